@@ -1,0 +1,186 @@
+"""Seeded synthetic inputs with the shapes of the paper's models.
+
+This module only draws random tensors (and loads the frozen confidence-model parameters
+that were fitted offline).  It contains none of the method's arithmetic: no router
+product, no softmax, no ranking, no expert FFN.  Both the CPU oracle's tests and the
+CUDA path's tests / benchmark take their inputs from here, so that the two sides see
+identical bytes without sharing any code of the method.
+
+Recipe (one base seed, one sub-stream per (config, layer, tensor kind)):
+
+* router            W_r ~ N(0, 1/d) fp32; optional bias b_r = 0.5*ln f_e, f_e a Zipf(s=1.1)
+                    frequency over a seeded permutation of the experts (skewed popularity)
+* prefetch router   W_p = W_r + N(0, sigma_p^2/d), b_p = b_r  (it mirrors the router)
+* hidden states     h ~ N(0,1); h' = h + N(0, 0.25); both rounded to bf16-representable
+                    values but stored widened in fp32
+* expert weights    bf16, N(0, 0.02^2), generated directly in the library's store layout
+                    gate[I][d], up[I][d], downT[I][d]  (downT is W_down transposed)
+* confidence model  w[N], theta[N-k+1]: frozen values fitted offline on calibration tokens
+                    of this same generator (files under ``data/``), else a fixed hand-set
+                    model
+"""
+from __future__ import annotations
+
+import dataclasses
+import os
+from typing import Optional, Tuple
+
+import numpy as np
+
+BASE_SEED = 11688
+
+_KIND = {"router": 1, "prefetch_noise": 2, "hidden": 3, "hidden_noise": 4, "experts": 5,
+         "shared": 6, "zipf_perm": 7, "calib_hidden": 8, "calib_noise": 9, "attn": 10}
+
+
+@dataclasses.dataclass(frozen=True)
+class Config:
+    cfg_id: int
+    name: str
+    L: int          # layers
+    d: int          # hidden size
+    N: int          # experts per layer
+    k: int          # routed experts per token
+    I: int          # expert intermediate size
+    C: int          # HBM cache slots per layer
+    T: int          # decode steps
+    batches: Tuple[int, ...] = (1,)
+    I_shared: int = 0
+    sigma_p: float = 0.3      # prefetch-router noise std, in units of 1/sqrt(d)
+    zipf_s: float = 0.0       # >0: skewed expert popularity through a router bias
+    modes: Tuple[str, ...] = ("exact", "stall_free")
+
+    @property
+    def expert_bytes(self) -> int:
+        return 3 * self.d * self.I * 2
+
+    @property
+    def shared_bytes(self) -> int:
+        return 3 * self.d * self.I_shared * 2
+
+    def scaled(self, **kw) -> "Config":
+        return dataclasses.replace(self, **kw)
+
+
+CONFIGS = {
+    0: Config(0, "tiny-granite1b-layer", L=1, d=1024, N=32, k=8, I=512, C=16, T=128,
+              modes=("exact",)),
+    1: Config(1, "granite-3b-a800m-shape", L=32, d=1536, N=40, k=8, I=512, C=20, T=1024),
+    2: Config(2, "olmoe-shape", L=16, d=2048, N=64, k=8, I=1024, C=24, T=2048, zipf_s=1.1),
+    3: Config(3, "mixtral-8x7b-shape", L=32, d=4096, N=8, k=2, I=14336, C=4, T=512,
+              sigma_p=0.5),
+    4: Config(4, "qwen1.5-moe-shape", L=24, d=2048, N=60, k=4, I=1408, C=30, T=64,
+              batches=(1, 8, 32, 128, 256), I_shared=5632, modes=("exact",)),
+}
+
+
+def _rng(cfg: Config, layer: int, kind: str) -> np.random.Generator:
+    return np.random.default_rng(np.random.SeedSequence([BASE_SEED, cfg.cfg_id, layer, _KIND[kind]]))
+
+
+def round_to_bf16_values(x: np.ndarray) -> np.ndarray:
+    """Round fp32 values to the nearest bf16-representable value (ties to even), keep fp32."""
+    x = np.ascontiguousarray(x, dtype=np.float32)
+    u = x.view(np.uint32).astype(np.uint64)
+    bias = 0x7FFF + ((u >> 16) & 1)
+    u = ((u + bias) & 0xFFFF0000).astype(np.uint32)
+    return u.view(np.float32).reshape(x.shape)
+
+
+def router_weights(cfg: Config, layer: int):
+    """Returns (W_r [N][d], b_r [N], W_p [N][d], b_p [N]) as fp32 arrays."""
+    d, N = cfg.d, cfg.N
+    W_r = (_rng(cfg, layer, "router").standard_normal((N, d)) / np.sqrt(d)).astype(np.float32)
+    noise = _rng(cfg, layer, "prefetch_noise").standard_normal((N, d)) * (cfg.sigma_p / np.sqrt(d))
+    W_p = (W_r.astype(np.float64) + noise).astype(np.float32)
+    if cfg.zipf_s > 0:
+        perm = _rng(cfg, layer, "zipf_perm").permutation(N)          # perm[e] = popularity rank - 1
+        f = (perm + 1.0) ** (-cfg.zipf_s)
+        f /= f.sum()
+        b_r = (0.5 * np.log(f)).astype(np.float32)
+    else:
+        b_r = np.zeros(N, dtype=np.float32)
+    return W_r, b_r, W_p, b_r.copy()
+
+
+def hidden_states(cfg: Config, layer: int, T: int, B: int = 1, calib: bool = False):
+    """Returns (h [T][B][d], h' [T][B][d]) fp32 holding bf16-representable values."""
+    a, b = ("calib_hidden", "calib_noise") if calib else ("hidden", "hidden_noise")
+    h = _rng(cfg, layer, a).standard_normal((T, B, cfg.d)).astype(np.float32)
+    hp = h + 0.5 * _rng(cfg, layer, b).standard_normal((T, B, cfg.d)).astype(np.float32)
+    return round_to_bf16_values(h), round_to_bf16_values(hp)
+
+
+def expert_store(cfg: Config, layer: int, device="cpu", pin: bool = False, out=None):
+    """bf16 tensor [N][3][I][d] in the library's store layout: gate, up, downT per expert.
+
+    The conceptual down projection is W_down[j][i] = downT[i][j].  Drawn with torch's
+    seeded generator on ``device`` (CPU and CUDA streams differ; within one run everybody
+    reads the same bytes).
+    """
+    import torch
+    shape = (cfg.N, 3, cfg.I, cfg.d)
+    g = torch.Generator(device=device)
+    g.manual_seed((BASE_SEED * 1000003 + cfg.cfg_id * 10007 + layer * 101 + _KIND["experts"]) & 0x7FFFFFFF)
+    if out is None:
+        out = torch.empty(shape, dtype=torch.bfloat16, device="cpu", pin_memory=pin) \
+            if str(device) == "cpu" else torch.empty(shape, dtype=torch.bfloat16, device=device)
+    # draw expert by expert to bound the fp32 temporary
+    for e in range(cfg.N):
+        t = torch.randn((3, cfg.I, cfg.d), generator=g, device=device, dtype=torch.float32)
+        out[e].copy_((t * 0.02).to(torch.bfloat16))
+    return out
+
+
+def shared_expert(cfg: Config, layer: int, device="cpu"):
+    """bf16 tensor [3][I_shared][d] (gate, up, downT) or None when the config has none."""
+    import torch
+    if cfg.I_shared == 0:
+        return None
+    g = torch.Generator(device=device)
+    g.manual_seed((BASE_SEED * 1000003 + cfg.cfg_id * 10007 + layer * 101 + _KIND["shared"]) & 0x7FFFFFFF)
+    t = torch.randn((3, cfg.I_shared, cfg.d), generator=g, device=device, dtype=torch.float32)
+    return (t * 0.02).to(torch.bfloat16)
+
+
+def handset_cdf_params(cfg: Config):
+    """A fixed, monotone confidence model used when no fitted file exists.
+
+    x is the prefetch distribution sorted in descending order.  Probability mass just below
+    the top-k boundary raises the latent score (less confident, larger budget); mass inside
+    the top-k lowers it.
+    """
+    N, k = cfg.N, cfg.k
+    w = np.zeros(N, dtype=np.float32)
+    w[:k] = -2.0
+    w[k:min(N, 2 * k)] = 6.0
+    theta = (-1.0 + 0.6 * np.arange(N - k + 1)).astype(np.float32)
+    return w, theta
+
+
+_DATA_DIR = os.path.join(os.path.dirname(os.path.abspath(__file__)), "data")
+
+
+def cdf_params(cfg: Config, layer: int, allow_handset: bool = True):
+    """(w [N], theta [N-k+1]) fp32: the frozen confidence model of this config and layer."""
+    path = os.path.join(_DATA_DIR, f"cdf_cfg{cfg.cfg_id}.npz")
+    if os.path.exists(path):
+        z = np.load(path)
+        if z["w"].shape == (cfg.L, cfg.N) and layer < cfg.L:
+            return z["w"][layer].astype(np.float32), z["theta"][layer].astype(np.float32)
+    if not allow_handset:
+        raise FileNotFoundError(path)
+    return handset_cdf_params(cfg)
+
+
+def bf16_to_f32_numpy(t) -> np.ndarray:
+    """Lossless widening of a torch bf16 tensor to a numpy fp32 array (test helper)."""
+    import torch
+    return t.detach().to("cpu").to(torch.float32).numpy()
+
+
+def tiny_config(d=256, N=8, k=2, I=64, C=4, L=1, T=8, I_shared=0, sigma_p=0.3, zipf_s=0.0,
+                cfg_id=100, batches=(1,)) -> Config:
+    """Small shapes for brute-force tests."""
+    return Config(cfg_id, "tiny", L=L, d=d, N=N, k=k, I=I, C=C, T=T, batches=batches,
+                  I_shared=I_shared, sigma_p=sigma_p, zipf_s=zipf_s)

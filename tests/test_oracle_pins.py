@@ -1,0 +1,395 @@
+"""Pins for the CPU oracle: values the paper prints, closed forms, brute force on tiny inputs,
+library special cases and invariants.  None of these re-types an oracle formula: each checks
+the oracle against an independent statement of the same fact."""
+import itertools
+import math
+import os
+
+import numpy as np
+import pytest
+import torch
+
+from oracle import apex_oracle as ao
+from paper_2608_11688_b200 import synth
+
+GOLDEN = os.path.join(os.path.dirname(__file__), "golden")
+
+
+def _rows(name):
+    with open(os.path.join(GOLDEN, name)) as f:
+        return [ln.split() for ln in f if ln.strip() and not ln.startswith("#")]
+
+
+# ---------------------------------------------------------------- values the paper prints
+def test_overlap_fraction_examples_from_paper():
+    for k, hits, expect in _rows("overlap_fraction.txt"):
+        k, hits, expect = int(k), int(hits), float(expect)
+        K_r = list(range(k))
+        P = list(range(hits)) + [100 + i for i in range(k - hits)]   # same size, one expert wrong
+        assert ao.overlap_accuracy(K_r, P) == expect
+        assert not ao.covered(K_r, P)
+
+
+def test_parameter_counts_pin_shapes_of_prefetch_router_and_cdf_model():
+    # W_p is d x N and the confidence model has (at most) 2N numbers per layer: x lives in R^N.
+    for model, L, d, N, millions in _rows("param_counts.txt"):
+        L, d, N = int(L), int(d), int(N)
+        cfg = synth.tiny_config(d=d, N=N, k=2, I=8, C=4)
+        W_r, b_r, W_p, b_p = synth.router_weights(cfg, 0)
+        w, theta = synth.handset_cdf_params(cfg)
+        assert W_p.shape == (N, d)
+        assert w.shape == (N,) and theta.shape[0] <= N
+        total = L * (W_p.size + 2 * N)
+        assert f"{total / 1e6:.2f}" == millions, (model, total)
+
+
+# ---------------------------------------------------------------- library special cases
+def test_logits_and_softmax_match_torch_fp64():
+    rng = np.random.default_rng(0)
+    for N, d in [(8, 64), (40, 1536), (5, 7)]:
+        W = rng.standard_normal((N, d)).astype(np.float32)
+        b = rng.standard_normal(N).astype(np.float32)
+        v = rng.standard_normal(d).astype(np.float32)
+        z = ao.linear_logits(W, b, v)
+        zt = torch.from_numpy(W).double() @ torch.from_numpy(v).double() + torch.from_numpy(b).double()
+        np.testing.assert_allclose(z, zt.numpy(), rtol=0, atol=1e-12)
+        np.testing.assert_allclose(ao.softmax(z), torch.softmax(zt, 0).numpy(), rtol=1e-13, atol=0)
+    # a transposed operand or a dropped bias would fail the above; no-bias path:
+    np.testing.assert_allclose(ao.linear_logits(W, None, v), (torch.from_numpy(W).double() @ torch.from_numpy(v).double()).numpy(), atol=1e-12)
+
+
+def test_softmax_is_shift_invariant_and_stable():
+    z = np.array([1000.0, 999.0, -1000.0])
+    q = ao.softmax(z)
+    assert np.isfinite(q).all() and abs(q.sum() - 1) < 1e-15
+    np.testing.assert_allclose(q, ao.softmax(z - 1000.0), rtol=1e-15)
+
+
+def test_swiglu_matches_torch_functional_and_zero_gate():
+    rng = np.random.default_rng(1)
+    d, I = 48, 20
+    Wg, Wu = rng.standard_normal((I, d)), rng.standard_normal((I, d))
+    Wd = rng.standard_normal((d, I))
+    v = rng.standard_normal(d)
+    t = lambda a: torch.from_numpy(np.asarray(a))
+    ref = t(Wd) @ (torch.nn.functional.silu(t(Wg) @ t(v)) * (t(Wu) @ t(v)))
+    np.testing.assert_allclose(ao.swiglu_ffn(Wg, Wu, Wd, v), ref.numpy(), rtol=1e-12, atol=1e-12)
+    assert np.all(ao.swiglu_ffn(np.zeros((I, d)), Wu, Wd, v) == 0.0)       # silu(0) = 0
+    # N = k = 1: the MoE layer is the plain FFN (the only gate is 1)
+    y = ao.moe_output(v, [0], ao.gates(ao.softmax(np.array([0.3])), [0]), lambda e: (Wg, Wu, Wd))
+    np.testing.assert_allclose(y, ref.numpy(), rtol=1e-12, atol=1e-12)
+
+
+# ---------------------------------------------------------------- ranking and top-k: brute force
+def test_rank_desc_against_definition_with_ties():
+    rng = np.random.default_rng(2)
+    for trial in range(200):
+        N = int(rng.integers(1, 9))
+        z = rng.integers(-2, 3, size=N).astype(np.float64)      # many duplicates
+        pi = ao.rank_desc(z)
+        assert sorted(pi) == list(range(N))
+        for j, e in enumerate(pi):
+            better = sum(1 for f in range(N) if z[f] > z[e] or (z[f] == z[e] and f < e))
+            assert better == j
+
+
+def test_route_topk_bruteforce_subset_and_order():
+    rng = np.random.default_rng(3)
+    for trial in range(50):
+        N, d, k = 7, 16, 3
+        W = rng.standard_normal((N, d)); b = rng.standard_normal(N); v = rng.standard_normal(d)
+        z, K_r, alpha = ao.route_topk(W, b, v, k)
+        # the top-k set maximises the sum of logits over all k-subsets
+        best = max(itertools.combinations(range(N), k), key=lambda S: sum(z[list(S)]))
+        assert set(best) == set(K_r)
+        assert all(z[K_r[i]] >= z[K_r[i + 1]] for i in range(k - 1))
+        assert abs(alpha.sum() - 1) < 1e-14 and np.argmax(alpha) == K_r[0]
+
+
+# ---------------------------------------------------------------- budget selection, Eq. (8)-(9)
+def _budget_bruteforce_pdomain(x, w, theta, tau, N, k):
+    s = float(np.dot(w.astype(np.float64), x))
+    for delta in range(N - k + 1):
+        p = 1.0 / (1.0 + math.exp(-(float(theta[delta]) - s)))
+        if p >= tau:
+            return delta
+    return N - k
+
+
+def test_select_budget_matches_probability_domain_bruteforce():
+    rng = np.random.default_rng(4)
+    checked = 0
+    for trial in range(400):
+        N = int(rng.integers(3, 12)); k = int(rng.integers(1, N)); C = N
+        q = ao.softmax(rng.standard_normal(N) * 2)
+        pi = ao.rank_desc(q)
+        w = rng.standard_normal(N).astype(np.float32) * 3
+        theta = np.sort(rng.standard_normal(N - k + 1).astype(np.float32) * 2)
+        tau = float(rng.uniform(0.05, 0.99))
+        sel = ao.select_budget(q, pi, w, theta, tau, k, C)
+        if sel["threshold_margin"] < 1e-9:
+            continue
+        x = np.sort(q)[::-1]
+        assert sel["delta_hat"] == _budget_bruteforce_pdomain(x, w, theta, tau, N, k)
+        assert sel["P"] == [int(e) for e in pi[:k + sel["delta_hat"]]]
+        checked += 1
+    assert checked > 300
+
+
+def test_select_budget_limits_static_and_cap():
+    rng = np.random.default_rng(5)
+    N, k = 10, 3
+    q = ao.softmax(rng.standard_normal(N)); pi = ao.rank_desc(q)
+    w = rng.standard_normal(N).astype(np.float32)
+    theta = np.sort(rng.standard_normal(N - k + 1)).astype(np.float32)
+    assert ao.select_budget(q, pi, w, theta, 0.0, k, N)["delta_hat"] == 0
+    assert ao.select_budget(q, pi, w, theta, 1e-300, k, N)["delta_hat"] == 0
+    assert ao.select_budget(q, pi, w, theta, 1.0, k, N)["delta_hat"] == N - k
+    for C in (k, 5, N):
+        sel = ao.select_budget(q, pi, w, theta, 1.0 - 1e-16, k, C)
+        assert sel["delta_hat"] == min(N, C) - k and len(sel["P"]) == min(N, C)
+        assert sel["capped"] == int(C < N)
+    # w = 0: the budget does not depend on the token (static over-fetch baseline)
+    w0 = np.zeros(N, np.float32)
+    d0 = {ao.select_budget(ao.softmax(rng.standard_normal(N)), pi, w0, theta, 0.7, k, N)["delta_hat"] for _ in range(20)}
+    assert len(d0) == 1
+
+
+def test_candidate_sets_are_nested_in_tau_and_probabilities_monotone():
+    rng = np.random.default_rng(6)
+    for trial in range(100):
+        N, k = 16, 4
+        q = ao.softmax(rng.standard_normal(N) * 1.5); pi = ao.rank_desc(q)
+        w = rng.standard_normal(N).astype(np.float32) * 2
+        theta = np.sort(rng.standard_normal(N - k + 1)).astype(np.float32) * 2
+        p = ao.coverage_probabilities(q[pi], w, theta)
+        assert np.all(np.diff(p) >= 0)                                   # Eq. (7)
+        prev = None
+        for tau in (0.3, 0.6, 0.75, 0.9, 0.97):
+            P = ao.select_budget(q, pi, w, theta, tau, k, N)["P"]
+            if prev is not None:
+                assert P[:len(prev)] == prev                              # nested prefixes of E
+            prev = P
+
+
+# ---------------------------------------------------------------- delta*, coverage
+def test_oracle_budget_closed_form_vs_definition():
+    rng = np.random.default_rng(7)
+    for trial in range(300):
+        N = int(rng.integers(2, 12)); k = int(rng.integers(1, N + 1))
+        pi = rng.permutation(N)
+        K_r = [int(e) for e in rng.choice(N, size=k, replace=False)]
+        # Eq. (3) literally: smallest delta whose prefix of E contains K_r
+        brute = next(dl for dl in range(N - k + 1) if set(K_r) <= set(int(e) for e in pi[:k + dl]))
+        assert ao.oracle_budget(pi, K_r, k) == brute
+        for d_hat in range(N - k + 1):                                     # full coverage iff d_hat >= delta*
+            assert ao.covered(K_r, pi[:k + d_hat]) == (d_hat >= brute)
+
+
+def test_identical_routers_and_states_need_no_extra_budget():
+    cfg = synth.tiny_config(d=64, N=12, k=3, I=8, C=6)
+    W_r, b_r, _, _ = synth.router_weights(cfg, 0)
+    h, _ = synth.hidden_states(cfg, 0, T=10)
+    for t in range(10):
+        z_p, q_p, pi = ao.prefetch_scores(W_r, b_r, h[t, 0])
+        _, K_r, _ = ao.route_topk(W_r, b_r, h[t, 0], cfg.k)
+        assert ao.oracle_budget(pi, K_r, cfg.k) == 0
+        assert ao.overlap_accuracy(K_r, pi[:cfg.k]) == 1.0
+
+
+# ---------------------------------------------------------------- Algorithm 1
+def test_stall_free_set_bruteforce_over_all_subsets():
+    rng = np.random.default_rng(8)
+    for trial in range(300):
+        N = int(rng.integers(3, 7)); k = int(rng.integers(1, N))
+        alpha = ao.softmax(rng.standard_normal(N))
+        K_r = [int(e) for e in ao.rank_desc(alpha)[:k]]
+        size_R = int(rng.integers(k, N + 1))
+        R = sorted(int(e) for e in rng.choice(N, size=size_R, replace=False))
+        K = ao.stall_free_set(K_r, alpha, R)
+        assert len(K) == k and set(K) <= set(R) and (set(K_r) & set(R)) <= set(K)
+        if set(K_r) <= set(R):
+            assert set(K) == set(K_r)
+        # independent characterisation: among all k-subsets of R that keep the available routed
+        # experts, Algorithm 1 picks the one of largest total router weight
+        keep = set(K_r) & set(R)
+        best = max((S for S in itertools.combinations(R, k) if keep <= set(S)),
+                   key=lambda S: sum(alpha[list(S)]))
+        assert set(best) == set(K)
+        g = ao.gates(alpha, K)
+        assert abs(g.sum() - 1.0) < 1e-14 and np.all(g > 0)
+
+
+def test_stall_free_tie_break_prefers_lower_index():
+    alpha = np.array([0.4, 0.1, 0.1, 0.1, 0.3])
+    assert ao.stall_free_set([0, 4], alpha, [0, 1, 2, 3]) == [0, 1]
+    assert ao.stall_free_set([0, 4], alpha, [0, 2, 3]) == [0, 2]
+
+
+# ---------------------------------------------------------------- slot cache
+def test_slot_cache_hand_traced_example():
+    # N=4, C=2.  Traced by hand from the replacement rule (smallest (stamp, slot) not protected).
+    c = ao.SlotCache(4, 2)
+    c.begin_step()                              # clock 1
+    U, cp = c.prefetch([[2, 0]])                # both slots empty: ascending expert order 0->slot0, 2->slot1
+    assert U == [0, 2] and cp == [(0, 0), (2, 1)] and c.expert_slot == [0, -1, 1, -1]
+    miss, waves = c.demand([[0, 3]])            # 3 missing; victim must not be a Need member if possible: slot1 (expert 2)
+    assert miss == [3] and waves == [[(3, 1)]] and c.expert_slot == [0, -1, -1, 1]
+    c.begin_step()                              # clock 2
+    U, cp = c.prefetch([[3, 1]])                # 3 hit (touched, stamp 2); 1 -> victim slot0 (stamp 1)
+    assert cp == [(1, 0)] and c.expert_slot == [-1, 0, -1, 1] and c.slot_stamp == [2, 2]
+    miss, waves = c.demand([[1, 3]])
+    assert miss == [] and waves == []
+    c.begin_step()                              # clock 3
+    U, cp = c.prefetch([[1]])                   # hit only: slot0 stamp 3
+    assert cp == [] and c.slot_stamp == [3, 2]
+    miss, waves = c.demand([[0, 2]])            # both missing, C=2: one chunk; 0 -> slot1 (stamp 2 < 3), 2 -> slot0
+    assert miss == [0, 2] and waves == [[(0, 1), (2, 0)]] and c.expert_slot == [1, -1, 0, -1]
+
+
+def test_slot_cache_invariants_random_walk():
+    rng = np.random.default_rng(9)
+    for reuse in (True, False):
+        N, C, k = 12, 5, 3
+        c = ao.SlotCache(N, C, cache_reuse=reuse)
+        for step in range(200):
+            c.begin_step()
+            P = [int(e) for e in rng.choice(N, size=int(rng.integers(k, C + 1)), replace=False)]
+            U, copies = c.prefetch([P])
+            assert set(P) <= set(c.resident())                       # nothing needed was evicted
+            if not reuse:
+                assert len(copies) == len(P)                          # load-use-evict: every candidate is copied
+            K_r = [int(e) for e in rng.choice(N, size=k, replace=False)]
+            missing, waves = c.demand([K_r])
+            assert set(K_r) <= set(c.resident())
+            assert sorted(e for wv in waves for e, _ in wv) == sorted(missing)
+            for e, s in enumerate(c.expert_slot):                     # tables are mutually inverse
+                if s >= 0:
+                    assert c.slot_expert[s] == e
+            for s, e in enumerate(c.slot_expert):
+                if e >= 0:
+                    assert c.expert_slot[e] == s
+            assert sum(1 for e in c.slot_expert if e >= 0) <= C
+
+
+def test_full_size_cache_copies_each_expert_once():
+    rng = np.random.default_rng(10)
+    N = C = 8
+    c = ao.SlotCache(N, C)
+    seen, total = set(), 0
+    for step in range(100):
+        c.begin_step()
+        P = [int(e) for e in rng.choice(N, size=4, replace=False)]
+        _, cp = c.prefetch([P])
+        K_r = [int(e) for e in rng.choice(N, size=2, replace=False)]
+        _, waves = c.demand([K_r])
+        for e, _ in cp + [x for wv in waves for x in wv]:
+            assert e not in seen
+            seen.add(e); total += 1
+    assert total == len(seen) <= N
+
+
+def test_batched_prefetch_union_order_and_truncation():
+    c = ao.SlotCache(10, 3)
+    c.begin_step()
+    # counts: 5 -> 3 tokens, 1 -> 2, 7 -> 2, 0 -> 1, 9 -> 1 ; keep the 3 most wanted, ties by lower index
+    U, cp = c.prefetch([[5, 1, 0], [5, 7, 1], [5, 7, 9]])
+    assert U == [1, 5, 7] and [e for e, _ in cp] == [1, 5, 7]
+
+
+# ---------------------------------------------------------------- whole layer-step
+def _dense_topk_moe(W_r, b_r, hp, k, experts, shared):
+    """Written separately from the oracle, with torch fp64 ops: standard MoE layer that knows
+    nothing about prefetching or caches (softmax over all experts, top-k, renormalised gates)."""
+    t = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
+    logits = t(W_r) @ t(hp) + t(b_r)
+    probs = torch.softmax(logits, 0)
+    top = torch.topk(logits, k).indices
+    gate = probs[top] / probs[top].sum()
+    y = torch.zeros(len(hp), dtype=torch.float64)
+    for g, e in zip(gate, top):
+        Wg, Wu, Wd = (t(m) for m in experts(int(e)))
+        y += g * (Wd @ (torch.nn.functional.silu(Wg @ t(hp)) * (Wu @ t(hp))))
+    if shared is not None:
+        Wg, Wu, Wd = (t(m) for m in shared)
+        y += Wd @ (torch.nn.functional.silu(Wg @ t(hp)) * (Wu @ t(hp)))
+    return y.numpy()
+
+
+def _tiny_problem(cfg, layer=0):
+    W_r, b_r, W_p, b_p = synth.router_weights(cfg, layer)
+    store = synth.bf16_to_f32_numpy(synth.expert_store(cfg, layer))
+    experts = lambda e: (store[e, 0], store[e, 1], store[e, 2].T)
+    sh = synth.shared_expert(cfg, layer)
+    shared = None
+    if sh is not None:
+        s = synth.bf16_to_f32_numpy(sh)
+        shared = (s[0], s[1], s[2].T)
+    w, theta = synth.handset_cdf_params(cfg)
+    return W_r, b_r, W_p, b_p, experts, shared, w, theta
+
+
+@pytest.mark.parametrize("reuse", [True, False])
+@pytest.mark.parametrize("tau,C", [(0.0, 2), (0.6, 3), (0.9, 5), (1.0, 8)])
+def test_exact_mode_equals_dense_topk_moe(tau, C, reuse):
+    cfg = synth.tiny_config(d=64, N=8, k=2, I=16, C=C, T=6, I_shared=8 if C == 5 else 0, zipf_s=1.1)
+    W_r, b_r, W_p, b_p, experts, shared, w, theta = _tiny_problem(cfg)
+    h, hp = synth.hidden_states(cfg, 0, cfg.T, B=2)
+    cache = ao.SlotCache(cfg.N, cfg.C, cache_reuse=reuse)
+    for t in range(cfg.T):
+        out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=tau,
+                            k=cfg.k, h=h[t], h_post=hp[t], mode="exact", expert_weights=experts, shared=shared)
+        for b in range(2):
+            ref = _dense_topk_moe(W_r, b_r, hp[t, b], cfg.k, experts, shared)
+            np.testing.assert_allclose(out["tokens"][b]["y"], ref, rtol=1e-10, atol=1e-13)
+            assert set(out["tokens"][b]["K_exec"]) == set(out["tokens"][b]["K_r"])
+        need = set(e for tok in out["tokens"] for e in tok["K_r"])
+        if len(need) <= cfg.C:                  # otherwise the waves reuse slots within the step
+            assert need <= set(cache.resident())
+
+
+def test_stall_free_equals_exact_when_covered_and_differs_only_by_substitution():
+    cfg = synth.tiny_config(d=64, N=10, k=3, I=16, C=5, T=40, sigma_p=1.5)
+    W_r, b_r, W_p, b_p, experts, shared, w, theta = _tiny_problem(cfg)
+    h, hp = synth.hidden_states(cfg, 0, cfg.T)
+    cache = ao.SlotCache(cfg.N, cfg.C)
+    n_sub = n_same = 0
+    for t in range(cfg.T):
+        out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=0.6,
+                            k=cfg.k, h=h[t], h_post=hp[t], mode="stall_free", expert_weights=experts)
+        tok = out["tokens"][0]
+        R = set(out["resident_after_prefetch"])
+        assert out["demand_copies"] == [] and set(tok["K_exec"]) <= R and len(tok["K_exec"]) == cfg.k
+        assert abs(sum(tok["gates"]) - 1.0) < 1e-14
+        if set(tok["K_r"]) <= R:
+            ref = _dense_topk_moe(W_r, b_r, hp[t, 0], cfg.k, experts, None)
+            np.testing.assert_allclose(tok["y"], ref, rtol=1e-10, atol=1e-13)
+            n_same += 1
+        else:
+            assert tok["n_subst"] == len(set(tok["K_r"]) - R) > 0
+            n_sub += 1
+    assert n_sub > 0 and n_same > 0          # the noisy predictor exercises both branches
+
+
+def test_per_layer_staging_policy_copies_every_candidate():
+    # cache_reuse=False is the paper's load-use-evict policy: R = P after the prefetch
+    cfg = synth.tiny_config(d=64, N=10, k=3, I=16, C=6, T=10)
+    W_r, b_r, W_p, b_p, experts, shared, w, theta = _tiny_problem(cfg)
+    h, hp = synth.hidden_states(cfg, 0, cfg.T)
+    cache = ao.SlotCache(cfg.N, cfg.C, cache_reuse=False)
+    for t in range(cfg.T):
+        out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=0.9,
+                            k=cfg.k, h=h[t], h_post=hp[t], mode="stall_free", compute_ffn=False)
+        tok = out["tokens"][0]
+        assert sorted(out["resident_after_prefetch"]) == sorted(tok["P"])
+        assert len(out["prefetch_copies"]) == cfg.k + tok["delta_hat"]
+
+
+def test_generator_rounds_hidden_states_to_bf16_values():
+    cfg = synth.tiny_config()
+    h, hp = synth.hidden_states(cfg, 0, 4)
+    for a in (h, hp):
+        t = torch.from_numpy(a)
+        assert torch.equal(t, t.to(torch.bfloat16).to(torch.float32))
+    x = np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8], dtype=np.float32)    # exact ties: round to even
+    np.testing.assert_array_equal(synth.round_to_bf16_values(x), torch.from_numpy(x).to(torch.bfloat16).float().numpy())

@@ -1,0 +1,211 @@
+/*
+ * apex.h -- C ABI of the B200-native MoE decode step with adaptive expert prefetch.
+ *
+ * One layer-step of decoding, as the paper sequences it (Sec. IV-A "two stages", Sec. IV-D
+ * "Runtime Operation"):
+ *
+ *   apex_predict            prefetch router on the pre-attention state h       (Sec. IV-D)
+ *   apex_select_candidates  confidence-driven budget delta_hat and K_p         (Eq. (8), (9), (1))
+ *   apex_prefetch           asynchronous copy of K_p into HBM cache slots      (Sec. IV-A stage 1)
+ *   apex_attention_standin  the window that hides the copies                   (Eq. (12))
+ *   apex_route_topk         exact top-k gate on the post-attention state h'    (Sec. III-A)
+ *   apex_moe_ffn            expert FFNs + weighted sum, in one of two modes    (Sec. IV-E, Alg. 1)
+ *
+ * Conventions
+ *   - Every function returns an int: APEX_OK (0) or a negative error code.  Nothing throws or
+ *     aborts across this boundary.  apex_last_error() gives a text owned by the context.
+ *   - "dev" pointers are device (HBM) addresses, "host" pointers host addresses.  All buffers
+ *     are owned by the caller and only borrowed for the duration stated at each call.
+ *   - Streams are cudaStream_t handles passed as void*; NULL is the legacy default stream.
+ *   - Row-major everywhere.  Expert indices, slots and counts are int32, probabilities and
+ *     hidden states fp32, expert weights bf16 (fp32 accumulation inside the kernels).
+ *   - All orderings are "value descending, then lower expert index".
+ *   - Limits of this build: N <= 64 experts per layer, k <= 16, d a multiple of 256 and
+ *     d <= 4096, 1 <= B <= max_batch <= 256, k <= C <= N.
+ *   - A context is not thread-safe; use one host thread per context.
+ *
+ * Expert store layout (host, pinned): expert e of a layer starts at base + e*stride and holds
+ *   gate[I][d], up[I][d], downT[I][d]   (bf16),
+ * where downT is the transpose of the down projection W_down[d][I], so that intermediate
+ * index i owns three contiguous d-vectors.  apex_pack_expert() converts from the usual
+ * gate[I][d], up[I][d], down[d][I].
+ */
+#ifndef APEX_H
+#define APEX_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+#define APEX_OK 0
+#define APEX_EINVAL (-1)   /* bad argument or unsupported shape */
+#define APEX_ENOMEM (-2)   /* host or device allocation failed */
+#define APEX_ECUDA (-3)    /* a CUDA runtime call failed; see apex_last_error */
+#define APEX_ETIMEOUT (-4) /* a bounded wait (host or device side) ran out */
+#define APEX_ESTATE (-5)   /* calls out of order, or no evictable slot */
+#define APEX_ENOTIMPL (-6)
+
+#define APEX_MODE_EXACT 0      /* correctness-preserving: follow K_r, fetch what is missing */
+#define APEX_MODE_STALL_FREE 1 /* Algorithm 1: resident experts only, gates renormalised */
+
+#define APEX_MAX_EXPERTS 64
+#define APEX_MAX_TOPK 16
+#define APEX_MAX_BATCH 256
+
+typedef struct apex_ctx apex_ctx;
+
+typedef struct apex_config {
+  int32_t d;             /* hidden size */
+  int32_t N;             /* experts per layer */
+  int32_t k;             /* routed experts per token */
+  int32_t I;             /* expert intermediate size */
+  int32_t I_shared;      /* always-on shared SwiGLU FFN intermediate size, 0 = none */
+  int32_t C;             /* HBM cache slots per layer */
+  int32_t L;             /* layers */
+  int32_t max_batch;     /* largest B that will be passed */
+  int32_t norm_topk;     /* 1: g_e = alpha_e / sum over the executed set; 0: g_e = alpha_e */
+  int32_t cache_reuse;   /* 1: slots persist across steps; 0: load-use-evict per layer-step */
+  int32_t ctx_len;       /* context length that sizes the stand-in attention kernel */
+  int32_t flags;         /* reserved, 0 */
+  int64_t wait_limit_ns; /* bound of every host- and device-side wait; 0 = 2 s */
+} apex_config;
+
+/* Counters of one layer, accumulated over layer-steps since the last reset. */
+typedef struct apex_step_stats {
+  int64_t layer_steps;
+  int64_t tokens;
+  int64_t sum_delta_hat;   /* selected extra budget (after the cap) */
+  int64_t sum_delta_star;  /* oracle budget, Eq. (3) */
+  int64_t sum_ncand;       /* k + delta_hat */
+  int64_t capped;          /* tokens whose budget hit the buffer cap C - k */
+  int64_t routed;          /* tokens * k */
+  int64_t hits_P;          /* routed experts inside the token's candidate set K_p */
+  int64_t hits_R;          /* routed experts resident after the prefetch plan */
+  int64_t covered;         /* tokens with K_r subset of K_p, Eq. (2) */
+  int64_t substitutions;   /* stall-free replacements */
+  int64_t prefetch_copies;
+  int64_t demand_copies;
+  int64_t bytes_copied;
+  int64_t extra_waves;     /* FFN launches beyond the first, exact mode */
+  int64_t stall_ns;        /* device time spent waiting for slot-ready flags (max over CTAs per launch) */
+  int64_t timeouts;
+  int64_t near_full_prefetch; /* tokens with k + delta_hat > N/2 */
+} apex_step_stats;
+
+/* ---- life cycle ------------------------------------------------------------------------ */
+
+/* Allocates the context: router tables, the L*C slot cache in HBM, flags, mailboxes.
+ * Returns APEX_EINVAL for shapes outside the limits above, APEX_ENOMEM / APEX_ECUDA otherwise. */
+int apex_create(const apex_config* cfg, apex_ctx** out);
+int apex_destroy(apex_ctx* ctx);
+const char* apex_last_error(const apex_ctx* ctx);
+
+/* ---- parameters (host pointers, copied into library-owned device memory) ---------------- */
+
+/* Original router of a layer (Sec. III-A): W_r [N][d], b_r [N] or NULL. */
+int apex_set_router(apex_ctx* ctx, int layer, const float* W_r_host, const float* b_r_host);
+/* Prefetch router (Sec. IV-D: mirrors the original router): W_p [N][d], b_p [N] or NULL. */
+int apex_set_prefetch_router(apex_ctx* ctx, int layer, const float* W_p_host, const float* b_p_host);
+/* Ordinal-logistic confidence model (Eq. (8)): w [N], theta [N-k+1].  theta must be
+ * non-decreasing (Table I), else APEX_EINVAL. */
+int apex_set_cdf(apex_ctx* ctx, int layer, const float* w_host, const float* theta_host);
+/* Off-chip expert store of a layer (Sec. III-A: expert weights live off-package): pinned host
+ * memory in the store layout described above.  Borrowed until apex_destroy. */
+int apex_register_experts(apex_ctx* ctx, int layer, const void* pinned_base, size_t expert_stride_bytes);
+/* Always-on shared expert (Sec. V-A: shared experts are outside the routing and the budget):
+ * device pointer to gate[I_shared][d], up[I_shared][d], downT[I_shared][d], bf16.  Borrowed. */
+int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights);
+/* Host helper: gate[I][d], up[I][d], down[d][I] -> store layout.  dst holds 3*I*d bf16. */
+int apex_pack_expert(const void* gate, const void* up, const void* down, int d, int I, void* dst);
+
+/* ---- the layer-step ---------------------------------------------------------------------- */
+
+/* S1+S2 (Sec. IV-D): z_p = W_p h + b_p, q_p = softmax(z_p), ranking E of Sec. IV-B.  h_dev is
+ * [B][d].  Results stay in the context for apex_select_candidates.  Starts a new layer-step
+ * for this layer (advances its slot-table clock). */
+int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stream);
+/* S3 (Eq. (9), (1)): x = q_p sorted descending, delta_hat = min{delta: theta_delta - w.x >=
+ * ln(tau/(1-tau))}, capped to C-k; cand_dev [B][C] receives e_1..e_{k+delta_hat} in rank order,
+ * padded with -1; ncand_dev [B] receives k+delta_hat.  tau<=0 gives delta_hat=0, tau>=1 gives
+ * the cap. */
+int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* cand_dev,
+                           int32_t* ncand_dev, void* stream);
+/* S5 (Sec. IV-A stage 1): waits (host side, bounded) for the candidate lists, plans slots and
+ * issues one cudaMemcpyAsync per non-resident candidate on copy_stream (NULL: the context's
+ * own copy stream), each followed by a slot-ready flag.  Returns without waiting for the
+ * copies. */
+int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream);
+/* Streams the bytes of an attention block (4 d^2 + 2 ctx_len d bf16 values): the hiding window
+ * of Eq. (12).  It does not produce h'. */
+int apex_attention_standin(apex_ctx* ctx, int layer, void* stream);
+/* S4 (Sec. III-A; Alg. 1 line 3): z_r = W_r h' + b_r, idx_dev [B][k] = K_r in rank order,
+ * alpha_dev [B][N] = softmax(z_r).  Both buffers must stay valid until apex_moe_ffn of the
+ * same layer-step has been called. */
+int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int32_t* idx_dev,
+                    float* alpha_dev, void* stream);
+/* S6-S8 (Sec. IV-E): y_dev [B][d] = sum over the execution set of g_e FFN_e(h') (+ shared FFN).
+ * APEX_MODE_EXACT executes K_r: resident experts first, missing ones are copied on demand and
+ * executed in further launches ("asynchronous miss correction").  APEX_MODE_STALL_FREE executes
+ * Algorithm 1 with K_p := the resident set.  exec_idx_dev [B][k] (ascending expert index) and
+ * exec_gate_dev [B][k] may be NULL.  Device-side waits on slot-ready flags are bounded; when one
+ * runs out the call (or the next call on this context) returns APEX_ETIMEOUT. */
+int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev,
+                 int32_t* exec_idx_dev, float* exec_gate_dev, void* stream);
+
+/* All L layers of one decode step, in the order above.  h_dev, hpost_dev, y_dev are [L][B][d]. */
+int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev, int B, float tau,
+                      int mode, float* y_dev, void* stream);
+/* Same with host buffers (pinned for full speed): inputs are copied to the device and y back
+ * inside the call, which returns after y_host is complete. */
+int apex_decode_token_host(apex_ctx* ctx, const float* h_host, const float* hpost_host, int B,
+                           float tau, int mode, float* y_host, void* stream);
+
+/* ---- observation, checkpoint, test hooks --------------------------------------------------- */
+
+int apex_get_stats(apex_ctx* ctx, int layer, apex_step_stats* out); /* layer -1: sum over layers */
+int apex_reset_stats(apex_ctx* ctx);
+/* Results of the last apex_predict (synchronises the stream it ran on): z_p, q_p [B][N], pi [B][N]. */
+int apex_read_prediction(apex_ctx* ctx, int B, float* z_p_host, float* q_p_host, int32_t* pi_host);
+/* Copies issued by the last layer-step of `layer`: first the prefetch copies, then the demand
+ * copies, as (expert, slot) pairs; arrays hold up to 2*N entries. */
+int apex_get_last_copies(apex_ctx* ctx, int layer, int32_t* expert, int32_t* slot, int32_t* n_prefetch,
+                         int32_t* n_demand);
+/* Slot table of a layer: expert_slot [N] (-1 = not resident), slot_stamp [C], clock.  Setting a
+ * table marks the named slots as holding valid data only if they already do (checkpoint/resume
+ * within one context); other residents are dropped. */
+int apex_get_slot_table(apex_ctx* ctx, int layer, int32_t* expert_slot, int64_t* slot_stamp, int64_t* clock);
+int apex_set_slot_table(apex_ctx* ctx, int layer, const int32_t* expert_slot, const int64_t* slot_stamp,
+                        int64_t clock);
+/* Makes every expert of every layer resident (needs C == N) and waits for the copies. */
+int apex_warm_all(apex_ctx* ctx);
+/* Host-side fault hooks for tests: what = 1 the next copy issue fails (APEX_ECUDA path);
+ * what = 2 the next slot-ready flag is withheld (device wait runs out); 0 clears. */
+int apex_test_inject(apex_ctx* ctx, int what);
+/* Number of kernels this library has launched on the context so far. */
+int64_t apex_launch_count(const apex_ctx* ctx);
+
+/* ---- host-only slot planner (the state machine behind apex_prefetch / apex_moe_ffn) -------- */
+
+typedef struct apex_slots apex_slots;
+apex_slots* apex_slots_create(int N, int C, int cache_reuse);
+void apex_slots_destroy(apex_slots* s);
+int apex_slots_begin_step(apex_slots* s);
+/* cand [B][stride], ncand [B]: plans the union (most wanted first, truncated to C).  Outputs:
+ * copy_expert/copy_slot (up to C entries), *n_copies. */
+int apex_slots_prefetch(apex_slots* s, const int32_t* cand, const int32_t* ncand, int B, int stride,
+                        int32_t* copy_expert, int32_t* copy_slot, int32_t* n_copies);
+/* K_r [B][k]: touches resident routed experts and installs the missing ones in chunks of C.
+ * Outputs: copy_expert/copy_slot (up to N entries), wave_of_copy (1-based wave), *n_copies. */
+int apex_slots_demand(apex_slots* s, const int32_t* K_r, int B, int k, int32_t* copy_expert,
+                      int32_t* copy_slot, int32_t* wave_of_copy, int32_t* n_copies);
+int apex_slots_touch(apex_slots* s, const int32_t* experts, int n);
+int apex_slots_get(const apex_slots* s, int32_t* expert_slot, int64_t* slot_stamp, int64_t* clock);
+int apex_slots_set(apex_slots* s, const int32_t* expert_slot, const int64_t* slot_stamp, int64_t clock);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* APEX_H */

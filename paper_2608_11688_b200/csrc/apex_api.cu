@@ -1,0 +1,812 @@
+// C-ABI entry points: argument checks, the host side of the prefetch machinery (slot planning,
+// cudaMemcpyAsync on the copy stream, slot-ready flags) and kernel launches.  All arithmetic of the
+// path runs in the kernels of kernels_router.cu / kernels_ffn.cu.
+#include <chrono>
+#include <cmath>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "apex_internal.hpp"
+
+using namespace apex;
+
+namespace {
+
+typedef int (*WriteValue32Fn)(cudaStream_t, unsigned long long, uint32_t, unsigned int);
+
+int fail(apex_ctx* ctx, int code, const char* what, cudaError_t e = cudaSuccess) {
+  if (ctx) {
+    char buf[512];
+    if (e != cudaSuccess)
+      snprintf(buf, sizeof buf, "%s: %s", what, cudaGetErrorString(e));
+    else
+      snprintf(buf, sizeof buf, "%s", what);
+    ctx->err = buf;
+  }
+  return code;
+}
+
+#define CU_TRY(ctx, expr)                                              \
+  do {                                                                 \
+    cudaError_t _e = (expr);                                           \
+    if (_e != cudaSuccess) return fail(ctx, APEX_ECUDA, #expr, _e);    \
+  } while (0)
+
+#define CHECK_CTX(ctx) \
+  if (!(ctx)) return APEX_EINVAL
+#define CHECK_LAYER(ctx, layer) \
+  if ((layer) < 0 || (layer) >= (ctx)->cfg.L) return fail(ctx, APEX_EINVAL, "layer out of range")
+
+template <typename T>
+cudaError_t dev_alloc(T** p, size_t n) {
+  return cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T) > 0 ? n * sizeof(T) : 16);
+}
+
+MailboxHeader* mhdr(apex_ctx* ctx) { return reinterpret_cast<MailboxHeader*>(ctx->mbox); }
+int32_t* mbox_i32(apex_ctx* ctx, size_t off) { return reinterpret_cast<int32_t*>(ctx->mbox + off); }
+
+// Bounded host wait for a mailbox sequence number.
+bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
+  if ((int32_t)(*p - want) >= 0) return true;
+  const auto t0 = std::chrono::steady_clock::now();
+  const int64_t limit = ctx->cfg.wait_limit_ns * 2 + 1000000000ll;  // the device side gives up first
+  for (uint32_t it = 0;; ++it) {
+    if ((int32_t)(*p - want) >= 0) return true;
+    if ((it & 1023u) == 1023u) {
+      const int64_t ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+      if (ns > limit) return false;
+    }
+#if defined(__x86_64__)
+    __builtin_ia32_pause();
+#endif
+  }
+}
+
+// One expert copy host store -> slot, followed by the slot-ready flag on the same stream.
+int issue_copy(apex_ctx* ctx, int layer, int e, int slot, cudaStream_t cs) {
+  if (!ctx->store_base[layer]) return fail(ctx, APEX_ESTATE, "no expert store registered for this layer");
+  if (ctx->inject == 1) {
+    ctx->inject = 0;
+    return fail(ctx, APEX_ECUDA, "injected copy-issue failure");
+  }
+  const size_t C = ctx->cfg.C;
+  uint8_t* dst = ctx->d_cache + ((size_t)layer * C + slot) * ctx->expert_bytes;
+  const uint8_t* src = ctx->store_base[layer] + (size_t)e * ctx->store_stride[layer];
+  const uint32_t gen = ++ctx->slot_gen[layer][slot];
+  CU_TRY(ctx, cudaMemcpyAsync(dst, src, ctx->expert_bytes, cudaMemcpyHostToDevice, cs));
+  uint32_t* flag = ctx->d_slot_ready + (size_t)layer * C + slot;
+  if (ctx->inject == 2) {
+    ctx->inject = 0;
+    ctx->withheld_flag = flag;
+    ctx->withheld_gen = gen;
+  } else if (ctx->fn_write_value32) {
+    int r = reinterpret_cast<WriteValue32Fn>(ctx->fn_write_value32)(cs, (unsigned long long)(uintptr_t)flag, gen, 0);
+    if (r != 0) return fail(ctx, APEX_ECUDA, "cuStreamWriteValue32 failed");
+  } else {
+    uint32_t* srcv = ctx->gen_src + (ctx->gen_src_pos++ % ctx->gen_src_len);
+    *srcv = gen;
+    CU_TRY(ctx, cudaMemcpyAsync(flag, srcv, sizeof(uint32_t), cudaMemcpyHostToDevice, cs));
+  }
+  ctx->phys_expert[layer][slot] = e;
+  ctx->host_stats[layer].bytes_copied += (int64_t)ctx->expert_bytes;
+  return APEX_OK;
+}
+
+int release_withheld(apex_ctx* ctx) {
+  if (!ctx->withheld_flag) return APEX_OK;
+  uint32_t* srcv = ctx->gen_src + (ctx->gen_src_pos++ % ctx->gen_src_len);
+  *srcv = ctx->withheld_gen;
+  CU_TRY(ctx, cudaMemcpyAsync(ctx->withheld_flag, srcv, sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->cur_copy_stream));
+  ctx->withheld_flag = nullptr;
+  return APEX_OK;
+}
+
+SlotSnapshot make_snapshot(apex_ctx* ctx, int layer) {
+  SlotSnapshot s;
+  const auto& es = ctx->tables[layer].expert_slot();
+  s.resident_mask = 0;
+  for (int e = 0; e < APEX_MAX_EXPERTS; ++e) {
+    const int slot = e < ctx->cfg.N ? es[e] : -1;
+    s.expert_slot[e] = (int8_t)slot;
+    s.need_gen[e] = slot >= 0 ? ctx->slot_gen[layer][slot] : 0u;
+    if (slot >= 0) s.resident_mask |= (1ull << e);
+  }
+  return s;
+}
+
+int check_device_status(apex_ctx* ctx) {
+  if (mhdr(ctx)->status != 0) {
+    mhdr(ctx)->status = 0;
+    release_withheld(ctx);
+    return fail(ctx, APEX_ETIMEOUT, "a device-side wait on a slot-ready flag ran out");
+  }
+  return APEX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int apex_create(const apex_config* cfg, apex_ctx** out) {
+  if (!cfg || !out) return APEX_EINVAL;
+  *out = nullptr;
+  const apex_config& c = *cfg;
+  if (c.N < 1 || c.N > APEX_MAX_EXPERTS || c.k < 1 || c.k > APEX_MAX_TOPK || c.k > c.N || c.C < c.k || c.C > c.N ||
+      c.L < 1 || c.I < 1 || c.I_shared < 0 || c.max_batch < 1 || c.max_batch > APEX_MAX_BATCH || !ffn_shape_supported(c.d) ||
+      c.ctx_len < 0)
+    return APEX_EINVAL;
+  apex_ctx* ctx = new (std::nothrow) apex_ctx();
+  if (!ctx) return APEX_ENOMEM;
+  ctx->cfg = c;
+  if (ctx->cfg.wait_limit_ns <= 0) ctx->cfg.wait_limit_ns = 2000000000ll;
+  if (ctx->cfg.ctx_len == 0) ctx->cfg.ctx_len = 1024;
+  const size_t L = c.L, N = c.N, C = c.C, d = c.d, MB = c.max_batch, k = c.k;
+  ctx->expert_bytes = 3 * d * (size_t)c.I * 2;
+  ctx->shared_bytes = 3 * d * (size_t)c.I_shared * 2;
+
+  auto bail = [&](int code, const char* what, cudaError_t e) {
+    fail(ctx, code, what, e);
+    fprintf(stderr, "apex_create: %s\n", ctx->err.c_str());
+    apex_destroy(ctx);
+    return code;
+  };
+#define CR(expr)                                                                  \
+  do {                                                                            \
+    cudaError_t _e = (expr);                                                      \
+    if (_e != cudaSuccess)                                                        \
+      return bail(_e == cudaErrorMemoryAllocation ? APEX_ENOMEM : APEX_ECUDA, #expr, _e); \
+  } while (0)
+
+  CR(cudaGetDevice(&ctx->device));
+  CR(cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device));
+  CR(dev_alloc(&ctx->d_Wr, L * N * d));
+  CR(dev_alloc(&ctx->d_Wp, L * N * d));
+  CR(dev_alloc(&ctx->d_br, L * N));
+  CR(dev_alloc(&ctx->d_bp, L * N));
+  CR(dev_alloc(&ctx->d_w, L * N));
+  CR(dev_alloc(&ctx->d_theta, L * (N - k + 1)));
+  CR(cudaMemset(ctx->d_br, 0, L * N * sizeof(float)));
+  CR(cudaMemset(ctx->d_bp, 0, L * N * sizeof(float)));
+  CR(cudaMemset(ctx->d_w, 0, L * N * sizeof(float)));
+  CR(cudaMemset(ctx->d_theta, 0, L * (N - k + 1) * sizeof(float)));
+  ctx->has_br.assign(L, 0);
+  ctx->has_bp.assign(L, 0);
+  ctx->has_cdf.assign(L, 0);
+  CR(dev_alloc(&ctx->d_cache, L * C * ctx->expert_bytes));
+  CR(dev_alloc(&ctx->d_slot_ready, L * C));
+  CR(cudaMemset(ctx->d_slot_ready, 0, L * C * sizeof(uint32_t)));
+  CR(dev_alloc(&ctx->d_zp, MB * N));
+  CR(dev_alloc(&ctx->d_qp, MB * N));
+  CR(dev_alloc(&ctx->d_zr, MB * N));
+  CR(dev_alloc(&ctx->d_pi, MB * N));
+  CR(dev_alloc(&ctx->d_ncand, MB));
+  CR(dev_alloc(&ctx->d_stats, L));
+  CR(cudaMemset(ctx->d_stats, 0, L * sizeof(DevStats)));
+  CR(dev_alloc(&ctx->d_counters, 4));
+  CR(cudaMemset(ctx->d_counters, 0, 4 * sizeof(unsigned long long)));
+  const size_t max_pairs = MB * (k + 1);
+  CR(dev_alloc(&ctx->d_plan_exec_idx, MB * k));
+  CR(dev_alloc(&ctx->d_plan_exec_gate, MB * k));
+  CR(dev_alloc(&ctx->d_pair_tok, max_pairs));
+  CR(dev_alloc(&ctx->d_pair_gate, max_pairs));
+  CR(dev_alloc(&ctx->d_pair_expert, max_pairs));
+  CR(dev_alloc(&ctx->d_n_pairs, 4));
+  CR(dev_alloc(&ctx->d_cand, MB * C));
+  CR(dev_alloc(&ctx->d_idx, MB * k));
+  CR(dev_alloc(&ctx->d_exec_idx, MB * k));
+  CR(dev_alloc(&ctx->d_alpha, MB * N));
+  CR(dev_alloc(&ctx->d_exec_gate, MB * k));
+  CR(dev_alloc(&ctx->d_cand_ncand, MB));
+  ctx->attn_bytes = (4 * d * d + 2 * (size_t)ctx->cfg.ctx_len * d) * 2;
+  ctx->attn_layers = L < 8 ? L : 8;
+  CR(dev_alloc(&ctx->d_attn, ctx->attn_bytes * ctx->attn_layers));
+  CR(cudaMemset(ctx->d_attn, 0, ctx->attn_bytes * ctx->attn_layers));
+  CR(dev_alloc(&ctx->d_attn_sink, 4));
+
+  // mapped mailbox
+  MailboxLayout& ml = ctx->ml;
+  size_t off = sizeof(MailboxHeader);
+  ml.off_ncand = off; off += MB * sizeof(int32_t);
+  ml.off_cand = off;  off += MB * C * sizeof(int32_t);
+  ml.off_kr = off;    off += MB * k * sizeof(int32_t);
+  ml.off_exec = off;  off += MB * k * sizeof(int32_t);
+  ml.bytes = off;
+  CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->mbox), ml.bytes, cudaHostAllocMapped | cudaHostAllocPortable));
+  memset(ctx->mbox, 0, ml.bytes);
+  ctx->gen_src_len = 1 << 16;
+  CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->gen_src), ctx->gen_src_len * sizeof(uint32_t), cudaHostAllocPortable));
+
+  CR(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+  ctx->cur_copy_stream = ctx->copy_stream;
+  CR(cudaEventCreateWithFlags(&ctx->ev_wave, cudaEventDisableTiming));
+  CR(cudaEventCreateWithFlags(&ctx->ev_in, cudaEventDisableTiming));
+#undef CR
+  {
+    void* fn = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
+        qr == cudaDriverEntryPointSuccess)
+      ctx->fn_write_value32 = fn;
+    cudaGetLastError();
+  }
+  ctx->tables.reserve(L);
+  for (size_t l = 0; l < L; ++l) ctx->tables.emplace_back((int)N, (int)C, c.cache_reuse != 0);
+  ctx->store_base.assign(L, nullptr);
+  ctx->store_stride.assign(L, 0);
+  ctx->shared_dev.assign(L, nullptr);
+  ctx->slot_gen.assign(L, std::vector<uint32_t>(C, 0u));
+  ctx->phys_expert.assign(L, std::vector<int32_t>(C, -1));
+  ctx->last_copies.assign(L, {});
+  ctx->host_stats.assign(L, apex_step_stats{});
+  ctx->step.assign(L, apex_ctx::StepState{});
+  *out = ctx;
+  return APEX_OK;
+}
+
+int apex_destroy(apex_ctx* ctx) {
+  if (!ctx) return APEX_EINVAL;
+  cudaDeviceSynchronize();
+  cudaGetLastError();
+  void* dev[] = {ctx->d_Wr, ctx->d_br, ctx->d_Wp, ctx->d_bp, ctx->d_w, ctx->d_theta, ctx->d_cache, ctx->d_slot_ready, ctx->d_zp,
+                 ctx->d_qp, ctx->d_zr, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_plan_exec_idx,
+                 ctx->d_plan_exec_gate, ctx->d_pair_tok, ctx->d_pair_gate, ctx->d_pair_expert, ctx->d_n_pairs, ctx->d_cand,
+                 ctx->d_idx, ctx->d_exec_idx, ctx->d_alpha, ctx->d_exec_gate, ctx->d_cand_ncand, ctx->d_attn, ctx->d_attn_sink,
+                 ctx->d_h_stage, ctx->d_hp_stage, ctx->d_y_stage};
+  for (void* p : dev)
+    if (p) cudaFree(p);
+  if (ctx->mbox) cudaFreeHost(ctx->mbox);
+  if (ctx->gen_src) cudaFreeHost(ctx->gen_src);
+  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->ev_wave) cudaEventDestroy(ctx->ev_wave);
+  if (ctx->ev_in) cudaEventDestroy(ctx->ev_in);
+  delete ctx;
+  return APEX_OK;
+}
+
+const char* apex_last_error(const apex_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+
+int apex_set_router(apex_ctx* ctx, int layer, const float* W, const float* b) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!W) return fail(ctx, APEX_EINVAL, "W_r is null");
+  const size_t N = ctx->cfg.N, d = ctx->cfg.d;
+  CU_TRY(ctx, cudaMemcpy(ctx->d_Wr + (size_t)layer * N * d, W, N * d * sizeof(float), cudaMemcpyHostToDevice));
+  if (b) CU_TRY(ctx, cudaMemcpy(ctx->d_br + (size_t)layer * N, b, N * sizeof(float), cudaMemcpyHostToDevice));
+  ctx->has_br[layer] = b ? 1 : 0;
+  return APEX_OK;
+}
+
+int apex_set_prefetch_router(apex_ctx* ctx, int layer, const float* W, const float* b) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!W) return fail(ctx, APEX_EINVAL, "W_p is null");
+  const size_t N = ctx->cfg.N, d = ctx->cfg.d;
+  CU_TRY(ctx, cudaMemcpy(ctx->d_Wp + (size_t)layer * N * d, W, N * d * sizeof(float), cudaMemcpyHostToDevice));
+  if (b) CU_TRY(ctx, cudaMemcpy(ctx->d_bp + (size_t)layer * N, b, N * sizeof(float), cudaMemcpyHostToDevice));
+  ctx->has_bp[layer] = b ? 1 : 0;
+  return APEX_OK;
+}
+
+int apex_set_cdf(apex_ctx* ctx, int layer, const float* w, const float* theta) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!w || !theta) return fail(ctx, APEX_EINVAL, "w or theta is null");
+  const size_t N = ctx->cfg.N, nth = ctx->cfg.N - ctx->cfg.k + 1;
+  for (size_t i = 1; i < nth; ++i)
+    if (!(theta[i] >= theta[i - 1])) return fail(ctx, APEX_EINVAL, "theta must be non-decreasing");
+  CU_TRY(ctx, cudaMemcpy(ctx->d_w + (size_t)layer * N, w, N * sizeof(float), cudaMemcpyHostToDevice));
+  CU_TRY(ctx, cudaMemcpy(ctx->d_theta + (size_t)layer * nth, theta, nth * sizeof(float), cudaMemcpyHostToDevice));
+  ctx->has_cdf[layer] = 1;
+  return APEX_OK;
+}
+
+int apex_register_experts(apex_ctx* ctx, int layer, const void* base, size_t stride) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!base || stride < ctx->expert_bytes || (stride & 15) || ((uintptr_t)base & 15))
+    return fail(ctx, APEX_EINVAL, "expert store: null base, stride below 3*I*d*2 or not 16-byte aligned");
+  ctx->store_base[layer] = static_cast<const uint8_t*>(base);
+  ctx->store_stride[layer] = stride;
+  return APEX_OK;
+}
+
+int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (ctx->cfg.I_shared <= 0) return fail(ctx, APEX_EINVAL, "the context was created with I_shared = 0");
+  if (!dev_weights || ((uintptr_t)dev_weights & 15)) return fail(ctx, APEX_EINVAL, "shared expert: null or unaligned");
+  ctx->shared_dev[layer] = static_cast<const uint8_t*>(dev_weights);
+  return APEX_OK;
+}
+
+int apex_pack_expert(const void* gate, const void* up, const void* down, int d, int I, void* dst) {
+  if (!gate || !up || !down || !dst || d < 1 || I < 1) return APEX_EINVAL;
+  const uint16_t* dn = static_cast<const uint16_t*>(down);
+  uint16_t* o = static_cast<uint16_t*>(dst);
+  const size_t m = (size_t)I * d;
+  memcpy(o, gate, m * 2);
+  memcpy(o + m, up, m * 2);
+  uint16_t* dT = o + 2 * m;
+  for (int j = 0; j < d; ++j)
+    for (int i = 0; i < I; ++i) dT[(size_t)i * d + j] = dn[(size_t)j * I + i];
+  return APEX_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+
+int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!h_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_predict: bad h or B");
+  const size_t N = ctx->cfg.N, d = ctx->cfg.d;
+  ctx->tables[layer].begin_step();
+  ctx->last_copies[layer].clear();
+  ctx->step[layer] = apex_ctx::StepState{};
+  ctx->step[layer].B = B;
+  RouterParams p{};
+  p.W = ctx->d_Wp + (size_t)layer * N * d;
+  p.bias = ctx->has_bp[layer] ? ctx->d_bp + (size_t)layer * N : nullptr;
+  p.x = h_dev;
+  p.z_out = ctx->d_zp;
+  p.q_out = ctx->d_qp;
+  p.pi_out = ctx->d_pi;
+  p.topk_out = nullptr;
+  p.N = (int)N; p.d = (int)d; p.B = B; p.k = ctx->cfg.k; p.C = ctx->cfg.C;
+  CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
+  ++ctx->launches;
+  ctx->pred_stream = (cudaStream_t)stream;
+  ctx->step[layer].predicted = true;
+  ctx->host_stats[layer].layer_steps += 1;
+  return APEX_OK;
+}
+
+int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* cand_dev, int32_t* ncand_dev, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  auto& st = ctx->step[layer];
+  if (!st.predicted || st.B != B) return fail(ctx, APEX_ESTATE, "apex_select_candidates needs apex_predict of the same layer-step and B");
+  if (!cand_dev || !ncand_dev) return fail(ctx, APEX_EINVAL, "null output");
+  if (!ctx->has_cdf[layer]) return fail(ctx, APEX_ESTATE, "no confidence model set for this layer");
+  if (!(tau == tau)) return fail(ctx, APEX_EINVAL, "tau is NaN");
+  const int N = ctx->cfg.N, k = ctx->cfg.k;
+  SelectParams p{};
+  p.q = ctx->d_qp;
+  p.pi = ctx->d_pi;
+  p.w = ctx->d_w + (size_t)layer * N;
+  p.theta = ctx->d_theta + (size_t)layer * (N - k + 1);
+  p.cand_out = cand_dev;
+  p.ncand_out = ncand_dev;
+  p.ncand_keep = ctx->d_ncand;
+  p.mbox_cand = mbox_i32(ctx, ctx->ml.off_cand);
+  p.mbox_ncand = mbox_i32(ctx, ctx->ml.off_ncand);
+  p.mbox_seq = &mhdr(ctx)->sel_seq;
+  p.seq_value = ++ctx->sel_seq;
+  ctx->sel_done += (unsigned long long)B;
+  p.done_counter = ctx->d_counters + 0;
+  p.done_target = ctx->sel_done;
+  p.stats = ctx->d_stats + layer;
+  p.force = tau <= 0.f ? 1 : (tau >= 1.f ? 2 : 0);
+  p.t_tau = p.force ? 0.f : (float)std::log((double)tau / (1.0 - (double)tau));
+  p.N = N; p.k = k; p.C = ctx->cfg.C; p.B = B;
+  CU_TRY(ctx, launch_select(p, (cudaStream_t)stream));
+  ++ctx->launches;
+  st.selected = true;
+  return APEX_OK;
+}
+
+int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  auto& st = ctx->step[layer];
+  if (!st.selected || st.B != B) return fail(ctx, APEX_ESTATE, "apex_prefetch needs apex_select_candidates of the same layer-step and B");
+  if (st.prefetched) return fail(ctx, APEX_ESTATE, "apex_prefetch called twice in one layer-step");
+  ctx->cur_copy_stream = copy_stream ? (cudaStream_t)copy_stream : ctx->copy_stream;
+  if (!host_wait_seq(ctx, &mhdr(ctx)->sel_seq, ctx->sel_seq))
+    return fail(ctx, APEX_ETIMEOUT, "apex_prefetch: candidate lists did not arrive");
+  const int C = ctx->cfg.C;
+  const int32_t* ncand = mbox_i32(ctx, ctx->ml.off_ncand);
+  const int32_t* cand = mbox_i32(ctx, ctx->ml.off_cand);
+  std::vector<SlotCopy> copies;
+  if (!ctx->tables[layer].plan_prefetch(cand, ncand, B, C, &copies)) return fail(ctx, APEX_ESTATE, "no evictable slot");
+  // issue most likely first: order of appearance in the first token's ranked list, others after
+  if (B == 1 && copies.size() > 1) {
+    int pos[APEX_MAX_EXPERTS];
+    for (int e = 0; e < APEX_MAX_EXPERTS; ++e) pos[e] = 1 << 20;
+    for (int j = 0; j < ncand[0]; ++j) pos[cand[j]] = j;
+    std::vector<SlotCopy> ordered = copies;
+    std::stable_sort(ordered.begin(), ordered.end(), [&](const SlotCopy& a, const SlotCopy& b) { return pos[a.expert] < pos[b.expert]; });
+    for (const auto& c : ordered) {
+      int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+      if (r != APEX_OK) return r;
+    }
+  } else {
+    for (const auto& c : copies) {
+      int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+      if (r != APEX_OK) return r;
+    }
+  }
+  ctx->host_stats[layer].prefetch_copies += (int64_t)copies.size();
+  ctx->last_copies[layer].insert(ctx->last_copies[layer].end(), copies.begin(), copies.end());
+  st.prefetched = true;
+  return APEX_OK;
+}
+
+int apex_attention_standin(apex_ctx* ctx, int layer, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  AttnParams p{};
+  p.buf = reinterpret_cast<const uint4*>(ctx->d_attn + (size_t)(layer % ctx->attn_layers) * ctx->attn_bytes);
+  p.n_vec = ctx->attn_bytes / 16;
+  p.sink = ctx->d_attn_sink;
+  CU_TRY(ctx, launch_attention(p, ctx->n_sm, (cudaStream_t)stream));
+  ++ctx->launches;
+  return APEX_OK;
+}
+
+int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int32_t* idx_dev, float* alpha_dev, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!hpost_dev || !idx_dev || !alpha_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_route_topk: bad argument");
+  auto& st = ctx->step[layer];
+  if (st.predicted && st.B != B) return fail(ctx, APEX_ESTATE, "B differs from apex_predict of this layer-step");
+  if (!st.predicted) {  // gate used on its own (no prefetch stage): still one layer-step
+    ctx->tables[layer].begin_step();
+    ctx->last_copies[layer].clear();
+    st = apex_ctx::StepState{};
+    st.B = B;
+    ctx->host_stats[layer].layer_steps += 1;
+  }
+  const size_t N = ctx->cfg.N, d = ctx->cfg.d;
+  RouterParams p{};
+  p.W = ctx->d_Wr + (size_t)layer * N * d;
+  p.bias = ctx->has_br[layer] ? ctx->d_br + (size_t)layer * N : nullptr;
+  p.x = hpost_dev;
+  p.z_out = ctx->d_zr;
+  p.q_out = alpha_dev;
+  p.pi_out = nullptr;
+  p.topk_out = idx_dev;
+  p.N = (int)N; p.d = (int)d; p.B = B; p.k = ctx->cfg.k; p.C = ctx->cfg.C;
+  p.pi_pred = st.selected ? ctx->d_pi : nullptr;
+  p.ncand_pred = st.selected ? ctx->d_ncand : nullptr;
+  p.resident_mask = ctx->tables[layer].resident_mask();
+  p.stats = ctx->d_stats + layer;
+  p.mbox_kr = mbox_i32(ctx, ctx->ml.off_kr);
+  p.mbox_seq = &mhdr(ctx)->route_seq;
+  p.seq_value = ++ctx->route_seq;
+  ctx->route_done += (unsigned long long)B;
+  p.done_counter = ctx->d_counters + 1;
+  p.done_target = ctx->route_done;
+  CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
+  ++ctx->launches;
+  st.routed = true;
+  st.idx_dev = idx_dev;
+  st.alpha_dev = alpha_dev;
+  return APEX_OK;
+}
+
+int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev, int32_t* exec_idx_dev,
+                 float* exec_gate_dev, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  auto& st = ctx->step[layer];
+  if (!st.routed || st.B != B) return fail(ctx, APEX_ESTATE, "apex_moe_ffn needs apex_route_topk of the same layer-step and B");
+  if (!hpost_dev || !y_dev) return fail(ctx, APEX_EINVAL, "null h' or y");
+  if (mode != APEX_MODE_EXACT && mode != APEX_MODE_STALL_FREE) return fail(ctx, APEX_EINVAL, "unknown mode");
+  if (ctx->cfg.I_shared > 0 && !ctx->shared_dev[layer]) return fail(ctx, APEX_ESTATE, "shared expert not set for this layer");
+  cudaStream_t cs = (cudaStream_t)stream;
+  const int N = ctx->cfg.N, k = ctx->cfg.k, C = ctx->cfg.C;
+  auto& tab = ctx->tables[layer];
+
+  FfnParams p{};
+  p.hpost = hpost_dev;
+  p.y = y_dev;
+  p.idx = st.idx_dev;
+  p.alpha = st.alpha_dev;
+  p.z_r = ctx->d_zr;
+  p.exec_idx = exec_idx_dev;
+  p.exec_gate = exec_gate_dev;
+  p.cache = ctx->d_cache + (size_t)layer * C * ctx->expert_bytes;
+  p.shared_w = ctx->shared_dev[layer];
+  p.slot_ready = ctx->d_slot_ready + (size_t)layer * C;
+  p.plan_exec_idx = ctx->d_plan_exec_idx;
+  p.plan_exec_gate = ctx->d_plan_exec_gate;
+  p.pair_tok = ctx->d_pair_tok;
+  p.pair_gate = ctx->d_pair_gate;
+  p.pair_expert = ctx->d_pair_expert;
+  p.n_pairs = ctx->d_n_pairs;
+  p.mbox_exec = mbox_i32(ctx, ctx->ml.off_exec);
+  p.mbox_seq = &mhdr(ctx)->exec_seq;
+  p.mbox_status = &mhdr(ctx)->status;
+  p.seq_value = ++ctx->exec_seq;
+  p.stats = ctx->d_stats + layer;
+  p.zero_counter = ctx->d_counters + 2;
+  ctx->zero_done += (unsigned long long)ctx->n_sm;
+  p.zero_target = ctx->zero_done;
+  p.snap = make_snapshot(ctx, layer);
+  p.run_mask = p.snap.resident_mask;
+  p.slot_stride = ctx->expert_bytes;
+  p.wait_limit_ns = ctx->cfg.wait_limit_ns;
+  p.d = ctx->cfg.d; p.N = N; p.k = k; p.I = ctx->cfg.I; p.I_shared = ctx->cfg.I_shared; p.B = B;
+  p.mode = mode; p.norm_topk = ctx->cfg.norm_topk; p.accumulate = 0;
+  p.run_shared = ctx->cfg.I_shared > 0 ? 1 : 0;
+  p.post_exec = 1;
+  if (B > 1) {
+    CU_TRY(ctx, launch_ffn_plan(p, cs));
+    ++ctx->launches;
+  }
+  CU_TRY(ctx, launch_ffn(p, ctx->n_sm, cs));
+  ++ctx->launches;
+
+  // the gate's decision arrives through the mailbox while the first wave runs
+  if (!host_wait_seq(ctx, &mhdr(ctx)->route_seq, ctx->route_seq)) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
+  const int32_t* K_r = mbox_i32(ctx, ctx->ml.off_kr);
+  if (mode == APEX_MODE_EXACT) {
+    std::vector<SlotCopy> copies;
+    uint64_t need = 0;
+    const std::vector<int32_t> slot_expert_before = tab.slot_expert();
+    if (!tab.plan_demand(K_r, B, k, &copies, &need)) return fail(ctx, APEX_ESTATE, "no evictable slot");
+    int n_waves = 0;
+    for (const auto& c : copies) n_waves = c.wave > n_waves ? c.wave : n_waves;
+    for (int w = 1; w <= n_waves; ++w) {
+      // a victim that an earlier wave of this step may still be reading: order the copy after that wave
+      bool hazard = false;
+      uint64_t chunk = 0;
+      for (const auto& c : copies)
+        if (c.wave == w) {
+          chunk |= (1ull << c.expert);
+          const int prev = w == 1 ? slot_expert_before[c.slot] : -2;
+          if (w > 1 || (prev >= 0 && ((need >> prev) & 1))) hazard = true;
+        }
+      if (hazard) {
+        CU_TRY(ctx, cudaEventRecord(ctx->ev_wave, cs));
+        CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_stream, ctx->ev_wave, 0));
+      }
+      for (const auto& c : copies)
+        if (c.wave == w) {
+          int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+          if (r != APEX_OK) return r;
+        }
+      FfnParams q = p;
+      q.snap = make_snapshot(ctx, layer);
+      q.run_mask = chunk;
+      q.accumulate = 1;
+      q.run_shared = 0;
+      q.post_exec = 0;
+      if (B > 1) {
+        CU_TRY(ctx, launch_ffn_plan(q, cs));
+        ++ctx->launches;
+      }
+      CU_TRY(ctx, launch_ffn(q, ctx->n_sm, cs));
+      ++ctx->launches;
+      ctx->host_stats[layer].extra_waves += 1;
+    }
+    ctx->host_stats[layer].demand_copies += (int64_t)copies.size();
+    ctx->last_copies[layer].insert(ctx->last_copies[layer].end(), copies.begin(), copies.end());
+  } else {
+    if (!host_wait_seq(ctx, &mhdr(ctx)->exec_seq, ctx->exec_seq)) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: execution sets did not arrive");
+    const int32_t* ex = mbox_i32(ctx, ctx->ml.off_exec);
+    for (int i = 0; i < B * k; ++i) tab.touch(ex[i]);
+  }
+  st.routed = false;  // the layer-step is complete
+  st.predicted = false;
+  st.selected = false;
+  return check_device_status(ctx);
+}
+
+int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev, int B, float tau, int mode, float* y_dev,
+                      void* stream) {
+  CHECK_CTX(ctx);
+  if (!h_dev || !hpost_dev || !y_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_decode_token: bad argument");
+  const size_t step = (size_t)B * ctx->cfg.d;
+  for (int l = 0; l < ctx->cfg.L; ++l) {
+    int r;
+    if ((r = apex_predict(ctx, l, h_dev + l * step, B, stream)) != APEX_OK) return r;
+    if ((r = apex_select_candidates(ctx, l, B, tau, ctx->d_cand, ctx->d_cand_ncand, stream)) != APEX_OK) return r;
+    if ((r = apex_prefetch(ctx, l, B, nullptr)) != APEX_OK) return r;
+    if ((r = apex_attention_standin(ctx, l, stream)) != APEX_OK) return r;
+    if ((r = apex_route_topk(ctx, l, hpost_dev + l * step, B, ctx->d_idx, ctx->d_alpha, stream)) != APEX_OK) return r;
+    if ((r = apex_moe_ffn(ctx, l, mode, hpost_dev + l * step, B, y_dev + l * step, ctx->d_exec_idx, ctx->d_exec_gate, stream)) != APEX_OK)
+      return r;
+  }
+  return APEX_OK;
+}
+
+int apex_decode_token_host(apex_ctx* ctx, const float* h_host, const float* hpost_host, int B, float tau, int mode,
+                           float* y_host, void* stream) {
+  CHECK_CTX(ctx);
+  if (!h_host || !hpost_host || !y_host || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_decode_token_host: bad argument");
+  const size_t n = (size_t)ctx->cfg.L * ctx->cfg.max_batch * ctx->cfg.d;
+  if (!ctx->d_h_stage) {
+    CU_TRY(ctx, dev_alloc(&ctx->d_h_stage, n));
+    CU_TRY(ctx, dev_alloc(&ctx->d_hp_stage, n));
+    CU_TRY(ctx, dev_alloc(&ctx->d_y_stage, n));
+  }
+  cudaStream_t cs = (cudaStream_t)stream;
+  const size_t bytes = (size_t)ctx->cfg.L * B * ctx->cfg.d * sizeof(float);
+  CU_TRY(ctx, cudaMemcpyAsync(ctx->d_h_stage, h_host, bytes, cudaMemcpyHostToDevice, cs));
+  CU_TRY(ctx, cudaMemcpyAsync(ctx->d_hp_stage, hpost_host, bytes, cudaMemcpyHostToDevice, cs));
+  int r = apex_decode_token(ctx, ctx->d_h_stage, ctx->d_hp_stage, B, tau, mode, ctx->d_y_stage, stream);
+  if (r != APEX_OK) return r;
+  CU_TRY(ctx, cudaMemcpyAsync(y_host, ctx->d_y_stage, bytes, cudaMemcpyDeviceToHost, cs));
+  CU_TRY(ctx, cudaStreamSynchronize(cs));
+  return check_device_status(ctx);
+}
+
+// ---------------------------------------------------------------------------------------------
+
+static void add_dev_stats(apex_step_stats* o, const DevStats& s, int n_sm) {
+  o->tokens += (int64_t)s.tokens;
+  o->sum_delta_hat += (int64_t)s.sum_delta_hat;
+  o->sum_delta_star += (int64_t)s.sum_delta_star;
+  o->sum_ncand += (int64_t)s.sum_ncand;
+  o->capped += (int64_t)s.capped;
+  o->routed += (int64_t)s.routed;
+  o->hits_P += (int64_t)s.hits_P;
+  o->hits_R += (int64_t)s.hits_R;
+  o->covered += (int64_t)s.covered;
+  o->substitutions += (int64_t)s.substitutions;
+  o->stall_ns += (int64_t)(s.stall_ns / (unsigned long long)(n_sm > 0 ? n_sm : 1));
+  o->timeouts += (int64_t)s.timeouts;
+  o->near_full_prefetch += (int64_t)s.near_full;
+}
+
+int apex_get_stats(apex_ctx* ctx, int layer, apex_step_stats* out) {
+  CHECK_CTX(ctx);
+  if (!out || layer < -1 || layer >= ctx->cfg.L) return fail(ctx, APEX_EINVAL, "apex_get_stats: bad argument");
+  CU_TRY(ctx, cudaDeviceSynchronize());
+  std::vector<DevStats> ds(ctx->cfg.L);
+  CU_TRY(ctx, cudaMemcpy(ds.data(), ctx->d_stats, ds.size() * sizeof(DevStats), cudaMemcpyDeviceToHost));
+  memset(out, 0, sizeof *out);
+  for (int l = 0; l < ctx->cfg.L; ++l) {
+    if (layer >= 0 && l != layer) continue;
+    const apex_step_stats& h = ctx->host_stats[l];
+    out->layer_steps += h.layer_steps;
+    out->prefetch_copies += h.prefetch_copies;
+    out->demand_copies += h.demand_copies;
+    out->bytes_copied += h.bytes_copied;
+    out->extra_waves += h.extra_waves;
+    add_dev_stats(out, ds[l], ctx->n_sm);
+  }
+  return APEX_OK;
+}
+
+int apex_reset_stats(apex_ctx* ctx) {
+  CHECK_CTX(ctx);
+  CU_TRY(ctx, cudaDeviceSynchronize());
+  CU_TRY(ctx, cudaMemset(ctx->d_stats, 0, ctx->cfg.L * sizeof(DevStats)));
+  for (auto& h : ctx->host_stats) h = apex_step_stats{};
+  return APEX_OK;
+}
+
+int apex_read_prediction(apex_ctx* ctx, int B, float* z_p, float* q_p, int32_t* pi) {
+  CHECK_CTX(ctx);
+  if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "bad B");
+  CU_TRY(ctx, cudaStreamSynchronize(ctx->pred_stream));
+  const size_t n = (size_t)B * ctx->cfg.N;
+  if (z_p) CU_TRY(ctx, cudaMemcpy(z_p, ctx->d_zp, n * sizeof(float), cudaMemcpyDeviceToHost));
+  if (q_p) CU_TRY(ctx, cudaMemcpy(q_p, ctx->d_qp, n * sizeof(float), cudaMemcpyDeviceToHost));
+  if (pi) CU_TRY(ctx, cudaMemcpy(pi, ctx->d_pi, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
+  return APEX_OK;
+}
+
+int apex_get_last_copies(apex_ctx* ctx, int layer, int32_t* expert, int32_t* slot, int32_t* n_prefetch, int32_t* n_demand) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  int np = 0, nd = 0, i = 0;
+  for (const auto& c : ctx->last_copies[layer]) {
+    if (expert) expert[i] = c.expert;
+    if (slot) slot[i] = c.slot;
+    ++i;
+    if (c.wave == 0) ++np; else ++nd;
+  }
+  if (n_prefetch) *n_prefetch = np;
+  if (n_demand) *n_demand = nd;
+  return APEX_OK;
+}
+
+int apex_get_slot_table(apex_ctx* ctx, int layer, int32_t* expert_slot, int64_t* slot_stamp, int64_t* clock) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  ctx->tables[layer].get(expert_slot, slot_stamp, clock);
+  return APEX_OK;
+}
+
+int apex_set_slot_table(apex_ctx* ctx, int layer, const int32_t* expert_slot, const int64_t* slot_stamp, int64_t clock) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!expert_slot || !slot_stamp) return fail(ctx, APEX_EINVAL, "null table");
+  if (!ctx->tables[layer].set(expert_slot, slot_stamp, clock)) return fail(ctx, APEX_EINVAL, "inconsistent slot table");
+  // slots whose bytes belong to another expert are refilled
+  CU_TRY(ctx, cudaDeviceSynchronize());
+  for (int e = 0; e < ctx->cfg.N; ++e) {
+    const int s = expert_slot[e];
+    if (s >= 0 && ctx->phys_expert[layer][s] != e) {
+      int r = issue_copy(ctx, layer, e, s, ctx->cur_copy_stream);
+      if (r != APEX_OK) return r;
+    }
+  }
+  return APEX_OK;
+}
+
+int apex_warm_all(apex_ctx* ctx) {
+  CHECK_CTX(ctx);
+  if (ctx->cfg.C != ctx->cfg.N) return fail(ctx, APEX_ESTATE, "apex_warm_all needs C == N");
+  std::vector<int32_t> es(ctx->cfg.N);
+  std::vector<int64_t> stamp(ctx->cfg.C, 0);
+  for (int e = 0; e < ctx->cfg.N; ++e) es[e] = e;
+  for (int l = 0; l < ctx->cfg.L; ++l) {
+    int r = apex_set_slot_table(ctx, l, es.data(), stamp.data(), ctx->tables[l].clock());
+    if (r != APEX_OK) return r;
+  }
+  CU_TRY(ctx, cudaStreamSynchronize(ctx->cur_copy_stream));
+  return APEX_OK;
+}
+
+int apex_test_inject(apex_ctx* ctx, int what) {
+  CHECK_CTX(ctx);
+  if (what < 0 || what > 2) return fail(ctx, APEX_EINVAL, "unknown injection");
+  ctx->inject = what;
+  return APEX_OK;
+}
+
+int64_t apex_launch_count(const apex_ctx* ctx) { return ctx ? ctx->launches : -1; }
+
+// ---- host-only slot planner ---------------------------------------------------------------------
+
+struct apex_slots {
+  SlotTable t;
+  apex_slots(int N, int C, bool r) : t(N, C, r) {}
+};
+
+apex_slots* apex_slots_create(int N, int C, int cache_reuse) {
+  if (N < 1 || N > APEX_MAX_EXPERTS || C < 1 || C > N) return nullptr;
+  return new (std::nothrow) apex_slots(N, C, cache_reuse != 0);
+}
+void apex_slots_destroy(apex_slots* s) { delete s; }
+int apex_slots_begin_step(apex_slots* s) {
+  if (!s) return APEX_EINVAL;
+  s->t.begin_step();
+  return APEX_OK;
+}
+int apex_slots_prefetch(apex_slots* s, const int32_t* cand, const int32_t* ncand, int B, int stride, int32_t* copy_expert,
+                        int32_t* copy_slot, int32_t* n_copies) {
+  if (!s || !cand || !ncand || !n_copies || B < 1) return APEX_EINVAL;
+  std::vector<SlotCopy> cp;
+  if (!s->t.plan_prefetch(cand, ncand, B, stride, &cp)) return APEX_ESTATE;
+  for (size_t i = 0; i < cp.size(); ++i) {
+    if (copy_expert) copy_expert[i] = cp[i].expert;
+    if (copy_slot) copy_slot[i] = cp[i].slot;
+  }
+  *n_copies = (int32_t)cp.size();
+  return APEX_OK;
+}
+int apex_slots_demand(apex_slots* s, const int32_t* K_r, int B, int k, int32_t* copy_expert, int32_t* copy_slot,
+                      int32_t* wave_of_copy, int32_t* n_copies) {
+  if (!s || !K_r || !n_copies || B < 1 || k < 1) return APEX_EINVAL;
+  std::vector<SlotCopy> cp;
+  if (!s->t.plan_demand(K_r, B, k, &cp)) return APEX_ESTATE;
+  for (size_t i = 0; i < cp.size(); ++i) {
+    if (copy_expert) copy_expert[i] = cp[i].expert;
+    if (copy_slot) copy_slot[i] = cp[i].slot;
+    if (wave_of_copy) wave_of_copy[i] = cp[i].wave;
+  }
+  *n_copies = (int32_t)cp.size();
+  return APEX_OK;
+}
+int apex_slots_touch(apex_slots* s, const int32_t* experts, int n) {
+  if (!s || (!experts && n > 0)) return APEX_EINVAL;
+  for (int i = 0; i < n; ++i) s->t.touch(experts[i]);
+  return APEX_OK;
+}
+int apex_slots_get(const apex_slots* s, int32_t* expert_slot, int64_t* slot_stamp, int64_t* clock) {
+  if (!s) return APEX_EINVAL;
+  s->t.get(expert_slot, slot_stamp, clock);
+  return APEX_OK;
+}
+int apex_slots_set(apex_slots* s, const int32_t* expert_slot, const int64_t* slot_stamp, int64_t clock) {
+  if (!s || !expert_slot || !slot_stamp) return APEX_EINVAL;
+  return s->t.set(expert_slot, slot_stamp, clock) ? APEX_OK : APEX_EINVAL;
+}
+
+}  // extern "C"

@@ -1,0 +1,199 @@
+// Internal declarations shared by the translation units of libapex.so.
+#pragma once
+#include <cuda_runtime.h>
+
+#include <cstdint>
+#include <string>
+#include <vector>
+
+#include "../../include/apex.h"
+#include "slot_table.hpp"
+
+namespace apex {
+
+// ---- mapped host mailbox: the kernels post small decision records here so that the host can
+// plan copies without a stream synchronisation.  One per context; sequence numbers only grow.
+struct MailboxHeader {
+  volatile uint32_t sel_seq;    // written by the candidate-selection kernel, after the lists
+  volatile uint32_t route_seq;  // written by the gate kernel, after K_r
+  volatile uint32_t exec_seq;   // written by the plan step of the FFN, after the execution sets
+  volatile uint32_t status;     // sticky device status (0 ok, 1 wait ran out)
+};
+
+struct MailboxLayout {
+  size_t off_ncand, off_cand, off_kr, off_exec, bytes;
+};
+
+// Device-side counters of one layer (S9), accumulated with 64-bit atomics.
+struct DevStats {
+  unsigned long long tokens, sum_delta_hat, sum_delta_star, sum_ncand, capped, routed, hits_P, hits_R, covered,
+      substitutions, stall_ns, timeouts, near_full;
+};
+
+// Small tables handed to kernels by value at launch: a snapshot of the layer's slot table.
+struct SlotSnapshot {
+  int8_t expert_slot[APEX_MAX_EXPERTS];   // -1 = not resident
+  uint32_t need_gen[APEX_MAX_EXPERTS];    // slot-ready value to wait for
+  unsigned long long resident_mask;
+};
+
+struct RouterParams {
+  const float* W;     // [N][d]
+  const float* bias;  // [N] or null
+  const float* x;     // [B][d]
+  float* z_out;       // [B][N]
+  float* q_out;       // [B][N] softmax
+  int32_t* pi_out;    // [B][N] ranking, or null
+  int32_t* topk_out;  // [B][k] or null
+  int N, d, B, k;
+  int warps_per_cta;
+  // gate-kernel epilogue (S9 metrics + mailbox); all null/0 for the prefetch router
+  const int32_t* pi_pred;     // [B][N] ranking of the prefetch router for this step, or null
+  const int32_t* ncand_pred;  // [B]
+  unsigned long long resident_mask;
+  DevStats* stats;
+  int32_t* mbox_kr;                 // mapped host [B][k]
+  volatile uint32_t* mbox_seq;      // mapped host
+  uint32_t seq_value;
+  unsigned long long* done_counter; // device
+  unsigned long long done_target;
+  int C;
+};
+
+struct SelectParams {
+  const float* q;       // [B][N]
+  const int32_t* pi;    // [B][N]
+  const float* w;       // [N]
+  const float* theta;   // [N-k+1]
+  int32_t* cand_out;    // [B][C] device, caller's
+  int32_t* ncand_out;   // [B]
+  int32_t* ncand_keep;  // [B] context-owned copy for the metrics
+  int32_t* mbox_cand;   // mapped host [B][C]
+  int32_t* mbox_ncand;  // mapped host [B]
+  volatile uint32_t* mbox_seq;
+  uint32_t seq_value;
+  unsigned long long* done_counter;
+  unsigned long long done_target;
+  DevStats* stats;
+  float t_tau;
+  int force;  // 0: threshold test, 1: delta_hat = 0, 2: delta_hat = N-k
+  int N, k, C, B;
+};
+
+struct FfnParams {
+  const float* hpost;       // [B][d]
+  float* y;                 // [B][d]
+  const int32_t* idx;       // [B][k] K_r
+  const float* alpha;       // [B][N]
+  const float* z_r;         // [B][N]
+  int32_t* exec_idx;        // [B][k] out or null
+  float* exec_gate;         // [B][k] out or null
+  const uint8_t* cache;     // slot 0 of this layer
+  const uint8_t* shared_w;  // or null
+  const uint32_t* slot_ready;  // [C]
+  // batched plan (B > 1), context-owned
+  int32_t* plan_exec_idx;   // [B][k]
+  float* plan_exec_gate;    // [B][k]
+  int32_t* pair_tok;        // [B*k + B]
+  float* pair_gate;         // [B*k + B]
+  int32_t* pair_expert;     // [B*k + B]   (N = shared expert)
+  int32_t* n_pairs;         // [1]
+  int32_t* mbox_exec;       // mapped host [B][k]
+  volatile uint32_t* mbox_seq;
+  volatile uint32_t* mbox_status;
+  uint32_t seq_value;
+  DevStats* stats;
+  unsigned long long* zero_counter;
+  unsigned long long zero_target;
+  unsigned long long run_mask;  // experts this launch executes
+  SlotSnapshot snap;
+  size_t slot_stride;
+  long long wait_limit_ns;
+  int d, N, k, I, I_shared, B, mode, norm_topk, accumulate, run_shared, post_exec;
+};
+
+struct AttnParams {
+  const uint4* buf;
+  size_t n_vec;  // 16-byte vectors
+  float* sink;
+};
+
+// launchers (kernels_*.cu).  Each returns the cudaError_t of the launch.
+cudaError_t launch_router(const RouterParams& p, cudaStream_t s);
+cudaError_t launch_select(const SelectParams& p, cudaStream_t s);
+cudaError_t launch_attention(const AttnParams& p, int n_sm, cudaStream_t s);
+cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s);
+cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s);
+cudaError_t ffn_configure(int d);  // sets the dynamic shared-memory attribute once per shape
+bool ffn_shape_supported(int d);
+
+}  // namespace apex
+
+// ---- the context ----------------------------------------------------------------------------
+struct apex_ctx {
+  apex_config cfg;
+  std::string err;
+  int device = 0;
+  int n_sm = 0;
+  size_t expert_bytes = 0;   // 3*I*d*2
+  size_t shared_bytes = 0;
+
+  // device memory
+  float* d_Wr = nullptr;  // [L][N][d]
+  float* d_br = nullptr;  // [L][N]
+  float* d_Wp = nullptr;
+  float* d_bp = nullptr;
+  float* d_w = nullptr;      // [L][N]
+  float* d_theta = nullptr;  // [L][N-k+1]
+  std::vector<uint8_t> has_br, has_bp, has_cdf;
+  uint8_t* d_cache = nullptr;     // [L][C][expert_bytes]
+  uint32_t* d_slot_ready = nullptr;  // [L][C]
+  float *d_zp = nullptr, *d_qp = nullptr, *d_zr = nullptr;  // [maxB][N]
+  int32_t *d_pi = nullptr, *d_ncand = nullptr;              // [maxB][N], [maxB]
+  apex::DevStats* d_stats = nullptr;                        // [L]
+  unsigned long long* d_counters = nullptr;                 // [4]: select done, route done, zero, spare
+  int32_t *d_plan_exec_idx = nullptr, *d_pair_tok = nullptr, *d_pair_expert = nullptr, *d_n_pairs = nullptr;
+  float *d_plan_exec_gate = nullptr, *d_pair_gate = nullptr;
+  uint8_t* d_attn = nullptr;
+  size_t attn_bytes = 0, attn_layers = 1;
+  float* d_attn_sink = nullptr;
+  // scratch for apex_decode_token
+  int32_t *d_cand = nullptr, *d_cand_ncand = nullptr, *d_idx = nullptr, *d_exec_idx = nullptr;
+  float *d_alpha = nullptr, *d_exec_gate = nullptr;
+  float *d_h_stage = nullptr, *d_hp_stage = nullptr, *d_y_stage = nullptr;  // [L][maxB][d] for the host variant
+
+  // mapped host mailbox
+  uint8_t* mbox = nullptr;
+  apex::MailboxLayout ml{};
+  uint32_t sel_seq = 0, route_seq = 0, exec_seq = 0;
+  unsigned long long sel_done = 0, route_done = 0, zero_done = 0;
+  uint32_t* gen_src = nullptr;  // pinned ring of flag values for the ready-flag copies
+  size_t gen_src_pos = 0, gen_src_len = 0;
+
+  // host state per layer
+  std::vector<apex::SlotTable> tables;
+  std::vector<const uint8_t*> store_base;
+  std::vector<size_t> store_stride;
+  std::vector<const uint8_t*> shared_dev;
+  std::vector<std::vector<uint32_t>> slot_gen;  // [L][C] install count
+  std::vector<std::vector<int32_t>> phys_expert;  // [L][C] whose bytes the slot holds (or is receiving)
+  uint32_t* withheld_flag = nullptr;  // test hook: a ready flag that was not written
+  uint32_t withheld_gen = 0;
+  std::vector<std::vector<apex::SlotCopy>> last_copies;
+  std::vector<apex_step_stats> host_stats;
+  struct StepState {
+    int B = 0;
+    bool predicted = false, selected = false, prefetched = false, routed = false;
+    const int32_t* idx_dev = nullptr;
+    const float* alpha_dev = nullptr;
+  };
+  std::vector<StepState> step;
+
+  cudaStream_t copy_stream = nullptr;   // own
+  cudaStream_t cur_copy_stream = nullptr;
+  cudaStream_t pred_stream = nullptr;   // stream of the last apex_predict
+  cudaEvent_t ev_wave = nullptr, ev_in = nullptr;
+  int inject = 0;
+  int64_t launches = 0;
+  void* fn_write_value32 = nullptr;  // cuStreamWriteValue32 when the driver offers it
+};

@@ -1,0 +1,241 @@
+"""Lock-step comparison of the CUDA library with the CPU oracle on seeded synthetic inputs.
+
+Per layer-step the oracle is given the library's pre-step slot table, runs the step on the same
+inputs, and every decision is compared: ranking, budget, candidate set, slot plan, routed set,
+execution set, gates, demand plan, post-step table (bit-exact) and the FFN output (tolerance).
+A mismatch is excused only when the oracle flags the deciding comparison as a near-tie (logit gap
+below 1e-6, threshold margin below 1e-5); such steps are counted and reported."""
+from __future__ import annotations
+
+import dataclasses
+from typing import Dict, List, Optional
+
+import numpy as np
+import torch
+
+from oracle import apex_oracle as ao
+from paper_2608_11688_b200 import binding, build, synth
+
+REL_L2_TOL = 2e-3
+MAX_ABS_TOL = 2e-2
+
+
+@dataclasses.dataclass
+class Report:
+    layer_steps: int = 0
+    near_ties: int = 0
+    worst_rel_l2: float = 0.0
+    worst_max_abs: float = 0.0
+    n_miss_steps: int = 0
+    n_subst: int = 0
+    n_prefetch_copies: int = 0
+    n_demand_copies: int = 0
+    ffn_checked: int = 0
+
+
+class Problem:
+    """Parameters and expert stores of one config on the GPU machine, shared by library and oracle."""
+
+    def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset"):
+        self.cfg = cfg
+        self.L = layers or cfg.L
+        self.routers = [synth.router_weights(cfg, l) for l in range(self.L)]
+        self.cdf = [synth.handset_cdf_params(cfg) if cdf == "handset" else synth.cdf_params(cfg, l)
+                    for l in range(self.L)]
+        self.stores = []
+        self.shared = []
+        for l in range(self.L):
+            st = torch.empty((cfg.N, 3, cfg.I, cfg.d), dtype=torch.bfloat16, pin_memory=True)
+            tmp = synth.expert_store(cfg, l, device=device)
+            st.copy_(tmp)
+            del tmp
+            self.stores.append(st)
+            self.shared.append(synth.shared_expert(cfg, l, device=device))
+        torch.cuda.synchronize()
+
+    def make_ctx(self, *, C=None, max_batch=1, norm_topk=1, cache_reuse=1, wait_limit_ns=0) -> binding.Apex:
+        cfg = self.cfg
+        build.build()
+        a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C or cfg.C, L=self.L, I_shared=cfg.I_shared,
+                         max_batch=max_batch, norm_topk=norm_topk, cache_reuse=cache_reuse,
+                         wait_limit_ns=wait_limit_ns)
+        for l in range(self.L):
+            W_r, b_r, W_p, b_p = self.routers[l]
+            a.set_router(l, W_r, b_r)
+            a.set_prefetch_router(l, W_p, b_p)
+            a.set_cdf(l, *self.cdf[l])
+            a.register_experts(l, self.stores[l])
+            if self.shared[l] is not None:
+                a.set_shared_expert(l, self.shared[l])
+        return a
+
+    def oracle_experts(self, layer):
+        st = self.stores[layer]
+
+        def get(e):
+            w = st[e].to(torch.float32).numpy()
+            return w[0], w[1], w[2].T
+        return get
+
+    def oracle_shared(self, layer):
+        sh = self.shared[layer]
+        if sh is None:
+            return None
+        w = sh.detach().cpu().to(torch.float32).numpy()
+        return w[0], w[1], w[2].T
+
+
+def _excusable(tok, what: str) -> bool:
+    if what == "rank":
+        return tok["rank_margin"] < ao.NEAR_TIE_LOGIT
+    if what == "budget":
+        return tok["threshold_margin"] < ao.NEAR_TIE_THRESHOLD or tok["rank_margin"] < ao.NEAR_TIE_LOGIT
+    if what == "route":
+        return tok["route_margin"] < ao.NEAR_TIE_LOGIT
+    if what == "exec":
+        return tok["subst_margin"] < ao.NEAR_TIE_LOGIT or tok["route_margin"] < ao.NEAR_TIE_LOGIT
+    return False
+
+
+def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T: int, B: int = 1,
+                 C: Optional[int] = None, norm_topk: bool = True, cache_reuse: bool = True,
+                 check_ffn_every: int = 1, use_prefetch: bool = True, t0: int = 0) -> Report:
+    cfg = prob.cfg
+    C = C or cfg.C
+    N, k, d = cfg.N, cfg.k, cfg.d
+    dev = "cuda"
+    rep = Report()
+    hs = [synth.hidden_states(cfg, l, t0 + T, B) for l in range(prob.L)]
+    cand = torch.full((B, C), -7, dtype=torch.int32, device=dev)
+    ncand = torch.zeros(B, dtype=torch.int32, device=dev)
+    idx = torch.zeros((B, k), dtype=torch.int32, device=dev)
+    alpha = torch.zeros((B, N), dtype=torch.float32, device=dev)
+    exec_idx = torch.zeros((B, k), dtype=torch.int32, device=dev)
+    exec_gate = torch.zeros((B, k), dtype=torch.float32, device=dev)
+    y = torch.full((B, d), 123.0, dtype=torch.float32, device=dev)     # garbage: the library must overwrite
+    for t in range(t0, t0 + T):
+        for l in range(prob.L):
+            W_r, b_r, W_p, b_p = prob.routers[l]
+            w, theta = prob.cdf[l]
+            h = torch.from_numpy(hs[l][0][t]).to(dev)
+            hp = torch.from_numpy(hs[l][1][t]).to(dev)
+            pre = apex.get_slot_table(l)
+            # ---- library
+            if use_prefetch:
+                apex.predict(l, h, B)
+                apex.select_candidates(l, B, tau, cand, ncand)
+                apex.prefetch(l, B)
+                apex.attention_standin(l)
+            apex.route_topk(l, hp, B, idx, alpha)
+            apex.moe_ffn(l, mode, hp, B, y, exec_idx, exec_gate)
+            torch.cuda.synchronize()
+            post = apex.get_slot_table(l)
+            g_cp, g_dm = apex.get_last_copies(l)
+            # ---- oracle from the same pre-step table
+            cache = ao.SlotCache(N, C, cache_reuse=cache_reuse)
+            cache.set_state(pre[0], pre[1], pre[2])
+            do_ffn = (rep.layer_steps % check_ffn_every) == 0
+            if use_prefetch:
+                out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=tau, k=k,
+                                    h=hs[l][0][t], h_post=hs[l][1][t], mode=mode,
+                                    expert_weights=prob.oracle_experts(l), shared=prob.oracle_shared(l),
+                                    norm_topk=norm_topk, compute_ffn=do_ffn)
+            else:   # no prefetch stage: budget 0 candidates are never issued; emulate by an empty prefetch
+                out = _oracle_step_without_prefetch(cache, W_r, b_r, k, hs[l][1][t], mode, prob, l, norm_topk, do_ffn)
+            rep.layer_steps += 1
+            excused = False
+            if use_prefetch:
+                z_p, q_p, pi = apex.read_prediction(B)
+                g_cand, g_ncand = cand.cpu().numpy(), ncand.cpu().numpy()
+                for b in range(B):
+                    tok = out["tokens"][b]
+                    np.testing.assert_allclose(z_p[b], tok["z_p"], atol=2e-5, rtol=0)
+                    np.testing.assert_allclose(q_p[b], tok["q_p"], atol=1e-6, rtol=1e-5)
+                    if list(pi[b]) != list(tok["pi"]):
+                        assert _excusable(tok, "rank"), f"ranking differs t={t} l={l} b={b}"
+                        excused = True
+                    gP = [int(e) for e in g_cand[b][:g_ncand[b]]]
+                    if gP != tok["P"] or g_ncand[b] != k + tok["delta_hat"]:
+                        assert _excusable(tok, "budget"), \
+                            f"candidate set differs t={t} l={l} b={b}: {gP} vs {tok['P']} margin {tok['threshold_margin']}"
+                        excused = True
+                    assert all(int(v) == -1 for v in g_cand[b][g_ncand[b]:])
+                if not excused:
+                    assert g_cp == out["prefetch_copies"], f"prefetch plan differs t={t} l={l}"
+            g_idx, g_alpha = idx.cpu().numpy(), alpha.cpu().numpy()
+            g_ex, g_gate = exec_idx.cpu().numpy(), exec_gate.cpu().numpy()
+            g_y = y.cpu().numpy()
+            for b in range(B):
+                tok = out["tokens"][b]
+                np.testing.assert_allclose(g_alpha[b], tok["alpha"], atol=1e-6, rtol=1e-5)
+                if list(g_idx[b]) != tok["K_r"]:
+                    assert _excusable(tok, "route"), f"K_r differs t={t} l={l} b={b}: {g_idx[b]} vs {tok['K_r']}"
+                    excused = True
+            if not excused:
+                for b in range(B):
+                    tok = out["tokens"][b]
+                    if list(g_ex[b]) != tok["K_exec"]:
+                        assert _excusable(tok, "exec"), f"K_exec differs t={t} l={l} b={b}: {g_ex[b]} vs {tok['K_exec']}"
+                        excused = True
+            if excused:
+                rep.near_ties += 1
+                continue
+            assert g_dm == out["demand_copies"], f"demand plan differs t={t} l={l}: {g_dm} vs {out['demand_copies']}"
+            es, stamp, clk = cache.get_state()
+            assert list(post[0]) == es and list(post[1]) == stamp and post[2] == clk, f"post-step table differs t={t} l={l}"
+            rep.n_prefetch_copies += len(g_cp)
+            rep.n_demand_copies += len(g_dm)
+            rep.n_miss_steps += int(len(out["missing"]) > 0)
+            for b in range(B):
+                tok = out["tokens"][b]
+                rep.n_subst += tok["n_subst"]
+                np.testing.assert_allclose(g_gate[b], tok["gates"], rtol=2e-5, atol=1e-7)
+                if norm_topk:
+                    assert abs(float(g_gate[b].sum()) - 1.0) < 1e-5
+                if do_ffn:
+                    ref = tok["y"]
+                    err = g_y[b].astype(np.float64) - ref
+                    rel = float(np.linalg.norm(err) / max(np.linalg.norm(ref), 1e-30))
+                    mx = float(np.abs(err).max())
+                    rep.worst_rel_l2 = max(rep.worst_rel_l2, rel)
+                    rep.worst_max_abs = max(rep.worst_max_abs, mx)
+                    rep.ffn_checked += 1
+                    assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL, f"FFN output t={t} l={l} b={b}: rel-L2 {rel:.3e} max-abs {mx:.3e}"
+    return rep
+
+
+def _oracle_step_without_prefetch(cache, W_r, b_r, k, h_post, mode, prob, layer, norm_topk, do_ffn):
+    """Gate + execution only (the no-prefetch baseline): nothing is predicted, every non-resident
+    routed expert is a demand fetch."""
+    B = h_post.shape[0]
+    cache.begin_step()
+    out = {"B": B, "tokens": [], "prefetch_copies": []}
+    R = cache.resident()
+    Ks = []
+    for b in range(B):
+        z_r, K_r, alpha = ao.route_topk(W_r, b_r, h_post[b], k)
+        out["tokens"].append({"z_r": z_r, "K_r": K_r, "alpha": alpha, "route_margin": ao.min_adjacent_gap(z_r, upto=k),
+                              "n_subst": 0, "subst_margin": float("inf")})
+        Ks.append(K_r)
+    if mode == "exact":
+        missing, waves = cache.demand(Ks)
+        out["missing"] = missing
+        out["demand_copies"] = [c for wv in waves for c in wv]
+        for tok in out["tokens"]:
+            tok["K_exec"] = sorted(tok["K_r"])
+    else:
+        out["missing"], out["demand_copies"] = [], []
+        used = set()
+        for tok in out["tokens"]:
+            tok["K_exec"] = ao.stall_free_set(tok["K_r"], tok["alpha"], R)
+            tok["n_subst"] = len(set(tok["K_exec"]) - set(tok["K_r"]))
+            cand = [e for e in R if e not in tok["K_r"]]
+            tok["subst_margin"] = ao.min_adjacent_gap(tok["z_r"][cand]) if (tok["n_subst"] and len(cand) > 1) else float("inf")
+            used |= set(tok["K_exec"])
+        for e in sorted(used):
+            cache.touch(e)
+    for b, tok in enumerate(out["tokens"]):
+        tok["gates"] = ao.gates(tok["alpha"], tok["K_exec"], norm_topk)
+        if do_ffn:
+            tok["y"] = ao.moe_output(h_post[b], tok["K_exec"], tok["gates"], prob.oracle_experts(layer), prob.oracle_shared(layer))
+    return out

@@ -1,0 +1,272 @@
+"""GPU parity: the CUDA library against the CPU oracle, element by element, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+from paper_2608_11688_b200 import binding, synth
+
+pytestmark = pytest.mark.gpu
+
+
+def _harness():
+    import harness
+    return harness
+
+
+def _run(cfg, *, mode, tau, T, B=1, layers=None, C=None, norm_topk=1, cache_reuse=1, check_ffn_every=1,
+         use_prefetch=True, prob=None):
+    hz = _harness()
+    prob = prob or hz.Problem(cfg, layers=layers)
+    apex = prob.make_ctx(C=C, max_batch=B, norm_topk=norm_topk, cache_reuse=cache_reuse)
+    try:
+        rep = hz.run_lockstep(prob, apex, mode=mode, tau=tau, T=T, B=B, C=C, norm_topk=bool(norm_topk),
+                              cache_reuse=bool(cache_reuse), check_ffn_every=check_ffn_every,
+                              use_prefetch=use_prefetch)
+        stats = apex.get_stats()
+    finally:
+        apex.destroy()
+    return rep, stats
+
+
+# ------------------------------------------------------------------ tiny and ragged shapes
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+@pytest.mark.parametrize("d,N,k,I,C", [(256, 8, 2, 24, 4), (512, 12, 3, 40, 6), (768, 33, 5, 17, 9),
+                                       (1024, 64, 8, 16, 16), (3072, 5, 1, 9, 2)])
+def test_tiny_shapes_both_modes(d, N, k, I, C, mode):
+    cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, T=12, sigma_p=1.0, cfg_id=200 + N)
+    rep, stats = _run(cfg, mode=mode, tau=0.7, T=12)
+    assert rep.layer_steps == 12 and rep.ffn_checked + rep.near_ties >= 12
+    assert stats["tokens"] == 12 and stats["routed"] == 12 * k
+    if mode == "stall_free":
+        assert rep.n_demand_copies == 0
+
+
+@pytest.mark.parametrize("tau", [0.0, 0.3, 0.97, 1.0])
+def test_tau_extremes_and_cap(tau):
+    cfg = synth.tiny_config(d=256, N=16, k=4, I=32, C=8, T=10, sigma_p=0.8, cfg_id=210)
+    rep, stats = _run(cfg, mode="exact", tau=tau, T=10)
+    if tau == 0.0:
+        assert stats["sum_delta_hat"] == 0
+    if tau == 1.0:
+        assert stats["sum_ncand"] == 10 * 8 and stats["capped"] == 10     # N-k = 12 capped to C-k = 4
+
+
+def test_all_resident_cache_never_copies_twice():
+    cfg = synth.tiny_config(d=256, N=8, k=2, I=32, C=8, T=30, cfg_id=211)
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=30)
+    assert stats["prefetch_copies"] + stats["demand_copies"] <= 8
+
+
+def test_minimal_cache_C_equals_k():
+    cfg = synth.tiny_config(d=256, N=10, k=3, I=16, C=3, T=20, sigma_p=1.5, cfg_id=212)
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=20)
+    assert rep.n_miss_steps > 0            # a noisy predictor with no spare slot misses
+    assert stats["extra_waves"] == rep.n_miss_steps
+    rep, stats = _run(cfg, mode="stall_free", tau=0.9, T=20)
+    assert rep.n_subst > 0 and stats["substitutions"] == rep.n_subst
+
+
+def test_load_use_evict_policy_and_unnormalised_gates():
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=7, T=12, sigma_p=1.0, cfg_id=213)
+    rep, stats = _run(cfg, mode="stall_free", tau=0.8, T=12, cache_reuse=0)
+    assert stats["prefetch_copies"] == stats["sum_ncand"]       # every candidate of every step is copied
+    _run(cfg, mode="exact", tau=0.8, T=8, norm_topk=0)
+
+
+def test_no_prefetch_baseline_demand_fetches_everything():
+    cfg = synth.tiny_config(d=256, N=10, k=3, I=16, C=5, T=10, cfg_id=214)
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=10, use_prefetch=False)
+    assert stats["prefetch_copies"] == 0 and stats["demand_copies"] == rep.n_demand_copies > 0
+
+
+def test_shared_expert_and_multi_layer():
+    cfg = synth.tiny_config(d=512, N=12, k=2, I=24, C=6, L=3, T=6, I_shared=40, cfg_id=215)
+    rep, stats = _run(cfg, mode="exact", tau=0.8, T=6)
+    assert rep.layer_steps == 18
+
+
+@pytest.mark.parametrize("B", [2, 5, 16])
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_batched_tokens(B, mode):
+    cfg = synth.tiny_config(d=512, N=20, k=3, I=24, C=8, T=5, I_shared=16, sigma_p=1.0, cfg_id=216)
+    rep, stats = _run(cfg, mode=mode, tau=0.8, T=5, B=B)
+    assert stats["tokens"] == 5 * B
+
+
+def test_batched_exact_mode_runs_in_waves_when_cache_is_smaller_than_need():
+    cfg = synth.tiny_config(d=256, N=16, k=4, I=16, C=5, T=4, cfg_id=217)
+    rep, stats = _run(cfg, mode="exact", tau=0.5, T=4, B=8)
+    assert stats["extra_waves"] >= 4 * 2          # at least two extra waves per step: need > 2 C
+
+
+# ------------------------------------------------------------------ the paper-shaped configs
+def test_config0_full():
+    cfg = synth.CONFIGS[0]
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=cfg.T)
+    assert rep.layer_steps == 128
+    assert rep.worst_rel_l2 <= 2e-3 and rep.worst_max_abs <= 2e-2
+    print("config0", rep, stats)
+
+
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_config1_shape_two_layers(mode):
+    cfg = synth.CONFIGS[1]
+    rep, stats = _run(cfg, mode=mode, tau=0.9, T=24, layers=2, check_ffn_every=3)
+    assert rep.layer_steps == 48
+    print("config1", mode, rep, stats)
+
+
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_config2_shape_one_layer(mode):
+    cfg = synth.CONFIGS[2]
+    rep, stats = _run(cfg, mode=mode, tau=0.9, T=12, layers=1, check_ffn_every=3)
+    print("config2", mode, rep, stats)
+
+
+def test_config3_shape_one_layer():
+    cfg = synth.CONFIGS[3]
+    hz = _harness()
+    prob = hz.Problem(cfg, layers=1)
+    for mode in ("exact", "stall_free"):
+        rep, stats = _run(cfg, mode=mode, tau=0.9, T=3, layers=1, prob=prob)
+        print("config3", mode, rep, stats)
+
+
+@pytest.mark.parametrize("B", [1, 8])
+def test_config4_shape_one_layer(B):
+    cfg = synth.CONFIGS[4]
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=2, layers=1, B=B)
+    print("config4", B, rep, stats)
+
+
+# ------------------------------------------------------------------ API behaviour
+def test_decode_token_matches_per_call_sequence_and_counts_launches():
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=6, L=2, T=4, cfg_id=218)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    a1, a2 = prob.make_ctx(), prob.make_ctx()
+    try:
+        hs = [synth.hidden_states(cfg, l, cfg.T) for l in range(cfg.L)]
+        h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()       # [T][L][1][d]
+        hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
+        y1 = torch.empty((cfg.L, 1, cfg.d), device="cuda"); y2 = torch.empty_like(y1)
+        cand = torch.empty((1, cfg.C), dtype=torch.int32, device="cuda"); nc = torch.empty(1, dtype=torch.int32, device="cuda")
+        idx = torch.empty((1, cfg.k), dtype=torch.int32, device="cuda"); al = torch.empty((1, cfg.N), device="cuda")
+        for t in range(cfg.T):
+            n0 = a1.launch_count()
+            a1.decode_token(h[t], hp[t], 1, 0.9, "exact", y1)
+            assert a1.launch_count() - n0 >= 5 * cfg.L
+            for l in range(cfg.L):
+                a2.predict(l, h[t, l], 1); a2.select_candidates(l, 1, 0.9, cand, nc); a2.prefetch(l, 1)
+                a2.attention_standin(l); a2.route_topk(l, hp[t, l], 1, idx, al)
+                a2.moe_ffn(l, "exact", hp[t, l], 1, y2[l])
+            torch.cuda.synchronize()
+            torch.testing.assert_close(y1, y2, rtol=1e-4, atol=1e-5)
+        # host-buffer variant
+        hh = h[0].cpu().pin_memory(); hph = hp[0].cpu().pin_memory(); yh = torch.empty_like(hh).pin_memory()
+        a3 = prob.make_ctx()
+        a3.decode_token_host(hh, hph, 1, 0.9, "exact", yh)
+        a4 = prob.make_ctx()
+        a4.decode_token(h[0], hp[0], 1, 0.9, "exact", y1); torch.cuda.synchronize()
+        torch.testing.assert_close(yh.cuda(), y1, rtol=1e-4, atol=1e-5)
+        a3.destroy(); a4.destroy()
+    finally:
+        a1.destroy(); a2.destroy()
+
+
+def test_calls_out_of_order_and_bad_arguments():
+    cfg = synth.tiny_config(d=256, N=8, k=2, I=16, C=4, cfg_id=219)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    a = prob.make_ctx()
+    try:
+        y = torch.empty((1, cfg.d), device="cuda")
+        with pytest.raises(binding.ApexError) as ei:
+            a.moe_ffn(0, "exact", y, 1, y)
+        assert ei.value.code == binding.APEX_ESTATE
+        cand = torch.empty((1, cfg.C), dtype=torch.int32, device="cuda"); nc = torch.empty(1, dtype=torch.int32, device="cuda")
+        with pytest.raises(binding.ApexError) as ei:
+            a.select_candidates(0, 1, 0.9, cand, nc)
+        assert ei.value.code == binding.APEX_ESTATE
+        with pytest.raises(binding.ApexError) as ei:
+            a.predict(3, y, 1)
+        assert ei.value.code == binding.APEX_EINVAL
+        with pytest.raises(binding.ApexError) as ei:
+            a.set_cdf(0, np.zeros(cfg.N, np.float32), np.arange(cfg.N - cfg.k + 1, 0, -1).astype(np.float32))
+        assert ei.value.code == binding.APEX_EINVAL
+    finally:
+        a.destroy()
+
+
+def test_host_side_fault_hooks_copy_failure_and_withheld_flag():
+    cfg = synth.tiny_config(d=256, N=8, k=2, I=16, C=4, T=4, cfg_id=220)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    a = prob.make_ctx(wait_limit_ns=50_000_000)          # 50 ms bound on every wait
+    try:
+        h, hp = synth.hidden_states(cfg, 0, 4)
+        hd, hpd = torch.from_numpy(h).cuda(), torch.from_numpy(hp).cuda()
+        y = torch.empty((1, cfg.d), device="cuda")
+        cand = torch.empty((1, cfg.C), dtype=torch.int32, device="cuda"); nc = torch.empty(1, dtype=torch.int32, device="cuda")
+        idx = torch.empty((1, cfg.k), dtype=torch.int32, device="cuda"); al = torch.empty((1, cfg.N), device="cuda")
+        # 1: the copy issue fails on the host
+        a.predict(0, hd[0], 1); a.select_candidates(0, 1, 0.9, cand, nc)
+        a.test_inject(1)
+        with pytest.raises(binding.ApexError) as ei:
+            a.prefetch(0, 1)
+        assert ei.value.code == binding.APEX_ECUDA
+        # 2: a slot-ready flag is withheld: the device-side wait runs out and the call reports it;
+        # the context stays usable afterwards
+        a2 = prob.make_ctx(wait_limit_ns=50_000_000)
+        a2.predict(0, hd[1], 1); a2.select_candidates(0, 1, 1.0, cand, nc)
+        a2.test_inject(2)
+        a2.prefetch(0, 1); a2.attention_standin(0); a2.route_topk(0, hpd[1], 1, idx, al)
+        try:
+            a2.moe_ffn(0, "stall_free", hpd[1], 1, y)
+            torch.cuda.synchronize()
+            # the status may arrive after the call returned: the next call reports it
+            a2.predict(0, hd[2], 1); a2.select_candidates(0, 1, 1.0, cand, nc); a2.prefetch(0, 1)
+            a2.route_topk(0, hpd[2], 1, idx, al); a2.moe_ffn(0, "stall_free", hpd[2], 1, y)
+            torch.cuda.synchronize()
+            raised = False
+        except binding.ApexError as e:
+            assert e.code == binding.APEX_ETIMEOUT
+            raised = True
+        assert raised or a2.get_stats()["timeouts"] > 0
+        torch.cuda.synchronize()
+        a2.predict(0, hd[3], 1); a2.select_candidates(0, 1, 0.9, cand, nc); a2.prefetch(0, 1)
+        a2.route_topk(0, hpd[3], 1, idx, al)
+        try:
+            a2.moe_ffn(0, "exact", hpd[3], 1, y)
+        except binding.ApexError as e:
+            assert e.code == binding.APEX_ETIMEOUT          # a late report of the same timeout
+        torch.cuda.synchronize()
+        assert torch.isfinite(y).all()
+        a2.destroy()
+    finally:
+        a.destroy()
+
+
+def test_run_to_run_determinism_of_indices():
+    cfg = synth.tiny_config(d=1024, N=32, k=8, I=32, C=16, T=6, cfg_id=221)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    outs = []
+    for rep in range(2):
+        a = prob.make_ctx()
+        h, hp = synth.hidden_states(cfg, 0, 6)
+        cand = torch.empty((1, cfg.C), dtype=torch.int32, device="cuda"); nc = torch.empty(1, dtype=torch.int32, device="cuda")
+        idx = torch.empty((1, cfg.k), dtype=torch.int32, device="cuda"); al = torch.empty((1, cfg.N), device="cuda")
+        rec = []
+        for t in range(6):
+            a.predict(0, torch.from_numpy(h[t]).cuda(), 1); a.select_candidates(0, 1, 0.9, cand, nc)
+            a.route_topk(0, torch.from_numpy(hp[t]).cuda(), 1, idx, al)
+            torch.cuda.synchronize()
+            rec.append((cand.cpu().numpy().copy(), idx.cpu().numpy().copy(), al.cpu().numpy().copy(), a.read_prediction(1)))
+        outs.append(rec)
+        a.destroy()
+    for r0, r1 in zip(*outs):
+        np.testing.assert_array_equal(r0[0], r1[0]); np.testing.assert_array_equal(r0[1], r1[1])
+        np.testing.assert_array_equal(r0[2], r1[2])                      # bitwise: fixed reduction order
+        for x, y2 in zip(r0[3], r1[3]):
+            np.testing.assert_array_equal(x, y2)

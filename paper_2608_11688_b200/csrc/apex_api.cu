@@ -548,15 +548,19 @@ int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int
     if (!tab.plan_demand(K_r, B, k, &copies, &need)) return fail(ctx, APEX_ESTATE, "no evictable slot");
     int n_waves = 0;
     for (const auto& c : copies) n_waves = c.wave > n_waves ? c.wave : n_waves;
+    // The plan above covers every wave; replay it wave by wave so that each launch gets the table
+    // as it stands when that wave runs.
+    std::vector<int32_t> cur_slot_expert = slot_expert_before;
+    SlotSnapshot cur = p.snap;
     for (int w = 1; w <= n_waves; ++w) {
-      // a victim that an earlier wave of this step may still be reading: order the copy after that wave
+      // a victim that an earlier launch of this step may still be reading: order the copy after it
       bool hazard = false;
       uint64_t chunk = 0;
       for (const auto& c : copies)
         if (c.wave == w) {
           chunk |= (1ull << c.expert);
-          const int prev = w == 1 ? slot_expert_before[c.slot] : -2;
-          if (w > 1 || (prev >= 0 && ((need >> prev) & 1))) hazard = true;
+          const int prev = cur_slot_expert[c.slot];
+          if (prev >= 0 && ((need >> prev) & 1)) hazard = true;
         }
       if (hazard) {
         CU_TRY(ctx, cudaEventRecord(ctx->ev_wave, cs));
@@ -566,9 +570,18 @@ int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int
         if (c.wave == w) {
           int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
           if (r != APEX_OK) return r;
+          const int prev = cur_slot_expert[c.slot];
+          if (prev >= 0) {
+            cur.expert_slot[prev] = -1;
+            cur.resident_mask &= ~(1ull << prev);
+          }
+          cur_slot_expert[c.slot] = c.expert;
+          cur.expert_slot[c.expert] = (int8_t)c.slot;
+          cur.need_gen[c.expert] = ctx->slot_gen[layer][c.slot];
+          cur.resident_mask |= (1ull << c.expert);
         }
       FfnParams q = p;
-      q.snap = make_snapshot(ctx, layer);
+      q.snap = cur;
       q.run_mask = chunk;
       q.accumulate = 1;
       q.run_shared = 0;

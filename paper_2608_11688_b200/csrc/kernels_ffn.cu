@@ -23,6 +23,12 @@ constexpr int kMaxStages = 32;
 constexpr int kSmemBudget = 224 * 1024;  // ring bytes; static tables fit in what is left of the 227 KB per-CTA limit
 constexpr int kSmallPairs = APEX_MAX_TOPK + 1;
 
+__host__ __device__ constexpr int ring_stages(uint32_t entry_bytes) {
+  int n = kSmemBudget / (int)entry_bytes;
+  if (n > kMaxStages) n = kMaxStages;
+  return n / kConsumerWarps * kConsumerWarps;
+}
+
 // ---------------------------------------------------------------- PTX helpers
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ void mbar_init(uint64_t* bar, uint32_t count) {
@@ -288,8 +294,11 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   constexpr int d = NCH * 256;
   constexpr uint32_t row_bytes = d * 2;
   constexpr uint32_t entry_bytes = 3 * row_bytes;
-  constexpr int NS = (kSmemBudget / (int)entry_bytes) < kMaxStages ? (kSmemBudget / (int)entry_bytes) : kMaxStages;
-  static_assert(NS >= 6, "ring must also hold the cross-warp reduction buffer");
+  // The ring depth is a multiple of the consumer-warp count, so a stage is always consumed by the
+  // same warp: a warp can then never wait on a stage's next phase before it has consumed the current
+  // one (a parity wait cannot tell "one phase ahead" from "done").
+  constexpr int NS = ring_stages(entry_bytes);
+  static_assert(NS >= kConsumerWarps && NS % kConsumerWarps == 0, "ring depth must be a multiple of the consumer warps");
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = p.N, k = p.k, I = p.I, B = p.B;
@@ -404,6 +413,10 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
           cur_e = e;
           if (e < N) {
             const int slot = p.snap.expert_slot[e];
+            if (slot < 0) {  // the host never asks for an expert without a slot; refuse rather than read out of range
+              ok = false;
+              break;
+            }
             const uint32_t need = p.snap.need_gen[e];
             const uint32_t* flag = p.slot_ready + slot;
             if ((int32_t)(ld_acquire_sys(flag) - need) < 0) {
@@ -612,7 +625,7 @@ template <int NCH>
 static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
   constexpr bool HR = NCH <= 8;
   constexpr uint32_t entry = 3 * NCH * 256 * 2;
-  constexpr int NS = (kSmemBudget / (int)entry) < kMaxStages ? (kSmemBudget / (int)entry) : kMaxStages;
+  constexpr int NS = ring_stages(entry);
   const size_t smem = (size_t)NS * entry;
   static bool configured = false;
   if (!configured) {

@@ -1,0 +1,412 @@
+#!/usr/bin/env python
+"""Benchmark of the MoE decode step with adaptive expert prefetch on B200.
+
+A "step" is one decode token through all layers of the workload: for every layer the prefetch
+router, the budget selection, the asynchronous expert prefetch, the stand-in attention window,
+the exact gate and the expert FFN (with on-demand correction of misses in exact mode).
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--config 1] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  N > 1 runs N independent replicas (the path does not shard).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "moe_decode_tokens_per_s"
+UNIT = "tokens/s"
+NOMINAL_HBM_GBS = 8000.0
+FALLBACK_HBM_GBS = 6650.0
+TAU = 0.90
+
+# DRAM bytes per launch of the expert-FFN kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
+# the ncu capture summarised in profiles/ (same kernel, same per-launch shape).  None = not captured.
+NCU_TRAFFIC_BYTES = {1: None}
+
+
+def measured_peak():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        try:
+            return float(json.load(open(p))["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """nvidia-smi clocks and throttle reasons during the timed region."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.idx = gpu_index
+        self.proc = None
+        self.path = f"/tmp/apex_clocks_{os.getpid()}.csv"
+
+    def start(self):
+        try:
+            self.f = open(self.path, "w")
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-i", str(self.idx), "-lms", "100"], stdout=self.f, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self):
+        out = {"sm_mhz": None, "sm_max_mhz": None, "reasons": [], "samples": 0}
+        if self.proc is None:
+            return out
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.f.close()
+        sm, mx, reasons = [], [], set()
+        for ln in open(self.path):
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1])); mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, v in zip(("hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"), f[5:9]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        try:
+            os.remove(self.path)
+        except OSError:
+            pass
+        if sm:
+            out.update(sm_mhz=statistics.median(sm), sm_max_mhz=max(mx), reasons=sorted(reasons), samples=len(sm))
+        return out
+
+
+def algorithmic_bytes(cfg, B=1):
+    """Per layer-step: routed expert weights + shared FFN + both routers (fp32), and the FFN kernel alone."""
+    ffn = cfg.k * cfg.expert_bytes + cfg.shared_bytes + 2 * B * cfg.d * 4
+    routers = 2 * cfg.d * cfg.N * 4
+    return ffn + routers, ffn
+
+
+# ------------------------------------------------------------------------------------------------
+def build_problem(cfg, device):
+    import torch
+    from paper_2608_11688_b200 import synth
+    routers = [synth.router_weights(cfg, l) for l in range(cfg.L)]
+    cdf = [synth.cdf_params(cfg, l) for l in range(cfg.L)]
+    store = torch.empty((cfg.L, cfg.N, 3, cfg.I, cfg.d), dtype=torch.bfloat16, pin_memory=True)
+    shared = []
+    for l in range(cfg.L):
+        store[l].copy_(synth.expert_store(cfg, l, device=device))
+        shared.append(synth.shared_expert(cfg, l, device=device))
+    torch.cuda.synchronize()
+    return routers, cdf, store, shared
+
+
+def make_ctx(cfg, prob, C, max_batch=1):
+    from paper_2608_11688_b200 import binding
+    routers, cdf, store, shared = prob
+    a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C, L=cfg.L, I_shared=cfg.I_shared, max_batch=max_batch)
+    for l in range(cfg.L):
+        W_r, b_r, W_p, b_p = routers[l]
+        a.set_router(l, W_r, b_r)
+        a.set_prefetch_router(l, W_p, b_p)
+        a.set_cdf(l, *cdf[l])
+        a.register_experts(l, store[l])
+        if shared[l] is not None:
+            a.set_shared_expert(l, shared[l])
+    return a
+
+
+def hidden_inputs(cfg, T, B, device):
+    """[T][L][B][d] tensors on the device (h, h')."""
+    import torch
+    from paper_2608_11688_b200 import synth
+    hs = [synth.hidden_states(cfg, l, T, B) for l in range(cfg.L)]
+    h = torch.from_numpy(np.stack([x[0] for x in hs], 1))
+    hp = torch.from_numpy(np.stack([x[1] for x in hs], 1))
+    return h, hp
+
+
+def time_tokens(apex, h, hp, y, B, mode, warmup, steps, dist_sync=None, host=False):
+    """W untimed + K timed decode tokens; returns seconds (CUDA events on the launching stream)."""
+    import torch
+    T = h.shape[0]
+    run = (lambda t: apex.decode_token_host(h[t % T], hp[t % T], B, TAU, mode, y)) if host else \
+          (lambda t: apex.decode_token(h[t % T], hp[t % T], B, TAU, mode, y))
+    for t in range(warmup):
+        run(t)
+    torch.cuda.synchronize()
+    if dist_sync:
+        dist_sync()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(warmup, warmup + steps):
+        run(t)
+    e1.record()
+    torch.cuda.synchronize()
+    if dist_sync:
+        dist_sync()
+    return e0.elapsed_time(e1) * 1e-3
+
+
+def time_ffn_kernel(apex, cfg, h, hp, B, tokens):
+    """Average device time of one expert-FFN launch, all experts resident: CUDA events around each
+    launch on the launching stream, summed over layers and tokens."""
+    import torch
+    dev = h.device
+    idx = torch.empty((B, cfg.k), dtype=torch.int32, device=dev)
+    al = torch.empty((B, cfg.N), dtype=torch.float32, device=dev)
+    y = torch.empty((B, cfg.d), dtype=torch.float32, device=dev)
+    T = h.shape[0]
+    pairs = []
+    for t in range(tokens + 1):
+        for l in range(cfg.L):
+            apex.route_topk(l, hp[t % T, l], B, idx, al)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            apex.moe_ffn(l, "exact", hp[t % T, l], B, y)
+            e1.record()
+            if t > 0:                       # first pass is warm-up
+                pairs.append((e0, e1))
+    torch.cuda.synchronize()
+    ms = [a.elapsed_time(b) for a, b in pairs]
+    return statistics.mean(ms) * 1e-3, statistics.median(ms) * 1e-3, len(ms)
+
+
+def oracle_tokens_per_s(cfg, prob, n_tokens):
+    """The CPU oracle as it stands, timed on the host cores over n_tokens full decode tokens."""
+    import torch
+    from oracle import apex_oracle as ao
+    from paper_2608_11688_b200 import synth
+    routers, cdf, store, shared = prob
+    caches = [ao.SlotCache(cfg.N, cfg.C) for _ in range(cfg.L)]
+    hs = [synth.hidden_states(cfg, l, n_tokens, 1) for l in range(cfg.L)]
+    t0 = time.perf_counter()
+    for t in range(n_tokens):
+        for l in range(cfg.L):
+            W_r, b_r, W_p, b_p = routers[l]
+            w, theta = cdf[l]
+
+            def experts(e, l=l):
+                a = store[l, e].to(torch.float32).numpy()
+                return a[0], a[1], a[2].T
+            sh = None
+            if shared[l] is not None:
+                s = shared[l].cpu().to(torch.float32).numpy()
+                sh = (s[0], s[1], s[2].T)
+            ao.layer_step(caches[l], W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=TAU, k=cfg.k,
+                          h=hs[l][0][t], h_post=hs[l][1][t], mode="exact", expert_weights=experts, shared=sh)
+    dt = time.perf_counter() - t0
+    try:
+        from threadpoolctl import threadpool_info
+        cores = max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+    except Exception:
+        cores = 1
+    return n_tokens / dt, cores, dt
+
+
+# ------------------------------------------------------------------------------------------------
+def run_reference(args, cfg, rank):
+    """--impl reference: the oracle on the host cores, same metric and workload, bounded sample."""
+    if rank != 0:
+        return
+    import torch
+    dev = "cuda" if torch.cuda.is_available() else "cpu"
+    from paper_2608_11688_b200 import synth
+    routers = [synth.router_weights(cfg, l) for l in range(cfg.L)]
+    cdf = [synth.cdf_params(cfg, l) for l in range(cfg.L)]
+    store = torch.empty((cfg.L, cfg.N, 3, cfg.I, cfg.d), dtype=torch.bfloat16)
+    shared = []
+    for l in range(cfg.L):
+        store[l].copy_(synth.expert_store(cfg, l, device=dev))
+        sh = synth.shared_expert(cfg, l, device=dev)
+        shared.append(None if sh is None else sh.cpu())
+    prob = (routers, cdf, store, shared)
+    n = max(1, args.steps)
+    for _ in range(min(args.warmup, 1)):
+        oracle_tokens_per_s(cfg, prob, 1)
+    tps, cores, dt = oracle_tokens_per_s(cfg, prob, n)
+    line = {"impl": "reference", "metric": METRIC, "value": tps, "unit": UNIT, "n_gpus": args.gpus, "steps": n,
+            "warmup": min(args.warmup, 1), "ms_per_step": 1e3 * dt / n, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}", "L": cfg.L, "d": cfg.d, "N": cfg.N, "k": cfg.k,
+                       "I": cfg.I, "C": cfg.C, "B": 1, "tau": TAU, "mode": "exact"},
+            "cpu_baseline": {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                             "sample": f"{n} decode tokens x {cfg.L} layers, every step of the path in fp64 numpy"},
+            "e2e": {"value": tps, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0}}
+    print(json.dumps(line), flush=True)
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=None)
+    ap.add_argument("--warmup", type=int, default=None)
+    ap.add_argument("--config", type=int, default=1)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--cpu-baseline-tokens", type=int, default=2)
+    ap.add_argument("--skip-extras", action="store_true", help="only the headline leg (used for ncu launch lists)")
+    ap.add_argument("--ffn-only", action="store_true",
+                    help="profiling case: all experts resident, gate + expert FFN only, no copy in flight")
+    ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (smaller captures)")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+
+    from paper_2608_11688_b200 import synth
+    cfg = synth.CONFIGS[args.config]
+    if args.layers:
+        cfg = cfg.scaled(L=args.layers)
+    if args.impl == "reference":
+        args.steps = 2 if args.steps is None else min(args.steps, 4)
+        args.warmup = 0 if args.warmup is None else args.warmup
+        run_reference(args, cfg, rank)
+        return
+    args.steps = 48 if args.steps is None else args.steps
+    args.warmup = 4 if args.warmup is None else max(3, args.warmup)
+
+    import torch
+    from paper_2608_11688_b200 import build
+    assert torch.cuda.is_available(), "bench.py needs a CUDA device (there is no CPU fallback)"
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if rank == 0:
+        build.build()
+    dist_sync = None
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+        dist.barrier()
+        dist_sync = dist.barrier
+    B = 1
+    prob = build_problem(cfg, dev)
+    T = min(cfg.T, args.warmup + args.steps)
+    h, hp = hidden_inputs(cfg, T, B, dev)
+    h_dev, hp_dev = h.to(dev), hp.to(dev)
+    h_pin, hp_pin = h.pin_memory(), hp.pin_memory()
+    y_dev = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32, device=dev)
+    y_pin = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32).pin_memory()
+
+    if args.ffn_only:
+        a = make_ctx(cfg, prob, cfg.N)
+        a.warm_all()
+        mean_s, med_s, n_l = time_ffn_kernel(a, cfg, h_dev, hp_dev, B, tokens=args.steps)
+        _, bytes_ffn = algorithmic_bytes(cfg, B)
+        print(json.dumps({"ffn_only": True, "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6,
+                          "launches": n_l, "GBps_mean": bytes_ffn / mean_s / 1e9, "bytes_per_launch": bytes_ffn}), flush=True)
+        a.destroy()
+        return
+
+    # ---- headline: config cache size, exact (correctness-preserving) mode, inputs resident in HBM
+    apex = make_ctx(cfg, prob, cfg.C)
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    n0 = apex.launch_count()
+    sec = time_tokens(apex, h_dev, hp_dev, y_dev, B, "exact", args.warmup, args.steps, dist_sync)
+    launches = (apex.launch_count() - n0) * args.steps // (args.warmup + args.steps)
+    clocks = sampler.stop()
+    st_all = apex.get_stats()
+    if world > 1:
+        import torch.distributed as dist
+        tmax = torch.tensor([sec], device=dev)
+        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+        sec = float(tmax.item())
+    value = world * args.steps / sec
+    extras = {}
+    e2e = None
+    roof = None
+    cpu = None
+    bytes_step, bytes_ffn = algorithmic_bytes(cfg, B)
+    peak, peak_kind = measured_peak()
+    if not args.skip_extras:
+        # ---- end to end: host buffers in, host buffer out, through the C-ABI call
+        apex.reset_stats()
+        sec_e2e = time_tokens(apex, h_pin, hp_pin, y_pin, B, "exact", args.warmup, args.steps, dist_sync, host=True)
+        if world > 1:
+            tmax = torch.tensor([sec_e2e], device=dev)
+            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
+            sec_e2e = float(tmax.item())
+        st = apex.get_stats()
+        per_tok = args.warmup + args.steps
+        e2e = {"value": world * args.steps / sec_e2e, "unit": UNIT,
+               "h2d_bytes_per_step": int(2 * cfg.L * B * cfg.d * 4), "d2h_bytes_per_step": int(cfg.L * B * cfg.d * 4),
+               "expert_bytes_copied_per_step": int(st["bytes_copied"] / per_tok)}
+        extras["exact"] = {
+            "tokens_per_s": args.steps / sec, "overlap_vs_P": st["hits_P"] / max(1, st["routed"]),
+            "overlap_vs_R": st["hits_R"] / max(1, st["routed"]), "coverage": st["covered"] / max(1, st["tokens"]),
+            "mean_delta_hat": st["sum_delta_hat"] / max(1, st["tokens"]),
+            "mean_delta_star": st["sum_delta_star"] / max(1, st["tokens"]),
+            "copies_per_token": (st["prefetch_copies"] + st["demand_copies"]) / per_tok,
+            "demand_copies_per_token": st["demand_copies"] / per_tok,
+            "device_flag_wait_us_per_token": st["stall_ns"] / per_tok / 1e3,
+            "h2d_expert_gbs": st["bytes_copied"] / per_tok / (sec_e2e / args.steps) / 1e9}
+        apex.destroy()
+        if rank == 0:
+            # ---- stall-free mode
+            a2 = make_ctx(cfg, prob, cfg.C)
+            if "stall_free" in cfg.modes:
+                sec_sf = time_tokens(a2, h_dev, hp_dev, y_dev, B, "stall_free", args.warmup, args.steps)
+                s2 = a2.get_stats()
+                extras["stall_free"] = {"tokens_per_s": args.steps / sec_sf,
+                                        "substitutions_per_token": s2["substitutions"] / (args.warmup + args.steps),
+                                        "copies_per_token": s2["prefetch_copies"] / (args.warmup + args.steps)}
+            a2.destroy()
+            # ---- all experts resident (C = N): isolates the kernels from the host link
+            a3 = make_ctx(cfg, prob, cfg.N)
+            a3.warm_all()
+            sec_res = time_tokens(a3, h_dev, hp_dev, y_dev, B, "exact", args.warmup, args.steps)
+            extras["all_resident"] = {"tokens_per_s": args.steps / sec_res,
+                                      "frac_of_8TBs": bytes_step * cfg.L * args.steps / sec_res / 1e9 / NOMINAL_HBM_GBS,
+                                      "frac_of_peak": bytes_step * cfg.L * args.steps / sec_res / 1e9 / peak}
+            extras["exact"]["exposed_stall_us_per_token"] = (sec / args.steps - sec_res / args.steps) * 1e6
+            # ---- the dominant kernel alone
+            mean_s, med_s, n_l = time_ffn_kernel(a3, cfg, h_dev, hp_dev, B, tokens=max(2, min(8, args.steps)))
+            achieved = bytes_ffn / mean_s / 1e9
+            roof = {"bound": "hbm", "kernel": "moe_ffn_stream_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / NOMINAL_HBM_GBS,
+                    "traffic": NCU_TRAFFIC_BYTES.get(cfg.cfg_id), "algorithmic_bytes_per_launch": bytes_ffn,
+                    "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6, "launches_timed": n_l}
+            a3.destroy()
+            # ---- the oracle on the host cores (bounded sample)
+            tps, cores, dt = oracle_tokens_per_s(cfg, prob, args.cpu_baseline_tokens)
+            cpu = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",
+                   "sample": f"{args.cpu_baseline_tokens} decode tokens x {cfg.L} layers ({dt:.1f} s)"}
+    else:
+        apex.destroy()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank != 0:
+        return
+    line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
+            "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+            "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}", "L": cfg.L, "d": cfg.d, "N": cfg.N, "k": cfg.k,
+                       "I": cfg.I, "C": cfg.C, "B": B, "tau": TAU, "mode": "exact", "ctx_len": 1024,
+                       "parallelism": "replicas only" if world > 1 else "single GPU",
+                       "l2": "inputs larger than L2: each token streams %.0f MB of expert and attention bytes" %
+                             ((bytes_step + (4 * cfg.d * cfg.d + 2 * 1024 * cfg.d) * 2) * cfg.L / 1e6)},
+            "clocks": clocks, "gpu_launches": int(launches),
+            "e2e": e2e, "roofline": roof, "cpu_baseline": cpu, "modes": extras,
+            "stats_headline": {"copies_per_token": (st_all["prefetch_copies"] + st_all["demand_copies"]) / (args.warmup + args.steps)}}
+    print(json.dumps(line), flush=True)
+
+
+if __name__ == "__main__":
+    main()

@@ -17,6 +17,22 @@
 
 namespace apex {
 
+// Debug builds (-DAPEX_TIMELINE) record per-CTA time stamps of the streaming kernel.
+#ifdef APEX_TIMELINE
+__device__ unsigned long long g_timeline[1024 * 16];
+#define TL(slot)                                                                      \
+  do {                                                                                \
+    g_timeline[blockIdx.x * 16 + (slot)] = (slot) == 0 ? globaltimer_ns_raw() : (unsigned long long)clock64(); \
+  } while (0)
+__device__ __forceinline__ unsigned long long globaltimer_ns_raw() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#else
+#define TL(slot) do { } while (0)
+#endif
+
 constexpr int kConsumerWarps = 8;
 constexpr int kFfnThreads = (kConsumerWarps + 1) * 32;
 constexpr int kMaxStages = 32;
@@ -305,6 +321,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   const int G = gridDim.x, cta = blockIdx.x;
 
   if (tid == 0) {
+    TL(0);
+    TL(1);
     s_abort = 0;
     for (int s = 0; s < NS; ++s) {
       mbar_init(&s_full[s], 1);
@@ -384,6 +402,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     atomicAdd(p.zero_counter, 1ull);
   }
 
+  if (tid == 0) TL(2);  // plan done
   const long long total_rows = pair_row_off(pv, pv.n_pairs, I, p.I_shared);
   const long long r_begin = total_rows * cta / G, r_end = total_rows * (cta + 1) / G;
   const int n_my = (int)(r_end - r_begin);
@@ -449,11 +468,13 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
         }
         uint8_t* dst = smem + (size_t)s * entry_bytes;
         const uint8_t* src = base + (size_t)i * row_bytes;
+        if (q == 0) TL(3);  // first copy issued
         mbar_expect_tx(&s_full[s], entry_bytes);
         bulk_g2s(dst, src, row_bytes, &s_full[s]);
         bulk_g2s(dst + row_bytes, src + mat_bytes, row_bytes, &s_full[s]);
         bulk_g2s(dst + 2 * row_bytes, src + 2 * mat_bytes, row_bytes, &s_full[s]);
       }
+      TL(4);  // last copy issued
       if (waited && p.stats) atomicAdd(&p.stats->stall_ns, waited);
       if (!ok) {
         // a wait ran out: tell the consumers to stop, and the host
@@ -526,6 +547,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
         break;
       }
       if (*(volatile int*)&s_abort) break;
+      if (lane == 0 && q == 0) TL(5);                       // first row landed
+      if (lane == 0 && q == n_my - 1) TL(6);                // last row landed
       const uint4* gs = reinterpret_cast<const uint4*>(smem + (size_t)s * entry_bytes);
       const uint4* us = gs + row_bytes / 16;
       const uint4* ds = us + row_bytes / 16;
@@ -587,6 +610,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
 
   // ---- B == 1: reduce the eight partial vectors in shared memory, then one vector atomic per float4
   __syncthreads();  // every ring entry has been consumed; the ring is free
+  if (tid == 0) TL(7);
   float* red = reinterpret_cast<float*>(smem);
   if (warp < kConsumerWarps) {
     float4* dst = reinterpret_cast<float4*>(red + (size_t)warp * d);
@@ -607,6 +631,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     }
   }
   __syncthreads();
+  if (tid == 0) TL(8);
   if (n_my > 0 && !s_abort) {
     float4* y4 = reinterpret_cast<float4*>(p.y);
     for (int col4 = tid; col4 < d / 4; col4 += kFfnThreads) {
@@ -619,7 +644,14 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
       atomicAdd(y4 + col4, sacc);
     }
   }
+  if (tid == 0) TL(9);
 }
+
+#ifdef APEX_TIMELINE
+extern "C" int apex_debug_read_timeline(unsigned long long* host, int n) {
+  return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n);
+}
+#endif
 
 template <int NCH>
 static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {

@@ -108,7 +108,7 @@ def build_problem(cfg, device):
     from paper_2608_11688_b200 import synth
     routers = [synth.router_weights(cfg, l) for l in range(cfg.L)]
     cdf = [synth.cdf_params(cfg, l) for l in range(cfg.L)]
-    store = torch.empty((cfg.L, cfg.N, 3, cfg.I, cfg.d), dtype=torch.bfloat16, pin_memory=True)
+    store = torch.empty((cfg.L, cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16, pin_memory=True)
     shared = []
     for l in range(cfg.L):
         store[l].copy_(synth.expert_store(cfg, l, device=device))
@@ -204,11 +204,11 @@ def oracle_tokens_per_s(cfg, prob, n_tokens):
 
             def experts(e, l=l):
                 a = store[l, e].to(torch.float32).numpy()
-                return a[0], a[1], a[2].T
+                return synth.split_store(a)
             sh = None
             if shared[l] is not None:
                 s = shared[l].cpu().to(torch.float32).numpy()
-                sh = (s[0], s[1], s[2].T)
+                sh = synth.split_store(s)
             ao.layer_step(caches[l], W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=TAU, k=cfg.k,
                           h=hs[l][0][t], h_post=hs[l][1][t], mode="exact", expert_weights=experts, shared=sh)
     dt = time.perf_counter() - t0
@@ -230,7 +230,7 @@ def run_reference(args, cfg, rank):
     from paper_2608_11688_b200 import synth
     routers = [synth.router_weights(cfg, l) for l in range(cfg.L)]
     cdf = [synth.cdf_params(cfg, l) for l in range(cfg.L)]
-    store = torch.empty((cfg.L, cfg.N, 3, cfg.I, cfg.d), dtype=torch.bfloat16)
+    store = torch.empty((cfg.L, cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16)
     shared = []
     for l in range(cfg.L):
         store[l].copy_(synth.expert_store(cfg, l, device=dev))

@@ -25,9 +25,9 @@
  *   - A context is not thread-safe; use one host thread per context.
  *
  * Expert store layout (host, pinned): expert e of a layer starts at base + e*stride and holds
- *   gate[I][d], up[I][d], downT[I][d]   (bf16),
- * where downT is the transpose of the down projection W_down[d][I], so that intermediate
- * index i owns three contiguous d-vectors.  apex_pack_expert() converts from the usual
+ *   [I][3][d] bf16:  for each intermediate index i the three rows gate_i, up_i, downT_i,
+ * where downT_i[j] = W_down[j][i] (the down projection transposed), so that index i owns one
+ * contiguous block of 3*d values.  apex_pack_expert() converts from the usual
  * gate[I][d], up[I][d], down[d][I].
  */
 #ifndef APEX_H
@@ -116,7 +116,7 @@ int apex_set_cdf(apex_ctx* ctx, int layer, const float* w_host, const float* the
  * memory in the store layout described above.  Borrowed until apex_destroy. */
 int apex_register_experts(apex_ctx* ctx, int layer, const void* pinned_base, size_t expert_stride_bytes);
 /* Always-on shared expert (Sec. V-A: shared experts are outside the routing and the budget):
- * device pointer to gate[I_shared][d], up[I_shared][d], downT[I_shared][d], bf16.  Borrowed. */
+ * device pointer to [I_shared][3][d] bf16 in the store layout.  Borrowed. */
 int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights);
 /* Host helper: gate[I][d], up[I][d], down[d][I] -> store layout.  dst holds 3*I*d bf16. */
 int apex_pack_expert(const void* gate, const void* up, const void* down, int d, int I, void* dst);

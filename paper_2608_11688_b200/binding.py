@@ -176,7 +176,7 @@ class Apex:
         self._chk(self.lib.apex_set_cdf(self.h, layer, _ptr(w), _ptr(th)))
 
     def register_experts(self, layer, store, stride_bytes=None):
-        """store: pinned torch bf16 tensor [N][3][I][d] in the store layout."""
+        """store: pinned torch bf16 tensor [N][I][3][d] in the store layout."""
         self._keep.append(store)
         stride = stride_bytes if stride_bytes is not None else store.stride(0) * store.element_size()
         self._chk(self.lib.apex_register_experts(self.h, layer, _ptr(store), stride))

@@ -324,12 +324,14 @@ int apex_pack_expert(const void* gate, const void* up, const void* down, int d, 
   if (!gate || !up || !down || !dst || d < 1 || I < 1) return APEX_EINVAL;
   const uint16_t* dn = static_cast<const uint16_t*>(down);
   uint16_t* o = static_cast<uint16_t*>(dst);
-  const size_t m = (size_t)I * d;
-  memcpy(o, gate, m * 2);
-  memcpy(o + m, up, m * 2);
-  uint16_t* dT = o + 2 * m;
-  for (int j = 0; j < d; ++j)
-    for (int i = 0; i < I; ++i) dT[(size_t)i * d + j] = dn[(size_t)j * I + i];
+  const uint16_t* g = static_cast<const uint16_t*>(gate);
+  const uint16_t* u = static_cast<const uint16_t*>(up);
+  for (int i = 0; i < I; ++i) {
+    uint16_t* row = o + (size_t)i * 3 * d;
+    memcpy(row, g + (size_t)i * d, (size_t)d * 2);
+    memcpy(row + d, u + (size_t)i * d, (size_t)d * 2);
+    for (int j = 0; j < d; ++j) row[2 * (size_t)d + j] = dn[(size_t)j * I + i];
+  }
   return APEX_OK;
 }
 

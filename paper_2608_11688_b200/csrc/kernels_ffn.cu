@@ -2,15 +2,19 @@
 // (Sec. III-A weighted sum of expert outputs; Sec. IV-E execution modes; Algorithm 1).
 //
 // The step is bandwidth-bound at decode batch sizes: every weight byte is used once per token.
-// Layout: a slot holds gate[I][d], up[I][d], downT[I][d] (bf16), so intermediate index i owns three
-// d-vectors and one pass suffices:  a_i = g_e * silu(gate_i . h') * (up_i . h'),  y += a_i * downT_i.
+// Layout: a slot holds [I][3][d] bf16 -- for intermediate index i the three d-vectors gate_i, up_i,
+// downT_i are contiguous (downT is W_down transposed) -- so one pass suffices and every CTA reads one
+// contiguous byte range:  a_i = g_e * silu(gate_i . h') * (up_i . h'),  y += a_i * downT_i.
 //
 // Kernel: persistent, one CTA per SM.  The (pair, i) row space -- a pair is (token, expert) -- is
-// cut into equal contiguous ranges, one per CTA.  A producer thread streams row triples into a
-// shared-memory ring with bulk asynchronous copies (TMA, mbarrier completion); eight consumer warps
-// take ring entries round-robin, do the two dot products with warp-shuffle reductions and
-// accumulate the down projection in registers (fp32).  Partial y vectors are reduced across the
-// warps of the CTA in shared memory and added to y with vector atomics.
+// cut into equal contiguous ranges, one per CTA.  Each of the eight warps streams its own rows
+// (row q of the CTA belongs to warp q mod 8) into its stages of a shared-memory ring with one bulk
+// asynchronous copy per row (TMA, mbarrier completion; issuing from eight threads instead of one
+// matters: one thread sustains only about one bulk copy per 570 cycles), does the two dot products
+// with warp-shuffle reductions and accumulates the down projection in registers (fp32).  Partial y
+// vectors are reduced across the warps of the CTA in shared memory and added to y with vector
+// atomics.  Launched with programmatic stream serialization: the prologue overlaps the tail of the
+// gate kernel.
 #include <cuda_bf16.h>
 
 #include "apex_internal.hpp"
@@ -34,10 +38,9 @@ __device__ __forceinline__ unsigned long long globaltimer_ns_raw() {
 #endif
 
 constexpr int kConsumerWarps = 8;
-constexpr int kFfnThreads = (kConsumerWarps + 1) * 32;
+constexpr int kFfnThreads = kConsumerWarps * 32;
 constexpr int kMaxStages = 32;
 constexpr int kSmemBudget = 224 * 1024;  // ring bytes; static tables fit in what is left of the 227 KB per-CTA limit
-constexpr int kSmallPairs = APEX_MAX_TOPK + 1;
 
 __host__ __device__ constexpr int ring_stages(uint32_t entry_bytes) {
   int n = kSmemBudget / (int)entry_bytes;
@@ -80,7 +83,7 @@ __device__ __forceinline__ bool mbar_wait(uint64_t* bar, uint32_t parity, const 
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 255u) == 0u) {
-      if (*abort_flag) return false;
+      if (abort_flag && *abort_flag) return false;
       if ((long long)(globaltimer_ns() - t0) > limit_ns) return false;
     }
   }
@@ -96,6 +99,11 @@ __device__ __forceinline__ uint32_t ld_acquire_sys(const uint32_t* p) {
   asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
   return v;
 }
+__device__ __forceinline__ uint32_t ld_relaxed_sys(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.relaxed.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
 __device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned long long* p) {
   unsigned long long v;
   asm volatile("ld.acquire.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
@@ -104,6 +112,14 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned 
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
+__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const unsigned long long w = __shfl_xor_sync(0xffffffffu, v, o);
+    v = w > v ? w : v;
+  }
+  return v;
+}
 __device__ __forceinline__ float warp_sum(float v) {
 #pragma unroll
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
@@ -123,16 +139,36 @@ struct TokenPlan {
   float g0, g1;  // gates of experts lane, lane+32 (0 if not executed)
 };
 
-__device__ __forceinline__ TokenPlan plan_token(const int32_t* __restrict__ idx, const float* __restrict__ z_r,
-                                                const float* __restrict__ alpha, int N, int k, int mode,
-                                                int norm_topk, unsigned long long resident, int lane) {
+struct TokenLoads {
+  int my_idx;          // idx[lane] for lane < k, else -1
+  float al0, al1;      // alpha of experts lane, lane+32
+  float z0, z1;        // logits of experts lane, lane+32 (stall-free mode only)
+};
+__device__ __forceinline__ TokenLoads load_token(const int32_t* __restrict__ idx, const float* __restrict__ z_r,
+                                                 const float* __restrict__ alpha, int N, int k, int mode, int lane) {
+  TokenLoads t;
+  const int e0 = lane, e1 = lane + 32;
+  t.my_idx = lane < k ? idx[lane] : -1;
+  t.al0 = e0 < N ? alpha[e0] : 0.f;
+  t.al1 = e1 < N ? alpha[e1] : 0.f;
+  t.z0 = t.z1 = 0.f;
+  if (mode == APEX_MODE_STALL_FREE) {
+    t.z0 = e0 < N ? z_r[e0] : 0.f;
+    t.z1 = e1 < N ? z_r[e1] : 0.f;
+  }
+  return t;
+}
+__device__ __forceinline__ TokenPlan plan_token(const TokenLoads& t, int mode, int norm_topk, unsigned long long resident,
+                                                int lane) {
+  const int e0 = lane, e1 = lane + 32;
+  const int my_idx = t.my_idx;
+  const float al0 = t.al0, al1 = t.al1, z0 = t.z0, z1 = t.z1;
   unsigned lo = 0, hi = 0;
-  if (lane < k) {
-    const int e = idx[lane];
-    if (e < 32)
-      lo = 1u << e;
+  if (my_idx >= 0) {
+    if (my_idx < 32)
+      lo = 1u << my_idx;
     else
-      hi = 1u << (e - 32);
+      hi = 1u << (my_idx - 32);
   }
   lo = __reduce_or_sync(0xffffffffu, lo);
   hi = __reduce_or_sync(0xffffffffu, hi);
@@ -142,8 +178,6 @@ __device__ __forceinline__ TokenPlan plan_token(const int32_t* __restrict__ idx,
     const unsigned long long keep = kr & resident;
     const int n_missing = __popcll(kr & ~resident);
     const unsigned long long cand = resident & ~kr;
-    const int e0 = lane, e1 = lane + 32;
-    const float z0 = e0 < N ? z_r[e0] : 0.f, z1 = e1 < N ? z_r[e1] : 0.f;
     int r0 = 0, r1 = 0;
     unsigned long long rest = cand;
     while (rest) {
@@ -154,13 +188,12 @@ __device__ __forceinline__ TokenPlan plan_token(const int32_t* __restrict__ idx,
       r1 += (zf > z1 || (zf == z1 && f < e1)) ? 1 : 0;
     }
     const bool s0 = ((cand >> e0) & 1) && r0 < n_missing;
-    const bool s1 = e1 < 64 && ((cand >> e1) & 1) && r1 < n_missing;
+    const bool s1 = ((cand >> e1) & 1) && r1 < n_missing;
     const unsigned b0 = __ballot_sync(0xffffffffu, s0), b1 = __ballot_sync(0xffffffffu, s1);
     exec = keep | (((unsigned long long)b1 << 32) | b0);
   }
-  const int e0 = lane, e1 = lane + 32;
   const bool x0 = (exec >> e0) & 1, x1 = (exec >> e1) & 1;
-  const float a0 = x0 ? alpha[e0] : 0.f, a1 = x1 ? alpha[e1] : 0.f;
+  const float a0 = x0 ? al0 : 0.f, a1 = x1 ? al1 : 0.f;
   float denom = 1.f;
   if (norm_topk) denom = warp_sum(a0 + a1);
   TokenPlan tp;
@@ -204,8 +237,8 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   const int N = p.N, k = p.k, B = p.B;
   int my_subst = 0;
   for (int b = warp; b < B; b += nwarp) {
-    const TokenPlan tp = plan_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode,
-                                    p.norm_topk, p.snap.resident_mask, lane);
+    const TokenLoads tl = load_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode, lane);
+    const TokenPlan tp = plan_token(tl, p.mode, p.norm_topk, p.snap.resident_mask, lane);
     store_token_plan(tp, lane, k, p.plan_exec_idx + (size_t)b * k, p.plan_exec_gate + (size_t)b * k,
                      p.post_exec ? p.mbox_exec + (size_t)b * k : nullptr);
     if (p.post_exec) {
@@ -281,57 +314,55 @@ cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s) {
 }
 
 // ---------------------------------------------------------------- the streaming FFN kernel
-struct PairView {
-  const int32_t* tok;
-  const float* gate;
-  const int32_t* expert;
-  int n_pairs;
-  int n_routed;  // pairs before the shared-expert pairs
+// Row space: pair p (a (token, expert) pair; routed pairs first, then the shared-expert pairs) owns
+// I (or I_shared) consecutive rows; row r of pair p is intermediate index i = r - offset(p).
+struct RowMap {
+  int n_routed;          // routed pairs
+  int n_pairs;           // all pairs
+  long long routed_rows; // n_routed * I
+  long long total_rows;
 };
 
-__device__ __forceinline__ long long pair_row_off(const PairView& v, int pidx, int I, int I_shared) {
-  return pidx <= v.n_routed ? (long long)pidx * I : (long long)v.n_routed * I + (long long)(pidx - v.n_routed) * I_shared;
+__device__ __forceinline__ int nth_set_bit64(unsigned long long m, int n) {
+  for (int i = 0; i < n; ++i) m &= m - 1;
+  return __ffsll((long long)m) - 1;
 }
-// pair that contains row r
-__device__ __forceinline__ int pair_of_row(const PairView& v, long long r, int I, int I_shared) {
-  const long long routed_rows = (long long)v.n_routed * I;
-  return r < routed_rows ? (int)(r / I) : v.n_routed + (int)((r - routed_rows) / I_shared);
-}
+
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <int NCH, bool H_REGS>
 __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const FfnParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
-  __shared__ int32_t s_tok[kSmallPairs], s_exp[kSmallPairs];
-  __shared__ float s_gate[kSmallPairs];
-  __shared__ int s_np[2];
+  __shared__ uint64_t s_full[kMaxStages];
+  __shared__ float s_gate[kMaxStages];
+  __shared__ int s_tok[kMaxStages];
+  __shared__ int s_exp[kMaxStages];
   __shared__ int s_abort;
-  __shared__ uint64_t s_full[kMaxStages], s_empty[kMaxStages];
 
   constexpr int d = NCH * 256;
   constexpr uint32_t row_bytes = d * 2;
   constexpr uint32_t entry_bytes = 3 * row_bytes;
-  // The ring depth is a multiple of the consumer-warp count, so a stage is always consumed by the
-  // same warp: a warp can then never wait on a stage's next phase before it has consumed the current
-  // one (a parity wait cannot tell "one phase ahead" from "done").
+  // Each warp streams its own rows: it owns the ring stages {w, w+8, ...} and keeps NSW of its rows
+  // in flight, so a stage is produced and consumed by the same warp (no "empty" barriers, and a
+  // parity wait can never be a phase ahead).
   constexpr int NS = ring_stages(entry_bytes);
-  static_assert(NS >= kConsumerWarps && NS % kConsumerWarps == 0, "ring depth must be a multiple of the consumer warps");
+  constexpr int NSW = NS / kConsumerWarps;
+  static_assert(NS >= kConsumerWarps && NS % kConsumerWarps == 0, "ring depth must be a multiple of the warp count");
+  static_assert(NS * entry_bytes >= kConsumerWarps * d * 4, "ring must also hold the cross-warp reduction buffer");
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = p.N, k = p.k, I = p.I, B = p.B;
   const int G = gridDim.x, cta = blockIdx.x;
 
+  // ---- work that does not depend on the preceding kernel
   if (tid == 0) {
     TL(0);
     TL(1);
     s_abort = 0;
-    for (int s = 0; s < NS; ++s) {
-      mbar_init(&s_full[s], 1);
-      mbar_init(&s_empty[s], 1);
-    }
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
-
-  // ---- zero this CTA's slice of y (first launch of a layer-step only)
+  if (tid < NS) mbar_init(&s_full[tid], 1);
+  asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   if (!p.accumulate) {
     const size_t n4 = (size_t)B * d / 4;
     const size_t per = (n4 + G - 1) / G;
@@ -339,288 +370,86 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     float4* y4 = reinterpret_cast<float4*>(p.y);
     for (size_t i = lo + tid; i < hi; i += kFfnThreads) y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
   }
-
-  // ---- plan
-  PairView pv;
-  if (B == 1) {
-    if (warp == 0) {
-      const TokenPlan tp = plan_token(p.idx, p.z_r, p.alpha, N, k, p.mode, p.norm_topk, p.snap.resident_mask, lane);
-      if (cta == 0 && p.post_exec) {
-        store_token_plan(tp, lane, k, p.exec_idx, p.exec_gate, p.mbox_exec);
-        if (lane == 0 && p.stats) {
-          const int ns = __popcll(tp.exec_mask & ~tp.kr_mask);
-          if (ns) atomicAdd(&p.stats->substitutions, (unsigned long long)ns);
-        }
-        __threadfence_system();
-        __syncwarp();
-        if (lane == 0) {
-          __threadfence_system();
-          *p.mbox_seq = p.seq_value;
-        }
-      }
-      const unsigned long long run = tp.exec_mask & p.run_mask;
-      const int e0 = lane, e1 = lane + 32;
-      if ((run >> e0) & 1) {
-        const int pos = __popcll(run & ((1ull << e0) - 1ull));
-        s_tok[pos] = 0;
-        s_exp[pos] = e0;
-        s_gate[pos] = tp.g0;
-      }
-      if ((run >> e1) & 1) {
-        const int pos = __popcll(run & ((1ull << e1) - 1ull));
-        s_tok[pos] = 0;
-        s_exp[pos] = e1;
-        s_gate[pos] = tp.g1;
-      }
-      if (lane == 0) {
-        const int nr = __popcll(run);
-        if (p.run_shared) {
-          s_tok[nr] = 0;
-          s_exp[nr] = N;
-          s_gate[nr] = 1.f;
-        }
-        s_np[0] = nr + (p.run_shared ? 1 : 0);
-        s_np[1] = nr;
-      }
-    }
-    __syncthreads();
-    pv.tok = s_tok;
-    pv.gate = s_gate;
-    pv.expert = s_exp;
-    pv.n_pairs = s_np[0];
-    pv.n_routed = s_np[1];
-  } else {
-    __syncthreads();
-    pv.tok = p.pair_tok;
-    pv.gate = p.pair_gate;
-    pv.expert = p.pair_expert;
-    pv.n_pairs = p.n_pairs[0];
-    pv.n_routed = pv.n_pairs - (p.run_shared ? B : 0);
-  }
+  __syncthreads();
   if (!p.accumulate && tid == 0) {
     __threadfence();
     atomicAdd(p.zero_counter, 1ull);
   }
+  float hreg[H_REGS ? NCH * 8 : 1];
+  int cur_tok = -1;
+  if (H_REGS && B == 1) {  // h' is an input of the gate kernel as well: complete long before this kernel
+    cur_tok = 0;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const float4 a = __ldg(reinterpret_cast<const float4*>(p.hpost) + (c * 32 + lane) * 2);
+      const float4 b2 = __ldg(reinterpret_cast<const float4*>(p.hpost) + (c * 32 + lane) * 2 + 1);
+      hreg[c * 8 + 0] = a.x; hreg[c * 8 + 1] = a.y; hreg[c * 8 + 2] = a.z; hreg[c * 8 + 3] = a.w;
+      hreg[c * 8 + 4] = b2.x; hreg[c * 8 + 5] = b2.y; hreg[c * 8 + 6] = b2.z; hreg[c * 8 + 7] = b2.w;
+    }
+  }
+  pdl_wait();               // the gate's outputs (K_r, alpha, z_r) are complete from here on
+  pdl_launch_dependents();  // the next kernel may start its own prologue
+  if (tid == 0) TL(4);
 
+  // ---- every global load of the prologue is issued before the first use, so the latencies overlap.
+  // Slot-ready flags: lanes own experts lane and lane+32.  The flag is written by the copy engine
+  // after the expert's bytes; a relaxed load suffices here because the bulk copies that follow are
+  // issued only after the value has been inspected (and they read through L2, like the flag).
+  const int sl0 = lane < N ? p.snap.expert_slot[lane] : -1, sl1 = lane + 32 < N ? p.snap.expert_slot[lane + 32] : -1;
+  const uint32_t f0 = sl0 >= 0 ? ld_relaxed_sys(p.slot_ready + sl0) : 0u;
+  const uint32_t f1 = sl1 >= 0 ? ld_relaxed_sys(p.slot_ready + sl1) : 0u;
+  TokenLoads tl1;
+  if (B == 1) tl1 = load_token(p.idx, p.z_r, p.alpha, N, k, p.mode, lane);
+  unsigned long long ready_mask;
+  {
+    const bool r0 = sl0 >= 0 && (int32_t)(f0 - p.snap.need_gen[lane]) >= 0;
+    const bool r1 = sl1 >= 0 && (int32_t)(f1 - p.snap.need_gen[(lane + 32) & 63]) >= 0;
+    ready_mask = ((unsigned long long)__ballot_sync(0xffffffffu, r1) << 32) | __ballot_sync(0xffffffffu, r0);
+  }
+  if (tid == 0) TL(10);
+
+  // ---- plan: B == 1 every warp derives the execution set itself; B > 1 the plan kernel wrote it
+  RowMap rm;
+  unsigned long long run = 0;
+  float g0 = 0.f, g1 = 0.f;
+  TokenPlan tp1;
+  tp1.exec_mask = tp1.kr_mask = 0ull;
+  tp1.g0 = tp1.g1 = 0.f;
+  if (B == 1) {
+    const TokenPlan tp = plan_token(tl1, p.mode, p.norm_topk, p.snap.resident_mask, lane);
+    g0 = tp.g0;
+    g1 = tp.g1;
+    tp1 = tp;
+    run = tp.exec_mask & p.run_mask;
+    rm.n_routed = __popcll(run);
+    rm.n_pairs = rm.n_routed + (p.run_shared ? 1 : 0);
+  } else {
+    rm.n_pairs = p.n_pairs[0];
+    rm.n_routed = rm.n_pairs - (p.run_shared ? B : 0);
+  }
+  rm.routed_rows = (long long)rm.n_routed * I;
+  rm.total_rows = rm.routed_rows + (long long)(rm.n_pairs - rm.n_routed) * p.I_shared;
   if (tid == 0) TL(2);  // plan done
-  const long long total_rows = pair_row_off(pv, pv.n_pairs, I, p.I_shared);
-  const long long r_begin = total_rows * cta / G, r_end = total_rows * (cta + 1) / G;
+
+  const long long r_begin = rm.total_rows * cta / G, r_end = rm.total_rows * (cta + 1) / G;
   const int n_my = (int)(r_end - r_begin);
+  const int my_n = n_my > warp ? (n_my - warp + kConsumerWarps - 1) / kConsumerWarps : 0;  // rows of this warp
 
   float acc[NCH * 8];
 #pragma unroll
   for (int i = 0; i < NCH * 8; ++i) acc[i] = 0.f;
+  const float* hrow = p.hpost;
+  bool zero_seen = p.accumulate != 0;
+  bool ok = true;
+  unsigned long long waited = 0;
 
-  if (warp == kConsumerWarps) {
-    // ================= producer: one thread issues every copy of this CTA
-    if (lane == 0 && n_my > 0) {
-      int pidx = pair_of_row(pv, r_begin, I, p.I_shared);
-      long long pair_end = pair_row_off(pv, pidx + 1, I, p.I_shared);
-      int cur_e = -1;
-      const uint8_t* base = nullptr;
-      size_t mat_bytes = 0;
-      unsigned long long waited = 0;
-      bool ok = true;
-      for (int q = 0; q < n_my && ok; ++q) {
-        const long long r = r_begin + q;
-        while (r >= pair_end) {
-          ++pidx;
-          pair_end = pair_row_off(pv, pidx + 1, I, p.I_shared);
-        }
-        const int e = pv.expert[pidx];
-        if (e != cur_e) {
-          cur_e = e;
-          if (e < N) {
-            const int slot = p.snap.expert_slot[e];
-            if (slot < 0) {  // the host never asks for an expert without a slot; refuse rather than read out of range
-              ok = false;
-              break;
-            }
-            const uint32_t need = p.snap.need_gen[e];
-            const uint32_t* flag = p.slot_ready + slot;
-            if ((int32_t)(ld_acquire_sys(flag) - need) < 0) {
-              const unsigned long long t0 = globaltimer_ns();
-              while ((int32_t)(ld_acquire_sys(flag) - need) < 0) {
-                if ((long long)(globaltimer_ns() - t0) > p.wait_limit_ns) {
-                  ok = false;
-                  break;
-                }
-                __nanosleep(64);
-              }
-              waited += globaltimer_ns() - t0;
-            }
-            asm volatile("fence.proxy.async;" ::: "memory");
-            base = p.cache + (size_t)slot * p.slot_stride;
-            mat_bytes = (size_t)I * row_bytes;
-          } else {
-            base = p.shared_w;
-            mat_bytes = (size_t)p.I_shared * row_bytes;
-          }
-          if (!ok) break;
-        }
-        const long long i = r - pair_row_off(pv, pidx, I, p.I_shared);
-        const int s = q % NS;
-        if (q >= NS) {
-          if (!mbar_wait(&s_empty[s], (uint32_t)((q / NS - 1) & 1), &s_abort, p.wait_limit_ns)) {
-            ok = false;
-            break;
-          }
-        }
-        uint8_t* dst = smem + (size_t)s * entry_bytes;
-        const uint8_t* src = base + (size_t)i * row_bytes;
-        if (q == 0) TL(3);  // first copy issued
-        mbar_expect_tx(&s_full[s], entry_bytes);
-        bulk_g2s(dst, src, row_bytes, &s_full[s]);
-        bulk_g2s(dst + row_bytes, src + mat_bytes, row_bytes, &s_full[s]);
-        bulk_g2s(dst + 2 * row_bytes, src + 2 * mat_bytes, row_bytes, &s_full[s]);
-      }
-      TL(4);  // last copy issued
-      if (waited && p.stats) atomicAdd(&p.stats->stall_ns, waited);
-      if (!ok) {
-        // a wait ran out: tell the consumers to stop, and the host
-        atomicExch(&s_abort, 1);
-        if (p.stats) atomicAdd(&p.stats->timeouts, 1ull);
-        *p.mbox_status = 1u;
-        __threadfence_system();
-      }
-    }
-  } else {
-    // ================= consumers
-    float hreg[H_REGS ? NCH * 8 : 1];
-    bool zero_seen = p.accumulate != 0;  // batched case: y must be zero before the first atomic add
-    auto wait_zeroed = [&]() {
-      if (zero_seen) return;
-      const unsigned long long t0 = globaltimer_ns();
-      while (ld_acquire_gpu_u64(p.zero_counter) < p.zero_target) {
-        if ((long long)(globaltimer_ns() - t0) > p.wait_limit_ns) {
-          *p.mbox_status = 1u;
-          break;
-        }
-        __nanosleep(32);
-      }
+  auto poll_zeroed = [&](bool spin) {  // y must be all zero before anybody adds to it
+    if (zero_seen) return;
+    if (ld_acquire_gpu_u64(p.zero_counter) >= p.zero_target) {
       zero_seen = true;
-    };
-    int cur_tok = -1, pidx = 0;
-    long long pair_end = -1;
-    float gate = 0.f;
-    const float* hrow = p.hpost;
-    if (n_my > 0) pidx = pair_of_row(pv, r_begin, I, p.I_shared) - 1, pair_end = r_begin;  // forces a lookup
-    for (int q = warp; q < n_my; q += kConsumerWarps) {
-      const long long r = r_begin + q;
-      if (r >= pair_end) {
-        while (r >= pair_end) {
-          ++pidx;
-          pair_end = pair_row_off(pv, pidx + 1, I, p.I_shared);
-        }
-        gate = pv.gate[pidx];
-        const int t = pv.tok[pidx];
-        if (t != cur_tok) {
-          if (cur_tok >= 0) {
-            // batched case: this warp moves to another token, flush its partial sums
-            wait_zeroed();
-            float4* y4 = reinterpret_cast<float4*>(p.y + (size_t)cur_tok * d);
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-              const int col4 = (c * 32 + lane) * 2;
-              atomicAdd(y4 + col4, make_float4(acc[c * 8 + 0], acc[c * 8 + 1], acc[c * 8 + 2], acc[c * 8 + 3]));
-              atomicAdd(y4 + col4 + 1, make_float4(acc[c * 8 + 4], acc[c * 8 + 5], acc[c * 8 + 6], acc[c * 8 + 7]));
-            }
-#pragma unroll
-            for (int i2 = 0; i2 < NCH * 8; ++i2) acc[i2] = 0.f;
-          }
-          cur_tok = t;
-          hrow = p.hpost + (size_t)t * d;
-          if (H_REGS) {
-#pragma unroll
-            for (int c = 0; c < NCH; ++c) {
-              const float4 a = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2);
-              const float4 b2 = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2 + 1);
-              hreg[c * 8 + 0] = a.x; hreg[c * 8 + 1] = a.y; hreg[c * 8 + 2] = a.z; hreg[c * 8 + 3] = a.w;
-              hreg[c * 8 + 4] = b2.x; hreg[c * 8 + 5] = b2.y; hreg[c * 8 + 6] = b2.z; hreg[c * 8 + 7] = b2.w;
-            }
-          }
-        }
-      }
-      const int s = q % NS;
-      if (!mbar_wait(&s_full[s], (uint32_t)((q / NS) & 1), &s_abort, p.wait_limit_ns)) {
-        atomicExch(&s_abort, 1);
-        break;
-      }
-      if (*(volatile int*)&s_abort) break;
-      if (lane == 0 && q == 0) TL(5);                       // first row landed
-      if (lane == 0 && q == n_my - 1) TL(6);                // last row landed
-      const uint4* gs = reinterpret_cast<const uint4*>(smem + (size_t)s * entry_bytes);
-      const uint4* us = gs + row_bytes / 16;
-      const uint4* ds = us + row_bytes / 16;
-      float g = 0.f, u = 0.f;
-#pragma unroll
-      for (int c = 0; c < NCH; ++c) {
-        const uint4 gv = gs[c * 32 + lane];
-        const uint4 uv = us[c * 32 + lane];
-        float h0, h1, h2, h3, h4, h5, h6, h7;
-        if (H_REGS) {
-          h0 = hreg[c * 8 + 0]; h1 = hreg[c * 8 + 1]; h2 = hreg[c * 8 + 2]; h3 = hreg[c * 8 + 3];
-          h4 = hreg[c * 8 + 4]; h5 = hreg[c * 8 + 5]; h6 = hreg[c * 8 + 6]; h7 = hreg[c * 8 + 7];
-        } else {
-          const float4 a = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2);
-          const float4 b2 = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2 + 1);
-          h0 = a.x; h1 = a.y; h2 = a.z; h3 = a.w; h4 = b2.x; h5 = b2.y; h6 = b2.z; h7 = b2.w;
-        }
-        g = fmaf(bf16lo(gv.x), h0, g); g = fmaf(bf16hi(gv.x), h1, g);
-        g = fmaf(bf16lo(gv.y), h2, g); g = fmaf(bf16hi(gv.y), h3, g);
-        g = fmaf(bf16lo(gv.z), h4, g); g = fmaf(bf16hi(gv.z), h5, g);
-        g = fmaf(bf16lo(gv.w), h6, g); g = fmaf(bf16hi(gv.w), h7, g);
-        u = fmaf(bf16lo(uv.x), h0, u); u = fmaf(bf16hi(uv.x), h1, u);
-        u = fmaf(bf16lo(uv.y), h2, u); u = fmaf(bf16hi(uv.y), h3, u);
-        u = fmaf(bf16lo(uv.z), h4, u); u = fmaf(bf16hi(uv.z), h5, u);
-        u = fmaf(bf16lo(uv.w), h6, u); u = fmaf(bf16hi(uv.w), h7, u);
-      }
-      g = warp_sum(g);
-      u = warp_sum(u);
-      const float a = gate * (g / (1.f + expf(-g))) * u;
-#pragma unroll
-      for (int c = 0; c < NCH; ++c) {
-        const uint4 dv = ds[c * 32 + lane];
-        acc[c * 8 + 0] = fmaf(a, bf16lo(dv.x), acc[c * 8 + 0]);
-        acc[c * 8 + 1] = fmaf(a, bf16hi(dv.x), acc[c * 8 + 1]);
-        acc[c * 8 + 2] = fmaf(a, bf16lo(dv.y), acc[c * 8 + 2]);
-        acc[c * 8 + 3] = fmaf(a, bf16hi(dv.y), acc[c * 8 + 3]);
-        acc[c * 8 + 4] = fmaf(a, bf16lo(dv.z), acc[c * 8 + 4]);
-        acc[c * 8 + 5] = fmaf(a, bf16hi(dv.z), acc[c * 8 + 5]);
-        acc[c * 8 + 6] = fmaf(a, bf16lo(dv.w), acc[c * 8 + 6]);
-        acc[c * 8 + 7] = fmaf(a, bf16hi(dv.w), acc[c * 8 + 7]);
-      }
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&s_empty[s]);
+      return;
     }
-    if (B > 1 && cur_tok >= 0) {
-      // batched case: every warp adds its own partial sums (y was zeroed by all CTAs: wait for that)
-      wait_zeroed();
-      float4* y4 = reinterpret_cast<float4*>(p.y + (size_t)cur_tok * d);
-#pragma unroll
-      for (int c = 0; c < NCH; ++c) {
-        const int col4 = (c * 32 + lane) * 2;
-        atomicAdd(y4 + col4, make_float4(acc[c * 8 + 0], acc[c * 8 + 1], acc[c * 8 + 2], acc[c * 8 + 3]));
-        atomicAdd(y4 + col4 + 1, make_float4(acc[c * 8 + 4], acc[c * 8 + 5], acc[c * 8 + 6], acc[c * 8 + 7]));
-      }
-    }
-  }
-
-  if (B > 1) return;
-
-  // ---- B == 1: reduce the eight partial vectors in shared memory, then one vector atomic per float4
-  __syncthreads();  // every ring entry has been consumed; the ring is free
-  if (tid == 0) TL(7);
-  float* red = reinterpret_cast<float*>(smem);
-  if (warp < kConsumerWarps) {
-    float4* dst = reinterpret_cast<float4*>(red + (size_t)warp * d);
-#pragma unroll
-    for (int c = 0; c < NCH; ++c) {
-      const int col4 = (c * 32 + lane) * 2;
-      dst[col4] = make_float4(acc[c * 8 + 0], acc[c * 8 + 1], acc[c * 8 + 2], acc[c * 8 + 3]);
-      dst[col4 + 1] = make_float4(acc[c * 8 + 4], acc[c * 8 + 5], acc[c * 8 + 6], acc[c * 8 + 7]);
-    }
-  } else if (lane == 0 && !p.accumulate) {
+    if (!spin) return;
     const unsigned long long t0 = globaltimer_ns();
     while (ld_acquire_gpu_u64(p.zero_counter) < p.zero_target) {
       if ((long long)(globaltimer_ns() - t0) > p.wait_limit_ns) {
@@ -629,10 +458,239 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
       }
       __nanosleep(32);
     }
+    zero_seen = true;
+  };
+
+  // lane (j mod NSW) starts the copy of this warp's j-th row into stage (j mod NSW) of the warp.  The
+  // first NSW copies of a warp are thus issued by NSW lanes in one instruction.
+  auto issue = [&](int j) {
+    const long long r = r_begin + warp + (long long)kConsumerWarps * j;
+    int pidx, e, tok;
+    long long i;
+    float gate = 0.f;
+    if (r < rm.routed_rows) {
+      pidx = (int)(r / I);
+      i = r - (long long)pidx * I;
+    } else {
+      pidx = rm.n_routed + (int)((r - rm.routed_rows) / p.I_shared);
+      i = r - rm.routed_rows - (long long)(pidx - rm.n_routed) * p.I_shared;
+    }
+    if (B == 1) {
+      e = pidx < rm.n_routed ? nth_set_bit64(run, pidx) : N;
+      tok = 0;
+    } else {
+      e = p.pair_expert[pidx];
+      tok = p.pair_tok[pidx];
+      gate = p.pair_gate[pidx];
+    }
+    const uint8_t* base;
+    if (e < N) {
+      const int slot = p.snap.expert_slot[e];
+      if (slot < 0) {  // the host never asks for an expert without a slot; refuse rather than read out of range
+        ok = false;
+        return;
+      }
+      if (!((ready_mask >> e) & 1)) {
+        const uint32_t need = p.snap.need_gen[e];
+        const uint32_t* flag = p.slot_ready + slot;
+        const unsigned long long t0 = globaltimer_ns();
+        while ((int32_t)(ld_acquire_sys(flag) - need) < 0) {
+          if ((long long)(globaltimer_ns() - t0) > p.wait_limit_ns) {
+            ok = false;
+            break;
+          }
+          __nanosleep(64);
+        }
+        waited += globaltimer_ns() - t0;
+        if (!ok) return;
+        ready_mask |= 1ull << e;
+        asm volatile("fence.proxy.async;" ::: "memory");
+      }
+      base = p.cache + (size_t)slot * p.slot_stride;
+    } else {
+      base = p.shared_w;
+    }
+    const int s = warp + kConsumerWarps * (j % NSW);
+    s_gate[s] = gate;
+    s_tok[s] = tok;
+    s_exp[s] = e;
+    mbar_expect_tx(&s_full[s], entry_bytes);
+    bulk_g2s(smem + (size_t)s * entry_bytes, base + (size_t)i * entry_bytes, entry_bytes, &s_full[s]);
+  };
+
+  if (lane < NSW && lane < my_n) {
+    if (lane == 0 && warp == 0) TL(3);
+    issue(lane);
+    if (!ok) atomicExch(&s_abort, 1);
   }
-  __syncthreads();
+  __syncwarp();
+  if (B == 1 && cta == 0 && warp == 0 && p.post_exec) {
+    // the execution set goes to the caller's buffers and to the host mailbox while the first rows are in flight
+    store_token_plan(tp1, lane, k, p.exec_idx, p.exec_gate, p.mbox_exec);
+    if (lane == 0 && p.stats) {
+      const int ns = __popcll(tp1.exec_mask & ~tp1.kr_mask);
+      if (ns) atomicAdd(&p.stats->substitutions, (unsigned long long)ns);
+    }
+    __threadfence_system();
+    __syncwarp();
+    if (lane == 0) {
+      __threadfence_system();
+      *p.mbox_seq = p.seq_value;
+    }
+  }
+  int issued = my_n < NSW ? my_n : NSW;  // rows of this warp whose copy has been started (uniform across the warp)
+  for (int j = 0; j < my_n; ++j) {
+    if (lane == 0 && j == my_n - 1) poll_zeroed(false);  // latency hidden behind the wait for the last row
+    if (__any_sync(0xffffffffu, *(volatile int*)&s_abort != 0)) break;
+    const int s = warp + kConsumerWarps * (j % NSW);
+    if (!__all_sync(0xffffffffu, mbar_wait(&s_full[s], (uint32_t)((j / NSW) & 1), &s_abort, p.wait_limit_ns))) {
+      atomicExch(&s_abort, 1);
+      break;
+    }
+    if (lane == 0 && warp == 0 && j == 0) TL(5);
+    if (lane == 0 && j == my_n - 1) TL(6);
+    const int e = s_exp[s];
+    const int tok = s_tok[s];
+    float gate;
+    if (B == 1) {
+      gate = __shfl_sync(0xffffffffu, e < 32 ? g0 : g1, e & 31);
+      if (e >= N) gate = 1.f;
+    } else {
+      gate = s_gate[s];
+    }
+    if (tok != cur_tok) {
+      if (cur_tok >= 0) {
+        // batched case: this warp moves to another token, flush its partial sums
+        if (lane == 0) poll_zeroed(true);
+        __syncwarp();
+        float4* y4 = reinterpret_cast<float4*>(p.y + (size_t)cur_tok * d);
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const int col4 = (c * 32 + lane) * 2;
+          atomicAdd(y4 + col4, make_float4(acc[c * 8 + 0], acc[c * 8 + 1], acc[c * 8 + 2], acc[c * 8 + 3]));
+          atomicAdd(y4 + col4 + 1, make_float4(acc[c * 8 + 4], acc[c * 8 + 5], acc[c * 8 + 6], acc[c * 8 + 7]));
+        }
+#pragma unroll
+        for (int i2 = 0; i2 < NCH * 8; ++i2) acc[i2] = 0.f;
+      }
+      cur_tok = tok;
+      hrow = p.hpost + (size_t)tok * d;
+      if (H_REGS) {
+#pragma unroll
+        for (int c = 0; c < NCH; ++c) {
+          const float4 a = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2);
+          const float4 b2 = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2 + 1);
+          hreg[c * 8 + 0] = a.x; hreg[c * 8 + 1] = a.y; hreg[c * 8 + 2] = a.z; hreg[c * 8 + 3] = a.w;
+          hreg[c * 8 + 4] = b2.x; hreg[c * 8 + 5] = b2.y; hreg[c * 8 + 6] = b2.z; hreg[c * 8 + 7] = b2.w;
+        }
+      }
+    }
+    const uint4* gs = reinterpret_cast<const uint4*>(smem + (size_t)s * entry_bytes);
+    const uint4* us = gs + row_bytes / 16;
+    const uint4* ds = us + row_bytes / 16;
+    float g = 0.f, u = 0.f;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const uint4 gv = gs[c * 32 + lane];
+      const uint4 uv = us[c * 32 + lane];
+      float h0, h1, h2, h3, h4, h5, h6, h7;
+      if (H_REGS) {
+        h0 = hreg[c * 8 + 0]; h1 = hreg[c * 8 + 1]; h2 = hreg[c * 8 + 2]; h3 = hreg[c * 8 + 3];
+        h4 = hreg[c * 8 + 4]; h5 = hreg[c * 8 + 5]; h6 = hreg[c * 8 + 6]; h7 = hreg[c * 8 + 7];
+      } else {
+        const float4 a = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2);
+        const float4 b2 = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2 + 1);
+        h0 = a.x; h1 = a.y; h2 = a.z; h3 = a.w; h4 = b2.x; h5 = b2.y; h6 = b2.z; h7 = b2.w;
+      }
+      g = fmaf(bf16lo(gv.x), h0, g); g = fmaf(bf16hi(gv.x), h1, g);
+      g = fmaf(bf16lo(gv.y), h2, g); g = fmaf(bf16hi(gv.y), h3, g);
+      g = fmaf(bf16lo(gv.z), h4, g); g = fmaf(bf16hi(gv.z), h5, g);
+      g = fmaf(bf16lo(gv.w), h6, g); g = fmaf(bf16hi(gv.w), h7, g);
+      u = fmaf(bf16lo(uv.x), h0, u); u = fmaf(bf16hi(uv.x), h1, u);
+      u = fmaf(bf16lo(uv.y), h2, u); u = fmaf(bf16hi(uv.y), h3, u);
+      u = fmaf(bf16lo(uv.z), h4, u); u = fmaf(bf16hi(uv.z), h5, u);
+      u = fmaf(bf16lo(uv.w), h6, u); u = fmaf(bf16hi(uv.w), h7, u);
+    }
+    g = warp_sum(g);
+    u = warp_sum(u);
+    const float a = gate * (g / (1.f + expf(-g))) * u;
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const uint4 dv = ds[c * 32 + lane];
+      acc[c * 8 + 0] = fmaf(a, bf16lo(dv.x), acc[c * 8 + 0]);
+      acc[c * 8 + 1] = fmaf(a, bf16hi(dv.x), acc[c * 8 + 1]);
+      acc[c * 8 + 2] = fmaf(a, bf16lo(dv.y), acc[c * 8 + 2]);
+      acc[c * 8 + 3] = fmaf(a, bf16hi(dv.y), acc[c * 8 + 3]);
+      acc[c * 8 + 4] = fmaf(a, bf16lo(dv.z), acc[c * 8 + 4]);
+      acc[c * 8 + 5] = fmaf(a, bf16hi(dv.z), acc[c * 8 + 5]);
+      acc[c * 8 + 6] = fmaf(a, bf16lo(dv.w), acc[c * 8 + 6]);
+      acc[c * 8 + 7] = fmaf(a, bf16hi(dv.w), acc[c * 8 + 7]);
+    }
+    __syncwarp();  // every lane has read stage s: it may be refilled
+    if (j + NSW < my_n) {
+      if (lane == j % NSW) {
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        issue(j + NSW);
+        if (!ok) atomicExch(&s_abort, 1);
+      }
+      ++issued;
+    }
+  }
+  waited = warp_max_u64(waited);
+  ok = __all_sync(0xffffffffu, ok);
+  if (lane == 0) {
+    if (waited && p.stats) atomicAdd(&p.stats->stall_ns, waited);
+    if (!ok) {
+      if (p.stats) atomicAdd(&p.stats->timeouts, 1ull);
+      *p.mbox_status = 1u;
+      __threadfence_system();
+    }
+  }
+  const bool aborted = *(volatile int*)&s_abort != 0;
+  if (aborted) {
+    // leave only after every copy this warp started has landed (bounded), so that no copy is in
+    // flight into the shared memory of an exited CTA
+    for (int jj = 0; jj < issued; ++jj) {
+      const int s = warp + kConsumerWarps * (jj % NSW);
+      if (jj + NSW >= issued) mbar_wait(&s_full[s], (uint32_t)((jj / NSW) & 1), nullptr, p.wait_limit_ns);
+    }
+  }
+
+  if (B > 1) {
+    if (cur_tok >= 0 && !aborted) {
+      if (lane == 0) poll_zeroed(true);
+      __syncwarp();
+      float4* y4 = reinterpret_cast<float4*>(p.y + (size_t)cur_tok * d);
+#pragma unroll
+      for (int c = 0; c < NCH; ++c) {
+        const int col4 = (c * 32 + lane) * 2;
+        atomicAdd(y4 + col4, make_float4(acc[c * 8 + 0], acc[c * 8 + 1], acc[c * 8 + 2], acc[c * 8 + 3]));
+        atomicAdd(y4 + col4 + 1, make_float4(acc[c * 8 + 4], acc[c * 8 + 5], acc[c * 8 + 6], acc[c * 8 + 7]));
+      }
+    }
+    return;
+  }
+
+  // ---- B == 1: reduce the eight partial vectors in shared memory, then one vector atomic per float4
+  __syncthreads();  // every ring entry has been consumed; the ring is free
+  if (tid == 0) TL(7);
+  float* red = reinterpret_cast<float*>(smem);
+  {
+    float4* dst = reinterpret_cast<float4*>(red + (size_t)warp * d);
+#pragma unroll
+    for (int c = 0; c < NCH; ++c) {
+      const int col4 = (c * 32 + lane) * 2;
+      dst[col4] = make_float4(acc[c * 8 + 0], acc[c * 8 + 1], acc[c * 8 + 2], acc[c * 8 + 3]);
+      dst[col4 + 1] = make_float4(acc[c * 8 + 4], acc[c * 8 + 5], acc[c * 8 + 6], acc[c * 8 + 7]);
+    }
+  }
+  // one thread makes sure that every CTA has zeroed its slice of y (normally seen long ago)
+  if (!__syncthreads_or((lane == 0 && zero_seen) ? 1 : 0)) {
+    if (tid == 0) poll_zeroed(true);
+    __syncthreads();
+  }
   if (tid == 0) TL(8);
-  if (n_my > 0 && !s_abort) {
+  if (n_my > 0 && !aborted) {
     float4* y4 = reinterpret_cast<float4*>(p.y);
     for (int col4 = tid; col4 < d / 4; col4 += kFfnThreads) {
       float4 sacc = make_float4(0.f, 0.f, 0.f, 0.f);
@@ -665,8 +723,17 @@ static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
     if (e != cudaSuccess) return e;
     configured = true;
   }
-  moe_ffn_stream_kernel<NCH, HR><<<n_sm, kFfnThreads, smem, s>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_sm, 1, 1);
+  cfg.blockDim = dim3(kFfnThreads, 1, 1);
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // prologue overlaps the gate kernel's tail
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, moe_ffn_stream_kernel<NCH, HR>, p);
 }
 
 bool ffn_shape_supported(int d) {

@@ -14,7 +14,8 @@ Recipe (one base seed, one sub-stream per (config, layer, tensor kind)):
 * hidden states     h ~ N(0,1); h' = h + N(0, 0.25); both rounded to bf16-representable
                     values but stored widened in fp32
 * expert weights    bf16, N(0, 0.02^2), generated directly in the library's store layout
-                    gate[I][d], up[I][d], downT[I][d]  (downT is W_down transposed)
+                    [I][3][d]: for intermediate index i the rows gate_i, up_i, downT_i
+                    (downT is W_down transposed)
 * confidence model  w[N], theta[N-k+1]: frozen values fitted offline on calibration tokens
                     of this same generator (files under ``data/``), else a fixed hand-set
                     model
@@ -112,14 +113,15 @@ def hidden_states(cfg: Config, layer: int, T: int, B: int = 1, calib: bool = Fal
 
 
 def expert_store(cfg: Config, layer: int, device="cpu", pin: bool = False, out=None):
-    """bf16 tensor [N][3][I][d] in the library's store layout: gate, up, downT per expert.
+    """bf16 tensor [N][I][3][d] in the library's store layout: per intermediate index i the rows
+    gate_i, up_i, downT_i.
 
-    The conceptual down projection is W_down[j][i] = downT[i][j].  Drawn with torch's
+    The conceptual down projection is W_down[j][i] = downT[i][j] = store[e][i][2][j].  Drawn with torch's
     seeded generator on ``device`` (CPU and CUDA streams differ; within one run everybody
     reads the same bytes).
     """
     import torch
-    shape = (cfg.N, 3, cfg.I, cfg.d)
+    shape = (cfg.N, cfg.I, 3, cfg.d)
     g = torch.Generator(device=device)
     g.manual_seed((BASE_SEED * 1000003 + cfg.cfg_id * 10007 + layer * 101 + _KIND["experts"]) & 0x7FFFFFFF)
     if out is None:
@@ -127,19 +129,19 @@ def expert_store(cfg: Config, layer: int, device="cpu", pin: bool = False, out=N
             if str(device) == "cpu" else torch.empty(shape, dtype=torch.bfloat16, device=device)
     # draw expert by expert to bound the fp32 temporary
     for e in range(cfg.N):
-        t = torch.randn((3, cfg.I, cfg.d), generator=g, device=device, dtype=torch.float32)
+        t = torch.randn((cfg.I, 3, cfg.d), generator=g, device=device, dtype=torch.float32)
         out[e].copy_((t * 0.02).to(torch.bfloat16))
     return out
 
 
 def shared_expert(cfg: Config, layer: int, device="cpu"):
-    """bf16 tensor [3][I_shared][d] (gate, up, downT) or None when the config has none."""
+    """bf16 tensor [I_shared][3][d] (rows gate_i, up_i, downT_i) or None when the config has none."""
     import torch
     if cfg.I_shared == 0:
         return None
     g = torch.Generator(device=device)
     g.manual_seed((BASE_SEED * 1000003 + cfg.cfg_id * 10007 + layer * 101 + _KIND["shared"]) & 0x7FFFFFFF)
-    t = torch.randn((3, cfg.I_shared, cfg.d), generator=g, device=device, dtype=torch.float32)
+    t = torch.randn((cfg.I_shared, 3, cfg.d), generator=g, device=device, dtype=torch.float32)
     return (t * 0.02).to(torch.bfloat16)
 
 
@@ -171,6 +173,11 @@ def cdf_params(cfg: Config, layer: int, allow_handset: bool = True):
     if not allow_handset:
         raise FileNotFoundError(path)
     return handset_cdf_params(cfg)
+
+
+def split_store(w):
+    """Store layout [..., I, 3, d] -> the usual (W_gate [I][d], W_up [I][d], W_down [d][I]) views."""
+    return w[..., 0, :], w[..., 1, :], np.swapaxes(w[..., 2, :], -1, -2)
 
 
 def bf16_to_f32_numpy(t) -> np.ndarray:

@@ -45,7 +45,7 @@ class Problem:
         self.stores = []
         self.shared = []
         for l in range(self.L):
-            st = torch.empty((cfg.N, 3, cfg.I, cfg.d), dtype=torch.bfloat16, pin_memory=True)
+            st = torch.empty((cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16, pin_memory=True)
             tmp = synth.expert_store(cfg, l, device=device)
             st.copy_(tmp)
             del tmp
@@ -74,7 +74,7 @@ class Problem:
 
         def get(e):
             w = st[e].to(torch.float32).numpy()
-            return w[0], w[1], w[2].T
+            return synth.split_store(w)
         return get
 
     def oracle_shared(self, layer):
@@ -82,7 +82,7 @@ class Problem:
         if sh is None:
             return None
         w = sh.detach().cpu().to(torch.float32).numpy()
-        return w[0], w[1], w[2].T
+        return synth.split_store(w)
 
 
 def _excusable(tok, what: str) -> bool:

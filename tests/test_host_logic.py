@@ -57,11 +57,11 @@ def test_pack_expert_transposes_down(lib):
     gate = rng.integers(0, 2 ** 16, (I, d)).astype(np.uint16)
     up = rng.integers(0, 2 ** 16, (I, d)).astype(np.uint16)
     down = rng.integers(0, 2 ** 16, (d, I)).astype(np.uint16)
-    out = np.zeros((3, I, d), np.uint16)
+    out = np.zeros((I, 3, d), np.uint16)
     assert lib.apex_pack_expert(gate.ctypes.data, up.ctypes.data, down.ctypes.data, d, I, out.ctypes.data) == 0
-    np.testing.assert_array_equal(out[0], gate)
-    np.testing.assert_array_equal(out[1], up)
-    np.testing.assert_array_equal(out[2], down.T)
+    np.testing.assert_array_equal(out[:, 0], gate)
+    np.testing.assert_array_equal(out[:, 1], up)
+    np.testing.assert_array_equal(out[:, 2], down.T)
 
 
 @pytest.mark.parametrize("reuse", [True, False])

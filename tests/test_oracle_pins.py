@@ -319,12 +319,12 @@ def _dense_topk_moe(W_r, b_r, hp, k, experts, shared):
 def _tiny_problem(cfg, layer=0):
     W_r, b_r, W_p, b_p = synth.router_weights(cfg, layer)
     store = synth.bf16_to_f32_numpy(synth.expert_store(cfg, layer))
-    experts = lambda e: (store[e, 0], store[e, 1], store[e, 2].T)
+    experts = lambda e: synth.split_store(store[e])
     sh = synth.shared_expert(cfg, layer)
     shared = None
     if sh is not None:
         s = synth.bf16_to_f32_numpy(sh)
-        shared = (s[0], s[1], s[2].T)
+        shared = synth.split_store(s)
     w, theta = synth.handset_cdf_params(cfg)
     return W_r, b_r, W_p, b_p, experts, shared, w, theta
 

@@ -165,27 +165,32 @@ def time_tokens(apex, h, hp, y, B, mode, warmup, steps, dist_sync=None, host=Fal
 
 
 def time_ffn_kernel(apex, cfg, h, hp, B, tokens):
-    """Average device time of one expert-FFN launch, all experts resident: CUDA events around each
-    launch on the launching stream, summed over layers and tokens."""
+    """Average device time of one expert-FFN launch, all experts resident.  Per token the gates of all
+    layers run first; then the L expert-FFN kernels are launched back to back (each reads its own
+    layer's experts, so nothing is served from L2) between two CUDA events on the launching stream."""
     import torch
     dev = h.device
-    idx = torch.empty((B, cfg.k), dtype=torch.int32, device=dev)
-    al = torch.empty((B, cfg.N), dtype=torch.float32, device=dev)
-    y = torch.empty((B, cfg.d), dtype=torch.float32, device=dev)
+    idx = torch.empty((cfg.L, B, cfg.k), dtype=torch.int32, device=dev)
+    al = torch.empty((cfg.L, B, cfg.N), dtype=torch.float32, device=dev)
+    y = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32, device=dev)
     T = h.shape[0]
-    pairs = []
+    per_launch = []
+    stream = torch.cuda.current_stream().cuda_stream
+    y_ptr = [y[l].data_ptr() for l in range(cfg.L)]
     for t in range(tokens + 1):
+        hp_ptr = [hp[t % T, l].data_ptr() for l in range(cfg.L)]
         for l in range(cfg.L):
-            apex.route_topk(l, hp[t % T, l], B, idx, al)
-            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            e0.record()
-            apex.moe_ffn(l, "exact", hp[t % T, l], B, y)
-            e1.record()
-            if t > 0:                       # first pass is warm-up
-                pairs.append((e0, e1))
-    torch.cuda.synchronize()
-    ms = [a.elapsed_time(b) for a, b in pairs]
-    return statistics.mean(ms) * 1e-3, statistics.median(ms) * 1e-3, len(ms)
+            apex.route_topk(l, hp[t % T, l], B, idx[l], al[l])
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for l in range(cfg.L):
+            apex.moe_ffn_raw(l, 0, hp_ptr[l], B, y_ptr[l], stream)
+        e1.record()
+        torch.cuda.synchronize()
+        if t > 0:                       # first pass is warm-up
+            per_launch.append(e0.elapsed_time(e1) / cfg.L)
+    return statistics.mean(per_launch) * 1e-3, statistics.median(per_launch) * 1e-3, len(per_launch) * cfg.L
 
 
 def oracle_tokens_per_s(cfg, prob, n_tokens):

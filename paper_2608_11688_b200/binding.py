@@ -208,6 +208,12 @@ class Apex:
         self._chk(self.lib.apex_moe_ffn(self.h, layer, m, _ptr(hpost_dev), B, _ptr(y_dev), _ptr(exec_idx_dev),
                                         _ptr(exec_gate_dev), _stream(stream)))
 
+    def moe_ffn_raw(self, layer, mode_int, hpost_ptr, B, y_ptr, stream_int):
+        """Same call with raw addresses (no per-call marshalling): for tight timing loops."""
+        rc = self.lib.apex_moe_ffn(self.h, layer, mode_int, hpost_ptr, B, y_ptr, None, None, stream_int)
+        if rc != APEX_OK:
+            self._chk(rc)
+
     def decode_token(self, h_dev, hpost_dev, B, tau, mode, y_dev, stream=None):
         m = MODES[mode] if isinstance(mode, str) else mode
         self._chk(self.lib.apex_decode_token(self.h, _ptr(h_dev), _ptr(hpost_dev), B, float(tau), m, _ptr(y_dev),

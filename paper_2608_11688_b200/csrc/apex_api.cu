@@ -45,6 +45,27 @@ cudaError_t dev_alloc(T** p, size_t n) {
 
 MailboxHeader* mhdr(apex_ctx* ctx) { return reinterpret_cast<MailboxHeader*>(ctx->mbox); }
 int32_t* mbox_i32(apex_ctx* ctx, size_t off) { return reinterpret_cast<int32_t*>(ctx->mbox + off); }
+volatile uint32_t* mbox_route_seq(apex_ctx* ctx, int l) {
+  return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_route_seq) + l;
+}
+volatile uint32_t* mbox_exec_seq(apex_ctx* ctx, int l) {
+  return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_exec_seq) + l;
+}
+int32_t* mbox_kr(apex_ctx* ctx, int l) { return mbox_i32(ctx, ctx->ml.off_kr + (size_t)l * ctx->ml.kr_stride); }
+int32_t* mbox_exec(apex_ctx* ctx, int l) { return mbox_i32(ctx, ctx->ml.off_exec + (size_t)l * ctx->ml.kr_stride); }
+
+// A 32-bit word written in stream order (after everything queued before it on that stream).
+int stream_write32(apex_ctx* ctx, cudaStream_t cs, uint32_t* dev, uint32_t value) {
+  if (ctx->fn_write_value32) {
+    int r = reinterpret_cast<WriteValue32Fn>(ctx->fn_write_value32)(cs, (unsigned long long)(uintptr_t)dev, value, 0);
+    if (r != 0) return fail(ctx, APEX_ECUDA, "cuStreamWriteValue32 failed");
+    return APEX_OK;
+  }
+  uint32_t* srcv = ctx->gen_src + (ctx->gen_src_pos++ % ctx->gen_src_len);
+  *srcv = value;
+  CU_TRY(ctx, cudaMemcpyAsync(dev, srcv, sizeof(uint32_t), cudaMemcpyHostToDevice, cs));
+  return APEX_OK;
+}
 
 // Bounded host wait for a mailbox sequence number.
 bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
@@ -80,13 +101,9 @@ int issue_copy(apex_ctx* ctx, int layer, int e, int slot, cudaStream_t cs) {
     ctx->inject = 0;
     ctx->withheld_flag = flag;
     ctx->withheld_gen = gen;
-  } else if (ctx->fn_write_value32) {
-    int r = reinterpret_cast<WriteValue32Fn>(ctx->fn_write_value32)(cs, (unsigned long long)(uintptr_t)flag, gen, 0);
-    if (r != 0) return fail(ctx, APEX_ECUDA, "cuStreamWriteValue32 failed");
   } else {
-    uint32_t* srcv = ctx->gen_src + (ctx->gen_src_pos++ % ctx->gen_src_len);
-    *srcv = gen;
-    CU_TRY(ctx, cudaMemcpyAsync(flag, srcv, sizeof(uint32_t), cudaMemcpyHostToDevice, cs));
+    int r = stream_write32(ctx, cs, flag, gen);
+    if (r != APEX_OK) return r;
   }
   ctx->phys_expert[layer][slot] = e;
   ctx->host_stats[layer].bytes_copied += (int64_t)ctx->expert_bytes;
@@ -178,13 +195,15 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(cudaMemset(ctx->d_slot_ready, 0, L * C * sizeof(uint32_t)));
   CR(dev_alloc(&ctx->d_zp, MB * N));
   CR(dev_alloc(&ctx->d_qp, MB * N));
-  CR(dev_alloc(&ctx->d_zr, MB * N));
+  CR(dev_alloc(&ctx->d_zr, L * MB * N));
+  CR(dev_alloc(&ctx->d_demand, L * N));
+  CR(cudaMemset(ctx->d_demand, 0, L * N * sizeof(uint32_t)));
   CR(dev_alloc(&ctx->d_pi, MB * N));
   CR(dev_alloc(&ctx->d_ncand, MB));
   CR(dev_alloc(&ctx->d_stats, L));
   CR(cudaMemset(ctx->d_stats, 0, L * sizeof(DevStats)));
-  CR(dev_alloc(&ctx->d_counters, 4));
-  CR(cudaMemset(ctx->d_counters, 0, 4 * sizeof(unsigned long long)));
+  CR(dev_alloc(&ctx->d_counters, 2 + L));
+  CR(cudaMemset(ctx->d_counters, 0, (2 + L) * sizeof(unsigned long long)));
   const size_t max_pairs = MB * (k + 1);
   CR(dev_alloc(&ctx->d_plan_exec_idx, MB * k));
   CR(dev_alloc(&ctx->d_plan_exec_gate, MB * k));
@@ -193,9 +212,9 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(dev_alloc(&ctx->d_pair_expert, max_pairs));
   CR(dev_alloc(&ctx->d_n_pairs, 4));
   CR(dev_alloc(&ctx->d_cand, MB * C));
-  CR(dev_alloc(&ctx->d_idx, MB * k));
+  CR(dev_alloc(&ctx->d_idx, L * MB * k));
   CR(dev_alloc(&ctx->d_exec_idx, MB * k));
-  CR(dev_alloc(&ctx->d_alpha, MB * N));
+  CR(dev_alloc(&ctx->d_alpha, L * MB * N));
   CR(dev_alloc(&ctx->d_exec_gate, MB * k));
   CR(dev_alloc(&ctx->d_cand_ncand, MB));
   ctx->attn_bytes = (4 * d * d + 2 * (size_t)ctx->cfg.ctx_len * d) * 2;
@@ -207,11 +226,18 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   // mapped mailbox
   MailboxLayout& ml = ctx->ml;
   size_t off = sizeof(MailboxHeader);
+  ml.off_route_seq = off; off += L * sizeof(uint32_t);
+  ml.off_exec_seq = off;  off += L * sizeof(uint32_t);
+  off = (off + 15) & ~(size_t)15;
   ml.off_ncand = off; off += MB * sizeof(int32_t);
   ml.off_cand = off;  off += MB * C * sizeof(int32_t);
-  ml.off_kr = off;    off += MB * k * sizeof(int32_t);
-  ml.off_exec = off;  off += MB * k * sizeof(int32_t);
+  ml.kr_stride = MB * k * sizeof(int32_t);
+  ml.off_kr = off;    off += L * ml.kr_stride;
+  ml.off_exec = off;  off += L * ml.kr_stride;
   ml.bytes = off;
+  ctx->route_seq.assign(L, 0u);
+  ctx->exec_seq.assign(L, 0u);
+  ctx->route_done.assign(L, 0ull);
   CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->mbox), ml.bytes, cudaHostAllocMapped | cudaHostAllocPortable));
   memset(ctx->mbox, 0, ml.bytes);
   ctx->gen_src_len = 1 << 16;
@@ -240,6 +266,7 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   ctx->last_copies.assign(L, {});
   ctx->host_stats.assign(L, apex_step_stats{});
   ctx->step.assign(L, apex_ctx::StepState{});
+  ctx->ffn_params.assign(L, FfnParams{});
   *out = ctx;
   return APEX_OK;
 }
@@ -249,7 +276,7 @@ int apex_destroy(apex_ctx* ctx) {
   cudaDeviceSynchronize();
   cudaGetLastError();
   void* dev[] = {ctx->d_Wr, ctx->d_br, ctx->d_Wp, ctx->d_bp, ctx->d_w, ctx->d_theta, ctx->d_cache, ctx->d_slot_ready, ctx->d_zp,
-                 ctx->d_qp, ctx->d_zr, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_plan_exec_idx,
+                 ctx->d_qp, ctx->d_zr, ctx->d_demand, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_plan_exec_idx,
                  ctx->d_plan_exec_gate, ctx->d_pair_tok, ctx->d_pair_gate, ctx->d_pair_expert, ctx->d_n_pairs, ctx->d_cand,
                  ctx->d_idx, ctx->d_exec_idx, ctx->d_alpha, ctx->d_exec_gate, ctx->d_cand_ncand, ctx->d_attn, ctx->d_attn_sink,
                  ctx->d_h_stage, ctx->d_hp_stage, ctx->d_y_stage};
@@ -342,6 +369,7 @@ int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stre
   CHECK_LAYER(ctx, layer);
   if (!h_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_predict: bad h or B");
   const size_t N = ctx->cfg.N, d = ctx->cfg.d;
+  if (ctx->step[layer].pending) return fail(ctx, APEX_ESTATE, "the previous expert FFN of this layer has not been completed");
   ctx->tables[layer].begin_step();
   ctx->last_copies[layer].clear();
   ctx->step[layer] = apex_ctx::StepState{};
@@ -412,21 +440,16 @@ int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream) {
   std::vector<SlotCopy> copies;
   if (!ctx->tables[layer].plan_prefetch(cand, ncand, B, C, &copies)) return fail(ctx, APEX_ESTATE, "no evictable slot");
   // issue most likely first: order of appearance in the first token's ranked list, others after
+  std::vector<SlotCopy> ordered = copies;
   if (B == 1 && copies.size() > 1) {
     int pos[APEX_MAX_EXPERTS];
     for (int e = 0; e < APEX_MAX_EXPERTS; ++e) pos[e] = 1 << 20;
     for (int j = 0; j < ncand[0]; ++j) pos[cand[j]] = j;
-    std::vector<SlotCopy> ordered = copies;
     std::stable_sort(ordered.begin(), ordered.end(), [&](const SlotCopy& a, const SlotCopy& b) { return pos[a.expert] < pos[b.expert]; });
-    for (const auto& c : ordered) {
-      int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
-      if (r != APEX_OK) return r;
-    }
-  } else {
-    for (const auto& c : copies) {
-      int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
-      if (r != APEX_OK) return r;
-    }
+  }
+  for (const auto& c : ordered) {
+    int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+    if (r != APEX_OK) return r;
   }
   ctx->host_stats[layer].prefetch_copies += (int64_t)copies.size();
   ctx->last_copies[layer].insert(ctx->last_copies[layer].end(), copies.begin(), copies.end());
@@ -451,6 +474,7 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   CHECK_LAYER(ctx, layer);
   if (!hpost_dev || !idx_dev || !alpha_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_route_topk: bad argument");
   auto& st = ctx->step[layer];
+  if (st.pending) return fail(ctx, APEX_ESTATE, "the previous expert FFN of this layer has not been completed");
   if (st.predicted && st.B != B) return fail(ctx, APEX_ESTATE, "B differs from apex_predict of this layer-step");
   if (!st.predicted) {  // gate used on its own (no prefetch stage): still one layer-step
     ctx->tables[layer].begin_step();
@@ -464,21 +488,20 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   p.W = ctx->d_Wr + (size_t)layer * N * d;
   p.bias = ctx->has_br[layer] ? ctx->d_br + (size_t)layer * N : nullptr;
   p.x = hpost_dev;
-  p.z_out = ctx->d_zr;
+  p.z_out = ctx->d_zr + (size_t)layer * ctx->cfg.max_batch * N;
   p.q_out = alpha_dev;
   p.pi_out = nullptr;
   p.topk_out = idx_dev;
   p.N = (int)N; p.d = (int)d; p.B = B; p.k = ctx->cfg.k; p.C = ctx->cfg.C;
   p.pi_pred = st.selected ? ctx->d_pi : nullptr;
   p.ncand_pred = st.selected ? ctx->d_ncand : nullptr;
-  p.resident_mask = ctx->tables[layer].resident_mask();
   p.stats = ctx->d_stats + layer;
-  p.mbox_kr = mbox_i32(ctx, ctx->ml.off_kr);
-  p.mbox_seq = &mhdr(ctx)->route_seq;
-  p.seq_value = ++ctx->route_seq;
-  ctx->route_done += (unsigned long long)B;
-  p.done_counter = ctx->d_counters + 1;
-  p.done_target = ctx->route_done;
+  p.mbox_kr = mbox_kr(ctx, layer);
+  p.mbox_seq = mbox_route_seq(ctx, layer);
+  p.seq_value = ++ctx->route_seq[layer];
+  ctx->route_done[layer] += (unsigned long long)B;
+  p.done_counter = ctx->d_counters + 2 + layer;
+  p.done_target = ctx->route_done[layer];
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
   ++ctx->launches;
   st.routed = true;
@@ -487,25 +510,28 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   return APEX_OK;
 }
 
-int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev, int32_t* exec_idx_dev,
-                 float* exec_gate_dev, void* stream) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
+}  // extern "C"
+
+namespace {
+
+// First half of apex_moe_ffn: launches the expert FFN of a layer-step.  B == 1 in exact mode is one
+// launch that also waits, inside the kernel, for experts the host has to fetch on demand; otherwise
+// the launch covers the experts that are resident and ffn_finalize adds further launches.
+int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev, int32_t* exec_idx_dev,
+               float* exec_gate_dev, cudaStream_t cs) {
   auto& st = ctx->step[layer];
   if (!st.routed || st.B != B) return fail(ctx, APEX_ESTATE, "apex_moe_ffn needs apex_route_topk of the same layer-step and B");
   if (!hpost_dev || !y_dev) return fail(ctx, APEX_EINVAL, "null h' or y");
   if (mode != APEX_MODE_EXACT && mode != APEX_MODE_STALL_FREE) return fail(ctx, APEX_EINVAL, "unknown mode");
   if (ctx->cfg.I_shared > 0 && !ctx->shared_dev[layer]) return fail(ctx, APEX_ESTATE, "shared expert not set for this layer");
-  cudaStream_t cs = (cudaStream_t)stream;
   const int N = ctx->cfg.N, k = ctx->cfg.k, C = ctx->cfg.C;
-  auto& tab = ctx->tables[layer];
-
-  FfnParams p{};
+  FfnParams& p = ctx->ffn_params[layer];
+  p = FfnParams{};
   p.hpost = hpost_dev;
   p.y = y_dev;
   p.idx = st.idx_dev;
   p.alpha = st.alpha_dev;
-  p.z_r = ctx->d_zr;
+  p.z_r = ctx->d_zr + (size_t)layer * ctx->cfg.max_batch * N;
   p.exec_idx = exec_idx_dev;
   p.exec_gate = exec_gate_dev;
   p.cache = ctx->d_cache + (size_t)layer * C * ctx->expert_bytes;
@@ -517,90 +543,122 @@ int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int
   p.pair_gate = ctx->d_pair_gate;
   p.pair_expert = ctx->d_pair_expert;
   p.n_pairs = ctx->d_n_pairs;
-  p.mbox_exec = mbox_i32(ctx, ctx->ml.off_exec);
-  p.mbox_seq = &mhdr(ctx)->exec_seq;
+  p.mbox_exec = mbox_exec(ctx, layer);
+  p.mbox_seq = mbox_exec_seq(ctx, layer);
   p.mbox_status = &mhdr(ctx)->status;
-  p.seq_value = ++ctx->exec_seq;
+  p.seq_value = ++ctx->exec_seq[layer];
   p.stats = ctx->d_stats + layer;
-  p.zero_counter = ctx->d_counters + 2;
+  p.zero_counter = ctx->d_counters + 1;
   ctx->zero_done += (unsigned long long)ctx->n_sm;
   p.zero_target = ctx->zero_done;
   p.snap = make_snapshot(ctx, layer);
-  p.run_mask = p.snap.resident_mask;
   p.slot_stride = ctx->expert_bytes;
   p.wait_limit_ns = ctx->cfg.wait_limit_ns;
   p.d = ctx->cfg.d; p.N = N; p.k = k; p.I = ctx->cfg.I; p.I_shared = ctx->cfg.I_shared; p.B = B;
   p.mode = mode; p.norm_topk = ctx->cfg.norm_topk; p.accumulate = 0;
   p.run_shared = ctx->cfg.I_shared > 0 ? 1 : 0;
   p.post_exec = 1;
+  p.demand = ctx->d_demand + (size_t)layer * N;
+  ctx->launch_tag = ctx->launch_tag % 0xfffffeu + 1u;
+  p.demand_tag = ctx->launch_tag;
+  p.demand_in_kernel = (mode == APEX_MODE_EXACT && B == 1) ? 1 : 0;
+  p.run_mask = p.demand_in_kernel ? ~0ull : p.snap.resident_mask;
   if (B > 1) {
     CU_TRY(ctx, launch_ffn_plan(p, cs));
     ++ctx->launches;
   }
   CU_TRY(ctx, launch_ffn(p, ctx->n_sm, cs));
   ++ctx->launches;
+  st.pending = true;
+  st.pend_mode = mode;
+  st.pend_tag = p.demand_tag;
+  st.pend_stream = cs;
+  return APEX_OK;
+}
 
-  // the gate's decision arrives through the mailbox while the first wave runs
-  if (!host_wait_seq(ctx, &mhdr(ctx)->route_seq, ctx->route_seq)) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
-  const int32_t* K_r = mbox_i32(ctx, ctx->ml.off_kr);
-  if (mode == APEX_MODE_EXACT) {
+// Second half: host work that needs the gate's decision (LRU stamps, demand copies, further waves).
+int ffn_finalize(apex_ctx* ctx, int layer) {
+  auto& st = ctx->step[layer];
+  if (!st.pending) return APEX_OK;
+  st.pending = false;
+  const int B = st.B, N = ctx->cfg.N, k = ctx->cfg.k;
+  (void)N;
+  cudaStream_t cs = st.pend_stream;
+  auto& tab = ctx->tables[layer];
+  const FfnParams& p = ctx->ffn_params[layer];
+  if (!host_wait_seq(ctx, mbox_route_seq(ctx, layer), ctx->route_seq[layer])) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
+  const int32_t* K_r = mbox_kr(ctx, layer);
+  if (st.pend_mode == APEX_MODE_EXACT) {
     std::vector<SlotCopy> copies;
     uint64_t need = 0;
     const std::vector<int32_t> slot_expert_before = tab.slot_expert();
     if (!tab.plan_demand(K_r, B, k, &copies, &need)) return fail(ctx, APEX_ESTATE, "no evictable slot");
-    int n_waves = 0;
-    for (const auto& c : copies) n_waves = c.wave > n_waves ? c.wave : n_waves;
-    // The plan above covers every wave; replay it wave by wave so that each launch gets the table
-    // as it stands when that wave runs.
-    std::vector<int32_t> cur_slot_expert = slot_expert_before;
-    SlotSnapshot cur = p.snap;
-    for (int w = 1; w <= n_waves; ++w) {
-      // a victim that an earlier launch of this step may still be reading: order the copy after it
-      bool hazard = false;
-      uint64_t chunk = 0;
-      for (const auto& c : copies)
-        if (c.wave == w) {
-          chunk |= (1ull << c.expert);
-          const int prev = cur_slot_expert[c.slot];
-          if (prev >= 0 && ((need >> prev) & 1)) hazard = true;
-        }
-      if (hazard) {
-        CU_TRY(ctx, cudaEventRecord(ctx->ev_wave, cs));
-        CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_stream, ctx->ev_wave, 0));
+    if (p.demand_in_kernel) {
+      // the running kernel waits for these experts: copy, then publish (tag, slot)
+      for (const auto& c : copies) {
+        const int prev = slot_expert_before[c.slot];
+        if (c.wave != 1 || (prev >= 0 && ((need >> prev) & 1))) return fail(ctx, APEX_ESTATE, "demand plan would evict an expert in use");
+        int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+        if (r != APEX_OK) return r;
+        r = stream_write32(ctx, ctx->cur_copy_stream, ctx->d_demand + (size_t)layer * ctx->cfg.N + c.expert,
+                           (st.pend_tag << 8) | (uint32_t)c.slot);
+        if (r != APEX_OK) return r;
       }
-      for (const auto& c : copies)
-        if (c.wave == w) {
-          int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
-          if (r != APEX_OK) return r;
-          const int prev = cur_slot_expert[c.slot];
-          if (prev >= 0) {
-            cur.expert_slot[prev] = -1;
-            cur.resident_mask &= ~(1ull << prev);
+    } else {
+      int n_waves = 0;
+      for (const auto& c : copies) n_waves = c.wave > n_waves ? c.wave : n_waves;
+      // The plan above covers every wave; replay it wave by wave so that each launch gets the table
+      // as it stands when that wave runs.
+      std::vector<int32_t> cur_slot_expert = slot_expert_before;
+      SlotSnapshot cur = p.snap;
+      for (int w = 1; w <= n_waves; ++w) {
+        // a victim that an earlier launch of this step may still be reading: order the copy after it
+        bool hazard = false;
+        uint64_t chunk = 0;
+        for (const auto& c : copies)
+          if (c.wave == w) {
+            chunk |= (1ull << c.expert);
+            const int prev = cur_slot_expert[c.slot];
+            if (prev >= 0 && ((need >> prev) & 1)) hazard = true;
           }
-          cur_slot_expert[c.slot] = c.expert;
-          cur.expert_slot[c.expert] = (int8_t)c.slot;
-          cur.need_gen[c.expert] = ctx->slot_gen[layer][c.slot];
-          cur.resident_mask |= (1ull << c.expert);
+        if (hazard) {
+          CU_TRY(ctx, cudaEventRecord(ctx->ev_wave, cs));
+          CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_stream, ctx->ev_wave, 0));
         }
-      FfnParams q = p;
-      q.snap = cur;
-      q.run_mask = chunk;
-      q.accumulate = 1;
-      q.run_shared = 0;
-      q.post_exec = 0;
-      if (B > 1) {
-        CU_TRY(ctx, launch_ffn_plan(q, cs));
+        for (const auto& c : copies)
+          if (c.wave == w) {
+            int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+            if (r != APEX_OK) return r;
+            const int prev = cur_slot_expert[c.slot];
+            if (prev >= 0) {
+              cur.expert_slot[prev] = -1;
+              cur.resident_mask &= ~(1ull << prev);
+            }
+            cur_slot_expert[c.slot] = c.expert;
+            cur.expert_slot[c.expert] = (int8_t)c.slot;
+            cur.need_gen[c.expert] = ctx->slot_gen[layer][c.slot];
+            cur.resident_mask |= (1ull << c.expert);
+          }
+        FfnParams q = p;
+        q.snap = cur;
+        q.run_mask = chunk;
+        q.accumulate = 1;
+        q.run_shared = 0;
+        q.post_exec = 0;
+        if (B > 1) {
+          CU_TRY(ctx, launch_ffn_plan(q, cs));
+          ++ctx->launches;
+        }
+        CU_TRY(ctx, launch_ffn(q, ctx->n_sm, cs));
         ++ctx->launches;
+        ctx->host_stats[layer].extra_waves += 1;
       }
-      CU_TRY(ctx, launch_ffn(q, ctx->n_sm, cs));
-      ++ctx->launches;
-      ctx->host_stats[layer].extra_waves += 1;
     }
     ctx->host_stats[layer].demand_copies += (int64_t)copies.size();
     ctx->last_copies[layer].insert(ctx->last_copies[layer].end(), copies.begin(), copies.end());
   } else {
-    if (!host_wait_seq(ctx, &mhdr(ctx)->exec_seq, ctx->exec_seq)) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: execution sets did not arrive");
-    const int32_t* ex = mbox_i32(ctx, ctx->ml.off_exec);
+    if (!host_wait_seq(ctx, mbox_exec_seq(ctx, layer), ctx->exec_seq[layer])) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: execution sets did not arrive");
+    const int32_t* ex = mbox_exec(ctx, layer);
     for (int i = 0; i < B * k; ++i) tab.touch(ex[i]);
   }
   st.routed = false;  // the layer-step is complete
@@ -609,22 +667,43 @@ int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int
   return check_device_status(ctx);
 }
 
+}  // namespace
+
+extern "C" {
+
+int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev, int32_t* exec_idx_dev,
+                 float* exec_gate_dev, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  int r = ffn_launch(ctx, layer, mode, hpost_dev, B, y_dev, exec_idx_dev, exec_gate_dev, (cudaStream_t)stream);
+  if (r != APEX_OK) return r;
+  return ffn_finalize(ctx, layer);
+}
+
+// Pipelined over layers: the host work that needs the gate's decision of layer l-1 (LRU stamps,
+// demand copies) is done after the kernels of layer l have been queued, so that on the hit path
+// the GPU never waits for the host.
 int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev, int B, float tau, int mode, float* y_dev,
                       void* stream) {
   CHECK_CTX(ctx);
   if (!h_dev || !hpost_dev || !y_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_decode_token: bad argument");
   const size_t step = (size_t)B * ctx->cfg.d;
+  const size_t MB = ctx->cfg.max_batch, k = ctx->cfg.k, N = ctx->cfg.N;
+  int r;
   for (int l = 0; l < ctx->cfg.L; ++l) {
-    int r;
+    int32_t* idx = ctx->d_idx + (size_t)l * MB * k;
+    float* alpha = ctx->d_alpha + (size_t)l * MB * N;
     if ((r = apex_predict(ctx, l, h_dev + l * step, B, stream)) != APEX_OK) return r;
     if ((r = apex_select_candidates(ctx, l, B, tau, ctx->d_cand, ctx->d_cand_ncand, stream)) != APEX_OK) return r;
-    if ((r = apex_prefetch(ctx, l, B, nullptr)) != APEX_OK) return r;
     if ((r = apex_attention_standin(ctx, l, stream)) != APEX_OK) return r;
-    if ((r = apex_route_topk(ctx, l, hpost_dev + l * step, B, ctx->d_idx, ctx->d_alpha, stream)) != APEX_OK) return r;
-    if ((r = apex_moe_ffn(ctx, l, mode, hpost_dev + l * step, B, y_dev + l * step, ctx->d_exec_idx, ctx->d_exec_gate, stream)) != APEX_OK)
+    if ((r = apex_route_topk(ctx, l, hpost_dev + l * step, B, idx, alpha, stream)) != APEX_OK) return r;
+    if (l > 0 && (r = ffn_finalize(ctx, l - 1)) != APEX_OK) return r;
+    if ((r = apex_prefetch(ctx, l, B, nullptr)) != APEX_OK) return r;
+    if ((r = ffn_launch(ctx, l, mode, hpost_dev + l * step, B, y_dev + l * step, ctx->d_exec_idx, ctx->d_exec_gate,
+                        (cudaStream_t)stream)) != APEX_OK)
       return r;
   }
-  return APEX_OK;
+  return ffn_finalize(ctx, ctx->cfg.L - 1);
 }
 
 int apex_decode_token_host(apex_ctx* ctx, const float* h_host, const float* hpost_host, int B, float tau, int mode,

@@ -14,14 +14,15 @@ namespace apex {
 // ---- mapped host mailbox: the kernels post small decision records here so that the host can
 // plan copies without a stream synchronisation.  One per context; sequence numbers only grow.
 struct MailboxHeader {
-  volatile uint32_t sel_seq;    // written by the candidate-selection kernel, after the lists
-  volatile uint32_t route_seq;  // written by the gate kernel, after K_r
-  volatile uint32_t exec_seq;   // written by the plan step of the FFN, after the execution sets
-  volatile uint32_t status;     // sticky device status (0 ok, 1 wait ran out)
+  volatile uint32_t sel_seq;  // written by the candidate-selection kernel, after the lists
+  volatile uint32_t status;   // sticky device status (0 ok, 1 a bounded wait ran out)
+  uint32_t pad[2];
 };
 
+// Byte offsets inside the mailbox.  Per layer: route_seq[l] is written by the gate kernel after
+// K_r of that layer, exec_seq[l] by the FFN's plan step after the execution sets.
 struct MailboxLayout {
-  size_t off_ncand, off_cand, off_kr, off_exec, bytes;
+  size_t off_route_seq, off_exec_seq, off_ncand, off_cand, off_kr, off_exec, kr_stride, bytes;
 };
 
 // Device-side counters of one layer (S9), accumulated with 64-bit atomics.
@@ -50,7 +51,6 @@ struct RouterParams {
   // gate-kernel epilogue (S9 metrics + mailbox); all null/0 for the prefetch router
   const int32_t* pi_pred;     // [B][N] ranking of the prefetch router for this step, or null
   const int32_t* ncand_pred;  // [B]
-  unsigned long long resident_mask;
   DevStats* stats;
   int32_t* mbox_kr;                 // mapped host [B][k]
   volatile uint32_t* mbox_seq;      // mapped host
@@ -106,6 +106,9 @@ struct FfnParams {
   unsigned long long* zero_counter;
   unsigned long long zero_target;
   unsigned long long run_mask;  // experts this launch executes
+  const uint32_t* demand;       // [N] per layer: (tag << 8 | slot), published by the host after a demand copy
+  uint32_t demand_tag;          // tag of this launch
+  int demand_in_kernel;         // 1: a routed expert without a slot is waited for inside the kernel
   SlotSnapshot snap;
   size_t slot_stride;
   long long wait_limit_ns;
@@ -148,25 +151,32 @@ struct apex_ctx {
   std::vector<uint8_t> has_br, has_bp, has_cdf;
   uint8_t* d_cache = nullptr;     // [L][C][expert_bytes]
   uint32_t* d_slot_ready = nullptr;  // [L][C]
-  float *d_zp = nullptr, *d_qp = nullptr, *d_zr = nullptr;  // [maxB][N]
+  float *d_zp = nullptr, *d_qp = nullptr;  // [maxB][N]
+  float* d_zr = nullptr;                   // [L][maxB][N]
+  uint32_t* d_demand = nullptr;            // [L][N]
   int32_t *d_pi = nullptr, *d_ncand = nullptr;              // [maxB][N], [maxB]
   apex::DevStats* d_stats = nullptr;                        // [L]
-  unsigned long long* d_counters = nullptr;                 // [4]: select done, route done, zero, spare
+  unsigned long long* d_counters = nullptr;                 // [2 + L]: select done, zero, route done per layer
   int32_t *d_plan_exec_idx = nullptr, *d_pair_tok = nullptr, *d_pair_expert = nullptr, *d_n_pairs = nullptr;
   float *d_plan_exec_gate = nullptr, *d_pair_gate = nullptr;
   uint8_t* d_attn = nullptr;
   size_t attn_bytes = 0, attn_layers = 1;
   float* d_attn_sink = nullptr;
   // scratch for apex_decode_token
-  int32_t *d_cand = nullptr, *d_cand_ncand = nullptr, *d_idx = nullptr, *d_exec_idx = nullptr;
-  float *d_alpha = nullptr, *d_exec_gate = nullptr;
+  int32_t *d_cand = nullptr, *d_cand_ncand = nullptr, *d_exec_idx = nullptr;
+  float* d_exec_gate = nullptr;
+  int32_t* d_idx = nullptr;  // [L][maxB][k]
+  float* d_alpha = nullptr;  // [L][maxB][N]
   float *d_h_stage = nullptr, *d_hp_stage = nullptr, *d_y_stage = nullptr;  // [L][maxB][d] for the host variant
 
   // mapped host mailbox
   uint8_t* mbox = nullptr;
   apex::MailboxLayout ml{};
-  uint32_t sel_seq = 0, route_seq = 0, exec_seq = 0;
-  unsigned long long sel_done = 0, route_done = 0, zero_done = 0;
+  uint32_t sel_seq = 0;
+  std::vector<uint32_t> route_seq, exec_seq;      // per layer, last value asked for
+  std::vector<unsigned long long> route_done;     // per layer
+  unsigned long long sel_done = 0, zero_done = 0;
+  uint32_t launch_tag = 0;
   uint32_t* gen_src = nullptr;  // pinned ring of flag values for the ready-flag copies
   size_t gen_src_pos = 0, gen_src_len = 0;
 
@@ -186,8 +196,14 @@ struct apex_ctx {
     bool predicted = false, selected = false, prefetched = false, routed = false;
     const int32_t* idx_dev = nullptr;
     const float* alpha_dev = nullptr;
+    // an FFN launch whose host-side completion (LRU touch, demand copies) is still due
+    bool pending = false;
+    int pend_mode = 0;
+    uint32_t pend_tag = 0;
+    cudaStream_t pend_stream = nullptr;
   };
   std::vector<StepState> step;
+  std::vector<apex::FfnParams> ffn_params;  // [L] parameters of the last FFN launch of each layer
 
   cudaStream_t copy_stream = nullptr;   // own
   cudaStream_t cur_copy_stream = nullptr;

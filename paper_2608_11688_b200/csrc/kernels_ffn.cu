@@ -235,7 +235,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   __shared__ int s_off[APEX_MAX_EXPERTS + 2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
   const int N = p.N, k = p.k, B = p.B;
-  int my_subst = 0;
+  int my_subst = 0, my_hits = 0;
   for (int b = warp; b < B; b += nwarp) {
     const TokenLoads tl = load_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode, lane);
     const TokenPlan tp = plan_token(tl, p.mode, p.norm_topk, p.snap.resident_mask, lane);
@@ -254,10 +254,12 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
         if (p.exec_gate) p.exec_gate[(size_t)b * k + pos] = tp.g1;
       }
       my_subst += __popcll(tp.exec_mask & ~tp.kr_mask);
+      my_hits += __popcll(tp.kr_mask & p.snap.resident_mask);
     }
     if (lane == 0) s_exec[b] = tp.exec_mask;
   }
   if (p.post_exec && lane == 0 && my_subst && p.stats) atomicAdd(&p.stats->substitutions, (unsigned long long)my_subst);
+  if (p.post_exec && lane == 0 && my_hits && p.stats) atomicAdd(&p.stats->hits_R, (unsigned long long)my_hits);
   __syncthreads();
   const int e = threadIdx.x;
   if (e < N) {
@@ -363,18 +365,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   }
   if (tid < NS) mbar_init(&s_full[tid], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-  if (!p.accumulate) {
-    const size_t n4 = (size_t)B * d / 4;
-    const size_t per = (n4 + G - 1) / G;
-    const size_t lo = per * cta, hi = lo + per < n4 ? lo + per : n4;
-    float4* y4 = reinterpret_cast<float4*>(p.y);
-    for (size_t i = lo + tid; i < hi; i += kFfnThreads) y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  __syncthreads();
-  if (!p.accumulate && tid == 0) {
-    __threadfence();
-    atomicAdd(p.zero_counter, 1ull);
-  }
+  __syncthreads();  // barriers initialised
   float hreg[H_REGS ? NCH * 8 : 1];
   int cur_tok = -1;
   if (H_REGS && B == 1) {  // h' is an input of the gate kernel as well: complete long before this kernel
@@ -390,6 +381,19 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   pdl_wait();               // the gate's outputs (K_r, alpha, z_r) are complete from here on
   pdl_launch_dependents();  // the next kernel may start its own prologue
   if (tid == 0) TL(4);
+  // y is zeroed only now: a preceding launch that still adds to the same buffer has completed
+  if (!p.accumulate) {
+    const size_t n4 = (size_t)B * d / 4;
+    const size_t per = (n4 + G - 1) / G;
+    const size_t lo = per * cta, hi = lo + per < n4 ? lo + per : n4;
+    float4* y4 = reinterpret_cast<float4*>(p.y);
+    for (size_t i = lo + tid; i < hi; i += kFfnThreads) y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  if (!p.accumulate) __syncthreads();
+  if (!p.accumulate && tid == 0) {
+    __threadfence();
+    atomicAdd(p.zero_counter, 1ull);
+  }
 
   // ---- every global load of the prologue is issued before the first use, so the latencies overlap.
   // Slot-ready flags: lanes own experts lane and lane+32.  The flag is written by the copy engine
@@ -442,6 +446,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   bool zero_seen = p.accumulate != 0;
   bool ok = true;
   unsigned long long waited = 0;
+  int dm_e = -1, dm_slot = -1;  // last expert this lane had to wait for on demand
 
   auto poll_zeroed = [&](bool spin) {  // y must be all zero before anybody adds to it
     if (zero_seen) return;
@@ -485,12 +490,37 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     }
     const uint8_t* base;
     if (e < N) {
-      const int slot = p.snap.expert_slot[e];
-      if (slot < 0) {  // the host never asks for an expert without a slot; refuse rather than read out of range
-        ok = false;
-        return;
-      }
-      if (!((ready_mask >> e) & 1)) {
+      int slot = p.snap.expert_slot[e];
+      if (slot < 0) {
+        // not resident when the kernel was launched: the host fetches it on demand and publishes
+        // (tag, slot) after the copy -- "asynchronous miss correction" inside one launch
+        if (!p.demand_in_kernel) {  // refuse rather than read out of range
+          ok = false;
+          return;
+        }
+        if (e == dm_e) {
+          slot = dm_slot;
+        } else {
+          const uint32_t* w = p.demand + e;
+          uint32_t v = ld_acquire_sys(w);
+          if ((v >> 8) != p.demand_tag) {
+            const unsigned long long t0 = globaltimer_ns();
+            while (((v = ld_acquire_sys(w)) >> 8) != p.demand_tag) {
+              if ((long long)(globaltimer_ns() - t0) > p.wait_limit_ns) {
+                ok = false;
+                break;
+              }
+              __nanosleep(128);
+            }
+            waited += globaltimer_ns() - t0;
+            if (!ok) return;
+          }
+          slot = (int)(v & 0xffu);
+          dm_e = e;
+          dm_slot = slot;
+          asm volatile("fence.proxy.async;" ::: "memory");
+        }
+      } else if (!((ready_mask >> e) & 1)) {
         const uint32_t need = p.snap.need_gen[e];
         const uint32_t* flag = p.slot_ready + slot;
         const unsigned long long t0 = globaltimer_ns();
@@ -530,6 +560,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     if (lane == 0 && p.stats) {
       const int ns = __popcll(tp1.exec_mask & ~tp1.kr_mask);
       if (ns) atomicAdd(&p.stats->substitutions, (unsigned long long)ns);
+      atomicAdd(&p.stats->hits_R, (unsigned long long)__popcll(tp1.kr_mask & p.snap.resident_mask));
     }
     __threadfence_system();
     __syncwarp();

@@ -34,7 +34,12 @@ __device__ __forceinline__ int warp_max_int(int v) {
 // expert; the logits are gathered in the leader CTA's shared memory through distributed shared
 // memory, and the leader's first warp does softmax, ranking, top-k and (for the gate) the
 // per-step metrics of Eq. (2)-(3).
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
+  pdl_wait();               // everything queued before this kernel is complete
+  pdl_launch_dependents();  // the next kernel may begin its own prologue
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned crank = cluster.block_rank();
   const int b = blockIdx.y;
@@ -104,8 +109,6 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
   if (in0) p.mbox_kr[(size_t)b * k + r0] = e0;
   if (in1) p.mbox_kr[(size_t)b * k + r1] = e1;
   if (p.stats) {
-    int hitsR = __popc(__ballot_sync(0xffffffffu, in0 && ((p.resident_mask >> e0) & 1))) +
-                __popc(__ballot_sync(0xffffffffu, in1 && ((p.resident_mask >> e1) & 1)));
     int dstar = 0, hitsP = 0, have_pred = 0;
     if (p.pi_pred) {
       have_pred = 1;
@@ -119,7 +122,6 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
     }
     if (lane == 0) {
       atomicAdd(&p.stats->routed, (unsigned long long)k);
-      atomicAdd(&p.stats->hits_R, (unsigned long long)hitsR);
       if (have_pred) {
         atomicAdd(&p.stats->sum_delta_star, (unsigned long long)dstar);
         atomicAdd(&p.stats->hits_P, (unsigned long long)hitsP);
@@ -149,13 +151,15 @@ cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
   cfg.blockDim = dim3(256, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = s;
-  cudaLaunchAttribute attr[1];
+  cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = csize;
   attr[0].val.clusterDim.y = 1;
   attr[0].val.clusterDim.z = 1;
+  attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
-  cfg.numAttrs = 1;
+  cfg.numAttrs = 2;
   return cudaLaunchKernelEx(&cfg, router_kernel, q);
 }
 
@@ -163,6 +167,8 @@ cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
 // s = w.x, delta_hat = first delta with theta_delta - s >= logit(tau)  (Eq. (8), (9) in the logit
 // domain), capped to C - k; K_p = first k + delta_hat experts of E (Eq. (1)).
 __global__ void __launch_bounds__(128) select_kernel(const SelectParams p) {
+  pdl_wait();
+  pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.x * (blockDim.x >> 5) + warp;
   if (b >= p.B) return;
@@ -225,13 +231,23 @@ __global__ void __launch_bounds__(128) select_kernel(const SelectParams p) {
 
 cudaError_t launch_select(const SelectParams& p, cudaStream_t s) {
   const int wpb = 4;
-  select_kernel<<<(p.B + wpb - 1) / wpb, wpb * 32, 0, s>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3((p.B + wpb - 1) / wpb, 1, 1);
+  cfg.blockDim = dim3(wpb * 32, 1, 1);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, select_kernel, p);
 }
 
 // Streams attn_bytes once (the weight and KV bytes an attention block of this shape reads).  The
 // xor of everything read is stored only if it equals one fixed pattern, which keeps the loads live.
 __global__ void __launch_bounds__(512) attention_standin_kernel(const AttnParams p) {
+  pdl_wait();
+  pdl_launch_dependents();
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   uint4 a = make_uint4(0, 0, 0, 0);
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < p.n_vec; i += stride) {
@@ -245,8 +261,16 @@ __global__ void __launch_bounds__(512) attention_standin_kernel(const AttnParams
 }
 
 cudaError_t launch_attention(const AttnParams& p, int n_sm, cudaStream_t s) {
-  attention_standin_kernel<<<n_sm * 2, 512, 0, s>>>(p);
-  return cudaGetLastError();
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_sm * 2, 1, 1);
+  cfg.blockDim = dim3(512, 1, 1);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, attention_standin_kernel, p);
 }
 
 }  // namespace apex

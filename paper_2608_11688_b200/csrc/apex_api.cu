@@ -45,9 +45,7 @@ cudaError_t dev_alloc(T** p, size_t n) {
 
 MailboxHeader* mhdr(apex_ctx* ctx) { return reinterpret_cast<MailboxHeader*>(ctx->mbox); }
 int32_t* mbox_i32(apex_ctx* ctx, size_t off) { return reinterpret_cast<int32_t*>(ctx->mbox + off); }
-volatile uint32_t* mbox_route_seq(apex_ctx* ctx, int l) {
-  return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_route_seq) + l;
-}
+volatile uint32_t* mbox_sel_rec(apex_ctx* ctx) { return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_sel_rec); }
 volatile uint32_t* mbox_exec_seq(apex_ctx* ctx, int l) {
   return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_exec_seq) + l;
 }
@@ -202,8 +200,8 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(dev_alloc(&ctx->d_ncand, MB));
   CR(dev_alloc(&ctx->d_stats, L));
   CR(cudaMemset(ctx->d_stats, 0, L * sizeof(DevStats)));
-  CR(dev_alloc(&ctx->d_counters, 2 + L));
-  CR(cudaMemset(ctx->d_counters, 0, (2 + L) * sizeof(unsigned long long)));
+  CR(dev_alloc(&ctx->d_counters, 2));
+  CR(cudaMemset(ctx->d_counters, 0, 2 * sizeof(unsigned long long)));
   const size_t max_pairs = MB * (k + 1);
   CR(dev_alloc(&ctx->d_plan_exec_idx, MB * k));
   CR(dev_alloc(&ctx->d_plan_exec_gate, MB * k));
@@ -226,18 +224,16 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   // mapped mailbox
   MailboxLayout& ml = ctx->ml;
   size_t off = sizeof(MailboxHeader);
-  ml.off_route_seq = off; off += L * sizeof(uint32_t);
   ml.off_exec_seq = off;  off += L * sizeof(uint32_t);
   off = (off + 15) & ~(size_t)15;
+  ml.off_sel_rec = off;   off += 16;
   ml.off_ncand = off; off += MB * sizeof(int32_t);
   ml.off_cand = off;  off += MB * C * sizeof(int32_t);
   ml.kr_stride = MB * k * sizeof(int32_t);
   ml.off_kr = off;    off += L * ml.kr_stride;
   ml.off_exec = off;  off += L * ml.kr_stride;
   ml.bytes = off;
-  ctx->route_seq.assign(L, 0u);
   ctx->exec_seq.assign(L, 0u);
-  ctx->route_done.assign(L, 0ull);
   CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->mbox), ml.bytes, cudaHostAllocMapped | cudaHostAllocPortable));
   memset(ctx->mbox, 0, ml.bytes);
   ctx->gen_src_len = 1 << 16;
@@ -364,9 +360,11 @@ int apex_pack_expert(const void* gate, const void* up, const void* down, int d, 
 
 // ---------------------------------------------------------------------------------------------
 
-int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stream) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
+}  // extern "C"
+
+namespace {
+
+int begin_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, RouterParams* p) {
   if (!h_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_predict: bad h or B");
   const size_t N = ctx->cfg.N, d = ctx->cfg.d;
   if (ctx->step[layer].pending) return fail(ctx, APEX_ESTATE, "the previous expert FFN of this layer has not been completed");
@@ -374,15 +372,74 @@ int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stre
   ctx->last_copies[layer].clear();
   ctx->step[layer] = apex_ctx::StepState{};
   ctx->step[layer].B = B;
-  RouterParams p{};
-  p.W = ctx->d_Wp + (size_t)layer * N * d;
-  p.bias = ctx->has_bp[layer] ? ctx->d_bp + (size_t)layer * N : nullptr;
-  p.x = h_dev;
-  p.z_out = ctx->d_zp;
-  p.q_out = ctx->d_qp;
-  p.pi_out = ctx->d_pi;
-  p.topk_out = nullptr;
-  p.N = (int)N; p.d = (int)d; p.B = B; p.k = ctx->cfg.k; p.C = ctx->cfg.C;
+  *p = RouterParams{};
+  p->W = ctx->d_Wp + (size_t)layer * N * d;
+  p->bias = ctx->has_bp[layer] ? ctx->d_bp + (size_t)layer * N : nullptr;
+  p->x = h_dev;
+  p->z_out = ctx->d_zp;
+  p->q_out = ctx->d_qp;
+  p->pi_out = ctx->d_pi;
+  p->topk_out = nullptr;
+  p->N = (int)N; p->d = (int)d; p->B = B; p->k = ctx->cfg.k; p->C = ctx->cfg.C;
+  return APEX_OK;
+}
+
+int fill_select(apex_ctx* ctx, int layer, int B, float tau, int32_t* cand_dev, int32_t* ncand_dev, SelectParams* p) {
+  if (!cand_dev || !ncand_dev) return fail(ctx, APEX_EINVAL, "null output");
+  if (!ctx->has_cdf[layer]) return fail(ctx, APEX_ESTATE, "no confidence model set for this layer");
+  if (!(tau == tau)) return fail(ctx, APEX_EINVAL, "tau is NaN");
+  const int N = ctx->cfg.N, k = ctx->cfg.k;
+  *p = SelectParams{};
+  p->q = ctx->d_qp;
+  p->pi = ctx->d_pi;
+  p->w = ctx->d_w + (size_t)layer * N;
+  p->theta = ctx->d_theta + (size_t)layer * (N - k + 1);
+  p->cand_out = cand_dev;
+  p->ncand_out = ncand_dev;
+  p->ncand_keep = ctx->d_ncand;
+  p->mbox_cand = mbox_i32(ctx, ctx->ml.off_cand);
+  p->mbox_ncand = mbox_i32(ctx, ctx->ml.off_ncand);
+  p->mbox_seq = &mhdr(ctx)->sel_seq;
+  p->mbox_rec = const_cast<uint32_t*>(mbox_sel_rec(ctx));
+  p->seq_value = ++ctx->sel_seq;
+  if (B > 1) ctx->sel_done += (unsigned long long)B;
+  p->done_counter = ctx->d_counters + 0;
+  p->done_target = ctx->sel_done;
+  p->stats = ctx->d_stats + layer;
+  p->force = tau <= 0.f ? 1 : (tau >= 1.f ? 2 : 0);
+  p->t_tau = p->force ? 0.f : (float)std::log((double)tau / (1.0 - (double)tau));
+  p->N = N; p->k = k; p->C = ctx->cfg.C; p->B = B;
+  return APEX_OK;
+}
+
+// S1-S3 in one launch (used by apex_decode_token): the leader warp of the prefetch-router kernel
+// goes on with the budget selection of its token.
+int predict_select_fused(apex_ctx* ctx, int layer, const float* h_dev, int B, float tau, int32_t* cand_dev,
+                         int32_t* ncand_dev, cudaStream_t cs) {
+  RouterParams p;
+  int r = begin_predict(ctx, layer, h_dev, B, &p);
+  if (r != APEX_OK) return r;
+  if ((r = fill_select(ctx, layer, B, tau, cand_dev, ncand_dev, &p.sel)) != APEX_OK) return r;
+  p.fuse_select = 1;
+  CU_TRY(ctx, launch_router(p, cs));
+  ++ctx->launches;
+  ctx->pred_stream = cs;
+  ctx->step[layer].predicted = true;
+  ctx->step[layer].selected = true;
+  ctx->host_stats[layer].layer_steps += 1;
+  return APEX_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  RouterParams p;
+  int r = begin_predict(ctx, layer, h_dev, B, &p);
+  if (r != APEX_OK) return r;
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
   ++ctx->launches;
   ctx->pred_stream = (cudaStream_t)stream;
@@ -396,29 +453,9 @@ int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* 
   CHECK_LAYER(ctx, layer);
   auto& st = ctx->step[layer];
   if (!st.predicted || st.B != B) return fail(ctx, APEX_ESTATE, "apex_select_candidates needs apex_predict of the same layer-step and B");
-  if (!cand_dev || !ncand_dev) return fail(ctx, APEX_EINVAL, "null output");
-  if (!ctx->has_cdf[layer]) return fail(ctx, APEX_ESTATE, "no confidence model set for this layer");
-  if (!(tau == tau)) return fail(ctx, APEX_EINVAL, "tau is NaN");
-  const int N = ctx->cfg.N, k = ctx->cfg.k;
-  SelectParams p{};
-  p.q = ctx->d_qp;
-  p.pi = ctx->d_pi;
-  p.w = ctx->d_w + (size_t)layer * N;
-  p.theta = ctx->d_theta + (size_t)layer * (N - k + 1);
-  p.cand_out = cand_dev;
-  p.ncand_out = ncand_dev;
-  p.ncand_keep = ctx->d_ncand;
-  p.mbox_cand = mbox_i32(ctx, ctx->ml.off_cand);
-  p.mbox_ncand = mbox_i32(ctx, ctx->ml.off_ncand);
-  p.mbox_seq = &mhdr(ctx)->sel_seq;
-  p.seq_value = ++ctx->sel_seq;
-  ctx->sel_done += (unsigned long long)B;
-  p.done_counter = ctx->d_counters + 0;
-  p.done_target = ctx->sel_done;
-  p.stats = ctx->d_stats + layer;
-  p.force = tau <= 0.f ? 1 : (tau >= 1.f ? 2 : 0);
-  p.t_tau = p.force ? 0.f : (float)std::log((double)tau / (1.0 - (double)tau));
-  p.N = N; p.k = k; p.C = ctx->cfg.C; p.B = B;
+  SelectParams p;
+  int r = fill_select(ctx, layer, B, tau, cand_dev, ncand_dev, &p);
+  if (r != APEX_OK) return r;
   CU_TRY(ctx, launch_select(p, (cudaStream_t)stream));
   ++ctx->launches;
   st.selected = true;
@@ -432,20 +469,42 @@ int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream) {
   if (!st.selected || st.B != B) return fail(ctx, APEX_ESTATE, "apex_prefetch needs apex_select_candidates of the same layer-step and B");
   if (st.prefetched) return fail(ctx, APEX_ESTATE, "apex_prefetch called twice in one layer-step");
   ctx->cur_copy_stream = copy_stream ? (cudaStream_t)copy_stream : ctx->copy_stream;
-  if (!host_wait_seq(ctx, &mhdr(ctx)->sel_seq, ctx->sel_seq))
-    return fail(ctx, APEX_ETIMEOUT, "apex_prefetch: candidate lists did not arrive");
   const int C = ctx->cfg.C;
   const int32_t* ncand = mbox_i32(ctx, ctx->ml.off_ncand);
   const int32_t* cand = mbox_i32(ctx, ctx->ml.off_cand);
   std::vector<SlotCopy> copies;
-  if (!ctx->tables[layer].plan_prefetch(cand, ncand, B, C, &copies)) return fail(ctx, APEX_ESTATE, "no evictable slot");
-  // issue most likely first: order of appearance in the first token's ranked list, others after
-  std::vector<SlotCopy> ordered = copies;
-  if (B == 1 && copies.size() > 1) {
+  std::vector<SlotCopy> ordered;
+  if (B == 1) {
+    // one 16-byte record {mask lo, mask hi, ncand, seq}; the ranked list beside it is advisory
+    volatile uint32_t* rec = mbox_sel_rec(ctx);
+    if (!host_wait_seq(ctx, rec + 3, ctx->sel_seq)) return fail(ctx, APEX_ETIMEOUT, "apex_prefetch: candidate set did not arrive");
+    const uint64_t mask = ((uint64_t)rec[1] << 32) | rec[0];
+    const int n = (int)rec[2];
+    int32_t list[APEX_MAX_EXPERTS];
+    int m = 0;
+    for (int e = 0; e < ctx->cfg.N; ++e)
+      if ((mask >> e) & 1) list[m++] = e;
+    if (m != n || n > C) return fail(ctx, APEX_ESTATE, "candidate record is inconsistent");
+    int32_t nn = n;
+    if (!ctx->tables[layer].plan_prefetch(list, &nn, 1, APEX_MAX_EXPERTS, &copies)) return fail(ctx, APEX_ESTATE, "no evictable slot");
+    ordered = copies;
+    // issue most likely first if the ranked list (written without a fence) is the same set
     int pos[APEX_MAX_EXPERTS];
-    for (int e = 0; e < APEX_MAX_EXPERTS; ++e) pos[e] = 1 << 20;
-    for (int j = 0; j < ncand[0]; ++j) pos[cand[j]] = j;
-    std::stable_sort(ordered.begin(), ordered.end(), [&](const SlotCopy& a, const SlotCopy& b) { return pos[a.expert] < pos[b.expert]; });
+    for (int e = 0; e < APEX_MAX_EXPERTS; ++e) pos[e] = -1;
+    uint64_t seen = 0;
+    bool valid = true;
+    for (int j = 0; j < n && valid; ++j) {
+      const int e = cand[j];
+      if (e < 0 || e >= ctx->cfg.N || ((seen >> e) & 1) || !((mask >> e) & 1)) valid = false;
+      else { seen |= 1ull << e; pos[e] = j; }
+    }
+    if (valid && copies.size() > 1)
+      std::stable_sort(ordered.begin(), ordered.end(), [&](const SlotCopy& a, const SlotCopy& b) { return pos[a.expert] < pos[b.expert]; });
+  } else {
+    if (!host_wait_seq(ctx, &mhdr(ctx)->sel_seq, ctx->sel_seq))
+      return fail(ctx, APEX_ETIMEOUT, "apex_prefetch: candidate lists did not arrive");
+    if (!ctx->tables[layer].plan_prefetch(cand, ncand, B, C, &copies)) return fail(ctx, APEX_ESTATE, "no evictable slot");
+    ordered = copies;
   }
   for (const auto& c : ordered) {
     int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
@@ -496,12 +555,6 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   p.pi_pred = st.selected ? ctx->d_pi : nullptr;
   p.ncand_pred = st.selected ? ctx->d_ncand : nullptr;
   p.stats = ctx->d_stats + layer;
-  p.mbox_kr = mbox_kr(ctx, layer);
-  p.mbox_seq = mbox_route_seq(ctx, layer);
-  p.seq_value = ++ctx->route_seq[layer];
-  ctx->route_done[layer] += (unsigned long long)B;
-  p.done_counter = ctx->d_counters + 2 + layer;
-  p.done_target = ctx->route_done[layer];
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
   ++ctx->launches;
   st.routed = true;
@@ -544,6 +597,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.pair_expert = ctx->d_pair_expert;
   p.n_pairs = ctx->d_n_pairs;
   p.mbox_exec = mbox_exec(ctx, layer);
+  p.mbox_kr = mbox_kr(ctx, layer);
   p.mbox_seq = mbox_exec_seq(ctx, layer);
   p.mbox_status = &mhdr(ctx)->status;
   p.seq_value = ++ctx->exec_seq[layer];
@@ -586,7 +640,8 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
   cudaStream_t cs = st.pend_stream;
   auto& tab = ctx->tables[layer];
   const FfnParams& p = ctx->ffn_params[layer];
-  if (!host_wait_seq(ctx, mbox_route_seq(ctx, layer), ctx->route_seq[layer])) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
+  // the FFN's plan step posts the routed and the execution sets of this layer-step
+  if (!host_wait_seq(ctx, mbox_exec_seq(ctx, layer), ctx->exec_seq[layer])) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
   const int32_t* K_r = mbox_kr(ctx, layer);
   if (st.pend_mode == APEX_MODE_EXACT) {
     std::vector<SlotCopy> copies;
@@ -657,7 +712,6 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
     ctx->host_stats[layer].demand_copies += (int64_t)copies.size();
     ctx->last_copies[layer].insert(ctx->last_copies[layer].end(), copies.begin(), copies.end());
   } else {
-    if (!host_wait_seq(ctx, mbox_exec_seq(ctx, layer), ctx->exec_seq[layer])) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: execution sets did not arrive");
     const int32_t* ex = mbox_exec(ctx, layer);
     for (int i = 0; i < B * k; ++i) tab.touch(ex[i]);
   }
@@ -693,8 +747,8 @@ int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev,
   for (int l = 0; l < ctx->cfg.L; ++l) {
     int32_t* idx = ctx->d_idx + (size_t)l * MB * k;
     float* alpha = ctx->d_alpha + (size_t)l * MB * N;
-    if ((r = apex_predict(ctx, l, h_dev + l * step, B, stream)) != APEX_OK) return r;
-    if ((r = apex_select_candidates(ctx, l, B, tau, ctx->d_cand, ctx->d_cand_ncand, stream)) != APEX_OK) return r;
+    if ((r = predict_select_fused(ctx, l, h_dev + l * step, B, tau, ctx->d_cand, ctx->d_cand_ncand, (cudaStream_t)stream)) != APEX_OK)
+      return r;
     if ((r = apex_attention_standin(ctx, l, stream)) != APEX_OK) return r;
     if ((r = apex_route_topk(ctx, l, hpost_dev + l * step, B, idx, alpha, stream)) != APEX_OK) return r;
     if (l > 0 && (r = ffn_finalize(ctx, l - 1)) != APEX_OK) return r;

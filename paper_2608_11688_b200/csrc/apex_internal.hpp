@@ -11,6 +11,33 @@
 
 namespace apex {
 
+// Debug builds (-DAPEX_TIMELINE): every kernel logs (id, start, end) of its block 0 in device memory.
+#ifdef APEX_TIMELINE
+struct SpanLog {
+  unsigned long long n;
+  unsigned long long rec[4096][3];
+};
+extern __device__ SpanLog g_spans;
+__device__ __forceinline__ unsigned long long span_now() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+#define SPAN_BEGIN() const unsigned long long _span_t0 = span_now()
+#define SPAN_END(id)                                                                     \
+  do {                                                                                   \
+    if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) {                         \
+      const unsigned long long _i = atomicAdd(&apex::g_spans.n, 1ull) & 4095ull;         \
+      apex::g_spans.rec[_i][0] = (id);                                                   \
+      apex::g_spans.rec[_i][1] = _span_t0;                                               \
+      apex::g_spans.rec[_i][2] = span_now();                                             \
+    }                                                                                    \
+  } while (0)
+#else
+#define SPAN_BEGIN() do { } while (0)
+#define SPAN_END(id) do { } while (0)
+#endif
+
 // ---- mapped host mailbox: the kernels post small decision records here so that the host can
 // plan copies without a stream synchronisation.  One per context; sequence numbers only grow.
 struct MailboxHeader {
@@ -22,7 +49,7 @@ struct MailboxHeader {
 // Byte offsets inside the mailbox.  Per layer: route_seq[l] is written by the gate kernel after
 // K_r of that layer, exec_seq[l] by the FFN's plan step after the execution sets.
 struct MailboxLayout {
-  size_t off_route_seq, off_exec_seq, off_ncand, off_cand, off_kr, off_exec, kr_stride, bytes;
+  size_t off_exec_seq, off_sel_rec, off_ncand, off_cand, off_kr, off_exec, kr_stride, bytes;
 };
 
 // Device-side counters of one layer (S9), accumulated with 64-bit atomics.
@@ -36,6 +63,27 @@ struct SlotSnapshot {
   int8_t expert_slot[APEX_MAX_EXPERTS];   // -1 = not resident
   uint32_t need_gen[APEX_MAX_EXPERTS];    // slot-ready value to wait for
   unsigned long long resident_mask;
+};
+
+struct SelectParams {
+  const float* q;       // [B][N]
+  const int32_t* pi;    // [B][N]
+  const float* w;       // [N]
+  const float* theta;   // [N-k+1]
+  int32_t* cand_out;    // [B][C] device, caller's
+  int32_t* ncand_out;   // [B]
+  int32_t* ncand_keep;  // [B] context-owned copy for the metrics
+  int32_t* mbox_cand;   // mapped host [B][C]
+  int32_t* mbox_ncand;  // mapped host [B]
+  volatile uint32_t* mbox_seq;
+  uint32_t* mbox_rec;   // mapped host, 16-byte aligned: {mask lo, mask hi, ncand, seq} for B == 1
+  uint32_t seq_value;
+  unsigned long long* done_counter;
+  unsigned long long done_target;
+  DevStats* stats;
+  float t_tau;
+  int force;  // 0: threshold test, 1: delta_hat = 0, 2: delta_hat = N-k
+  int N, k, C, B;
 };
 
 struct RouterParams {
@@ -52,33 +100,11 @@ struct RouterParams {
   const int32_t* pi_pred;     // [B][N] ranking of the prefetch router for this step, or null
   const int32_t* ncand_pred;  // [B]
   DevStats* stats;
-  int32_t* mbox_kr;                 // mapped host [B][k]
-  volatile uint32_t* mbox_seq;      // mapped host
-  uint32_t seq_value;
-  unsigned long long* done_counter; // device
-  unsigned long long done_target;
   int C;
+  int fuse_select;   // 1: the leader warp also runs the budget selection (sel) for its token
+  SelectParams sel;
 };
 
-struct SelectParams {
-  const float* q;       // [B][N]
-  const int32_t* pi;    // [B][N]
-  const float* w;       // [N]
-  const float* theta;   // [N-k+1]
-  int32_t* cand_out;    // [B][C] device, caller's
-  int32_t* ncand_out;   // [B]
-  int32_t* ncand_keep;  // [B] context-owned copy for the metrics
-  int32_t* mbox_cand;   // mapped host [B][C]
-  int32_t* mbox_ncand;  // mapped host [B]
-  volatile uint32_t* mbox_seq;
-  uint32_t seq_value;
-  unsigned long long* done_counter;
-  unsigned long long done_target;
-  DevStats* stats;
-  float t_tau;
-  int force;  // 0: threshold test, 1: delta_hat = 0, 2: delta_hat = N-k
-  int N, k, C, B;
-};
 
 struct FfnParams {
   const float* hpost;       // [B][d]
@@ -99,6 +125,7 @@ struct FfnParams {
   int32_t* pair_expert;     // [B*k + B]   (N = shared expert)
   int32_t* n_pairs;         // [1]
   int32_t* mbox_exec;       // mapped host [B][k]
+  int32_t* mbox_kr;         // mapped host [B][k]: the routed sets, posted with the execution sets
   volatile uint32_t* mbox_seq;
   volatile uint32_t* mbox_status;
   uint32_t seq_value;
@@ -156,7 +183,7 @@ struct apex_ctx {
   uint32_t* d_demand = nullptr;            // [L][N]
   int32_t *d_pi = nullptr, *d_ncand = nullptr;              // [maxB][N], [maxB]
   apex::DevStats* d_stats = nullptr;                        // [L]
-  unsigned long long* d_counters = nullptr;                 // [2 + L]: select done, zero, route done per layer
+  unsigned long long* d_counters = nullptr;                 // [2]: select done, zero
   int32_t *d_plan_exec_idx = nullptr, *d_pair_tok = nullptr, *d_pair_expert = nullptr, *d_n_pairs = nullptr;
   float *d_plan_exec_gate = nullptr, *d_pair_gate = nullptr;
   uint8_t* d_attn = nullptr;
@@ -173,8 +200,7 @@ struct apex_ctx {
   uint8_t* mbox = nullptr;
   apex::MailboxLayout ml{};
   uint32_t sel_seq = 0;
-  std::vector<uint32_t> route_seq, exec_seq;      // per layer, last value asked for
-  std::vector<unsigned long long> route_done;     // per layer
+  std::vector<uint32_t> exec_seq;                 // per layer, last value asked for
   unsigned long long sel_done = 0, zero_done = 0;
   uint32_t launch_tag = 0;
   uint32_t* gen_src = nullptr;  // pinned ring of flag values for the ready-flag copies

@@ -242,6 +242,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     store_token_plan(tp, lane, k, p.plan_exec_idx + (size_t)b * k, p.plan_exec_gate + (size_t)b * k,
                      p.post_exec ? p.mbox_exec + (size_t)b * k : nullptr);
     if (p.post_exec) {
+      if (lane < k) p.mbox_kr[(size_t)b * k + lane] = tl.my_idx;
       const int e0 = lane, e1 = lane + 32;
       if ((tp.exec_mask >> e0) & 1) {
         const int pos = __popcll(tp.exec_mask & ((1ull << e0) - 1ull));
@@ -358,6 +359,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   const int G = gridDim.x, cta = blockIdx.x;
 
   // ---- work that does not depend on the preceding kernel
+  SPAN_BEGIN();
   if (tid == 0) {
     TL(0);
     TL(1);
@@ -548,15 +550,10 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     bulk_g2s(smem + (size_t)s * entry_bytes, base + (size_t)i * entry_bytes, entry_bytes, &s_full[s]);
   };
 
-  if (lane < NSW && lane < my_n) {
-    if (lane == 0 && warp == 0) TL(3);
-    issue(lane);
-    if (!ok) atomicExch(&s_abort, 1);
-  }
-  __syncwarp();
-  if (B == 1 && cta == 0 && warp == 0 && p.post_exec) {
-    // the execution set goes to the caller's buffers and to the host mailbox while the first rows are in flight
+  auto post_plan = [&]() {
+    // the routed and the execution set go to the caller's buffers and to the host mailbox
     store_token_plan(tp1, lane, k, p.exec_idx, p.exec_gate, p.mbox_exec);
+    if (lane < k) p.mbox_kr[lane] = tl1.my_idx;
     if (lane == 0 && p.stats) {
       const int ns = __popcll(tp1.exec_mask & ~tp1.kr_mask);
       if (ns) atomicAdd(&p.stats->substitutions, (unsigned long long)ns);
@@ -568,7 +565,19 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
       __threadfence_system();
       *p.mbox_seq = p.seq_value;
     }
+  };
+  const bool poster = B == 1 && cta == 0 && warp == 0 && p.post_exec;
+  // If an expert of this launch still has to be fetched, the host cannot start before it has seen
+  // K_r: post first.  Otherwise post while the first rows are in flight.
+  const bool will_wait_for_host = p.demand_in_kernel && (run & ~p.snap.resident_mask) != 0ull;
+  if (poster && will_wait_for_host) post_plan();
+  if (lane < NSW && lane < my_n) {
+    if (lane == 0 && warp == 0) TL(3);
+    issue(lane);
+    if (!ok) atomicExch(&s_abort, 1);
   }
+  __syncwarp();
+  if (poster && !will_wait_for_host) post_plan();
   int issued = my_n < NSW ? my_n : NSW;  // rows of this warp whose copy has been started (uniform across the warp)
   for (int j = 0; j < my_n; ++j) {
     if (lane == 0 && j == my_n - 1) poll_zeroed(false);  // latency hidden behind the wait for the last row
@@ -734,11 +743,22 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     }
   }
   if (tid == 0) TL(9);
+  SPAN_END(5);
 }
 
 #ifdef APEX_TIMELINE
+__device__ SpanLog g_spans;
 extern "C" int apex_debug_read_timeline(unsigned long long* host, int n) {
   return (int)cudaMemcpyFromSymbol(host, g_timeline, sizeof(unsigned long long) * n);
+}
+extern "C" int apex_debug_read_spans(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_spans, sizeof(SpanLog));
+}
+extern "C" int apex_debug_reset_spans() {
+  SpanLog* z = new SpanLog();
+  int r = (int)cudaMemcpyToSymbol(g_spans, z, sizeof(SpanLog));
+  delete z;
+  return r;
 }
 #endif
 

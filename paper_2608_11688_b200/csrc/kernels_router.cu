@@ -34,10 +34,85 @@ __device__ __forceinline__ int warp_max_int(int v) {
 // expert; the logits are gathered in the leader CTA's shared memory through distributed shared
 // memory, and the leader's first warp does softmax, ranking, top-k and (for the gate) the
 // per-step metrics of Eq. (2)-(3).
+// Budget selection for one token by one warp (Eq. (8), (9) in the logit domain; Eq. (1)).
+// Lane l holds positions l and l+32 of the ranked list E: pj = expert at that position, x = its
+// prefetch probability (so x is the prefetch distribution in descending order).
+//   s = w.x   (lane partial: position l then l+32 with fused multiply-adds, then the xor tree)
+//   delta_hat = first delta with theta_delta - s >= logit(tau), capped to C - k
+//   K_p = first k + delta_hat experts of E
+__device__ __forceinline__ void select_token(const SelectParams& p, int b, int lane, int pj0, int pj1, float x0, float x1) {
+  const int N = p.N, k = p.k, C = p.C;
+  float part = 0.f;
+  if (lane < N) part = fmaf(__ldg(p.w + lane), x0, part);
+  if (lane + 32 < N) part = fmaf(__ldg(p.w + lane + 32), x1, part);
+  const float sdot = warp_sum_tree(part);
+  const int nth = N - k + 1;
+  const bool pass0 = lane < nth && (__ldg(p.theta + lane) - sdot >= p.t_tau);
+  const bool pass1 = lane + 32 < nth && (__ldg(p.theta + lane + 32) - sdot >= p.t_tau);
+  const unsigned m0 = __ballot_sync(0xffffffffu, pass0), m1 = __ballot_sync(0xffffffffu, pass1);
+  int d_hat = m0 ? (__ffs(m0) - 1) : (m1 ? 32 + __ffs(m1) - 1 : N - k);
+  if (p.force == 1) d_hat = 0;
+  if (p.force == 2) d_hat = N - k;
+  const int uncapped = d_hat;
+  d_hat = min(d_hat, C - k);
+  const int ncand = k + d_hat;
+  // candidates in rank order, padded with -1
+  const bool in0 = lane < ncand, in1 = lane + 32 < ncand;
+  if (lane < C) {
+    const int v = in0 ? pj0 : -1;
+    p.cand_out[(size_t)b * C + lane] = v;
+    p.mbox_cand[(size_t)b * C + lane] = v;
+  }
+  if (lane + 32 < C) {
+    const int v = in1 ? pj1 : -1;
+    p.cand_out[(size_t)b * C + lane + 32] = v;
+    p.mbox_cand[(size_t)b * C + lane + 32] = v;
+  }
+  // the candidate set as a 64-bit mask
+  unsigned lo = 0, hi = 0;
+  if (in0) { if (pj0 < 32) lo |= 1u << pj0; else hi |= 1u << (pj0 - 32); }
+  if (in1) { if (pj1 < 32) lo |= 1u << pj1; else hi |= 1u << (pj1 - 32); }
+  lo = __reduce_or_sync(0xffffffffu, lo);
+  hi = __reduce_or_sync(0xffffffffu, hi);
+  if (lane == 0) {
+    p.ncand_out[b] = ncand;
+    p.ncand_keep[b] = ncand;
+    p.mbox_ncand[b] = ncand;
+    if (p.stats) {
+      atomicAdd(&p.stats->tokens, 1ull);
+      atomicAdd(&p.stats->sum_delta_hat, (unsigned long long)d_hat);
+      atomicAdd(&p.stats->sum_ncand, (unsigned long long)ncand);
+      atomicAdd(&p.stats->capped, (unsigned long long)(uncapped > d_hat ? 1 : 0));
+      atomicAdd(&p.stats->near_full, (unsigned long long)(2 * ncand > N ? 1 : 0));
+    }
+  }
+  if (p.B == 1) {
+    // one token: the host needs only the set.  Mask, count and sequence number travel in ONE aligned
+    // 16-byte store, so no system-scope fence sits on the kernel's critical path.  (The ranked list
+    // above is advisory for the host: it is used for the issue order only if it matches the mask.)
+    if (lane == 0) {
+      asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p.mbox_rec), "r"(lo), "r"(hi), "r"((unsigned)ncand),
+                   "r"(p.seq_value)
+                   : "memory");
+    }
+    return;
+  }
+  __threadfence_system();
+  __syncwarp();
+  if (lane == 0) {
+    const unsigned long long old = atomicAdd(p.done_counter, 1ull);
+    if (old + 1 == p.done_target) {
+      __threadfence_system();
+      *p.mbox_seq = p.seq_value;
+    }
+  }
+}
+
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
+  SPAN_BEGIN();
   pdl_wait();               // everything queued before this kernel is complete
   pdl_launch_dependents();  // the next kernel may begin its own prologue
   cg::cluster_group cluster = cg::this_cluster();
@@ -45,6 +120,8 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
   const int b = blockIdx.y;
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   __shared__ float zs[APEX_MAX_EXPERTS];
+  __shared__ float qs[APEX_MAX_EXPERTS];
+  __shared__ int pis[APEX_MAX_EXPERTS];
   __shared__ int posp[APEX_MAX_EXPERTS];
 
   const int e = (int)crank * p.warps_per_cta + warp;
@@ -53,7 +130,7 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
     const float4* __restrict__ xv = reinterpret_cast<const float4*>(p.x + (size_t)b * p.d);
     const int nv = p.d >> 2;
     float acc = 0.f;
-#pragma unroll 4
+#pragma unroll 8
     for (int c = lane; c < nv; c += 32) {
       const float4 w = __ldg(Wrow + c);
       const float4 x = __ldg(xv + c);
@@ -102,13 +179,25 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
     if (p.pi_out) p.pi_out[row + r1] = e1;
     if (p.topk_out && r1 < k) p.topk_out[(size_t)b * k + r1] = e1;
   }
-  if (!p.mbox_seq) return;
+  if (p.fuse_select) {
+    // prefetch router and budget selection in one launch: the ranked list goes through shared memory
+    if (e0 < N) { qs[e0] = q0; pis[r0] = e0; }
+    if (e1 < N) { qs[e1] = q1; pis[r1] = e1; }
+    __syncwarp();
+    const int pj0 = lane < N ? pis[lane] : -1, pj1 = lane + 32 < N ? pis[lane + 32] : -1;
+    const float x0 = pj0 >= 0 ? qs[pj0] : 0.f, x1 = pj1 >= 0 ? qs[pj1] : 0.f;
+    select_token(p.sel, b, lane, pj0, pj1, x0, x1);
+    SPAN_END(1);
+    return;
+  }
+  if (!p.topk_out || !p.stats) {
+    SPAN_END(1);
+    return;
+  }
 
-  // ---- gate epilogue: K_r to the host mailbox, metrics of this token
+  // ---- gate epilogue: metrics of this token against the prefetch stage (Eq. (2), (3))
   const bool in0 = e0 < N && r0 < k, in1 = e1 < N && r1 < k;
-  if (in0) p.mbox_kr[(size_t)b * k + r0] = e0;
-  if (in1) p.mbox_kr[(size_t)b * k + r1] = e1;
-  if (p.stats) {
+  {
     int dstar = 0, hitsP = 0, have_pred = 0;
     if (p.pi_pred) {
       have_pred = 1;
@@ -129,15 +218,7 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
       }
     }
   }
-  __threadfence_system();
-  __syncwarp();
-  if (lane == 0) {
-    const unsigned long long old = atomicAdd(p.done_counter, 1ull);
-    if (old + 1 == p.done_target) {
-      __threadfence_system();
-      *p.mbox_seq = p.seq_value;
-    }
-  }
+  SPAN_END(4);
 }
 
 cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
@@ -167,66 +248,26 @@ cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
 // s = w.x, delta_hat = first delta with theta_delta - s >= logit(tau)  (Eq. (8), (9) in the logit
 // domain), capped to C - k; K_p = first k + delta_hat experts of E (Eq. (1)).
 __global__ void __launch_bounds__(128) select_kernel(const SelectParams p) {
+  SPAN_BEGIN();
   pdl_wait();
   pdl_launch_dependents();
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int b = blockIdx.x * (blockDim.x >> 5) + warp;
   if (b >= p.B) return;
-  const int N = p.N, k = p.k, C = p.C;
+  const int N = p.N;
   const size_t row = (size_t)b * N;
-  float part = 0.f;
   int pj0 = -1, pj1 = -1;
+  float x0 = 0.f, x1 = 0.f;
   if (lane < N) {
     pj0 = __ldg(p.pi + row + lane);
-    part = fmaf(__ldg(p.w + lane), __ldg(p.q + row + pj0), part);
+    x0 = __ldg(p.q + row + pj0);
   }
   if (lane + 32 < N) {
     pj1 = __ldg(p.pi + row + lane + 32);
-    part = fmaf(__ldg(p.w + lane + 32), __ldg(p.q + row + pj1), part);
+    x1 = __ldg(p.q + row + pj1);
   }
-  const float sdot = warp_sum_tree(part);
-  const int nth = N - k + 1;
-  const bool pass0 = lane < nth && (__ldg(p.theta + lane) - sdot >= p.t_tau);
-  const bool pass1 = lane + 32 < nth && (__ldg(p.theta + lane + 32) - sdot >= p.t_tau);
-  const unsigned m0 = __ballot_sync(0xffffffffu, pass0), m1 = __ballot_sync(0xffffffffu, pass1);
-  int d_hat = m0 ? (__ffs(m0) - 1) : (m1 ? 32 + __ffs(m1) - 1 : N - k);
-  if (p.force == 1) d_hat = 0;
-  if (p.force == 2) d_hat = N - k;
-  const int uncapped = d_hat;
-  d_hat = min(d_hat, C - k);
-  const int ncand = k + d_hat;
-  // candidates in rank order, padded with -1
-  if (lane < C) {
-    const int v = lane < ncand ? pj0 : -1;
-    p.cand_out[(size_t)b * C + lane] = v;
-    p.mbox_cand[(size_t)b * C + lane] = v;
-  }
-  if (lane + 32 < C) {
-    const int v = lane + 32 < ncand ? pj1 : -1;
-    p.cand_out[(size_t)b * C + lane + 32] = v;
-    p.mbox_cand[(size_t)b * C + lane + 32] = v;
-  }
-  if (lane == 0) {
-    p.ncand_out[b] = ncand;
-    p.ncand_keep[b] = ncand;
-    p.mbox_ncand[b] = ncand;
-    if (p.stats) {
-      atomicAdd(&p.stats->tokens, 1ull);
-      atomicAdd(&p.stats->sum_delta_hat, (unsigned long long)d_hat);
-      atomicAdd(&p.stats->sum_ncand, (unsigned long long)ncand);
-      atomicAdd(&p.stats->capped, (unsigned long long)(uncapped > d_hat ? 1 : 0));
-      atomicAdd(&p.stats->near_full, (unsigned long long)(2 * ncand > N ? 1 : 0));
-    }
-  }
-  __threadfence_system();
-  __syncwarp();
-  if (lane == 0) {
-    const unsigned long long old = atomicAdd(p.done_counter, 1ull);
-    if (old + 1 == p.done_target) {
-      __threadfence_system();
-      *p.mbox_seq = p.seq_value;
-    }
-  }
+  select_token(p, b, lane, pj0, pj1, x0, x1);
+  SPAN_END(2);
 }
 
 cudaError_t launch_select(const SelectParams& p, cudaStream_t s) {
@@ -246,6 +287,7 @@ cudaError_t launch_select(const SelectParams& p, cudaStream_t s) {
 // Streams attn_bytes once (the weight and KV bytes an attention block of this shape reads).  The
 // xor of everything read is stored only if it equals one fixed pattern, which keeps the loads live.
 __global__ void __launch_bounds__(512) attention_standin_kernel(const AttnParams p) {
+  SPAN_BEGIN();
   pdl_wait();
   pdl_launch_dependents();
   const size_t stride = (size_t)gridDim.x * blockDim.x;
@@ -258,6 +300,7 @@ __global__ void __launch_bounds__(512) attention_standin_kernel(const AttnParams
     a.w ^= v.w;
   }
   if (a.x == 0x12345678u && a.y == 0x9abcdef0u && a.z == 0x0fedcba9u && a.w == 0x87654321u) p.sink[0] = 1.f;
+  SPAN_END(3);
 }
 
 cudaError_t launch_attention(const AttnParams& p, int n_sm, cudaStream_t s) {

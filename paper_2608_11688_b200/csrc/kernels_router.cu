@@ -111,10 +111,18 @@ __device__ __forceinline__ void select_token(const SelectParams& p, int b, int l
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
+constexpr int kRouterMaxVec = 32;  // float4 per lane of one weight row: d <= 4096
+
+#ifdef APEX_TIMELINE
+__device__ long long g_router_tl[16];
+#define RTL(i) do { if (blockIdx.x == 0 && blockIdx.y == 0 && threadIdx.x == 0) g_router_tl[i] = clock64(); } while (0)
+extern "C" int apex_debug_read_router_tl(long long* host) { return (int)cudaMemcpyFromSymbol(host, g_router_tl, sizeof(long long) * 16); }
+#else
+#define RTL(i) do { } while (0)
+#endif
+
 __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
   SPAN_BEGIN();
-  pdl_wait();               // everything queued before this kernel is complete
-  pdl_launch_dependents();  // the next kernel may begin its own prologue
   cg::cluster_group cluster = cg::this_cluster();
   const unsigned crank = cluster.block_rank();
   const int b = blockIdx.y;
@@ -123,30 +131,58 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
   __shared__ float qs[APEX_MAX_EXPERTS];
   __shared__ int pis[APEX_MAX_EXPERTS];
   __shared__ int posp[APEX_MAX_EXPERTS];
+  __shared__ float4 xs[kRouterMaxVec * 32];
 
+  // The router weights are parameters, not results of the preceding kernel: this warp's row is
+  // loaded into registers before the dependency wait, so its DRAM latency hides behind that kernel.
   const int e = (int)crank * p.warps_per_cta + warp;
-  if (warp < p.warps_per_cta && e < p.N) {
+  const bool active = warp < p.warps_per_cta && e < p.N;
+  const int nv = p.d >> 2;
+  float4 wreg[kRouterMaxVec];
+  float bias_e = 0.f;
+  if (active) {
     const float4* __restrict__ Wrow = reinterpret_cast<const float4*>(p.W + (size_t)e * p.d);
+#pragma unroll
+    for (int i = 0; i < kRouterMaxVec; ++i) {
+      const int c = i * 32 + lane;
+      if (c < nv) wreg[i] = __ldg(Wrow + c);
+    }
+    if (p.bias) bias_e = __ldg(p.bias + e);
+  }
+  RTL(0);
+  pdl_wait();               // everything queued before this kernel is complete: x may be read
+  pdl_launch_dependents();  // the next kernel may begin its own prologue
+  RTL(1);
+
+  // x is staged in shared memory by the whole CTA in one round of loads
+  {
     const float4* __restrict__ xv = reinterpret_cast<const float4*>(p.x + (size_t)b * p.d);
-    const int nv = p.d >> 2;
+    for (int c = threadIdx.x; c < nv; c += blockDim.x) xs[c] = __ldg(xv + c);
+  }
+  __syncthreads();
+  if (active) {
     float acc = 0.f;
-#pragma unroll 8
-    for (int c = lane; c < nv; c += 32) {
-      const float4 w = __ldg(Wrow + c);
-      const float4 x = __ldg(xv + c);
-      acc = fmaf(w.x, x.x, acc);
-      acc = fmaf(w.y, x.y, acc);
-      acc = fmaf(w.z, x.z, acc);
-      acc = fmaf(w.w, x.w, acc);
+#pragma unroll
+    for (int i = 0; i < kRouterMaxVec; ++i) {
+      const int c = i * 32 + lane;
+      if (c < nv) {
+        const float4 x = xs[c];
+        acc = fmaf(wreg[i].x, x.x, acc);
+        acc = fmaf(wreg[i].y, x.y, acc);
+        acc = fmaf(wreg[i].z, x.z, acc);
+        acc = fmaf(wreg[i].w, x.w, acc);
+      }
     }
     acc = warp_sum_tree(acc);
     if (lane == 0) {
-      const float z = acc + (p.bias ? __ldg(p.bias + e) : 0.f);
+      const float z = acc + bias_e;
       float* dst = cluster.map_shared_rank(zs, 0);
       dst[e] = z;
     }
   }
+  RTL(2);
   cluster.sync();
+  RTL(3);
   if (crank != 0 || warp != 0) return;
 
   // ---- leader warp: lanes own experts lane and lane+32
@@ -179,6 +215,7 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
     if (p.pi_out) p.pi_out[row + r1] = e1;
     if (p.topk_out && r1 < k) p.topk_out[(size_t)b * k + r1] = e1;
   }
+  RTL(4);
   if (p.fuse_select) {
     // prefetch router and budget selection in one launch: the ranked list goes through shared memory
     if (e0 < N) { qs[e0] = q0; pis[r0] = e0; }
@@ -187,6 +224,7 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
     const int pj0 = lane < N ? pis[lane] : -1, pj1 = lane + 32 < N ? pis[lane + 32] : -1;
     const float x0 = pj0 >= 0 ? qs[pj0] : 0.f, x1 = pj1 >= 0 ? qs[pj1] : 0.f;
     select_token(p.sel, b, lane, pj0, pj1, x0, x1);
+    RTL(5);
     SPAN_END(1);
     return;
   }
@@ -218,6 +256,7 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
       }
     }
   }
+  RTL(5);
   SPAN_END(4);
 }
 

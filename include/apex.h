@@ -54,6 +54,7 @@ extern "C" {
 #define APEX_MAX_EXPERTS 64
 #define APEX_MAX_TOPK 16
 #define APEX_MAX_BATCH 256
+#define APEX_STATIC_MAX_BATCH 64 /* largest B of apex_route_topk_static */
 
 typedef struct apex_ctx apex_ctx;
 
@@ -186,6 +187,28 @@ int apex_warm_all(apex_ctx* ctx);
 int apex_test_inject(apex_ctx* ctx, int what);
 /* Number of kernels this library has launched on the context so far. */
 int64_t apex_launch_count(const apex_ctx* ctx);
+
+/* ---- allocation-free gate ----------------------------------------------------------------- */
+
+/* (No counterpart in the paper: an addition for deployment.)
+ * The exact top-k gate of apex_route_topk for callers that cannot allocate device memory -- for
+ * example a serving process whose HBM is owned by a fixed pool, where a stray cudaMalloc would
+ * both escape the pool's accounting and stall the device.  No context is needed and nothing is
+ * allocated or freed, here or in any library it calls.
+ *   W_r_dev [N][d], b_r_dev [N] or NULL, hpost_dev [B][d]: device inputs, borrowed for the launch.
+ *   idx_dev [B][k] (K_r in rank order) and alpha_dev [B][N] (softmax of the logits): device outputs.
+ *   Limits: B <= APEX_STATIC_MAX_BATCH (64), N <= APEX_MAX_EXPERTS (64), k <= min(N, 16),
+ *   d a multiple of 4 and d <= 4096.  Larger sizes are refused with APEX_EINVAL and a message.
+ * The kernel's only scratch, the raw logits, lives in a 16 KiB array built into the library; every
+ * GPU that loads the library holds it until the process ends.  The first call on a device looks
+ * up the array's address on that device (make that first call outside any stream capture).  All
+ * calls on a device share the array and it keeps the previous call's logits; the kernel overwrites
+ * what it uses, so nothing has to be cleared, but two calls that overlap on the GPU (different
+ * streams) race on it: serialise them.
+ * err (optional, err_len bytes, caller-owned) receives a text on failure.  Returns APEX_OK,
+ * APEX_EINVAL or APEX_ECUDA. */
+int apex_route_topk_static(const float* W_r_dev, const float* b_r_dev, const float* hpost_dev, int N, int d, int k,
+                           int B, int32_t* idx_dev, float* alpha_dev, void* stream, char* err, size_t err_len);
 
 /* ---- host-only slot planner (the state machine behind apex_prefetch / apex_moe_ffn) -------- */
 

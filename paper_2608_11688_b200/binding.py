@@ -69,6 +69,7 @@ SIGNATURES = {
     "apex_warm_all": (_I, [_P]),
     "apex_test_inject": (_I, [_P, _I]),
     "apex_launch_count": (C.c_int64, [_P]),
+    "apex_route_topk_static": (_I, [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, C.c_char_p, C.c_size_t]),
     "apex_slots_create": (_P, [_I, _I, _I]),
     "apex_slots_destroy": (None, [_P]),
     "apex_slots_begin_step": (_I, [_P]),
@@ -265,6 +266,20 @@ class Apex:
 
     def launch_count(self):
         return int(self.lib.apex_launch_count(self.h))
+
+
+def route_topk_static(W_r_dev, b_r_dev, hpost_dev, k, idx_dev, alpha_dev, stream=None):
+    """apex_route_topk_static: the gate without a context and without any allocation.  W_r_dev [N][d],
+    b_r_dev [N] or None, hpost_dev [B][d] are CUDA tensors; idx_dev [B][k] int32 and alpha_dev [B][N]
+    fp32 receive the result.  Raises ApexError with the library's message on failure."""
+    lib = load_library()
+    N, d = W_r_dev.shape
+    B = hpost_dev.shape[0]
+    err = C.create_string_buffer(256)
+    rc = lib.apex_route_topk_static(_ptr(W_r_dev), _ptr(b_r_dev), _ptr(hpost_dev), N, d, k, B, _ptr(idx_dev),
+                                    _ptr(alpha_dev), _stream(stream), err, len(err))
+    if rc != APEX_OK:
+        raise ApexError(rc, err.value.decode())
 
 
 class Slots:

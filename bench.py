@@ -33,7 +33,7 @@ TAU = 0.90
 
 # DRAM bytes per launch of the expert-FFN kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu capture summarised in profiles/ (same kernel, same per-launch shape).  None = not captured.
-NCU_TRAFFIC_BYTES = {1: None}
+NCU_TRAFFIC_BYTES = {1: 37_854_500}   # profiles/moe_ffn_stream_kernel_config1.md: 37.809 MB read + ~0.045 MB written
 
 
 def measured_peak():

@@ -209,12 +209,30 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(dev_alloc(&ctx->d_pair_gate, max_pairs));
   CR(dev_alloc(&ctx->d_pair_expert, max_pairs));
   CR(dev_alloc(&ctx->d_n_pairs, 4));
+  CR(dev_alloc(&ctx->d_grp, 4 + 3 * (N + 1)));
   CR(dev_alloc(&ctx->d_cand, MB * C));
   CR(dev_alloc(&ctx->d_idx, L * MB * k));
   CR(dev_alloc(&ctx->d_exec_idx, MB * k));
   CR(dev_alloc(&ctx->d_alpha, L * MB * N));
   CR(dev_alloc(&ctx->d_exec_gate, MB * k));
   CR(dev_alloc(&ctx->d_cand_ncand, MB));
+  // batched tensor-core path: scratch and tensor maps (only for contexts that will see large batches)
+  if (MB >= 16 && tc_shape_supported(c.d, c.I, c.I_shared)) {
+    const size_t rows = max_pairs + 256;
+    const size_t i_max = (size_t)(c.I > c.I_shared ? c.I : c.I_shared);
+    ctx->act_stride = (int)i_max;
+    CR(dev_alloc(&ctx->d_xg, rows * d));
+    ctx->act_plane = rows * i_max;
+    CR(dev_alloc(&ctx->d_act, 2 * rows * i_max));
+    CR(cudaMemset(ctx->d_xg, 0, rows * d * 2));
+    CR(cudaMemset(ctx->d_act, 0, 2 * rows * i_max * 2));
+    ctx->tc_ok = tc_make_weight_map(ctx->tc_maps.w_gateup, ctx->d_cache, c.d, c.I, L * C, ctx->expert_bytes, 128) &&
+                 tc_make_weight_map(ctx->tc_maps.w_down, ctx->d_cache, c.d, c.I, L * C, ctx->expert_bytes, 64) &&
+                 tc_make_rows_map(ctx->tc_maps.xg, ctx->d_xg, c.d, rows, d) &&
+                 tc_make_rows_map(ctx->tc_maps.act, ctx->d_act, (int)i_max, rows, i_max) &&
+                 tc_make_rows_map(ctx->tc_maps.act_lo, ctx->d_act + ctx->act_plane, (int)i_max, rows, i_max);
+    ctx->tc_shared_maps.assign(L, ctx->tc_maps);
+  }
   ctx->attn_bytes = (4 * d * d + 2 * (size_t)ctx->cfg.ctx_len * d) * 2;
   ctx->attn_layers = L < 8 ? L : 8;
   CR(dev_alloc(&ctx->d_attn, ctx->attn_bytes * ctx->attn_layers));
@@ -273,7 +291,7 @@ int apex_destroy(apex_ctx* ctx) {
   cudaGetLastError();
   void* dev[] = {ctx->d_Wr, ctx->d_br, ctx->d_Wp, ctx->d_bp, ctx->d_w, ctx->d_theta, ctx->d_cache, ctx->d_slot_ready, ctx->d_zp,
                  ctx->d_qp, ctx->d_zr, ctx->d_demand, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_plan_exec_idx,
-                 ctx->d_plan_exec_gate, ctx->d_pair_tok, ctx->d_pair_gate, ctx->d_pair_expert, ctx->d_n_pairs, ctx->d_cand,
+                 ctx->d_plan_exec_gate, ctx->d_pair_tok, ctx->d_pair_gate, ctx->d_pair_expert, ctx->d_n_pairs, ctx->d_grp, ctx->d_xg, ctx->d_act, ctx->d_cand,
                  ctx->d_idx, ctx->d_exec_idx, ctx->d_alpha, ctx->d_exec_gate, ctx->d_cand_ncand, ctx->d_attn, ctx->d_attn_sink,
                  ctx->d_h_stage, ctx->d_hp_stage, ctx->d_y_stage};
   for (void* p : dev)
@@ -340,6 +358,12 @@ int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights) {
   if (ctx->cfg.I_shared <= 0) return fail(ctx, APEX_EINVAL, "the context was created with I_shared = 0");
   if (!dev_weights || ((uintptr_t)dev_weights & 15)) return fail(ctx, APEX_EINVAL, "shared expert: null or unaligned");
   ctx->shared_dev[layer] = static_cast<const uint8_t*>(dev_weights);
+  if (ctx->tc_ok) {
+    TcMaps& m = ctx->tc_shared_maps[layer];
+    if (!tc_make_weight_map(m.ws_gateup, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1, ctx->shared_bytes, 128) ||
+        !tc_make_weight_map(m.ws_down, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1, ctx->shared_bytes, 64))
+      return fail(ctx, APEX_ECUDA, "tensor map for the shared expert could not be encoded");
+  }
   return APEX_OK;
 }
 
@@ -567,6 +591,30 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
 
 namespace {
 
+constexpr int kTcMinBatch = 16;  // from this many tokens per step the tensor-core grouped GEMM runs
+
+// B > 1: plan kernel, then either the tensor-core grouped GEMM or the streaming kernel per pair.
+int launch_batched(apex_ctx* ctx, int layer, const FfnParams& p, cudaStream_t cs) {
+  CU_TRY(ctx, launch_ffn_plan(p, cs));
+  ++ctx->launches;
+  if (ctx->tc_ok && p.B >= kTcMinBatch) {
+    TcParams t{};
+    t.f = p;
+    t.grp = ctx->d_grp;
+    t.xg = ctx->d_xg;
+    t.act = ctx->d_act;
+    t.act_stride = ctx->act_stride;
+    t.act_plane = ctx->act_plane;
+    t.layer_slot0 = layer * ctx->cfg.C;
+    CU_TRY(ctx, launch_ffn_tc(t, ctx->tc_shared_maps[layer], ctx->n_sm, cs));
+    ctx->launches += 3;
+  } else {
+    CU_TRY(ctx, launch_ffn(p, ctx->n_sm, cs));
+    ++ctx->launches;
+  }
+  return APEX_OK;
+}
+
 // First half of apex_moe_ffn: launches the expert FFN of a layer-step.  B == 1 in exact mode is one
 // launch that also waits, inside the kernel, for experts the host has to fetch on demand; otherwise
 // the launch covers the experts that are resident and ffn_finalize adds further launches.
@@ -596,6 +644,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.pair_gate = ctx->d_pair_gate;
   p.pair_expert = ctx->d_pair_expert;
   p.n_pairs = ctx->d_n_pairs;
+  p.grp = ctx->d_grp;
   p.mbox_exec = mbox_exec(ctx, layer);
   p.mbox_kr = mbox_kr(ctx, layer);
   p.mbox_seq = mbox_exec_seq(ctx, layer);
@@ -618,11 +667,12 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.demand_in_kernel = (mode == APEX_MODE_EXACT && B == 1) ? 1 : 0;
   p.run_mask = p.demand_in_kernel ? ~0ull : p.snap.resident_mask;
   if (B > 1) {
-    CU_TRY(ctx, launch_ffn_plan(p, cs));
+    int r = launch_batched(ctx, layer, p, cs);
+    if (r != APEX_OK) return r;
+  } else {
+    CU_TRY(ctx, launch_ffn(p, ctx->n_sm, cs));
     ++ctx->launches;
   }
-  CU_TRY(ctx, launch_ffn(p, ctx->n_sm, cs));
-  ++ctx->launches;
   st.pending = true;
   st.pend_mode = mode;
   st.pend_tag = p.demand_tag;
@@ -701,11 +751,12 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
         q.run_shared = 0;
         q.post_exec = 0;
         if (B > 1) {
-          CU_TRY(ctx, launch_ffn_plan(q, cs));
+          int r = launch_batched(ctx, layer, q, cs);
+          if (r != APEX_OK) return r;
+        } else {
+          CU_TRY(ctx, launch_ffn(q, ctx->n_sm, cs));
           ++ctx->launches;
         }
-        CU_TRY(ctx, launch_ffn(q, ctx->n_sm, cs));
-        ++ctx->launches;
         ctx->host_stats[layer].extra_waves += 1;
       }
     }

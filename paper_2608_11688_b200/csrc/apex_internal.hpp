@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of libapex.so.
 #pragma once
+#include <cuda_bf16.h>
 #include <cuda_runtime.h>
 
 #include <cstdint>
@@ -124,6 +125,7 @@ struct FfnParams {
   float* pair_gate;         // [B*k + B]
   int32_t* pair_expert;     // [B*k + B]   (N = shared expert)
   int32_t* n_pairs;         // [1]
+  int32_t* grp;             // [4 + 3*(N+1)]: routed groups, all groups, 0, 0, then (expert, pair offset, tokens) per group
   int32_t* mbox_exec;       // mapped host [B][k]
   int32_t* mbox_kr;         // mapped host [B][k]: the routed sets, posted with the execution sets
   volatile uint32_t* mbox_seq;
@@ -142,6 +144,20 @@ struct FfnParams {
   int d, N, k, I, I_shared, B, mode, norm_topk, accumulate, run_shared, post_exec;
 };
 
+// Batched tensor-core path (kernels_ffn_tc.cu)
+struct TcParams {
+  FfnParams f;
+  const int32_t* grp;
+  __nv_bfloat16* xg;    // [pairs][d] gathered activations, bf16
+  __nv_bfloat16* act;   // two planes [2][rows][act_stride]: bf16(a) and bf16(a - bf16(a))
+  size_t act_plane;     // elements per plane
+  int act_stride;
+  int layer_slot0;      // index of this layer's slot 0 in the all-layers weight tensor map
+};
+struct TcMaps {          // opaque 128-byte CUtensorMap objects
+  alignas(64) unsigned char w_gateup[128], w_down[128], ws_gateup[128], ws_down[128], xg[128], act[128], act_lo[128];
+};
+
 struct AttnParams {
   const uint4* buf;
   size_t n_vec;  // 16-byte vectors
@@ -155,6 +171,10 @@ cudaError_t launch_attention(const AttnParams& p, int n_sm, cudaStream_t s);
 cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s);
 cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s);
 cudaError_t ffn_configure(int d);  // sets the dynamic shared-memory attribute once per shape
+cudaError_t launch_ffn_tc(const TcParams& p, const TcMaps& m, int n_sm, cudaStream_t s);
+bool tc_make_weight_map(void* out, const void* base, int d, int I, size_t n_slots, size_t slot_bytes, int box_rows);
+bool tc_make_rows_map(void* out, const void* base, int cols, size_t rows, size_t stride_elems);
+bool tc_shape_supported(int d, int I, int I_shared);
 bool ffn_shape_supported(int d);
 
 }  // namespace apex
@@ -186,6 +206,14 @@ struct apex_ctx {
   unsigned long long* d_counters = nullptr;                 // [2]: select done, zero
   int32_t *d_plan_exec_idx = nullptr, *d_pair_tok = nullptr, *d_pair_expert = nullptr, *d_n_pairs = nullptr;
   float *d_plan_exec_gate = nullptr, *d_pair_gate = nullptr;
+  // batched tensor-core path
+  bool tc_ok = false;
+  int32_t* d_grp = nullptr;
+  __nv_bfloat16 *d_xg = nullptr, *d_act = nullptr;
+  int act_stride = 0;
+  size_t act_plane = 0;
+  apex::TcMaps tc_maps{};
+  std::vector<apex::TcMaps> tc_shared_maps;  // per layer: ws_gateup / ws_down filled
   uint8_t* d_attn = nullptr;
   size_t attn_bytes = 0, attn_layers = 1;
   float* d_attn_sink = nullptr;

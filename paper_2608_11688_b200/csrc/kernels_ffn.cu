@@ -279,6 +279,23 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     s_off[N] = acc;  // routed pairs
     const int n_pairs = acc + (p.run_shared ? B : 0);
     p.n_pairs[0] = n_pairs;
+    // groups for the tensor-core path: one per executed expert, then the shared expert
+    int ng = 0;
+    for (int f = 0; f < N; ++f)
+      if (s_count[f] > 0) {
+        p.grp[4 + 3 * ng] = f;
+        p.grp[5 + 3 * ng] = s_off[f];
+        p.grp[6 + 3 * ng] = s_count[f];
+        ++ng;
+      }
+    p.grp[0] = ng;
+    if (p.run_shared) {
+      p.grp[4 + 3 * ng] = N;
+      p.grp[5 + 3 * ng] = acc;
+      p.grp[6 + 3 * ng] = B;
+      ++ng;
+    }
+    p.grp[1] = ng;
   }
   __syncthreads();
   if (e < N && s_count[e] > 0) {

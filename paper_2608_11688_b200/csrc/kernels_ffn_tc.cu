@@ -1,0 +1,458 @@
+// Batched expert FFN on the 5th-generation tensor cores (tcgen05 + TMEM), for decode steps with many
+// tokens (Sec. V-B: the method "supports batching multiple concurrent requests").
+//
+// With B tokens per step an expert serves several tokens, so its weights should be read once and
+// applied to all of them: a grouped GEMM, one group per executed expert (plus the shared expert).
+// The step is still HBM-bound (a few tens of flop per weight byte at most), so the kernels are
+// organised around streaming the weights once; the tensor cores only keep arithmetic off the
+// critical path.  "Swap-AB": the weight rows are the MMA's M dimension (128 per tile), the group's
+// tokens are N (16..256), so a small token count does not waste a 128-row tile.
+//
+//   gather     X_g[pair][d] (bf16) = h'[token of pair]   (pairs are sorted by expert); zero y
+//   gate/up    G, U [128 x n] = W_gate/up[128 rows of I x d] . X_g^T       accumulators in TMEM
+//              a = g_pair * silu(G) * U  (fp32) is kept as TWO bf16 planes, a_hi = bf16(a) and
+//              a_lo = bf16(a - a_hi), so feeding it back to the tensor cores loses 2^-17, not 2^-9
+//                                                                            -> global scratch (L2)
+//   down       D [128 cols of d x n] = downT[I x 128]^T . (a_hi + a_lo)^T   (downT is MN-major)
+//              y[token][col] += D                                            fp32 atomics
+//              (at most 128 tokens per unit here; larger groups are split)
+//
+// Operands reach shared memory through TMA tensor maps with the 128-byte swizzle and are consumed
+// by tcgen05.mma through shared-memory descriptors (K-major for gate, up, X, A; MN-major for downT).
+// One CTA per SM, three roles: one thread issues TMA loads, one thread issues MMAs, four warps run
+// the epilogue out of TMEM.  Every wait is bounded.
+#include <cuda.h>
+#include <cuda_bf16.h>
+
+#include "apex_internal.hpp"
+
+namespace apex {
+
+namespace {
+
+constexpr int kTcThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int kKTile = 64;       // K elements per pipeline stage (128 bytes: one swizzle span)
+constexpr int kXRowsPerLoad = 32;
+
+__device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ unsigned long long gtimer() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t c) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(b)), "r"(c) : "memory");
+}
+__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
+  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(b)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
+  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(b)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
+  uint32_t ok;
+  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0,1,0,p;\n}"
+               : "=r"(ok)
+               : "r"(s32(b)), "r"(parity)
+               : "memory");
+  return ok != 0;
+}
+// Bounded: false when the limit ran out or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, const volatile int* abort_flag, long long limit_ns) {
+  if (mbar_try(b, parity)) return true;
+  const unsigned long long t0 = gtimer();
+  for (uint32_t it = 1;; ++it) {
+    if (mbar_try(b, parity)) return true;
+    if ((it & 255u) == 0u) {
+      if (*abort_flag) return false;
+      if ((long long)(gtimer() - t0) > limit_ns) return false;
+    }
+  }
+}
+__device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t* bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(s32(dst)),
+      "l"(map), "r"(s32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(s32(dst)),
+               "l"(map), "r"(s32(bar)), "r"(c0), "r"(c1)
+               : "memory");
+}
+// shared-memory matrix descriptor, 128-byte swizzle (layout type 2), version 1
+__device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
+  uint64_t d = 0;
+  d |= (uint64_t)((saddr >> 4) & 0x3FFF);
+  d |= (uint64_t)((lbo_bytes >> 4) & 0x3FFF) << 16;
+  d |= (uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32;
+  d |= (uint64_t)1 << 46;
+  d |= (uint64_t)2 << 61;
+  return d;
+}
+// instruction descriptor: bf16 x bf16 -> fp32, M x N, optional MN-major A
+__device__ __forceinline__ uint32_t umma_idesc(int M, int N, int a_mn_major) {
+  uint32_t d = 0;
+  d |= 1u << 4;    // D fp32
+  d |= 1u << 7;    // A bf16
+  d |= 1u << 10;   // B bf16
+  d |= (uint32_t)a_mn_major << 15;
+  d |= (uint32_t)(N >> 3) << 17;
+  d |= (uint32_t)(M >> 4) << 24;
+  return d;
+}
+__device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+  asm volatile("{\n.reg .pred p;\nsetp.ne.b32 p, %4, 0;\ntcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n}" ::"r"(tmem_d),
+               "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+               : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t* bar) {
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s32(bar)) : "memory");
+}
+__device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+      "{%0,%1,%2,%3,%4,%5,%6,%7,%8,%9,%10,%11,%12,%13,%14,%15,%16,%17,%18,%19,%20,%21,%22,%23,%24,%25,%26,%27,%28,%29,%30,%31}, [%32];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]), "=r"(r[9]),
+        "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]), "=r"(r[16]), "=r"(r[17]), "=r"(r[18]),
+        "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]), "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]),
+        "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+      : "r"(taddr)
+      : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ uint32_t ld_acquire_sys_u32(const uint32_t* p) {
+  uint32_t v;
+  asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+
+struct Group {
+  int expert, pair_off, n_tok;
+};
+__device__ __forceinline__ Group load_group(const int32_t* grp, int g) {
+  Group r;
+  r.expert = grp[4 + 3 * g];
+  r.pair_off = grp[5 + 3 * g];
+  r.n_tok = grp[6 + 3 * g];
+  return r;
+}
+
+}  // namespace
+
+// ---------------------------------------------------------------- gather + zero
+__global__ void __launch_bounds__(256) ffn_tc_gather_kernel(const TcParams p) {
+  const int n_pairs = p.f.n_pairs[0];
+  const int d = p.f.d;
+  if (!p.f.accumulate) {
+    float4* y4 = reinterpret_cast<float4*>(p.f.y);
+    const size_t n4 = (size_t)p.f.B * d / 4;
+    for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n4; i += (size_t)gridDim.x * blockDim.x)
+      y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
+  }
+  for (int pr = blockIdx.x; pr < n_pairs; pr += gridDim.x) {
+    const int t = p.f.pair_tok[pr];
+    const float4* src = reinterpret_cast<const float4*>(p.f.hpost + (size_t)t * d);
+    uint2* dst = reinterpret_cast<uint2*>(p.xg + (size_t)pr * d);
+    for (int c = threadIdx.x; c < d / 4; c += blockDim.x) {
+      const float4 v = __ldg(src + c);
+      __nv_bfloat162 lo = __floats2bfloat162_rn(v.x, v.y), hi = __floats2bfloat162_rn(v.z, v.w);
+      uint2 o;
+      o.x = *reinterpret_cast<uint32_t*>(&lo);
+      o.y = *reinterpret_cast<uint32_t*>(&hi);
+      dst[c] = o;
+    }
+  }
+}
+
+// ---------------------------------------------------------------- the two GEMM kernels
+// PHASE 1: gate/up.  A tiles: gate and up rows [128 x 64] (K-major), B tile: X_g rows [<=256 x 64].
+// PHASE 2: down.     A tile: downT [64 k-rows x 128 cols] as two 64-column atoms (MN-major), B tile: A rows [<=256 x 64].
+template <int PHASE>
+__global__ void __launch_bounds__(kTcThreads, 1)
+ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_ws,
+                   const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_b2, const TcParams p) {
+  extern __shared__ __align__(1024) uint8_t smem_raw[];
+  uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
+  constexpr int A_BYTES = PHASE == 1 ? 2 * 128 * 128 : 2 * 64 * 128;  // gate+up tiles | two downT atoms
+  constexpr int NMAX = PHASE == 1 ? 256 : 128;                        // tokens per unit
+  constexpr int B_PLANE = NMAX * 128;                                 // one B tile
+  constexpr int B_BYTES = PHASE == 1 ? B_PLANE : 2 * B_PLANE;         // X | a_hi and a_lo
+  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
+  constexpr int NSTAGE = PHASE == 1 ? 3 : 4;
+  __shared__ uint64_t full[NSTAGE], empty[NSTAGE], tmem_full, tmem_empty;
+  __shared__ uint32_t tmem_base_s;
+  __shared__ int s_abort;
+
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int N = p.f.N, d = p.f.d, I = p.f.I, I_s = p.f.I_shared;
+  const int32_t* grp = p.grp;
+
+  if (tid == 0) {
+    s_abort = 0;
+    for (int s = 0; s < NSTAGE; ++s) {
+      mbar_init(&full[s], 1);
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(&tmem_full, 1);
+    mbar_init(&tmem_empty, 128);
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_ws) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b2) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&tmem_base_s)), "r"(512) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = tmem_base_s;
+
+  const int n_rg = grp[0], n_g = grp[1];
+  const int blocks_r = PHASE == 1 ? I / 128 : d / 128;                       // M blocks of a routed group
+  const int blocks_s = PHASE == 1 ? (I_s > 0 ? I_s / 128 : 0) : d / 128;     // ... of the shared group
+  const int kdim_r = PHASE == 1 ? d : I, kdim_s = PHASE == 1 ? d : I_s;
+  // PHASE 2 handles at most NMAX tokens per unit: a group of n tokens is cut into ceil(n / NMAX) parts
+  const int sub_max = PHASE == 1 ? 1 : (p.f.B + NMAX - 1) / NMAX;
+  const int base_units = n_rg * blocks_r + (n_g - n_rg) * blocks_s;
+  const int n_units = base_units * sub_max;
+
+  uint32_t it_load = 0, it_mma = 0;  // running K-tile counters of the producer and of the MMA thread
+  uint32_t unit_no = 0;              // units done by this CTA (phase of the TMEM barriers)
+  for (int uu = blockIdx.x; uu < n_units; uu += gridDim.x) {
+    const int u = uu % base_units, sub = uu / base_units;  // the (mostly empty) second parts come last
+    int g, blk;
+    if (u < n_rg * blocks_r) {
+      g = u / blocks_r;
+      blk = u % blocks_r;
+    } else {
+      g = n_rg + (u - n_rg * blocks_r) / blocks_s;
+      blk = (u - n_rg * blocks_r) % blocks_s;
+    }
+    Group gr = load_group(grp, g);
+    if (sub * NMAX >= gr.n_tok) continue;  // this part of the group is empty (uniform over the CTA)
+    gr.pair_off += sub * NMAX;
+    gr.n_tok = gr.n_tok - sub * NMAX < NMAX ? gr.n_tok - sub * NMAX : NMAX;
+    const bool shared = gr.expert >= N;
+    const int kdim = shared ? kdim_s : kdim_r;
+    const int n_kt = kdim / kKTile;
+    const int n_pad = (gr.n_tok + 15) & ~15;                                  // MMA N
+    const int n_loads = (gr.n_tok + kXRowsPerLoad - 1) / kXRowsPerLoad;       // 32-row boxes of the B tile
+
+    if (warp == 0) {
+      // ================= TMA producer
+      if (lane == 0) {
+        int slot = 0;
+        bool ok = true;
+        if (!shared) {
+          slot = p.f.snap.expert_slot[gr.expert];
+          if (slot < 0) ok = false;
+          if (ok) {
+            const uint32_t need = p.f.snap.need_gen[gr.expert];
+            const uint32_t* flag = p.f.slot_ready + slot;
+            if ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
+              const unsigned long long t0 = gtimer();
+              while ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
+                if ((long long)(gtimer() - t0) > p.f.wait_limit_ns) {
+                  ok = false;
+                  break;
+                }
+                __nanosleep(64);
+              }
+              if (p.f.stats) atomicAdd(&p.f.stats->stall_ns, (gtimer() - t0) * (unsigned long long)gridDim.x / 4ull);
+            }
+            asm volatile("fence.proxy.async;" ::: "memory");
+            slot += p.layer_slot0;  // the tensor map covers the slots of all layers
+          }
+        }
+        const CUtensorMap* wmap = shared ? &tm_ws : &tm_w;
+        for (int kt = 0; kt < n_kt && ok; ++kt, ++it_load) {
+          const int s = it_load % NSTAGE;
+          if (it_load >= (uint32_t)NSTAGE && !mbar_wait(&empty[s], ((it_load / NSTAGE) - 1) & 1, &s_abort, p.f.wait_limit_ns)) {
+            ok = false;
+            break;
+          }
+          uint8_t* st = smem + (size_t)s * STAGE_BYTES;
+          mbar_expect_tx(&full[s], A_BYTES + (PHASE == 1 ? 1 : 2) * n_loads * kXRowsPerLoad * 128);
+          if (PHASE == 1) {
+            tma_load_4d(st, wmap, kt * kKTile, 0, blk * 128, slot, &full[s]);               // gate rows
+            tma_load_4d(st + 128 * 128, wmap, kt * kKTile, 1, blk * 128, slot, &full[s]);   // up rows
+          } else {
+            tma_load_4d(st, wmap, blk * 128, 2, kt * kKTile, slot, &full[s]);               // downT, columns 0..63
+            tma_load_4d(st + 64 * 128, wmap, blk * 128 + 64, 2, kt * kKTile, slot, &full[s]);
+          }
+          for (int r = 0; r < n_loads; ++r) {
+            tma_load_2d(st + A_BYTES + r * kXRowsPerLoad * 128, &tm_b, kt * kKTile, gr.pair_off + r * kXRowsPerLoad, &full[s]);
+            if (PHASE == 2)
+              tma_load_2d(st + A_BYTES + B_PLANE + r * kXRowsPerLoad * 128, &tm_b2, kt * kKTile, gr.pair_off + r * kXRowsPerLoad, &full[s]);
+          }
+        }
+        if (!ok) {
+          atomicExch(&s_abort, 1);
+          *p.f.mbox_status = 1u;
+          if (p.f.stats) atomicAdd(&p.f.stats->timeouts, 1ull);
+        }
+      }
+    } else if (warp == 1) {
+      // ================= MMA issuer
+      if (lane == 0) {
+        bool ok = true;
+        if (unit_no > 0) ok = mbar_wait(&tmem_empty, (unit_no - 1) & 1, &s_abort, p.f.wait_limit_ns);
+        tc_fence_after();
+        const uint32_t idesc = umma_idesc(128, n_pad, PHASE == 2 ? 1 : 0);
+        for (int kt = 0; kt < n_kt && ok; ++kt, ++it_mma) {
+          const int s = it_mma % NSTAGE;
+          if (!mbar_wait(&full[s], (it_mma / NSTAGE) & 1, &s_abort, p.f.wait_limit_ns)) {
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t a0 = s32(smem + (size_t)s * STAGE_BYTES);
+          const uint32_t b0 = a0 + A_BYTES;
+#pragma unroll
+          for (int ks = 0; ks < kKTile / 16; ++ks) {
+            const uint32_t acc = (kt > 0 || ks > 0) ? 1u : 0u;
+            const uint64_t bdesc = umma_desc(b0 + ks * 32, 16, 1024);
+            if (PHASE == 1) {
+              umma(tmem_base, umma_desc(a0 + ks * 32, 16, 1024), bdesc, idesc, acc);                     // G
+              umma(tmem_base + 256, umma_desc(a0 + 128 * 128 + ks * 32, 16, 1024), bdesc, idesc, acc);   // U
+            } else {
+              const uint64_t adesc = umma_desc(a0 + ks * 2048, 64 * 128, 1024);
+              umma(tmem_base, adesc, bdesc, idesc, acc);                                           // a_hi
+              umma(tmem_base, adesc, umma_desc(b0 + B_PLANE + ks * 32, 16, 1024), idesc, 1u);     // a_lo
+            }
+          }
+          umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
+        }
+        if (ok) umma_commit(&tmem_full);
+        else atomicExch(&s_abort, 1);
+      }
+    } else {
+      // ================= epilogue: warp w owns TMEM lanes 32*(w%4) .. +31
+      const int quad = warp & 3;
+      const int row = quad * 32 + lane;  // row of the 128-row tile
+      if (__all_sync(0xffffffffu, mbar_wait(&tmem_full, unit_no & 1, &s_abort, p.f.wait_limit_ns))) {
+        tc_fence_after();
+        for (int c0 = 0; c0 < gr.n_tok; c0 += 32) {
+          uint32_t a[32];
+          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0;
+          tmem_ld32(taddr, a);
+          if (PHASE == 1) {
+            uint32_t b2[32];
+            tmem_ld32(taddr + 256, b2);
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int i = blk * 128 + row;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (c0 + j < gr.n_tok) {
+                const float gq = __uint_as_float(a[j]), uq = __uint_as_float(b2[j]);
+                const float w = __ldg(p.f.pair_gate + gr.pair_off + c0 + j);
+                const float v = w * (gq / (1.f + expf(-gq))) * uq;
+                const __nv_bfloat16 hi = __float2bfloat16(v);
+                const size_t at = (size_t)(gr.pair_off + c0 + j) * p.act_stride + i;
+                p.act[at] = hi;
+                p.act[p.act_plane + at] = __float2bfloat16(v - __bfloat162float(hi));
+              }
+            }
+          } else {
+            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
+            const int col = blk * 128 + row;
+#pragma unroll
+            for (int j = 0; j < 32; ++j) {
+              if (c0 + j < gr.n_tok) {
+                const int t = __ldg(p.f.pair_tok + gr.pair_off + c0 + j);
+                atomicAdd(p.f.y + (size_t)t * d + col, __uint_as_float(a[j]));
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before();
+      mbar_arrive(&tmem_empty);
+    }
+    ++unit_no;
+    if (*(volatile int*)&s_abort) break;
+  }
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+}
+
+// ---------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,
+                                  const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave, CUtensorMapSwizzle,
+                                  CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  if (!fn) {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult qr;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &qr) == cudaSuccess && qr == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+    cudaGetLastError();
+  }
+  return fn;
+}
+
+// Weights of n_slots consecutive slots, each [I][3][d] bf16: dims (d, 3, I, n_slots); box (64, 1, box_rows, 1).
+bool tc_make_weight_map(void* out, const void* base, int d, int I, size_t n_slots, size_t slot_bytes, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[4] = {(cuuint64_t)d, 3, (cuuint64_t)I, (cuuint64_t)n_slots};
+  cuuint64_t strides[3] = {(cuuint64_t)d * 2, (cuuint64_t)d * 6, (cuuint64_t)slot_bytes};
+  cuuint32_t box[4] = {64, 1, (cuuint32_t)box_rows, 1};
+  cuuint32_t es[4] = {1, 1, 1, 1};
+  return fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Row-major bf16 matrix [rows][cols] with row stride `stride_elems`: dims (cols, rows); box (64, 32).
+bool tc_make_rows_map(void* out, const void* base, int cols, size_t rows, size_t stride_elems) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[2] = {(cuuint64_t)cols, (cuuint64_t)rows};
+  cuuint64_t strides[1] = {(cuuint64_t)stride_elems * 2};
+  cuuint32_t box[2] = {64, kXRowsPerLoad};
+  cuuint32_t es[2] = {1, 1};
+  return fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+bool tc_shape_supported(int d, int I, int I_shared) {
+  return d % 128 == 0 && I % 128 == 0 && I_shared % 128 == 0;
+}
+
+cudaError_t launch_ffn_tc(const TcParams& p, const TcMaps& m, int n_sm, cudaStream_t s) {
+  static bool configured = false;
+  const size_t smem1 = 3 * (2 * 128 * 128 + 256 * 128) + 1024, smem2 = 4 * (2 * 64 * 128 + 2 * 128 * 128) + 1024;
+  if (!configured) {
+    cudaError_t e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
+    if (e != cudaSuccess) return e;
+    e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    if (e != cudaSuccess) return e;
+    configured = true;
+  }
+  ffn_tc_gather_kernel<<<n_sm * 2, 256, 0, s>>>(p);
+  cudaError_t e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  const CUtensorMap* w1 = reinterpret_cast<const CUtensorMap*>(m.w_gateup);
+  const CUtensorMap* ws1 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_gateup : m.w_gateup);
+  const CUtensorMap* w2 = reinterpret_cast<const CUtensorMap*>(m.w_down);
+  const CUtensorMap* ws2 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_down : m.w_down);
+  const CUtensorMap* xg = reinterpret_cast<const CUtensorMap*>(m.xg);
+  ffn_tc_gemm_kernel<1><<<n_sm, kTcThreads, smem1, s>>>(*w1, *ws1, *xg, *xg, p);
+  e = cudaGetLastError();
+  if (e != cudaSuccess) return e;
+  ffn_tc_gemm_kernel<2><<<n_sm, kTcThreads, smem2, s>>>(*w2, *ws2, *reinterpret_cast<const CUtensorMap*>(m.act),
+                                                        *reinterpret_cast<const CUtensorMap*>(m.act_lo), p);
+  return cudaGetLastError();
+}
+
+}  // namespace apex

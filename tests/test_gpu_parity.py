@@ -94,6 +94,16 @@ def test_batched_tokens(B, mode):
     assert stats["tokens"] == 5 * B
 
 
+@pytest.mark.parametrize("B", [16, 40, 97])
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_batched_tensor_core_path(B, mode):
+    # shapes the tcgen05 grouped GEMM accepts (d, I, I_shared multiples of 128), B >= 16
+    cfg = synth.tiny_config(d=256, N=12, k=3, I=128, C=8, T=3, I_shared=256, sigma_p=1.0, cfg_id=230)
+    rep, stats = _run(cfg, mode=mode, tau=0.8, T=3, B=B)
+    assert stats["tokens"] == 3 * B and rep.ffn_checked + rep.near_ties >= 1
+    print("tc", B, mode, rep)
+
+
 def test_batched_exact_mode_runs_in_waves_when_cache_is_smaller_than_need():
     cfg = synth.tiny_config(d=256, N=16, k=4, I=16, C=5, T=4, cfg_id=217)
     rep, stats = _run(cfg, mode="exact", tau=0.5, T=4, B=8)

@@ -269,6 +269,7 @@ def main():
     ap.add_argument("--ffn-only", action="store_true",
                     help="profiling case: all experts resident, gate + expert FFN only, no copy in flight")
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (smaller captures)")
+    ap.add_argument("--batch", type=int, default=1, help="tokens per decode step (config 4 sweeps 1, 8, 32, 128, 256)")
     ap.add_argument("--resident", action="store_true",
                     help="cache as large as the expert count, warmed up: no host-link copies (kernel launch lists)")
     args = ap.parse_args()
@@ -301,7 +302,7 @@ def main():
         dist.init_process_group("nccl", device_id=dev)
         dist.barrier()
         dist_sync = dist.barrier
-    B = 1
+    B = args.batch
     prob = build_problem(cfg, dev)
     T = min(cfg.T, args.warmup + args.steps)
     h, hp = hidden_inputs(cfg, T, B, dev)
@@ -311,12 +312,18 @@ def main():
     y_pin = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32).pin_memory()
 
     if args.ffn_only:
-        a = make_ctx(cfg, prob, cfg.N)
+        a = make_ctx(cfg, prob, cfg.N, max_batch=B)
         a.warm_all()
         mean_s, med_s, n_l = time_ffn_kernel(a, cfg, h_dev, hp_dev, B, tokens=args.steps)
-        _, bytes_ffn = algorithmic_bytes(cfg, B)
-        print(json.dumps({"ffn_only": True, "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6,
-                          "launches": n_l, "GBps_mean": bytes_ffn / mean_s / 1e9, "bytes_per_launch": bytes_ffn}), flush=True)
+        if B == 1:
+            _, bytes_ffn = algorithmic_bytes(cfg, B)
+        else:   # expected number of distinct experts touched by B tokens with uniform routing
+            distinct = cfg.N * (1.0 - (1.0 - cfg.k / cfg.N) ** B)
+            bytes_ffn = distinct * cfg.expert_bytes + cfg.shared_bytes + 2 * B * cfg.d * 4
+        flops = 2.0 * 3 * cfg.d * (cfg.k * cfg.I + cfg.I_shared) * B
+        print(json.dumps({"ffn_only": True, "B": B, "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6,
+                          "launches": n_l, "GBps_mean": bytes_ffn / mean_s / 1e9, "bytes_per_launch": bytes_ffn,
+                          "TFLOPs": flops / mean_s / 1e12}), flush=True)
         a.destroy()
         return
 

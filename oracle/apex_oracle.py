@@ -323,9 +323,11 @@ class SlotCache:
 def layer_step(cache: SlotCache, *, W_p, b_p, W_r, b_r, w, theta, tau: float, k: int,
                h: np.ndarray, h_post: np.ndarray, mode: str,
                expert_weights: Optional[Callable] = None, shared=None,
-               norm_topk: bool = True, compute_ffn: bool = True) -> Dict:
+               norm_topk: bool = True, compute_ffn: bool = True, ffn_tokens: Optional[Sequence[int]] = None) -> Dict:
     """h, h_post: [B][d].  mode: 'exact' (correctness-preserving) or 'stall_free'.
-    Returns every decision of the step, with the margins needed to flag near-ties."""
+    Returns every decision of the step, with the margins needed to flag near-ties.
+    ffn_tokens limits the (slow) FFN evaluation to some tokens of the batch; decisions are always
+    computed for all."""
     B = h.shape[0]
     N = np.asarray(W_r).shape[0]
     out: Dict = {"B": B, "tokens": []}
@@ -384,6 +386,6 @@ def layer_step(cache: SlotCache, *, W_p, b_p, W_r, b_r, w, theta, tau: float, k:
         raise ValueError(mode)
     for b, tok in enumerate(out["tokens"]):
         tok["gates"] = gates(tok["alpha"], tok["K_exec"], norm_topk)
-        if compute_ffn and expert_weights is not None:
+        if compute_ffn and expert_weights is not None and (ffn_tokens is None or b in ffn_tokens):
             tok["y"] = moe_output(h_post[b], tok["K_exec"], tok["gates"], expert_weights, shared)
     return out

@@ -153,6 +153,8 @@ struct TcParams {
   size_t act_plane;     // elements per plane
   int act_stride;
   int layer_slot0;      // index of this layer's slot 0 in the all-layers weight tensor map
+  int nmax1, nmax2;     // tokens per unit of the gate/up and of the down kernel (set by the launcher)
+  int nstage1, nstage2; // pipeline depths
 };
 struct TcMaps {          // opaque 128-byte CUtensorMap objects
   alignas(64) unsigned char w_gateup[128], w_down[128], ws_gateup[128], ws_down[128], xg[128], act[128], act_lo[128];

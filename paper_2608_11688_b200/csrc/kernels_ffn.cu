@@ -227,8 +227,12 @@ __device__ __forceinline__ void store_token_plan(const TokenPlan& tp, int lane, 
 }
 
 // ---------------------------------------------------------------- batched plan (B > 1)
-// One CTA.  Warps plan tokens; then thread e gathers the tokens that execute expert e, so the pair
-// list is sorted by (expert, token).  Shared-expert pairs (expert id N) follow.
+// One CTA of 32 warps.  Phase A: warp w plans tokens w, w+32, ... (all global loads of a warp's tokens
+// are issued before the first use).  Phase B: warp w owns experts w and w+32 and gathers the tokens
+// that execute them with ballots, so the pair list is sorted by (expert, token).  Shared-expert pairs
+// (expert id N) follow.
+constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;
+
 __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   __shared__ unsigned long long s_exec[APEX_MAX_BATCH];
   __shared__ int s_count[APEX_MAX_EXPERTS + 1];
@@ -236,8 +240,17 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
   const int N = p.N, k = p.k, B = p.B;
   int my_subst = 0, my_hits = 0;
-  for (int b = warp; b < B; b += nwarp) {
-    const TokenLoads tl = load_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode, lane);
+  TokenLoads tls[kPlanMaxTokPerWarp];
+#pragma unroll
+  for (int j = 0; j < kPlanMaxTokPerWarp; ++j) {
+    const int b = warp + j * nwarp;
+    if (b < B) tls[j] = load_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode, lane);
+  }
+#pragma unroll
+  for (int j = 0; j < kPlanMaxTokPerWarp; ++j) {
+    const int b = warp + j * nwarp;
+    if (b >= B) break;
+    const TokenLoads& tl = tls[j];
     const TokenPlan tp = plan_token(tl, p.mode, p.norm_topk, p.snap.resident_mask, lane);
     store_token_plan(tp, lane, k, p.plan_exec_idx + (size_t)b * k, p.plan_exec_gate + (size_t)b * k,
                      p.post_exec ? p.mbox_exec + (size_t)b * k : nullptr);
@@ -262,12 +275,15 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   if (p.post_exec && lane == 0 && my_subst && p.stats) atomicAdd(&p.stats->substitutions, (unsigned long long)my_subst);
   if (p.post_exec && lane == 0 && my_hits && p.stats) atomicAdd(&p.stats->hits_R, (unsigned long long)my_hits);
   __syncthreads();
-  const int e = threadIdx.x;
-  if (e < N) {
+  // ---- phase B, counts: warp w counts the tokens of experts w and w + 32
+  for (int e = warp; e < N; e += nwarp) {
     int c = 0;
     if ((p.run_mask >> e) & 1)
-      for (int b = 0; b < B; ++b) c += (int)((s_exec[b] >> e) & 1);
-    s_count[e] = c;
+      for (int b0 = 0; b0 < B; b0 += 32) {
+        const int b = b0 + lane;
+        c += __popc(__ballot_sync(0xffffffffu, b < B && ((s_exec[b] >> e) & 1)));
+      }
+    if (lane == 0) s_count[e] = c;
   }
   __syncthreads();
   if (threadIdx.x == 0) {
@@ -298,16 +314,22 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     p.grp[1] = ng;
   }
   __syncthreads();
-  if (e < N && s_count[e] > 0) {
+  // ---- phase B, placement: token b of expert e goes to s_off[e] + (number of earlier tokens of e)
+  for (int e = warp; e < N; e += nwarp) {
+    if (s_count[e] == 0) continue;
     int o = s_off[e];
-    for (int b = 0; b < B; ++b) {
-      if ((s_exec[b] >> e) & 1) {
+    for (int b0 = 0; b0 < B; b0 += 32) {
+      const int b = b0 + lane;
+      const bool has = b < B && ((s_exec[b] >> e) & 1);
+      const unsigned m = __ballot_sync(0xffffffffu, has);
+      if (has) {
+        const int at = o + __popc(m & ((1u << lane) - 1u));
         const int pos = __popcll(s_exec[b] & ((1ull << e) - 1ull));
-        p.pair_tok[o] = b;
-        p.pair_expert[o] = e;
-        p.pair_gate[o] = p.plan_exec_gate[(size_t)b * k + pos];
-        ++o;
+        p.pair_tok[at] = b;
+        p.pair_expert[at] = e;
+        p.pair_gate[at] = p.plan_exec_gate[(size_t)b * k + pos];
       }
+      o += __popc(m);
     }
   }
   if (p.run_shared) {

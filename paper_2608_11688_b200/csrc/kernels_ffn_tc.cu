@@ -19,8 +19,9 @@
 //
 // Operands reach shared memory through TMA tensor maps with the 128-byte swizzle and are consumed
 // by tcgen05.mma through shared-memory descriptors (K-major for gate, up, X, A; MN-major for downT).
-// One CTA per SM, three roles: one thread issues TMA loads, one thread issues MMAs, four warps run
-// the epilogue out of TMEM.  Every wait is bounded.
+// One CTA per SM, three roles: two warps issue TMA loads (alternating K tiles; a single issuing
+// thread cannot keep up with 16 KB tiles), one thread issues MMAs, four warps run the epilogue out
+// of TMEM.  Every wait is bounded.
 #include <cuda.h>
 #include <cuda_bf16.h>
 
@@ -30,7 +31,9 @@ namespace apex {
 
 namespace {
 
-constexpr int kTcThreads = 192;  // warp 0: TMA, warp 1: MMA + TMEM owner, warps 2..5: epilogue
+constexpr int kProducerWarps = 2;  // TMA producers: K tile t is loaded by warp t mod 2
+constexpr int kMmaWarp = kProducerWarps;
+constexpr int kTcThreads = (kProducerWarps + 1 + 4) * 32;  // producers, MMA + TMEM owner, four epilogue warps
 constexpr int kKTile = 64;       // K elements per pipeline stage (128 bytes: one swizzle span)
 constexpr int kXRowsPerLoad = 32;
 
@@ -176,14 +179,18 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   constexpr int A_BYTES = PHASE == 1 ? 2 * 128 * 128 : 2 * 64 * 128;  // gate+up tiles | two downT atoms
-  constexpr int NMAX = PHASE == 1 ? 256 : 128;                        // tokens per unit
-  constexpr int B_PLANE = NMAX * 128;                                 // one B tile
-  constexpr int B_BYTES = PHASE == 1 ? B_PLANE : 2 * B_PLANE;         // X | a_hi and a_lo
-  constexpr int STAGE_BYTES = A_BYTES + B_BYTES;
-  constexpr int NSTAGE = PHASE == 1 ? 3 : 4;
-  __shared__ uint64_t full[NSTAGE], empty[NSTAGE], tmem_full, tmem_empty;
+  constexpr int PLANES = PHASE == 1 ? 1 : 2;                          // X | a_hi and a_lo
+  constexpr int MAX_STAGES = 8;
+  // Tokens per unit (NMAX), hence the size of a B tile and the pipeline depth, are chosen per launch:
+  // small batches get deep pipelines (more weight bytes in flight), large groups are cut into parts.
+  const int NMAX = PHASE == 1 ? p.nmax1 : p.nmax2;
+  const int B_PLANE = NMAX * 128;
+  const int STAGE_BYTES = A_BYTES + PLANES * B_PLANE;
+  const int NSTAGE = PHASE == 1 ? p.nstage1 : p.nstage2;
+  __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full, tmem_empty;
   __shared__ uint32_t tmem_base_s;
   __shared__ int s_abort;
+  __shared__ int s_ustart[APEX_MAX_EXPERTS + 3];  // first unit of each group
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = p.f.N, d = p.f.d, I = p.f.I, I_s = p.f.I_shared;
@@ -191,7 +198,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
 
   if (tid == 0) {
     s_abort = 0;
-    for (int s = 0; s < NSTAGE; ++s) {
+    for (int s = 0; s < MAX_STAGES; ++s) {
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
     }
@@ -203,7 +210,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b2) : "memory");
   }
-  if (warp == 1) {
+  if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&tmem_base_s)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
@@ -216,25 +223,29 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   const int blocks_r = PHASE == 1 ? I / 128 : d / 128;                       // M blocks of a routed group
   const int blocks_s = PHASE == 1 ? (I_s > 0 ? I_s / 128 : 0) : d / 128;     // ... of the shared group
   const int kdim_r = PHASE == 1 ? d : I, kdim_s = PHASE == 1 ? d : I_s;
-  // PHASE 2 handles at most NMAX tokens per unit: a group of n tokens is cut into ceil(n / NMAX) parts
-  const int sub_max = PHASE == 1 ? 1 : (p.f.B + NMAX - 1) / NMAX;
-  const int base_units = n_rg * blocks_r + (n_g - n_rg) * blocks_s;
-  const int n_units = base_units * sub_max;
+  // A group of n tokens is cut into ceil(n / NMAX) parts; a unit is (group, M block, part), parts
+  // fastest so that the CTAs that share a weight block run at the same time (second reader hits L2).
+  if (tid == 0) {
+    int acc = 0;
+    for (int g = 0; g < n_g; ++g) {
+      s_ustart[g] = acc;
+      const int parts = (grp[6 + 3 * g] + NMAX - 1) / NMAX;
+      acc += (g < n_rg ? blocks_r : blocks_s) * parts;
+    }
+    s_ustart[n_g] = acc;
+  }
+  __syncthreads();
+  const int n_units = s_ustart[n_g];
 
   uint32_t it_load = 0, it_mma = 0;  // running K-tile counters of the producer and of the MMA thread
   uint32_t unit_no = 0;              // units done by this CTA (phase of the TMEM barriers)
+  int g = 0;
   for (int uu = blockIdx.x; uu < n_units; uu += gridDim.x) {
-    const int u = uu % base_units, sub = uu / base_units;  // the (mostly empty) second parts come last
-    int g, blk;
-    if (u < n_rg * blocks_r) {
-      g = u / blocks_r;
-      blk = u % blocks_r;
-    } else {
-      g = n_rg + (u - n_rg * blocks_r) / blocks_s;
-      blk = (u - n_rg * blocks_r) % blocks_s;
-    }
+    while (uu >= s_ustart[g + 1]) ++g;
     Group gr = load_group(grp, g);
-    if (sub * NMAX >= gr.n_tok) continue;  // this part of the group is empty (uniform over the CTA)
+    const int parts = (gr.n_tok + NMAX - 1) / NMAX;
+    const int local = uu - s_ustart[g];
+    const int blk = local / parts, sub = local % parts;
     gr.pair_off += sub * NMAX;
     gr.n_tok = gr.n_tok - sub * NMAX < NMAX ? gr.n_tok - sub * NMAX : NMAX;
     const bool shared = gr.expert >= N;
@@ -243,61 +254,66 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     const int n_pad = (gr.n_tok + 15) & ~15;                                  // MMA N
     const int n_loads = (gr.n_tok + kXRowsPerLoad - 1) / kXRowsPerLoad;       // 32-row boxes of the B tile
 
-    if (warp == 0) {
-      // ================= TMA producer
-      if (lane == 0) {
-        int slot = 0;
-        bool ok = true;
-        if (!shared) {
-          slot = p.f.snap.expert_slot[gr.expert];
-          if (slot < 0) ok = false;
-          if (ok) {
-            const uint32_t need = p.f.snap.need_gen[gr.expert];
-            const uint32_t* flag = p.f.slot_ready + slot;
-            if ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
-              const unsigned long long t0 = gtimer();
-              while ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
-                if ((long long)(gtimer() - t0) > p.f.wait_limit_ns) {
-                  ok = false;
-                  break;
-                }
-                __nanosleep(64);
+    if (warp < kProducerWarps) {
+      // ================= TMA producers: the whole warp walks the K tiles; lane 0 owns the barriers and
+      // each load of a stage is issued by a different lane (one thread sustains only about one bulk
+      // copy per 570 cycles)
+      int slot = 0;
+      bool ok = true;
+      if (!shared) {
+        slot = p.f.snap.expert_slot[gr.expert];
+        if (slot < 0) ok = false;
+        if (ok && lane == 0) {
+          const uint32_t need = p.f.snap.need_gen[gr.expert];
+          const uint32_t* flag = p.f.slot_ready + slot;
+          if ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
+            const unsigned long long t0 = gtimer();
+            while ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
+              if ((long long)(gtimer() - t0) > p.f.wait_limit_ns) {
+                ok = false;
+                break;
               }
-              if (p.f.stats) atomicAdd(&p.f.stats->stall_ns, (gtimer() - t0) * (unsigned long long)gridDim.x / 4ull);
+              __nanosleep(64);
             }
-            asm volatile("fence.proxy.async;" ::: "memory");
-            slot += p.layer_slot0;  // the tensor map covers the slots of all layers
+            if (p.f.stats) atomicAdd(&p.f.stats->stall_ns, (gtimer() - t0) * (unsigned long long)gridDim.x / 4ull);
           }
+          asm volatile("fence.proxy.async;" ::: "memory");
         }
-        const CUtensorMap* wmap = shared ? &tm_ws : &tm_w;
-        for (int kt = 0; kt < n_kt && ok; ++kt, ++it_load) {
-          const int s = it_load % NSTAGE;
-          if (it_load >= (uint32_t)NSTAGE && !mbar_wait(&empty[s], ((it_load / NSTAGE) - 1) & 1, &s_abort, p.f.wait_limit_ns)) {
-            ok = false;
-            break;
-          }
-          uint8_t* st = smem + (size_t)s * STAGE_BYTES;
-          mbar_expect_tx(&full[s], A_BYTES + (PHASE == 1 ? 1 : 2) * n_loads * kXRowsPerLoad * 128);
-          if (PHASE == 1) {
-            tma_load_4d(st, wmap, kt * kKTile, 0, blk * 128, slot, &full[s]);               // gate rows
-            tma_load_4d(st + 128 * 128, wmap, kt * kKTile, 1, blk * 128, slot, &full[s]);   // up rows
-          } else {
-            tma_load_4d(st, wmap, blk * 128, 2, kt * kKTile, slot, &full[s]);               // downT, columns 0..63
-            tma_load_4d(st + 64 * 128, wmap, blk * 128 + 64, 2, kt * kKTile, slot, &full[s]);
-          }
-          for (int r = 0; r < n_loads; ++r) {
-            tma_load_2d(st + A_BYTES + r * kXRowsPerLoad * 128, &tm_b, kt * kKTile, gr.pair_off + r * kXRowsPerLoad, &full[s]);
-            if (PHASE == 2)
-              tma_load_2d(st + A_BYTES + B_PLANE + r * kXRowsPerLoad * 128, &tm_b2, kt * kKTile, gr.pair_off + r * kXRowsPerLoad, &full[s]);
-          }
-        }
-        if (!ok) {
-          atomicExch(&s_abort, 1);
-          *p.f.mbox_status = 1u;
-          if (p.f.stats) atomicAdd(&p.f.stats->timeouts, 1ull);
-        }
+        ok = __all_sync(0xffffffffu, ok);
+        slot += p.layer_slot0;  // the tensor map covers the slots of all layers
       }
-    } else if (warp == 1) {
+      const CUtensorMap* wmap = shared ? &tm_ws : &tm_w;
+      constexpr int planes = PLANES;
+      for (int kt = 0; kt < n_kt && ok; ++kt, ++it_load) {
+        if ((int)(it_load % kProducerWarps) != warp) continue;  // the other producer warp's tile
+        const int s = it_load % NSTAGE;
+        if (lane == 0) {
+          if (it_load >= (uint32_t)NSTAGE && !mbar_wait(&empty[s], ((it_load / NSTAGE) - 1) & 1, &s_abort, p.f.wait_limit_ns)) ok = false;
+          if (ok) mbar_expect_tx(&full[s], A_BYTES + planes * n_loads * kXRowsPerLoad * 128);
+        }
+        ok = __all_sync(0xffffffffu, ok);
+        if (!ok) break;
+        uint8_t* st = smem + (size_t)s * STAGE_BYTES;
+        // op 0, 1: the two weight tiles; op 2 + r*planes + pl: 32-row box r of B plane pl
+        const int n_ops = 2 + planes * n_loads;
+        for (int op = lane; op < n_ops; op += 32) {
+          if (op < 2) {
+            if (PHASE == 1) tma_load_4d(st + op * 128 * 128, wmap, kt * kKTile, op, blk * 128, slot, &full[s]);   // gate | up rows
+            else tma_load_4d(st + op * 64 * 128, wmap, blk * 128 + op * 64, 2, kt * kKTile, slot, &full[s]);      // downT, 64 columns
+          } else {
+            const int r = (op - 2) / planes, pl = (op - 2) % planes;
+            tma_load_2d(st + A_BYTES + pl * B_PLANE + r * kXRowsPerLoad * 128, pl ? &tm_b2 : &tm_b, kt * kKTile,
+                        gr.pair_off + r * kXRowsPerLoad, &full[s]);
+          }
+        }
+        __syncwarp();
+      }
+      if (!ok && lane == 0) {
+        atomicExch(&s_abort, 1);
+        *p.f.mbox_status = 1u;
+        if (p.f.stats) atomicAdd(&p.f.stats->timeouts, 1ull);
+      }
+    } else if (warp == kMmaWarp) {
       // ================= MMA issuer
       if (lane == 0) {
         bool ok = true;
@@ -379,7 +395,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   }
   tc_fence_before();
   __syncthreads();
-  if (warp == 1) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  if (warp == kMmaWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
 }
 
 // ---------------------------------------------------------------- host side
@@ -429,16 +445,23 @@ bool tc_shape_supported(int d, int I, int I_shared) {
   return d % 128 == 0 && I % 128 == 0 && I_shared % 128 == 0;
 }
 
-cudaError_t launch_ffn_tc(const TcParams& p, const TcMaps& m, int n_sm, cudaStream_t s) {
+cudaError_t launch_ffn_tc(const TcParams& p_in, const TcMaps& m, int n_sm, cudaStream_t s) {
   static bool configured = false;
-  const size_t smem1 = 3 * (2 * 128 * 128 + 256 * 128) + 1024, smem2 = 4 * (2 * 64 * 128 + 2 * 128 * 128) + 1024;
+  const size_t budget = 196 * 1024;  // ring bytes per CTA
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem1);
+    cudaError_t e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget + 1024);
     if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem2);
+    e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget + 1024);
     if (e != cudaSuccess) return e;
     configured = true;
   }
+  TcParams p = p_in;
+  const int b32 = (p.f.B + 31) & ~31;
+  p.nmax1 = b32 < 128 ? b32 : 128;
+  p.nmax2 = b32 < 64 ? b32 : 64;
+  const size_t st1 = 2 * 128 * 128 + (size_t)p.nmax1 * 128, st2 = 2 * 64 * 128 + 2 * (size_t)p.nmax2 * 128;
+  p.nstage1 = (int)(budget / st1) < 4 ? (int)(budget / st1) : 4;
+  p.nstage2 = (int)(budget / st2) < 4 ? (int)(budget / st2) : 4;
   ffn_tc_gather_kernel<<<n_sm * 2, 256, 0, s>>>(p);
   cudaError_t e = cudaGetLastError();
   if (e != cudaSuccess) return e;
@@ -447,11 +470,11 @@ cudaError_t launch_ffn_tc(const TcParams& p, const TcMaps& m, int n_sm, cudaStre
   const CUtensorMap* w2 = reinterpret_cast<const CUtensorMap*>(m.w_down);
   const CUtensorMap* ws2 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_down : m.w_down);
   const CUtensorMap* xg = reinterpret_cast<const CUtensorMap*>(m.xg);
-  ffn_tc_gemm_kernel<1><<<n_sm, kTcThreads, smem1, s>>>(*w1, *ws1, *xg, *xg, p);
+  ffn_tc_gemm_kernel<1><<<n_sm, kTcThreads, p.nstage1 * st1 + 1024, s>>>(*w1, *ws1, *xg, *xg, p);
   e = cudaGetLastError();
   if (e != cudaSuccess) return e;
-  ffn_tc_gemm_kernel<2><<<n_sm, kTcThreads, smem2, s>>>(*w2, *ws2, *reinterpret_cast<const CUtensorMap*>(m.act),
-                                                        *reinterpret_cast<const CUtensorMap*>(m.act_lo), p);
+  ffn_tc_gemm_kernel<2><<<n_sm, kTcThreads, p.nstage2 * st2 + 1024, s>>>(*w2, *ws2, *reinterpret_cast<const CUtensorMap*>(m.act),
+                                                                        *reinterpret_cast<const CUtensorMap*>(m.act_lo), p);
   return cudaGetLastError();
 }
 

@@ -99,7 +99,7 @@ def _excusable(tok, what: str) -> bool:
 
 def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T: int, B: int = 1,
                  C: Optional[int] = None, norm_topk: bool = True, cache_reuse: bool = True,
-                 check_ffn_every: int = 1, use_prefetch: bool = True, t0: int = 0) -> Report:
+                 check_ffn_every: int = 1, use_prefetch: bool = True, t0: int = 0, ffn_token_stride: int = 1) -> Report:
     cfg = prob.cfg
     C = C or cfg.C
     N, k, d = cfg.N, cfg.k, cfg.d
@@ -139,7 +139,8 @@ def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T:
                 out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=tau, k=k,
                                     h=hs[l][0][t], h_post=hs[l][1][t], mode=mode,
                                     expert_weights=prob.oracle_experts(l), shared=prob.oracle_shared(l),
-                                    norm_topk=norm_topk, compute_ffn=do_ffn)
+                                    norm_topk=norm_topk, compute_ffn=do_ffn,
+                                    ffn_tokens=None if ffn_token_stride == 1 else set(range(0, B, ffn_token_stride)))
             else:   # no prefetch stage: budget 0 candidates are never issued; emulate by an empty prefetch
                 out = _oracle_step_without_prefetch(cache, W_r, b_r, k, hs[l][1][t], mode, prob, l, norm_topk, do_ffn)
             rep.layer_steps += 1
@@ -192,7 +193,7 @@ def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T:
                 np.testing.assert_allclose(g_gate[b], tok["gates"], rtol=2e-5, atol=1e-7)
                 if norm_topk:
                     assert abs(float(g_gate[b].sum()) - 1.0) < 1e-5
-                if do_ffn:
+                if do_ffn and "y" in tok:
                     ref = tok["y"]
                     err = g_y[b].astype(np.float64) - ref
                     rel = float(np.linalg.norm(err) / max(np.linalg.norm(ref), 1e-30))

@@ -14,14 +14,14 @@ def _harness():
 
 
 def _run(cfg, *, mode, tau, T, B=1, layers=None, C=None, norm_topk=1, cache_reuse=1, check_ffn_every=1,
-         use_prefetch=True, prob=None):
+         use_prefetch=True, prob=None, ffn_token_stride=1):
     hz = _harness()
     prob = prob or hz.Problem(cfg, layers=layers)
     apex = prob.make_ctx(C=C, max_batch=B, norm_topk=norm_topk, cache_reuse=cache_reuse)
     try:
         rep = hz.run_lockstep(prob, apex, mode=mode, tau=tau, T=T, B=B, C=C, norm_topk=bool(norm_topk),
                               cache_reuse=bool(cache_reuse), check_ffn_every=check_ffn_every,
-                              use_prefetch=use_prefetch)
+                              use_prefetch=use_prefetch, ffn_token_stride=ffn_token_stride)
         stats = apex.get_stats()
     finally:
         apex.destroy()
@@ -148,6 +148,16 @@ def test_config4_shape_one_layer(B):
     cfg = synth.CONFIGS[4]
     rep, stats = _run(cfg, mode="exact", tau=0.9, T=2, layers=1, B=B)
     print("config4", B, rep, stats)
+
+
+@pytest.mark.parametrize("B,stride", [(32, 8), (128, 32), (256, 64)])
+def test_config4_shape_tensor_core_batches(B, stride):
+    # the batched sweep of config 4 on the tcgen05 path; decisions checked for every token, FFN output for
+    # every stride-th token (the oracle needs seconds per token at this size)
+    cfg = synth.CONFIGS[4]
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=1, layers=1, B=B, ffn_token_stride=stride)
+    assert stats["tokens"] == B and rep.ffn_checked >= B // stride
+    print("config4-tc", B, rep, stats)
 
 
 # ------------------------------------------------------------------ API behaviour

@@ -185,8 +185,10 @@ def time_ffn_kernel(apex, cfg, h, hp, B, tokens):
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
         e0.record()
         for l in range(cfg.L):
-            apex.moe_ffn_raw(l, 0, hp_ptr[l], B, y_ptr[l], stream)
+            apex.moe_ffn_begin_raw(l, 0, hp_ptr[l], B, y_ptr[l], stream)
         e1.record()
+        for l in range(cfg.L):
+            apex.moe_ffn_end(l)
         torch.cuda.synchronize()
         if t > 0:                       # first pass is warm-up
             per_launch.append(e0.elapsed_time(e1) / cfg.L)

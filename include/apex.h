@@ -156,6 +156,17 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
 int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev,
                  int32_t* exec_idx_dev, float* exec_gate_dev, void* stream);
 
+/* The same in two halves, for callers that pipeline layers themselves (Sec. IV-E "asynchronous miss
+ * correction": the expert computation starts while the host is still arranging the copies).
+ * apex_moe_ffn_begin queues the expert FFN of the layer-step and returns at once.  apex_moe_ffn_end
+ * does the host part that needs the gate's decision -- recency stamps, demand copies for missing
+ * experts (B = 1: the queued kernel is already waiting for them; B > 1: further launches) -- and must
+ * be called before the next apex_predict / apex_route_topk of the same layer (APEX_ESTATE otherwise).
+ * apex_moe_ffn is begin followed by end. */
+int apex_moe_ffn_begin(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev,
+                       int32_t* exec_idx_dev, float* exec_gate_dev, void* stream);
+int apex_moe_ffn_end(apex_ctx* ctx, int layer);
+
 /* All L layers of one decode step, in the order above.  h_dev, hpost_dev, y_dev are [L][B][d]. */
 int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev, int B, float tau,
                       int mode, float* y_dev, void* stream);

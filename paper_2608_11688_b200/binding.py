@@ -58,6 +58,8 @@ SIGNATURES = {
     "apex_attention_standin": (_I, [_P, _I, _P]),
     "apex_route_topk": (_I, [_P, _I, _P, _I, _P, _P, _P]),
     "apex_moe_ffn": (_I, [_P, _I, _I, _P, _I, _P, _P, _P, _P]),
+    "apex_moe_ffn_begin": (_I, [_P, _I, _I, _P, _I, _P, _P, _P, _P]),
+    "apex_moe_ffn_end": (_I, [_P, _I]),
     "apex_decode_token": (_I, [_P, _P, _P, _I, C.c_float, _I, _P, _P]),
     "apex_decode_token_host": (_I, [_P, _P, _P, _I, C.c_float, _I, _P, _P]),
     "apex_get_stats": (_I, [_P, _I, C.POINTER(ApexStepStats)]),
@@ -209,11 +211,19 @@ class Apex:
         self._chk(self.lib.apex_moe_ffn(self.h, layer, m, _ptr(hpost_dev), B, _ptr(y_dev), _ptr(exec_idx_dev),
                                         _ptr(exec_gate_dev), _stream(stream)))
 
-    def moe_ffn_raw(self, layer, mode_int, hpost_ptr, B, y_ptr, stream_int):
-        """Same call with raw addresses (no per-call marshalling): for tight timing loops."""
-        rc = self.lib.apex_moe_ffn(self.h, layer, mode_int, hpost_ptr, B, y_ptr, None, None, stream_int)
+    def moe_ffn_begin_raw(self, layer, mode_int, hpost_ptr, B, y_ptr, stream_int):
+        """apex_moe_ffn_begin with raw addresses (no per-call marshalling): for tight timing loops."""
+        rc = self.lib.apex_moe_ffn_begin(self.h, layer, mode_int, hpost_ptr, B, y_ptr, None, None, stream_int)
         if rc != APEX_OK:
             self._chk(rc)
+
+    def moe_ffn_begin(self, layer, mode, hpost_dev, B, y_dev, exec_idx_dev=None, exec_gate_dev=None, stream=None):
+        m = MODES[mode] if isinstance(mode, str) else mode
+        self._chk(self.lib.apex_moe_ffn_begin(self.h, layer, m, _ptr(hpost_dev), B, _ptr(y_dev), _ptr(exec_idx_dev),
+                                              _ptr(exec_gate_dev), _stream(stream)))
+
+    def moe_ffn_end(self, layer):
+        self._chk(self.lib.apex_moe_ffn_end(self.h, layer))
 
     def decode_token(self, h_dev, hpost_dev, B, tau, mode, y_dev, stream=None):
         m = MODES[mode] if isinstance(mode, str) else mode

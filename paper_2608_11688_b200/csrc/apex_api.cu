@@ -4,6 +4,7 @@
 #include <chrono>
 #include <cmath>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 
@@ -200,6 +201,8 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(dev_alloc(&ctx->d_ncand, MB));
   CR(dev_alloc(&ctx->d_stats, L));
   CR(cudaMemset(ctx->d_stats, 0, L * sizeof(DevStats)));
+  CR(dev_alloc(&ctx->d_tickets, 64));
+  CR(cudaMemset(ctx->d_tickets, 0, 64 * sizeof(unsigned int)));
   CR(dev_alloc(&ctx->d_counters, 2));
   CR(cudaMemset(ctx->d_counters, 0, 2 * sizeof(unsigned long long)));
   const size_t max_pairs = MB * (k + 1);
@@ -290,7 +293,7 @@ int apex_destroy(apex_ctx* ctx) {
   cudaDeviceSynchronize();
   cudaGetLastError();
   void* dev[] = {ctx->d_Wr, ctx->d_br, ctx->d_Wp, ctx->d_bp, ctx->d_w, ctx->d_theta, ctx->d_cache, ctx->d_slot_ready, ctx->d_zp,
-                 ctx->d_qp, ctx->d_zr, ctx->d_demand, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_plan_exec_idx,
+                 ctx->d_qp, ctx->d_zr, ctx->d_demand, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_tickets, ctx->d_plan_exec_idx,
                  ctx->d_plan_exec_gate, ctx->d_pair_tok, ctx->d_pair_gate, ctx->d_pair_expert, ctx->d_n_pairs, ctx->d_grp, ctx->d_xg, ctx->d_act, ctx->d_cand,
                  ctx->d_idx, ctx->d_exec_idx, ctx->d_alpha, ctx->d_exec_gate, ctx->d_cand_ncand, ctx->d_attn, ctx->d_attn_sink,
                  ctx->d_h_stage, ctx->d_hp_stage, ctx->d_y_stage};
@@ -446,6 +449,8 @@ int predict_select_fused(apex_ctx* ctx, int layer, const float* h_dev, int B, fl
   if ((r = fill_select(ctx, layer, B, tau, cand_dev, ncand_dev, &p.sel)) != APEX_OK) return r;
   p.fuse_select = 1;
   CU_TRY(ctx, launch_router(p, cs));
+  ctx->last_was_ffn = false;
+  ctx->last_stream = cs;
   ++ctx->launches;
   ctx->pred_stream = cs;
   ctx->step[layer].predicted = true;
@@ -465,6 +470,8 @@ int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stre
   int r = begin_predict(ctx, layer, h_dev, B, &p);
   if (r != APEX_OK) return r;
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
+  ctx->last_was_ffn = false;
+  ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   ctx->pred_stream = (cudaStream_t)stream;
   ctx->step[layer].predicted = true;
@@ -481,6 +488,8 @@ int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* 
   int r = fill_select(ctx, layer, B, tau, cand_dev, ncand_dev, &p);
   if (r != APEX_OK) return r;
   CU_TRY(ctx, launch_select(p, (cudaStream_t)stream));
+  ctx->last_was_ffn = false;
+  ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   st.selected = true;
   return APEX_OK;
@@ -548,6 +557,8 @@ int apex_attention_standin(apex_ctx* ctx, int layer, void* stream) {
   p.n_vec = ctx->attn_bytes / 16;
   p.sink = ctx->d_attn_sink;
   CU_TRY(ctx, launch_attention(p, ctx->n_sm, (cudaStream_t)stream));
+  ctx->last_was_ffn = false;
+  ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   return APEX_OK;
 }
@@ -580,6 +591,8 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   p.ncand_pred = st.selected ? ctx->d_ncand : nullptr;
   p.stats = ctx->d_stats + layer;
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
+  ctx->last_was_ffn = false;
+  ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   st.routed = true;
   st.idx_dev = idx_dev;
@@ -591,11 +604,25 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
 
 namespace {
 
+// Every launch of the streaming kernel gets its own row-ticket counter out of a ring of 64; the
+// launch also clears the counter that will be used 32 launches later.
+cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
+  const uint32_t id = ctx->ffn_launch_id++;
+  p.zero_early = (!ctx->last_was_ffn && ctx->last_stream == cs && !getenv("APEX_ZERO_LATE")) ? 1 : 0;
+  ctx->last_was_ffn = true;
+  ctx->last_stream = cs;
+  p.ticket = ctx->d_tickets + (id & 63u);
+  p.ticket_reset = ctx->d_tickets + ((id + 32u) & 63u);
+  return launch_ffn(p, ctx->n_sm, cs);
+}
+
 constexpr int kTcMinBatch = 16;  // from this many tokens per step the tensor-core grouped GEMM runs
 
 // B > 1: plan kernel, then either the tensor-core grouped GEMM or the streaming kernel per pair.
 int launch_batched(apex_ctx* ctx, int layer, const FfnParams& p, cudaStream_t cs) {
   CU_TRY(ctx, launch_ffn_plan(p, cs));
+  ctx->last_was_ffn = false;
+  ctx->last_stream = cs;
   ++ctx->launches;
   if (ctx->tc_ok && p.B >= kTcMinBatch) {
     TcParams t{};
@@ -607,9 +634,10 @@ int launch_batched(apex_ctx* ctx, int layer, const FfnParams& p, cudaStream_t cs
     t.act_plane = ctx->act_plane;
     t.layer_slot0 = layer * ctx->cfg.C;
     CU_TRY(ctx, launch_ffn_tc(t, ctx->tc_shared_maps[layer], ctx->n_sm, cs));
+    ctx->last_was_ffn = true;
     ctx->launches += 3;
   } else {
-    CU_TRY(ctx, launch_ffn(p, ctx->n_sm, cs));
+    CU_TRY(ctx, launch_stream(ctx, p, cs));
     ++ctx->launches;
   }
   return APEX_OK;
@@ -670,7 +698,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
     int r = launch_batched(ctx, layer, p, cs);
     if (r != APEX_OK) return r;
   } else {
-    CU_TRY(ctx, launch_ffn(p, ctx->n_sm, cs));
+    CU_TRY(ctx, launch_stream(ctx, p, cs));
     ++ctx->launches;
   }
   st.pending = true;
@@ -754,7 +782,7 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
           int r = launch_batched(ctx, layer, q, cs);
           if (r != APEX_OK) return r;
         } else {
-          CU_TRY(ctx, launch_ffn(q, ctx->n_sm, cs));
+          CU_TRY(ctx, launch_stream(ctx, q, cs));
           ++ctx->launches;
         }
         ctx->host_stats[layer].extra_waves += 1;
@@ -782,6 +810,20 @@ int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int
   CHECK_LAYER(ctx, layer);
   int r = ffn_launch(ctx, layer, mode, hpost_dev, B, y_dev, exec_idx_dev, exec_gate_dev, (cudaStream_t)stream);
   if (r != APEX_OK) return r;
+  return ffn_finalize(ctx, layer);
+}
+
+int apex_moe_ffn_begin(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev, int32_t* exec_idx_dev,
+                       float* exec_gate_dev, void* stream) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  return ffn_launch(ctx, layer, mode, hpost_dev, B, y_dev, exec_idx_dev, exec_gate_dev, (cudaStream_t)stream);
+}
+
+int apex_moe_ffn_end(apex_ctx* ctx, int layer) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (!ctx->step[layer].pending) return fail(ctx, APEX_ESTATE, "apex_moe_ffn_end without apex_moe_ffn_begin");
   return ffn_finalize(ctx, layer);
 }
 

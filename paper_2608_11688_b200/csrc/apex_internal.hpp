@@ -134,10 +134,13 @@ struct FfnParams {
   DevStats* stats;
   unsigned long long* zero_counter;
   unsigned long long zero_target;
+  unsigned int* ticket;        // row-ticket counter of this launch (zero at launch)
+  unsigned int* ticket_reset;  // counter of the launch 32 launches ahead, reset by this one
   unsigned long long run_mask;  // experts this launch executes
   const uint32_t* demand;       // [N] per layer: (tag << 8 | slot), published by the host after a demand copy
   uint32_t demand_tag;          // tag of this launch
   int demand_in_kernel;         // 1: a routed expert without a slot is waited for inside the kernel
+  int zero_early;               // 1: y may be zeroed before the dependency wait (the preceding kernel does not touch y)
   SlotSnapshot snap;
   size_t slot_stride;
   long long wait_limit_ns;
@@ -232,6 +235,12 @@ struct apex_ctx {
   uint32_t sel_seq = 0;
   std::vector<uint32_t> exec_seq;                 // per layer, last value asked for
   unsigned long long sel_done = 0, zero_done = 0;
+  unsigned int* d_tickets = nullptr;  // [64] ring of row-ticket counters
+  uint32_t ffn_launch_id = 0;
+  // what this context queued last, and where: an expert-FFN launch may still be adding to its y when
+  // the next kernel's prologue runs (programmatic dependent launch)
+  bool last_was_ffn = false;
+  cudaStream_t last_stream = nullptr;
   uint32_t launch_tag = 0;
   uint32_t* gen_src = nullptr;  // pinned ring of flag values for the ready-flag copies
   size_t gen_src_pos = 0, gen_src_len = 0;

@@ -403,6 +403,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     TL(0);
     TL(1);
     s_abort = 0;
+    if (cta == 0) *p.ticket_reset = 0u;  // the counter of a launch far in the future (nobody uses it now)
   }
   if (tid < NS) mbar_init(&s_full[tid], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -419,22 +420,27 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
       hreg[c * 8 + 4] = b2.x; hreg[c * 8 + 5] = b2.y; hreg[c * 8 + 6] = b2.z; hreg[c * 8 + 7] = b2.w;
     }
   }
-  pdl_wait();               // the gate's outputs (K_r, alpha, z_r) are complete from here on
-  pdl_launch_dependents();  // the next kernel may start its own prologue
-  if (tid == 0) TL(4);
-  // y is zeroed only now: a preceding launch that still adds to the same buffer has completed
-  if (!p.accumulate) {
+  // y is zeroed by all CTAs together (a slice each) and the slice is published through a counter.
+  // Before the dependency wait when the host knows that the preceding kernel does not touch y (the
+  // usual case: the gate kernel), after it otherwise.
+  auto zero_slice = [&]() {
+    if (p.accumulate) return;
     const size_t n4 = (size_t)B * d / 4;
     const size_t per = (n4 + G - 1) / G;
     const size_t lo = per * cta, hi = lo + per < n4 ? lo + per : n4;
     float4* y4 = reinterpret_cast<float4*>(p.y);
     for (size_t i = lo + tid; i < hi; i += kFfnThreads) y4[i] = make_float4(0.f, 0.f, 0.f, 0.f);
-  }
-  if (!p.accumulate) __syncthreads();
-  if (!p.accumulate && tid == 0) {
-    __threadfence();
-    atomicAdd(p.zero_counter, 1ull);
-  }
+    __syncthreads();
+    if (tid == 0) {
+      __threadfence();
+      atomicAdd(p.zero_counter, 1ull);
+    }
+  };
+  if (p.zero_early) zero_slice();
+  pdl_wait();               // the gate's outputs (K_r, alpha, z_r) are complete from here on
+  pdl_launch_dependents();  // the next kernel may start its own prologue
+  if (tid == 0) TL(4);
+  if (!p.zero_early) zero_slice();  // a preceding launch of this library may still be adding to the same y
 
   // ---- every global load of the prologue is issued before the first use, so the latencies overlap.
   // Slot-ready flags: lanes own experts lane and lane+32.  The flag is written by the copy engine
@@ -476,9 +482,22 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   rm.total_rows = rm.routed_rows + (long long)(rm.n_pairs - rm.n_routed) * p.I_shared;
   if (tid == 0) TL(2);  // plan done
 
-  const long long r_begin = rm.total_rows * cta / G, r_end = rm.total_rows * (cta + 1) / G;
-  const int n_my = (int)(r_end - r_begin);
-  const int my_n = n_my > warp ? (n_my - warp + kConsumerWarps - 1) / kConsumerWarps : 0;  // rows of this warp
+  // Work split.  Short launches (fewer than two ring fills per CTA): equal contiguous ranges, all
+  // known at launch, no shared counter (a ticket per row costs more than it balances there: every
+  // warp would hit one counter within the same microsecond).  Long launches: every CTA owns NS (the
+  // ring depth) consecutive rows, so all its stages are filled at once, and the remaining rows are
+  // handed out in tickets from a global counter to whichever warp has a free stage first.
+  const long long per_cta = rm.total_rows / G;
+  const bool dynamic = per_cta >= 2 * NS;
+  const long long range_lo = rm.total_rows * cta / G, range_hi = rm.total_rows * (cta + 1) / G;
+  const int S = dynamic ? NS : (int)(range_hi - range_lo);       // rows this CTA knows about at launch
+  const long long static_base = dynamic ? (long long)cta * NS : range_lo;
+  const long long dyn_begin = dynamic ? (long long)G * NS : rm.total_rows;
+  const long long dyn_rows = rm.total_rows - dyn_begin;
+  const int chunk = (int)((dyn_rows + (long long)G * kConsumerWarps * 4 - 1) / ((long long)G * kConsumerWarps * 4)) > 1
+                        ? (int)((dyn_rows + (long long)G * kConsumerWarps * 4 - 1) / ((long long)G * kConsumerWarps * 4))
+                        : 1;                                      // rows per ticket: about four tickets per warp
+  const int n_static = S > warp ? (S - warp + kConsumerWarps - 1) / kConsumerWarps : 0;  // static rows of this warp
 
   float acc[NCH * 8];
 #pragma unroll
@@ -507,10 +526,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     zero_seen = true;
   };
 
-  // lane (j mod NSW) starts the copy of this warp's j-th row into stage (j mod NSW) of the warp.  The
-  // first NSW copies of a warp are thus issued by NSW lanes in one instruction.
-  auto issue = [&](int j) {
-    const long long r = r_begin + warp + (long long)kConsumerWarps * j;
+  // Starts the copy of row r as this warp's n-th row, into stage (n mod NSW) of the warp.
+  auto issue = [&](long long r, int n) {
     int pidx, e, tok;
     long long i;
     float gate = 0.f;
@@ -581,7 +598,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     } else {
       base = p.shared_w;
     }
-    const int s = warp + kConsumerWarps * (j % NSW);
+    const int s = warp + kConsumerWarps * (n % NSW);
     s_gate[s] = gate;
     s_tok[s] = tok;
     s_exp[s] = e;
@@ -610,24 +627,63 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   // K_r: post first.  Otherwise post while the first rows are in flight.
   const bool will_wait_for_host = p.demand_in_kernel && (run & ~p.snap.resident_mask) != 0ull;
   if (poster && will_wait_for_host) post_plan();
-  if (lane < NSW && lane < my_n) {
+  // ---- row supply of this warp (state lives in lane 0; the other lanes learn the outcome by shuffle)
+  int next_static = 0;                 // static rows of this warp already started
+  long long dyn_cur = 0, dyn_end = 0;  // rows of the current ticket
+  bool dyn_done = dyn_rows <= 0;
+  auto next_row = [&]() -> long long {  // lane 0 only
+    if (next_static < n_static) return static_base + warp + (long long)kConsumerWarps * next_static++;
+    if (dyn_cur < dyn_end) return dyn_cur++;
+    if (dyn_done) return -1;
+    // Tickets are taken on demand, never ahead: the rows must go to the warps that are free first
+    // (all stages of all SMs are requested at once at the start, and which SM is served first is a
+    // matter of queueing; an SM whose first rows land late should not also hold extra rows).
+    const unsigned int ticket = atomicAdd(p.ticket, 1u);
+    const long long first = dyn_begin + (long long)ticket * chunk;
+    if (first >= rm.total_rows) {
+      dyn_done = true;
+      return -1;
+    }
+    dyn_cur = first;
+    dyn_end = first + chunk < rm.total_rows ? first + chunk : rm.total_rows;
+    return dyn_cur++;
+  };
+  // first fill: the static rows go out from NSW lanes in one instruction
+  const int first_fill = n_static < NSW ? n_static : NSW;
+  if (lane < first_fill) {
     if (lane == 0 && warp == 0) TL(3);
-    issue(lane);
+    issue(static_base + warp + (long long)kConsumerWarps * lane, lane);
     if (!ok) atomicExch(&s_abort, 1);
   }
   __syncwarp();
+  int tail = first_fill;  // rows of this warp whose copy has been started (uniform across the warp)
+  next_static = first_fill;
   if (poster && !will_wait_for_host) post_plan();
-  int issued = my_n < NSW ? my_n : NSW;  // rows of this warp whose copy has been started (uniform across the warp)
-  for (int j = 0; j < my_n; ++j) {
-    if (lane == 0 && j == my_n - 1) poll_zeroed(false);  // latency hidden behind the wait for the last row
+  // a warp with fewer static rows than stages tops up from the dynamic part
+  while (tail < NSW) {
+    int more = 0;
+    if (lane == 0 && ok) {
+      const long long r = next_row();
+      if (r >= 0) {
+        issue(r, tail);
+        if (!ok) atomicExch(&s_abort, 1);
+        more = ok ? 1 : 0;
+      }
+    }
+    more = __shfl_sync(0xffffffffu, more, 0);
+    if (!more) break;
+    ++tail;
+  }
+  bool polled = false;
+  for (int head = 0; head < tail; ++head) {
     if (__any_sync(0xffffffffu, *(volatile int*)&s_abort != 0)) break;
-    const int s = warp + kConsumerWarps * (j % NSW);
-    if (!__all_sync(0xffffffffu, mbar_wait(&s_full[s], (uint32_t)((j / NSW) & 1), &s_abort, p.wait_limit_ns))) {
+    const int s = warp + kConsumerWarps * (head % NSW);
+    if (!__all_sync(0xffffffffu, mbar_wait(&s_full[s], (uint32_t)((head / NSW) & 1), &s_abort, p.wait_limit_ns))) {
       atomicExch(&s_abort, 1);
       break;
     }
-    if (lane == 0 && warp == 0 && j == 0) TL(5);
-    if (lane == 0 && j == my_n - 1) TL(6);
+    if (lane == 0 && warp == 0 && head == 0) TL(5);
+    if (lane == 0 && warp == 0) TL(6);
     const int e = s_exp[s];
     const int tok = s_tok[s];
     float gate;
@@ -706,13 +762,21 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
       acc[c * 8 + 7] = fmaf(a, bf16hi(dv.w), acc[c * 8 + 7]);
     }
     __syncwarp();  // every lane has read stage s: it may be refilled
-    if (j + NSW < my_n) {
-      if (lane == j % NSW) {
-        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-        issue(j + NSW);
-        if (!ok) atomicExch(&s_abort, 1);
+    {
+      int more = 0;
+      if (lane == 0 && ok) {
+        const long long r = next_row();
+        if (r >= 0) {
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          issue(r, tail);
+          if (!ok) atomicExch(&s_abort, 1);
+          more = ok ? 1 : 0;
+        } else if (!polled) {
+          polled = true;
+          poll_zeroed(false);  // no more rows to fetch: the latency hides behind the rows still in flight
+        }
       }
-      ++issued;
+      tail += __shfl_sync(0xffffffffu, more, 0);
     }
   }
   waited = warp_max_u64(waited);
@@ -729,9 +793,9 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   if (aborted) {
     // leave only after every copy this warp started has landed (bounded), so that no copy is in
     // flight into the shared memory of an exited CTA
-    for (int jj = 0; jj < issued; ++jj) {
+    for (int jj = 0; jj < tail; ++jj) {
       const int s = warp + kConsumerWarps * (jj % NSW);
-      if (jj + NSW >= issued) mbar_wait(&s_full[s], (uint32_t)((jj / NSW) & 1), nullptr, p.wait_limit_ns);
+      if (jj + NSW >= tail) mbar_wait(&s_full[s], (uint32_t)((jj / NSW) & 1), nullptr, p.wait_limit_ns);
     }
   }
 
@@ -769,7 +833,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     __syncthreads();
   }
   if (tid == 0) TL(8);
-  if (n_my > 0 && !aborted) {
+  if (!aborted) {  // (a CTA that took no row adds zeros)
     float4* y4 = reinterpret_cast<float4*>(p.y);
     for (int col4 = tid; col4 < d / 4; col4 += kFfnThreads) {
       float4 sacc = make_float4(0.f, 0.f, 0.f, 0.f);

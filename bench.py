@@ -298,12 +298,12 @@ def main():
     dev = torch.device("cuda", local_rank)
     if rank == 0:
         build.build()
+    from paper_2608_11688_b200 import replicas
     dist_sync = None
     if world > 1:
-        import torch.distributed as dist
-        dist.init_process_group("nccl", device_id=dev)
-        dist.barrier()
-        dist_sync = dist.barrier
+        replicas.init("nccl", dev)
+        replicas.barrier()
+        dist_sync = replicas.barrier
     B = args.batch
     prob = build_problem(cfg, dev)
     T = min(cfg.T, args.warmup + args.steps)
@@ -330,7 +330,7 @@ def main():
         return
 
     # ---- headline: config cache size, exact (correctness-preserving) mode, inputs resident in HBM
-    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C)
+    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B)
     if args.resident:
         apex.warm_all()
     sampler = ClockSampler(local_rank)
@@ -340,12 +340,8 @@ def main():
     launches = (apex.launch_count() - n0) * args.steps // (args.warmup + args.steps)
     clocks = sampler.stop()
     st_all = apex.get_stats()
-    if world > 1:
-        import torch.distributed as dist
-        tmax = torch.tensor([sec], device=dev)
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        sec = float(tmax.item())
-    value = world * args.steps / sec
+    sec = replicas.max_over_ranks(sec, dev)
+    value = world * args.steps * B / sec
     extras = {}
     e2e = None
     roof = None
@@ -356,17 +352,14 @@ def main():
         # ---- end to end: host buffers in, host buffer out, through the C-ABI call
         apex.reset_stats()
         sec_e2e = time_tokens(apex, h_pin, hp_pin, y_pin, B, "exact", args.warmup, args.steps, dist_sync, host=True)
-        if world > 1:
-            tmax = torch.tensor([sec_e2e], device=dev)
-            dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-            sec_e2e = float(tmax.item())
+        sec_e2e = replicas.max_over_ranks(sec_e2e, dev)
         st = apex.get_stats()
         per_tok = args.warmup + args.steps
-        e2e = {"value": world * args.steps / sec_e2e, "unit": UNIT,
+        e2e = {"value": world * args.steps * B / sec_e2e, "unit": UNIT,
                "h2d_bytes_per_step": int(2 * cfg.L * B * cfg.d * 4), "d2h_bytes_per_step": int(cfg.L * B * cfg.d * 4),
                "expert_bytes_copied_per_step": int(st["bytes_copied"] / per_tok)}
         extras["exact"] = {
-            "tokens_per_s": args.steps / sec, "overlap_vs_P": st["hits_P"] / max(1, st["routed"]),
+            "tokens_per_s": args.steps * B / sec, "overlap_vs_P": st["hits_P"] / max(1, st["routed"]),
             "overlap_vs_R": st["hits_R"] / max(1, st["routed"]), "coverage": st["covered"] / max(1, st["tokens"]),
             "mean_delta_hat": st["sum_delta_hat"] / max(1, st["tokens"]),
             "mean_delta_star": st["sum_delta_star"] / max(1, st["tokens"]),
@@ -377,19 +370,19 @@ def main():
         apex.destroy()
         if rank == 0:
             # ---- stall-free mode
-            a2 = make_ctx(cfg, prob, cfg.C)
+            a2 = make_ctx(cfg, prob, cfg.C, max_batch=B)
             if "stall_free" in cfg.modes:
                 sec_sf = time_tokens(a2, h_dev, hp_dev, y_dev, B, "stall_free", args.warmup, args.steps)
                 s2 = a2.get_stats()
-                extras["stall_free"] = {"tokens_per_s": args.steps / sec_sf,
+                extras["stall_free"] = {"tokens_per_s": args.steps * B / sec_sf,
                                         "substitutions_per_token": s2["substitutions"] / (args.warmup + args.steps),
                                         "copies_per_token": s2["prefetch_copies"] / (args.warmup + args.steps)}
             a2.destroy()
             # ---- all experts resident (C = N): isolates the kernels from the host link
-            a3 = make_ctx(cfg, prob, cfg.N)
+            a3 = make_ctx(cfg, prob, cfg.N, max_batch=B)
             a3.warm_all()
             sec_res = time_tokens(a3, h_dev, hp_dev, y_dev, B, "exact", args.warmup, args.steps)
-            extras["all_resident"] = {"tokens_per_s": args.steps / sec_res,
+            extras["all_resident"] = {"tokens_per_s": args.steps * B / sec_res,
                                       "frac_of_8TBs": bytes_step * cfg.L * args.steps / sec_res / 1e9 / NOMINAL_HBM_GBS,
                                       "frac_of_peak": bytes_step * cfg.L * args.steps / sec_res / 1e9 / peak}
             extras["exact"]["exposed_stall_us_per_token"] = (sec / args.steps - sec_res / args.steps) * 1e6
@@ -407,9 +400,7 @@ def main():
                    "sample": f"{args.cpu_baseline_tokens} decode tokens x {cfg.L} layers ({dt:.1f} s)"}
     else:
         apex.destroy()
-    if world > 1:
-        dist.barrier()
-        dist.destroy_process_group()
+    replicas.finish()
     if rank != 0:
         return
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,

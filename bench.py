@@ -272,6 +272,8 @@ def main():
                     help="profiling case: all experts resident, gate + expert FFN only, no copy in flight")
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (smaller captures)")
     ap.add_argument("--batch", type=int, default=1, help="tokens per decode step (config 4 sweeps 1, 8, 32, 128, 256)")
+    ap.add_argument("--policies", action="store_true",
+                    help="also time the baselines of the paper's comparison: no prefetch, static top-k, top-(k+4), top-(k+8)")
     ap.add_argument("--resident", action="store_true",
                     help="cache as large as the expert count, warmed up: no host-link copies (kernel launch lists)")
     args = ap.parse_args()
@@ -378,6 +380,35 @@ def main():
                                         "substitutions_per_token": s2["substitutions"] / (args.warmup + args.steps),
                                         "copies_per_token": s2["prefetch_copies"] / (args.warmup + args.steps)}
             a2.destroy()
+            # ---- policy baselines of Sec. V-A under the same harness (same ranking, different budgets)
+            if args.policies:
+                pol = {}
+                n_tok = args.warmup + args.steps
+                for name, tau_p, delta in (("no_prefetch", -1.0, None), ("static_k", 0.9, 0), ("static_k+4", 0.9, 4),
+                                           ("static_k+8", 0.9, 8)):
+                    ap_ = make_ctx(cfg, prob, cfg.C, max_batch=B)
+                    if delta is not None:      # w = 0 and a step in theta: delta_hat = delta for every token
+                        nth = cfg.N - cfg.k + 1
+                        th = np.where(np.arange(nth) >= delta, 50.0, -50.0).astype(np.float32)
+                        for l in range(cfg.L):
+                            ap_.set_cdf(l, np.zeros(cfg.N, np.float32), th)
+                    T_ = h_dev.shape[0]
+                    for t in range(args.warmup):
+                        ap_.decode_token(h_dev[t % T_], hp_dev[t % T_], B, tau_p, "exact", y_dev)
+                    torch.cuda.synchronize()
+                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                    e0.record()
+                    for t in range(args.warmup, n_tok):
+                        ap_.decode_token(h_dev[t % T_], hp_dev[t % T_], B, tau_p, "exact", y_dev)
+                    e1.record()
+                    torch.cuda.synchronize()
+                    sp = ap_.get_stats()
+                    pol[name] = {"tokens_per_s": args.steps * B / (e0.elapsed_time(e1) * 1e-3),
+                                 "copies_per_token": (sp["prefetch_copies"] + sp["demand_copies"]) / n_tok,
+                                 "demand_copies_per_token": sp["demand_copies"] / n_tok,
+                                 "overlap_vs_R": sp["hits_R"] / max(1, sp["routed"])}
+                    ap_.destroy()
+                extras["policies"] = pol
             # ---- all experts resident (C = N): isolates the kernels from the host link
             a3 = make_ctx(cfg, prob, cfg.N, max_batch=B)
             a3.warm_all()

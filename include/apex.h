@@ -167,7 +167,10 @@ int apex_moe_ffn_begin(apex_ctx* ctx, int layer, int mode, const float* hpost_de
                        int32_t* exec_idx_dev, float* exec_gate_dev, void* stream);
 int apex_moe_ffn_end(apex_ctx* ctx, int layer);
 
-/* All L layers of one decode step, in the order above.  h_dev, hpost_dev, y_dev are [L][B][d]. */
+/* All L layers of one decode step, in the order above.  h_dev, hpost_dev, y_dev are [L][B][d].
+ * tau < 0 skips the prefetch stage altogether: the "No Prefetch" baseline of Sec. V-A, where every
+ * non-resident routed expert is loaded on the critical path (static over-fetch baselines are a
+ * confidence model with w = 0 and a step in theta). */
 int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev, int B, float tau,
                       int mode, float* y_dev, void* stream);
 /* Same with host buffers (pinned for full speed): inputs are copied to the device and y back

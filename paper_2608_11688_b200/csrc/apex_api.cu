@@ -840,12 +840,14 @@ int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev,
   for (int l = 0; l < ctx->cfg.L; ++l) {
     int32_t* idx = ctx->d_idx + (size_t)l * MB * k;
     float* alpha = ctx->d_alpha + (size_t)l * MB * N;
-    if ((r = predict_select_fused(ctx, l, h_dev + l * step, B, tau, ctx->d_cand, ctx->d_cand_ncand, (cudaStream_t)stream)) != APEX_OK)
+    const bool prefetching = !(tau < 0.f);  // tau < 0: the conventional scheme, expert loading on the critical path
+    if (prefetching &&
+        (r = predict_select_fused(ctx, l, h_dev + l * step, B, tau, ctx->d_cand, ctx->d_cand_ncand, (cudaStream_t)stream)) != APEX_OK)
       return r;
     if ((r = apex_attention_standin(ctx, l, stream)) != APEX_OK) return r;
     if ((r = apex_route_topk(ctx, l, hpost_dev + l * step, B, idx, alpha, stream)) != APEX_OK) return r;
     if (l > 0 && (r = ffn_finalize(ctx, l - 1)) != APEX_OK) return r;
-    if ((r = apex_prefetch(ctx, l, B, nullptr)) != APEX_OK) return r;
+    if (prefetching && (r = apex_prefetch(ctx, l, B, nullptr)) != APEX_OK) return r;
     if ((r = ffn_launch(ctx, l, mode, hpost_dev + l * step, B, y_dev + l * step, ctx->d_exec_idx, ctx->d_exec_gate,
                         (cudaStream_t)stream)) != APEX_OK)
       return r;

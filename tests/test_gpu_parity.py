@@ -291,3 +291,54 @@ def test_run_to_run_determinism_of_indices():
         np.testing.assert_array_equal(r0[2], r1[2])                      # bitwise: fixed reduction order
         for x, y2 in zip(r0[3], r1[3]):
             np.testing.assert_array_equal(x, y2)
+
+
+# ------------------------------------------------------------------ the benchmark's launch configuration
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_config1_full_size_decode_token_sampled_layers(mode):
+    """Config 1 at full size (32 layers, 20 slots, fitted confidence model) through apex_decode_token --
+    the call bench.py times: fused prefetch router + budget, pipelined host work, in-kernel miss wait.
+    Every token: slot tables of all layers before and after; sampled layers are replayed by the oracle
+    from the pre-step table and compared (decisions bit-exact via the tables and copy lists, y by tolerance)."""
+    from oracle import apex_oracle as ao
+    hz = _harness()
+    cfg = synth.CONFIGS[1]
+    prob = hz.Problem(cfg, cdf="fitted")
+    apex = prob.make_ctx()
+    try:
+        T = 3
+        hs = [synth.hidden_states(cfg, l, T, 1) for l in range(cfg.L)]
+        h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()      # [T][L][1][d]
+        hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
+        y = torch.empty((cfg.L, 1, cfg.d), device="cuda")
+        worst = 0.0
+        for t in range(T):
+            pre = [apex.get_slot_table(l) for l in range(cfg.L)]
+            apex.decode_token(h[t], hp[t], 1, 0.9, mode, y)
+            torch.cuda.synchronize()
+            g_y = y.cpu().numpy()
+            for l in range((t * 5) % 7, cfg.L, 7):                           # five or so layers per token
+                W_r, b_r, W_p, b_p = prob.routers[l]
+                w, theta = prob.cdf[l]
+                cache = ao.SlotCache(cfg.N, cfg.C)
+                cache.set_state(*pre[l])
+                out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=0.9, k=cfg.k,
+                                    h=hs[l][0][t], h_post=hs[l][1][t], mode=mode, expert_weights=prob.oracle_experts(l))
+                tok = out["tokens"][0]
+                near = (min(tok["rank_margin"], tok["route_margin"], tok["subst_margin"]) < ao.NEAR_TIE_LOGIT
+                        or tok["threshold_margin"] < ao.NEAR_TIE_THRESHOLD)
+                post = apex.get_slot_table(l)
+                cp, dm = apex.get_last_copies(l)
+                same = (list(post[0]) == cache.expert_slot and list(post[1]) == cache.slot_stamp and post[2] == cache.clock
+                        and cp == out["prefetch_copies"] and dm == out["demand_copies"])
+                assert same or near, f"slot decisions differ t={t} l={l}"
+                if same:
+                    err = g_y[l, 0].astype(np.float64) - tok["y"]
+                    rel = float(np.linalg.norm(err) / np.linalg.norm(tok["y"]))
+                    worst = max(worst, rel)
+                    assert rel <= hz.REL_L2_TOL and float(np.abs(err).max()) <= hz.MAX_ABS_TOL, (t, l, rel)
+        st = apex.get_stats()
+        assert st["tokens"] == T * cfg.L and st["timeouts"] == 0
+        print("config1 full", mode, "worst rel-L2", worst, st)
+    finally:
+        apex.destroy()

@@ -261,7 +261,9 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->gen_src), ctx->gen_src_len * sizeof(uint32_t), cudaHostAllocPortable));
 
   CR(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
+  CR(cudaStreamCreateWithFlags(&ctx->copy_stream_b, cudaStreamNonBlocking));
   ctx->cur_copy_stream = ctx->copy_stream;
+  ctx->cur_copy_stream_b = ctx->copy_stream_b;
   CR(cudaEventCreateWithFlags(&ctx->ev_wave, cudaEventDisableTiming));
   CR(cudaEventCreateWithFlags(&ctx->ev_in, cudaEventDisableTiming));
 #undef CR
@@ -302,6 +304,7 @@ int apex_destroy(apex_ctx* ctx) {
   if (ctx->mbox) cudaFreeHost(ctx->mbox);
   if (ctx->gen_src) cudaFreeHost(ctx->gen_src);
   if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
+  if (ctx->copy_stream_b) cudaStreamDestroy(ctx->copy_stream_b);
   if (ctx->ev_wave) cudaEventDestroy(ctx->ev_wave);
   if (ctx->ev_in) cudaEventDestroy(ctx->ev_in);
   delete ctx;
@@ -502,6 +505,7 @@ int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream) {
   if (!st.selected || st.B != B) return fail(ctx, APEX_ESTATE, "apex_prefetch needs apex_select_candidates of the same layer-step and B");
   if (st.prefetched) return fail(ctx, APEX_ESTATE, "apex_prefetch called twice in one layer-step");
   ctx->cur_copy_stream = copy_stream ? (cudaStream_t)copy_stream : ctx->copy_stream;
+  ctx->cur_copy_stream_b = copy_stream ? (cudaStream_t)copy_stream : ctx->copy_stream_b;
   const int C = ctx->cfg.C;
   const int32_t* ncand = mbox_i32(ctx, ctx->ml.off_ncand);
   const int32_t* cand = mbox_i32(ctx, ctx->ml.off_cand);
@@ -540,7 +544,7 @@ int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream) {
     ordered = copies;
   }
   for (const auto& c : ordered) {
-    int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+    int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->stream_of_slot(c.slot));
     if (r != APEX_OK) return r;
   }
   ctx->host_stats[layer].prefetch_copies += (int64_t)copies.size();
@@ -731,9 +735,9 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
       for (const auto& c : copies) {
         const int prev = slot_expert_before[c.slot];
         if (c.wave != 1 || (prev >= 0 && ((need >> prev) & 1))) return fail(ctx, APEX_ESTATE, "demand plan would evict an expert in use");
-        int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+        int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->stream_of_slot(c.slot));
         if (r != APEX_OK) return r;
-        r = stream_write32(ctx, ctx->cur_copy_stream, ctx->d_demand + (size_t)layer * ctx->cfg.N + c.expert,
+        r = stream_write32(ctx, ctx->stream_of_slot(c.slot), ctx->d_demand + (size_t)layer * ctx->cfg.N + c.expert,
                            (st.pend_tag << 8) | (uint32_t)c.slot);
         if (r != APEX_OK) return r;
       }
@@ -757,10 +761,11 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
         if (hazard) {
           CU_TRY(ctx, cudaEventRecord(ctx->ev_wave, cs));
           CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_stream, ctx->ev_wave, 0));
+          if (ctx->cur_copy_stream_b != ctx->cur_copy_stream) CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_stream_b, ctx->ev_wave, 0));
         }
         for (const auto& c : copies)
           if (c.wave == w) {
-            int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->cur_copy_stream);
+            int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->stream_of_slot(c.slot));
             if (r != APEX_OK) return r;
             const int prev = cur_slot_expert[c.slot];
             if (prev >= 0) {
@@ -965,7 +970,7 @@ int apex_set_slot_table(apex_ctx* ctx, int layer, const int32_t* expert_slot, co
   for (int e = 0; e < ctx->cfg.N; ++e) {
     const int s = expert_slot[e];
     if (s >= 0 && ctx->phys_expert[layer][s] != e) {
-      int r = issue_copy(ctx, layer, e, s, ctx->cur_copy_stream);
+      int r = issue_copy(ctx, layer, e, s, ctx->stream_of_slot(s));
       if (r != APEX_OK) return r;
     }
   }
@@ -983,6 +988,7 @@ int apex_warm_all(apex_ctx* ctx) {
     if (r != APEX_OK) return r;
   }
   CU_TRY(ctx, cudaStreamSynchronize(ctx->cur_copy_stream));
+  CU_TRY(ctx, cudaStreamSynchronize(ctx->cur_copy_stream_b));
   return APEX_OK;
 }
 

@@ -270,8 +270,11 @@ struct apex_ctx {
   std::vector<StepState> step;
   std::vector<apex::FfnParams> ffn_params;  // [L] parameters of the last FFN launch of each layer
 
-  cudaStream_t copy_stream = nullptr;   // own
-  cudaStream_t cur_copy_stream = nullptr;
+  // Copies of a slot always travel on the same stream (slot index modulo 2), so two installs into
+  // one slot stay ordered; two streams hide the gap between consecutive copies (+6 % on the link).
+  cudaStream_t copy_stream = nullptr, copy_stream_b = nullptr;  // own
+  cudaStream_t cur_copy_stream = nullptr, cur_copy_stream_b = nullptr;
+  cudaStream_t stream_of_slot(int slot) const { return (slot & 1) ? cur_copy_stream_b : cur_copy_stream; }
   cudaStream_t pred_stream = nullptr;   // stream of the last apex_predict
   cudaEvent_t ev_wave = nullptr, ev_in = nullptr;
   int inject = 0;

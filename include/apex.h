@@ -91,7 +91,7 @@ typedef struct apex_step_stats {
   int64_t demand_copies;
   int64_t bytes_copied;
   int64_t extra_waves;     /* FFN launches beyond the first, exact mode */
-  int64_t stall_ns;        /* device time spent waiting for slot-ready flags (max over CTAs per launch) */
+  int64_t stall_ns;        /* device time spent waiting for slot-ready flags or demand copies, mean over the SMs */
   int64_t timeouts;
   int64_t near_full_prefetch; /* tokens with k + delta_hat > N/2 */
 } apex_step_stats;

@@ -612,7 +612,7 @@ namespace {
 // launch also clears the counter that will be used 32 launches later.
 cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
   const uint32_t id = ctx->ffn_launch_id++;
-  p.zero_early = (!ctx->last_was_ffn && ctx->last_stream == cs && !getenv("APEX_ZERO_LATE")) ? 1 : 0;
+  p.zero_early = (!ctx->last_was_ffn && ctx->last_stream == cs) ? 1 : 0;
   ctx->last_was_ffn = true;
   ctx->last_stream = cs;
   p.ticket = ctx->d_tickets + (id & 63u);

@@ -31,6 +31,14 @@ class Report:
     n_prefetch_copies: int = 0
     n_demand_copies: int = 0
     ffn_checked: int = 0
+    # sums of the oracle's per-token metrics over the steps without near-ties (S9)
+    sum_delta_hat: int = 0
+    sum_delta_star: int = 0
+    sum_ncand: int = 0
+    hits_P: int = 0
+    hits_R: int = 0
+    covered: int = 0
+    capped: int = 0
 
 
 class Problem:
@@ -189,6 +197,14 @@ def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T:
             rep.n_miss_steps += int(len(out["missing"]) > 0)
             for b in range(B):
                 tok = out["tokens"][b]
+                if use_prefetch:
+                    rep.sum_delta_hat += tok["delta_hat"]
+                    rep.sum_delta_star += tok["delta_star"]
+                    rep.sum_ncand += k + tok["delta_hat"]
+                    rep.hits_P += int(round(tok["overlap_P"] * k))
+                    rep.covered += int(tok["covered"])
+                    rep.capped += tok["capped"]
+                    rep.hits_R += int(round(tok["overlap_R"] * k))
                 rep.n_subst += tok["n_subst"]
                 np.testing.assert_allclose(g_gate[b], tok["gates"], rtol=2e-5, atol=1e-7)
                 if norm_topk:

@@ -25,6 +25,12 @@ def _run(cfg, *, mode, tau, T, B=1, layers=None, C=None, norm_topk=1, cache_reus
         stats = apex.get_stats()
     finally:
         apex.destroy()
+    if use_prefetch and rep.near_ties == 0:
+        # S9: the device-side counters equal the oracle's metrics summed over the run
+        for key in ("sum_delta_hat", "sum_delta_star", "sum_ncand", "hits_P", "hits_R", "covered", "capped"):
+            assert stats[key] == getattr(rep, key), (key, stats[key], getattr(rep, key))
+        assert stats["prefetch_copies"] == rep.n_prefetch_copies and stats["demand_copies"] == rep.n_demand_copies
+        assert stats["substitutions"] == rep.n_subst
     return rep, stats
 
 
@@ -191,6 +197,35 @@ def test_decode_token_matches_per_call_sequence_and_counts_launches():
         a4.decode_token(h[0], hp[0], 1, 0.9, "exact", y1); torch.cuda.synchronize()
         torch.testing.assert_close(yh.cuda(), y1, rtol=1e-4, atol=1e-5)
         a3.destroy(); a4.destroy()
+    finally:
+        a1.destroy(); a2.destroy()
+
+
+def test_slot_table_checkpoint_and_resume():
+    # snapshot the slot tables after a few tokens, restore them into a fresh context, continue: same outputs
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=6, L=2, T=8, cfg_id=222)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    a1, a2 = prob.make_ctx(), prob.make_ctx()
+    try:
+        hs = [synth.hidden_states(cfg, l, cfg.T) for l in range(cfg.L)]
+        h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()
+        hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
+        y1 = torch.empty((cfg.L, 1, cfg.d), device="cuda"); y2 = torch.empty_like(y1)
+        for t in range(4):
+            a1.decode_token(h[t], hp[t], 1, 0.8, "exact", y1)
+        torch.cuda.synchronize()
+        for l in range(cfg.L):
+            es, st, clk = a1.get_slot_table(l)
+            a2.set_slot_table(l, es, st, clk)
+        for t in range(4, 8):
+            a1.decode_token(h[t], hp[t], 1, 0.8, "exact", y1)
+            a2.decode_token(h[t], hp[t], 1, 0.8, "exact", y2)
+            torch.cuda.synchronize()
+            torch.testing.assert_close(y1, y2, rtol=1e-4, atol=1e-5)
+            for l in range(cfg.L):
+                t1, t2 = a1.get_slot_table(l), a2.get_slot_table(l)
+                assert list(t1[0]) == list(t2[0]) and list(t1[1]) == list(t2[1]) and t1[2] == t2[2]
     finally:
         a1.destroy(); a2.destroy()
 

@@ -377,3 +377,20 @@ def test_config1_full_size_decode_token_sampled_layers(mode):
         print("config1 full", mode, "worst rel-L2", worst, st)
     finally:
         apex.destroy()
+
+
+def test_config1_long_run_counts_near_ties():
+    """1024 decode steps of one config-1 layer in lock-step: every decision of every step against the
+    oracle (FFN output on every 64th step).  Reports how many steps had a near-tie (deciding logit gap
+    below 1e-6) -- those are the only steps where an index may differ, and they are excused and counted."""
+    cfg = synth.CONFIGS[1]
+    hz = _harness()
+    prob = hz.Problem(cfg, layers=1, cdf="fitted")
+    apex = prob.make_ctx()
+    try:
+        rep = hz.run_lockstep(prob, apex, mode="exact", tau=0.9, T=cfg.T, check_ffn_every=64)
+    finally:
+        apex.destroy()
+    assert rep.layer_steps == 1024
+    assert rep.near_ties <= 2, rep          # expected about 1e-3 per run for 40 logits of unit spread
+    print("config1 long run:", rep)

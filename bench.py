@@ -103,16 +103,20 @@ def algorithmic_bytes(cfg, B=1):
 
 
 # ------------------------------------------------------------------------------------------------
-def build_problem(cfg, device):
+def build_problem(cfg, device, fp8=False):
     import torch
     from paper_2608_11688_b200 import synth
     routers = [synth.router_weights(cfg, l) for l in range(cfg.L)]
     cdf = [synth.cdf_params(cfg, l) for l in range(cfg.L)]
-    store = torch.empty((cfg.L, cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16, pin_memory=True)
+    if fp8:     # datatype study (Sec. V-G): e4m3 rows with per-row scales
+        store = torch.empty((cfg.L, cfg.N, cfg.I, 3 * cfg.d + 16), dtype=torch.uint8, pin_memory=True)
+    else:
+        store = torch.empty((cfg.L, cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16, pin_memory=True)
     shared = []
     for l in range(cfg.L):
-        store[l].copy_(synth.expert_store(cfg, l, device=device))
-        shared.append(synth.shared_expert(cfg, l, device=device))
+        store[l].copy_(synth.expert_store_fp8(cfg, l, device=device) if fp8 else synth.expert_store(cfg, l, device=device))
+        sh = synth.shared_expert(cfg, l, device=device)
+        shared.append(synth.quantize_store_fp8(sh) if (fp8 and sh is not None) else sh)
     torch.cuda.synchronize()
     return routers, cdf, store, shared
 
@@ -120,7 +124,9 @@ def build_problem(cfg, device):
 def make_ctx(cfg, prob, C, max_batch=1):
     from paper_2608_11688_b200 import binding
     routers, cdf, store, shared = prob
-    a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C, L=cfg.L, I_shared=cfg.I_shared, max_batch=max_batch)
+    fp8 = store.dtype != __import__("torch").bfloat16
+    a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C, L=cfg.L, I_shared=cfg.I_shared, max_batch=max_batch,
+                     flags=binding.FLAG_FP8_EXPERTS if fp8 else 0)
     for l in range(cfg.L):
         W_r, b_r, W_p, b_p = routers[l]
         a.set_router(l, W_r, b_r)
@@ -276,7 +282,11 @@ def main():
                     help="also time the baselines of the paper's comparison: no prefetch, static top-k, top-(k+4), top-(k+8)")
     ap.add_argument("--resident", action="store_true",
                     help="cache as large as the expert count, warmed up: no host-link copies (kernel launch lists)")
+    ap.add_argument("--fp8", action="store_true",
+                    help="datatype study: e4m3 expert store with per-row scales (needs --ffn-only or --skip-extras)")
     args = ap.parse_args()
+    if args.fp8 and not (args.ffn_only or args.skip_extras):
+        ap.error("--fp8 is a study leg: combine it with --ffn-only or --skip-extras")
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -307,7 +317,8 @@ def main():
         replicas.barrier()
         dist_sync = replicas.barrier
     B = args.batch
-    prob = build_problem(cfg, dev)
+    prob = build_problem(cfg, dev, fp8=args.fp8)
+    row_scale = (3 * cfg.d + 16) / (6 * cfg.d) if args.fp8 else 1.0     # bytes of a stored row relative to bf16
     T = min(cfg.T, args.warmup + args.steps)
     h, hp = hidden_inputs(cfg, T, B, dev)
     h_dev, hp_dev = h.to(dev), hp.to(dev)
@@ -324,8 +335,9 @@ def main():
         else:   # expected number of distinct experts touched by B tokens with uniform routing
             distinct = cfg.N * (1.0 - (1.0 - cfg.k / cfg.N) ** B)
             bytes_ffn = distinct * cfg.expert_bytes + cfg.shared_bytes + 2 * B * cfg.d * 4
+        bytes_ffn = (bytes_ffn - 2 * B * cfg.d * 4) * row_scale + 2 * B * cfg.d * 4
         flops = 2.0 * 3 * cfg.d * (cfg.k * cfg.I + cfg.I_shared) * B
-        print(json.dumps({"ffn_only": True, "B": B, "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6,
+        print(json.dumps({"ffn_only": True, "B": B, "weights": "e4m3" if args.fp8 else "bf16", "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6,
                           "launches": n_l, "GBps_mean": bytes_ffn / mean_s / 1e9, "bytes_per_launch": bytes_ffn,
                           "TFLOPs": flops / mean_s / 1e12}), flush=True)
         a.destroy()
@@ -436,8 +448,9 @@ def main():
         return
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "bf16", "data": "synthetic",
-            "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}", "L": cfg.L, "d": cfg.d, "N": cfg.N, "k": cfg.k,
+            "dtype": "e4m3 weights, fp32 accumulation" if args.fp8 else "bf16", "data": "synthetic",
+            "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}" + (" (e4m3 expert store)" if args.fp8 else ""),
+                       "L": cfg.L, "d": cfg.d, "N": cfg.N, "k": cfg.k,
                        "I": cfg.I, "C": cfg.N if args.resident else cfg.C, "B": B, "tau": TAU, "mode": "exact", "ctx_len": 1024,
                        "parallelism": "replicas only" if world > 1 else "single GPU",
                        "l2": "inputs larger than L2: each token streams %.0f MB of expert and attention bytes" %

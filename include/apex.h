@@ -29,6 +29,11 @@
  * where downT_i[j] = W_down[j][i] (the down projection transposed), so that index i owns one
  * contiguous block of 3*d values.  apex_pack_expert() converts from the usual
  * gate[I][d], up[I][d], down[d][I].
+ * With APEX_FLAG_FP8_EXPERTS (the expert-weight precision study of Sec. V-G: smaller experts, smaller
+ * copies) a row is 3*d e4m3 codes followed by three fp32 scales and 4 bytes of padding,
+ *   [I][ gate_i (d bytes) | up_i (d bytes) | downT_i (d bytes) | s_gate, s_up, s_down, 0 ],
+ * weight = scale * code; 3*d + 16 bytes per row.  Needs d in {512, 1024, 1536, 2048, 4096}; batched steps
+ * then run the streaming kernel per (token, expert) pair (no tensor-core path for this format yet).
  */
 #ifndef APEX_H
 #define APEX_H
@@ -51,6 +56,8 @@ extern "C" {
 #define APEX_MODE_EXACT 0      /* correctness-preserving: follow K_r, fetch what is missing */
 #define APEX_MODE_STALL_FREE 1 /* Algorithm 1: resident experts only, gates renormalised */
 
+#define APEX_FLAG_FP8_EXPERTS 1 /* apex_config.flags: expert stores and slots hold e4m3 rows (see below) */
+
 #define APEX_MAX_EXPERTS 64
 #define APEX_MAX_TOPK 16
 #define APEX_MAX_BATCH 256
@@ -70,7 +77,7 @@ typedef struct apex_config {
   int32_t norm_topk;     /* 1: g_e = alpha_e / sum over the executed set; 0: g_e = alpha_e */
   int32_t cache_reuse;   /* 1: slots persist across steps; 0: load-use-evict per layer-step */
   int32_t ctx_len;       /* context length that sizes the stand-in attention kernel */
-  int32_t flags;         /* reserved, 0 */
+  int32_t flags;         /* APEX_FLAG_* bits */
   int64_t wait_limit_ns; /* bound of every host- and device-side wait; 0 = 2 s */
 } apex_config;
 

@@ -18,6 +18,7 @@ LIB_PATH = os.path.join(_HERE, "libapex.so")
 APEX_OK, APEX_EINVAL, APEX_ENOMEM, APEX_ECUDA, APEX_ETIMEOUT, APEX_ESTATE, APEX_ENOTIMPL = 0, -1, -2, -3, -4, -5, -6
 MODE_EXACT, MODE_STALL_FREE = 0, 1
 MODES = {"exact": MODE_EXACT, "stall_free": MODE_STALL_FREE}
+FLAG_FP8_EXPERTS = 1
 ERR_NAMES = {0: "APEX_OK", -1: "APEX_EINVAL", -2: "APEX_ENOMEM", -3: "APEX_ECUDA", -4: "APEX_ETIMEOUT",
              -5: "APEX_ESTATE", -6: "APEX_ENOTIMPL"}
 
@@ -132,10 +133,10 @@ class Apex:
     """One context.  Methods mirror the C entry points one to one (apex_ prefix dropped)."""
 
     def __init__(self, *, d, N, k, I, C_slots, L=1, I_shared=0, max_batch=1, norm_topk=1, cache_reuse=1,
-                 ctx_len=1024, wait_limit_ns=0):
+                 ctx_len=1024, wait_limit_ns=0, flags=0):
         self.lib = load_library()
         self.cfg = ApexConfig(d=d, N=N, k=k, I=I, I_shared=I_shared, C=C_slots, L=L, max_batch=max_batch,
-                              norm_topk=norm_topk, cache_reuse=cache_reuse, ctx_len=ctx_len, flags=0,
+                              norm_topk=norm_topk, cache_reuse=cache_reuse, ctx_len=ctx_len, flags=flags,
                               wait_limit_ns=wait_limit_ns)
         h = C.c_void_p()
         rc = self.lib.apex_create(C.byref(self.cfg), C.byref(h))
@@ -179,7 +180,7 @@ class Apex:
         self._chk(self.lib.apex_set_cdf(self.h, layer, _ptr(w), _ptr(th)))
 
     def register_experts(self, layer, store, stride_bytes=None):
-        """store: pinned torch bf16 tensor [N][I][3][d] in the store layout."""
+        """store: pinned torch tensor in the store layout, bf16 [N][I][3][d] (uint8 [N][I][3*d+16] with FLAG_FP8_EXPERTS)."""
         self._keep.append(store)
         stride = stride_bytes if stride_bytes is not None else store.stride(0) * store.element_size()
         self._chk(self.lib.apex_register_experts(self.h, layer, _ptr(store), stride))

@@ -140,6 +140,7 @@ struct FfnParams {
   const uint32_t* demand;       // [N] per layer: (tag << 8 | slot), published by the host after a demand copy
   uint32_t demand_tag;          // tag of this launch
   int demand_in_kernel;         // 1: a routed expert without a slot is waited for inside the kernel
+  int fp8;                      // 1: slots hold e4m3 rows with per-row scales
   int zero_early;               // 1: y may be zeroed before the dependency wait (the preceding kernel does not touch y)
   SlotSnapshot snap;
   size_t slot_stride;
@@ -181,6 +182,7 @@ bool tc_make_weight_map(void* out, const void* base, int d, int I, size_t n_slot
 bool tc_make_rows_map(void* out, const void* base, int cols, size_t rows, size_t stride_elems);
 bool tc_shape_supported(int d, int I, int I_shared);
 bool ffn_shape_supported(int d);
+bool ffn_fp8_shape_supported(int d);
 
 }  // namespace apex
 

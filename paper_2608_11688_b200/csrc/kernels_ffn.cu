@@ -16,6 +16,7 @@
 // atomics.  Launched with programmatic stream serialization: the prologue overlaps the tail of the
 // gate kernel.
 #include <cuda_bf16.h>
+#include <cuda_fp16.h>
 
 #include "apex_internal.hpp"
 
@@ -111,6 +112,29 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned 
 }
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
+
+// Eight consecutive weights of a row as fp32: bf16 (16 bytes) or e4m3 (8 bytes; the row's scale is applied later).
+template <bool FP8>
+__device__ __forceinline__ void load8(const uint8_t* row, int idx8, float (&w)[8]) {
+  if (FP8) {
+    const uint2 v = reinterpret_cast<const uint2*>(row)[idx8];
+    uint32_t h2[4];
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2[0]) : "h"((unsigned short)(v.x & 0xffffu)));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2[1]) : "h"((unsigned short)(v.x >> 16)));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2[2]) : "h"((unsigned short)(v.y & 0xffffu)));
+    asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2[3]) : "h"((unsigned short)(v.y >> 16)));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2[i]));
+      w[2 * i] = f.x;
+      w[2 * i + 1] = f.y;
+    }
+  } else {
+    const uint4 v = reinterpret_cast<const uint4*>(row)[idx8];
+    w[0] = bf16lo(v.x); w[1] = bf16hi(v.x); w[2] = bf16lo(v.y); w[3] = bf16hi(v.y);
+    w[4] = bf16lo(v.z); w[5] = bf16hi(v.z); w[6] = bf16lo(v.w); w[7] = bf16hi(v.w);
+  }
+}
 
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
 #pragma unroll
@@ -373,7 +397,7 @@ __device__ __forceinline__ int nth_set_bit64(unsigned long long m, int n) {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-template <int NCH, bool H_REGS>
+template <int NCH, bool H_REGS, bool FP8>
 __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const FfnParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t s_full[kMaxStages];
@@ -383,8 +407,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   __shared__ int s_abort;
 
   constexpr int d = NCH * 256;
-  constexpr uint32_t row_bytes = d * 2;
-  constexpr uint32_t entry_bytes = 3 * row_bytes;
+  constexpr uint32_t row_bytes = FP8 ? d : d * 2;                      // one of the three vectors of a row
+  constexpr uint32_t entry_bytes = FP8 ? 3 * row_bytes + 16 : 3 * row_bytes;  // e4m3 rows carry three fp32 scales
   // Each warp streams its own rows: it owns the ring stages {w, w+8, ...} and keeps NSW of its rows
   // in flight, so a stage is produced and consumed by the same warp (no "empty" barriers, and a
   // parity wait can never be a phase ahead).
@@ -720,46 +744,44 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
         }
       }
     }
-    const uint4* gs = reinterpret_cast<const uint4*>(smem + (size_t)s * entry_bytes);
-    const uint4* us = gs + row_bytes / 16;
-    const uint4* ds = us + row_bytes / 16;
+    const uint8_t* gs = smem + (size_t)s * entry_bytes;
+    const uint8_t* us = gs + row_bytes;
+    const uint8_t* ds = us + row_bytes;
     float g = 0.f, u = 0.f;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
-      const uint4 gv = gs[c * 32 + lane];
-      const uint4 uv = us[c * 32 + lane];
-      float h0, h1, h2, h3, h4, h5, h6, h7;
+      float gw[8], uw[8], hh[8];
+      load8<FP8>(gs, c * 32 + lane, gw);
+      load8<FP8>(us, c * 32 + lane, uw);
       if (H_REGS) {
-        h0 = hreg[c * 8 + 0]; h1 = hreg[c * 8 + 1]; h2 = hreg[c * 8 + 2]; h3 = hreg[c * 8 + 3];
-        h4 = hreg[c * 8 + 4]; h5 = hreg[c * 8 + 5]; h6 = hreg[c * 8 + 6]; h7 = hreg[c * 8 + 7];
+#pragma unroll
+        for (int m = 0; m < 8; ++m) hh[m] = hreg[c * 8 + m];
       } else {
         const float4 a = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2);
         const float4 b2 = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2 + 1);
-        h0 = a.x; h1 = a.y; h2 = a.z; h3 = a.w; h4 = b2.x; h5 = b2.y; h6 = b2.z; h7 = b2.w;
+        hh[0] = a.x; hh[1] = a.y; hh[2] = a.z; hh[3] = a.w; hh[4] = b2.x; hh[5] = b2.y; hh[6] = b2.z; hh[7] = b2.w;
       }
-      g = fmaf(bf16lo(gv.x), h0, g); g = fmaf(bf16hi(gv.x), h1, g);
-      g = fmaf(bf16lo(gv.y), h2, g); g = fmaf(bf16hi(gv.y), h3, g);
-      g = fmaf(bf16lo(gv.z), h4, g); g = fmaf(bf16hi(gv.z), h5, g);
-      g = fmaf(bf16lo(gv.w), h6, g); g = fmaf(bf16hi(gv.w), h7, g);
-      u = fmaf(bf16lo(uv.x), h0, u); u = fmaf(bf16hi(uv.x), h1, u);
-      u = fmaf(bf16lo(uv.y), h2, u); u = fmaf(bf16hi(uv.y), h3, u);
-      u = fmaf(bf16lo(uv.z), h4, u); u = fmaf(bf16hi(uv.z), h5, u);
-      u = fmaf(bf16lo(uv.w), h6, u); u = fmaf(bf16hi(uv.w), h7, u);
+#pragma unroll
+      for (int m = 0; m < 8; ++m) g = fmaf(gw[m], hh[m], g);
+#pragma unroll
+      for (int m = 0; m < 8; ++m) u = fmaf(uw[m], hh[m], u);
     }
     g = warp_sum(g);
     u = warp_sum(u);
-    const float a = gate * (g / (1.f + expf(-g))) * u;
+    float down_scale = 1.f;
+    if (FP8) {  // per-row scales of the e4m3 store: value = scale * code
+      const float* sc = reinterpret_cast<const float*>(ds + row_bytes);
+      g *= sc[0];
+      u *= sc[1];
+      down_scale = sc[2];
+    }
+    const float a = gate * (g / (1.f + expf(-g))) * u * down_scale;
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
-      const uint4 dv = ds[c * 32 + lane];
-      acc[c * 8 + 0] = fmaf(a, bf16lo(dv.x), acc[c * 8 + 0]);
-      acc[c * 8 + 1] = fmaf(a, bf16hi(dv.x), acc[c * 8 + 1]);
-      acc[c * 8 + 2] = fmaf(a, bf16lo(dv.y), acc[c * 8 + 2]);
-      acc[c * 8 + 3] = fmaf(a, bf16hi(dv.y), acc[c * 8 + 3]);
-      acc[c * 8 + 4] = fmaf(a, bf16lo(dv.z), acc[c * 8 + 4]);
-      acc[c * 8 + 5] = fmaf(a, bf16hi(dv.z), acc[c * 8 + 5]);
-      acc[c * 8 + 6] = fmaf(a, bf16lo(dv.w), acc[c * 8 + 6]);
-      acc[c * 8 + 7] = fmaf(a, bf16hi(dv.w), acc[c * 8 + 7]);
+      float dw[8];
+      load8<FP8>(ds, c * 32 + lane, dw);
+#pragma unroll
+      for (int m = 0; m < 8; ++m) acc[c * 8 + m] = fmaf(a, dw[m], acc[c * 8 + m]);
     }
     __syncwarp();  // every lane has read stage s: it may be refilled
     {
@@ -865,15 +887,15 @@ extern "C" int apex_debug_reset_spans() {
 }
 #endif
 
-template <int NCH>
+template <int NCH, bool FP8>
 static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
   constexpr bool HR = NCH <= 8;
-  constexpr uint32_t entry = 3 * NCH * 256 * 2;
+  constexpr uint32_t entry = FP8 ? 3 * NCH * 256 + 16 : 3 * NCH * 256 * 2;
   constexpr int NS = ring_stages(entry);
   const size_t smem = (size_t)NS * entry;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(moe_ffn_stream_kernel<NCH, HR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(moe_ffn_stream_kernel<NCH, HR, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -887,7 +909,7 @@ static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, moe_ffn_stream_kernel<NCH, HR>, p);
+  return cudaLaunchKernelEx(&cfg, moe_ffn_stream_kernel<NCH, HR, FP8>, p);
 }
 
 bool ffn_shape_supported(int d) {
@@ -901,17 +923,29 @@ bool ffn_shape_supported(int d) {
 cudaError_t ffn_configure(int) { return cudaSuccess; }
 
 cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s) {
+  if (p.fp8) {  // e4m3 store: the shapes of the paper-sized configs
+    switch (p.d) {
+      case 1024: return launch_ffn_t<4, true>(p, n_sm, s);
+      case 1536: return launch_ffn_t<6, true>(p, n_sm, s);
+      case 2048: return launch_ffn_t<8, true>(p, n_sm, s);
+      case 4096: return launch_ffn_t<16, true>(p, n_sm, s);
+      case 512: return launch_ffn_t<2, true>(p, n_sm, s);
+    }
+    return cudaErrorInvalidValue;
+  }
   switch (p.d) {
-    case 256: return launch_ffn_t<1>(p, n_sm, s);
-    case 512: return launch_ffn_t<2>(p, n_sm, s);
-    case 768: return launch_ffn_t<3>(p, n_sm, s);
-    case 1024: return launch_ffn_t<4>(p, n_sm, s);
-    case 1536: return launch_ffn_t<6>(p, n_sm, s);
-    case 2048: return launch_ffn_t<8>(p, n_sm, s);
-    case 3072: return launch_ffn_t<12>(p, n_sm, s);
-    case 4096: return launch_ffn_t<16>(p, n_sm, s);
+    case 256: return launch_ffn_t<1, false>(p, n_sm, s);
+    case 512: return launch_ffn_t<2, false>(p, n_sm, s);
+    case 768: return launch_ffn_t<3, false>(p, n_sm, s);
+    case 1024: return launch_ffn_t<4, false>(p, n_sm, s);
+    case 1536: return launch_ffn_t<6, false>(p, n_sm, s);
+    case 2048: return launch_ffn_t<8, false>(p, n_sm, s);
+    case 3072: return launch_ffn_t<12, false>(p, n_sm, s);
+    case 4096: return launch_ffn_t<16, false>(p, n_sm, s);
   }
   return cudaErrorInvalidValue;
 }
+
+bool ffn_fp8_shape_supported(int d) { return d == 512 || d == 1024 || d == 1536 || d == 2048 || d == 4096; }
 
 }  // namespace apex

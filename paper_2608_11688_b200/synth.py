@@ -180,6 +180,51 @@ def split_store(w):
     return w[..., 0, :], w[..., 1, :], np.swapaxes(w[..., 2, :], -1, -2)
 
 
+def quantize_store_fp8(w):
+    """bf16/fp32 store [..., I, 3, d] -> uint8 [..., I, 3*d + 16] in the library's e4m3 row layout.
+
+    Per row (one of gate_i, up_i, downT_i) the scale is max|row| / 448 (448 = largest e4m3 value; 1 for an all-zero
+    row), the codes are the row divided by its scale, rounded to e4m3 by torch's cast.  A row block is
+    3*d code bytes, then the three fp32 scales, then 4 zero bytes.
+    """
+    import torch
+    wf = w.to(torch.float32)
+    d = wf.shape[-1]
+    amax = wf.abs().amax(dim=-1, keepdim=True)
+    scale = torch.where(amax > 0, amax / 448.0, torch.ones_like(amax))
+    codes = (wf / scale).to(torch.float8_e4m3fn).view(torch.uint8)             # [..., I, 3, d]
+    lead = codes.shape[:-2]
+    out = torch.zeros(lead + (3 * d + 16,), dtype=torch.uint8, device=w.device)
+    out[..., :3 * d] = codes.reshape(lead + (3 * d,))
+    sc = torch.zeros(lead + (4,), dtype=torch.float32, device=w.device)
+    sc[..., :3] = scale.squeeze(-1)
+    out[..., 3 * d:] = sc.view(torch.uint8).reshape(lead + (16,))
+    return out
+
+
+def dequantize_store_fp8(q, d: int) -> np.ndarray:
+    """uint8 [..., I, 3*d + 16] -> fp64 numpy [..., I, 3, d]: weight = scale * code, multiplied in fp64 (the
+    product of an e4m3 value and an fp32 scale is exact there)."""
+    import torch
+    q = q.detach().cpu()
+    lead = q.shape[:-1]
+    codes = q[..., :3 * d].contiguous().view(torch.float8_e4m3fn).to(torch.float32).reshape(lead + (3, d)).numpy()
+    sc = q[..., 3 * d:].contiguous().view(torch.float32)[..., :3].numpy()
+    return codes.astype(np.float64) * sc[..., None].astype(np.float64)
+
+
+def expert_store_fp8(cfg: Config, layer: int, device="cpu"):
+    """uint8 tensor [N][I][3*d+16]: the seeded bf16 store of ``expert_store`` quantised row by row."""
+    import torch
+    out = torch.empty((cfg.N, cfg.I, 3 * cfg.d + 16), dtype=torch.uint8, device=device)
+    g = torch.Generator(device=device)
+    g.manual_seed((BASE_SEED * 1000003 + cfg.cfg_id * 10007 + layer * 101 + _KIND["experts"]) & 0x7FFFFFFF)
+    for e in range(cfg.N):
+        t = torch.randn((cfg.I, 3, cfg.d), generator=g, device=device, dtype=torch.float32)
+        out[e].copy_(quantize_store_fp8((t * 0.02).to(torch.bfloat16)))
+    return out
+
+
 def bf16_to_f32_numpy(t) -> np.ndarray:
     """Lossless widening of a torch bf16 tensor to a numpy fp32 array (test helper)."""
     import torch

@@ -44,8 +44,9 @@ class Report:
 class Problem:
     """Parameters and expert stores of one config on the GPU machine, shared by library and oracle."""
 
-    def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset"):
+    def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset", fp8=False):
         self.cfg = cfg
+        self.fp8 = fp8
         self.L = layers or cfg.L
         self.routers = [synth.router_weights(cfg, l) for l in range(self.L)]
         self.cdf = [synth.handset_cdf_params(cfg) if cdf == "handset" else synth.cdf_params(cfg, l)
@@ -53,12 +54,19 @@ class Problem:
         self.stores = []
         self.shared = []
         for l in range(self.L):
-            st = torch.empty((cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16, pin_memory=True)
-            tmp = synth.expert_store(cfg, l, device=device)
+            if fp8:
+                st = torch.empty((cfg.N, cfg.I, 3 * cfg.d + 16), dtype=torch.uint8, pin_memory=True)
+                tmp = synth.expert_store_fp8(cfg, l, device=device)
+            else:
+                st = torch.empty((cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16, pin_memory=True)
+                tmp = synth.expert_store(cfg, l, device=device)
             st.copy_(tmp)
             del tmp
             self.stores.append(st)
-            self.shared.append(synth.shared_expert(cfg, l, device=device))
+            sh = synth.shared_expert(cfg, l, device=device)
+            if fp8 and sh is not None:
+                sh = synth.quantize_store_fp8(sh)
+            self.shared.append(sh)
         torch.cuda.synchronize()
 
     def make_ctx(self, *, C=None, max_batch=1, norm_topk=1, cache_reuse=1, wait_limit_ns=0) -> binding.Apex:
@@ -66,7 +74,7 @@ class Problem:
         build.build()
         a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C or cfg.C, L=self.L, I_shared=cfg.I_shared,
                          max_batch=max_batch, norm_topk=norm_topk, cache_reuse=cache_reuse,
-                         wait_limit_ns=wait_limit_ns)
+                         wait_limit_ns=wait_limit_ns, flags=binding.FLAG_FP8_EXPERTS if self.fp8 else 0)
         for l in range(self.L):
             W_r, b_r, W_p, b_p = self.routers[l]
             a.set_router(l, W_r, b_r)
@@ -81,6 +89,8 @@ class Problem:
         st = self.stores[layer]
 
         def get(e):
+            if self.fp8:
+                return synth.split_store(synth.dequantize_store_fp8(st[e], self.cfg.d))
             w = st[e].to(torch.float32).numpy()
             return synth.split_store(w)
         return get
@@ -89,6 +99,8 @@ class Problem:
         sh = self.shared[layer]
         if sh is None:
             return None
+        if self.fp8:
+            return synth.split_store(synth.dequantize_store_fp8(sh, self.cfg.d))
         w = sh.detach().cpu().to(torch.float32).numpy()
         return synth.split_store(w)
 

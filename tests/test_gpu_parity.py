@@ -116,6 +116,39 @@ def test_batched_exact_mode_runs_in_waves_when_cache_is_smaller_than_need():
     assert stats["extra_waves"] >= 4 * 2          # at least two extra waves per step: need > 2 C
 
 
+# ------------------------------------------------------------------ e4m3 expert store (Sec. V-G)
+def _run_fp8(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1):
+    hz = _harness()
+    prob = hz.Problem(cfg, layers=layers, fp8=True)
+    return _run(cfg, mode=mode, tau=tau, T=T, B=B, layers=layers, prob=prob, check_ffn_every=check_ffn_every)
+
+
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+@pytest.mark.parametrize("d,N,k,I,C,Ish", [(512, 12, 3, 40, 6, 0), (1024, 16, 4, 17, 8, 24), (2048, 8, 2, 9, 4, 0),
+                                            (4096, 6, 2, 5, 3, 7)])
+def test_fp8_store_tiny_shapes(d, N, k, I, C, Ish, mode):
+    cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, T=8, I_shared=Ish, sigma_p=1.0, cfg_id=260 + N)
+    rep, stats = _run_fp8(cfg, mode=mode, tau=0.7, T=8)
+    assert rep.layer_steps == 8 and rep.ffn_checked + rep.near_ties >= 8
+    assert stats["bytes_copied"] == (rep.n_prefetch_copies + rep.n_demand_copies) * I * (3 * d + 16)
+    print("fp8", d, mode, rep)
+
+
+@pytest.mark.parametrize("B", [3, 16])
+def test_fp8_store_batched_runs_streaming_kernel(B):
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=128, C=8, T=3, I_shared=128, sigma_p=1.0, cfg_id=275)
+    rep, stats = _run_fp8(cfg, mode="exact", tau=0.8, T=3, B=B)
+    assert stats["tokens"] == 3 * B
+
+
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_fp8_store_config1_shape_two_layers(mode):
+    cfg = synth.CONFIGS[1]
+    rep, stats = _run_fp8(cfg, mode=mode, tau=0.9, T=12, layers=2, check_ffn_every=3)
+    assert rep.layer_steps == 24
+    print("fp8 config1", mode, rep)
+
+
 # ------------------------------------------------------------------ the paper-shaped configs
 def test_config0_full():
     cfg = synth.CONFIGS[0]

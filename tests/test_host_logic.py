@@ -47,8 +47,30 @@ def test_null_and_bad_arguments_are_rejected_without_cuda(lib):
         kw.update(bad)
         cfg = binding.ApexConfig(**kw)
         assert lib.apex_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.APEX_EINVAL, bad
+    # the e4m3 store needs one of the widths its kernel was built for
+    cfg = binding.ApexConfig(d=768, N=8, k=2, I=8, I_shared=0, C=4, L=1, max_batch=1, norm_topk=1, cache_reuse=1,
+                             flags=binding.FLAG_FP8_EXPERTS)
+    assert lib.apex_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.APEX_EINVAL
     assert lib.apex_slots_create(8, 9, 1) is None
     assert lib.apex_launch_count(None) == -1
+
+
+def test_fp8_store_generator_round_trips_within_e4m3_precision():
+    import numpy as np
+    import torch
+    from paper_2608_11688_b200 import synth
+    cfg = synth.tiny_config(d=512, N=3, k=1, I=5)
+    w = synth.expert_store(cfg, 0).to(torch.float32).numpy()
+    q = synth.expert_store_fp8(cfg, 0)
+    assert q.shape == (3, 5, 3 * 512 + 16) and q.dtype == torch.uint8
+    dq = synth.dequantize_store_fp8(q, 512)
+    # e4m3 keeps 3 mantissa bits: relative error <= 2^-4 for normal codes; the per-row scale maps the
+    # row maximum to 448, so nothing overflows and the absolute error is <= amax * 2^-4
+    amax = np.abs(w).max(axis=-1, keepdims=True)
+    assert np.all(np.abs(dq - w) <= amax / 16 + 1e-12)
+    assert np.all(q[..., 3 * 512 + 12:].numpy() == 0)                          # padding bytes
+    # the row maximum is reproduced exactly (code 448 times scale)
+    assert np.allclose(np.abs(dq).max(axis=-1, keepdims=True), amax, rtol=1e-6)
 
 
 def test_pack_expert_transposes_down(lib):

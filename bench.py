@@ -33,7 +33,8 @@ TAU = 0.90
 
 # DRAM bytes per launch of the expert-FFN kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu capture summarised in profiles/ (same kernel, same per-launch shape).  None = not captured.
-NCU_TRAFFIC_BYTES = {1: 37_854_500}   # profiles/moe_ffn_stream_kernel_config1.md: 37.809 MB read + ~0.045 MB written
+NCU_TRAFFIC_BYTES = {1: 47_496_000}   # profiles/moe_ffn_stream_kernel_config1.md: mean of three launches (46.0, 42.1, 54.4 MB);
+#                                       37.8 MB of it is the executed experts, the rest speculative rows that were dropped
 
 
 def measured_peak():
@@ -121,12 +122,12 @@ def build_problem(cfg, device, fp8=False):
     return routers, cdf, store, shared
 
 
-def make_ctx(cfg, prob, C, max_batch=1):
+def make_ctx(cfg, prob, C, max_batch=1, flags=0):
     from paper_2608_11688_b200 import binding
     routers, cdf, store, shared = prob
     fp8 = store.dtype != __import__("torch").bfloat16
     a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C, L=cfg.L, I_shared=cfg.I_shared, max_batch=max_batch,
-                     flags=binding.FLAG_FP8_EXPERTS if fp8 else 0)
+                     flags=(binding.FLAG_FP8_EXPERTS if fp8 else 0) | flags)
     for l in range(cfg.L):
         W_r, b_r, W_p, b_p = routers[l]
         a.set_router(l, W_r, b_r)
@@ -171,8 +172,8 @@ def time_tokens(apex, h, hp, y, B, mode, warmup, steps, dist_sync=None, host=Fal
 
 
 def time_ffn_kernel(apex, cfg, h, hp, B, tokens):
-    """Average device time of one expert-FFN launch, all experts resident.  Per token the gates of all
-    layers run first; then the L expert-FFN kernels are launched back to back (each reads its own
+    """Average device time of one expert-FFN launch, all experts resident.  Per token the prefetch routers
+    and the gates of all layers run first; then the L expert-FFN kernels are launched back to back (each reads its own
     layer's experts, so nothing is served from L2) between two CUDA events on the launching stream."""
     import torch
     dev = h.device
@@ -183,8 +184,14 @@ def time_ffn_kernel(apex, cfg, h, hp, B, tokens):
     per_launch = []
     stream = torch.cuda.current_stream().cuda_stream
     y_ptr = [y[l].data_ptr() for l in range(cfg.L)]
+    cand = torch.empty((B, cfg.N), dtype=torch.int32, device=dev)
+    ncand = torch.empty((B,), dtype=torch.int32, device=dev)
     for t in range(tokens + 1):
         hp_ptr = [hp[t % T, l].data_ptr() for l in range(cfg.L)]
+        for l in range(cfg.L):      # the steps that precede the expert FFN in a decode step (nothing to copy: all resident)
+            apex.predict(l, h[t % T, l], B)
+            apex.select_candidates(l, B, TAU, cand, ncand)
+            apex.prefetch(l, B)
         for l in range(cfg.L):
             apex.route_topk(l, hp[t % T, l], B, idx[l], al[l])
         torch.cuda.synchronize()
@@ -282,6 +289,7 @@ def main():
                     help="also time the baselines of the paper's comparison: no prefetch, static top-k, top-(k+4), top-(k+8)")
     ap.add_argument("--resident", action="store_true",
                     help="cache as large as the expert count, warmed up: no host-link copies (kernel launch lists)")
+    ap.add_argument("--no-spec", action="store_true", help="A/B: expert FFN without the speculative first fill")
     ap.add_argument("--fp8", action="store_true",
                     help="datatype study: e4m3 expert store with per-row scales (needs --ffn-only or --skip-extras)")
     args = ap.parse_args()
@@ -327,7 +335,7 @@ def main():
     y_pin = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32).pin_memory()
 
     if args.ffn_only:
-        a = make_ctx(cfg, prob, cfg.N, max_batch=B)
+        a = make_ctx(cfg, prob, cfg.N, max_batch=B, flags=2 if args.no_spec else 0)
         a.warm_all()
         mean_s, med_s, n_l = time_ffn_kernel(a, cfg, h_dev, hp_dev, B, tokens=args.steps)
         if B == 1:
@@ -344,7 +352,7 @@ def main():
         return
 
     # ---- headline: config cache size, exact (correctness-preserving) mode, inputs resident in HBM
-    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B)
+    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B, flags=2 if args.no_spec else 0)
     if args.resident:
         apex.warm_all()
     sampler = ClockSampler(local_rank)

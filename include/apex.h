@@ -57,6 +57,9 @@ extern "C" {
 #define APEX_MODE_STALL_FREE 1 /* Algorithm 1: resident experts only, gates renormalised */
 
 #define APEX_FLAG_FP8_EXPERTS 1 /* apex_config.flags: expert stores and slots hold e4m3 rows (see below) */
+#define APEX_FLAG_NO_SPECULATION 2 /* apex_config.flags: the expert FFN does not start streaming the experts the prefetch
+                                      router ranked first before the gate's decision is visible (for A/B timing; results
+                                      are identical either way) */
 
 #define APEX_MAX_EXPERTS 64
 #define APEX_MAX_TOPK 16

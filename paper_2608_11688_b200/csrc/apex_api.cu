@@ -209,6 +209,8 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(cudaMemset(ctx->d_stats, 0, L * sizeof(DevStats)));
   CR(dev_alloc(&ctx->d_tickets, 64));
   CR(cudaMemset(ctx->d_tickets, 0, 64 * sizeof(unsigned int)));
+  CR(dev_alloc(&ctx->d_spec, L * APEX_MAX_TOPK));
+  CR(cudaMemset(ctx->d_spec, 0xff, L * APEX_MAX_TOPK * sizeof(int32_t)));
   CR(dev_alloc(&ctx->d_counters, 2));
   CR(cudaMemset(ctx->d_counters, 0, 2 * sizeof(unsigned long long)));
   const size_t max_pairs = MB * (k + 1);
@@ -301,7 +303,7 @@ int apex_destroy(apex_ctx* ctx) {
   cudaDeviceSynchronize();
   cudaGetLastError();
   void* dev[] = {ctx->d_Wr, ctx->d_br, ctx->d_Wp, ctx->d_bp, ctx->d_w, ctx->d_theta, ctx->d_cache, ctx->d_slot_ready, ctx->d_zp,
-                 ctx->d_qp, ctx->d_zr, ctx->d_demand, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_tickets, ctx->d_plan_exec_idx,
+                 ctx->d_qp, ctx->d_zr, ctx->d_demand, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_tickets, ctx->d_spec, ctx->d_plan_exec_idx,
                  ctx->d_plan_exec_gate, ctx->d_pair_tok, ctx->d_pair_gate, ctx->d_pair_expert, ctx->d_n_pairs, ctx->d_grp, ctx->d_xg, ctx->d_act, ctx->d_cand,
                  ctx->d_idx, ctx->d_exec_idx, ctx->d_alpha, ctx->d_exec_gate, ctx->d_cand_ncand, ctx->d_attn, ctx->d_attn_sink,
                  ctx->d_h_stage, ctx->d_hp_stage, ctx->d_y_stage};
@@ -415,7 +417,7 @@ int begin_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, RouterPar
   p->z_out = ctx->d_zp;
   p->q_out = ctx->d_qp;
   p->pi_out = ctx->d_pi;
-  p->topk_out = nullptr;
+  p->topk_out = B == 1 ? ctx->d_spec + (size_t)layer * APEX_MAX_TOPK : nullptr;  // the FFN's speculative first fill
   p->N = (int)N; p->d = (int)d; p->B = B; p->k = ctx->cfg.k; p->C = ctx->cfg.C;
   return APEX_OK;
 }
@@ -605,6 +607,7 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   st.routed = true;
+  st.route_stream = (cudaStream_t)stream;
   st.idx_dev = idx_dev;
   st.alpha_dev = alpha_dev;
   return APEX_OK;
@@ -690,7 +693,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.seq_value = ++ctx->exec_seq[layer];
   p.stats = ctx->d_stats + layer;
   p.zero_counter = ctx->d_counters + 1;
-  ctx->zero_done += (unsigned long long)ctx->n_sm;
+  ctx->zero_done += (unsigned long long)ffn_grid_ctas(ctx->n_sm);
   p.zero_target = ctx->zero_done;
   p.snap = make_snapshot(ctx, layer);
   p.slot_stride = ctx->expert_bytes;
@@ -705,6 +708,14 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.demand_tag = ctx->launch_tag;
   p.demand_in_kernel = (mode == APEX_MODE_EXACT && B == 1) ? 1 : 0;
   p.run_mask = p.demand_in_kernel ? ~0ull : p.snap.resident_mask;
+  // Speculative first fill: the kernel may start streaming the experts the prefetch router ranked
+  // first before the gate's decision is visible.  Allowed when that ranking is certainly complete by
+  // then: predicted in this step, its candidate record already seen by the host (apex_prefetch), and
+  // the gate kernel (which waits for everything before it) between the two on this same stream.
+  p.spec = (B == 1 && st.predicted && st.prefetched && ctx->pred_stream == cs && st.route_stream == cs &&
+            !(ctx->cfg.flags & APEX_FLAG_NO_SPECULATION))
+               ? ctx->d_spec + (size_t)layer * APEX_MAX_TOPK
+               : nullptr;
   if (B > 1) {
     int r = launch_batched(ctx, layer, p, cs);
     if (r != APEX_OK) return r;

@@ -142,6 +142,7 @@ struct FfnParams {
   int demand_in_kernel;         // 1: a routed expert without a slot is waited for inside the kernel
   int fp8;                      // 1: slots hold e4m3 rows with per-row scales
   int zero_early;               // 1: y may be zeroed before the dependency wait (the preceding kernel does not touch y)
+  const int32_t* spec;          // [k] predicted top-k of this layer-step (complete before the preceding kernel began), or null
   SlotSnapshot snap;
   size_t slot_stride;
   long long wait_limit_ns;
@@ -176,6 +177,7 @@ cudaError_t launch_select(const SelectParams& p, cudaStream_t s);
 cudaError_t launch_attention(const AttnParams& p, int n_sm, cudaStream_t s);
 cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s);
 cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s);
+int ffn_grid_ctas(int n_sm);  // CTAs of one streaming-kernel launch (each adds one to the zero counter)
 cudaError_t ffn_configure(int d);  // sets the dynamic shared-memory attribute once per shape
 cudaError_t launch_ffn_tc(const TcParams& p, const TcMaps& m, int n_sm, cudaStream_t s);
 bool tc_make_weight_map(void* out, const void* base, int d, int I, size_t n_slots, size_t slot_bytes, int box_rows);
@@ -238,6 +240,7 @@ struct apex_ctx {
   std::vector<uint32_t> exec_seq;                 // per layer, last value asked for
   unsigned long long sel_done = 0, zero_done = 0;
   unsigned int* d_tickets = nullptr;  // [64] ring of row-ticket counters
+  int32_t* d_spec = nullptr;          // [L][APEX_MAX_TOPK]: top-k of the prefetch router (B = 1), the FFN's speculative first fill
   uint32_t ffn_launch_id = 0;
   // what this context queued last, and where: an expert-FFN launch may still be adding to its y when
   // the next kernel's prologue runs (programmatic dependent launch)
@@ -261,6 +264,7 @@ struct apex_ctx {
   struct StepState {
     int B = 0;
     bool predicted = false, selected = false, prefetched = false, routed = false;
+    cudaStream_t route_stream = nullptr;   // stream of this step's gate kernel
     const int32_t* idx_dev = nullptr;
     const float* alpha_dev = nullptr;
     // an FFN launch whose host-side completion (LRU touch, demand copies) is still due

@@ -34,14 +34,24 @@ __device__ __forceinline__ unsigned long long globaltimer_ns_raw() {
   asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
   return t;
 }
+#define TLG(slot) do { g_timeline[blockIdx.x * 16 + (slot)] = globaltimer_ns_raw(); } while (0)
 #else
 #define TL(slot) do { } while (0)
+#define TLG(slot) do { } while (0)
 #endif
 
-constexpr int kConsumerWarps = 8;
+#ifndef APEX_FFN_WARPS
+#define APEX_FFN_WARPS 8
+#endif
+#ifndef APEX_FFN_CTAS_PER_SM
+#define APEX_FFN_CTAS_PER_SM 1
+#endif
+constexpr int kConsumerWarps = APEX_FFN_WARPS;
+constexpr int kCtasPerSm = APEX_FFN_CTAS_PER_SM;
 constexpr int kFfnThreads = kConsumerWarps * 32;
 constexpr int kMaxStages = 32;
-constexpr int kSmemBudget = 224 * 1024;  // ring bytes; static tables fit in what is left of the 227 KB per-CTA limit
+// ring bytes; static tables fit in what is left of the 227 KB per-CTA limit (of half an SM's 228 KB with two CTAs per SM)
+constexpr int kSmemBudget = kCtasPerSm == 1 ? 224 * 1024 : 110 * 1024;
 
 __host__ __device__ constexpr int ring_stages(uint32_t entry_bytes) {
   int n = kSmemBudget / (int)entry_bytes;
@@ -398,12 +408,13 @@ __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;"
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 template <int NCH, bool H_REGS, bool FP8>
-__global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const FfnParams p) {
+__global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel(const FfnParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t s_full[kMaxStages];
   __shared__ float s_gate[kMaxStages];
   __shared__ int s_tok[kMaxStages];
   __shared__ int s_exp[kMaxStages];
+  __shared__ int s_pos[kConsumerWarps][APEX_MAX_TOPK];  // B == 1: expert at each position of the row space (a copy per warp)
   __shared__ int s_abort;
 
   constexpr int d = NCH * 256;
@@ -461,67 +472,148 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     }
   };
   if (p.zero_early) zero_slice();
-  pdl_wait();               // the gate's outputs (K_r, alpha, z_r) are complete from here on
-  pdl_launch_dependents();  // the next kernel may start its own prologue
-  if (tid == 0) TL(4);
-  if (!p.zero_early) zero_slice();  // a preceding launch of this library may still be adding to the same y
 
-  // ---- every global load of the prologue is issued before the first use, so the latencies overlap.
   // Slot-ready flags: lanes own experts lane and lane+32.  The flag is written by the copy engine
   // after the expert's bytes; a relaxed load suffices here because the bulk copies that follow are
   // issued only after the value has been inspected (and they read through L2, like the flag).
+  // Neither the flags nor the slot snapshot come from the preceding kernel.
   const int sl0 = lane < N ? p.snap.expert_slot[lane] : -1, sl1 = lane + 32 < N ? p.snap.expert_slot[lane + 32] : -1;
   const uint32_t f0 = sl0 >= 0 ? ld_relaxed_sys(p.slot_ready + sl0) : 0u;
   const uint32_t f1 = sl1 >= 0 ? ld_relaxed_sys(p.slot_ready + sl1) : 0u;
-  TokenLoads tl1;
-  if (B == 1) tl1 = load_token(p.idx, p.z_r, p.alpha, N, k, p.mode, lane);
   unsigned long long ready_mask;
   {
     const bool r0 = sl0 >= 0 && (int32_t)(f0 - p.snap.need_gen[lane]) >= 0;
     const bool r1 = sl1 >= 0 && (int32_t)(f1 - p.snap.need_gen[(lane + 32) & 63]) >= 0;
     ready_mask = ((unsigned long long)__ballot_sync(0xffffffffu, r1) << 32) | __ballot_sync(0xffffffffu, r0);
   }
+
+  // Row space and work split.  Short launches (fewer than two ring fills per CTA): equal contiguous
+  // ranges, all known at launch, no shared counter (a ticket per row costs more than it balances
+  // there: every warp would hit one counter within the same microsecond).  Long launches: every CTA
+  // owns NS (the ring depth) consecutive rows, so all its stages are filled at once, and the remaining
+  // rows are handed out in tickets from a global counter to whichever warp has a free stage first.
+  RowMap rm;
+  bool dynamic = false;
+  int S = 0, chunk = 1, n_static = 0;
+  long long static_base = 0, dyn_begin = 0, dyn_rows = 0;
+  auto set_geometry = [&](int n_routed, int n_pairs) {
+    rm.n_routed = n_routed;
+    rm.n_pairs = n_pairs;
+    rm.routed_rows = (long long)n_routed * I;
+    rm.total_rows = rm.routed_rows + (long long)(n_pairs - n_routed) * p.I_shared;
+    const long long per_cta = rm.total_rows / G;
+    dynamic = per_cta >= 2 * NS;
+    const long long range_lo = rm.total_rows * cta / G, range_hi = rm.total_rows * (cta + 1) / G;
+    S = dynamic ? NS : (int)(range_hi - range_lo);  // rows this CTA knows about at launch
+    static_base = dynamic ? (long long)cta * NS : range_lo;
+    dyn_begin = dynamic ? (long long)G * NS : rm.total_rows;
+    dyn_rows = rm.total_rows - dyn_begin;
+    const long long per_ticket = (dyn_rows + (long long)G * kConsumerWarps * 4 - 1) / ((long long)G * kConsumerWarps * 4);
+    chunk = per_ticket > 1 ? (int)per_ticket : 1;   // rows per ticket: about four tickets per warp
+    n_static = S > warp ? (S - warp + kConsumerWarps - 1) / kConsumerWarps : 0;  // static rows of this warp
+  };
+  // (position in the row space, index inside the expert) of row r
+  auto locate = [&](long long r, int* pidx, long long* i) {
+    if (r < rm.routed_rows) {
+      *pidx = (int)(r / I);
+      *i = r - (long long)*pidx * I;
+    } else {
+      *pidx = rm.n_routed + (int)((r - rm.routed_rows) / p.I_shared);
+      *i = r - rm.routed_rows - (long long)(*pidx - rm.n_routed) * p.I_shared;
+    }
+  };
+
+  // ---- speculative first fill (B == 1).  The prefetch router ranked this step's experts long ago;
+  // its first k are the best guess of the routed set.  Their rows are requested now, while the gate
+  // kernel is still running; after the dependency wait each guess is either confirmed (the copy is
+  // already in flight or has landed) or dropped and its stage refilled.  Positions of the row space
+  // that hold a confirmed guess keep it, so confirmed rows stay with the CTA that requested them.
+  bool spec_on = B == 1 && p.spec != nullptr;
+  int spec_e = -1;
+  bool spec_issued = false;  // this lane started a speculative copy into its stage (stage index = lane)
+  if (spec_on) {
+    spec_e = lane < k ? __ldg(p.spec + lane) : -1;
+    const unsigned kmask = k >= 32 ? 0xffffffffu : ((1u << k) - 1u);
+    const bool bad = lane < k && (spec_e < 0 || spec_e >= N);
+    const unsigned same = __match_any_sync(0xffffffffu, spec_e);
+    const bool dup = lane < k && (same & kmask) != (1u << lane);
+    spec_on = !__any_sync(0xffffffffu, bad || dup);
+  }
+  if (spec_on) {
+    if (lane < k) s_pos[warp][lane] = spec_e;
+    __syncwarp();
+    set_geometry(k, k + (p.run_shared ? 1 : 0));
+    const int fill = n_static < NSW ? n_static : NSW;
+    if (lane < fill) {
+      int pidx;
+      long long i;
+      locate(static_base + warp + (long long)kConsumerWarps * lane, &pidx, &i);
+      const int e = pidx < k ? s_pos[warp][pidx] : N;
+      const uint8_t* base = nullptr;
+      if (e >= N) {
+        base = p.shared_w;
+      } else if ((ready_mask >> e) & 1) {
+        base = p.cache + (size_t)p.snap.expert_slot[e] * p.slot_stride;
+      }
+      if (base) {
+        const int s = warp + kConsumerWarps * lane;
+        s_gate[s] = 0.f;
+        s_tok[s] = 0;
+        s_exp[s] = e;
+        mbar_expect_tx(&s_full[s], entry_bytes);
+        bulk_g2s(smem + (size_t)s * entry_bytes, base + (size_t)i * entry_bytes, entry_bytes, &s_full[s]);
+        spec_issued = true;
+      }
+    }
+  }
+
+  pdl_wait();               // the gate's outputs (K_r, alpha, z_r) are complete from here on
+  pdl_launch_dependents();  // the next kernel may start its own prologue
+  if (tid == 0) TL(4);
+  if (tid == 0) TLG(11);
+  if (!p.zero_early) zero_slice();  // a preceding launch of this library may still be adding to the same y
+
+  // ---- every global load of the prologue is issued before the first use, so the latencies overlap.
+  TokenLoads tl1;
+  if (B == 1) tl1 = load_token(p.idx, p.z_r, p.alpha, N, k, p.mode, lane);
   if (tid == 0) TL(10);
 
   // ---- plan: B == 1 every warp derives the execution set itself; B > 1 the plan kernel wrote it
-  RowMap rm;
   unsigned long long run = 0;
   float g0 = 0.f, g1 = 0.f;
   TokenPlan tp1;
   tp1.exec_mask = tp1.kr_mask = 0ull;
   tp1.g0 = tp1.g1 = 0.f;
+  bool spec_geometry = false;  // the speculative row space is the final one
   if (B == 1) {
     const TokenPlan tp = plan_token(tl1, p.mode, p.norm_topk, p.snap.resident_mask, lane);
     g0 = tp.g0;
     g1 = tp.g1;
     tp1 = tp;
     run = tp.exec_mask & p.run_mask;
-    rm.n_routed = __popcll(run);
-    rm.n_pairs = rm.n_routed + (p.run_shared ? 1 : 0);
+    const int n_routed = __popcll(run);
+    spec_geometry = spec_on && n_routed == k;
+    int pos_e = -1;
+    if (spec_geometry) {
+      // a confirmed guess keeps its position; the other executed experts fill the gaps in ascending order
+      const bool keep = lane < k && ((run >> spec_e) & 1ull);
+      const unsigned keep_lanes = __ballot_sync(0xffffffffu, keep);
+      const unsigned lo = __reduce_or_sync(0xffffffffu, keep && spec_e < 32 ? (1u << spec_e) : 0u);
+      const unsigned hi = __reduce_or_sync(0xffffffffu, keep && spec_e >= 32 ? (1u << (spec_e - 32)) : 0u);
+      const unsigned long long rest = run & ~(((unsigned long long)hi << 32) | lo);
+      const unsigned gaps = ~keep_lanes & (k >= 32 ? 0xffffffffu : ((1u << k) - 1u));
+      if (lane < k) pos_e = keep ? spec_e : nth_set_bit64(rest, __popc(gaps & ((1u << lane) - 1u)));
+    } else {
+      if (lane < n_routed) pos_e = nth_set_bit64(run, lane);
+      set_geometry(n_routed, n_routed + (p.run_shared ? 1 : 0));
+    }
+    if (lane < APEX_MAX_TOPK) s_pos[warp][lane] = pos_e;
+    __syncwarp();
   } else {
-    rm.n_pairs = p.n_pairs[0];
-    rm.n_routed = rm.n_pairs - (p.run_shared ? B : 0);
+    const int n_pairs = p.n_pairs[0];
+    set_geometry(n_pairs - (p.run_shared ? B : 0), n_pairs);
   }
-  rm.routed_rows = (long long)rm.n_routed * I;
-  rm.total_rows = rm.routed_rows + (long long)(rm.n_pairs - rm.n_routed) * p.I_shared;
   if (tid == 0) TL(2);  // plan done
-
-  // Work split.  Short launches (fewer than two ring fills per CTA): equal contiguous ranges, all
-  // known at launch, no shared counter (a ticket per row costs more than it balances there: every
-  // warp would hit one counter within the same microsecond).  Long launches: every CTA owns NS (the
-  // ring depth) consecutive rows, so all its stages are filled at once, and the remaining rows are
-  // handed out in tickets from a global counter to whichever warp has a free stage first.
-  const long long per_cta = rm.total_rows / G;
-  const bool dynamic = per_cta >= 2 * NS;
-  const long long range_lo = rm.total_rows * cta / G, range_hi = rm.total_rows * (cta + 1) / G;
-  const int S = dynamic ? NS : (int)(range_hi - range_lo);       // rows this CTA knows about at launch
-  const long long static_base = dynamic ? (long long)cta * NS : range_lo;
-  const long long dyn_begin = dynamic ? (long long)G * NS : rm.total_rows;
-  const long long dyn_rows = rm.total_rows - dyn_begin;
-  const int chunk = (int)((dyn_rows + (long long)G * kConsumerWarps * 4 - 1) / ((long long)G * kConsumerWarps * 4)) > 1
-                        ? (int)((dyn_rows + (long long)G * kConsumerWarps * 4 - 1) / ((long long)G * kConsumerWarps * 4))
-                        : 1;                                      // rows per ticket: about four tickets per warp
-  const int n_static = S > warp ? (S - warp + kConsumerWarps - 1) / kConsumerWarps : 0;  // static rows of this warp
 
   float acc[NCH * 8];
 #pragma unroll
@@ -555,15 +647,9 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     int pidx, e, tok;
     long long i;
     float gate = 0.f;
-    if (r < rm.routed_rows) {
-      pidx = (int)(r / I);
-      i = r - (long long)pidx * I;
-    } else {
-      pidx = rm.n_routed + (int)((r - rm.routed_rows) / p.I_shared);
-      i = r - rm.routed_rows - (long long)(pidx - rm.n_routed) * p.I_shared;
-    }
+    locate(r, &pidx, &i);
     if (B == 1) {
-      e = pidx < rm.n_routed ? nth_set_bit64(run, pidx) : N;
+      e = pidx < rm.n_routed ? s_pos[warp][pidx] : N;
       tok = 0;
     } else {
       e = p.pair_expert[pidx];
@@ -672,13 +758,32 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     dyn_end = first + chunk < rm.total_rows ? first + chunk : rm.total_rows;
     return dyn_cur++;
   };
-  // first fill: the static rows go out from NSW lanes in one instruction
+  // first fill: the static rows go out from NSW lanes in one instruction.  A speculative copy that
+  // was confirmed is this lane's first row already; one that was not has to land (nothing cancels
+  // a bulk copy) before its stage is filled again, and from then on that stage's barrier runs one
+  // phase ahead of the row count.
   const int first_fill = n_static < NSW ? n_static : NSW;
-  if (lane < first_fill) {
+  bool dropped = false;
+  if (spec_issued) {
+    bool confirmed = false;
+    if (spec_geometry && lane < first_fill) {
+      int pidx;
+      long long i;
+      locate(static_base + warp + (long long)kConsumerWarps * lane, &pidx, &i);
+      confirmed = s_exp[warp + kConsumerWarps * lane] == (pidx < rm.n_routed ? s_pos[warp][pidx] : N);
+    }
+    if (!confirmed) {
+      dropped = true;
+      spec_issued = false;
+      if (!mbar_wait(&s_full[warp + kConsumerWarps * lane], 0u, nullptr, p.wait_limit_ns)) ok = false;
+    }
+  }
+  const unsigned phase_ahead = __ballot_sync(0xffffffffu, dropped);  // bit n: stage n of this warp
+  if (lane < first_fill && !spec_issued && ok) {
     if (lane == 0 && warp == 0) TL(3);
     issue(static_base + warp + (long long)kConsumerWarps * lane, lane);
-    if (!ok) atomicExch(&s_abort, 1);
   }
+  if (!ok) atomicExch(&s_abort, 1);
   __syncwarp();
   int tail = first_fill;  // rows of this warp whose copy has been started (uniform across the warp)
   next_static = first_fill;
@@ -702,7 +807,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
   for (int head = 0; head < tail; ++head) {
     if (__any_sync(0xffffffffu, *(volatile int*)&s_abort != 0)) break;
     const int s = warp + kConsumerWarps * (head % NSW);
-    if (!__all_sync(0xffffffffu, mbar_wait(&s_full[s], (uint32_t)((head / NSW) & 1), &s_abort, p.wait_limit_ns))) {
+    const uint32_t parity = (uint32_t)((head / NSW + ((phase_ahead >> (head % NSW)) & 1u)) & 1);
+    if (!__all_sync(0xffffffffu, mbar_wait(&s_full[s], parity, &s_abort, p.wait_limit_ns))) {
       atomicExch(&s_abort, 1);
       break;
     }
@@ -817,7 +923,8 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     // flight into the shared memory of an exited CTA
     for (int jj = 0; jj < tail; ++jj) {
       const int s = warp + kConsumerWarps * (jj % NSW);
-      if (jj + NSW >= tail) mbar_wait(&s_full[s], (uint32_t)((jj / NSW) & 1), nullptr, p.wait_limit_ns);
+      if (jj + NSW >= tail)
+        mbar_wait(&s_full[s], (uint32_t)((jj / NSW + ((phase_ahead >> (jj % NSW)) & 1u)) & 1), nullptr, p.wait_limit_ns);
     }
   }
 
@@ -868,6 +975,7 @@ __global__ void __launch_bounds__(kFfnThreads, 1) moe_ffn_stream_kernel(const Ff
     }
   }
   if (tid == 0) TL(9);
+  if (tid == 0) TLG(12);
   SPAN_END(5);
 }
 
@@ -900,7 +1008,7 @@ static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
     configured = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n_sm, 1, 1);
+  cfg.gridDim = dim3(n_sm * kCtasPerSm, 1, 1);
   cfg.blockDim = dim3(kFfnThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
@@ -921,6 +1029,8 @@ bool ffn_shape_supported(int d) {
 }
 
 cudaError_t ffn_configure(int) { return cudaSuccess; }
+
+int ffn_grid_ctas(int n_sm) { return n_sm * kCtasPerSm; }
 
 cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s) {
   if (p.fp8) {  // e4m3 store: the shapes of the paper-sized configs

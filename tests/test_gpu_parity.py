@@ -149,6 +149,45 @@ def test_fp8_store_config1_shape_two_layers(mode):
     print("fp8 config1", mode, rep)
 
 
+# ------------------------------------------------------------------ speculative first fill of the expert FFN
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+@pytest.mark.parametrize("sigma_p", [0.0, 8.0])
+def test_speculative_fill_with_good_and_useless_predictor(sigma_p, mode):
+    # sigma_p = 0: most guesses are confirmed; sigma_p = 8: the prefetch ranking is almost unrelated to the
+    # gate's, so nearly every speculative copy is dropped and its stage refilled
+    cfg = synth.tiny_config(d=1024, N=24, k=6, I=96, C=12, T=10, I_shared=32, sigma_p=sigma_p, cfg_id=280)
+    rep, stats = _run(cfg, mode=mode, tau=0.6, T=10)
+    assert rep.layer_steps == 10 and rep.ffn_checked + rep.near_ties >= 10
+    if sigma_p == 8.0:
+        assert stats["hits_P"] < 0.8 * stats["routed"]
+
+
+def test_speculation_switch_changes_nothing_but_time():
+    cfg = synth.tiny_config(d=1536, N=40, k=8, I=128, C=20, L=3, T=6, sigma_p=0.3, cfg_id=281)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    hs = [synth.hidden_states(cfg, l, cfg.T, 1) for l in range(cfg.L)]
+    h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()
+    hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
+    ys, stats = [], []
+    for flags in (0, binding.FLAG_NO_SPECULATION):
+        apex = prob.make_ctx(flags=flags)
+        try:
+            y = torch.zeros((cfg.T, cfg.L, 1, cfg.d), dtype=torch.float32, device="cuda")
+            for t in range(cfg.T):
+                apex.decode_token(h[t], hp[t], 1, 0.8, "exact", y[t])
+            torch.cuda.synchronize()
+            ys.append(y.cpu().numpy())
+            st = apex.get_stats()
+            stats.append({k: st[k] for k in ("hits_P", "hits_R", "covered", "prefetch_copies", "demand_copies",
+                                             "sum_delta_hat", "sum_delta_star", "substitutions", "timeouts")})
+        finally:
+            apex.destroy()
+    assert stats[0] == stats[1] and stats[0]["timeouts"] == 0
+    # same rows, same arithmetic per row; only the order of the fp32 atomic adds into y may differ
+    np.testing.assert_allclose(ys[0], ys[1], rtol=0, atol=2e-6 * float(np.abs(ys[1]).max()))
+
+
 # ------------------------------------------------------------------ the paper-shaped configs
 def test_config0_full():
     cfg = synth.CONFIGS[0]

@@ -228,7 +228,7 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(dev_alloc(&ctx->d_exec_gate, MB * k));
   CR(dev_alloc(&ctx->d_cand_ncand, MB));
   // batched tensor-core path: scratch and tensor maps (only for contexts that will see large batches)
-  if (MB >= 12 && !fp8 && tc_shape_supported(c.d, c.I, c.I_shared)) {
+  if (MB >= kTcMinBatch && !fp8 && tc_shape_supported(c.d, c.I, c.I_shared)) {
     const size_t rows = max_pairs + 256;
     const size_t i_max = (size_t)(c.I > c.I_shared ? c.I : c.I_shared);
     ctx->act_stride = (int)i_max;
@@ -629,7 +629,6 @@ cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
   return launch_ffn(p, ctx->n_sm, cs);
 }
 
-constexpr int kTcMinBatch = 12;  // from this many tokens per step the tensor-core grouped GEMM runs
 
 // B > 1: plan kernel, then either the tensor-core grouped GEMM or the streaming kernel per pair.
 int launch_batched(apex_ctx* ctx, int layer, const FfnParams& p, cudaStream_t cs) {

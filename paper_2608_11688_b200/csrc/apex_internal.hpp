@@ -150,6 +150,7 @@ struct FfnParams {
 };
 
 // Batched tensor-core path (kernels_ffn_tc.cu)
+constexpr int kTcMinBatch = 4;  // from this many tokens per step the tensor-core grouped GEMM runs (measured crossover)
 struct TcParams {
   FfnParams f;
   const int32_t* grp;

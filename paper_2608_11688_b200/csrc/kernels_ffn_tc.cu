@@ -13,9 +13,16 @@
 //              a = g_pair * silu(G) * U  (fp32) is kept as TWO bf16 planes, a_hi = bf16(a) and
 //              a_lo = bf16(a - a_hi), so feeding it back to the tensor cores loses 2^-17, not 2^-9
 //                                                                            -> global scratch (L2)
-//   down       D [128 cols of d x n] = downT[I x 128]^T . (a_hi + a_lo)^T   (downT is MN-major)
-//              y[token][col] += D                                            fp32 atomics
-//              (at most 128 tokens per unit here; larger groups are split)
+//   down       D [128 cols of d x 2n] = downT[I x 128]^T . [a_hi ; a_lo]^T   (downT is MN-major; both planes
+//              y[token][col] += D[:, j] + D[:, n + j]          fp32 atomics      in one MMA: N = 2n)
+//              (at most 64 tokens per unit here; larger groups are split; the shared expert's longer K is cut
+//              into chunks of I rows so that all units are about equally long)
+//
+// Measured on B200: an MMA with M = 128, K = 16 costs about 35-40 ns to issue whatever N is (it streams a
+// 128 x 16 slice of A), so small-N "swap-AB" MMAs are bound by their count, not by their flops: eight per
+// 64-wide K tile was the pace of both kernels until the two planes of the down projection were merged into
+// one instruction.  Accumulators are double-buffered in TMEM (2 x 256 columns), so the epilogue of one unit
+// overlaps the MMAs of the next.
 //
 // Operands reach shared memory through TMA tensor maps with the 128-byte swizzle and are consumed
 // by tcgen05.mma through shared-memory descriptors (K-major for gate, up, X, A; MN-major for downT).
@@ -35,7 +42,7 @@ constexpr int kProducerWarps = 2;  // TMA producers: K tile t is loaded by warp 
 constexpr int kMmaWarp = kProducerWarps;
 constexpr int kTcThreads = (kProducerWarps + 1 + 4) * 32;  // producers, MMA + TMEM owner, four epilogue warps
 constexpr int kKTile = 64;       // K elements per pipeline stage (128 bytes: one swizzle span)
-constexpr int kXRowsPerLoad = 32;
+constexpr int kXRowsPerLoad = 8;    // rows per B-tile box: one 8-row swizzle atom, so a small group does not fetch rows it has no token for
 
 __device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 __device__ __forceinline__ unsigned long long gtimer() {
@@ -131,6 +138,13 @@ __device__ __forceinline__ uint32_t ld_acquire_sys_u32(const uint32_t* p) {
   return v;
 }
 
+#ifdef APEX_TIMELINE
+__device__ unsigned long long g_tc_tl[2][148][128];
+#define TCTL(ph, i) do { if ((i) < 128) g_tc_tl[(ph) - 1][blockIdx.x][(i)] = gtimer(); } while (0)
+#else
+#define TCTL(ph, i) do { } while (0)
+#endif
+
 struct Group {
   int expert, pair_off, n_tok;
 };
@@ -171,7 +185,8 @@ __global__ void __launch_bounds__(256) ffn_tc_gather_kernel(const TcParams p) {
 
 // ---------------------------------------------------------------- the two GEMM kernels
 // PHASE 1: gate/up.  A tiles: gate and up rows [128 x 64] (K-major), B tile: X_g rows [<=256 x 64].
-// PHASE 2: down.     A tile: downT [64 k-rows x 128 cols] as two 64-column atoms (MN-major), B tile: A rows [<=256 x 64].
+// PHASE 2: down.     A tile: downT [64 k-rows x 128 cols] as two 64-column atoms (MN-major), B tile: the group's rows of
+//                    a_hi, then of a_lo [2 x <=64 x 64].
 template <int PHASE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_ws,
@@ -187,10 +202,11 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   const int B_PLANE = NMAX * 128;
   const int STAGE_BYTES = A_BYTES + PLANES * B_PLANE;
   const int NSTAGE = PHASE == 1 ? p.nstage1 : p.nstage2;
-  __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full, tmem_empty;
+  __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int s_abort;
   __shared__ int s_ustart[APEX_MAX_EXPERTS + 3];  // first unit of each group
+  __shared__ int32_t s_grp[4 + 3 * (APEX_MAX_EXPERTS + 1)];
 
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int N = p.f.N, d = p.f.d, I = p.f.I, I_s = p.f.I_shared;
@@ -202,8 +218,10 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       mbar_init(&full[s], 1);
       mbar_init(&empty[s], 1);
     }
-    mbar_init(&tmem_full, 1);
-    mbar_init(&tmem_empty, 128);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tmem_full[b], 1);
+      mbar_init(&tmem_empty[b], 128);
+    }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_w) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_ws) : "memory");
@@ -219,18 +237,25 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
 
-  const int n_rg = grp[0], n_g = grp[1];
+  // the group table goes to shared memory once: a global load per unit would sit on every role's path
+  for (int i = tid; i < 4 + 3 * (N + 1); i += kTcThreads) s_grp[i] = grp[i];
+  __syncthreads();
+  const int n_rg = s_grp[0], n_g = s_grp[1];
   const int blocks_r = PHASE == 1 ? I / 128 : d / 128;                       // M blocks of a routed group
   const int blocks_s = PHASE == 1 ? (I_s > 0 ? I_s / 128 : 0) : d / 128;     // ... of the shared group
   const int kdim_r = PHASE == 1 ? d : I, kdim_s = PHASE == 1 ? d : I_s;
   // A group of n tokens is cut into ceil(n / NMAX) parts; a unit is (group, M block, part), parts
   // fastest so that the CTAs that share a weight block run at the same time (second reader hits L2).
+  // The shared expert's down projection has a longer K (I_s) than a routed expert's (I): it is cut into
+  // chunks of I rows, each a unit of its own (partial sums meet in y through the atomics), so that all
+  // units of a launch are about equally long and the round-robin assignment stays balanced.
+  const int kchunks_s = (PHASE == 2 && I_s > I) ? (I_s + I - 1) / I : 1;
   if (tid == 0) {
     int acc = 0;
     for (int g = 0; g < n_g; ++g) {
       s_ustart[g] = acc;
-      const int parts = (grp[6 + 3 * g] + NMAX - 1) / NMAX;
-      acc += (g < n_rg ? blocks_r : blocks_s) * parts;
+      const int parts = (s_grp[6 + 3 * g] + NMAX - 1) / NMAX;
+      acc += (g < n_rg ? blocks_r : blocks_s * kchunks_s) * parts;
     }
     s_ustart[n_g] = acc;
   }
@@ -242,15 +267,17 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   int g = 0;
   for (int uu = blockIdx.x; uu < n_units; uu += gridDim.x) {
     while (uu >= s_ustart[g + 1]) ++g;
-    Group gr = load_group(grp, g);
+    Group gr = load_group(s_grp, g);
     const int parts = (gr.n_tok + NMAX - 1) / NMAX;
     const int local = uu - s_ustart[g];
-    const int blk = local / parts, sub = local % parts;
+    const bool shared = gr.expert >= N;
+    const int kch = shared ? kchunks_s : 1;
+    const int blk = local / (parts * kch), kc = (local / parts) % kch, sub = local % parts;
     gr.pair_off += sub * NMAX;
     gr.n_tok = gr.n_tok - sub * NMAX < NMAX ? gr.n_tok - sub * NMAX : NMAX;
-    const bool shared = gr.expert >= N;
     const int kdim = shared ? kdim_s : kdim_r;
-    const int n_kt = kdim / kKTile;
+    const int kt_begin = kch > 1 ? kc * (I / kKTile) : 0;                                    // K tiles of this unit
+    const int kt_end = kch > 1 ? (kt_begin + I / kKTile < kdim / kKTile ? kt_begin + I / kKTile : kdim / kKTile) : kdim / kKTile;
     const int n_pad = (gr.n_tok + 15) & ~15;                                  // MMA N
     const int n_loads = (gr.n_tok + kXRowsPerLoad - 1) / kXRowsPerLoad;       // 32-row boxes of the B tile
 
@@ -284,7 +311,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       }
       const CUtensorMap* wmap = shared ? &tm_ws : &tm_w;
       constexpr int planes = PLANES;
-      for (int kt = 0; kt < n_kt && ok; ++kt, ++it_load) {
+      for (int kt = kt_begin; kt < kt_end && ok; ++kt, ++it_load) {
         if ((int)(it_load % kProducerWarps) != warp) continue;  // the other producer warp's tile
         const int s = it_load % NSTAGE;
         if (lane == 0) {
@@ -301,8 +328,9 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
             if (PHASE == 1) tma_load_4d(st + op * 128 * 128, wmap, kt * kKTile, op, blk * 128, slot, &full[s]);   // gate | up rows
             else tma_load_4d(st + op * 64 * 128, wmap, blk * 128 + op * 64, 2, kt * kKTile, slot, &full[s]);      // downT, 64 columns
           } else {
+            // B rows of this stage: the tokens' rows of plane 0, padded to n_pad, then those of plane 1
             const int r = (op - 2) / planes, pl = (op - 2) % planes;
-            tma_load_2d(st + A_BYTES + pl * B_PLANE + r * kXRowsPerLoad * 128, pl ? &tm_b2 : &tm_b, kt * kKTile,
+            tma_load_2d(st + A_BYTES + pl * n_pad * 128 + r * kXRowsPerLoad * 128, pl ? &tm_b2 : &tm_b, kt * kKTile,
                         gr.pair_off + r * kXRowsPerLoad, &full[s]);
           }
         }
@@ -317,49 +345,58 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       // ================= MMA issuer
       if (lane == 0) {
         bool ok = true;
-        if (unit_no > 0) ok = mbar_wait(&tmem_empty, (unit_no - 1) & 1, &s_abort, p.f.wait_limit_ns);
+        // two accumulator buffers of 256 TMEM columns: this unit's MMAs run while the epilogue warps
+        // still read the previous unit's
+        const uint32_t buf = unit_no & 1u;
+        if (unit_no >= 2) ok = mbar_wait(&tmem_empty[buf], ((unit_no >> 1) - 1) & 1, &s_abort, p.f.wait_limit_ns);
         tc_fence_after();
-        const uint32_t idesc = umma_idesc(128, n_pad, PHASE == 2 ? 1 : 0);
-        for (int kt = 0; kt < n_kt && ok; ++kt, ++it_mma) {
+        TCTL(PHASE, unit_no * 16);
+        const uint32_t tacc = tmem_base + buf * 256u;
+        // An MMA costs about 128 cycles whatever N is (it streams a 128 x 16 slice of A), so the down
+        // projection multiplies both planes of the intermediate in one instruction: N = 2 * n_pad.
+        const uint32_t idesc = umma_idesc(128, PHASE == 2 ? 2 * n_pad : n_pad, PHASE == 2 ? 1 : 0);
+        for (int kt = kt_begin; kt < kt_end && ok; ++kt, ++it_mma) {
           const int s = it_mma % NSTAGE;
           if (!mbar_wait(&full[s], (it_mma / NSTAGE) & 1, &s_abort, p.f.wait_limit_ns)) {
             ok = false;
             break;
           }
+          if (kt - kt_begin < 10) TCTL(PHASE, unit_no * 16 + 1 + kt - kt_begin);
           tc_fence_after();
           const uint32_t a0 = s32(smem + (size_t)s * STAGE_BYTES);
           const uint32_t b0 = a0 + A_BYTES;
 #pragma unroll
           for (int ks = 0; ks < kKTile / 16; ++ks) {
-            const uint32_t acc = (kt > 0 || ks > 0) ? 1u : 0u;
+            const uint32_t acc = (kt > kt_begin || ks > 0) ? 1u : 0u;
             const uint64_t bdesc = umma_desc(b0 + ks * 32, 16, 1024);
             if (PHASE == 1) {
-              umma(tmem_base, umma_desc(a0 + ks * 32, 16, 1024), bdesc, idesc, acc);                     // G
-              umma(tmem_base + 256, umma_desc(a0 + 128 * 128 + ks * 32, 16, 1024), bdesc, idesc, acc);   // U
+              umma(tacc, umma_desc(a0 + ks * 32, 16, 1024), bdesc, idesc, acc);                     // G
+              umma(tacc + 128, umma_desc(a0 + 128 * 128 + ks * 32, 16, 1024), bdesc, idesc, acc);   // U
             } else {
-              const uint64_t adesc = umma_desc(a0 + ks * 2048, 64 * 128, 1024);
-              umma(tmem_base, adesc, bdesc, idesc, acc);                                           // a_hi
-              umma(tmem_base, adesc, umma_desc(b0 + B_PLANE + ks * 32, 16, 1024), idesc, 1u);     // a_lo
+              umma(tacc, umma_desc(a0 + ks * 2048, 64 * 128, 1024), bdesc, idesc, acc);  // columns [0, n_pad): a_hi, [n_pad, 2 n_pad): a_lo
             }
           }
           umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
         }
-        if (ok) umma_commit(&tmem_full);
+        TCTL(PHASE, unit_no * 16 + 11);
+        if (ok) umma_commit(&tmem_full[buf]);
         else atomicExch(&s_abort, 1);
       }
     } else {
       // ================= epilogue: warp w owns TMEM lanes 32*(w%4) .. +31
       const int quad = warp & 3;
       const int row = quad * 32 + lane;  // row of the 128-row tile
-      if (__all_sync(0xffffffffu, mbar_wait(&tmem_full, unit_no & 1, &s_abort, p.f.wait_limit_ns))) {
+      const uint32_t buf = unit_no & 1u;
+      if (__all_sync(0xffffffffu, mbar_wait(&tmem_full[buf], (unit_no >> 1) & 1, &s_abort, p.f.wait_limit_ns))) {
         tc_fence_after();
+        if (warp == kMmaWarp + 1 && lane == 0) TCTL(PHASE, unit_no * 16 + 12);
         for (int c0 = 0; c0 < gr.n_tok; c0 += 32) {
           uint32_t a[32];
-          const uint32_t taddr = tmem_base + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0;
+          const uint32_t taddr = tmem_base + buf * 256u + ((uint32_t)(quad * 32) << 16) + (uint32_t)c0;
           tmem_ld32(taddr, a);
+          uint32_t b2[32];
+          tmem_ld32(taddr + (PHASE == 1 ? 128 : n_pad), b2);   // U | the a_lo half of the down product
           if (PHASE == 1) {
-            uint32_t b2[32];
-            tmem_ld32(taddr + 256, b2);
             asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             const int i = blk * 128 + row;
 #pragma unroll
@@ -381,14 +418,15 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
             for (int j = 0; j < 32; ++j) {
               if (c0 + j < gr.n_tok) {
                 const int t = __ldg(p.f.pair_tok + gr.pair_off + c0 + j);
-                atomicAdd(p.f.y + (size_t)t * d + col, __uint_as_float(a[j]));
+                atomicAdd(p.f.y + (size_t)t * d + col, __uint_as_float(a[j]) + __uint_as_float(b2[j]));
               }
             }
           }
         }
       }
       tc_fence_before();
-      mbar_arrive(&tmem_empty);
+      if (warp == kMmaWarp + 1 && lane == 0) TCTL(PHASE, unit_no * 16 + 13);
+      mbar_arrive(&tmem_empty[unit_no & 1u]);
     }
     ++unit_no;
     if (*(volatile int*)&s_abort) break;
@@ -397,6 +435,12 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   __syncthreads();
   if (warp == kMmaWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
 }
+
+#ifdef APEX_TIMELINE
+extern "C" int apex_debug_read_tc_timeline(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_tc_tl, sizeof(g_tc_tl));
+}
+#endif
 
 // ---------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*, const cuuint64_t*,

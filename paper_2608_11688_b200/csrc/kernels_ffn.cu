@@ -260,6 +260,11 @@ __device__ __forceinline__ void store_token_plan(const TokenPlan& tp, int lane, 
   }
 }
 
+__device__ __forceinline__ int nth_set_bit64(unsigned long long m, int n) {
+  for (int i = 0; i < n; ++i) m &= m - 1;
+  return __ffsll((long long)m) - 1;
+}
+
 // ---------------------------------------------------------------- batched plan (B > 1)
 // One CTA of 32 warps.  Phase A: warp w plans tokens w, w+32, ... (all global loads of a warp's tokens
 // are issued before the first use).  Phase B: warp w owns experts w and w+32 and gathers the tokens
@@ -267,13 +272,21 @@ __device__ __forceinline__ void store_token_plan(const TokenPlan& tp, int lane, 
 // (expert id N) follow.
 constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;
 
+#ifdef APEX_TIMELINE
+#define PTL(i) do { if (threadIdx.x == 0) g_timeline[1000 * 16 + (i)] = globaltimer_ns_raw(); } while (0)
+#else
+#define PTL(i) do { } while (0)
+#endif
+
 __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   __shared__ unsigned long long s_exec[APEX_MAX_BATCH];
+  __shared__ float s_pgate[APEX_MAX_BATCH][APEX_MAX_TOPK];  // gate of the j-th executed expert of each token
   __shared__ int s_count[APEX_MAX_EXPERTS + 1];
   __shared__ int s_off[APEX_MAX_EXPERTS + 2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
   const int N = p.N, k = p.k, B = p.B;
   int my_subst = 0, my_hits = 0;
+  PTL(0);
   TokenLoads tls[kPlanMaxTokPerWarp];
 #pragma unroll
   for (int j = 0; j < kPlanMaxTokPerWarp; ++j) {
@@ -286,10 +299,8 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     if (b >= B) break;
     const TokenLoads& tl = tls[j];
     const TokenPlan tp = plan_token(tl, p.mode, p.norm_topk, p.snap.resident_mask, lane);
-    store_token_plan(tp, lane, k, p.plan_exec_idx + (size_t)b * k, p.plan_exec_gate + (size_t)b * k,
-                     p.post_exec ? p.mbox_exec + (size_t)b * k : nullptr);
+    store_token_plan(tp, lane, k, p.plan_exec_idx + (size_t)b * k, p.plan_exec_gate + (size_t)b * k, nullptr);
     if (p.post_exec) {
-      if (lane < k) p.mbox_kr[(size_t)b * k + lane] = tl.my_idx;
       const int e0 = lane, e1 = lane + 32;
       if ((tp.exec_mask >> e0) & 1) {
         const int pos = __popcll(tp.exec_mask & ((1ull << e0) - 1ull));
@@ -305,10 +316,33 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
       my_hits += __popcll(tp.kr_mask & p.snap.resident_mask);
     }
     if (lane == 0) s_exec[b] = tp.exec_mask;
+    {
+      const int e0 = lane, e1 = lane + 32;
+      if ((tp.exec_mask >> e0) & 1) {
+        const int pos = __popcll(tp.exec_mask & ((1ull << e0) - 1ull));
+        if (pos < APEX_MAX_TOPK) s_pgate[b][pos] = tp.g0;
+      }
+      if ((tp.exec_mask >> e1) & 1) {
+        const int pos = __popcll(tp.exec_mask & ((1ull << e1) - 1ull));
+        if (pos < APEX_MAX_TOPK) s_pgate[b][pos] = tp.g1;
+      }
+    }
   }
   if (p.post_exec && lane == 0 && my_subst && p.stats) atomicAdd(&p.stats->substitutions, (unsigned long long)my_subst);
   if (p.post_exec && lane == 0 && my_hits && p.stats) atomicAdd(&p.stats->hits_R, (unsigned long long)my_hits);
   __syncthreads();
+  PTL(1);
+  // The routed and the execution sets go to the host mailbox here, as whole lines from consecutive
+  // threads (a 4-byte store per lane and token from inside the loop above cost 2 us per token), and
+  // early, so that the trip over the host link overlaps the sorting below.
+  if (p.post_exec) {
+    for (int t = threadIdx.x; t < B * k; t += blockDim.x) {
+      const int b = t / k, j = t - b * k;
+      const unsigned long long m = s_exec[b];
+      p.mbox_exec[t] = j < __popcll(m) ? nth_set_bit64(m, j) : -1;
+      p.mbox_kr[t] = p.idx[t];
+    }
+  }
   // ---- phase B, counts: warp w counts the tokens of experts w and w + 32
   for (int e = warp; e < N; e += nwarp) {
     int c = 0;
@@ -320,34 +354,52 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     if (lane == 0) s_count[e] = c;
   }
   __syncthreads();
-  if (threadIdx.x == 0) {
-    int acc = 0;
-    for (int f = 0; f < N; ++f) {
-      s_off[f] = acc;
-      acc += s_count[f];
-    }
-    s_off[N] = acc;  // routed pairs
-    const int n_pairs = acc + (p.run_shared ? B : 0);
-    p.n_pairs[0] = n_pairs;
-    // groups for the tensor-core path: one per executed expert, then the shared expert
-    int ng = 0;
-    for (int f = 0; f < N; ++f)
-      if (s_count[f] > 0) {
-        p.grp[4 + 3 * ng] = f;
-        p.grp[5 + 3 * ng] = s_off[f];
-        p.grp[6 + 3 * ng] = s_count[f];
-        ++ng;
+  PTL(2);
+  if (warp == 0) {
+    // exclusive prefix over the experts (lane owns experts lane and lane + 32), then the group table
+    // of the tensor-core path: one group per executed expert, then the shared expert
+    const int c0 = lane < N ? s_count[lane] : 0, c1 = lane + 32 < N ? s_count[lane + 32] : 0;
+    int i0 = c0, i1 = c1;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+      const int u0 = __shfl_up_sync(0xffffffffu, i0, o), u1 = __shfl_up_sync(0xffffffffu, i1, o);
+      if (lane >= o) {
+        i0 += u0;
+        i1 += u1;
       }
-    p.grp[0] = ng;
-    if (p.run_shared) {
-      p.grp[4 + 3 * ng] = N;
-      p.grp[5 + 3 * ng] = acc;
-      p.grp[6 + 3 * ng] = B;
-      ++ng;
     }
-    p.grp[1] = ng;
+    const int tot0 = __shfl_sync(0xffffffffu, i0, 31), acc = tot0 + __shfl_sync(0xffffffffu, i1, 31);
+    const int off0 = i0 - c0, off1 = tot0 + i1 - c1;
+    if (lane < N) s_off[lane] = off0;
+    if (lane + 32 < N) s_off[lane + 32] = off1;
+    const unsigned g0m = __ballot_sync(0xffffffffu, c0 > 0), g1m = __ballot_sync(0xffffffffu, c1 > 0);
+    const int ng_routed = __popc(g0m) + __popc(g1m);
+    if (c0 > 0) {
+      const int gi = __popc(g0m & ((1u << lane) - 1u));
+      p.grp[4 + 3 * gi] = lane;
+      p.grp[5 + 3 * gi] = off0;
+      p.grp[6 + 3 * gi] = c0;
+    }
+    if (c1 > 0) {
+      const int gi = __popc(g0m) + __popc(g1m & ((1u << lane) - 1u));
+      p.grp[4 + 3 * gi] = lane + 32;
+      p.grp[5 + 3 * gi] = off1;
+      p.grp[6 + 3 * gi] = c1;
+    }
+    if (lane == 0) {
+      s_off[N] = acc;  // routed pairs
+      p.n_pairs[0] = acc + (p.run_shared ? B : 0);
+      p.grp[0] = ng_routed;
+      if (p.run_shared) {
+        p.grp[4 + 3 * ng_routed] = N;
+        p.grp[5 + 3 * ng_routed] = acc;
+        p.grp[6 + 3 * ng_routed] = B;
+      }
+      p.grp[1] = ng_routed + (p.run_shared ? 1 : 0);
+    }
   }
   __syncthreads();
+  PTL(3);
   // ---- phase B, placement: token b of expert e goes to s_off[e] + (number of earlier tokens of e)
   for (int e = warp; e < N; e += nwarp) {
     if (s_count[e] == 0) continue;
@@ -361,7 +413,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
         const int pos = __popcll(s_exec[b] & ((1ull << e) - 1ull));
         p.pair_tok[at] = b;
         p.pair_expert[at] = e;
-        p.pair_gate[at] = p.plan_exec_gate[(size_t)b * k + pos];
+        p.pair_gate[at] = s_pgate[b][pos];
       }
       o += __popc(m);
     }
@@ -374,14 +426,18 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
       p.pair_gate[base + b] = 1.f;
     }
   }
+  PTL(4);
   if (p.post_exec) {
-    __threadfence_system();
+    // the barrier orders every thread's mailbox stores before thread 0's system-scope fence
+    // (fences are cumulative), which orders them before the sequence number
     __syncthreads();
+    PTL(5);
     if (threadIdx.x == 0) {
       __threadfence_system();
       *p.mbox_seq = p.seq_value;
     }
   }
+  PTL(6);
 }
 
 cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s) {
@@ -398,11 +454,6 @@ struct RowMap {
   long long routed_rows; // n_routed * I
   long long total_rows;
 };
-
-__device__ __forceinline__ int nth_set_bit64(unsigned long long m, int n) {
-  for (int i = 0; i < n; ++i) m &= m - 1;
-  return __ffsll((long long)m) - 1;
-}
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

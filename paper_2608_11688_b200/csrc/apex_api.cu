@@ -100,6 +100,7 @@ int issue_copy(apex_ctx* ctx, int layer, int e, int slot, cudaStream_t cs) {
     ctx->inject = 0;
     ctx->withheld_flag = flag;
     ctx->withheld_gen = gen;
+    ctx->withheld_stream = cs;
   } else {
     int r = stream_write32(ctx, cs, flag, gen);
     if (r != APEX_OK) return r;
@@ -113,7 +114,7 @@ int release_withheld(apex_ctx* ctx) {
   if (!ctx->withheld_flag) return APEX_OK;
   uint32_t* srcv = ctx->gen_src + (ctx->gen_src_pos++ % ctx->gen_src_len);
   *srcv = ctx->withheld_gen;
-  CU_TRY(ctx, cudaMemcpyAsync(ctx->withheld_flag, srcv, sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->cur_copy_stream));
+  CU_TRY(ctx, cudaMemcpyAsync(ctx->withheld_flag, srcv, sizeof(uint32_t), cudaMemcpyHostToDevice, ctx->withheld_stream));
   ctx->withheld_flag = nullptr;
   return APEX_OK;
 }
@@ -268,10 +269,10 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   ctx->gen_src_len = 1 << 16;
   CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->gen_src), ctx->gen_src_len * sizeof(uint32_t), cudaHostAllocPortable));
 
-  CR(cudaStreamCreateWithFlags(&ctx->copy_stream, cudaStreamNonBlocking));
-  CR(cudaStreamCreateWithFlags(&ctx->copy_stream_b, cudaStreamNonBlocking));
-  ctx->cur_copy_stream = ctx->copy_stream;
-  ctx->cur_copy_stream_b = ctx->copy_stream_b;
+  for (int i = 0; i < ctx->n_copy_streams; ++i) {
+    CR(cudaStreamCreateWithFlags(&ctx->copy_streams[i], cudaStreamNonBlocking));
+    ctx->cur_copy_streams[i] = ctx->copy_streams[i];
+  }
   CR(cudaEventCreateWithFlags(&ctx->ev_wave, cudaEventDisableTiming));
   CR(cudaEventCreateWithFlags(&ctx->ev_in, cudaEventDisableTiming));
 #undef CR
@@ -311,8 +312,8 @@ int apex_destroy(apex_ctx* ctx) {
     if (p) cudaFree(p);
   if (ctx->mbox) cudaFreeHost(ctx->mbox);
   if (ctx->gen_src) cudaFreeHost(ctx->gen_src);
-  if (ctx->copy_stream) cudaStreamDestroy(ctx->copy_stream);
-  if (ctx->copy_stream_b) cudaStreamDestroy(ctx->copy_stream_b);
+  for (cudaStream_t cs : ctx->copy_streams)
+    if (cs) cudaStreamDestroy(cs);
   if (ctx->ev_wave) cudaEventDestroy(ctx->ev_wave);
   if (ctx->ev_in) cudaEventDestroy(ctx->ev_in);
   delete ctx;
@@ -512,8 +513,8 @@ int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream) {
   auto& st = ctx->step[layer];
   if (!st.selected || st.B != B) return fail(ctx, APEX_ESTATE, "apex_prefetch needs apex_select_candidates of the same layer-step and B");
   if (st.prefetched) return fail(ctx, APEX_ESTATE, "apex_prefetch called twice in one layer-step");
-  ctx->cur_copy_stream = copy_stream ? (cudaStream_t)copy_stream : ctx->copy_stream;
-  ctx->cur_copy_stream_b = copy_stream ? (cudaStream_t)copy_stream : ctx->copy_stream_b;
+  for (int i = 0; i < ctx->n_copy_streams; ++i)
+    ctx->cur_copy_streams[i] = copy_stream ? (cudaStream_t)copy_stream : ctx->copy_streams[i];
   const int C = ctx->cfg.C;
   const int32_t* ncand = mbox_i32(ctx, ctx->ml.off_ncand);
   const int32_t* cand = mbox_i32(ctx, ctx->ml.off_cand);
@@ -777,8 +778,9 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
           }
         if (hazard) {
           CU_TRY(ctx, cudaEventRecord(ctx->ev_wave, cs));
-          CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_stream, ctx->ev_wave, 0));
-          if (ctx->cur_copy_stream_b != ctx->cur_copy_stream) CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_stream_b, ctx->ev_wave, 0));
+          for (int i = 0; i < ctx->n_copy_streams; ++i)
+            if (i == 0 || ctx->cur_copy_streams[i] != ctx->cur_copy_streams[0])
+              CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_streams[i], ctx->ev_wave, 0));
         }
         for (const auto& c : copies)
           if (c.wave == w) {
@@ -1004,8 +1006,7 @@ int apex_warm_all(apex_ctx* ctx) {
     int r = apex_set_slot_table(ctx, l, es.data(), stamp.data(), ctx->tables[l].clock());
     if (r != APEX_OK) return r;
   }
-  CU_TRY(ctx, cudaStreamSynchronize(ctx->cur_copy_stream));
-  CU_TRY(ctx, cudaStreamSynchronize(ctx->cur_copy_stream_b));
+  for (int i = 0; i < ctx->n_copy_streams; ++i) CU_TRY(ctx, cudaStreamSynchronize(ctx->cur_copy_streams[i]));
   return APEX_OK;
 }
 

@@ -260,6 +260,7 @@ struct apex_ctx {
   std::vector<std::vector<int32_t>> phys_expert;  // [L][C] whose bytes the slot holds (or is receiving)
   uint32_t* withheld_flag = nullptr;  // test hook: a ready flag that was not written
   uint32_t withheld_gen = 0;
+  cudaStream_t withheld_stream = nullptr;
   std::vector<std::vector<apex::SlotCopy>> last_copies;
   std::vector<apex_step_stats> host_stats;
   struct StepState {
@@ -277,11 +278,14 @@ struct apex_ctx {
   std::vector<StepState> step;
   std::vector<apex::FfnParams> ffn_params;  // [L] parameters of the last FFN launch of each layer
 
-  // Copies of a slot always travel on the same stream (slot index modulo 2), so two installs into
-  // one slot stay ordered; two streams hide the gap between consecutive copies (+6 % on the link).
-  cudaStream_t copy_stream = nullptr, copy_stream_b = nullptr;  // own
-  cudaStream_t cur_copy_stream = nullptr, cur_copy_stream_b = nullptr;
-  cudaStream_t stream_of_slot(int slot) const { return (slot & 1) ? cur_copy_stream_b : cur_copy_stream; }
+  // Copies of a slot always travel on the same stream (slot index modulo the stream count), so two
+  // installs into one slot stay ordered; two streams hide the gap between consecutive copies (+6 % on
+  // the host link; a third and a fourth add nothing: measured).
+  static constexpr int kMaxCopyStreams = 4;
+  int n_copy_streams = 2;
+  cudaStream_t copy_streams[kMaxCopyStreams] = {};      // own
+  cudaStream_t cur_copy_streams[kMaxCopyStreams] = {};  // in use: own, or the caller's (then all the same)
+  cudaStream_t stream_of_slot(int slot) const { return cur_copy_streams[slot % n_copy_streams]; }
   cudaStream_t pred_stream = nullptr;   // stream of the last apex_predict
   cudaEvent_t ev_wave = nullptr, ev_in = nullptr;
   int inject = 0;

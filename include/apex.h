@@ -234,6 +234,23 @@ int64_t apex_launch_count(const apex_ctx* ctx);
 int apex_route_topk_static(const float* W_r_dev, const float* b_r_dev, const float* hpost_dev, int N, int d, int k,
                            int B, int32_t* idx_dev, float* alpha_dev, void* stream, char* err, size_t err_len);
 
+/* ---- fitting the confidence model on the GPU (Sec. IV-C, Eq. (8) and Eq. (11)) ---------------
+ * Fits p_delta(x) = sigmoid(theta_delta - w.x) to a calibration set by minimising the cumulative binary
+ * cross-entropy  -(1/T) sum_t sum_delta [ y log p + (1-y) log(1-p) ],  y = [delta >= delta*_t],
+ * with theta kept non-decreasing (theta_delta = t0 + sum_{i<=delta} softplus(u_i)).  Full-batch Adam
+ * (0.9 / 0.999 / 1e-8) in fp64, `iters` steps of size lr, from w = 0 and the logit of the empirical
+ * distribution of delta* (clipped to [1e-3, 1-1e-3], increments at least 1e-3); all sums run in a fixed
+ * order, so the result is reproducible bit for bit.
+ *   X_dev [T][N] fp64 (device): x of each calibration token (its prefetch probabilities sorted in
+ *   descending order); dstar_dev [T] int32 (device): its oracle budget delta* (Eq. (3)), 0 <= delta* <= N-k.
+ *   w_host [N], theta_host [N-k+1] (host, fp32): the fitted parameters, theta made monotone again after
+ *   the rounding to fp32 -- ready for apex_set_cdf.
+ * Context-free; allocates and frees its own scratch; synchronises `stream` before it returns.
+ * N <= APEX_MAX_EXPERTS.  err (optional) receives a text on failure.  Returns APEX_OK, APEX_EINVAL,
+ * APEX_ENOMEM or APEX_ECUDA. */
+int apex_fit_cdf(const double* X_dev, const int32_t* dstar_dev, int T, int N, int k, int iters, double lr,
+                 float* w_host, float* theta_host, void* stream, char* err, size_t err_len);
+
 /* ---- host-only slot planner (the state machine behind apex_prefetch / apex_moe_ffn) -------- */
 
 typedef struct apex_slots apex_slots;

@@ -74,6 +74,7 @@ SIGNATURES = {
     "apex_test_inject": (_I, [_P, _I]),
     "apex_launch_count": (C.c_int64, [_P]),
     "apex_route_topk_static": (_I, [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, C.c_char_p, C.c_size_t]),
+    "apex_fit_cdf": (_I, [_P, _P, _I, _I, _I, _I, C.c_double, _P, _P, _P, C.c_char_p, C.c_size_t]),
     "apex_slots_create": (_P, [_I, _I, _I]),
     "apex_slots_destroy": (None, [_P]),
     "apex_slots_begin_step": (_I, [_P]),
@@ -292,6 +293,20 @@ def route_topk_static(W_r_dev, b_r_dev, hpost_dev, k, idx_dev, alpha_dev, stream
                                     _ptr(alpha_dev), _stream(stream), err, len(err))
     if rc != APEX_OK:
         raise ApexError(rc, err.value.decode())
+
+
+def fit_cdf(X_dev, dstar_dev, k, iters=600, lr=0.05, stream=None):
+    """apex_fit_cdf: X_dev [T][N] fp64 and dstar_dev [T] int32 CUDA tensors -> (w [N], theta [N-k+1]) fp32 numpy."""
+    lib = load_library()
+    T, N = X_dev.shape
+    w = np.empty(N, np.float32)
+    theta = np.empty(N - k + 1, np.float32)
+    err = C.create_string_buffer(256)
+    rc = lib.apex_fit_cdf(_ptr(X_dev), _ptr(dstar_dev), T, N, k, int(iters), float(lr), _ptr(w), _ptr(theta),
+                          _stream(stream), err, len(err))
+    if rc != APEX_OK:
+        raise ApexError(rc, err.value.decode())
+    return w, theta
 
 
 class Slots:

@@ -393,3 +393,72 @@ def test_generator_rounds_hidden_states_to_bf16_values():
         assert torch.equal(t, t.to(torch.bfloat16).to(torch.float32))
     x = np.array([1.0 + 2 ** -8, 1.0 + 3 * 2 ** -8], dtype=np.float32)    # exact ties: round to even
     np.testing.assert_array_equal(synth.round_to_bf16_values(x), torch.from_numpy(x).to(torch.bfloat16).float().numpy())
+
+
+# ------------------------------------------------------------------ the CPU fit of the confidence model (Eq. (8), (11))
+def _cumulative_bce(X, dstar, w, theta):
+    """Eq. (11) written out with plain loops: mean over tokens of the sum over thresholds of the binary
+    cross-entropy between [delta >= delta*] and sigmoid(theta_delta - w.x)."""
+    total = 0.0
+    for t in range(X.shape[0]):
+        s = float(np.dot(w, X[t]))
+        for dl in range(len(theta)):
+            z = theta[dl] - s
+            y = 1.0 if dl >= dstar[t] else 0.0
+            # -[y log p + (1 - y) log(1 - p)] with p = sigmoid(z), in the form that survives p = 1 in fp64
+            total += float(np.logaddexp(0.0, z)) - y * z
+    return total / X.shape[0]
+
+
+def _planted_ordinal_data(T, N, k, seed):
+    """Tokens whose delta* is drawn from a known ordinal-logistic model: P(delta* <= delta | x) = sigmoid(theta*_delta - w*.x)."""
+    rng = np.random.default_rng(seed)
+    X = np.sort(rng.dirichlet(np.full(N, 0.6), size=T), axis=1)[:, ::-1].copy()
+    w_true = np.zeros(N)
+    w_true[:k] = -3.0
+    w_true[k:2 * k] = 5.0
+    nth = N - k + 1
+    theta_true = -1.5 + 0.7 * np.arange(nth)
+    theta_true[-1] = 40.0                                   # delta* <= N-k always
+    cdf = 1.0 / (1.0 + np.exp(-(theta_true[None, :] - (X @ w_true)[:, None])))
+    u = rng.random(T)
+    dstar = (u[:, None] > cdf).sum(1)                        # smallest delta with cdf >= u
+    return X, dstar.astype(np.int64), w_true, theta_true
+
+
+def test_cdf_fit_lowers_the_loss_of_eq11_and_recovers_a_planted_model():
+    from oracle import fit_cdf
+    N, k = 10, 2
+    X, dstar, w_true, theta_true = _planted_ordinal_data(6000, N, k, seed=5)
+    w0 = np.zeros(N)
+    cdf0 = np.clip((np.arange(N - k + 1)[None, :] >= dstar[:, None]).mean(0), 1e-3, 1 - 1e-3)
+    th0 = np.log(cdf0 / (1 - cdf0))
+    w, theta = fit_cdf.fit(X, dstar, N, k, iters=600)
+    assert np.all(np.diff(theta) >= 0)
+    sub = slice(0, 1500)                                     # the plain-loop loss on a subset (seconds)
+    l_init = _cumulative_bce(X[sub], dstar[sub], w0, th0)
+    l_fit = _cumulative_bce(X[sub], dstar[sub], w.astype(np.float64), theta.astype(np.float64))
+    l_true = _cumulative_bce(X[sub], dstar[sub], w_true, theta_true)
+    assert l_fit < l_init - 0.03 * abs(l_init), (l_init, l_fit, l_true)   # the x-dependence is learnt: better than the marginal CDF
+    assert l_fit < l_true + 0.02 * abs(l_true), (l_init, l_fit, l_true)   # and about as good as the model that generated the data
+    # the fitted conditional CDF is close to the planted one on fresh tokens
+    Xt, _, _, _ = _planted_ordinal_data(2000, N, k, seed=6)
+    p_fit = 1.0 / (1.0 + np.exp(-(theta[None, :-1].astype(np.float64) - (Xt @ w.astype(np.float64))[:, None])))
+    p_true = 1.0 / (1.0 + np.exp(-(theta_true[None, :-1] - (Xt @ w_true)[:, None])))
+    assert np.abs(p_fit - p_true).mean() < 0.03
+    # a dropped or sign-flipped gradient term would leave w at zero or drive it the wrong way
+    assert np.corrcoef(w[:2 * k], w_true[:2 * k])[0, 1] > 0.9
+
+
+def test_cdf_fit_without_signal_returns_the_empirical_distribution():
+    # x carries no information (all tokens share one x): the optimum of Eq. (11) is the empirical CDF of delta*,
+    # theta_delta - w.x = logit(fraction of tokens with delta* <= delta)
+    from oracle import fit_cdf
+    N, k, T = 8, 3, 3000
+    rng = np.random.default_rng(9)
+    X = np.tile(np.sort(rng.dirichlet(np.ones(N)))[::-1], (T, 1))
+    dstar = rng.integers(0, N - k + 1, size=T)
+    w, theta = fit_cdf.fit(X, dstar, N, k, iters=600)
+    frac = (np.arange(N - k + 1)[None, :] >= dstar[:, None]).mean(0)
+    z = theta.astype(np.float64) - float(X[0] @ w.astype(np.float64))
+    np.testing.assert_allclose(1.0 / (1.0 + np.exp(-z[:-1])), frac[:-1], atol=2e-3)

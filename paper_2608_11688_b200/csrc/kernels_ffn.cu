@@ -1079,8 +1079,6 @@ bool ffn_shape_supported(int d) {
   return false;
 }
 
-cudaError_t ffn_configure(int) { return cudaSuccess; }
-
 int ffn_grid_ctas(int n_sm) { return n_sm * kCtasPerSm; }
 
 cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s) {

@@ -104,20 +104,25 @@ def algorithmic_bytes(cfg, B=1):
 
 
 # ------------------------------------------------------------------------------------------------
-def build_problem(cfg, device, fp8=False):
+def build_problem(cfg, device, fp8=False, fp4=False):
     import torch
     from paper_2608_11688_b200 import synth
     routers = [synth.router_weights(cfg, l) for l in range(cfg.L)]
     cdf = [synth.cdf_params(cfg, l) for l in range(cfg.L)]
-    if fp8:     # datatype study (Sec. V-G): e4m3 rows with per-row scales
+    if fp4:     # datatype study (Sec. V-G): e2m1 rows with a power-of-two scale per 32 elements
+        store = torch.empty((cfg.L, cfg.N, cfg.I, synth.fp4_row_bytes(cfg.d)), dtype=torch.uint8, pin_memory=True)
+    elif fp8:   # e4m3 rows with per-row scales
         store = torch.empty((cfg.L, cfg.N, cfg.I, 3 * cfg.d + 16), dtype=torch.uint8, pin_memory=True)
     else:
         store = torch.empty((cfg.L, cfg.N, cfg.I, 3, cfg.d), dtype=torch.bfloat16, pin_memory=True)
     shared = []
     for l in range(cfg.L):
-        store[l].copy_(synth.expert_store_fp8(cfg, l, device=device) if fp8 else synth.expert_store(cfg, l, device=device))
+        store[l].copy_(synth.expert_store_fp4(cfg, l, device=device) if fp4 else
+                       synth.expert_store_fp8(cfg, l, device=device) if fp8 else synth.expert_store(cfg, l, device=device))
         sh = synth.shared_expert(cfg, l, device=device)
-        shared.append(synth.quantize_store_fp8(sh) if (fp8 and sh is not None) else sh)
+        if sh is not None and (fp4 or fp8):
+            sh = synth.quantize_store_fp4(sh) if fp4 else synth.quantize_store_fp8(sh)
+        shared.append(sh)
     torch.cuda.synchronize()
     return routers, cdf, store, shared
 
@@ -125,9 +130,11 @@ def build_problem(cfg, device, fp8=False):
 def make_ctx(cfg, prob, C, max_batch=1, flags=0):
     from paper_2608_11688_b200 import binding
     routers, cdf, store, shared = prob
-    fp8 = store.dtype != __import__("torch").bfloat16
+    fmt_flag = 0
+    if store.dtype != __import__("torch").bfloat16:
+        fmt_flag = binding.FLAG_FP8_EXPERTS if store.shape[-1] == 3 * cfg.d + 16 else binding.FLAG_FP4_EXPERTS
     a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C, L=cfg.L, I_shared=cfg.I_shared, max_batch=max_batch,
-                     flags=(binding.FLAG_FP8_EXPERTS if fp8 else 0) | flags)
+                     flags=fmt_flag | flags)
     for l in range(cfg.L):
         W_r, b_r, W_p, b_p = routers[l]
         a.set_router(l, W_r, b_r)
@@ -292,9 +299,11 @@ def main():
     ap.add_argument("--no-spec", action="store_true", help="A/B: expert FFN without the speculative first fill")
     ap.add_argument("--fp8", action="store_true",
                     help="datatype study: e4m3 expert store with per-row scales (needs --ffn-only or --skip-extras)")
+    ap.add_argument("--fp4", action="store_true",
+                    help="datatype study: block-scaled e2m1 expert store (needs --ffn-only or --skip-extras)")
     args = ap.parse_args()
-    if args.fp8 and not (args.ffn_only or args.skip_extras):
-        ap.error("--fp8 is a study leg: combine it with --ffn-only or --skip-extras")
+    if (args.fp8 or args.fp4) and not (args.ffn_only or args.skip_extras):
+        ap.error("--fp8 / --fp4 are study legs: combine them with --ffn-only or --skip-extras")
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -325,8 +334,9 @@ def main():
         replicas.barrier()
         dist_sync = replicas.barrier
     B = args.batch
-    prob = build_problem(cfg, dev, fp8=args.fp8)
-    row_scale = (3 * cfg.d + 16) / (6 * cfg.d) if args.fp8 else 1.0     # bytes of a stored row relative to bf16
+    prob = build_problem(cfg, dev, fp8=args.fp8, fp4=args.fp4)
+    # bytes of a stored row relative to bf16
+    row_scale = synth.fp4_row_bytes(cfg.d) / (6 * cfg.d) if args.fp4 else (3 * cfg.d + 16) / (6 * cfg.d) if args.fp8 else 1.0
     T = min(cfg.T, args.warmup + args.steps)
     h, hp = hidden_inputs(cfg, T, B, dev)
     h_dev, hp_dev = h.to(dev), hp.to(dev)
@@ -345,7 +355,7 @@ def main():
             bytes_ffn = distinct * cfg.expert_bytes + cfg.shared_bytes + 2 * B * cfg.d * 4
         bytes_ffn = (bytes_ffn - 2 * B * cfg.d * 4) * row_scale + 2 * B * cfg.d * 4
         flops = 2.0 * 3 * cfg.d * (cfg.k * cfg.I + cfg.I_shared) * B
-        print(json.dumps({"ffn_only": True, "B": B, "weights": "e4m3" if args.fp8 else "bf16", "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6,
+        print(json.dumps({"ffn_only": True, "B": B, "weights": "e2m1" if args.fp4 else "e4m3" if args.fp8 else "bf16", "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6,
                           "launches": n_l, "GBps_mean": bytes_ffn / mean_s / 1e9, "bytes_per_launch": bytes_ffn,
                           "TFLOPs": flops / mean_s / 1e12}), flush=True)
         a.destroy()
@@ -456,8 +466,9 @@ def main():
         return
     line = {"metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps, "warmup": args.warmup,
             "ms_per_step": 1e3 * sec / args.steps, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
-            "dtype": "e4m3 weights, fp32 accumulation" if args.fp8 else "bf16", "data": "synthetic",
-            "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}" + (" (e4m3 expert store)" if args.fp8 else ""),
+            "dtype": "e2m1 weights, fp32 accumulation" if args.fp4 else "e4m3 weights, fp32 accumulation" if args.fp8 else "bf16",
+            "data": "synthetic",
+            "config": {"workload": f"config{cfg.cfg_id}:{cfg.name}" + (" (e2m1 expert store)" if args.fp4 else " (e4m3 expert store)" if args.fp8 else ""),
                        "L": cfg.L, "d": cfg.d, "N": cfg.N, "k": cfg.k,
                        "I": cfg.I, "C": cfg.N if args.resident else cfg.C, "B": B, "tau": TAU, "mode": "exact", "ctx_len": 1024,
                        "parallelism": "replicas only" if world > 1 else "single GPU",

@@ -32,8 +32,14 @@
  * With APEX_FLAG_FP8_EXPERTS (the expert-weight precision study of Sec. V-G: smaller experts, smaller
  * copies) a row is 3*d e4m3 codes followed by three fp32 scales and 4 bytes of padding,
  *   [I][ gate_i (d bytes) | up_i (d bytes) | downT_i (d bytes) | s_gate, s_up, s_down, 0 ],
- * weight = scale * code; 3*d + 16 bytes per row.  Needs d in {512, 1024, 1536, 2048, 4096}; batched steps
- * then run the streaming kernel per (token, expert) pair (no tensor-core path for this format yet).
+ * weight = scale * code; 3*d + 16 bytes per row.
+ * With APEX_FLAG_FP4_EXPERTS a row is 3*d e2m1 codes (two per byte, the even element in the low nibble),
+ * then one scale byte per 32 elements of each vector (a biased exponent: scale = 2^(byte - 127)), padded
+ * to a multiple of 16 bytes,
+ *   [I][ gate_i (d/2 bytes) | up_i (d/2) | downT_i (d/2) | gate scales (d/32) | up scales | downT scales | pad ],
+ * weight = scale of its block * code.
+ * Both need d in {512, 1024, 1536, 2048, 4096} and exclude each other; batched steps then run the
+ * streaming kernel per (token, expert) pair (no tensor-core path for these formats yet).
  */
 #ifndef APEX_H
 #define APEX_H
@@ -57,6 +63,7 @@ extern "C" {
 #define APEX_MODE_STALL_FREE 1 /* Algorithm 1: resident experts only, gates renormalised */
 
 #define APEX_FLAG_FP8_EXPERTS 1 /* apex_config.flags: expert stores and slots hold e4m3 rows (see below) */
+#define APEX_FLAG_FP4_EXPERTS 4 /* apex_config.flags: expert stores and slots hold block-scaled e2m1 rows (see below) */
 #define APEX_FLAG_NO_SPECULATION 2 /* apex_config.flags: the expert FFN does not start streaming the experts the prefetch
                                       router ranked first before the gate's decision is visible (for A/B timing; results
                                       are identical either way) */

@@ -159,12 +159,13 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   if (ctx->cfg.wait_limit_ns <= 0) ctx->cfg.wait_limit_ns = 2000000000ll;
   if (ctx->cfg.ctx_len == 0) ctx->cfg.ctx_len = 1024;
   const size_t L = c.L, N = c.N, C = c.C, d = c.d, MB = c.max_batch, k = c.k;
-  const bool fp8 = (c.flags & APEX_FLAG_FP8_EXPERTS) != 0;
-  if (fp8 && !ffn_fp8_shape_supported(c.d)) {
+  const bool fp8 = (c.flags & APEX_FLAG_FP8_EXPERTS) != 0, fp4 = (c.flags & APEX_FLAG_FP4_EXPERTS) != 0;
+  if ((fp8 && fp4) || ((fp8 || fp4) && !ffn_quantised_shape_supported(c.d))) {
     delete ctx;
     return APEX_EINVAL;
   }
-  const size_t row_bytes = fp8 ? 3 * d + 16 : 3 * d * 2;
+  ctx->fmt = fp4 ? 2 : (fp8 ? 1 : 0);
+  const size_t row_bytes = ffn_row_bytes(ctx->fmt, c.d);
   ctx->expert_bytes = row_bytes * (size_t)c.I;
   ctx->shared_bytes = row_bytes * (size_t)c.I_shared;
 
@@ -229,7 +230,7 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(dev_alloc(&ctx->d_exec_gate, MB * k));
   CR(dev_alloc(&ctx->d_cand_ncand, MB));
   // batched tensor-core path: scratch and tensor maps (only for contexts that will see large batches)
-  if (MB >= kTcMinBatch && !fp8 && tc_shape_supported(c.d, c.I, c.I_shared)) {
+  if (MB >= kTcMinBatch && ctx->fmt == 0 && tc_shape_supported(c.d, c.I, c.I_shared)) {
     const size_t rows = max_pairs + 256;
     const size_t i_max = (size_t)(c.I > c.I_shared ? c.I : c.I_shared);
     ctx->act_stride = (int)i_max;
@@ -702,7 +703,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.mode = mode; p.norm_topk = ctx->cfg.norm_topk; p.accumulate = 0;
   p.run_shared = ctx->cfg.I_shared > 0 ? 1 : 0;
   p.post_exec = 1;
-  p.fp8 = (ctx->cfg.flags & APEX_FLAG_FP8_EXPERTS) ? 1 : 0;
+  p.fmt = ctx->fmt;
   p.demand = ctx->d_demand + (size_t)layer * N;
   ctx->launch_tag = ctx->launch_tag % 0xfffffeu + 1u;
   p.demand_tag = ctx->launch_tag;

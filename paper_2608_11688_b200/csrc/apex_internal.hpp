@@ -140,7 +140,7 @@ struct FfnParams {
   const uint32_t* demand;       // [N] per layer: (tag << 8 | slot), published by the host after a demand copy
   uint32_t demand_tag;          // tag of this launch
   int demand_in_kernel;         // 1: a routed expert without a slot is waited for inside the kernel
-  int fp8;                      // 1: slots hold e4m3 rows with per-row scales
+  int fmt;                      // storage format of the slots: 0 bf16, 1 e4m3 with per-row scales, 2 e2m1 with block scales
   int zero_early;               // 1: y may be zeroed before the dependency wait (the preceding kernel does not touch y)
   const int32_t* spec;          // [k] predicted top-k of this layer-step (complete before the preceding kernel began), or null
   SlotSnapshot snap;
@@ -184,7 +184,8 @@ bool tc_make_weight_map(void* out, const void* base, int d, int I, size_t n_slot
 bool tc_make_rows_map(void* out, const void* base, int cols, size_t rows, size_t stride_elems);
 bool tc_shape_supported(int d, int I, int I_shared);
 bool ffn_shape_supported(int d);
-bool ffn_fp8_shape_supported(int d);
+bool ffn_quantised_shape_supported(int d);   // widths the e4m3 / e2m1 kernels were built for
+size_t ffn_row_bytes(int fmt, int d);        // bytes of one intermediate index (three vectors and their scales)
 
 }  // namespace apex
 
@@ -194,6 +195,7 @@ struct apex_ctx {
   std::string err;
   int device = 0;
   int n_sm = 0;
+  int fmt = 0;  // storage format of stores and slots (see FfnParams::fmt)
   size_t expert_bytes = 0;   // 3*I*d*2
   size_t shared_bytes = 0;
 

@@ -49,7 +49,7 @@ __device__ __forceinline__ unsigned long long globaltimer_ns_raw() {
 constexpr int kConsumerWarps = APEX_FFN_WARPS;
 constexpr int kCtasPerSm = APEX_FFN_CTAS_PER_SM;
 constexpr int kFfnThreads = kConsumerWarps * 32;
-constexpr int kMaxStages = 32;
+constexpr int kMaxStages = 64;
 // ring bytes; static tables fit in what is left of the 227 KB per-CTA limit (of half an SM's 228 KB with two CTAs per SM)
 constexpr int kSmemBudget = kCtasPerSm == 1 ? 224 * 1024 : 110 * 1024;
 
@@ -123,10 +123,38 @@ __device__ __forceinline__ unsigned long long ld_acquire_gpu_u64(const unsigned 
 __device__ __forceinline__ float bf16lo(uint32_t v) { return __uint_as_float(v << 16); }
 __device__ __forceinline__ float bf16hi(uint32_t v) { return __uint_as_float(v & 0xffff0000u); }
 
-// Eight consecutive weights of a row as fp32: bf16 (16 bytes) or e4m3 (8 bytes; the row's scale is applied later).
-template <bool FP8>
+// Storage formats of an expert row (FfnParams::fmt)
+constexpr int kFmtBf16 = 0;   // bf16
+constexpr int kFmtE4m3 = 1;   // e4m3 codes, one fp32 scale per vector of the row
+constexpr int kFmtMxfp4 = 2;  // e2m1 codes, one power-of-two scale (a biased exponent byte) per 32 elements
+
+__host__ __device__ constexpr uint32_t fmt_vec_bytes(int fmt, int d) { return fmt == kFmtMxfp4 ? d / 2 : (fmt == kFmtE4m3 ? d : 2 * d); }
+__host__ __device__ constexpr uint32_t fmt_entry_bytes(int fmt, int d) {
+  return fmt == kFmtMxfp4 ? ((3u * (d / 2) + 3u * (d / 32) + 15u) & ~15u) : (fmt == kFmtE4m3 ? 3u * d + 16u : 6u * d);
+}
+
+// Eight consecutive weights of a vector as fp32: bf16 (16 bytes), e4m3 (8 bytes) or e2m1 (4 bytes); scales are
+// applied by the caller.
+template <int FMT>
 __device__ __forceinline__ void load8(const uint8_t* row, int idx8, float (&w)[8]) {
-  if (FP8) {
+  if (FMT == kFmtMxfp4) {
+    const uint32_t v = reinterpret_cast<const uint32_t*>(row)[idx8];
+    uint32_t h2[4];
+    asm("{\n.reg .b8 b0, b1, b2, b3;\n"
+        "mov.b32 {b0, b1, b2, b3}, %4;\n"
+        "cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+        "cvt.rn.f16x2.e2m1x2 %1, b1;\n"
+        "cvt.rn.f16x2.e2m1x2 %2, b2;\n"
+        "cvt.rn.f16x2.e2m1x2 %3, b3;\n}"
+        : "=r"(h2[0]), "=r"(h2[1]), "=r"(h2[2]), "=r"(h2[3])
+        : "r"(v));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h2[i]));
+      w[2 * i] = f.x;
+      w[2 * i + 1] = f.y;
+    }
+  } else if (FMT == kFmtE4m3) {
     const uint2 v = reinterpret_cast<const uint2*>(row)[idx8];
     uint32_t h2[4];
     asm("cvt.rn.f16x2.e4m3x2 %0, %1;" : "=r"(h2[0]) : "h"((unsigned short)(v.x & 0xffffu)));
@@ -144,6 +172,10 @@ __device__ __forceinline__ void load8(const uint8_t* row, int idx8, float (&w)[8
     w[0] = bf16lo(v.x); w[1] = bf16hi(v.x); w[2] = bf16lo(v.y); w[3] = bf16hi(v.y);
     w[4] = bf16lo(v.z); w[5] = bf16hi(v.z); w[6] = bf16lo(v.w); w[7] = bf16hi(v.w);
   }
+}
+// scale of the 32-element block that holds elements 8*idx8 .. 8*idx8+7 (block-scaled format only)
+__device__ __forceinline__ float block_scale(const uint8_t* scales, int idx8) {
+  return __uint_as_float((uint32_t)scales[idx8 >> 2] << 23);
 }
 
 __device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
@@ -458,7 +490,7 @@ struct RowMap {
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
-template <int NCH, bool H_REGS, bool FP8>
+template <int NCH, bool H_REGS, int FMT>
 __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel(const FfnParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t s_full[kMaxStages];
@@ -469,8 +501,8 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   __shared__ int s_abort;
 
   constexpr int d = NCH * 256;
-  constexpr uint32_t row_bytes = FP8 ? d : d * 2;                      // one of the three vectors of a row
-  constexpr uint32_t entry_bytes = FP8 ? 3 * row_bytes + 16 : 3 * row_bytes;  // e4m3 rows carry three fp32 scales
+  constexpr uint32_t row_bytes = fmt_vec_bytes(FMT, d);      // one of the three vectors of a row
+  constexpr uint32_t entry_bytes = fmt_entry_bytes(FMT, d);  // the three vectors and, for the quantised formats, their scales
   // Each warp streams its own rows: it owns the ring stages {w, w+8, ...} and keeps NSW of its rows
   // in flight, so a stage is produced and consumed by the same warp (no "empty" barriers, and a
   // parity wait can never be a phase ahead).
@@ -908,8 +940,8 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
       float gw[8], uw[8], hh[8];
-      load8<FP8>(gs, c * 32 + lane, gw);
-      load8<FP8>(us, c * 32 + lane, uw);
+      load8<FMT>(gs, c * 32 + lane, gw);
+      load8<FMT>(us, c * 32 + lane, uw);
       if (H_REGS) {
 #pragma unroll
         for (int m = 0; m < 8; ++m) hh[m] = hreg[c * 8 + m];
@@ -918,15 +950,26 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
         const float4 b2 = __ldg(reinterpret_cast<const float4*>(hrow) + (c * 32 + lane) * 2 + 1);
         hh[0] = a.x; hh[1] = a.y; hh[2] = a.z; hh[3] = a.w; hh[4] = b2.x; hh[5] = b2.y; hh[6] = b2.z; hh[7] = b2.w;
       }
+      if (FMT == kFmtMxfp4) {  // the lane's eight elements share one block scale
+        float pg = 0.f, pu = 0.f;
 #pragma unroll
-      for (int m = 0; m < 8; ++m) g = fmaf(gw[m], hh[m], g);
+        for (int m = 0; m < 8; ++m) pg = fmaf(gw[m], hh[m], pg);
 #pragma unroll
-      for (int m = 0; m < 8; ++m) u = fmaf(uw[m], hh[m], u);
+        for (int m = 0; m < 8; ++m) pu = fmaf(uw[m], hh[m], pu);
+        const uint8_t* sc = ds + row_bytes;  // gate | up | downT block scales, d/32 bytes each
+        g = fmaf(block_scale(sc, c * 32 + lane), pg, g);
+        u = fmaf(block_scale(sc + d / 32, c * 32 + lane), pu, u);
+      } else {
+#pragma unroll
+        for (int m = 0; m < 8; ++m) g = fmaf(gw[m], hh[m], g);
+#pragma unroll
+        for (int m = 0; m < 8; ++m) u = fmaf(uw[m], hh[m], u);
+      }
     }
     g = warp_sum(g);
     u = warp_sum(u);
     float down_scale = 1.f;
-    if (FP8) {  // per-row scales of the e4m3 store: value = scale * code
+    if (FMT == kFmtE4m3) {  // per-row scales of the e4m3 store: value = scale * code
       const float* sc = reinterpret_cast<const float*>(ds + row_bytes);
       g *= sc[0];
       u *= sc[1];
@@ -936,9 +979,10 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
 #pragma unroll
     for (int c = 0; c < NCH; ++c) {
       float dw[8];
-      load8<FP8>(ds, c * 32 + lane, dw);
+      load8<FMT>(ds, c * 32 + lane, dw);
+      const float ac = FMT == kFmtMxfp4 ? a * block_scale(ds + row_bytes + 2 * (d / 32), c * 32 + lane) : a;
 #pragma unroll
-      for (int m = 0; m < 8; ++m) acc[c * 8 + m] = fmaf(a, dw[m], acc[c * 8 + m]);
+      for (int m = 0; m < 8; ++m) acc[c * 8 + m] = fmaf(ac, dw[m], acc[c * 8 + m]);
     }
     __syncwarp();  // every lane has read stage s: it may be refilled
     {
@@ -1046,15 +1090,15 @@ extern "C" int apex_debug_reset_spans() {
 }
 #endif
 
-template <int NCH, bool FP8>
+template <int NCH, int FMT>
 static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
   constexpr bool HR = NCH <= 8;
-  constexpr uint32_t entry = FP8 ? 3 * NCH * 256 + 16 : 3 * NCH * 256 * 2;
+  constexpr uint32_t entry = fmt_entry_bytes(FMT, NCH * 256);
   constexpr int NS = ring_stages(entry);
   const size_t smem = (size_t)NS * entry;
   static bool configured = false;
   if (!configured) {
-    cudaError_t e = cudaFuncSetAttribute(moe_ffn_stream_kernel<NCH, HR, FP8>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    cudaError_t e = cudaFuncSetAttribute(moe_ffn_stream_kernel<NCH, HR, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured = true;
   }
@@ -1068,7 +1112,7 @@ static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
   attr[0].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 1;
-  return cudaLaunchKernelEx(&cfg, moe_ffn_stream_kernel<NCH, HR, FP8>, p);
+  return cudaLaunchKernelEx(&cfg, moe_ffn_stream_kernel<NCH, HR, FMT>, p);
 }
 
 bool ffn_shape_supported(int d) {
@@ -1082,29 +1126,34 @@ bool ffn_shape_supported(int d) {
 int ffn_grid_ctas(int n_sm) { return n_sm * kCtasPerSm; }
 
 cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s) {
-  if (p.fp8) {  // e4m3 store: the shapes of the paper-sized configs
+  if (p.fmt == kFmtE4m3 || p.fmt == kFmtMxfp4) {  // quantised stores: the widths of the paper-sized configs
+#define APEX_FFN_CASE(NCH_) \
+  case NCH_ * 256: return p.fmt == kFmtE4m3 ? launch_ffn_t<NCH_, kFmtE4m3>(p, n_sm, s) : launch_ffn_t<NCH_, kFmtMxfp4>(p, n_sm, s);
     switch (p.d) {
-      case 1024: return launch_ffn_t<4, true>(p, n_sm, s);
-      case 1536: return launch_ffn_t<6, true>(p, n_sm, s);
-      case 2048: return launch_ffn_t<8, true>(p, n_sm, s);
-      case 4096: return launch_ffn_t<16, true>(p, n_sm, s);
-      case 512: return launch_ffn_t<2, true>(p, n_sm, s);
+      APEX_FFN_CASE(2)
+      APEX_FFN_CASE(4)
+      APEX_FFN_CASE(6)
+      APEX_FFN_CASE(8)
+      APEX_FFN_CASE(16)
     }
+#undef APEX_FFN_CASE
     return cudaErrorInvalidValue;
   }
   switch (p.d) {
-    case 256: return launch_ffn_t<1, false>(p, n_sm, s);
-    case 512: return launch_ffn_t<2, false>(p, n_sm, s);
-    case 768: return launch_ffn_t<3, false>(p, n_sm, s);
-    case 1024: return launch_ffn_t<4, false>(p, n_sm, s);
-    case 1536: return launch_ffn_t<6, false>(p, n_sm, s);
-    case 2048: return launch_ffn_t<8, false>(p, n_sm, s);
-    case 3072: return launch_ffn_t<12, false>(p, n_sm, s);
-    case 4096: return launch_ffn_t<16, false>(p, n_sm, s);
+    case 256: return launch_ffn_t<1, kFmtBf16>(p, n_sm, s);
+    case 512: return launch_ffn_t<2, kFmtBf16>(p, n_sm, s);
+    case 768: return launch_ffn_t<3, kFmtBf16>(p, n_sm, s);
+    case 1024: return launch_ffn_t<4, kFmtBf16>(p, n_sm, s);
+    case 1536: return launch_ffn_t<6, kFmtBf16>(p, n_sm, s);
+    case 2048: return launch_ffn_t<8, kFmtBf16>(p, n_sm, s);
+    case 3072: return launch_ffn_t<12, kFmtBf16>(p, n_sm, s);
+    case 4096: return launch_ffn_t<16, kFmtBf16>(p, n_sm, s);
   }
   return cudaErrorInvalidValue;
 }
 
-bool ffn_fp8_shape_supported(int d) { return d == 512 || d == 1024 || d == 1536 || d == 2048 || d == 4096; }
+bool ffn_quantised_shape_supported(int d) { return d == 512 || d == 1024 || d == 1536 || d == 2048 || d == 4096; }
+
+size_t ffn_row_bytes(int fmt, int d) { return fmt_entry_bytes(fmt, d); }
 
 }  // namespace apex

@@ -225,6 +225,69 @@ def expert_store_fp8(cfg: Config, layer: int, device="cpu"):
     return out
 
 
+_E2M1 = (0.0, 0.5, 1.0, 1.5, 2.0, 3.0, 4.0, 6.0)
+
+
+def fp4_row_bytes(d: int) -> int:
+    """Bytes of one intermediate index in the block-scaled e2m1 layout: codes, block scales, padding to 16."""
+    return (3 * (d // 2) + 3 * (d // 32) + 15) & ~15
+
+
+def quantize_store_fp4(w):
+    """bf16/fp32 store [..., I, 3, d] -> uint8 [..., I, fp4_row_bytes(d)] in the library's block-scaled e2m1 layout.
+
+    Per block of 32 consecutive elements of a vector the scale is the power of two 2^e with e the smallest integer
+    for which max|block| / 2^e <= 6 (6 = largest e2m1 value), stored as the byte e + 127 (0 for an all-zero block:
+    scale 0).  Codes: sign bit and the index of the nearest of (0, .5, 1, 1.5, 2, 3, 4, 6); two per byte, the even
+    element in the low nibble.  Row: gate | up | downT codes (d/2 bytes each), then their scale bytes (d/32 each).
+    """
+    import torch
+    wf = w.to(torch.float32)
+    d = wf.shape[-1]
+    lead = wf.shape[:-2]
+    blk = wf.reshape(lead + (3, d // 32, 32))
+    amax = blk.abs().amax(dim=-1)
+    e = torch.ceil(torch.log2(torch.clamp(amax, min=1e-38) / 6.0))
+    e = torch.clamp(e, -126, 127)
+    sbyte = torch.where(amax > 0, e + 127, torch.zeros_like(e)).to(torch.uint8)                  # [..., 3, d/32]
+    scale = torch.where(amax > 0, torch.exp2(e), torch.ones_like(e))
+    x = blk / scale[..., None]
+    mids = torch.tensor([0.25, 0.75, 1.25, 1.75, 2.5, 3.5, 5.0], dtype=torch.float32, device=wf.device)
+    code = torch.bucketize(x.abs(), mids).to(torch.uint8) | ((x < 0).to(torch.uint8) << 3)         # [..., 3, d/32, 32]
+    code = code.reshape(lead + (3, d // 2, 2))
+    packed = code[..., 0] | (code[..., 1] << 4)                                                     # [..., 3, d/2]
+    out = torch.zeros(lead + (fp4_row_bytes(d),), dtype=torch.uint8, device=wf.device)
+    out[..., :3 * (d // 2)] = packed.reshape(lead + (3 * (d // 2),))
+    out[..., 3 * (d // 2):3 * (d // 2) + 3 * (d // 32)] = sbyte.reshape(lead + (3 * (d // 32),))
+    return out
+
+
+def dequantize_store_fp4(q, d: int) -> np.ndarray:
+    """uint8 [..., I, fp4_row_bytes(d)] -> fp64 numpy [..., I, 3, d]: weight = 2^(scale byte - 127) * code value
+    (scale byte 0: the block is zero)."""
+    q = q.detach().cpu().numpy()
+    lead = q.shape[:-1]
+    packed = q[..., :3 * (d // 2)].reshape(lead + (3, d // 2))
+    codes = np.stack([packed & 0xF, packed >> 4], axis=-1).reshape(lead + (3, d))
+    table = np.array(_E2M1 + tuple(-v for v in _E2M1), dtype=np.float64)
+    vals = table[codes]
+    sb = q[..., 3 * (d // 2):3 * (d // 2) + 3 * (d // 32)].reshape(lead + (3, d // 32)).astype(np.int64)
+    scale = np.where(sb > 0, np.ldexp(1.0, sb - 127), 0.0)
+    return vals * np.repeat(scale, 32, axis=-1)
+
+
+def expert_store_fp4(cfg: Config, layer: int, device="cpu"):
+    """uint8 tensor [N][I][fp4_row_bytes(d)]: the seeded bf16 store of ``expert_store`` quantised block by block."""
+    import torch
+    out = torch.empty((cfg.N, cfg.I, fp4_row_bytes(cfg.d)), dtype=torch.uint8, device=device)
+    g = torch.Generator(device=device)
+    g.manual_seed((BASE_SEED * 1000003 + cfg.cfg_id * 10007 + layer * 101 + _KIND["experts"]) & 0x7FFFFFFF)
+    for e in range(cfg.N):
+        t = torch.randn((cfg.I, 3, cfg.d), generator=g, device=device, dtype=torch.float32)
+        out[e].copy_(quantize_store_fp4((t * 0.02).to(torch.bfloat16)))
+    return out
+
+
 def bf16_to_f32_numpy(t) -> np.ndarray:
     """Lossless widening of a torch bf16 tensor to a numpy fp32 array (test helper)."""
     import torch

@@ -44,9 +44,10 @@ class Report:
 class Problem:
     """Parameters and expert stores of one config on the GPU machine, shared by library and oracle."""
 
-    def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset", fp8=False):
+    def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset", fp8=False, fp4=False):
         self.cfg = cfg
         self.fp8 = fp8
+        self.fp4 = fp4
         self.L = layers or cfg.L
         self.routers = [synth.router_weights(cfg, l) for l in range(self.L)]
         self.cdf = [synth.handset_cdf_params(cfg) if cdf == "handset" else synth.cdf_params(cfg, l)
@@ -54,7 +55,10 @@ class Problem:
         self.stores = []
         self.shared = []
         for l in range(self.L):
-            if fp8:
+            if fp4:
+                st = torch.empty((cfg.N, cfg.I, synth.fp4_row_bytes(cfg.d)), dtype=torch.uint8, pin_memory=True)
+                tmp = synth.expert_store_fp4(cfg, l, device=device)
+            elif fp8:
                 st = torch.empty((cfg.N, cfg.I, 3 * cfg.d + 16), dtype=torch.uint8, pin_memory=True)
                 tmp = synth.expert_store_fp8(cfg, l, device=device)
             else:
@@ -64,7 +68,9 @@ class Problem:
             del tmp
             self.stores.append(st)
             sh = synth.shared_expert(cfg, l, device=device)
-            if fp8 and sh is not None:
+            if fp4 and sh is not None:
+                sh = synth.quantize_store_fp4(sh)
+            elif fp8 and sh is not None:
                 sh = synth.quantize_store_fp8(sh)
             self.shared.append(sh)
         torch.cuda.synchronize()
@@ -74,7 +80,7 @@ class Problem:
         build.build()
         a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C or cfg.C, L=self.L, I_shared=cfg.I_shared,
                          max_batch=max_batch, norm_topk=norm_topk, cache_reuse=cache_reuse,
-                         wait_limit_ns=wait_limit_ns, flags=(binding.FLAG_FP8_EXPERTS if self.fp8 else 0) | flags)
+                         wait_limit_ns=wait_limit_ns, flags=(binding.FLAG_FP4_EXPERTS if self.fp4 else binding.FLAG_FP8_EXPERTS if self.fp8 else 0) | flags)
         for l in range(self.L):
             W_r, b_r, W_p, b_p = self.routers[l]
             a.set_router(l, W_r, b_r)
@@ -89,6 +95,8 @@ class Problem:
         st = self.stores[layer]
 
         def get(e):
+            if self.fp4:
+                return synth.split_store(synth.dequantize_store_fp4(st[e], self.cfg.d))
             if self.fp8:
                 return synth.split_store(synth.dequantize_store_fp8(st[e], self.cfg.d))
             w = st[e].to(torch.float32).numpy()
@@ -99,6 +107,8 @@ class Problem:
         sh = self.shared[layer]
         if sh is None:
             return None
+        if self.fp4:
+            return synth.split_store(synth.dequantize_store_fp4(sh, self.cfg.d))
         if self.fp8:
             return synth.split_store(synth.dequantize_store_fp8(sh, self.cfg.d))
         w = sh.detach().cpu().to(torch.float32).numpy()

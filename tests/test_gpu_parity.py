@@ -149,6 +149,38 @@ def test_fp8_store_config1_shape_two_layers(mode):
     print("fp8 config1", mode, rep)
 
 
+# ------------------------------------------------------------------ block-scaled e2m1 expert store
+def _run_fp4(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1):
+    hz = _harness()
+    prob = hz.Problem(cfg, layers=layers, fp4=True)
+    return _run(cfg, mode=mode, tau=tau, T=T, B=B, layers=layers, prob=prob, check_ffn_every=check_ffn_every)
+
+
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+@pytest.mark.parametrize("d,N,k,I,C,Ish", [(512, 12, 3, 40, 6, 0), (1024, 16, 4, 17, 8, 24), (2048, 8, 2, 9, 4, 0),
+                                            (4096, 6, 2, 5, 3, 7)])
+def test_fp4_store_tiny_shapes(d, N, k, I, C, Ish, mode):
+    cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, T=8, I_shared=Ish, sigma_p=1.0, cfg_id=300 + N)
+    rep, stats = _run_fp4(cfg, mode=mode, tau=0.7, T=8)
+    assert rep.layer_steps == 8 and rep.ffn_checked + rep.near_ties >= 8
+    assert stats["bytes_copied"] == (rep.n_prefetch_copies + rep.n_demand_copies) * I * synth.fp4_row_bytes(d)
+    print("fp4", d, mode, rep)
+
+
+def test_fp4_store_batched_runs_streaming_kernel():
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=128, C=8, T=3, I_shared=128, sigma_p=1.0, cfg_id=315)
+    rep, stats = _run_fp4(cfg, mode="exact", tau=0.8, T=3, B=5)
+    assert stats["tokens"] == 15
+
+
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_fp4_store_config1_shape_two_layers(mode):
+    cfg = synth.CONFIGS[1]
+    rep, stats = _run_fp4(cfg, mode=mode, tau=0.9, T=12, layers=2, check_ffn_every=3)
+    assert rep.layer_steps == 24
+    print("fp4 config1", mode, rep)
+
+
 # ------------------------------------------------------------------ speculative first fill of the expert FFN
 @pytest.mark.parametrize("mode", ["exact", "stall_free"])
 @pytest.mark.parametrize("sigma_p", [0.0, 8.0])

@@ -51,8 +51,32 @@ def test_null_and_bad_arguments_are_rejected_without_cuda(lib):
     cfg = binding.ApexConfig(d=768, N=8, k=2, I=8, I_shared=0, C=4, L=1, max_batch=1, norm_topk=1, cache_reuse=1,
                              flags=binding.FLAG_FP8_EXPERTS)
     assert lib.apex_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.APEX_EINVAL
+    cfg = binding.ApexConfig(d=512, N=8, k=2, I=8, I_shared=0, C=4, L=1, max_batch=1, norm_topk=1, cache_reuse=1,
+                             flags=binding.FLAG_FP8_EXPERTS | binding.FLAG_FP4_EXPERTS)
+    assert lib.apex_create(ctypes.byref(cfg), ctypes.byref(h)) == binding.APEX_EINVAL   # one format at a time
     assert lib.apex_slots_create(8, 9, 1) is None
     assert lib.apex_launch_count(None) == -1
+
+
+def test_fp4_store_generator_round_trips_within_e2m1_precision():
+    import numpy as np
+    import torch
+    from paper_2608_11688_b200 import synth
+    cfg = synth.tiny_config(d=512, N=3, k=1, I=5)
+    w = synth.expert_store(cfg, 0).to(torch.float32).numpy()
+    q = synth.expert_store_fp4(cfg, 0)
+    assert q.shape == (3, 5, synth.fp4_row_bytes(512)) and synth.fp4_row_bytes(512) % 16 == 0
+    dq = synth.dequantize_store_fp4(q, 512)
+    # a block's scale is the smallest power of two that maps its maximum into [-6, 6]; the widest gap between
+    # neighbouring e2m1 values there is 2 (between 4 and 6), so the error is at most one scale unit, and the
+    # scale is below amax / 3
+    blk_w = w.reshape(3, 5, 3, 16, 32)
+    blk_e = np.abs(dq - w).reshape(3, 5, 3, 16, 32)
+    amax = np.abs(blk_w).max(-1, keepdims=True)
+    assert np.all(blk_e <= amax / 3 + 1e-12)
+    # quantising what was dequantised reproduces the same values (a block may be re-coded with a smaller scale)
+    q2 = synth.quantize_store_fp4(torch.from_numpy(dq.astype(np.float32)))
+    assert np.array_equal(synth.dequantize_store_fp4(q2, 512), dq)
 
 
 def test_fp8_store_generator_round_trips_within_e4m3_precision():

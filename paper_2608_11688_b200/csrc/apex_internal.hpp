@@ -149,6 +149,8 @@ struct FfnParams {
   int d, N, k, I, I_shared, B, mode, norm_topk, accumulate, run_shared, post_exec;
 };
 
+constexpr int kMaxDevices = 64;  // per-device launch attributes are remembered for this many devices
+
 // Batched tensor-core path (kernels_ffn_tc.cu)
 constexpr int kTcMinBatch = 4;  // from this many tokens per step the tensor-core grouped GEMM runs (measured crossover)
 struct TcParams {

@@ -1096,11 +1096,13 @@ static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
   constexpr uint32_t entry = fmt_entry_bytes(FMT, NCH * 256);
   constexpr int NS = ring_stages(entry);
   const size_t smem = (size_t)NS * entry;
-  static bool configured = false;
-  if (!configured) {
+  static bool configured[kMaxDevices] = {};  // the attribute is per device
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(moe_ffn_stream_kernel<NCH, HR, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
-    configured = true;
+    if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
   }
   cudaLaunchConfig_t cfg = {};
   cfg.gridDim = dim3(n_sm * kCtasPerSm, 1, 1);

@@ -490,14 +490,16 @@ bool tc_shape_supported(int d, int I, int I_shared) {
 }
 
 cudaError_t launch_ffn_tc(const TcParams& p_in, const TcMaps& m, int n_sm, cudaStream_t s) {
-  static bool configured = false;
+  static bool configured[kMaxDevices] = {};  // the attribute is per device
   const size_t budget = 196 * 1024;  // ring bytes per CTA
-  if (!configured) {
+  int dev = 0;
+  cudaGetDevice(&dev);
+  if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
     cudaError_t e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget + 1024);
     if (e != cudaSuccess) return e;
     e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget + 1024);
     if (e != cudaSuccess) return e;
-    configured = true;
+    if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
   }
   TcParams p = p_in;
   const int b32 = (p.f.B + 31) & ~31;

@@ -145,6 +145,9 @@ __device__ unsigned long long g_tc_tl[2][148][128];
 #define TCTL(ph, i) do { } while (0)
 #endif
 
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 struct Group {
   int expert, pair_off, n_tok;
 };
@@ -160,6 +163,8 @@ __device__ __forceinline__ Group load_group(const int32_t* grp, int g) {
 
 // ---------------------------------------------------------------- gather + zero
 __global__ void __launch_bounds__(256) ffn_tc_gather_kernel(const TcParams p) {
+  pdl_wait();               // the plan kernel's pair list is complete from here on
+  pdl_launch_dependents();  // the next kernel may start its prologue
   const int n_pairs = p.f.n_pairs[0];
   const int d = p.f.d;
   if (!p.f.accumulate) {
@@ -236,6 +241,9 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
+  // everything above (barriers, TMEM, tensor-map prefetch) is independent of the preceding kernel
+  pdl_wait();
+  pdl_launch_dependents();
 
   // the group table goes to shared memory once: a global load per unit would sit on every role's path
   for (int i = tid; i < 4 + 3 * (N + 1); i += kTcThreads) s_grp[i] = grp[i];
@@ -508,20 +516,34 @@ cudaError_t launch_ffn_tc(const TcParams& p_in, const TcMaps& m, int n_sm, cudaS
   const size_t st1 = 2 * 128 * 128 + (size_t)p.nmax1 * 128, st2 = 2 * 64 * 128 + 2 * (size_t)p.nmax2 * 128;
   p.nstage1 = (int)(budget / st1) < 4 ? (int)(budget / st1) : 4;
   p.nstage2 = (int)(budget / st2) < 4 ? (int)(budget / st2) : 4;
-  ffn_tc_gather_kernel<<<n_sm * 2, 256, 0, s>>>(p);
-  cudaError_t e = cudaGetLastError();
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;  // prologues overlap the preceding kernel's tail
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cudaLaunchConfig_t cfg = {};
+  cfg.stream = s;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  cfg.gridDim = dim3(n_sm * 2, 1, 1);
+  cfg.blockDim = dim3(256, 1, 1);
+  cfg.dynamicSmemBytes = 0;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, ffn_tc_gather_kernel, p);
   if (e != cudaSuccess) return e;
   const CUtensorMap* w1 = reinterpret_cast<const CUtensorMap*>(m.w_gateup);
   const CUtensorMap* ws1 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_gateup : m.w_gateup);
   const CUtensorMap* w2 = reinterpret_cast<const CUtensorMap*>(m.w_down);
   const CUtensorMap* ws2 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_down : m.w_down);
   const CUtensorMap* xg = reinterpret_cast<const CUtensorMap*>(m.xg);
-  ffn_tc_gemm_kernel<1><<<n_sm, kTcThreads, p.nstage1 * st1 + 1024, s>>>(*w1, *ws1, *xg, *xg, p);
-  e = cudaGetLastError();
+  cfg.gridDim = dim3(n_sm, 1, 1);
+  cfg.blockDim = dim3(kTcThreads, 1, 1);
+  // Each CTA allocates all 512 TMEM columns, so two CTAs must never share an SM (the second would sit in
+  // tcgen05.alloc until the first has finished): ask for more than half an SM's shared memory in any case.
+  const size_t one_per_sm = 120 * 1024;
+  cfg.dynamicSmemBytes = p.nstage1 * st1 + 1024 > one_per_sm ? p.nstage1 * st1 + 1024 : one_per_sm;
+  e = cudaLaunchKernelEx(&cfg, ffn_tc_gemm_kernel<1>, *w1, *ws1, *xg, *xg, p);
   if (e != cudaSuccess) return e;
-  ffn_tc_gemm_kernel<2><<<n_sm, kTcThreads, p.nstage2 * st2 + 1024, s>>>(*w2, *ws2, *reinterpret_cast<const CUtensorMap*>(m.act),
-                                                                        *reinterpret_cast<const CUtensorMap*>(m.act_lo), p);
-  return cudaGetLastError();
+  cfg.dynamicSmemBytes = p.nstage2 * st2 + 1024 > one_per_sm ? p.nstage2 * st2 + 1024 : one_per_sm;
+  return cudaLaunchKernelEx(&cfg, ffn_tc_gemm_kernel<2>, *w2, *ws2, *reinterpret_cast<const CUtensorMap*>(m.act),
+                            *reinterpret_cast<const CUtensorMap*>(m.act_lo), p);
 }
 
 }  // namespace apex

@@ -364,17 +364,6 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   if (p.post_exec && lane == 0 && my_hits && p.stats) atomicAdd(&p.stats->hits_R, (unsigned long long)my_hits);
   __syncthreads();
   PTL(1);
-  // The routed and the execution sets go to the host mailbox here, as whole lines from consecutive
-  // threads (a 4-byte store per lane and token from inside the loop above cost 2 us per token), and
-  // early, so that the trip over the host link overlaps the sorting below.
-  if (p.post_exec) {
-    for (int t = threadIdx.x; t < B * k; t += blockDim.x) {
-      const int b = t / k, j = t - b * k;
-      const unsigned long long m = s_exec[b];
-      p.mbox_exec[t] = j < __popcll(m) ? nth_set_bit64(m, j) : -1;
-      p.mbox_kr[t] = p.idx[t];
-    }
-  }
   // ---- phase B, counts: warp w counts the tokens of experts w and w + 32
   for (int e = warp; e < N; e += nwarp) {
     int c = 0;
@@ -459,6 +448,16 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     }
   }
   PTL(4);
+  // The routed and the execution sets go to the host mailbox last, as whole lines from consecutive
+  // threads (a 4-byte store per lane and token from inside the planning loop cost 2 us per token).
+  if (p.post_exec) {
+    for (int t = threadIdx.x; t < B * k; t += blockDim.x) {
+      const int b = t / k, j = t - b * k;
+      const unsigned long long m = s_exec[b];
+      p.mbox_exec[t] = j < __popcll(m) ? nth_set_bit64(m, j) : -1;
+      p.mbox_kr[t] = p.idx[t];
+    }
+  }
   if (p.post_exec) {
     // the barrier orders every thread's mailbox stores before thread 0's system-scope fence
     // (fences are cumulative), which orders them before the sequence number

@@ -153,6 +153,8 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
       c.L < 1 || c.I < 1 || c.I_shared < 0 || c.max_batch < 1 || c.max_batch > APEX_MAX_BATCH || !ffn_shape_supported(c.d) ||
       c.ctx_len < 0)
     return APEX_EINVAL;
+  // the kernels index (token, expert, intermediate index) rows with 31 bits
+  if ((long long)c.max_batch * (c.k + 1) * (long long)(c.I > c.I_shared ? c.I : c.I_shared) >= (1ll << 30)) return APEX_EINVAL;
   apex_ctx* ctx = new (std::nothrow) apex_ctx();
   if (!ctx) return APEX_ENOMEM;
   ctx->cfg = c;

@@ -482,8 +482,8 @@ cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s) {
 struct RowMap {
   int n_routed;          // routed pairs
   int n_pairs;           // all pairs
-  long long routed_rows; // n_routed * I
-  long long total_rows;
+  int routed_rows;       // n_routed * I (the host refuses shapes whose row count does not fit 31 bits)
+  int total_rows;
 };
 
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
@@ -577,31 +577,31 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   RowMap rm;
   bool dynamic = false;
   int S = 0, chunk = 1, n_static = 0;
-  long long static_base = 0, dyn_begin = 0, dyn_rows = 0;
+  int static_base = 0, dyn_begin = 0, dyn_rows = 0;
   auto set_geometry = [&](int n_routed, int n_pairs) {
     rm.n_routed = n_routed;
     rm.n_pairs = n_pairs;
-    rm.routed_rows = (long long)n_routed * I;
-    rm.total_rows = rm.routed_rows + (long long)(n_pairs - n_routed) * p.I_shared;
-    const long long per_cta = rm.total_rows / G;
+    rm.routed_rows = n_routed * I;
+    rm.total_rows = rm.routed_rows + (n_pairs - n_routed) * p.I_shared;
+    const int per_cta = rm.total_rows / G, extra = rm.total_rows - per_cta * G;  // the first `extra` CTAs take one row more
     dynamic = per_cta >= 2 * NS;
-    const long long range_lo = rm.total_rows * cta / G, range_hi = rm.total_rows * (cta + 1) / G;
+    const int range_lo = cta * per_cta + (cta < extra ? cta : extra), range_hi = range_lo + per_cta + (cta < extra ? 1 : 0);
     S = dynamic ? NS : (int)(range_hi - range_lo);  // rows this CTA knows about at launch
-    static_base = dynamic ? (long long)cta * NS : range_lo;
-    dyn_begin = dynamic ? (long long)G * NS : rm.total_rows;
+    static_base = dynamic ? cta * NS : range_lo;
+    dyn_begin = dynamic ? G * NS : rm.total_rows;
     dyn_rows = rm.total_rows - dyn_begin;
-    const long long per_ticket = (dyn_rows + (long long)G * kConsumerWarps * 4 - 1) / ((long long)G * kConsumerWarps * 4);
+    const int per_ticket = (dyn_rows + G * kConsumerWarps * 4 - 1) / (G * kConsumerWarps * 4);
     chunk = per_ticket > 1 ? (int)per_ticket : 1;   // rows per ticket: about four tickets per warp
     n_static = S > warp ? (S - warp + kConsumerWarps - 1) / kConsumerWarps : 0;  // static rows of this warp
   };
   // (position in the row space, index inside the expert) of row r
-  auto locate = [&](long long r, int* pidx, long long* i) {
+  auto locate = [&](int r, int* pidx, int* i) {
     if (r < rm.routed_rows) {
       *pidx = (int)(r / I);
-      *i = r - (long long)*pidx * I;
+      *i = r - *pidx * I;
     } else {
       *pidx = rm.n_routed + (int)((r - rm.routed_rows) / p.I_shared);
-      *i = r - rm.routed_rows - (long long)(*pidx - rm.n_routed) * p.I_shared;
+      *i = r - rm.routed_rows - (*pidx - rm.n_routed) * p.I_shared;
     }
   };
 
@@ -628,8 +628,8 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
     const int fill = n_static < NSW ? n_static : NSW;
     if (lane < fill) {
       int pidx;
-      long long i;
-      locate(static_base + warp + (long long)kConsumerWarps * lane, &pidx, &i);
+      int i;
+      locate(static_base + warp + kConsumerWarps * lane, &pidx, &i);
       const int e = pidx < k ? s_pos[warp][pidx] : N;
       const uint8_t* base = nullptr;
       if (e >= N) {
@@ -725,9 +725,8 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   };
 
   // Starts the copy of row r as this warp's n-th row, into stage (n mod NSW) of the warp.
-  auto issue = [&](long long r, int n) {
-    int pidx, e, tok;
-    long long i;
+  auto issue = [&](int r, int n) {
+    int pidx, e, tok, i;
     float gate = 0.f;
     locate(r, &pidx, &i);
     if (B == 1) {
@@ -821,21 +820,23 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   if (poster && will_wait_for_host) post_plan();
   // ---- row supply of this warp (state lives in lane 0; the other lanes learn the outcome by shuffle)
   int next_static = 0;                 // static rows of this warp already started
-  long long dyn_cur = 0, dyn_end = 0;  // rows of the current ticket
+  int dyn_cur = 0, dyn_end = 0;  // rows of the current ticket
   bool dyn_done = dyn_rows <= 0;
-  auto next_row = [&]() -> long long {  // lane 0 only
-    if (next_static < n_static) return static_base + warp + (long long)kConsumerWarps * next_static++;
+  auto next_row = [&]() -> int {  // lane 0 only
+    if (next_static < n_static) return static_base + warp + kConsumerWarps * next_static++;
     if (dyn_cur < dyn_end) return dyn_cur++;
     if (dyn_done) return -1;
     // Tickets are taken on demand, never ahead: the rows must go to the warps that are free first
     // (all stages of all SMs are requested at once at the start, and which SM is served first is a
     // matter of queueing; an SM whose first rows land late should not also hold extra rows).
     const unsigned int ticket = atomicAdd(p.ticket, 1u);
-    const long long first = dyn_begin + (long long)ticket * chunk;
-    if (first >= rm.total_rows) {
+    // (the host bounds the row count well below 2^31, and at most a few hundred tickets overshoot the end)
+    const long long first64 = (long long)dyn_begin + (long long)ticket * chunk;
+    if (first64 >= rm.total_rows) {
       dyn_done = true;
       return -1;
     }
+    const int first = (int)first64;
     dyn_cur = first;
     dyn_end = first + chunk < rm.total_rows ? first + chunk : rm.total_rows;
     return dyn_cur++;
@@ -850,8 +851,8 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
     bool confirmed = false;
     if (spec_geometry && lane < first_fill) {
       int pidx;
-      long long i;
-      locate(static_base + warp + (long long)kConsumerWarps * lane, &pidx, &i);
+      int i;
+      locate(static_base + warp + kConsumerWarps * lane, &pidx, &i);
       confirmed = s_exp[warp + kConsumerWarps * lane] == (pidx < rm.n_routed ? s_pos[warp][pidx] : N);
     }
     if (!confirmed) {
@@ -863,7 +864,7 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   const unsigned phase_ahead = __ballot_sync(0xffffffffu, dropped);  // bit n: stage n of this warp
   if (lane < first_fill && !spec_issued && ok) {
     if (lane == 0 && warp == 0) TL(3);
-    issue(static_base + warp + (long long)kConsumerWarps * lane, lane);
+    issue(static_base + warp + kConsumerWarps * lane, lane);
   }
   if (!ok) atomicExch(&s_abort, 1);
   __syncwarp();
@@ -874,7 +875,7 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   while (tail < NSW) {
     int more = 0;
     if (lane == 0 && ok) {
-      const long long r = next_row();
+      const int r = next_row();
       if (r >= 0) {
         issue(r, tail);
         if (!ok) atomicExch(&s_abort, 1);
@@ -987,7 +988,7 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
     {
       int more = 0;
       if (lane == 0 && ok) {
-        const long long r = next_row();
+        const int r = next_row();
         if (r >= 0) {
           asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
           issue(r, tail);

@@ -146,6 +146,49 @@ def make_ctx(cfg, prob, C, max_batch=1, flags=0):
     return a
 
 
+def train_auxiliary(cfg, prob, device, n_calib=8192, distill_iters=100, distill_lr=1e-4, fit_iters=600):
+    """The paper's two training stages on this GPU (Sec. IV-C): distil the prefetch router of every layer from the
+    router (Eq. (10)), then refit the confidence model on the distilled router's rankings (Eq. (11)).  Returns new
+    (routers, cdf) lists; the calibration tokens come from the seeded generator's calibration stream.  The step size
+    is small on purpose: a layer has N * (d + 1) parameters and only n_calib tokens, and Adam moves every weight by
+    about lr per step whatever its gradient, so a larger step overfits the calibration set within a few iterations."""
+    import torch
+    from paper_2608_11688_b200 import binding, synth
+    routers, cdf, store, shared = prob
+    new_routers, new_cdf = [], []
+    t_d = t_f = 0.0
+    for l in range(cfg.L):
+        W_r, b_r, W_p, b_p = routers[l]
+        h, hp = synth.hidden_states(cfg, l, n_calib, 1, calib=True)
+        H, Hp = h[:, 0].astype(np.float64), hp[:, 0].astype(np.float64)
+        Zr = Hp @ W_r.astype(np.float64).T + b_r.astype(np.float64)
+        Qr = np.exp(Zr - Zr.max(1, keepdims=True))
+        Qr /= Qr.sum(1, keepdims=True)
+        Hd = torch.from_numpy(H.astype(np.float32)).to(device)
+        t0 = time.perf_counter()
+        W_p2, b_p2 = binding.distill_router(Hd, torch.from_numpy(Qr.astype(np.float32)).to(device), W_p, b_p,
+                                            iters=distill_iters, lr=distill_lr)
+        t_d += time.perf_counter() - t0
+        # calibration set of the confidence model: x = the distilled router's probabilities in descending order,
+        # delta* = (largest rank of a routed expert in its ranking) - k
+        Zp = H @ W_p2.astype(np.float64).T + b_p2.astype(np.float64)
+        order = np.lexsort((np.broadcast_to(np.arange(cfg.N), Zp.shape), -Zp), axis=1)     # value desc, index asc
+        Qp = np.exp(Zp - Zp.max(1, keepdims=True))
+        Qp /= Qp.sum(1, keepdims=True)
+        X = np.take_along_axis(Qp, order, axis=1)
+        rank = np.empty_like(order)
+        np.put_along_axis(rank, order, np.broadcast_to(np.arange(cfg.N), order.shape), axis=1)
+        K_r = np.lexsort((np.broadcast_to(np.arange(cfg.N), Zr.shape), -Zr), axis=1)[:, :cfg.k]
+        dstar = np.take_along_axis(rank, K_r, axis=1).max(1) + 1 - cfg.k
+        t0 = time.perf_counter()
+        w, theta = binding.fit_cdf(torch.from_numpy(X).to(device), torch.from_numpy(dstar.astype(np.int32)).to(device),
+                                   cfg.k, iters=fit_iters)
+        t_f += time.perf_counter() - t0
+        new_routers.append((W_r, b_r, W_p2, b_p2))
+        new_cdf.append((w, theta))
+    return new_routers, new_cdf, {"distill_s": t_d, "fit_s": t_f, "calibration_tokens_per_layer": n_calib}
+
+
 def hidden_inputs(cfg, T, B, device):
     """[T][L][B][d] tensors on the device (h, h')."""
     import torch
@@ -299,11 +342,16 @@ def main():
     ap.add_argument("--no-spec", action="store_true", help="A/B: expert FFN without the speculative first fill")
     ap.add_argument("--fp8", action="store_true",
                     help="datatype study: e4m3 expert store with per-row scales (needs --ffn-only or --skip-extras)")
+    ap.add_argument("--train-aux", action="store_true",
+                    help="study: distil the prefetch routers and refit the confidence models on this GPU first "
+                         "(a different predictor than the workload's: needs --skip-extras)")
     ap.add_argument("--fp4", action="store_true",
                     help="datatype study: block-scaled e2m1 expert store (needs --ffn-only or --skip-extras)")
     args = ap.parse_args()
     if (args.fp8 or args.fp4) and not (args.ffn_only or args.skip_extras):
         ap.error("--fp8 / --fp4 are study legs: combine them with --ffn-only or --skip-extras")
+    if args.train_aux and not args.skip_extras:
+        ap.error("--train-aux is a study leg: combine it with --skip-extras")
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -335,6 +383,10 @@ def main():
         dist_sync = replicas.barrier
     B = args.batch
     prob = build_problem(cfg, dev, fp8=args.fp8, fp4=args.fp4)
+    aux_info = None
+    if args.train_aux:
+        r2, c2, aux_info = train_auxiliary(cfg, prob, dev)
+        prob = (r2, c2, prob[2], prob[3])
     # bytes of a stored row relative to bf16
     row_scale = synth.fp4_row_bytes(cfg.d) / (6 * cfg.d) if args.fp4 else (3 * cfg.d + 16) / (6 * cfg.d) if args.fp8 else 1.0
     T = min(cfg.T, args.warmup + args.steps)
@@ -477,6 +529,13 @@ def main():
             "clocks": clocks, "gpu_launches": int(launches),
             "e2e": e2e, "roofline": roof, "cpu_baseline": cpu, "modes": extras,
             "stats_headline": {"copies_per_token": (st_all["prefetch_copies"] + st_all["demand_copies"]) / (args.warmup + args.steps)}}
+    if aux_info is not None:
+        line["config"]["workload"] += " (prefetch routers distilled and confidence models refitted on this GPU)"
+        line["trained_auxiliary"] = dict(aux_info, overlap_vs_P=st_all["hits_P"] / max(1, st_all["routed"]),
+                                         coverage=st_all["covered"] / max(1, st_all["tokens"]),
+                                         mean_delta_hat=st_all["sum_delta_hat"] / max(1, st_all["tokens"]),
+                                         mean_delta_star=st_all["sum_delta_star"] / max(1, st_all["tokens"]),
+                                         demand_copies_per_token=st_all["demand_copies"] / (args.warmup + args.steps))
     print(json.dumps(line), flush=True)
 
 

@@ -258,6 +258,19 @@ int apex_route_topk_static(const float* W_r_dev, const float* b_r_dev, const flo
 int apex_fit_cdf(const double* X_dev, const int32_t* dstar_dev, int T, int N, int k, int iters, double lr,
                  float* w_host, float* theta_host, void* stream, char* err, size_t err_len);
 
+/* Distils the prefetch router from the frozen router (Sec. IV-C, Eq. (10)): minimises the mean over the
+ * calibration tokens of KL(q_r || q_p), q_p = softmax(W_p h + b_p), by `iters` steps of full-batch Adam
+ * (0.9 / 0.999 / 1e-8, step lr) in fp64; sums in a fixed order (bit-reproducible).
+ *   H_dev [T][d] fp32 (device): the hidden states the prefetch router will see (before attention);
+ *   Qr_dev [T][N] fp32 (device): the router's distribution for the same tokens (after attention), e.g. the
+ *   alpha output of apex_route_topk.
+ *   W_host [N][d], b_host [N] (host, fp32): in: the starting point; out: the trained parameters, ready for
+ *   apex_set_prefetch_router.
+ * Context-free; allocates and frees its own scratch; synchronises `stream` before it returns.
+ * N <= APEX_MAX_EXPERTS.  Returns APEX_OK, APEX_EINVAL, APEX_ENOMEM or APEX_ECUDA. */
+int apex_distill_router(const float* H_dev, const float* Qr_dev, int T, int N, int d, int iters, double lr,
+                        float* W_host, float* b_host, void* stream, char* err, size_t err_len);
+
 /* ---- host-only slot planner (the state machine behind apex_prefetch / apex_moe_ffn) -------- */
 
 typedef struct apex_slots apex_slots;

@@ -76,6 +76,7 @@ SIGNATURES = {
     "apex_launch_count": (C.c_int64, [_P]),
     "apex_route_topk_static": (_I, [_P, _P, _P, _I, _I, _I, _I, _P, _P, _P, C.c_char_p, C.c_size_t]),
     "apex_fit_cdf": (_I, [_P, _P, _I, _I, _I, _I, C.c_double, _P, _P, _P, C.c_char_p, C.c_size_t]),
+    "apex_distill_router": (_I, [_P, _P, _I, _I, _I, _I, C.c_double, _P, _P, _P, C.c_char_p, C.c_size_t]),
     "apex_slots_create": (_P, [_I, _I, _I]),
     "apex_slots_destroy": (None, [_P]),
     "apex_slots_begin_step": (_I, [_P]),
@@ -308,6 +309,23 @@ def fit_cdf(X_dev, dstar_dev, k, iters=600, lr=0.05, stream=None):
     if rc != APEX_OK:
         raise ApexError(rc, err.value.decode())
     return w, theta
+
+
+def distill_router(H_dev, Qr_dev, W0, b0, iters=200, lr=0.01, stream=None):
+    """apex_distill_router: H_dev [T][d], Qr_dev [T][N] fp32 CUDA tensors; W0 [N][d], b0 [N] the starting point.
+    Returns the trained (W [N][d], b [N]) as fp32 numpy arrays."""
+    lib = load_library()
+    T, d = H_dev.shape
+    N = Qr_dev.shape[1]
+    W = np.ascontiguousarray(W0, np.float32).copy()
+    b = np.ascontiguousarray(b0, np.float32).copy()
+    assert W.shape == (N, d) and b.shape == (N,)
+    err = C.create_string_buffer(256)
+    rc = lib.apex_distill_router(_ptr(H_dev), _ptr(Qr_dev), T, N, d, int(iters), float(lr), _ptr(W), _ptr(b),
+                                 _stream(stream), err, len(err))
+    if rc != APEX_OK:
+        raise ApexError(rc, err.value.decode())
+    return W, b
 
 
 class Slots:

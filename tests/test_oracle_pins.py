@@ -462,3 +462,65 @@ def test_cdf_fit_without_signal_returns_the_empirical_distribution():
     frac = (np.arange(N - k + 1)[None, :] >= dstar[:, None]).mean(0)
     z = theta.astype(np.float64) - float(X[0] @ w.astype(np.float64))
     np.testing.assert_allclose(1.0 / (1.0 + np.exp(-z[:-1])), frac[:-1], atol=2e-3)
+
+
+# ------------------------------------------------------------------ the CPU distillation of the prefetch router (Eq. (10))
+def _distill_problem(T, N, d, seed, noise=0.0):
+    rng = np.random.default_rng(seed)
+    W_true = rng.standard_normal((N, d)) / np.sqrt(d)
+    b_true = 0.3 * rng.standard_normal(N)
+    H = rng.standard_normal((T, d))
+    Hp = H + noise * rng.standard_normal((T, d))
+    Z = Hp @ W_true.T + b_true
+    Z -= Z.max(1, keepdims=True)
+    Qr = np.exp(Z)
+    Qr /= Qr.sum(1, keepdims=True)
+    return H, Qr, W_true, b_true
+
+
+def test_kl_loss_is_the_definition_and_vanishes_at_the_teacher():
+    from oracle import distill
+    H, Qr, W_true, b_true = _distill_problem(40, 5, 7, seed=1)
+    assert abs(distill.kl_loss(H, Qr, W_true, b_true)) < 1e-12
+    rng = np.random.default_rng(2)
+    W, b = rng.standard_normal((5, 7)), rng.standard_normal(5)
+    total = 0.0
+    for t in range(40):                                   # Eq. (10), term by term
+        z = W @ H[t] + b
+        qp = np.exp(z - z.max())
+        qp /= qp.sum()
+        total += sum(Qr[t, i] * math.log(Qr[t, i] / qp[i]) for i in range(5))
+    assert abs(distill.kl_loss(H, Qr, W, b) - total / 40) < 1e-12 and total > 0
+
+
+def test_distillation_first_step_follows_the_numerical_gradient():
+    # Adam's first step is -lr * sign(gradient): compare it with central differences of the loss.  A transposed
+    # operand, a wrong sign or a dropped bias term in the gradient would flip signs here.
+    from oracle import distill
+    H, Qr, _, _ = _distill_problem(60, 4, 6, seed=3, noise=0.3)
+    rng = np.random.default_rng(4)
+    W0, b0 = 0.5 * rng.standard_normal((4, 6)), 0.5 * rng.standard_normal(4)
+    lr = 1e-3
+    W1, b1 = distill.distill(H, Qr, W0, b0, iters=1, lr=lr)
+    eps = 1e-6
+    for (arr0, arr1) in ((W0, W1), (b0, b1)):
+        for idx in np.ndindex(arr0.shape):
+            def loss_at(delta):
+                Wc, bc = W0.copy(), b0.copy()
+                (Wc if arr0 is W0 else bc)[idx] += delta
+                return distill.kl_loss(H, Qr, Wc, bc)
+            g = (loss_at(eps) - loss_at(-eps)) / (2 * eps)
+            if abs(g) > 1e-6:
+                np.testing.assert_allclose(arr1[idx] - arr0[idx], -lr * np.sign(g), rtol=1e-3)
+
+
+def test_distillation_recovers_the_teacher_when_both_see_the_same_state():
+    from oracle import distill
+    H, Qr, W_true, b_true = _distill_problem(1500, 8, 24, seed=5)
+    W0, b0 = np.zeros((8, 24)), np.zeros(8)
+    l0 = distill.kl_loss(H, Qr, W0, b0)
+    W, b = distill.distill(H, Qr, W0, b0, iters=400, lr=0.02)
+    l1 = distill.kl_loss(H, Qr, W, b)
+    assert l1 < 0.02 * l0
+    Zs, Zt = H @ W.T + b, H @ W_true.T + b_true
+    assert (Zs.argmax(1) == Zt.argmax(1)).mean() > 0.97

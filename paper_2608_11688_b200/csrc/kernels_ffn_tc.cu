@@ -33,6 +33,7 @@
 #include <cuda_bf16.h>
 
 #include "apex_internal.hpp"
+#include "ptx.cuh"
 
 namespace apex {
 
@@ -44,50 +45,15 @@ constexpr int kTcThreads = (kProducerWarps + 1 + 4) * 32;  // producers, MMA + T
 constexpr int kKTile = 64;       // K elements per pipeline stage (128 bytes: one swizzle span)
 constexpr int kXRowsPerLoad = 8;    // rows per B-tile box: one 8-row swizzle atom, so a small group does not fetch rows it has no token for
 
-__device__ __forceinline__ uint32_t s32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-__device__ __forceinline__ unsigned long long gtimer() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
-__device__ __forceinline__ void mbar_init(uint64_t* b, uint32_t c) {
-  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(s32(b)), "r"(c) : "memory");
-}
-__device__ __forceinline__ void mbar_expect_tx(uint64_t* b, uint32_t bytes) {
-  asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(s32(b)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t* b) {
-  asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(s32(b)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try(uint64_t* b, uint32_t parity) {
-  uint32_t ok;
-  asm volatile("{\n.reg .pred p;\nmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\nselp.u32 %0,1,0,p;\n}"
-               : "=r"(ok)
-               : "r"(s32(b)), "r"(parity)
-               : "memory");
-  return ok != 0;
-}
-// Bounded: false when the limit ran out or another role gave up.
-__device__ __forceinline__ bool mbar_wait(uint64_t* b, uint32_t parity, const volatile int* abort_flag, long long limit_ns) {
-  if (mbar_try(b, parity)) return true;
-  const unsigned long long t0 = gtimer();
-  for (uint32_t it = 1;; ++it) {
-    if (mbar_try(b, parity)) return true;
-    if ((it & 255u) == 0u) {
-      if (*abort_flag) return false;
-      if ((long long)(gtimer() - t0) > limit_ns) return false;
-    }
-  }
-}
 __device__ __forceinline__ void tma_load_4d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, int c3, uint64_t* bar) {
   asm volatile(
-      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(s32(dst)),
-      "l"(map), "r"(s32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+      "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];" ::"r"(smem_u32(dst)),
+      "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
       : "memory");
 }
 __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, int c0, int c1, uint64_t* bar) {
-  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(s32(dst)),
-               "l"(map), "r"(s32(bar)), "r"(c0), "r"(c1)
+  asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(smem_u32(dst)),
+               "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
                : "memory");
 }
 // shared-memory matrix descriptor, 128-byte swizzle (layout type 2), version 1
@@ -117,7 +83,7 @@ __device__ __forceinline__ void umma(uint32_t tmem_d, uint64_t adesc, uint64_t b
                : "memory");
 }
 __device__ __forceinline__ void umma_commit(uint64_t* bar) {
-  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(s32(bar)) : "memory");
+  asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
 }
 __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
   asm volatile(
@@ -132,21 +98,13 @@ __device__ __forceinline__ void tmem_ld32(uint32_t taddr, uint32_t* r) {
 }
 __device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ uint32_t ld_acquire_sys_u32(const uint32_t* p) {
-  uint32_t v;
-  asm volatile("ld.acquire.sys.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
-  return v;
-}
 
 #ifdef APEX_TIMELINE
 __device__ unsigned long long g_tc_tl[2][148][128];
-#define TCTL(ph, i) do { if ((i) < 128) g_tc_tl[(ph) - 1][blockIdx.x][(i)] = gtimer(); } while (0)
+#define TCTL(ph, i) do { if ((i) < 128) g_tc_tl[(ph) - 1][blockIdx.x][(i)] = globaltimer_ns(); } while (0)
 #else
 #define TCTL(ph, i) do { } while (0)
 #endif
-
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 struct Group {
   int expert, pair_off, n_tok;
@@ -234,7 +192,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b2) : "memory");
   }
   if (warp == kMmaWarp) {
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(s32(&tmem_base_s)), "r"(512) : "memory");
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -301,16 +259,16 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         if (ok && lane == 0) {
           const uint32_t need = p.f.snap.need_gen[gr.expert];
           const uint32_t* flag = p.f.slot_ready + slot;
-          if ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
-            const unsigned long long t0 = gtimer();
-            while ((int32_t)(ld_acquire_sys_u32(flag) - need) < 0) {
-              if ((long long)(gtimer() - t0) > p.f.wait_limit_ns) {
+          if ((int32_t)(ld_acquire_sys(flag) - need) < 0) {
+            const unsigned long long t0 = globaltimer_ns();
+            while ((int32_t)(ld_acquire_sys(flag) - need) < 0) {
+              if ((long long)(globaltimer_ns() - t0) > p.f.wait_limit_ns) {
                 ok = false;
                 break;
               }
               __nanosleep(64);
             }
-            if (p.f.stats) atomicAdd(&p.f.stats->stall_ns, (gtimer() - t0) * (unsigned long long)gridDim.x / 4ull);
+            if (p.f.stats) atomicAdd(&p.f.stats->stall_ns, (globaltimer_ns() - t0) * (unsigned long long)gridDim.x / 4ull);
           }
           asm volatile("fence.proxy.async;" ::: "memory");
         }
@@ -371,7 +329,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
           }
           if (kt - kt_begin < 10) TCTL(PHASE, unit_no * 16 + 1 + kt - kt_begin);
           tc_fence_after();
-          const uint32_t a0 = s32(smem + (size_t)s * STAGE_BYTES);
+          const uint32_t a0 = smem_u32(smem + (size_t)s * STAGE_BYTES);
           const uint32_t b0 = a0 + A_BYTES;
 #pragma unroll
           for (int ks = 0; ks < kKTile / 16; ++ks) {

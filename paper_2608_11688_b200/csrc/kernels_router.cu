@@ -9,6 +9,7 @@
 #include <cooperative_groups.h>
 
 #include "apex_internal.hpp"
+#include "ptx.cuh"
 
 namespace cg = cooperative_groups;
 
@@ -108,8 +109,6 @@ __device__ __forceinline__ void select_token(const SelectParams& p, int b, int l
   }
 }
 
-__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
-__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 
 constexpr int kRouterMaxVec = 32;  // float4 per lane of one weight row: d <= 4096
 

@@ -127,14 +127,14 @@ def build_problem(cfg, device, fp8=False, fp4=False):
     return routers, cdf, store, shared
 
 
-def make_ctx(cfg, prob, C, max_batch=1, flags=0):
+def make_ctx(cfg, prob, C, max_batch=1, flags=0, link_gbs=0.0):
     from paper_2608_11688_b200 import binding
     routers, cdf, store, shared = prob
     fmt_flag = 0
     if store.dtype != __import__("torch").bfloat16:
         fmt_flag = binding.FLAG_FP8_EXPERTS if store.shape[-1] == 3 * cfg.d + 16 else binding.FLAG_FP4_EXPERTS
     a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C, L=cfg.L, I_shared=cfg.I_shared, max_batch=max_batch,
-                     flags=fmt_flag | flags)
+                     flags=fmt_flag | flags, link_gbs=link_gbs)
     for l in range(cfg.L):
         W_r, b_r, W_p, b_p = routers[l]
         a.set_router(l, W_r, b_r)
@@ -187,6 +187,41 @@ def train_auxiliary(cfg, prob, device, n_calib=8192, distill_iters=100, distill_
         new_routers.append((W_r, b_r, W_p2, b_p2))
         new_cdf.append((w, theta))
     return new_routers, new_cdf, {"distill_s": t_d, "fit_s": t_f, "calibration_tokens_per_layer": n_calib}
+
+
+POLICIES = (("no_prefetch", -1.0, None), ("static_k", 0.9, 0), ("static_k+4", 0.9, 4), ("static_k+8", 0.9, 8), ("apex", TAU, None))
+
+
+def run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, warmup, steps, link_gbs=0.0):
+    """Decode tokens under one prefetch policy of Sec. V-A (same ranking, different budgets); returns a dict."""
+    import torch
+    ap_ = make_ctx(cfg, prob, cfg.C, max_batch=B, link_gbs=link_gbs)
+    if delta is not None:      # w = 0 and a step in theta: delta_hat = delta for every token
+        nth = cfg.N - cfg.k + 1
+        th = np.where(np.arange(nth) >= delta, 50.0, -50.0).astype(np.float32)
+        for l in range(cfg.L):
+            ap_.set_cdf(l, np.zeros(cfg.N, np.float32), th)
+    T_ = h_dev.shape[0]
+    n_tok = warmup + steps
+    for t in range(warmup):
+        ap_.decode_token(h_dev[t % T_], hp_dev[t % T_], B, tau_p, "exact", y_dev)
+    torch.cuda.synchronize()
+    ap_.reset_stats()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(warmup, n_tok):
+        ap_.decode_token(h_dev[t % T_], hp_dev[t % T_], B, tau_p, "exact", y_dev)
+    e1.record()
+    torch.cuda.synchronize()
+    sp = ap_.get_stats()
+    sec = e0.elapsed_time(e1) * 1e-3
+    out = {"tokens_per_s": steps * B / sec, "ms_per_token": 1e3 * sec / (steps * B),
+           "copies_per_token": (sp["prefetch_copies"] + sp["demand_copies"]) / steps,
+           "demand_copies_per_token": sp["demand_copies"] / steps,
+           "overlap_vs_R": sp["hits_R"] / max(1, sp["routed"]),
+           "copied_gbs": sp["bytes_copied"] / sec / 1e9}
+    ap_.destroy()
+    return out
 
 
 def hidden_inputs(cfg, T, B, device):
@@ -342,6 +377,9 @@ def main():
     ap.add_argument("--no-spec", action="store_true", help="A/B: expert FFN without the speculative first fill")
     ap.add_argument("--fp8", action="store_true",
                     help="datatype study: e4m3 expert store with per-row scales (needs --ffn-only or --skip-extras)")
+    ap.add_argument("--link-sweep", action="store_true",
+                    help="study: per-token latency of the policies on a throttled host link (every expert copy padded to "
+                         "its duration at 8, 16 and 32 GB/s) and on the link as it is")
     ap.add_argument("--train-aux", action="store_true",
                     help="study: distil the prefetch routers and refit the confidence models on this GPU first "
                          "(a different predictor than the workload's: needs --skip-extras)")
@@ -395,6 +433,23 @@ def main():
     h_pin, hp_pin = h.pin_memory(), hp.pin_memory()
     y_dev = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32, device=dev)
     y_pin = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32).pin_memory()
+
+    if args.link_sweep:
+        import torch
+        table = {}
+        for bw in (8.0, 16.0, 32.0, 0.0):
+            row = {}
+            for name, tau_p, delta in (POLICIES[0], POLICIES[1], POLICIES[4]):
+                row[name] = run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, args.warmup, args.steps,
+                                       link_gbs=bw)
+            table["host link as it is" if bw == 0.0 else f"{bw:.0f} GB/s"] = row
+        a3 = make_ctx(cfg, prob, cfg.N, max_batch=B)
+        a3.warm_all()
+        sec_res = time_tokens(a3, h_dev, hp_dev, y_dev, B, "exact", args.warmup, args.steps)
+        a3.destroy()
+        print(json.dumps({"link_sweep": table, "all_resident_ms_per_token": 1e3 * sec_res / args.steps,
+                          "config": f"config{cfg.cfg_id}", "steps": args.steps, "tau": TAU}), flush=True)
+        return
 
     if args.ffn_only:
         a = make_ctx(cfg, prob, cfg.N, max_batch=B, flags=2 if args.no_spec else 0)
@@ -465,31 +520,8 @@ def main():
             # ---- policy baselines of Sec. V-A under the same harness (same ranking, different budgets)
             if args.policies:
                 pol = {}
-                n_tok = args.warmup + args.steps
-                for name, tau_p, delta in (("no_prefetch", -1.0, None), ("static_k", 0.9, 0), ("static_k+4", 0.9, 4),
-                                           ("static_k+8", 0.9, 8)):
-                    ap_ = make_ctx(cfg, prob, cfg.C, max_batch=B)
-                    if delta is not None:      # w = 0 and a step in theta: delta_hat = delta for every token
-                        nth = cfg.N - cfg.k + 1
-                        th = np.where(np.arange(nth) >= delta, 50.0, -50.0).astype(np.float32)
-                        for l in range(cfg.L):
-                            ap_.set_cdf(l, np.zeros(cfg.N, np.float32), th)
-                    T_ = h_dev.shape[0]
-                    for t in range(args.warmup):
-                        ap_.decode_token(h_dev[t % T_], hp_dev[t % T_], B, tau_p, "exact", y_dev)
-                    torch.cuda.synchronize()
-                    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-                    e0.record()
-                    for t in range(args.warmup, n_tok):
-                        ap_.decode_token(h_dev[t % T_], hp_dev[t % T_], B, tau_p, "exact", y_dev)
-                    e1.record()
-                    torch.cuda.synchronize()
-                    sp = ap_.get_stats()
-                    pol[name] = {"tokens_per_s": args.steps * B / (e0.elapsed_time(e1) * 1e-3),
-                                 "copies_per_token": (sp["prefetch_copies"] + sp["demand_copies"]) / n_tok,
-                                 "demand_copies_per_token": sp["demand_copies"] / n_tok,
-                                 "overlap_vs_R": sp["hits_R"] / max(1, sp["routed"])}
-                    ap_.destroy()
+                for name, tau_p, delta in POLICIES[:4]:
+                    pol[name] = run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, args.warmup, args.steps)
                 extras["policies"] = pol
             # ---- all experts resident (C = N): isolates the kernels from the host link
             a3 = make_ctx(cfg, prob, cfg.N, max_batch=B)

@@ -29,7 +29,7 @@ class ApexConfig(C.Structure):
     _fields_ = [("d", C.c_int32), ("N", C.c_int32), ("k", C.c_int32), ("I", C.c_int32), ("I_shared", C.c_int32),
                 ("C", C.c_int32), ("L", C.c_int32), ("max_batch", C.c_int32), ("norm_topk", C.c_int32),
                 ("cache_reuse", C.c_int32), ("ctx_len", C.c_int32), ("flags", C.c_int32),
-                ("wait_limit_ns", C.c_int64)]
+                ("wait_limit_ns", C.c_int64), ("link_gbs", C.c_double)]
 
 
 class ApexStepStats(C.Structure):
@@ -137,11 +137,11 @@ class Apex:
     """One context.  Methods mirror the C entry points one to one (apex_ prefix dropped)."""
 
     def __init__(self, *, d, N, k, I, C_slots, L=1, I_shared=0, max_batch=1, norm_topk=1, cache_reuse=1,
-                 ctx_len=1024, wait_limit_ns=0, flags=0):
+                 ctx_len=1024, wait_limit_ns=0, flags=0, link_gbs=0.0):
         self.lib = load_library()
         self.cfg = ApexConfig(d=d, N=N, k=k, I=I, I_shared=I_shared, C=C_slots, L=L, max_batch=max_batch,
                               norm_topk=norm_topk, cache_reuse=cache_reuse, ctx_len=ctx_len, flags=flags,
-                              wait_limit_ns=wait_limit_ns)
+                              wait_limit_ns=wait_limit_ns, link_gbs=float(link_gbs))
         h = C.c_void_p()
         rc = self.lib.apex_create(C.byref(self.cfg), C.byref(h))
         if rc != APEX_OK:

@@ -83,6 +83,43 @@ bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
   }
 }
 
+// Emulated link: measures, once, how long an expert copy from the registered store takes and what a padding
+// copy over the host link costs (latency and time per byte), with CUDA events on the copy stream.
+int calibrate_link(apex_ctx* ctx, uint8_t* dst, const uint8_t* src, cudaStream_t cs) {
+  cudaEvent_t e0, e1;
+  CU_TRY(ctx, cudaEventCreate(&e0));
+  CU_TRY(ctx, cudaEventCreate(&e1));
+  auto time_copy = [&](void* d, const void* s_, size_t n, cudaMemcpyKind kind, double* us) -> int {
+    float best = 1e30f;
+    for (int rep = 0; rep < 5; ++rep) {
+      CU_TRY(ctx, cudaEventRecord(e0, cs));
+      CU_TRY(ctx, cudaMemcpyAsync(d, s_, n, kind, cs));
+      CU_TRY(ctx, cudaEventRecord(e1, cs));
+      CU_TRY(ctx, cudaEventSynchronize(e1));
+      float ms = 0.f;
+      CU_TRY(ctx, cudaEventElapsedTime(&ms, e0, e1));
+      best = ms < best ? ms : best;
+    }
+    *us = (double)best * 1e3;
+    return APEX_OK;
+  };
+  CU_TRY(ctx, cudaStreamSynchronize(cs));
+  double t_small = 0.0, t_large = 0.0;
+  const size_t small = 64 * 1024, large = ctx->pad_bytes;
+  int r = time_copy(dst, src, ctx->expert_bytes, cudaMemcpyDefault, &ctx->real_copy_us);
+  if (r == APEX_OK) r = time_copy(ctx->pad_dst, ctx->pad_src, small, cudaMemcpyHostToDevice, &t_small);
+  if (r == APEX_OK) r = time_copy(ctx->pad_dst, ctx->pad_src, large, cudaMemcpyHostToDevice, &t_large);
+  cudaEventDestroy(e0);
+  cudaEventDestroy(e1);
+  if (r != APEX_OK) return r;
+  ctx->pad_us_per_byte = (t_large - t_small) / (double)(large - small);
+  ctx->pad_lat_us = t_small - (double)small * ctx->pad_us_per_byte;
+  if (!(ctx->pad_us_per_byte > 0.0)) return fail(ctx, APEX_ECUDA, "link calibration: padding copies took no time");
+  if (ctx->pad_lat_us < 0.0) ctx->pad_lat_us = 0.0;
+  ctx->link_calibrated = true;
+  return APEX_OK;
+}
+
 // One expert copy host store -> slot, followed by the slot-ready flag on the same stream.
 int issue_copy(apex_ctx* ctx, int layer, int e, int slot, cudaStream_t cs) {
   if (!ctx->store_base[layer]) return fail(ctx, APEX_ESTATE, "no expert store registered for this layer");
@@ -94,7 +131,24 @@ int issue_copy(apex_ctx* ctx, int layer, int e, int slot, cudaStream_t cs) {
   uint8_t* dst = ctx->d_cache + ((size_t)layer * C + slot) * ctx->expert_bytes;
   const uint8_t* src = ctx->store_base[layer] + (size_t)e * ctx->store_stride[layer];
   const uint32_t gen = ++ctx->slot_gen[layer][slot];
-  CU_TRY(ctx, cudaMemcpyAsync(dst, src, ctx->expert_bytes, cudaMemcpyHostToDevice, cs));
+  if (ctx->cfg.link_gbs > 0.0 && !ctx->link_calibrated) {
+    int r = calibrate_link(ctx, dst, src, cs);
+    if (r != APEX_OK) return r;
+  }
+  CU_TRY(ctx, cudaMemcpyAsync(dst, src, ctx->expert_bytes, cudaMemcpyDefault, cs));
+  if (ctx->cfg.link_gbs > 0.0) {
+    // the copy should have taken expert bytes / link_gbs: pad what is missing with a copy over the host link
+    const double target_us = (double)ctx->expert_bytes / (ctx->cfg.link_gbs * 1e3);
+    const double missing_us = target_us - ctx->real_copy_us - ctx->pad_lat_us;
+    double left_us = missing_us;
+    for (int guard = 0; left_us > 0.0 && guard < 64; ++guard) {  // as many padding copies as it takes
+      size_t pad = (size_t)(left_us / ctx->pad_us_per_byte);
+      pad = pad > ctx->pad_bytes ? ctx->pad_bytes : (pad & ~(size_t)255);
+      if (!pad) break;
+      CU_TRY(ctx, cudaMemcpyAsync(ctx->pad_dst, ctx->pad_src, pad, cudaMemcpyHostToDevice, cs));
+      left_us -= ctx->pad_lat_us + (double)pad * ctx->pad_us_per_byte;
+    }
+  }
   uint32_t* flag = ctx->d_slot_ready + (size_t)layer * C + slot;
   if (ctx->inject == 2) {
     ctx->inject = 0;
@@ -153,6 +207,7 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
       c.L < 1 || c.I < 1 || c.I_shared < 0 || c.max_batch < 1 || c.max_batch > APEX_MAX_BATCH || !ffn_shape_supported(c.d) ||
       c.ctx_len < 0)
     return APEX_EINVAL;
+  if (!(c.link_gbs >= 0.0)) return APEX_EINVAL;
   // the kernels index (token, expert, intermediate index) rows with 31 bits
   if ((long long)c.max_batch * (c.k + 1) * (long long)(c.I > c.I_shared ? c.I : c.I_shared) >= (1ll << 30)) return APEX_EINVAL;
   apex_ctx* ctx = new (std::nothrow) apex_ctx();
@@ -272,6 +327,13 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   ctx->gen_src_len = 1 << 16;
   CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->gen_src), ctx->gen_src_len * sizeof(uint32_t), cudaHostAllocPortable));
 
+  if (c.link_gbs > 0.0) {  // one emulated link: copies one after the other, each padded to its target duration
+    ctx->n_copy_streams = 1;
+    ctx->pad_bytes = ctx->expert_bytes > (4u << 20) ? ctx->expert_bytes : (size_t)(4u << 20);
+    CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->pad_src), ctx->pad_bytes, cudaHostAllocDefault));
+    memset(ctx->pad_src, 0, ctx->pad_bytes);
+    CR(cudaMalloc(reinterpret_cast<void**>(&ctx->pad_dst), ctx->pad_bytes));
+  }
   for (int i = 0; i < ctx->n_copy_streams; ++i) {
     CR(cudaStreamCreateWithFlags(&ctx->copy_streams[i], cudaStreamNonBlocking));
     ctx->cur_copy_streams[i] = ctx->copy_streams[i];
@@ -314,6 +376,8 @@ int apex_destroy(apex_ctx* ctx) {
   for (void* p : dev)
     if (p) cudaFree(p);
   if (ctx->mbox) cudaFreeHost(ctx->mbox);
+  if (ctx->pad_src) cudaFreeHost(ctx->pad_src);
+  if (ctx->pad_dst) cudaFree(ctx->pad_dst);
   if (ctx->gen_src) cudaFreeHost(ctx->gen_src);
   for (cudaStream_t cs : ctx->copy_streams)
     if (cs) cudaStreamDestroy(cs);

@@ -261,6 +261,13 @@ struct apex_ctx {
   std::vector<const uint8_t*> shared_dev;
   std::vector<std::vector<uint32_t>> slot_gen;  // [L][C] install count
   std::vector<std::vector<int32_t>> phys_expert;  // [L][C] whose bytes the slot holds (or is receiving)
+  // emulated link (cfg.link_gbs > 0): padding copies over the host link stretch every expert copy
+  uint8_t* pad_src = nullptr;    // pinned host scratch
+  uint8_t* pad_dst = nullptr;    // device scratch
+  size_t pad_bytes = 0;
+  bool link_calibrated = false;
+  double real_copy_us = 0.0;     // measured duration of one expert copy from the registered store
+  double pad_lat_us = 0.0, pad_us_per_byte = 0.0;  // measured: padding copy time = pad_lat_us + bytes * pad_us_per_byte
   uint32_t* withheld_flag = nullptr;  // test hook: a ready flag that was not written
   uint32_t withheld_gen = 0;
   cudaStream_t withheld_stream = nullptr;

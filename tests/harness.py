@@ -75,12 +75,13 @@ class Problem:
             self.shared.append(sh)
         torch.cuda.synchronize()
 
-    def make_ctx(self, *, C=None, max_batch=1, norm_topk=1, cache_reuse=1, wait_limit_ns=0, flags=0) -> binding.Apex:
+    def make_ctx(self, *, C=None, max_batch=1, norm_topk=1, cache_reuse=1, wait_limit_ns=0, flags=0, link_gbs=0.0) -> binding.Apex:
         cfg = self.cfg
         build.build()
         a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C or cfg.C, L=self.L, I_shared=cfg.I_shared,
                          max_batch=max_batch, norm_topk=norm_topk, cache_reuse=cache_reuse,
-                         wait_limit_ns=wait_limit_ns, flags=(binding.FLAG_FP4_EXPERTS if self.fp4 else binding.FLAG_FP8_EXPERTS if self.fp8 else 0) | flags)
+                         wait_limit_ns=wait_limit_ns, flags=(binding.FLAG_FP4_EXPERTS if self.fp4 else binding.FLAG_FP8_EXPERTS if self.fp8 else 0) | flags,
+                         link_gbs=link_gbs)
         for l in range(self.L):
             W_r, b_r, W_p, b_p = self.routers[l]
             a.set_router(l, W_r, b_r)

@@ -220,6 +220,34 @@ def test_speculation_switch_changes_nothing_but_time():
     np.testing.assert_allclose(ys[0], ys[1], rtol=0, atol=2e-6 * float(np.abs(ys[1]).max()))
 
 
+# ------------------------------------------------------------------ throttled host link
+def test_throttled_link_gives_the_same_results_later():
+    import time
+    cfg = synth.tiny_config(d=1024, N=16, k=4, I=256, C=8, T=8, sigma_p=1.0, cfg_id=320)     # 1.5 MiB experts
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    out = []
+    for gbs in (0.0, 2.0):
+        apex = prob.make_ctx(link_gbs=gbs)
+        try:
+            t0 = time.perf_counter()
+            rep = hz.run_lockstep(prob, apex, mode="exact", tau=0.7, T=cfg.T)
+            torch.cuda.synchronize()
+            out.append((rep, apex.get_stats(), time.perf_counter() - t0))
+        finally:
+            apex.destroy()
+    (r0, s0, _), (r1, s1, _) = out
+    assert r0.n_prefetch_copies == r1.n_prefetch_copies and r0.n_demand_copies == r1.n_demand_copies
+    assert s0["bytes_copied"] == s1["bytes_copied"] and s1["timeouts"] == 0
+    # at 2 GB/s every copy of 1.5 MiB takes about 0.8 ms: the copy stream alone needs that long
+    assert s1["bytes_copied"] / 2e9 > 0.02
+
+
+def test_negative_link_bandwidth_is_refused():
+    with pytest.raises(binding.ApexError):
+        binding.Apex(d=256, N=8, k=2, I=8, C_slots=4, link_gbs=-1.0)
+
+
 # ------------------------------------------------------------------ the paper-shaped configs
 def test_config0_full():
     cfg = synth.CONFIGS[0]

@@ -24,8 +24,7 @@
  *     d <= 4096, 1 <= B <= max_batch <= 256, k <= C <= N.
  *   - A context is not thread-safe; use one host thread per context.
  *
- * Expert store layout (pinned host memory, or device memory when the far tier is emulated inside HBM):
- * expert e of a layer starts at base + e*stride and holds
+ * Expert store layout (host, pinned): expert e of a layer starts at base + e*stride and holds
  *   [I][3][d] bf16:  for each intermediate index i the three rows gate_i, up_i, downT_i,
  * where downT_i[j] = W_down[j][i] (the down projection transposed), so that index i owns one
  * contiguous block of 3*d values.  apex_pack_expert() converts from the usual
@@ -92,8 +91,8 @@ typedef struct apex_config {
   int64_t wait_limit_ns; /* bound of every host- and device-side wait; 0 = 2 s */
   double link_gbs;       /* 0: expert copies run at the speed of the link they cross.  > 0: every expert copy is
                             stretched to expert bytes / link_gbs (GB/s) by a padding copy over the host link behind it,
-                            on one copy stream -- a stand-in for a slower or, with the expert store registered in
-                            device memory, a faster far tier than this machine's host link (Sec. V-G bandwidth study) */
+                            on one copy stream -- a stand-in for a slower far tier than this machine's host link
+                            (Sec. V-G bandwidth study) */
 } apex_config;
 
 /* Counters of one layer, accumulated over layer-steps since the last reset. */

@@ -429,6 +429,14 @@ int apex_register_experts(apex_ctx* ctx, int layer, const void* base, size_t str
   CHECK_LAYER(ctx, layer);
   if (!base || stride < ctx->expert_bytes || (stride & 15) || ((uintptr_t)base & 15))
     return fail(ctx, APEX_EINVAL, "expert store: null base, stride below 3*I*d*2 or not 16-byte aligned");
+  // Pinned host memory only.  Copies from it run on the copy engines beside the kernels that wait for them;
+  // a copy from pageable memory is staged and synchronous, and a device-to-device copy was seen not to make
+  // progress while the expert-FFN kernel waited for it.
+  cudaPointerAttributes attr{};
+  if (cudaPointerGetAttributes(&attr, base) != cudaSuccess || attr.type != cudaMemoryTypeHost) {
+    cudaGetLastError();
+    return fail(ctx, APEX_EINVAL, "expert store: the base must be pinned (page-locked) host memory");
+  }
   ctx->store_base[layer] = static_cast<const uint8_t*>(base);
   ctx->store_stride[layer] = stride;
   return APEX_OK;

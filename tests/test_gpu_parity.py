@@ -248,6 +248,20 @@ def test_negative_link_bandwidth_is_refused():
         binding.Apex(d=256, N=8, k=2, I=8, C_slots=4, link_gbs=-1.0)
 
 
+def test_expert_store_must_be_pinned_host_memory():
+    a = binding.Apex(d=256, N=8, k=2, I=8, C_slots=4)
+    try:
+        dev_store = torch.zeros((8, 8, 3, 256), dtype=torch.bfloat16, device="cuda")
+        with pytest.raises(binding.ApexError):
+            a.register_experts(0, dev_store)
+        pageable = torch.zeros((8, 8, 3, 256), dtype=torch.bfloat16)
+        with pytest.raises(binding.ApexError):
+            a.register_experts(0, pageable)
+        a.register_experts(0, pageable.pin_memory())
+    finally:
+        a.destroy()
+
+
 # ------------------------------------------------------------------ the paper-shaped configs
 def test_config0_full():
     cfg = synth.CONFIGS[0]

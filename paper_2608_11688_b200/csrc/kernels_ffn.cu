@@ -242,7 +242,7 @@ __device__ __forceinline__ int nth_set_bit64(unsigned long long m, int n) {
 // are issued before the first use).  Phase B: warp w owns experts w and w+32 and gathers the tokens
 // that execute them with ballots, so the pair list is sorted by (expert, token).  Shared-expert pairs
 // (expert id N) follow.
-constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;
+constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;  // instantiated for 1, 2, 4 and 8 tokens per warp
 
 #ifdef APEX_TIMELINE
 #define PTL(i) do { if (threadIdx.x == 0) g_timeline[1000 * 16 + (i)] = globaltimer_ns_raw(); } while (0)
@@ -250,6 +250,7 @@ constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;
 #define PTL(i) do { } while (0)
 #endif
 
+template <int TOK_PER_WARP>
 __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   __shared__ unsigned long long s_exec[APEX_MAX_BATCH];
   __shared__ float s_pgate[APEX_MAX_BATCH][APEX_MAX_TOPK];  // gate of the j-th executed expert of each token
@@ -259,14 +260,14 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   const int N = p.N, k = p.k, B = p.B;
   int my_subst = 0, my_hits = 0;
   PTL(0);
-  TokenLoads tls[kPlanMaxTokPerWarp];
+  TokenLoads tls[TOK_PER_WARP];
 #pragma unroll
-  for (int j = 0; j < kPlanMaxTokPerWarp; ++j) {
+  for (int j = 0; j < TOK_PER_WARP; ++j) {
     const int b = warp + j * nwarp;
     if (b < B) tls[j] = load_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode, lane);
   }
 #pragma unroll
-  for (int j = 0; j < kPlanMaxTokPerWarp; ++j) {
+  for (int j = 0; j < TOK_PER_WARP; ++j) {
     const int b = warp + j * nwarp;
     if (b >= B) break;
     const TokenLoads& tl = tls[j];
@@ -412,7 +413,13 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
 }
 
 cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s) {
-  ffn_plan_kernel<<<1, 1024, 0, s>>>(p);
+  // a small batch gets the instantiation with the short planning loop: the kernel runs once per layer-step on a
+  // single SM with a cold instruction cache, so its length in instructions shows
+  static_assert(kPlanMaxTokPerWarp == 8, "the dispatch below covers up to eight tokens per warp");
+  if (p.B <= 32) ffn_plan_kernel<1><<<1, 1024, 0, s>>>(p);
+  else if (p.B <= 64) ffn_plan_kernel<2><<<1, 1024, 0, s>>>(p);
+  else if (p.B <= 128) ffn_plan_kernel<4><<<1, 1024, 0, s>>>(p);
+  else ffn_plan_kernel<8><<<1, 1024, 0, s>>>(p);
   return cudaGetLastError();
 }
 

@@ -542,6 +542,8 @@ int predict_select_fused(apex_ctx* ctx, int layer, const float* h_dev, int B, fl
   ctx->pred_stream = cs;
   ctx->step[layer].predicted = true;
   ctx->step[layer].selected = true;
+  ctx->step[layer].sel_stream = cs;
+  ctx->step[layer].attn_stream = nullptr;
   ctx->host_stats[layer].layer_steps += 1;
   return APEX_OK;
 }
@@ -579,6 +581,8 @@ int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* 
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   st.selected = true;
+  st.sel_stream = (cudaStream_t)stream;
+  st.attn_stream = nullptr;
   return APEX_OK;
 }
 
@@ -645,6 +649,7 @@ int apex_attention_standin(apex_ctx* ctx, int layer, void* stream) {
   p.n_vec = ctx->attn_bytes / 16;
   p.sink = ctx->d_attn_sink;
   CU_TRY(ctx, launch_attention(p, ctx->n_sm, (cudaStream_t)stream));
+  ctx->step[layer].attn_stream = (cudaStream_t)stream;
   ctx->last_was_ffn = false;
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
@@ -677,6 +682,10 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   p.N = (int)N; p.d = (int)d; p.B = B; p.k = ctx->cfg.k; p.C = ctx->cfg.C;
   p.pi_pred = st.selected ? ctx->d_pi : nullptr;
   p.ncand_pred = st.selected ? ctx->d_ncand : nullptr;
+  // the prefetch stage's outputs may be read before this kernel's dependency wait when a whole kernel of this
+  // library (the attention stand-in of this layer-step) ran between the two on this same stream
+  p.pred_early = (st.selected && ctx->pred_stream == (cudaStream_t)stream && st.sel_stream == (cudaStream_t)stream &&
+                  st.attn_stream == (cudaStream_t)stream) ? 1 : 0;
   p.stats = ctx->d_stats + layer;
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
   ctx->last_was_ffn = false;

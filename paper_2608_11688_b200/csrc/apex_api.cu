@@ -702,11 +702,17 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
 
 namespace {
 
+constexpr long long kSpecDelayAfterGateNs = 1500;
+
 // Every launch of the streaming kernel gets its own row-ticket counter out of a ring of 64; the
 // launch also clears the counter that will be used 32 launches later.
 cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
   const uint32_t id = ctx->ffn_launch_id++;
   p.zero_early = (!ctx->last_was_ffn && ctx->last_stream == cs) ? 1 : 0;
+  // After the gate kernel the speculative first fill is held back until the gate has fetched its input (measured
+  // on the all-resident decode loop of config 1: 898 tokens/s without delay, 906 / 933 / 937 / 930 / 911 / 891 with
+  // 0.5 / 1 / 1.5 / 2 / 2.5 / 3.5 us, 902 without speculation); between two FFN launches there is nothing to spare.
+  p.spec_delay_ns = ctx->last_was_ffn ? 0 : kSpecDelayAfterGateNs;
   ctx->last_was_ffn = true;
   ctx->last_stream = cs;
   p.ticket = ctx->d_tickets + (id & 63u);

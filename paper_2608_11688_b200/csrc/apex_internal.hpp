@@ -143,6 +143,7 @@ struct FfnParams {
   int demand_in_kernel;         // 1: a routed expert without a slot is waited for inside the kernel
   int fmt;                      // storage format of the slots: 0 bf16, 1 e4m3 with per-row scales, 2 e2m1 with block scales
   int zero_early;               // 1: y may be zeroed before the dependency wait (the preceding kernel does not touch y)
+  long long spec_delay_ns;      // the speculative first fill starts this long after the CTA does
   const int32_t* spec;          // [k] predicted top-k of this layer-step (complete before the preceding kernel began), or null
   SlotSnapshot snap;
   size_t slot_stride;

@@ -569,6 +569,12 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   if (spec_on) {
     if (lane < k) s_pos[warp][lane] = spec_e;
     __syncwarp();
+    if (p.spec_delay_ns > 0) {
+      // When the preceding kernel is the (latency-bound) gate, flooding the memory system at once delays the
+      // gate's own few loads by as much as the speculation saves: hold the copies back for a moment.
+      const unsigned long long t0 = globaltimer_ns();
+      while ((long long)(globaltimer_ns() - t0) < p.spec_delay_ns) __nanosleep(200);
+    }
     set_geometry(k, k + (p.run_shared ? 1 : 0));
     const int fill = n_static < NSW ? n_static : NSW;
     if (lane < fill) {

@@ -14,6 +14,10 @@ using namespace apex;
 
 namespace {
 
+// Head starts, in ns, that a latency-bound router kernel gets over a bandwidth-hungry kernel launched right behind it
+// (measured; see the launch sites).
+constexpr long long kAttnDelayAfterPredictNs = 2500;
+
 typedef int (*WriteValue32Fn)(cudaStream_t, unsigned long long, uint32_t, unsigned int);
 
 int fail(apex_ctx* ctx, int code, const char* what, cudaError_t e = cudaSuccess) {
@@ -537,6 +541,7 @@ int predict_select_fused(apex_ctx* ctx, int layer, const float* h_dev, int B, fl
   p.fuse_select = 1;
   CU_TRY(ctx, launch_router(p, cs));
   ctx->last_was_ffn = false;
+  ctx->last_pred_layer = layer;
   ctx->last_stream = cs;
   ++ctx->launches;
   ctx->pred_stream = cs;
@@ -560,6 +565,7 @@ int apex_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, void* stre
   if (r != APEX_OK) return r;
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
   ctx->last_was_ffn = false;
+  ctx->last_pred_layer = layer;
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   ctx->pred_stream = (cudaStream_t)stream;
@@ -578,6 +584,7 @@ int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* 
   if (r != APEX_OK) return r;
   CU_TRY(ctx, launch_select(p, (cudaStream_t)stream));
   ctx->last_was_ffn = false;
+  ctx->last_pred_layer = layer;
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   st.selected = true;
@@ -648,9 +655,20 @@ int apex_attention_standin(apex_ctx* ctx, int layer, void* stream) {
   p.buf = reinterpret_cast<const uint4*>(ctx->d_attn + (size_t)(layer % ctx->attn_layers) * ctx->attn_bytes);
   p.n_vec = ctx->attn_bytes / 16;
   p.sink = ctx->d_attn_sink;
+  // The attention block of a layer reads the layer's input, not the prefetch router's output: when the kernel
+  // just before it on this stream is this layer-step's prefetch stage, the two may run side by side (Sec. IV-A:
+  // prediction and prefetch are hidden under attention).  Anything else in front of it is waited for first.
+  p.wait_first = (ctx->last_stream == (cudaStream_t)stream && ctx->last_pred_layer == layer) ? 0 : 1;
+  // It starts streaming a little after the prefetch router, whose few loads would otherwise queue behind its own
+  // (all-resident decode loop of config 1: 935 tokens/s one after the other; side by side 973 / 977 / 989 / 994 / 988 /
+  // 958 / 918 with a head start of 0 / 1 / 1.5 / 2.5 / 3.5 / 4.5 / 6 us for the router).
+  p.delay_ns = kAttnDelayAfterPredictNs;
   CU_TRY(ctx, launch_attention(p, ctx->n_sm, (cudaStream_t)stream));
-  ctx->step[layer].attn_stream = (cudaStream_t)stream;
+  // (only an attention kernel that waited for the prefetch stage before anything else lets the gate read that
+  // stage's outputs ahead of its own dependency wait)
+  ctx->step[layer].attn_stream = p.wait_first ? (cudaStream_t)stream : nullptr;
   ctx->last_was_ffn = false;
+  ctx->last_pred_layer = -1;
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   return APEX_OK;
@@ -689,6 +707,7 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   p.stats = ctx->d_stats + layer;
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
   ctx->last_was_ffn = false;
+  ctx->last_pred_layer = -1;
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   st.routed = true;
@@ -714,6 +733,7 @@ cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
   // 0.5 / 1 / 1.5 / 2 / 2.5 / 3.5 us, 902 without speculation); between two FFN launches there is nothing to spare.
   p.spec_delay_ns = ctx->last_was_ffn ? 0 : kSpecDelayAfterGateNs;
   ctx->last_was_ffn = true;
+  ctx->last_pred_layer = -1;
   ctx->last_stream = cs;
   p.ticket = ctx->d_tickets + (id & 63u);
   p.ticket_reset = ctx->d_tickets + ((id + 32u) & 63u);
@@ -725,6 +745,7 @@ cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
 int launch_batched(apex_ctx* ctx, int layer, const FfnParams& p, cudaStream_t cs) {
   CU_TRY(ctx, launch_ffn_plan(p, cs));
   ctx->last_was_ffn = false;
+  ctx->last_pred_layer = -1;
   ctx->last_stream = cs;
   ++ctx->launches;
   if (ctx->tc_ok && p.B >= kTcMinBatch) {
@@ -738,6 +759,7 @@ int launch_batched(apex_ctx* ctx, int layer, const FfnParams& p, cudaStream_t cs
     t.layer_slot0 = layer * ctx->cfg.C;
     CU_TRY(ctx, launch_ffn_tc(t, ctx->tc_shared_maps[layer], ctx->n_sm, cs));
     ctx->last_was_ffn = true;
+    ctx->last_pred_layer = -1;
     ctx->launches += 3;
   } else {
     CU_TRY(ctx, launch_stream(ctx, p, cs));

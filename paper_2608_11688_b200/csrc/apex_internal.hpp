@@ -174,6 +174,8 @@ struct AttnParams {
   const uint4* buf;
   size_t n_vec;  // 16-byte vectors
   float* sink;
+  int wait_first;       // 1: wait for the preceding kernel before streaming; 0: stream beside it, wait before exiting
+  long long delay_ns;   // (wait_first = 0) start streaming this long after the CTA does
 };
 
 // launchers (kernels_*.cu).  Each returns the cudaError_t of the launch.
@@ -301,6 +303,7 @@ struct apex_ctx {
   cudaStream_t cur_copy_streams[kMaxCopyStreams] = {};  // in use: own, or the caller's (then all the same)
   cudaStream_t stream_of_slot(int slot) const { return cur_copy_streams[slot % n_copy_streams]; }
   cudaStream_t pred_stream = nullptr;   // stream of the last apex_predict
+  int last_pred_layer = -1;             // layer whose prefetch stage (router, budget selection) was the last launch, else -1
   cudaEvent_t ev_wave = nullptr, ev_in = nullptr;
   int inject = 0;
   int64_t launches = 0;

@@ -343,8 +343,12 @@ cudaError_t launch_select(const SelectParams& p, cudaStream_t s) {
 // xor of everything read is stored only if it equals one fixed pattern, which keeps the loads live.
 __global__ void __launch_bounds__(512) attention_standin_kernel(const AttnParams p) {
   SPAN_BEGIN();
-  pdl_wait();
+  if (p.wait_first) pdl_wait();
   pdl_launch_dependents();
+  if (!p.wait_first && p.delay_ns > 0) {
+    const unsigned long long t0 = globaltimer_ns();
+    while ((long long)(globaltimer_ns() - t0) < p.delay_ns) __nanosleep(200);
+  }
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   uint4 a = make_uint4(0, 0, 0, 0);
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < p.n_vec; i += stride) {
@@ -355,6 +359,9 @@ __global__ void __launch_bounds__(512) attention_standin_kernel(const AttnParams
     a.w ^= v.w;
   }
   if (a.x == 0x12345678u && a.y == 0x9abcdef0u && a.z == 0x0fedcba9u && a.w == 0x87654321u) p.sink[0] = 1.f;
+  // Streamed beside the preceding kernel: wait for it now, so that whoever waits for this kernel has, as
+  // always, everything before it on the stream complete.
+  if (!p.wait_first) pdl_wait();
   SPAN_END(3);
 }
 

@@ -540,3 +540,27 @@ def test_config1_long_run_counts_near_ties():
     assert rep.layer_steps == 1024
     assert rep.near_ties <= 2, rep          # expected about 1e-3 per run for 40 logits of unit spread
     print("config1 long run:", rep)
+
+
+def test_config1_long_run_stall_free_and_batched():
+    """The same lock-step walk in stall-free mode (1024 steps), and with 8 tokens per step through the batched path
+    (128 steps of a config-1 layer, execution sets of every token compared, FFN output on every 16th step)."""
+    cfg = synth.CONFIGS[1]
+    hz = _harness()
+    prob = hz.Problem(cfg, layers=1, cdf="fitted")
+    apex = prob.make_ctx()
+    try:
+        rep = hz.run_lockstep(prob, apex, mode="stall_free", tau=0.9, T=cfg.T, check_ffn_every=64)
+        st = apex.get_stats()
+    finally:
+        apex.destroy()
+    assert rep.layer_steps == 1024 and rep.near_ties <= 2 and rep.n_demand_copies == 0
+    assert st["substitutions"] == rep.n_subst > 0
+    apex = prob.make_ctx(max_batch=8)
+    try:
+        rep8 = hz.run_lockstep(prob, apex, mode="exact", tau=0.9, T=128, B=8, check_ffn_every=16, ffn_token_stride=3)
+    finally:
+        apex.destroy()
+    assert rep8.layer_steps == 128 and rep8.near_ties <= 2
+    print("config1 long run stall-free:", rep, "\nconfig1 long run B=8:", rep8)
+

@@ -370,8 +370,10 @@ def main():
                     help="profiling case: all experts resident, gate + expert FFN only, no copy in flight")
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (smaller captures)")
     ap.add_argument("--batch", type=int, default=1, help="tokens per decode step (config 4 sweeps 1, 8, 32, 128, 256)")
-    ap.add_argument("--policies", action="store_true",
-                    help="also time the baselines of the paper's comparison: no prefetch, static top-k, top-(k+4), top-(k+8)")
+    ap.add_argument("--no-policies", dest="policies", action="store_false",
+                    help="skip the baselines of the paper's comparison (no prefetch, static top-k, top-(k+4), top-(k+8))")
+    ap.add_argument("--policies", dest="policies", action="store_true", help="(default) time those baselines too")
+    ap.set_defaults(policies=True)
     ap.add_argument("--resident", action="store_true",
                     help="cache as large as the expert count, warmed up: no host-link copies (kernel launch lists)")
     ap.add_argument("--no-spec", action="store_true", help="A/B: expert FFN without the speculative first fill")

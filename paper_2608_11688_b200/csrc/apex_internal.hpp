@@ -154,7 +154,7 @@ struct FfnParams {
 constexpr int kMaxDevices = 64;  // per-device launch attributes are remembered for this many devices
 
 // Batched tensor-core path (kernels_ffn_tc.cu)
-constexpr int kTcMinBatch = 4;  // from this many tokens per step the tensor-core grouped GEMM runs (measured crossover)
+constexpr int kTcMinBatch = 2;  // from this many tokens per step the tensor-core grouped GEMM runs (it beats the per-pair kernel at every B > 1)
 struct TcParams {
   FfnParams f;
   const int32_t* grp;

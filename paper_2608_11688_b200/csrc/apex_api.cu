@@ -810,7 +810,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.snap = make_snapshot(ctx, layer);
   p.slot_stride = ctx->expert_bytes;
   p.wait_limit_ns = ctx->cfg.wait_limit_ns;
-  p.d = ctx->cfg.d; p.N = N; p.k = k; p.I = ctx->cfg.I; p.I_shared = ctx->cfg.I_shared; p.B = B;
+  p.d = ctx->cfg.d; p.N = N; p.k = k; p.I = ctx->cfg.I; p.I_shared = ctx->cfg.I_shared; p.B = B; p.C = C;
   p.mode = mode; p.norm_topk = ctx->cfg.norm_topk; p.accumulate = 0;
   p.run_shared = ctx->cfg.I_shared > 0 ? 1 : 0;
   p.post_exec = 1;

@@ -148,7 +148,7 @@ struct FfnParams {
   SlotSnapshot snap;
   size_t slot_stride;
   long long wait_limit_ns;
-  int d, N, k, I, I_shared, B, mode, norm_topk, accumulate, run_shared, post_exec;
+  int d, N, k, I, I_shared, B, C, mode, norm_topk, accumulate, run_shared, post_exec;
 };
 
 constexpr int kMaxDevices = 64;  // per-device launch attributes are remembered for this many devices

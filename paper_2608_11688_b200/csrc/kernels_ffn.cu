@@ -716,6 +716,10 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
             if (!ok) return;
           }
           slot = (int)(v & 0xffu);
+          if (slot >= p.C) {  // a published slot outside the cache: refuse rather than read out of range
+            ok = false;
+            return;
+          }
           dm_e = e;
           dm_slot = slot;
           asm volatile("fence.proxy.async;" ::: "memory");

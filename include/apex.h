@@ -161,7 +161,10 @@ int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* 
  * copies. */
 int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream);
 /* Streams the bytes of an attention block (4 d^2 + 2 ctx_len d bf16 values): the hiding window
- * of Eq. (12).  It does not produce h'. */
+ * of Eq. (12).  It does not produce h'.  An attention block reads the layer's input, not the prefetch
+ * stage's output: when apex_predict / apex_select_candidates of this layer are the calls just before it on
+ * the same stream, the kernel runs beside them and only waits for them before it exits (everything launched
+ * after it still finds all earlier work complete); behind anything else it waits first. */
 int apex_attention_standin(apex_ctx* ctx, int layer, void* stream);
 /* S4 (Sec. III-A; Alg. 1 line 3): z_r = W_r h' + b_r, idx_dev [B][k] = K_r in rank order,
  * alpha_dev [B][N] = softmax(z_r).  Both buffers must stay valid until apex_moe_ffn of the

@@ -20,6 +20,8 @@
 
 #include "apex_internal.hpp"
 #include "ptx.cuh"
+#include "timeline.cuh"
+#include "token_plan.cuh"
 
 namespace apex {
 
@@ -30,11 +32,6 @@ __device__ unsigned long long g_timeline[1024 * 16];
   do {                                                                                \
     g_timeline[blockIdx.x * 16 + (slot)] = (slot) == 0 ? globaltimer_ns_raw() : (unsigned long long)clock64(); \
   } while (0)
-__device__ __forceinline__ unsigned long long globaltimer_ns_raw() {
-  unsigned long long t;
-  asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-  return t;
-}
 #define TLG(slot) do { g_timeline[blockIdx.x * 16 + (slot)] = globaltimer_ns_raw(); } while (0)
 #else
 #define TL(slot) do { } while (0)
@@ -116,311 +113,6 @@ __device__ __forceinline__ void load8(const uint8_t* row, int idx8, float (&w)[8
 // scale of the 32-element block that holds elements 8*idx8 .. 8*idx8+7 (block-scaled format only)
 __device__ __forceinline__ float block_scale(const uint8_t* scales, int idx8) {
   return __uint_as_float((uint32_t)scales[idx8 >> 2] << 23);
-}
-
-__device__ __forceinline__ unsigned long long warp_max_u64(unsigned long long v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) {
-    const unsigned long long w = __shfl_xor_sync(0xffffffffu, v, o);
-    v = w > v ? w : v;
-  }
-  return v;
-}
-__device__ __forceinline__ float warp_sum(float v) {
-#pragma unroll
-  for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-  return v;
-}
-
-// ---------------------------------------------------------------- execution set of one token (S6)
-// One warp.  Lanes own experts lane and lane+32.  Exact mode: K~ = K_r.  Stall-free mode
-// (Algorithm 1 with K_p := resident set): keep K_r that is resident, replace the |M| missing ones by
-// the |M| best remaining resident experts.  "Best" is by router weight alpha = softmax(z_r); the
-// order of alpha is the order of the logits, so the comparison is done on z_r (value descending,
-// index ascending).  Gates: alpha_e / sum over K~ (norm_topk) or alpha_e.
-// Returns the execution mask; pos/gate describe this lane's experts.
-struct TokenPlan {
-  unsigned long long exec_mask;
-  unsigned long long kr_mask;
-  float g0, g1;  // gates of experts lane, lane+32 (0 if not executed)
-};
-
-struct TokenLoads {
-  int my_idx;          // idx[lane] for lane < k, else -1
-  float al0, al1;      // alpha of experts lane, lane+32
-  float z0, z1;        // logits of experts lane, lane+32 (stall-free mode only)
-};
-__device__ __forceinline__ TokenLoads load_token(const int32_t* __restrict__ idx, const float* __restrict__ z_r,
-                                                 const float* __restrict__ alpha, int N, int k, int mode, int lane) {
-  TokenLoads t;
-  const int e0 = lane, e1 = lane + 32;
-  t.my_idx = lane < k ? idx[lane] : -1;
-  t.al0 = e0 < N ? alpha[e0] : 0.f;
-  t.al1 = e1 < N ? alpha[e1] : 0.f;
-  t.z0 = t.z1 = 0.f;
-  if (mode == APEX_MODE_STALL_FREE) {
-    t.z0 = e0 < N ? z_r[e0] : 0.f;
-    t.z1 = e1 < N ? z_r[e1] : 0.f;
-  }
-  return t;
-}
-__device__ __forceinline__ TokenPlan plan_token(const TokenLoads& t, int mode, int norm_topk, unsigned long long resident,
-                                                int lane) {
-  const int e0 = lane, e1 = lane + 32;
-  const int my_idx = t.my_idx;
-  const float al0 = t.al0, al1 = t.al1, z0 = t.z0, z1 = t.z1;
-  unsigned lo = 0, hi = 0;
-  if (my_idx >= 0) {
-    if (my_idx < 32)
-      lo = 1u << my_idx;
-    else
-      hi = 1u << (my_idx - 32);
-  }
-  lo = __reduce_or_sync(0xffffffffu, lo);
-  hi = __reduce_or_sync(0xffffffffu, hi);
-  const unsigned long long kr = ((unsigned long long)hi << 32) | lo;
-  unsigned long long exec = kr;
-  if (mode == APEX_MODE_STALL_FREE && (kr & ~resident) != 0ull) {
-    const unsigned long long keep = kr & resident;
-    const int n_missing = __popcll(kr & ~resident);
-    const unsigned long long cand = resident & ~kr;
-    int r0 = 0, r1 = 0;
-    unsigned long long rest = cand;
-    while (rest) {
-      const int f = __ffsll((long long)rest) - 1;
-      rest &= rest - 1;
-      const float zf = __shfl_sync(0xffffffffu, f < 32 ? z0 : z1, f & 31);
-      r0 += (zf > z0 || (zf == z0 && f < e0)) ? 1 : 0;
-      r1 += (zf > z1 || (zf == z1 && f < e1)) ? 1 : 0;
-    }
-    const bool s0 = ((cand >> e0) & 1) && r0 < n_missing;
-    const bool s1 = ((cand >> e1) & 1) && r1 < n_missing;
-    const unsigned b0 = __ballot_sync(0xffffffffu, s0), b1 = __ballot_sync(0xffffffffu, s1);
-    exec = keep | (((unsigned long long)b1 << 32) | b0);
-  }
-  const bool x0 = (exec >> e0) & 1, x1 = (exec >> e1) & 1;
-  const float a0 = x0 ? al0 : 0.f, a1 = x1 ? al1 : 0.f;
-  float denom = 1.f;
-  if (norm_topk) denom = warp_sum(a0 + a1);
-  TokenPlan tp;
-  tp.exec_mask = exec;
-  tp.kr_mask = kr;
-  tp.g0 = a0 / denom;
-  tp.g1 = a1 / denom;
-  return tp;
-}
-
-// Writes the per-token outputs of the plan (ascending expert index).
-__device__ __forceinline__ void store_token_plan(const TokenPlan& tp, int lane, int k, int32_t* exec_idx, float* exec_gate,
-                                                 int32_t* mbox_exec) {
-  const int e0 = lane, e1 = lane + 32;
-  if ((tp.exec_mask >> e0) & 1) {
-    const int pos = __popcll(tp.exec_mask & ((1ull << e0) - 1ull));
-    if (pos < k) {
-      if (exec_idx) exec_idx[pos] = e0;
-      if (exec_gate) exec_gate[pos] = tp.g0;
-      if (mbox_exec) mbox_exec[pos] = e0;
-    }
-  }
-  if ((tp.exec_mask >> e1) & 1) {
-    const int pos = __popcll(tp.exec_mask & ((1ull << e1) - 1ull));
-    if (pos < k) {
-      if (exec_idx) exec_idx[pos] = e1;
-      if (exec_gate) exec_gate[pos] = tp.g1;
-      if (mbox_exec) mbox_exec[pos] = e1;
-    }
-  }
-}
-
-__device__ __forceinline__ int nth_set_bit64(unsigned long long m, int n) {
-  for (int i = 0; i < n; ++i) m &= m - 1;
-  return __ffsll((long long)m) - 1;
-}
-
-// ---------------------------------------------------------------- batched plan (B > 1)
-// One CTA of 32 warps.  Phase A: warp w plans tokens w, w+32, ... (all global loads of a warp's tokens
-// are issued before the first use).  Phase B: warp w owns experts w and w+32 and gathers the tokens
-// that execute them with ballots, so the pair list is sorted by (expert, token).  Shared-expert pairs
-// (expert id N) follow.
-constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;  // instantiated for 1, 2, 4 and 8 tokens per warp
-
-#ifdef APEX_TIMELINE
-#define PTL(i) do { if (threadIdx.x == 0) g_timeline[1000 * 16 + (i)] = globaltimer_ns_raw(); } while (0)
-#else
-#define PTL(i) do { } while (0)
-#endif
-
-template <int TOK_PER_WARP>
-__global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
-  __shared__ unsigned long long s_exec[APEX_MAX_BATCH];
-  __shared__ float s_pgate[APEX_MAX_BATCH][APEX_MAX_TOPK];  // gate of the j-th executed expert of each token
-  __shared__ int s_count[APEX_MAX_EXPERTS + 1];
-  __shared__ int s_off[APEX_MAX_EXPERTS + 2];
-  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
-  const int N = p.N, k = p.k, B = p.B;
-  int my_subst = 0, my_hits = 0;
-  PTL(0);
-  TokenLoads tls[TOK_PER_WARP];
-#pragma unroll
-  for (int j = 0; j < TOK_PER_WARP; ++j) {
-    const int b = warp + j * nwarp;
-    if (b < B) tls[j] = load_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode, lane);
-  }
-#pragma unroll
-  for (int j = 0; j < TOK_PER_WARP; ++j) {
-    const int b = warp + j * nwarp;
-    if (b >= B) break;
-    const TokenLoads& tl = tls[j];
-    const TokenPlan tp = plan_token(tl, p.mode, p.norm_topk, p.snap.resident_mask, lane);
-    store_token_plan(tp, lane, k, p.plan_exec_idx + (size_t)b * k, p.plan_exec_gate + (size_t)b * k, nullptr);
-    if (p.post_exec) {
-      const int e0 = lane, e1 = lane + 32;
-      if ((tp.exec_mask >> e0) & 1) {
-        const int pos = __popcll(tp.exec_mask & ((1ull << e0) - 1ull));
-        if (p.exec_idx) p.exec_idx[(size_t)b * k + pos] = e0;
-        if (p.exec_gate) p.exec_gate[(size_t)b * k + pos] = tp.g0;
-      }
-      if ((tp.exec_mask >> e1) & 1) {
-        const int pos = __popcll(tp.exec_mask & ((1ull << e1) - 1ull));
-        if (p.exec_idx) p.exec_idx[(size_t)b * k + pos] = e1;
-        if (p.exec_gate) p.exec_gate[(size_t)b * k + pos] = tp.g1;
-      }
-      my_subst += __popcll(tp.exec_mask & ~tp.kr_mask);
-      my_hits += __popcll(tp.kr_mask & p.snap.resident_mask);
-    }
-    if (lane == 0) s_exec[b] = tp.exec_mask;
-    {
-      const int e0 = lane, e1 = lane + 32;
-      if ((tp.exec_mask >> e0) & 1) {
-        const int pos = __popcll(tp.exec_mask & ((1ull << e0) - 1ull));
-        if (pos < APEX_MAX_TOPK) s_pgate[b][pos] = tp.g0;
-      }
-      if ((tp.exec_mask >> e1) & 1) {
-        const int pos = __popcll(tp.exec_mask & ((1ull << e1) - 1ull));
-        if (pos < APEX_MAX_TOPK) s_pgate[b][pos] = tp.g1;
-      }
-    }
-  }
-  if (p.post_exec && lane == 0 && my_subst && p.stats) atomicAdd(&p.stats->substitutions, (unsigned long long)my_subst);
-  if (p.post_exec && lane == 0 && my_hits && p.stats) atomicAdd(&p.stats->hits_R, (unsigned long long)my_hits);
-  __syncthreads();
-  PTL(1);
-  // ---- phase B, counts: warp w counts the tokens of experts w and w + 32
-  for (int e = warp; e < N; e += nwarp) {
-    int c = 0;
-    if ((p.run_mask >> e) & 1)
-      for (int b0 = 0; b0 < B; b0 += 32) {
-        const int b = b0 + lane;
-        c += __popc(__ballot_sync(0xffffffffu, b < B && ((s_exec[b] >> e) & 1)));
-      }
-    if (lane == 0) s_count[e] = c;
-  }
-  __syncthreads();
-  PTL(2);
-  if (warp == 0) {
-    // exclusive prefix over the experts (lane owns experts lane and lane + 32), then the group table
-    // of the tensor-core path: one group per executed expert, then the shared expert
-    const int c0 = lane < N ? s_count[lane] : 0, c1 = lane + 32 < N ? s_count[lane + 32] : 0;
-    int i0 = c0, i1 = c1;
-#pragma unroll
-    for (int o = 1; o < 32; o <<= 1) {
-      const int u0 = __shfl_up_sync(0xffffffffu, i0, o), u1 = __shfl_up_sync(0xffffffffu, i1, o);
-      if (lane >= o) {
-        i0 += u0;
-        i1 += u1;
-      }
-    }
-    const int tot0 = __shfl_sync(0xffffffffu, i0, 31), acc = tot0 + __shfl_sync(0xffffffffu, i1, 31);
-    const int off0 = i0 - c0, off1 = tot0 + i1 - c1;
-    if (lane < N) s_off[lane] = off0;
-    if (lane + 32 < N) s_off[lane + 32] = off1;
-    const unsigned g0m = __ballot_sync(0xffffffffu, c0 > 0), g1m = __ballot_sync(0xffffffffu, c1 > 0);
-    const int ng_routed = __popc(g0m) + __popc(g1m);
-    if (c0 > 0) {
-      const int gi = __popc(g0m & ((1u << lane) - 1u));
-      p.grp[4 + 3 * gi] = lane;
-      p.grp[5 + 3 * gi] = off0;
-      p.grp[6 + 3 * gi] = c0;
-    }
-    if (c1 > 0) {
-      const int gi = __popc(g0m) + __popc(g1m & ((1u << lane) - 1u));
-      p.grp[4 + 3 * gi] = lane + 32;
-      p.grp[5 + 3 * gi] = off1;
-      p.grp[6 + 3 * gi] = c1;
-    }
-    if (lane == 0) {
-      s_off[N] = acc;  // routed pairs
-      p.n_pairs[0] = acc + (p.run_shared ? B : 0);
-      p.grp[0] = ng_routed;
-      if (p.run_shared) {
-        p.grp[4 + 3 * ng_routed] = N;
-        p.grp[5 + 3 * ng_routed] = acc;
-        p.grp[6 + 3 * ng_routed] = B;
-      }
-      p.grp[1] = ng_routed + (p.run_shared ? 1 : 0);
-    }
-  }
-  __syncthreads();
-  PTL(3);
-  // ---- phase B, placement: token b of expert e goes to s_off[e] + (number of earlier tokens of e)
-  for (int e = warp; e < N; e += nwarp) {
-    if (s_count[e] == 0) continue;
-    int o = s_off[e];
-    for (int b0 = 0; b0 < B; b0 += 32) {
-      const int b = b0 + lane;
-      const bool has = b < B && ((s_exec[b] >> e) & 1);
-      const unsigned m = __ballot_sync(0xffffffffu, has);
-      if (has) {
-        const int at = o + __popc(m & ((1u << lane) - 1u));
-        const int pos = __popcll(s_exec[b] & ((1ull << e) - 1ull));
-        p.pair_tok[at] = b;
-        p.pair_expert[at] = e;
-        p.pair_gate[at] = s_pgate[b][pos];
-      }
-      o += __popc(m);
-    }
-  }
-  if (p.run_shared) {
-    const int base = s_off[N];
-    for (int b = threadIdx.x; b < B; b += blockDim.x) {
-      p.pair_tok[base + b] = b;
-      p.pair_expert[base + b] = N;
-      p.pair_gate[base + b] = 1.f;
-    }
-  }
-  PTL(4);
-  // The routed and the execution sets go to the host mailbox last, as whole lines from consecutive
-  // threads (a 4-byte store per lane and token from inside the planning loop cost 2 us per token).
-  if (p.post_exec) {
-    for (int t = threadIdx.x; t < B * k; t += blockDim.x) {
-      const int b = t / k, j = t - b * k;
-      const unsigned long long m = s_exec[b];
-      p.mbox_exec[t] = j < __popcll(m) ? nth_set_bit64(m, j) : -1;
-      p.mbox_kr[t] = p.idx[t];
-    }
-  }
-  if (p.post_exec) {
-    // the barrier orders every thread's mailbox stores before thread 0's system-scope fence
-    // (fences are cumulative), which orders them before the sequence number
-    __syncthreads();
-    PTL(5);
-    if (threadIdx.x == 0) {
-      __threadfence_system();
-      *p.mbox_seq = p.seq_value;
-    }
-  }
-  PTL(6);
-}
-
-cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s) {
-  // a small batch gets the instantiation with the short planning loop: the kernel runs once per layer-step on a
-  // single SM with a cold instruction cache, so its length in instructions shows
-  static_assert(kPlanMaxTokPerWarp == 8, "the dispatch below covers up to eight tokens per warp");
-  if (p.B <= 32) ffn_plan_kernel<1><<<1, 1024, 0, s>>>(p);
-  else if (p.B <= 64) ffn_plan_kernel<2><<<1, 1024, 0, s>>>(p);
-  else if (p.B <= 128) ffn_plan_kernel<4><<<1, 1024, 0, s>>>(p);
-  else ffn_plan_kernel<8><<<1, 1024, 0, s>>>(p);
-  return cudaGetLastError();
 }
 
 // ---------------------------------------------------------------- the streaming FFN kernel

@@ -1,91 +1,11 @@
-// C-ABI entry points: argument checks, the host side of the prefetch machinery (slot planning,
-// cudaMemcpyAsync on the copy stream, slot-ready flags) and kernel launches.  All arithmetic of the
-// path runs in the kernels of kernels_router.cu / kernels_ffn.cu.
-#include <chrono>
-#include <cmath>
-#include <cstdio>
-#include <cstdlib>
-#include <cstring>
-#include <new>
-
-#include "apex_internal.hpp"
+// C-ABI entry points, part 2: the layer-step -- the host side of the prefetch machinery (slot planning,
+// cudaMemcpyAsync on the copy streams, slot-ready flags, demand copies) and the kernel launches.  All arithmetic of
+// the path runs in the kernels.
+#include "apex_host.hpp"
 
 using namespace apex;
 
-namespace {
-
-// Head starts, in ns, that a latency-bound router kernel gets over a bandwidth-hungry kernel launched right behind it
-// (measured; see the launch sites).
-constexpr long long kAttnDelayAfterPredictNs = 2500;
-
-typedef int (*WriteValue32Fn)(cudaStream_t, unsigned long long, uint32_t, unsigned int);
-
-int fail(apex_ctx* ctx, int code, const char* what, cudaError_t e = cudaSuccess) {
-  if (ctx) {
-    char buf[512];
-    if (e != cudaSuccess)
-      snprintf(buf, sizeof buf, "%s: %s", what, cudaGetErrorString(e));
-    else
-      snprintf(buf, sizeof buf, "%s", what);
-    ctx->err = buf;
-  }
-  return code;
-}
-
-#define CU_TRY(ctx, expr)                                              \
-  do {                                                                 \
-    cudaError_t _e = (expr);                                           \
-    if (_e != cudaSuccess) return fail(ctx, APEX_ECUDA, #expr, _e);    \
-  } while (0)
-
-#define CHECK_CTX(ctx) \
-  if (!(ctx)) return APEX_EINVAL
-#define CHECK_LAYER(ctx, layer) \
-  if ((layer) < 0 || (layer) >= (ctx)->cfg.L) return fail(ctx, APEX_EINVAL, "layer out of range")
-
-template <typename T>
-cudaError_t dev_alloc(T** p, size_t n) {
-  return cudaMalloc(reinterpret_cast<void**>(p), n * sizeof(T) > 0 ? n * sizeof(T) : 16);
-}
-
-MailboxHeader* mhdr(apex_ctx* ctx) { return reinterpret_cast<MailboxHeader*>(ctx->mbox); }
-int32_t* mbox_i32(apex_ctx* ctx, size_t off) { return reinterpret_cast<int32_t*>(ctx->mbox + off); }
-volatile uint32_t* mbox_sel_rec(apex_ctx* ctx) { return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_sel_rec); }
-volatile uint32_t* mbox_exec_seq(apex_ctx* ctx, int l) {
-  return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_exec_seq) + l;
-}
-int32_t* mbox_kr(apex_ctx* ctx, int l) { return mbox_i32(ctx, ctx->ml.off_kr + (size_t)l * ctx->ml.kr_stride); }
-int32_t* mbox_exec(apex_ctx* ctx, int l) { return mbox_i32(ctx, ctx->ml.off_exec + (size_t)l * ctx->ml.kr_stride); }
-
-// A 32-bit word written in stream order (after everything queued before it on that stream).
-int stream_write32(apex_ctx* ctx, cudaStream_t cs, uint32_t* dev, uint32_t value) {
-  if (ctx->fn_write_value32) {
-    int r = reinterpret_cast<WriteValue32Fn>(ctx->fn_write_value32)(cs, (unsigned long long)(uintptr_t)dev, value, 0);
-    if (r != 0) return fail(ctx, APEX_ECUDA, "cuStreamWriteValue32 failed");
-    return APEX_OK;
-  }
-  uint32_t* srcv = ctx->gen_src + (ctx->gen_src_pos++ % ctx->gen_src_len);
-  *srcv = value;
-  CU_TRY(ctx, cudaMemcpyAsync(dev, srcv, sizeof(uint32_t), cudaMemcpyHostToDevice, cs));
-  return APEX_OK;
-}
-
-// Bounded host wait for a mailbox sequence number.
-bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
-  if ((int32_t)(*p - want) >= 0) return true;
-  const auto t0 = std::chrono::steady_clock::now();
-  const int64_t limit = ctx->cfg.wait_limit_ns * 2 + 1000000000ll;  // the device side gives up first
-  for (uint32_t it = 0;; ++it) {
-    if ((int32_t)(*p - want) >= 0) return true;
-    if ((it & 1023u) == 1023u) {
-      const int64_t ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
-      if (ns > limit) return false;
-    }
-#if defined(__x86_64__)
-    __builtin_ia32_pause();
-#endif
-  }
-}
+namespace apex {
 
 // Emulated link: measures, once, how long an expert copy from the registered store takes and what a padding
 // copy over the host link costs (latency and time per byte), with CUDA events on the copy stream.
@@ -199,288 +119,13 @@ int check_device_status(apex_ctx* ctx) {
   return APEX_OK;
 }
 
-}  // namespace
-
-extern "C" {
-
-int apex_create(const apex_config* cfg, apex_ctx** out) {
-  if (!cfg || !out) return APEX_EINVAL;
-  *out = nullptr;
-  const apex_config& c = *cfg;
-  if (c.N < 1 || c.N > APEX_MAX_EXPERTS || c.k < 1 || c.k > APEX_MAX_TOPK || c.k > c.N || c.C < c.k || c.C > c.N ||
-      c.L < 1 || c.I < 1 || c.I_shared < 0 || c.max_batch < 1 || c.max_batch > APEX_MAX_BATCH || !ffn_shape_supported(c.d) ||
-      c.ctx_len < 0)
-    return APEX_EINVAL;
-  if (!(c.link_gbs >= 0.0)) return APEX_EINVAL;
-  // the kernels index (token, expert, intermediate index) rows with 31 bits
-  if ((long long)c.max_batch * (c.k + 1) * (long long)(c.I > c.I_shared ? c.I : c.I_shared) >= (1ll << 30)) return APEX_EINVAL;
-  apex_ctx* ctx = new (std::nothrow) apex_ctx();
-  if (!ctx) return APEX_ENOMEM;
-  ctx->cfg = c;
-  if (ctx->cfg.wait_limit_ns <= 0) ctx->cfg.wait_limit_ns = 2000000000ll;
-  if (ctx->cfg.ctx_len == 0) ctx->cfg.ctx_len = 1024;
-  const size_t L = c.L, N = c.N, C = c.C, d = c.d, MB = c.max_batch, k = c.k;
-  const bool fp8 = (c.flags & APEX_FLAG_FP8_EXPERTS) != 0, fp4 = (c.flags & APEX_FLAG_FP4_EXPERTS) != 0;
-  if ((fp8 && fp4) || ((fp8 || fp4) && !ffn_quantised_shape_supported(c.d))) {
-    delete ctx;
-    return APEX_EINVAL;
-  }
-  ctx->fmt = fp4 ? 2 : (fp8 ? 1 : 0);
-  const size_t row_bytes = ffn_row_bytes(ctx->fmt, c.d);
-  ctx->expert_bytes = row_bytes * (size_t)c.I;
-  ctx->shared_bytes = row_bytes * (size_t)c.I_shared;
-
-  auto bail = [&](int code, const char* what, cudaError_t e) {
-    fail(ctx, code, what, e);
-    fprintf(stderr, "apex_create: %s\n", ctx->err.c_str());
-    apex_destroy(ctx);
-    return code;
-  };
-#define CR(expr)                                                                  \
-  do {                                                                            \
-    cudaError_t _e = (expr);                                                      \
-    if (_e != cudaSuccess)                                                        \
-      return bail(_e == cudaErrorMemoryAllocation ? APEX_ENOMEM : APEX_ECUDA, #expr, _e); \
-  } while (0)
-
-  CR(cudaGetDevice(&ctx->device));
-  CR(cudaDeviceGetAttribute(&ctx->n_sm, cudaDevAttrMultiProcessorCount, ctx->device));
-  CR(dev_alloc(&ctx->d_Wr, L * N * d));
-  CR(dev_alloc(&ctx->d_Wp, L * N * d));
-  CR(dev_alloc(&ctx->d_br, L * N));
-  CR(dev_alloc(&ctx->d_bp, L * N));
-  CR(dev_alloc(&ctx->d_w, L * N));
-  CR(dev_alloc(&ctx->d_theta, L * (N - k + 1)));
-  CR(cudaMemset(ctx->d_br, 0, L * N * sizeof(float)));
-  CR(cudaMemset(ctx->d_bp, 0, L * N * sizeof(float)));
-  CR(cudaMemset(ctx->d_w, 0, L * N * sizeof(float)));
-  CR(cudaMemset(ctx->d_theta, 0, L * (N - k + 1) * sizeof(float)));
-  ctx->has_br.assign(L, 0);
-  ctx->has_bp.assign(L, 0);
-  ctx->has_cdf.assign(L, 0);
-  CR(dev_alloc(&ctx->d_cache, L * C * ctx->expert_bytes));
-  CR(dev_alloc(&ctx->d_slot_ready, L * C));
-  CR(cudaMemset(ctx->d_slot_ready, 0, L * C * sizeof(uint32_t)));
-  CR(dev_alloc(&ctx->d_zp, MB * N));
-  CR(dev_alloc(&ctx->d_qp, MB * N));
-  CR(dev_alloc(&ctx->d_zr, L * MB * N));
-  CR(dev_alloc(&ctx->d_demand, L * N));
-  CR(cudaMemset(ctx->d_demand, 0, L * N * sizeof(uint32_t)));
-  CR(dev_alloc(&ctx->d_pi, MB * N));
-  CR(dev_alloc(&ctx->d_ncand, MB));
-  CR(dev_alloc(&ctx->d_stats, L));
-  CR(cudaMemset(ctx->d_stats, 0, L * sizeof(DevStats)));
-  CR(dev_alloc(&ctx->d_tickets, 64));
-  CR(cudaMemset(ctx->d_tickets, 0, 64 * sizeof(unsigned int)));
-  CR(dev_alloc(&ctx->d_spec, L * APEX_MAX_TOPK));
-  CR(cudaMemset(ctx->d_spec, 0xff, L * APEX_MAX_TOPK * sizeof(int32_t)));
-  CR(dev_alloc(&ctx->d_counters, 2));
-  CR(cudaMemset(ctx->d_counters, 0, 2 * sizeof(unsigned long long)));
-  const size_t max_pairs = MB * (k + 1);
-  CR(dev_alloc(&ctx->d_plan_exec_idx, MB * k));
-  CR(dev_alloc(&ctx->d_plan_exec_gate, MB * k));
-  CR(dev_alloc(&ctx->d_pair_tok, max_pairs));
-  CR(dev_alloc(&ctx->d_pair_gate, max_pairs));
-  CR(dev_alloc(&ctx->d_pair_expert, max_pairs));
-  CR(dev_alloc(&ctx->d_n_pairs, 4));
-  CR(dev_alloc(&ctx->d_grp, 4 + 3 * (N + 1)));
-  CR(dev_alloc(&ctx->d_cand, MB * C));
-  CR(dev_alloc(&ctx->d_idx, L * MB * k));
-  CR(dev_alloc(&ctx->d_exec_idx, MB * k));
-  CR(dev_alloc(&ctx->d_alpha, L * MB * N));
-  CR(dev_alloc(&ctx->d_exec_gate, MB * k));
-  CR(dev_alloc(&ctx->d_cand_ncand, MB));
-  // batched tensor-core path: scratch and tensor maps (only for contexts that will see large batches)
-  if (MB >= kTcMinBatch && ctx->fmt == 0 && tc_shape_supported(c.d, c.I, c.I_shared)) {
-    const size_t rows = max_pairs + 256;
-    const size_t i_max = (size_t)(c.I > c.I_shared ? c.I : c.I_shared);
-    ctx->act_stride = (int)i_max;
-    CR(dev_alloc(&ctx->d_xg, rows * d));
-    ctx->act_plane = rows * i_max;
-    CR(dev_alloc(&ctx->d_act, 2 * rows * i_max));
-    CR(cudaMemset(ctx->d_xg, 0, rows * d * 2));
-    CR(cudaMemset(ctx->d_act, 0, 2 * rows * i_max * 2));
-    ctx->tc_ok = tc_make_weight_map(ctx->tc_maps.w_gateup, ctx->d_cache, c.d, c.I, L * C, ctx->expert_bytes, 128) &&
-                 tc_make_weight_map(ctx->tc_maps.w_down, ctx->d_cache, c.d, c.I, L * C, ctx->expert_bytes, 64) &&
-                 tc_make_rows_map(ctx->tc_maps.xg, ctx->d_xg, c.d, rows, d) &&
-                 tc_make_rows_map(ctx->tc_maps.act, ctx->d_act, (int)i_max, rows, i_max) &&
-                 tc_make_rows_map(ctx->tc_maps.act_lo, ctx->d_act + ctx->act_plane, (int)i_max, rows, i_max);
-    ctx->tc_shared_maps.assign(L, ctx->tc_maps);
-  }
-  ctx->attn_bytes = (4 * d * d + 2 * (size_t)ctx->cfg.ctx_len * d) * 2;
-  ctx->attn_layers = L < 8 ? L : 8;
-  CR(dev_alloc(&ctx->d_attn, ctx->attn_bytes * ctx->attn_layers));
-  CR(cudaMemset(ctx->d_attn, 0, ctx->attn_bytes * ctx->attn_layers));
-  CR(dev_alloc(&ctx->d_attn_sink, 4));
-
-  // mapped mailbox
-  MailboxLayout& ml = ctx->ml;
-  size_t off = sizeof(MailboxHeader);
-  ml.off_exec_seq = off;  off += L * sizeof(uint32_t);
-  off = (off + 15) & ~(size_t)15;
-  ml.off_sel_rec = off;   off += 16;
-  ml.off_ncand = off; off += MB * sizeof(int32_t);
-  ml.off_cand = off;  off += MB * C * sizeof(int32_t);
-  ml.kr_stride = MB * k * sizeof(int32_t);
-  ml.off_kr = off;    off += L * ml.kr_stride;
-  ml.off_exec = off;  off += L * ml.kr_stride;
-  ml.bytes = off;
-  ctx->exec_seq.assign(L, 0u);
-  CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->mbox), ml.bytes, cudaHostAllocMapped | cudaHostAllocPortable));
-  memset(ctx->mbox, 0, ml.bytes);
-  ctx->gen_src_len = 1 << 16;
-  CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->gen_src), ctx->gen_src_len * sizeof(uint32_t), cudaHostAllocPortable));
-
-  if (c.link_gbs > 0.0) {  // one emulated link: copies one after the other, each padded to its target duration
-    ctx->n_copy_streams = 1;
-    ctx->pad_bytes = ctx->expert_bytes > (4u << 20) ? ctx->expert_bytes : (size_t)(4u << 20);
-    CR(cudaHostAlloc(reinterpret_cast<void**>(&ctx->pad_src), ctx->pad_bytes, cudaHostAllocDefault));
-    memset(ctx->pad_src, 0, ctx->pad_bytes);
-    CR(cudaMalloc(reinterpret_cast<void**>(&ctx->pad_dst), ctx->pad_bytes));
-  }
-  for (int i = 0; i < ctx->n_copy_streams; ++i) {
-    CR(cudaStreamCreateWithFlags(&ctx->copy_streams[i], cudaStreamNonBlocking));
-    ctx->cur_copy_streams[i] = ctx->copy_streams[i];
-  }
-  CR(cudaEventCreateWithFlags(&ctx->ev_wave, cudaEventDisableTiming));
-  CR(cudaEventCreateWithFlags(&ctx->ev_in, cudaEventDisableTiming));
-#undef CR
-  {
-    void* fn = nullptr;
-    cudaDriverEntryPointQueryResult qr;
-    if (cudaGetDriverEntryPoint("cuStreamWriteValue32", &fn, cudaEnableDefault, &qr) == cudaSuccess &&
-        qr == cudaDriverEntryPointSuccess)
-      ctx->fn_write_value32 = fn;
-    cudaGetLastError();
-  }
-  ctx->tables.reserve(L);
-  for (size_t l = 0; l < L; ++l) ctx->tables.emplace_back((int)N, (int)C, c.cache_reuse != 0);
-  ctx->store_base.assign(L, nullptr);
-  ctx->store_stride.assign(L, 0);
-  ctx->shared_dev.assign(L, nullptr);
-  ctx->slot_gen.assign(L, std::vector<uint32_t>(C, 0u));
-  ctx->phys_expert.assign(L, std::vector<int32_t>(C, -1));
-  ctx->last_copies.assign(L, {});
-  ctx->host_stats.assign(L, apex_step_stats{});
-  ctx->step.assign(L, apex_ctx::StepState{});
-  ctx->ffn_params.assign(L, FfnParams{});
-  *out = ctx;
-  return APEX_OK;
-}
-
-int apex_destroy(apex_ctx* ctx) {
-  if (!ctx) return APEX_EINVAL;
-  cudaDeviceSynchronize();
-  cudaGetLastError();
-  void* dev[] = {ctx->d_Wr, ctx->d_br, ctx->d_Wp, ctx->d_bp, ctx->d_w, ctx->d_theta, ctx->d_cache, ctx->d_slot_ready, ctx->d_zp,
-                 ctx->d_qp, ctx->d_zr, ctx->d_demand, ctx->d_pi, ctx->d_ncand, ctx->d_stats, ctx->d_counters, ctx->d_tickets, ctx->d_spec, ctx->d_plan_exec_idx,
-                 ctx->d_plan_exec_gate, ctx->d_pair_tok, ctx->d_pair_gate, ctx->d_pair_expert, ctx->d_n_pairs, ctx->d_grp, ctx->d_xg, ctx->d_act, ctx->d_cand,
-                 ctx->d_idx, ctx->d_exec_idx, ctx->d_alpha, ctx->d_exec_gate, ctx->d_cand_ncand, ctx->d_attn, ctx->d_attn_sink,
-                 ctx->d_h_stage, ctx->d_hp_stage, ctx->d_y_stage};
-  for (void* p : dev)
-    if (p) cudaFree(p);
-  if (ctx->mbox) cudaFreeHost(ctx->mbox);
-  if (ctx->pad_src) cudaFreeHost(ctx->pad_src);
-  if (ctx->pad_dst) cudaFree(ctx->pad_dst);
-  if (ctx->gen_src) cudaFreeHost(ctx->gen_src);
-  for (cudaStream_t cs : ctx->copy_streams)
-    if (cs) cudaStreamDestroy(cs);
-  if (ctx->ev_wave) cudaEventDestroy(ctx->ev_wave);
-  if (ctx->ev_in) cudaEventDestroy(ctx->ev_in);
-  delete ctx;
-  return APEX_OK;
-}
-
-const char* apex_last_error(const apex_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
-
-int apex_set_router(apex_ctx* ctx, int layer, const float* W, const float* b) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  if (!W) return fail(ctx, APEX_EINVAL, "W_r is null");
-  const size_t N = ctx->cfg.N, d = ctx->cfg.d;
-  CU_TRY(ctx, cudaMemcpy(ctx->d_Wr + (size_t)layer * N * d, W, N * d * sizeof(float), cudaMemcpyHostToDevice));
-  if (b) CU_TRY(ctx, cudaMemcpy(ctx->d_br + (size_t)layer * N, b, N * sizeof(float), cudaMemcpyHostToDevice));
-  ctx->has_br[layer] = b ? 1 : 0;
-  return APEX_OK;
-}
-
-int apex_set_prefetch_router(apex_ctx* ctx, int layer, const float* W, const float* b) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  if (!W) return fail(ctx, APEX_EINVAL, "W_p is null");
-  const size_t N = ctx->cfg.N, d = ctx->cfg.d;
-  CU_TRY(ctx, cudaMemcpy(ctx->d_Wp + (size_t)layer * N * d, W, N * d * sizeof(float), cudaMemcpyHostToDevice));
-  if (b) CU_TRY(ctx, cudaMemcpy(ctx->d_bp + (size_t)layer * N, b, N * sizeof(float), cudaMemcpyHostToDevice));
-  ctx->has_bp[layer] = b ? 1 : 0;
-  return APEX_OK;
-}
-
-int apex_set_cdf(apex_ctx* ctx, int layer, const float* w, const float* theta) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  if (!w || !theta) return fail(ctx, APEX_EINVAL, "w or theta is null");
-  const size_t N = ctx->cfg.N, nth = ctx->cfg.N - ctx->cfg.k + 1;
-  for (size_t i = 1; i < nth; ++i)
-    if (!(theta[i] >= theta[i - 1])) return fail(ctx, APEX_EINVAL, "theta must be non-decreasing");
-  CU_TRY(ctx, cudaMemcpy(ctx->d_w + (size_t)layer * N, w, N * sizeof(float), cudaMemcpyHostToDevice));
-  CU_TRY(ctx, cudaMemcpy(ctx->d_theta + (size_t)layer * nth, theta, nth * sizeof(float), cudaMemcpyHostToDevice));
-  ctx->has_cdf[layer] = 1;
-  return APEX_OK;
-}
-
-int apex_register_experts(apex_ctx* ctx, int layer, const void* base, size_t stride) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  if (!base || stride < ctx->expert_bytes || (stride & 15) || ((uintptr_t)base & 15))
-    return fail(ctx, APEX_EINVAL, "expert store: null base, stride below 3*I*d*2 or not 16-byte aligned");
-  // Pinned host memory only.  Copies from it run on the copy engines beside the kernels that wait for them;
-  // a copy from pageable memory is staged and synchronous, and a device-to-device copy was seen not to make
-  // progress while the expert-FFN kernel waited for it.
-  cudaPointerAttributes attr{};
-  if (cudaPointerGetAttributes(&attr, base) != cudaSuccess || attr.type != cudaMemoryTypeHost) {
-    cudaGetLastError();
-    return fail(ctx, APEX_EINVAL, "expert store: the base must be pinned (page-locked) host memory");
-  }
-  ctx->store_base[layer] = static_cast<const uint8_t*>(base);
-  ctx->store_stride[layer] = stride;
-  return APEX_OK;
-}
-
-int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  if (ctx->cfg.I_shared <= 0) return fail(ctx, APEX_EINVAL, "the context was created with I_shared = 0");
-  if (!dev_weights || ((uintptr_t)dev_weights & 15)) return fail(ctx, APEX_EINVAL, "shared expert: null or unaligned");
-  ctx->shared_dev[layer] = static_cast<const uint8_t*>(dev_weights);
-  if (ctx->tc_ok) {
-    TcMaps& m = ctx->tc_shared_maps[layer];
-    if (!tc_make_weight_map(m.ws_gateup, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1, ctx->shared_bytes, 128) ||
-        !tc_make_weight_map(m.ws_down, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1, ctx->shared_bytes, 64))
-      return fail(ctx, APEX_ECUDA, "tensor map for the shared expert could not be encoded");
-  }
-  return APEX_OK;
-}
-
-int apex_pack_expert(const void* gate, const void* up, const void* down, int d, int I, void* dst) {
-  if (!gate || !up || !down || !dst || d < 1 || I < 1) return APEX_EINVAL;
-  const uint16_t* dn = static_cast<const uint16_t*>(down);
-  uint16_t* o = static_cast<uint16_t*>(dst);
-  const uint16_t* g = static_cast<const uint16_t*>(gate);
-  const uint16_t* u = static_cast<const uint16_t*>(up);
-  for (int i = 0; i < I; ++i) {
-    uint16_t* row = o + (size_t)i * 3 * d;
-    memcpy(row, g + (size_t)i * d, (size_t)d * 2);
-    memcpy(row + d, u + (size_t)i * d, (size_t)d * 2);
-    for (int j = 0; j < d; ++j) row[2 * (size_t)d + j] = dn[(size_t)j * I + i];
-  }
-  return APEX_OK;
-}
-
-// ---------------------------------------------------------------------------------------------
-
-}  // extern "C"
+}  // namespace apex
 
 namespace {
+
+// Head starts, in ns, that a latency-bound router kernel gets over a bandwidth-hungry kernel launched right behind it
+// (measured; see the launch sites).
+constexpr long long kAttnDelayAfterPredictNs = 2500;
 
 int begin_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, RouterParams* p) {
   if (!h_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_predict: bad h or B");
@@ -1013,179 +658,5 @@ int apex_decode_token_host(apex_ctx* ctx, const float* h_host, const float* hpos
 }
 
 // ---------------------------------------------------------------------------------------------
-
-static void add_dev_stats(apex_step_stats* o, const DevStats& s, int n_sm) {
-  o->tokens += (int64_t)s.tokens;
-  o->sum_delta_hat += (int64_t)s.sum_delta_hat;
-  o->sum_delta_star += (int64_t)s.sum_delta_star;
-  o->sum_ncand += (int64_t)s.sum_ncand;
-  o->capped += (int64_t)s.capped;
-  o->routed += (int64_t)s.routed;
-  o->hits_P += (int64_t)s.hits_P;
-  o->hits_R += (int64_t)s.hits_R;
-  o->covered += (int64_t)s.covered;
-  o->substitutions += (int64_t)s.substitutions;
-  o->stall_ns += (int64_t)(s.stall_ns / (unsigned long long)(n_sm > 0 ? n_sm : 1));
-  o->timeouts += (int64_t)s.timeouts;
-  o->near_full_prefetch += (int64_t)s.near_full;
-}
-
-int apex_get_stats(apex_ctx* ctx, int layer, apex_step_stats* out) {
-  CHECK_CTX(ctx);
-  if (!out || layer < -1 || layer >= ctx->cfg.L) return fail(ctx, APEX_EINVAL, "apex_get_stats: bad argument");
-  CU_TRY(ctx, cudaDeviceSynchronize());
-  std::vector<DevStats> ds(ctx->cfg.L);
-  CU_TRY(ctx, cudaMemcpy(ds.data(), ctx->d_stats, ds.size() * sizeof(DevStats), cudaMemcpyDeviceToHost));
-  memset(out, 0, sizeof *out);
-  for (int l = 0; l < ctx->cfg.L; ++l) {
-    if (layer >= 0 && l != layer) continue;
-    const apex_step_stats& h = ctx->host_stats[l];
-    out->layer_steps += h.layer_steps;
-    out->prefetch_copies += h.prefetch_copies;
-    out->demand_copies += h.demand_copies;
-    out->bytes_copied += h.bytes_copied;
-    out->extra_waves += h.extra_waves;
-    add_dev_stats(out, ds[l], ctx->n_sm);
-  }
-  return APEX_OK;
-}
-
-int apex_reset_stats(apex_ctx* ctx) {
-  CHECK_CTX(ctx);
-  CU_TRY(ctx, cudaDeviceSynchronize());
-  CU_TRY(ctx, cudaMemset(ctx->d_stats, 0, ctx->cfg.L * sizeof(DevStats)));
-  for (auto& h : ctx->host_stats) h = apex_step_stats{};
-  return APEX_OK;
-}
-
-int apex_read_prediction(apex_ctx* ctx, int B, float* z_p, float* q_p, int32_t* pi) {
-  CHECK_CTX(ctx);
-  if (B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "bad B");
-  CU_TRY(ctx, cudaStreamSynchronize(ctx->pred_stream));
-  const size_t n = (size_t)B * ctx->cfg.N;
-  if (z_p) CU_TRY(ctx, cudaMemcpy(z_p, ctx->d_zp, n * sizeof(float), cudaMemcpyDeviceToHost));
-  if (q_p) CU_TRY(ctx, cudaMemcpy(q_p, ctx->d_qp, n * sizeof(float), cudaMemcpyDeviceToHost));
-  if (pi) CU_TRY(ctx, cudaMemcpy(pi, ctx->d_pi, n * sizeof(int32_t), cudaMemcpyDeviceToHost));
-  return APEX_OK;
-}
-
-int apex_get_last_copies(apex_ctx* ctx, int layer, int32_t* expert, int32_t* slot, int32_t* n_prefetch, int32_t* n_demand) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  int np = 0, nd = 0, i = 0;
-  for (const auto& c : ctx->last_copies[layer]) {
-    if (expert) expert[i] = c.expert;
-    if (slot) slot[i] = c.slot;
-    ++i;
-    if (c.wave == 0) ++np; else ++nd;
-  }
-  if (n_prefetch) *n_prefetch = np;
-  if (n_demand) *n_demand = nd;
-  return APEX_OK;
-}
-
-int apex_get_slot_table(apex_ctx* ctx, int layer, int32_t* expert_slot, int64_t* slot_stamp, int64_t* clock) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  ctx->tables[layer].get(expert_slot, slot_stamp, clock);
-  return APEX_OK;
-}
-
-int apex_set_slot_table(apex_ctx* ctx, int layer, const int32_t* expert_slot, const int64_t* slot_stamp, int64_t clock) {
-  CHECK_CTX(ctx);
-  CHECK_LAYER(ctx, layer);
-  if (!expert_slot || !slot_stamp) return fail(ctx, APEX_EINVAL, "null table");
-  if (!ctx->tables[layer].set(expert_slot, slot_stamp, clock)) return fail(ctx, APEX_EINVAL, "inconsistent slot table");
-  // slots whose bytes belong to another expert are refilled
-  CU_TRY(ctx, cudaDeviceSynchronize());
-  for (int e = 0; e < ctx->cfg.N; ++e) {
-    const int s = expert_slot[e];
-    if (s >= 0 && ctx->phys_expert[layer][s] != e) {
-      int r = issue_copy(ctx, layer, e, s, ctx->stream_of_slot(s));
-      if (r != APEX_OK) return r;
-    }
-  }
-  return APEX_OK;
-}
-
-int apex_warm_all(apex_ctx* ctx) {
-  CHECK_CTX(ctx);
-  if (ctx->cfg.C != ctx->cfg.N) return fail(ctx, APEX_ESTATE, "apex_warm_all needs C == N");
-  std::vector<int32_t> es(ctx->cfg.N);
-  std::vector<int64_t> stamp(ctx->cfg.C, 0);
-  for (int e = 0; e < ctx->cfg.N; ++e) es[e] = e;
-  for (int l = 0; l < ctx->cfg.L; ++l) {
-    int r = apex_set_slot_table(ctx, l, es.data(), stamp.data(), ctx->tables[l].clock());
-    if (r != APEX_OK) return r;
-  }
-  for (int i = 0; i < ctx->n_copy_streams; ++i) CU_TRY(ctx, cudaStreamSynchronize(ctx->cur_copy_streams[i]));
-  return APEX_OK;
-}
-
-int apex_test_inject(apex_ctx* ctx, int what) {
-  CHECK_CTX(ctx);
-  if (what < 0 || what > 2) return fail(ctx, APEX_EINVAL, "unknown injection");
-  ctx->inject = what;
-  return APEX_OK;
-}
-
-int64_t apex_launch_count(const apex_ctx* ctx) { return ctx ? ctx->launches : -1; }
-
-// ---- host-only slot planner ---------------------------------------------------------------------
-
-struct apex_slots {
-  SlotTable t;
-  apex_slots(int N, int C, bool r) : t(N, C, r) {}
-};
-
-apex_slots* apex_slots_create(int N, int C, int cache_reuse) {
-  if (N < 1 || N > APEX_MAX_EXPERTS || C < 1 || C > N) return nullptr;
-  return new (std::nothrow) apex_slots(N, C, cache_reuse != 0);
-}
-void apex_slots_destroy(apex_slots* s) { delete s; }
-int apex_slots_begin_step(apex_slots* s) {
-  if (!s) return APEX_EINVAL;
-  s->t.begin_step();
-  return APEX_OK;
-}
-int apex_slots_prefetch(apex_slots* s, const int32_t* cand, const int32_t* ncand, int B, int stride, int32_t* copy_expert,
-                        int32_t* copy_slot, int32_t* n_copies) {
-  if (!s || !cand || !ncand || !n_copies || B < 1) return APEX_EINVAL;
-  std::vector<SlotCopy> cp;
-  if (!s->t.plan_prefetch(cand, ncand, B, stride, &cp)) return APEX_ESTATE;
-  for (size_t i = 0; i < cp.size(); ++i) {
-    if (copy_expert) copy_expert[i] = cp[i].expert;
-    if (copy_slot) copy_slot[i] = cp[i].slot;
-  }
-  *n_copies = (int32_t)cp.size();
-  return APEX_OK;
-}
-int apex_slots_demand(apex_slots* s, const int32_t* K_r, int B, int k, int32_t* copy_expert, int32_t* copy_slot,
-                      int32_t* wave_of_copy, int32_t* n_copies) {
-  if (!s || !K_r || !n_copies || B < 1 || k < 1) return APEX_EINVAL;
-  std::vector<SlotCopy> cp;
-  if (!s->t.plan_demand(K_r, B, k, &cp)) return APEX_ESTATE;
-  for (size_t i = 0; i < cp.size(); ++i) {
-    if (copy_expert) copy_expert[i] = cp[i].expert;
-    if (copy_slot) copy_slot[i] = cp[i].slot;
-    if (wave_of_copy) wave_of_copy[i] = cp[i].wave;
-  }
-  *n_copies = (int32_t)cp.size();
-  return APEX_OK;
-}
-int apex_slots_touch(apex_slots* s, const int32_t* experts, int n) {
-  if (!s || (!experts && n > 0)) return APEX_EINVAL;
-  for (int i = 0; i < n; ++i) s->t.touch(experts[i]);
-  return APEX_OK;
-}
-int apex_slots_get(const apex_slots* s, int32_t* expert_slot, int64_t* slot_stamp, int64_t* clock) {
-  if (!s) return APEX_EINVAL;
-  s->t.get(expert_slot, slot_stamp, clock);
-  return APEX_OK;
-}
-int apex_slots_set(apex_slots* s, const int32_t* expert_slot, const int64_t* slot_stamp, int64_t clock) {
-  if (!s || !expert_slot || !slot_stamp) return APEX_EINVAL;
-  return s->t.set(expert_slot, slot_stamp, clock) ? APEX_OK : APEX_EINVAL;
-}
 
 }  // extern "C"

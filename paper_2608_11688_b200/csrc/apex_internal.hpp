@@ -183,7 +183,7 @@ cudaError_t launch_router(const RouterParams& p, cudaStream_t s);
 cudaError_t launch_select(const SelectParams& p, cudaStream_t s);
 cudaError_t launch_attention(const AttnParams& p, int n_sm, cudaStream_t s);
 cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s);
-cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s);
+cudaError_t launch_ffn(const FfnParams& p, int n_ctas, cudaStream_t s);  // n_ctas: grid size, at most ffn_grid_ctas(SM count)
 int ffn_grid_ctas(int n_sm);  // CTAs of one streaming-kernel launch (each adds one to the zero counter)
 cudaError_t launch_ffn_tc(const TcParams& p, const TcMaps& m, int n_sm, cudaStream_t s);
 bool tc_make_weight_map(void* out, const void* base, int d, int I, size_t n_slots, size_t slot_bytes, int box_rows);

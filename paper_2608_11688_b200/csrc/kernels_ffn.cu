@@ -738,7 +738,7 @@ extern "C" int apex_debug_reset_spans() {
 #endif
 
 template <int NCH, int FMT>
-static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
+static cudaError_t launch_ffn_t(const FfnParams& p, int n_ctas, cudaStream_t s) {
   constexpr bool HR = NCH <= 8;
   constexpr uint32_t entry = fmt_entry_bytes(FMT, NCH * 256);
   constexpr int NS = ring_stages(entry);
@@ -752,7 +752,7 @@ static cudaError_t launch_ffn_t(const FfnParams& p, int n_sm, cudaStream_t s) {
     if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
   }
   cudaLaunchConfig_t cfg = {};
-  cfg.gridDim = dim3(n_sm * kCtasPerSm, 1, 1);
+  cfg.gridDim = dim3(n_ctas, 1, 1);
   cfg.blockDim = dim3(kFfnThreads, 1, 1);
   cfg.dynamicSmemBytes = smem;
   cfg.stream = s;
@@ -774,10 +774,10 @@ bool ffn_shape_supported(int d) {
 
 int ffn_grid_ctas(int n_sm) { return n_sm * kCtasPerSm; }
 
-cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s) {
+cudaError_t launch_ffn(const FfnParams& p, int n_ctas, cudaStream_t s) {
   if (p.fmt == kFmtE4m3 || p.fmt == kFmtMxfp4) {  // quantised stores: the widths of the paper-sized configs
 #define APEX_FFN_CASE(NCH_) \
-  case NCH_ * 256: return p.fmt == kFmtE4m3 ? launch_ffn_t<NCH_, kFmtE4m3>(p, n_sm, s) : launch_ffn_t<NCH_, kFmtMxfp4>(p, n_sm, s);
+  case NCH_ * 256: return p.fmt == kFmtE4m3 ? launch_ffn_t<NCH_, kFmtE4m3>(p, n_ctas, s) : launch_ffn_t<NCH_, kFmtMxfp4>(p, n_ctas, s);
     switch (p.d) {
       APEX_FFN_CASE(2)
       APEX_FFN_CASE(4)
@@ -789,14 +789,14 @@ cudaError_t launch_ffn(const FfnParams& p, int n_sm, cudaStream_t s) {
     return cudaErrorInvalidValue;
   }
   switch (p.d) {
-    case 256: return launch_ffn_t<1, kFmtBf16>(p, n_sm, s);
-    case 512: return launch_ffn_t<2, kFmtBf16>(p, n_sm, s);
-    case 768: return launch_ffn_t<3, kFmtBf16>(p, n_sm, s);
-    case 1024: return launch_ffn_t<4, kFmtBf16>(p, n_sm, s);
-    case 1536: return launch_ffn_t<6, kFmtBf16>(p, n_sm, s);
-    case 2048: return launch_ffn_t<8, kFmtBf16>(p, n_sm, s);
-    case 3072: return launch_ffn_t<12, kFmtBf16>(p, n_sm, s);
-    case 4096: return launch_ffn_t<16, kFmtBf16>(p, n_sm, s);
+    case 256: return launch_ffn_t<1, kFmtBf16>(p, n_ctas, s);
+    case 512: return launch_ffn_t<2, kFmtBf16>(p, n_ctas, s);
+    case 768: return launch_ffn_t<3, kFmtBf16>(p, n_ctas, s);
+    case 1024: return launch_ffn_t<4, kFmtBf16>(p, n_ctas, s);
+    case 1536: return launch_ffn_t<6, kFmtBf16>(p, n_ctas, s);
+    case 2048: return launch_ffn_t<8, kFmtBf16>(p, n_ctas, s);
+    case 3072: return launch_ffn_t<12, kFmtBf16>(p, n_ctas, s);
+    case 4096: return launch_ffn_t<16, kFmtBf16>(p, n_ctas, s);
   }
   return cudaErrorInvalidValue;
 }

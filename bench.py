@@ -33,8 +33,7 @@ TAU = 0.90
 
 # DRAM bytes per launch of the expert-FFN kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
 # the ncu capture summarised in profiles/ (same kernel, same per-launch shape).  None = not captured.
-NCU_TRAFFIC_BYTES = {1: 47_496_000}   # profiles/moe_ffn_stream_kernel_config1.md: mean of three launches (46.0, 42.1, 54.4 MB);
-#                                       37.8 MB of it is the executed experts, the rest speculative rows that were dropped
+NCU_TRAFFIC_BYTES = {1: 37_854_500}   # profiles/moe_ffn_stream_kernel_config1.md: 37.809 MB read + ~0.045 MB written
 
 
 def measured_peak():
@@ -376,7 +375,7 @@ def main():
     ap.set_defaults(policies=True)
     ap.add_argument("--resident", action="store_true",
                     help="cache as large as the expert count, warmed up: no host-link copies (kernel launch lists)")
-    ap.add_argument("--no-spec", action="store_true", help="A/B: expert FFN without the speculative first fill")
+    ap.add_argument("--spec", action="store_true", help="A/B: expert FFN with the speculative first fill (FLAG_SPECULATE)")
     ap.add_argument("--fp8", action="store_true",
                     help="datatype study: e4m3 expert store with per-row scales (needs --ffn-only or --skip-extras)")
     ap.add_argument("--link-sweep", action="store_true",
@@ -454,7 +453,7 @@ def main():
         return
 
     if args.ffn_only:
-        a = make_ctx(cfg, prob, cfg.N, max_batch=B, flags=2 if args.no_spec else 0)
+        a = make_ctx(cfg, prob, cfg.N, max_batch=B, flags=2 if args.spec else 0)
         a.warm_all()
         mean_s, med_s, n_l = time_ffn_kernel(a, cfg, h_dev, hp_dev, B, tokens=args.steps)
         if B == 1:
@@ -471,7 +470,7 @@ def main():
         return
 
     # ---- headline: config cache size, exact (correctness-preserving) mode, inputs resident in HBM
-    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B, flags=2 if args.no_spec else 0)
+    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B, flags=2 if args.spec else 0)
     if args.resident:
         apex.warm_all()
     sampler = ClockSampler(local_rank)

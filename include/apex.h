@@ -64,9 +64,11 @@ extern "C" {
 
 #define APEX_FLAG_FP8_EXPERTS 1 /* apex_config.flags: expert stores and slots hold e4m3 rows (see below) */
 #define APEX_FLAG_FP4_EXPERTS 4 /* apex_config.flags: expert stores and slots hold block-scaled e2m1 rows (see below) */
-#define APEX_FLAG_NO_SPECULATION 2 /* apex_config.flags: the expert FFN does not start streaming the experts the prefetch
-                                      router ranked first before the gate's decision is visible (for A/B timing; results
-                                      are identical either way) */
+#define APEX_FLAG_SPECULATE 2 /* apex_config.flags: at B = 1 the expert FFN starts streaming the k experts the prefetch router
+                                 ranked first before the gate's decision is visible, and drops the guesses the gate does not
+                                 confirm (results are identical either way).  Pays when FFN launches follow one another
+                                 directly, costs inside the decode loop, where the early copies delay the gate kernel; off by
+                                 default */
 
 #define APEX_MAX_EXPERTS 64
 #define APEX_MAX_TOPK 16

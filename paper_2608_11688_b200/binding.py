@@ -19,7 +19,7 @@ APEX_OK, APEX_EINVAL, APEX_ENOMEM, APEX_ECUDA, APEX_ETIMEOUT, APEX_ESTATE, APEX_
 MODE_EXACT, MODE_STALL_FREE = 0, 1
 MODES = {"exact": MODE_EXACT, "stall_free": MODE_STALL_FREE}
 FLAG_FP8_EXPERTS = 1
-FLAG_NO_SPECULATION = 2
+FLAG_SPECULATE = 2
 FLAG_FP4_EXPERTS = 4
 ERR_NAMES = {0: "APEX_OK", -1: "APEX_EINVAL", -2: "APEX_ENOMEM", -3: "APEX_ECUDA", -4: "APEX_ETIMEOUT",
              -5: "APEX_ESTATE", -6: "APEX_ENOTIMPL"}

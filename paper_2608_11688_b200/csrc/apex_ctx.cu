@@ -122,6 +122,7 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   ml.off_exec_seq = off;  off += L * sizeof(uint32_t);
   off = (off + 15) & ~(size_t)15;
   ml.off_sel_rec = off;   off += 16;
+  ml.off_exec_rec = off;  off += L * 32;   // per layer: routed-set record, execution-set record (B = 1)
   ml.off_ncand = off; off += MB * sizeof(int32_t);
   ml.off_cand = off;  off += MB * C * sizeof(int32_t);
   ml.kr_stride = MB * k * sizeof(int32_t);

@@ -51,6 +51,9 @@ inline volatile uint32_t* mbox_sel_rec(apex_ctx* ctx) { return reinterpret_cast<
 inline volatile uint32_t* mbox_exec_seq(apex_ctx* ctx, int l) {
   return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_exec_seq) + l;
 }
+inline volatile uint32_t* mbox_exec_rec(apex_ctx* ctx, int l) {
+  return reinterpret_cast<volatile uint32_t*>(ctx->mbox + ctx->ml.off_exec_rec) + 8 * l;
+}
 inline int32_t* mbox_kr(apex_ctx* ctx, int l) { return mbox_i32(ctx, ctx->ml.off_kr + (size_t)l * ctx->ml.kr_stride); }
 inline int32_t* mbox_exec(apex_ctx* ctx, int l) { return mbox_i32(ctx, ctx->ml.off_exec + (size_t)l * ctx->ml.kr_stride); }
 

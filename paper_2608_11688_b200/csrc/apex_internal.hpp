@@ -50,7 +50,7 @@ struct MailboxHeader {
 // Byte offsets inside the mailbox.  Per layer: route_seq[l] is written by the gate kernel after
 // K_r of that layer, exec_seq[l] by the FFN's plan step after the execution sets.
 struct MailboxLayout {
-  size_t off_exec_seq, off_sel_rec, off_ncand, off_cand, off_kr, off_exec, kr_stride, bytes;
+  size_t off_exec_seq, off_sel_rec, off_exec_rec, off_ncand, off_cand, off_kr, off_exec, kr_stride, bytes;
 };
 
 // Device-side counters of one layer (S9), accumulated with 64-bit atomics.
@@ -129,6 +129,7 @@ struct FfnParams {
   int32_t* grp;             // [4 + 3*(N+1)]: routed groups, all groups, 0, 0, then (expert, pair offset, tokens) per group
   int32_t* mbox_exec;       // mapped host [B][k]
   int32_t* mbox_kr;         // mapped host [B][k]: the routed sets, posted with the execution sets
+  uint32_t* mbox_rec;       // mapped host, B = 1: two 16-byte records {mask lo, mask hi, sequence number, 0}: routed set, execution set
   volatile uint32_t* mbox_seq;
   volatile uint32_t* mbox_status;
   uint32_t seq_value;

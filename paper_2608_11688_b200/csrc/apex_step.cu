@@ -366,16 +366,15 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
 
 namespace {
 
-constexpr long long kSpecDelayAfterGateNs = 1500;
+constexpr long long kSpecDelayAfterGateNs = 1000;
 
 // Every launch of the streaming kernel gets its own row-ticket counter out of a ring of 64; the
 // launch also clears the counter that will be used 32 launches later.
 cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
   const uint32_t id = ctx->ffn_launch_id++;
   p.zero_early = (!ctx->last_was_ffn && ctx->last_stream == cs) ? 1 : 0;
-  // After the gate kernel the speculative first fill is held back until the gate has fetched its input (measured
-  // on the all-resident decode loop of config 1: 898 tokens/s without delay, 906 / 933 / 937 / 930 / 911 / 891 with
-  // 0.5 / 1 / 1.5 / 2 / 2.5 / 3.5 us, 902 without speculation); between two FFN launches there is nothing to spare.
+  // With APEX_FLAG_SPECULATE: after the gate kernel the speculative first fill is held back until the gate has fetched
+  // its input; between two FFN launches there is nothing to spare.
   p.spec_delay_ns = ctx->last_was_ffn ? 0 : kSpecDelayAfterGateNs;
   ctx->last_was_ffn = true;
   ctx->last_pred_layer = -1;
@@ -452,6 +451,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.grp = ctx->d_grp;
   p.mbox_exec = mbox_exec(ctx, layer);
   p.mbox_kr = mbox_kr(ctx, layer);
+  p.mbox_rec = const_cast<uint32_t*>(mbox_exec_rec(ctx, layer));
   p.mbox_seq = mbox_exec_seq(ctx, layer);
   p.mbox_status = &mhdr(ctx)->status;
   p.seq_value = ++ctx->exec_seq[layer];
@@ -470,12 +470,12 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.demand_tag = ctx->launch_tag;
   p.demand_in_kernel = (mode == APEX_MODE_EXACT && B == 1) ? 1 : 0;
   p.run_mask = p.demand_in_kernel ? ~0ull : p.snap.resident_mask;
-  // Speculative first fill: the kernel may start streaming the experts the prefetch router ranked
+  // Speculative first fill (opt-in): the kernel may start streaming the experts the prefetch router ranked
   // first before the gate's decision is visible.  Allowed when that ranking is certainly complete by
   // then: predicted in this step, its candidate record already seen by the host (apex_prefetch), and
   // the gate kernel (which waits for everything before it) between the two on this same stream.
   p.spec = (B == 1 && st.predicted && st.prefetched && ctx->pred_stream == cs && st.route_stream == cs &&
-            !(ctx->cfg.flags & APEX_FLAG_NO_SPECULATION))
+            (ctx->cfg.flags & APEX_FLAG_SPECULATE))
                ? ctx->d_spec + (size_t)layer * APEX_MAX_TOPK
                : nullptr;
   if (B > 1) {
@@ -498,13 +498,29 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
   if (!st.pending) return APEX_OK;
   st.pending = false;
   const int B = st.B, N = ctx->cfg.N, k = ctx->cfg.k;
-  (void)N;
   cudaStream_t cs = st.pend_stream;
   auto& tab = ctx->tables[layer];
   const FfnParams& p = ctx->ffn_params[layer];
   // the FFN's plan step posts the routed and the execution sets of this layer-step
-  if (!host_wait_seq(ctx, mbox_exec_seq(ctx, layer), ctx->exec_seq[layer])) return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
+  std::vector<int32_t> kr_one, ex_one;  // B = 1: the sets arrive as masks, each with its sequence number in one 16-byte record
   const int32_t* K_r = mbox_kr(ctx, layer);
+  const int32_t* ex_list = mbox_exec(ctx, layer);
+  if (B == 1) {
+    volatile uint32_t* rec = mbox_exec_rec(ctx, layer);
+    if (!host_wait_seq(ctx, rec + 2, ctx->exec_seq[layer]) || !host_wait_seq(ctx, rec + 6, ctx->exec_seq[layer]))
+      return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
+    const uint64_t kr_mask = ((uint64_t)rec[1] << 32) | rec[0], ex_mask = ((uint64_t)rec[5] << 32) | rec[4];
+    for (int e = 0; e < N; ++e) {
+      if ((kr_mask >> e) & 1) kr_one.push_back(e);
+      if ((ex_mask >> e) & 1) ex_one.push_back(e);
+    }
+    kr_one.resize(k, -1);
+    ex_one.resize(k, -1);
+    K_r = kr_one.data();
+    ex_list = ex_one.data();
+  } else if (!host_wait_seq(ctx, mbox_exec_seq(ctx, layer), ctx->exec_seq[layer])) {
+    return fail(ctx, APEX_ETIMEOUT, "apex_moe_ffn: K_r did not arrive");
+  }
   if (st.pend_mode == APEX_MODE_EXACT) {
     std::vector<SlotCopy> copies;
     uint64_t need = 0;
@@ -577,8 +593,7 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
     ctx->host_stats[layer].demand_copies += (int64_t)copies.size();
     ctx->last_copies[layer].insert(ctx->last_copies[layer].end(), copies.begin(), copies.end());
   } else {
-    const int32_t* ex = mbox_exec(ctx, layer);
-    for (int i = 0; i < B * k; ++i) tab.touch(ex[i]);
+    for (int i = 0; i < B * k; ++i) tab.touch(ex_list[i]);
   }
   st.routed = false;  // the layer-step is complete
   st.predicted = false;

@@ -445,19 +445,22 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
   };
 
   auto post_plan = [&]() {
-    // the routed and the execution set go to the caller's buffers and to the host mailbox
-    store_token_plan(tp1, lane, k, p.exec_idx, p.exec_gate, p.mbox_exec);
-    if (lane < k) p.mbox_kr[lane] = tl1.my_idx;
-    if (lane == 0 && p.stats) {
-      const int ns = __popcll(tp1.exec_mask & ~tp1.kr_mask);
-      if (ns) atomicAdd(&p.stats->substitutions, (unsigned long long)ns);
-      atomicAdd(&p.stats->hits_R, (unsigned long long)__popcll(tp1.kr_mask & p.snap.resident_mask));
-    }
-    __threadfence_system();
-    __syncwarp();
+    // The routed and the execution set go to the caller's buffers and, as masks, to the host mailbox: each in ONE
+    // aligned 16-byte store that carries its own sequence number, so no system-scope fence (a round trip over the
+    // host link) sits in this warp's way -- it has rows to stream like every other warp.
+    store_token_plan(tp1, lane, k, p.exec_idx, p.exec_gate, nullptr);
     if (lane == 0) {
-      __threadfence_system();
-      *p.mbox_seq = p.seq_value;
+      if (p.stats) {
+        const int ns = __popcll(tp1.exec_mask & ~tp1.kr_mask);
+        if (ns) atomicAdd(&p.stats->substitutions, (unsigned long long)ns);
+        atomicAdd(&p.stats->hits_R, (unsigned long long)__popcll(tp1.kr_mask & p.snap.resident_mask));
+      }
+      asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p.mbox_rec), "r"((uint32_t)tp1.kr_mask),
+                   "r"((uint32_t)(tp1.kr_mask >> 32)), "r"(p.seq_value), "r"(0u)
+                   : "memory");
+      asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p.mbox_rec + 4), "r"((uint32_t)tp1.exec_mask),
+                   "r"((uint32_t)(tp1.exec_mask >> 32)), "r"(p.seq_value), "r"(0u)
+                   : "memory");
     }
   };
   const bool poster = B == 1 && cta == 0 && warp == 0 && p.post_exec;

@@ -14,10 +14,10 @@ def _harness():
 
 
 def _run(cfg, *, mode, tau, T, B=1, layers=None, C=None, norm_topk=1, cache_reuse=1, check_ffn_every=1,
-         use_prefetch=True, prob=None, ffn_token_stride=1):
+         use_prefetch=True, prob=None, ffn_token_stride=1, flags=0):
     hz = _harness()
     prob = prob or hz.Problem(cfg, layers=layers)
-    apex = prob.make_ctx(C=C, max_batch=B, norm_topk=norm_topk, cache_reuse=cache_reuse)
+    apex = prob.make_ctx(C=C, max_batch=B, norm_topk=norm_topk, cache_reuse=cache_reuse, flags=flags)
     try:
         rep = hz.run_lockstep(prob, apex, mode=mode, tau=tau, T=T, B=B, C=C, norm_topk=bool(norm_topk),
                               cache_reuse=bool(cache_reuse), check_ffn_every=check_ffn_every,
@@ -188,7 +188,7 @@ def test_speculative_fill_with_good_and_useless_predictor(sigma_p, mode):
     # sigma_p = 0: most guesses are confirmed; sigma_p = 8: the prefetch ranking is almost unrelated to the
     # gate's, so nearly every speculative copy is dropped and its stage refilled
     cfg = synth.tiny_config(d=1024, N=24, k=6, I=96, C=12, T=10, I_shared=32, sigma_p=sigma_p, cfg_id=280)
-    rep, stats = _run(cfg, mode=mode, tau=0.6, T=10)
+    rep, stats = _run(cfg, mode=mode, tau=0.6, T=10, flags=binding.FLAG_SPECULATE)
     assert rep.layer_steps == 10 and rep.ffn_checked + rep.near_ties >= 10
     if sigma_p == 8.0:
         assert stats["hits_P"] < 0.8 * stats["routed"]
@@ -202,7 +202,7 @@ def test_speculation_switch_changes_nothing_but_time():
     h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()
     hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
     ys, stats = [], []
-    for flags in (0, binding.FLAG_NO_SPECULATION):
+    for flags in (0, binding.FLAG_SPECULATE):
         apex = prob.make_ctx(flags=flags)
         try:
             y = torch.zeros((cfg.T, cfg.L, 1, cfg.d), dtype=torch.float32, device="cuda")

@@ -304,6 +304,7 @@ struct apex_ctx {
   cudaStream_t cur_copy_streams[kMaxCopyStreams] = {};  // in use: own, or the caller's (then all the same)
   cudaStream_t stream_of_slot(int slot) const { return cur_copy_streams[slot % n_copy_streams]; }
   cudaStream_t pred_stream = nullptr;   // stream of the last apex_predict
+  uintptr_t last_ffn_y_lo = 0, last_ffn_y_hi = 0;  // output range of the last streaming-kernel launch
   int last_pred_layer = -1;             // layer whose prefetch stage (router, budget selection) was the last launch, else -1
   cudaEvent_t ev_wave = nullptr, ev_in = nullptr;
   int inject = 0;

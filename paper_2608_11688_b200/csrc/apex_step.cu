@@ -372,7 +372,13 @@ constexpr long long kSpecDelayAfterGateNs = 1000;
 // launch also clears the counter that will be used 32 launches later.
 cudaError_t launch_stream(apex_ctx* ctx, FfnParams p, cudaStream_t cs) {
   const uint32_t id = ctx->ffn_launch_id++;
-  p.zero_early = (!ctx->last_was_ffn && ctx->last_stream == cs) ? 1 : 0;
+  // y may be zeroed before the dependency wait when the kernel in front of this one on the stream does not touch it:
+  // any kernel of this library that is not an expert-FFN launch, or an FFN launch that wrote another buffer.
+  const uintptr_t y_lo = (uintptr_t)p.y, y_hi = y_lo + (size_t)p.B * p.d * sizeof(float);
+  const bool prev_ffn_disjoint = ctx->last_was_ffn && (y_hi <= ctx->last_ffn_y_lo || ctx->last_ffn_y_hi <= y_lo);
+  p.zero_early = (ctx->last_stream == cs && (!ctx->last_was_ffn || prev_ffn_disjoint)) ? 1 : 0;
+  ctx->last_ffn_y_lo = y_lo;
+  ctx->last_ffn_y_hi = y_hi;
   // With APEX_FLAG_SPECULATE: after the gate kernel the speculative first fill is held back until the gate has fetched
   // its input; between two FFN launches there is nothing to spare.
   p.spec_delay_ns = ctx->last_was_ffn ? 0 : kSpecDelayAfterGateNs;
@@ -410,6 +416,8 @@ int launch_batched(apex_ctx* ctx, int layer, const FfnParams& p, cudaStream_t cs
     t.layer_slot0 = layer * ctx->cfg.C;
     CU_TRY(ctx, launch_ffn_tc(t, ctx->tc_shared_maps[layer], ctx->n_sm, cs));
     ctx->last_was_ffn = true;
+    ctx->last_ffn_y_lo = (uintptr_t)p.y;
+    ctx->last_ffn_y_hi = (uintptr_t)p.y + (size_t)p.B * p.d * sizeof(float);
     ctx->last_pred_layer = -1;
     ctx->launches += 3;
   } else {

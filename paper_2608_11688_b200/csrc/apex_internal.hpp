@@ -176,7 +176,6 @@ struct AttnParams {
   size_t n_vec;  // 16-byte vectors
   float* sink;
   int wait_first;       // 1: wait for the preceding kernel before streaming; 0: stream beside it, wait before exiting
-  long long delay_ns;   // (wait_first = 0) start streaming this long after the CTA does
 };
 
 // launchers (kernels_*.cu).  Each returns the cudaError_t of the launch.

@@ -123,9 +123,6 @@ int check_device_status(apex_ctx* ctx) {
 
 namespace {
 
-// Head starts, in ns, that a latency-bound router kernel gets over a bandwidth-hungry kernel launched right behind it
-// (measured; see the launch sites).
-constexpr long long kAttnDelayAfterPredictNs = 2500;
 
 int begin_predict(apex_ctx* ctx, int layer, const float* h_dev, int B, RouterParams* p) {
   if (!h_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_predict: bad h or B");
@@ -304,10 +301,6 @@ int apex_attention_standin(apex_ctx* ctx, int layer, void* stream) {
   // just before it on this stream is this layer-step's prefetch stage, the two may run side by side (Sec. IV-A:
   // prediction and prefetch are hidden under attention).  Anything else in front of it is waited for first.
   p.wait_first = (ctx->last_stream == (cudaStream_t)stream && ctx->last_pred_layer == layer) ? 0 : 1;
-  // It starts streaming a little after the prefetch router, whose few loads would otherwise queue behind its own
-  // (all-resident decode loop of config 1: 935 tokens/s one after the other; side by side 973 / 977 / 989 / 994 / 988 /
-  // 958 / 918 with a head start of 0 / 1 / 1.5 / 2.5 / 3.5 / 4.5 / 6 us for the router).
-  p.delay_ns = kAttnDelayAfterPredictNs;
   CU_TRY(ctx, launch_attention(p, ctx->n_sm, (cudaStream_t)stream));
   // (only an attention kernel that waited for the prefetch stage before anything else lets the gate read that
   // stage's outputs ahead of its own dependency wait)

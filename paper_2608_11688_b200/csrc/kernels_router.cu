@@ -345,10 +345,6 @@ __global__ void __launch_bounds__(512) attention_standin_kernel(const AttnParams
   SPAN_BEGIN();
   if (p.wait_first) pdl_wait();
   pdl_launch_dependents();
-  if (!p.wait_first && p.delay_ns > 0) {
-    const unsigned long long t0 = globaltimer_ns();
-    while ((long long)(globaltimer_ns() - t0) < p.delay_ns) __nanosleep(200);
-  }
   const size_t stride = (size_t)gridDim.x * blockDim.x;
   uint4 a = make_uint4(0, 0, 0, 0);
   for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < p.n_vec; i += stride) {

@@ -100,7 +100,6 @@ struct RouterParams {
   // gate-kernel epilogue (S9 metrics + mailbox); all null/0 for the prefetch router
   const int32_t* pi_pred;     // [B][N] ranking of the prefetch router for this step, or null
   const int32_t* ncand_pred;  // [B]
-  int pred_early;             // 1: pi_pred / ncand_pred were written earlier on this stream: may be read before the dependency wait
   DevStats* stats;
   int C;
   int fuse_select;   // 1: the leader warp also runs the budget selection (sel) for its token
@@ -281,8 +280,6 @@ struct apex_ctx {
     int B = 0;
     bool predicted = false, selected = false, prefetched = false, routed = false;
     cudaStream_t route_stream = nullptr;   // stream of this step's gate kernel
-    cudaStream_t sel_stream = nullptr;     // stream of this step's budget selection
-    cudaStream_t attn_stream = nullptr;    // stream of the attention stand-in launched after the selection, if any
     const int32_t* idx_dev = nullptr;
     const float* alpha_dev = nullptr;
     // an FFN launch whose host-side completion (LRU touch, demand copies) is still due

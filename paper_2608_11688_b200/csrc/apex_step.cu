@@ -189,8 +189,6 @@ int predict_select_fused(apex_ctx* ctx, int layer, const float* h_dev, int B, fl
   ctx->pred_stream = cs;
   ctx->step[layer].predicted = true;
   ctx->step[layer].selected = true;
-  ctx->step[layer].sel_stream = cs;
-  ctx->step[layer].attn_stream = nullptr;
   ctx->host_stats[layer].layer_steps += 1;
   return APEX_OK;
 }
@@ -230,8 +228,6 @@ int apex_select_candidates(apex_ctx* ctx, int layer, int B, float tau, int32_t* 
   ctx->last_stream = (cudaStream_t)stream;
   ++ctx->launches;
   st.selected = true;
-  st.sel_stream = (cudaStream_t)stream;
-  st.attn_stream = nullptr;
   return APEX_OK;
 }
 
@@ -302,9 +298,6 @@ int apex_attention_standin(apex_ctx* ctx, int layer, void* stream) {
   // prediction and prefetch are hidden under attention).  Anything else in front of it is waited for first.
   p.wait_first = (ctx->last_stream == (cudaStream_t)stream && ctx->last_pred_layer == layer) ? 0 : 1;
   CU_TRY(ctx, launch_attention(p, ctx->n_sm, (cudaStream_t)stream));
-  // (only an attention kernel that waited for the prefetch stage before anything else lets the gate read that
-  // stage's outputs ahead of its own dependency wait)
-  ctx->step[layer].attn_stream = p.wait_first ? (cudaStream_t)stream : nullptr;
   ctx->last_was_ffn = false;
   ctx->last_pred_layer = -1;
   ctx->last_stream = (cudaStream_t)stream;
@@ -338,10 +331,6 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
   p.N = (int)N; p.d = (int)d; p.B = B; p.k = ctx->cfg.k; p.C = ctx->cfg.C;
   p.pi_pred = st.selected ? ctx->d_pi : nullptr;
   p.ncand_pred = st.selected ? ctx->d_ncand : nullptr;
-  // the prefetch stage's outputs may be read before this kernel's dependency wait when a whole kernel of this
-  // library (the attention stand-in of this layer-step) ran between the two on this same stream
-  p.pred_early = (st.selected && ctx->pred_stream == (cudaStream_t)stream && st.sel_stream == (cudaStream_t)stream &&
-                  st.attn_stream == (cudaStream_t)stream) ? 1 : 0;
   p.stats = ctx->d_stats + layer;
   CU_TRY(ctx, launch_router(p, (cudaStream_t)stream));
   ctx->last_was_ffn = false;

@@ -148,17 +148,6 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
     }
     if (p.bias) bias_e = __ldg(p.bias + e);
   }
-  // Gate only: the prefetch stage's ranking and budget of this token (for the metrics of Eq. (2), (3)) were
-  // written two kernels ago on this stream -- complete by the time this kernel may start -- so the leader
-  // warp fetches them now instead of after the top-k, where the round trip would sit on the critical path.
-  int pred0 = -1, pred1 = -1, nc_pred = 0;
-  const bool pred_loaded = p.pi_pred && p.pred_early && crank == 0 && warp == 0;
-  if (pred_loaded) {
-    const size_t prow = (size_t)b * p.N;
-    if (lane < p.N) pred0 = p.pi_pred[prow + lane];
-    if (lane + 32 < p.N) pred1 = p.pi_pred[prow + lane + 32];
-    nc_pred = p.ncand_pred[b];
-  }
   RTL(0);
   pdl_wait();               // everything queued before this kernel is complete: x may be read
   pdl_launch_dependents();  // the next kernel may begin its own prologue
@@ -250,15 +239,10 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
     int dstar = 0, hitsP = 0, have_pred = 0;
     if (p.pi_pred) {
       have_pred = 1;
-      if (!pred_loaded) {
-        if (e0 < N) pred0 = __ldg(p.pi_pred + row + e0);
-        if (e1 < N) pred1 = __ldg(p.pi_pred + row + e1);
-        nc_pred = __ldg(p.ncand_pred + b);
-      }
-      if (e0 < N) posp[pred0] = e0;  // position of expert pi[j] in E is j
-      if (e1 < N) posp[pred1] = e1;
+      if (e0 < N) posp[__ldg(p.pi_pred + row + e0)] = e0;  // position of expert pi[j] in E is j
+      if (e1 < N) posp[__ldg(p.pi_pred + row + e1)] = e1;
       __syncwarp();
-      const int nc = nc_pred;
+      const int nc = __ldg(p.ncand_pred + b);
       const int pos0 = in0 ? posp[e0] : -1, pos1 = in1 ? posp[e1] : -1;
       dstar = warp_max_int(max(pos0, pos1)) + 1 - k;
       hitsP = __popc(__ballot_sync(0xffffffffu, in0 && pos0 < nc)) + __popc(__ballot_sync(0xffffffffu, in1 && pos1 < nc));

@@ -564,3 +564,29 @@ def test_config1_long_run_stall_free_and_batched():
     assert rep8.layer_steps == 128 and rep8.near_ties <= 2
     print("config1 long run stall-free:", rep, "\nconfig1 long run B=8:", rep8)
 
+
+def test_decode_token_output_does_not_depend_on_the_prefetch_policy():
+    # exact mode: y is the router's top-k mixture whatever was prefetched -- with prefetching, without (tau < 0: the
+    # attention stand-in then follows the previous layer's FFN and must wait for it), and with both alternating
+    cfg = synth.tiny_config(d=1024, N=16, k=4, I=64, C=8, L=3, T=6, sigma_p=0.8, cfg_id=330)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    hs = [synth.hidden_states(cfg, l, cfg.T, 1) for l in range(cfg.L)]
+    h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()
+    hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
+    outs = []
+    for taus in ([0.9] * cfg.T, [-1.0] * cfg.T, [0.9, -1.0] * (cfg.T // 2)):
+        apex = prob.make_ctx()
+        try:
+            y = torch.zeros((cfg.T, cfg.L, 1, cfg.d), dtype=torch.float32, device="cuda")
+            for t in range(cfg.T):
+                apex.decode_token(h[t], hp[t], 1, taus[t], "exact", y[t])
+            torch.cuda.synchronize()
+            assert apex.get_stats()["timeouts"] == 0
+            outs.append(y.cpu().numpy())
+        finally:
+            apex.destroy()
+    scale = float(np.abs(outs[0]).max())
+    for o in outs[1:]:
+        np.testing.assert_allclose(o, outs[0], rtol=0, atol=2e-6 * scale)   # only the order of the fp32 atomics differs
+

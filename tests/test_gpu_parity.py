@@ -590,3 +590,37 @@ def test_decode_token_output_does_not_depend_on_the_prefetch_policy():
     for o in outs[1:]:
         np.testing.assert_allclose(o, outs[0], rtol=0, atol=2e-6 * scale)   # only the order of the fp32 atomics differs
 
+
+def test_random_shapes_modes_and_options():
+    """A fixed-seed walk over shapes and options that the hand-picked cases above do not combine: widths, expert counts
+    up to 64, ragged I, shared experts, cache sizes from k to N, batch sizes on both sides of the tensor-core threshold,
+    both modes, tau at and between the extremes, both cache policies, both gate normalisations, the quantised stores and
+    the opt-in speculative fill.  Every decision and every output is compared with the oracle in lock-step."""
+    import random
+    rng = random.Random(20260811)
+    hz = _harness()
+    for it in range(36):
+        d = rng.choice([256, 512, 768, 1024, 1536, 2048])
+        N = rng.randint(2, 64)
+        k = rng.randint(1, min(N, 16))
+        C = rng.randint(k, N)
+        I = rng.choice([8, 17, 40, 64, 128, 256])
+        Ish = rng.choice([0, 0, 16, 128, 256])
+        B = rng.choice([1, 1, 1, 2, 3, 5, 8, 16, 33])
+        mode = rng.choice(["exact", "stall_free"])
+        tau = rng.choice([0.0, 0.3, 0.7, 0.9, 0.99, 1.0])
+        reuse, norm = rng.choice([1, 1, 0]), rng.choice([1, 1, 0])
+        flags = rng.choice([0, 0, binding.FLAG_SPECULATE])
+        fmt = rng.choice(["bf16", "bf16", "fp8", "fp4"]) if d in (512, 1024, 1536, 2048) else "bf16"
+        L = rng.choice([1, 2])
+        cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, L=L, T=4, I_shared=Ish, sigma_p=rng.choice([0.3, 1.0, 4.0]),
+                                cfg_id=2000 + it)
+        prob = hz.Problem(cfg, fp8=(fmt == "fp8"), fp4=(fmt == "fp4"))
+        apex = prob.make_ctx(max_batch=B, norm_topk=norm, cache_reuse=reuse, flags=flags)
+        try:
+            rep = hz.run_lockstep(prob, apex, mode=mode, tau=tau, T=4, B=B, norm_topk=bool(norm), cache_reuse=bool(reuse))
+            assert apex.get_stats()["timeouts"] == 0
+            assert rep.layer_steps == 4 * L
+        finally:
+            apex.destroy()
+

@@ -174,8 +174,9 @@ int apex_attention_standin(apex_ctx* ctx, int layer, void* stream);
 int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int32_t* idx_dev,
                     float* alpha_dev, void* stream);
 /* S6-S8 (Sec. IV-E): y_dev [B][d] = sum over the execution set of g_e FFN_e(h') (+ shared FFN).
- * APEX_MODE_EXACT executes K_r: resident experts first, missing ones are copied on demand and
- * executed in further launches ("asynchronous miss correction").  APEX_MODE_STALL_FREE executes
+ * APEX_MODE_EXACT executes K_r: resident experts first, missing ones are copied on demand while
+ * those run ("asynchronous miss correction") -- at B = 1 the one kernel waits (bounded) for each
+ * missing expert and then executes it, at B > 1 further launches follow.  APEX_MODE_STALL_FREE executes
  * Algorithm 1 with K_p := the resident set.  exec_idx_dev [B][k] (ascending expert index) and
  * exec_gate_dev [B][k] may be NULL.  Device-side waits on slot-ready flags are bounded; when one
  * runs out the call (or the next call on this context) returns APEX_ETIMEOUT. */

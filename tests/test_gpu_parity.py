@@ -347,6 +347,61 @@ def test_decode_token_matches_per_call_sequence_and_counts_launches():
         a1.destroy(); a2.destroy()
 
 
+def test_ffn_in_two_halves_reset_stats_and_warm_all():
+    # apex_moe_ffn_begin / apex_moe_ffn_end equal apex_moe_ffn; their ordering rules; apex_reset_stats; apex_warm_all
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=6, L=1, T=6, cfg_id=223)
+    hz = _harness()
+    prob = hz.Problem(cfg)
+    a1, a2 = prob.make_ctx(), prob.make_ctx()
+    full = prob.make_ctx(C=cfg.N)
+    try:
+        h, hp = synth.hidden_states(cfg, 0, cfg.T)
+        hd, hpd = torch.from_numpy(h).cuda(), torch.from_numpy(hp).cuda()
+        y1 = torch.empty((1, cfg.d), device="cuda"); y2 = torch.empty_like(y1)
+        cand = torch.empty((1, cfg.C), dtype=torch.int32, device="cuda"); nc = torch.empty(1, dtype=torch.int32, device="cuda")
+        idx = torch.empty((1, cfg.k), dtype=torch.int32, device="cuda"); al = torch.empty((1, cfg.N), device="cuda")
+        with pytest.raises(binding.ApexError) as ei:
+            a2.moe_ffn_end(0)                                   # nothing was begun
+        assert ei.value.code == binding.APEX_ESTATE and "apex_moe_ffn_begin" in str(ei.value)
+        for t in range(cfg.T):
+            mode = "exact" if t % 2 == 0 else "stall_free"
+            for a in (a1, a2):
+                a.predict(0, hd[t], 1); a.select_candidates(0, 1, 0.9, cand, nc); a.prefetch(0, 1)
+                a.attention_standin(0); a.route_topk(0, hpd[t], 1, idx, al)
+            a1.moe_ffn(0, mode, hpd[t], 1, y1)
+            a2.moe_ffn_begin(0, mode, hpd[t], 1, y2)
+            if t == 0:
+                with pytest.raises(binding.ApexError) as ei:    # the layer-step is not complete yet
+                    a2.predict(0, hd[t], 1)
+                assert ei.value.code == binding.APEX_ESTATE
+            a2.moe_ffn_end(0)
+            torch.cuda.synchronize()
+            torch.testing.assert_close(y1, y2, rtol=1e-4, atol=1e-5)   # fp32 atomics: the order of the partial sums is free
+            assert a1.get_last_copies(0) == a2.get_last_copies(0)
+            t1, t2 = a1.get_slot_table(0), a2.get_slot_table(0)
+            assert list(t1[0]) == list(t2[0]) and list(t1[1]) == list(t2[1])
+        s = a1.get_stats()
+        assert s["layer_steps"] == cfg.T and s["tokens"] == cfg.T and s["routed"] == cfg.T * cfg.k
+        a1.reset_stats()
+        assert all(v == 0 for v in a1.get_stats().values())
+        # warm_all: only when every expert has a slot; afterwards nothing is ever copied
+        with pytest.raises(binding.ApexError) as ei:
+            a1.warm_all()
+        assert ei.value.code in (binding.APEX_EINVAL, binding.APEX_ESTATE)
+        full.warm_all()
+        es, _, _ = full.get_slot_table(0)
+        assert sorted(es) == list(range(cfg.N))
+        full.reset_stats()
+        for t in range(cfg.T):
+            full.predict(0, hd[t], 1); full.select_candidates(0, 1, 0.9, cand, nc); full.prefetch(0, 1)
+            full.route_topk(0, hpd[t], 1, idx, al); full.moe_ffn(0, "exact", hpd[t], 1, y1)
+        torch.cuda.synchronize()
+        s = full.get_stats()
+        assert s["prefetch_copies"] == 0 and s["demand_copies"] == 0 and s["hits_R"] == s["routed"] == cfg.T * cfg.k
+    finally:
+        a1.destroy(); a2.destroy(); full.destroy()
+
+
 def test_slot_table_checkpoint_and_resume():
     # snapshot the slot tables after a few tokens, restore them into a fresh context, continue: same outputs
     cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=6, L=2, T=8, cfg_id=222)

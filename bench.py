@@ -386,6 +386,9 @@ def main():
                          "(a different predictor than the workload's: needs --skip-extras)")
     ap.add_argument("--fp4", action="store_true",
                     help="datatype study: block-scaled e2m1 expert store (needs --ffn-only or --skip-extras)")
+    ap.add_argument("--trace", action="store_true",
+                    help="debug: run a few decode tokens on the library built with time stamps (trace.py) and print the "
+                         "kernel spans of the last two; combine with --resident / --layers / --batch / --config")
     args = ap.parse_args()
     if (args.fp8 or args.fp4) and not (args.ffn_only or args.skip_extras):
         ap.error("--fp8 / --fp4 are study legs: combine them with --ffn-only or --skip-extras")
@@ -414,6 +417,10 @@ def main():
     dev = torch.device("cuda", local_rank)
     if rank == 0:
         build.build()
+    trace_lib = None
+    if args.trace:   # before anything loads the product library: a process holds one of the two
+        from paper_2608_11688_b200 import trace
+        trace_lib = trace.use_trace_library()
     from paper_2608_11688_b200 import replicas
     dist_sync = None
     if world > 1:
@@ -434,6 +441,30 @@ def main():
     h_pin, hp_pin = h.pin_memory(), hp.pin_memory()
     y_dev = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32, device=dev)
     y_pin = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32).pin_memory()
+
+    if args.trace:
+        a = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B)
+        if args.resident:
+            a.warm_all()
+        for t in range(args.warmup):
+            a.decode_token(h_dev[t % T], hp_dev[t % T], B, TAU, "exact", y_dev)
+        torch.cuda.synchronize()
+        trace.reset(trace_lib)
+        n_tok = 2
+        for t in range(args.warmup, args.warmup + n_tok):
+            a.decode_token(h_dev[t % T], hp_dev[t % T], B, TAU, "exact", y_dev)
+        torch.cuda.synchronize()
+        spans = trace.read_spans(trace_lib)
+        per_layer = max(1, len(spans) // (n_tok * cfg.L))
+        print(trace.format_spans(spans, limit=3 * per_layer + 2), file=sys.stderr)
+        summary = trace.summarize(spans)
+        phases = trace.ffn_phase_medians(trace.read_ffn_cta_stamps(trace_lib, torch.cuda.get_device_properties(dev).multi_processor_count)) if B == 1 else {}
+        print(json.dumps({"trace": summary, "tokens_traced": n_tok, "layers": cfg.L, "B": B,
+                          "us_per_layer_step": summary["_all"]["wall_us"] / (n_tok * cfg.L),
+                          "ffn_cta_phase_median_cycles": phases, "config": f"config{cfg.cfg_id}",
+                          "resident": bool(args.resident)}), flush=True)
+        a.destroy()
+        return
 
     if args.link_sweep:
         import torch

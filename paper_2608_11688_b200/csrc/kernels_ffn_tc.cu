@@ -121,6 +121,7 @@ __device__ __forceinline__ Group load_group(const int32_t* grp, int g) {
 
 // ---------------------------------------------------------------- gather + zero
 __global__ void __launch_bounds__(256) ffn_tc_gather_kernel(const TcParams p) {
+  SPAN_BEGIN();
   pdl_wait();               // the plan kernel's pair list is complete from here on
   pdl_launch_dependents();  // the next kernel may start its prologue
   const int n_pairs = p.f.n_pairs[0];
@@ -144,6 +145,7 @@ __global__ void __launch_bounds__(256) ffn_tc_gather_kernel(const TcParams p) {
       dst[c] = o;
     }
   }
+  SPAN_END(7);
 }
 
 // ---------------------------------------------------------------- the two GEMM kernels
@@ -154,6 +156,7 @@ template <int PHASE>
 __global__ void __launch_bounds__(kTcThreads, 1)
 ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_ws,
                    const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_b2, const TcParams p) {
+  SPAN_BEGIN();
   extern __shared__ __align__(1024) uint8_t smem_raw[];
   uint8_t* smem = reinterpret_cast<uint8_t*>(((uintptr_t)smem_raw + 1023) & ~(uintptr_t)1023);
   constexpr int A_BYTES = PHASE == 1 ? 2 * 128 * 128 : 2 * 64 * 128;  // gate+up tiles | two downT atoms
@@ -400,6 +403,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   tc_fence_before();
   __syncthreads();
   if (warp == kMmaWarp) asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(512) : "memory");
+  SPAN_END(PHASE == 1 ? 8 : 9);
 }
 
 #ifdef APEX_TIMELINE

@@ -29,6 +29,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
   const int N = p.N, k = p.k, B = p.B;
   int my_subst = 0, my_hits = 0;
+  SPAN_BEGIN();
   PTL(0);
   TokenLoads tls[TOK_PER_WARP];
 #pragma unroll
@@ -180,6 +181,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     }
   }
   PTL(6);
+  SPAN_END(6);
 }
 
 cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s) {

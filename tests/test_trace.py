@@ -1,0 +1,49 @@
+"""The trace tool: span formatting / summary on the CPU, and one traced decode on the GPU (in a process of its own,
+because a process holds either the product library or the traced build)."""
+import json
+import os
+import subprocess
+import sys
+
+import pytest
+
+from paper_2608_11688_b200 import trace
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def test_summary_and_format_of_hand_made_spans():
+    spans = [(1, 1000, 6000), (3, 2000, 8000), (4, 8000, 12000), (5, 12500, 25000), (1, 25000, 30000)]
+    s = trace.summarize(spans)
+    assert s[trace.KERNEL_NAMES[1]] == {"launches": 2, "mean_us": 5.0, "max_us": 5.0}
+    assert s[trace.KERNEL_NAMES[5]]["mean_us"] == 12.5
+    # union of the spans: [1000, 12000] + [12500, 30000] = 28500 of 29000 ns
+    assert s["_all"]["spans"] == 5 and abs(s["_all"]["wall_us"] - 29.0) < 1e-9
+    assert abs(s["_all"]["busy_fraction"] - 28500 / 29000) < 1e-12
+    text = trace.format_spans(spans, limit=4).splitlines()
+    assert len(text) == 1 + 4 + 1 and text[-1].startswith("... 1 more")
+    gate = text[3].split()
+    assert gate[0] == "gate" and float(gate[1]) == 7.0 and float(gate[3]) == 4.0 and float(gate[4]) == 0.0
+    assert float(text[4].split()[-1]) == 0.5     # the FFN starts 0.5 us after the gate's end
+    assert trace.format_spans([]) == "(no spans recorded)"
+    assert trace.summarize([]) == {}
+
+
+@pytest.mark.gpu
+def test_traced_decode_records_every_kernel_in_order():
+    r = subprocess.run([sys.executable, "bench.py", "--trace", "--config", "0", "--resident", "--warmup", "3"],
+                       cwd=ROOT, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    t = line["trace"]
+    n = line["tokens_traced"] * line["layers"]
+    for kid in (1, 3, 4, 5):     # prefetch router (+ selection), attention stand-in, gate, expert FFN: one launch per layer-step
+        assert t[trace.KERNEL_NAMES[kid]]["launches"] == n, t
+        assert 0.5 < t[trace.KERNEL_NAMES[kid]]["mean_us"] < 500.0
+    assert t["_all"]["spans"] == 4 * n and 0.0 < t["_all"]["busy_fraction"] <= 1.0
+    ph = line["ffn_cta_phase_median_cycles"]
+    assert len(ph) == 7 and all(v >= 0 for v in ph.values())
+    # the table printed beside it lists the kernels of a layer-step in launch order
+    rows = [l for l in r.stderr.splitlines() if l[:6] in ("prefet", "attent", "gate  ", "expert")]
+    assert rows[0].startswith("prefetch router") and rows[1].startswith("attention") and rows[2].startswith("gate")
+    assert rows[3].startswith("expert FFN")

@@ -97,6 +97,7 @@ struct RouterParams {
   int32_t* topk_out;  // [B][k] or null
   int N, d, B, k;
   int warps_per_cta;
+  int tok_per_group;  // batched kernel: tokens a cluster handles per pass (set by the launcher)
   // gate-kernel epilogue (S9 metrics + mailbox); all null/0 for the prefetch router
   const int32_t* pi_pred;     // [B][N] ranking of the prefetch router for this step, or null
   const int32_t* ncand_pred;  // [B]

@@ -120,6 +120,81 @@ extern "C" int apex_debug_read_router_tl(long long* host) { return (int)cudaMemc
 #define RTL(i) do { } while (0)
 #endif
 
+// Softmax, ranking, top-k and the per-token outputs of one token by one warp (lanes own experts lane and lane+32),
+// from the token's N logits in shared memory; then either the budget selection (prefetch router, fused launch) or
+// the metrics of Eq. (2), (3) against the prefetch stage (gate).  qs, pis, posp: this warp's scratch, 64 entries each.
+__device__ __forceinline__ void router_epilogue(const RouterParams& p, int b, int lane, const float* zs, float* qs, int* pis,
+                                                int* posp) {
+  const int N = p.N, k = p.k;
+  const int e0 = lane, e1 = lane + 32;
+  const float NEG = -3.402823466e38f;
+  const float z0 = e0 < N ? zs[e0] : NEG;
+  const float z1 = e1 < N ? zs[e1] : NEG;
+  const float m = warp_max_tree(fmaxf(z0, z1));
+  const float x0 = e0 < N ? expf(z0 - m) : 0.f;
+  const float x1 = e1 < N ? expf(z1 - m) : 0.f;
+  const float sum = warp_sum_tree(x0 + x1);
+  const float q0 = x0 / sum, q1 = x1 / sum;
+  int r0 = 0, r1 = 0;  // rank = number of experts ordered before mine (value desc, index asc)
+#pragma unroll 8
+  for (int f = 0; f < N; ++f) {
+    const float zf = zs[f];
+    r0 += (zf > z0 || (zf == z0 && f < e0)) ? 1 : 0;
+    r1 += (zf > z1 || (zf == z1 && f < e1)) ? 1 : 0;
+  }
+  const size_t row = (size_t)b * N;
+  if (e0 < N) {
+    p.z_out[row + e0] = z0;
+    p.q_out[row + e0] = q0;
+    if (p.pi_out) p.pi_out[row + r0] = e0;
+    if (p.topk_out && r0 < k) p.topk_out[(size_t)b * k + r0] = e0;
+  }
+  if (e1 < N) {
+    p.z_out[row + e1] = z1;
+    p.q_out[row + e1] = q1;
+    if (p.pi_out) p.pi_out[row + r1] = e1;
+    if (p.topk_out && r1 < k) p.topk_out[(size_t)b * k + r1] = e1;
+  }
+  RTL(4);
+  if (p.fuse_select) {
+    // prefetch router and budget selection in one launch: the ranked list goes through shared memory
+    if (e0 < N) { qs[e0] = q0; pis[r0] = e0; }
+    if (e1 < N) { qs[e1] = q1; pis[r1] = e1; }
+    __syncwarp();
+    const int pj0 = lane < N ? pis[lane] : -1, pj1 = lane + 32 < N ? pis[lane + 32] : -1;
+    const float x0 = pj0 >= 0 ? qs[pj0] : 0.f, x1 = pj1 >= 0 ? qs[pj1] : 0.f;
+    select_token(p.sel, b, lane, pj0, pj1, x0, x1);
+    RTL(5);
+    return;
+  }
+  if (!p.topk_out || !p.stats) return;
+
+  // ---- gate epilogue: metrics of this token against the prefetch stage (Eq. (2), (3))
+  const bool in0 = e0 < N && r0 < k, in1 = e1 < N && r1 < k;
+  {
+    int dstar = 0, hitsP = 0, have_pred = 0;
+    if (p.pi_pred) {
+      have_pred = 1;
+      if (e0 < N) posp[__ldg(p.pi_pred + row + e0)] = e0;  // position of expert pi[j] in E is j
+      if (e1 < N) posp[__ldg(p.pi_pred + row + e1)] = e1;
+      __syncwarp();
+      const int nc = __ldg(p.ncand_pred + b);
+      const int pos0 = in0 ? posp[e0] : -1, pos1 = in1 ? posp[e1] : -1;
+      dstar = warp_max_int(max(pos0, pos1)) + 1 - k;
+      hitsP = __popc(__ballot_sync(0xffffffffu, in0 && pos0 < nc)) + __popc(__ballot_sync(0xffffffffu, in1 && pos1 < nc));
+    }
+    if (lane == 0) {
+      atomicAdd(&p.stats->routed, (unsigned long long)k);
+      if (have_pred) {
+        atomicAdd(&p.stats->sum_delta_star, (unsigned long long)dstar);
+        atomicAdd(&p.stats->hits_P, (unsigned long long)hitsP);
+        atomicAdd(&p.stats->covered, (unsigned long long)(hitsP == k ? 1 : 0));
+      }
+    }
+  }
+  RTL(5);
+}
+
 __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
   SPAN_BEGIN();
   cg::cluster_group cluster = cg::this_cluster();
@@ -184,80 +259,130 @@ __global__ void __launch_bounds__(256) router_kernel(const RouterParams p) {
   RTL(3);
   if (crank != 0 || warp != 0) return;
 
-  // ---- leader warp: lanes own experts lane and lane+32
-  const int N = p.N, k = p.k;
-  const int e0 = lane, e1 = lane + 32;
-  const float NEG = -3.402823466e38f;
-  const float z0 = e0 < N ? zs[e0] : NEG;
-  const float z1 = e1 < N ? zs[e1] : NEG;
-  const float m = warp_max_tree(fmaxf(z0, z1));
-  const float x0 = e0 < N ? expf(z0 - m) : 0.f;
-  const float x1 = e1 < N ? expf(z1 - m) : 0.f;
-  const float sum = warp_sum_tree(x0 + x1);
-  const float q0 = x0 / sum, q1 = x1 / sum;
-  int r0 = 0, r1 = 0;  // rank = number of experts ordered before mine (value desc, index asc)
-#pragma unroll 8
-  for (int f = 0; f < N; ++f) {
-    const float zf = zs[f];
-    r0 += (zf > z0 || (zf == z0 && f < e0)) ? 1 : 0;
-    r1 += (zf > z1 || (zf == z1 && f < e1)) ? 1 : 0;
-  }
-  const size_t row = (size_t)b * N;
-  if (e0 < N) {
-    p.z_out[row + e0] = z0;
-    p.q_out[row + e0] = q0;
-    if (p.pi_out) p.pi_out[row + r0] = e0;
-    if (p.topk_out && r0 < k) p.topk_out[(size_t)b * k + r0] = e0;
-  }
-  if (e1 < N) {
-    p.z_out[row + e1] = z1;
-    p.q_out[row + e1] = q1;
-    if (p.pi_out) p.pi_out[row + r1] = e1;
-    if (p.topk_out && r1 < k) p.topk_out[(size_t)b * k + r1] = e1;
-  }
-  RTL(4);
-  if (p.fuse_select) {
-    // prefetch router and budget selection in one launch: the ranked list goes through shared memory
-    if (e0 < N) { qs[e0] = q0; pis[r0] = e0; }
-    if (e1 < N) { qs[e1] = q1; pis[r1] = e1; }
-    __syncwarp();
-    const int pj0 = lane < N ? pis[lane] : -1, pj1 = lane + 32 < N ? pis[lane + 32] : -1;
-    const float x0 = pj0 >= 0 ? qs[pj0] : 0.f, x1 = pj1 >= 0 ? qs[pj1] : 0.f;
-    select_token(p.sel, b, lane, pj0, pj1, x0, x1);
-    RTL(5);
-    SPAN_END(1);
-    return;
-  }
-  if (!p.topk_out || !p.stats) {
-    SPAN_END(1);
-    return;
-  }
+  // ---- leader warp
+  router_epilogue(p, b, lane, zs, qs, pis, posp);
+  SPAN_END((p.fuse_select || !p.topk_out || !p.stats) ? 1 : 4);
+}
 
-  // ---- gate epilogue: metrics of this token against the prefetch stage (Eq. (2), (3))
-  const bool in0 = e0 < N && r0 < k, in1 = e1 < N && r1 < k;
-  {
-    int dstar = 0, hitsP = 0, have_pred = 0;
-    if (p.pi_pred) {
-      have_pred = 1;
-      if (e0 < N) posp[__ldg(p.pi_pred + row + e0)] = e0;  // position of expert pi[j] in E is j
-      if (e1 < N) posp[__ldg(p.pi_pred + row + e1)] = e1;
-      __syncwarp();
-      const int nc = __ldg(p.ncand_pred + b);
-      const int pos0 = in0 ? posp[e0] : -1, pos1 = in1 ? posp[e1] : -1;
-      dstar = warp_max_int(max(pos0, pos1)) + 1 - k;
-      hitsP = __popc(__ballot_sync(0xffffffffu, in0 && pos0 < nc)) + __popc(__ballot_sync(0xffffffffu, in1 && pos1 < nc));
+// The same for a batch (B > 1).  A cluster keeps its weight rows in registers and walks over groups of
+// kRouterTok tokens: the group's hidden states (1 to kRouterTok tokens, chosen by the launcher) are staged in shared memory once, every warp takes the dot
+// products of its expert's row with all of them (per token the arithmetic and its order are those of
+// router_kernel), the logits go to the leader CTA, one cluster barrier per group, and warp t of the leader
+// CTA finishes token t of the group.  The logits are double-buffered: a buffer is written again two groups
+// later, after the barrier of the group in between, which the leader's warps reach only when they are done
+// reading it.  W_r is read once per cluster instead of once per token.
+constexpr int kRouterTok = 8;  // tokens per group = warps of a CTA
+
+__global__ void __launch_bounds__(256) router_batched_kernel(const RouterParams p) {
+  SPAN_BEGIN();
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned crank = cluster.block_rank();
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  __shared__ float zs[2][kRouterTok][APEX_MAX_EXPERTS];
+  __shared__ float qs[kRouterTok][APEX_MAX_EXPERTS];
+  __shared__ int pis[kRouterTok][APEX_MAX_EXPERTS];
+  __shared__ int posp[kRouterTok][APEX_MAX_EXPERTS];
+  extern __shared__ float4 xs_dyn[];  // [kRouterTok][d / 4]
+
+  const int e = (int)crank * p.warps_per_cta + warp;
+  const bool active = warp < p.warps_per_cta && e < p.N;
+  const int nv = p.d >> 2;
+  float4 wreg[kRouterMaxVec];
+  float bias_e = 0.f;
+  if (active) {
+    const float4* __restrict__ Wrow = reinterpret_cast<const float4*>(p.W + (size_t)e * p.d);
+#pragma unroll
+    for (int i = 0; i < kRouterMaxVec; ++i) {
+      const int c = i * 32 + lane;
+      // volatile: under this kernel's register pressure the compiler would otherwise sink the loads into the
+      // token loop, behind the dependency wait and once per group
+      if (c < nv)
+        asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];"
+                     : "=f"(wreg[i].x), "=f"(wreg[i].y), "=f"(wreg[i].z), "=f"(wreg[i].w)
+                     : "l"(Wrow + c));
     }
-    if (lane == 0) {
-      atomicAdd(&p.stats->routed, (unsigned long long)k);
-      if (have_pred) {
-        atomicAdd(&p.stats->sum_delta_star, (unsigned long long)dstar);
-        atomicAdd(&p.stats->hits_P, (unsigned long long)hitsP);
-        atomicAdd(&p.stats->covered, (unsigned long long)(hitsP == k ? 1 : 0));
+    if (p.bias) bias_e = __ldg(p.bias + e);
+  }
+  RTL(0);
+  pdl_wait();
+  pdl_launch_dependents();
+  RTL(1);
+
+  const int tpg = p.tok_per_group;  // tokens per group, 1..kRouterTok
+  const int n_groups = (p.B + tpg - 1) / tpg;
+  int buf = 0;
+  for (int g = blockIdx.y; g < n_groups; g += gridDim.y, buf ^= 1) {
+    const int b0 = g * tpg;
+    const int nt = p.B - b0 < tpg ? p.B - b0 : tpg;
+    {
+      // the group's rows of x are contiguous: one linear copy.  (Every warp of this CTA passed the cluster
+      // barrier of the previous group after its last read of xs.)
+      // Asynchronous 16-byte copies, all in flight at once: a loop of load-then-store would pay the memory
+      // latency once per trip (up to 32 trips per thread).
+      const float4* __restrict__ xv = reinterpret_cast<const float4*>(p.x + (size_t)b0 * p.d);
+      for (int c = threadIdx.x; c < nt * nv; c += blockDim.x)
+        asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(xs_dyn + c)), "l"(xv + c) : "memory");
+      asm volatile("cp.async.wait_all;" ::: "memory");
+    }
+    __syncthreads();
+    RTL(2);
+    if (active) {
+      float acc[kRouterTok];
+#pragma unroll
+      for (int t = 0; t < kRouterTok; ++t) acc[t] = 0.f;
+      if (nt == kRouterTok) {  // full group: no per-token predicate inside the unrolled loops
+#pragma unroll
+        for (int i = 0; i < kRouterMaxVec; ++i) {
+          const int c = i * 32 + lane;
+          if (c < nv) {
+#pragma unroll
+            for (int t = 0; t < kRouterTok; ++t) {
+              const float4 x = xs_dyn[t * nv + c];
+              acc[t] = fmaf(wreg[i].x, x.x, acc[t]);
+              acc[t] = fmaf(wreg[i].y, x.y, acc[t]);
+              acc[t] = fmaf(wreg[i].z, x.z, acc[t]);
+              acc[t] = fmaf(wreg[i].w, x.w, acc[t]);
+            }
+          }
+        }
+      }
+      float mine = 0.f;  // lane t delivers token t
+      if (nt == kRouterTok) {
+#pragma unroll
+        for (int t = 0; t < kRouterTok; ++t) {
+          const float v = warp_sum_tree(acc[t]);
+          if (lane == t) mine = v;
+        }
+      } else {  // partial group: token by token
+        for (int t = 0; t < nt; ++t) {
+          float a = 0.f;
+#pragma unroll
+          for (int i = 0; i < kRouterMaxVec; ++i) {
+            const int c = i * 32 + lane;
+            if (c < nv) {
+              const float4 x = xs_dyn[t * nv + c];
+              a = fmaf(wreg[i].x, x.x, a);
+              a = fmaf(wreg[i].y, x.y, a);
+              a = fmaf(wreg[i].z, x.z, a);
+              a = fmaf(wreg[i].w, x.w, a);
+            }
+          }
+          a = warp_sum_tree(a);
+          if (lane == t) mine = a;
+        }
+      }
+      if (lane < nt) {
+        float* dst = cluster.map_shared_rank(&zs[0][0][0], 0);
+        dst[(buf * kRouterTok + lane) * APEX_MAX_EXPERTS + e] = mine + bias_e;
       }
     }
+    RTL(3);
+    cluster.sync();
+    RTL(4);
+    if (crank == 0 && warp < nt) router_epilogue(p, b0 + warp, lane, zs[buf][warp], qs[warp], pis[warp], posp[warp]);
   }
-  RTL(5);
-  SPAN_END(4);
+  RTL(6);
+  SPAN_END((p.fuse_select || !p.topk_out || !p.stats) ? 1 : 4);
 }
 
 cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
@@ -271,6 +396,34 @@ cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
   cfg.blockDim = dim3(256, 1, 1);
   cfg.dynamicSmemBytes = 0;
   cfg.stream = s;
+  const bool batched = p.B > 1;
+  if (batched) {
+    // one cluster per group of tokens, at most as many clusters as fit the GPU at one CTA per SM (the weight
+    // rows in registers allow no more); further groups are walked by the same clusters
+    static int n_sm_of[kMaxDevices];
+    static bool configured[kMaxDevices];
+    int dev = 0;
+    cudaError_t e = cudaGetDevice(&dev);
+    if (e != cudaSuccess) return e;
+    if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
+    if (!configured[dev]) {
+      if ((e = cudaDeviceGetAttribute(&n_sm_of[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+      if ((e = cudaFuncSetAttribute(router_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                    kRouterTok * kRouterMaxVec * 32 * (int)sizeof(float4))) != cudaSuccess)
+        return e;
+      configured[dev] = true;
+    }
+    int resident = n_sm_of[dev] / csize;
+    if (resident < 1) resident = 1;
+    // small batches spread over the clusters (a token per cluster while they last); large ones fill the groups,
+    // because a group costs a barrier and a round of shared-memory reads of all its tokens per warp
+    int tpg = (p.B + resident - 1) / resident;
+    tpg = tpg > kRouterTok ? kRouterTok : tpg;
+    q.tok_per_group = tpg;
+    const int n_groups = (p.B + tpg - 1) / tpg;
+    cfg.gridDim = dim3(csize, n_groups < resident ? n_groups : resident, 1);
+    cfg.dynamicSmemBytes = (size_t)tpg * p.d * sizeof(float);
+  }
   cudaLaunchAttribute attr[2];
   attr[0].id = cudaLaunchAttributeClusterDimension;
   attr[0].val.clusterDim.x = csize;
@@ -280,7 +433,7 @@ cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
   attr[1].val.programmaticStreamSerializationAllowed = 1;
   cfg.attrs = attr;
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, router_kernel, q);
+  return batched ? cudaLaunchKernelEx(&cfg, router_batched_kernel, q) : cudaLaunchKernelEx(&cfg, router_kernel, q);
 }
 
 // One warp per token: x_j = q_p[pi[j]] (the prefetch distribution in descending order),

@@ -312,6 +312,19 @@ def test_config4_shape_tensor_core_batches(B, stride):
     print("config4-tc", B, rep, stats)
 
 
+@pytest.mark.parametrize("d,N,k,C,B", [(768, 64, 8, 24, 200),    # clusters of 8: groups of 8 tokens, two passes, a ragged last group
+                                        (512, 12, 3, 6, 250),     # clusters of 2: groups of 4 tokens, ragged
+                                        (1024, 33, 4, 10, 131),   # clusters of 8, groups of 8, one ragged group
+                                        (256, 5, 2, 3, 97)])      # one CTA per token
+def test_batched_router_group_shapes(d, N, k, C, B):
+    # the batched router / gate kernel walks groups of tokens per cluster: every token's ranking, budget, top-k and
+    # gates against the oracle for group counts above and below the number of clusters the GPU holds
+    cfg = synth.tiny_config(d=d, N=N, k=k, I=128, C=C, T=2, sigma_p=1.0, cfg_id=300 + N)
+    for mode in ("exact", "stall_free"):
+        rep, stats = _run(cfg, mode=mode, tau=0.8, T=2, B=B, ffn_token_stride=max(1, B // 8))
+        assert stats["tokens"] == 2 * B and stats["routed"] == 2 * B * k
+
+
 # ------------------------------------------------------------------ API behaviour
 def test_decode_token_matches_per_call_sequence_and_counts_launches():
     cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=6, L=2, T=4, cfg_id=218)

@@ -1,18 +1,24 @@
 // ffn_plan_kernel: the execution sets of a batched step (B > 1) and the (expert, token) pair list sorted by expert,
 // for the tensor-core grouped GEMMs and for the per-pair streaming kernel.
+#include <cooperative_groups.h>
+
 #include "apex_internal.hpp"
 #include "ptx.cuh"
 #include "timeline.cuh"
 #include "token_plan.cuh"
 
+namespace cg = cooperative_groups;
+
 namespace apex {
 
 // ---------------------------------------------------------------- batched plan (B > 1)
-// One CTA of 32 warps.  Phase A: warp w plans tokens w, w+32, ... (all global loads of a warp's tokens
-// are issued before the first use).  Phase B: warp w owns experts w and w+32 and gathers the tokens
-// that execute them with ballots, so the pair list is sorted by (expert, token).  Shared-expert pairs
-// (expert id N) follow.
-constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;  // instantiated for 1, 2, 4 and 8 tokens per warp
+// A cluster of ceil(B / 32) CTAs (at most 8) of 32 warps.  Phase A: every warp of the cluster plans one token (planning
+// a token costs a warp 2-3 us of dependent latency, so eight tokens per warp on one SM were 16 us at B = 256) and puts
+// its execution mask and gates into the leader CTA's shared memory through distributed shared memory.  Phase B, leader
+// CTA only: warp w owns experts w and w+32 and gathers the tokens that execute them with ballots, so the pair list is
+// sorted by (expert, token).  Shared-expert pairs (expert id N) follow.
+constexpr int kPlanMaxCtas = APEX_MAX_BATCH / 32;
+static_assert(kPlanMaxCtas <= 8, "one token per warp needs a cluster of at most 8 CTAs");
 
 #ifdef APEX_TIMELINE
 #define PTL(i) do { if (threadIdx.x == 0) g_timeline[1000 * 16 + (i)] = globaltimer_ns_raw(); } while (0)
@@ -20,8 +26,10 @@ constexpr int kPlanMaxTokPerWarp = APEX_MAX_BATCH / 32;  // instantiated for 1, 
 #define PTL(i) do { } while (0)
 #endif
 
-template <int TOK_PER_WARP>
 __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
+  constexpr int TOK_PER_WARP = 1;
+  cg::cluster_group cluster = cg::this_cluster();
+  const unsigned crank = cluster.block_rank();
   __shared__ unsigned long long s_exec[APEX_MAX_BATCH];
   __shared__ float s_pgate[APEX_MAX_BATCH][APEX_MAX_TOPK];  // gate of the j-th executed expert of each token
   __shared__ int s_count[APEX_MAX_EXPERTS + 1];
@@ -29,17 +37,20 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
   const int N = p.N, k = p.k, B = p.B;
   int my_subst = 0, my_hits = 0;
+  // the leader's copies of the per-token results
+  unsigned long long* l_exec = cluster.map_shared_rank(&s_exec[0], 0);
+  float* l_pgate = cluster.map_shared_rank(&s_pgate[0][0], 0);
   SPAN_BEGIN();
   PTL(0);
   TokenLoads tls[TOK_PER_WARP];
 #pragma unroll
   for (int j = 0; j < TOK_PER_WARP; ++j) {
-    const int b = warp + j * nwarp;
+    const int b = (int)crank * nwarp + warp + j * nwarp * (int)cluster.num_blocks();
     if (b < B) tls[j] = load_token(p.idx + (size_t)b * k, p.z_r + (size_t)b * N, p.alpha + (size_t)b * N, N, k, p.mode, lane);
   }
 #pragma unroll
   for (int j = 0; j < TOK_PER_WARP; ++j) {
-    const int b = warp + j * nwarp;
+    const int b = (int)crank * nwarp + warp + j * nwarp * (int)cluster.num_blocks();
     if (b >= B) break;
     const TokenLoads& tl = tls[j];
     const TokenPlan tp = plan_token(tl, p.mode, p.norm_topk, p.snap.resident_mask, lane);
@@ -59,22 +70,23 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
       my_subst += __popcll(tp.exec_mask & ~tp.kr_mask);
       my_hits += __popcll(tp.kr_mask & p.snap.resident_mask);
     }
-    if (lane == 0) s_exec[b] = tp.exec_mask;
+    if (lane == 0) l_exec[b] = tp.exec_mask;
     {
       const int e0 = lane, e1 = lane + 32;
       if ((tp.exec_mask >> e0) & 1) {
         const int pos = __popcll(tp.exec_mask & ((1ull << e0) - 1ull));
-        if (pos < APEX_MAX_TOPK) s_pgate[b][pos] = tp.g0;
+        if (pos < APEX_MAX_TOPK) l_pgate[b * APEX_MAX_TOPK + pos] = tp.g0;
       }
       if ((tp.exec_mask >> e1) & 1) {
         const int pos = __popcll(tp.exec_mask & ((1ull << e1) - 1ull));
-        if (pos < APEX_MAX_TOPK) s_pgate[b][pos] = tp.g1;
+        if (pos < APEX_MAX_TOPK) l_pgate[b * APEX_MAX_TOPK + pos] = tp.g1;
       }
     }
   }
   if (p.post_exec && lane == 0 && my_subst && p.stats) atomicAdd(&p.stats->substitutions, (unsigned long long)my_subst);
   if (p.post_exec && lane == 0 && my_hits && p.stats) atomicAdd(&p.stats->hits_R, (unsigned long long)my_hits);
-  __syncthreads();
+  cluster.sync();  // every token's mask and gates are in the leader's shared memory
+  if (crank != 0) return;
   PTL(1);
   // ---- phase B, counts: warp w counts the tokens of experts w and w + 32
   for (int e = warp; e < N; e += nwarp) {
@@ -185,14 +197,20 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
 }
 
 cudaError_t launch_ffn_plan(const FfnParams& p, cudaStream_t s) {
-  // a small batch gets the instantiation with the short planning loop: the kernel runs once per layer-step on a
-  // single SM with a cold instruction cache, so its length in instructions shows
-  static_assert(kPlanMaxTokPerWarp == 8, "the dispatch below covers up to eight tokens per warp");
-  if (p.B <= 32) ffn_plan_kernel<1><<<1, 1024, 0, s>>>(p);
-  else if (p.B <= 64) ffn_plan_kernel<2><<<1, 1024, 0, s>>>(p);
-  else if (p.B <= 128) ffn_plan_kernel<4><<<1, 1024, 0, s>>>(p);
-  else ffn_plan_kernel<8><<<1, 1024, 0, s>>>(p);
-  return cudaGetLastError();
+  int n_cta = (p.B + 31) / 32;
+  n_cta = n_cta < 1 ? 1 : (n_cta > kPlanMaxCtas ? kPlanMaxCtas : n_cta);
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(n_cta, 1, 1);
+  cfg.blockDim = dim3(1024, 1, 1);
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = n_cta;
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, ffn_plan_kernel, p);
 }
 
 }  // namespace apex

@@ -109,6 +109,11 @@ __device__ unsigned long long g_tc_tl[2][148][128];
 struct Group {
   int expert, pair_off, n_tok;
 };
+// One unit of work of a GEMM CTA: the (part of a) group, the M block and the K-tile range.
+struct UnitDesc {
+  int expert, pair_off, n_tok, blk, kt_begin, kt_end;
+};
+constexpr int kUnitChunk = 32;  // unit descriptors held in shared memory at a time
 __device__ __forceinline__ Group load_group(const int32_t* grp, int g) {
   Group r;
   r.expert = grp[4 + 3 * g];
@@ -171,6 +176,8 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int s_abort;
+  __shared__ UnitDesc s_unit[kUnitChunk];
+  __shared__ unsigned long long s_ready_mask;  // experts whose slot was seen ready in the prologue
   __shared__ int s_ustart[APEX_MAX_EXPERTS + 3];  // first unit of each group
   __shared__ int32_t s_grp[4 + 3 * (APEX_MAX_EXPERTS + 1)];
 
@@ -198,11 +205,29 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
+  // Slot-ready flags of all resident experts in one round of loads (neither the flags nor the snapshot come from the
+  // preceding kernel): the producers then skip the per-unit check, a system-scope load and a proxy fence on their path
+  // at every unit boundary, for every expert already seen ready here.
+  if (warp == 0) {
+    bool r0 = false, r1 = false;
+    const int e0 = lane, e1 = lane + 32;
+    if (e0 < N) {
+      const int sl = p.f.snap.expert_slot[e0];
+      if (sl >= 0) r0 = (int32_t)(ld_acquire_sys(p.f.slot_ready + sl) - p.f.snap.need_gen[e0]) >= 0;
+    }
+    if (e1 < N) {
+      const int sl = p.f.snap.expert_slot[e1];
+      if (sl >= 0) r1 = (int32_t)(ld_acquire_sys(p.f.slot_ready + sl) - p.f.snap.need_gen[e1]) >= 0;
+    }
+    const unsigned m0 = __ballot_sync(0xffffffffu, r0), m1 = __ballot_sync(0xffffffffu, r1);
+    if (lane == 0) s_ready_mask = ((unsigned long long)m1 << 32) | m0;
+    asm volatile("fence.proxy.async;" ::: "memory");  // the tensor-map loads that follow the barrier read what the flags cover
+  }
   tc_fence_before();
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = tmem_base_s;
-  // everything above (barriers, TMEM, tensor-map prefetch) is independent of the preceding kernel
+  // everything above (barriers, TMEM, tensor-map prefetch, flags) is independent of the preceding kernel
   pdl_wait();
   pdl_launch_dependents();
 
@@ -233,20 +258,41 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
 
   uint32_t it_load = 0, it_mma = 0;  // running K-tile counters of the producer and of the MMA thread
   uint32_t unit_no = 0;              // units done by this CTA (phase of the TMEM barriers)
-  int g = 0;
-  for (int uu = blockIdx.x; uu < n_units; uu += gridDim.x) {
-    while (uu >= s_ustart[g + 1]) ++g;
-    Group gr = load_group(s_grp, g);
-    const int parts = (gr.n_tok + NMAX - 1) / NMAX;
-    const int local = uu - s_ustart[g];
+  // The units of this CTA (uu = blockIdx.x, + gridDim.x, ...) are described once, kUnitChunk at a time and a thread
+  // per unit: group lookup and index arithmetic are then off every role's path at the unit boundaries, where that
+  // cold code cost each role more than a microsecond per unit.
+  for (int chunk0 = blockIdx.x; chunk0 < n_units; chunk0 += (int)gridDim.x * kUnitChunk) {
+    if (tid < kUnitChunk) {
+      const int uu = chunk0 + tid * (int)gridDim.x;
+      UnitDesc ud = {};
+      if (uu < n_units) {
+        int g = 0;
+        while (uu >= s_ustart[g + 1]) ++g;
+        Group gr = load_group(s_grp, g);
+        const int parts = (gr.n_tok + NMAX - 1) / NMAX;
+        const int local = uu - s_ustart[g];
+        const bool shared = gr.expert >= N;
+        const int kch = shared ? kchunks_s : 1;
+        const int blk = local / (parts * kch), kc = (local / parts) % kch, sub = local % parts;
+        const int kdim = shared ? kdim_s : kdim_r;
+        ud.expert = gr.expert;
+        ud.pair_off = gr.pair_off + sub * NMAX;
+        ud.n_tok = gr.n_tok - sub * NMAX < NMAX ? gr.n_tok - sub * NMAX : NMAX;
+        ud.blk = blk;
+        ud.kt_begin = kch > 1 ? kc * (I / kKTile) : 0;  // K tiles of this unit
+        ud.kt_end = kch > 1 ? (ud.kt_begin + I / kKTile < kdim / kKTile ? ud.kt_begin + I / kKTile : kdim / kKTile) : kdim / kKTile;
+      }
+      s_unit[tid] = ud;
+    }
+    __syncthreads();
+  for (int uj = 0; uj < kUnitChunk && chunk0 + uj * (int)gridDim.x < n_units && !*(volatile int*)&s_abort; ++uj) {
+    const UnitDesc ud = s_unit[uj];
+    Group gr;
+    gr.expert = ud.expert;
+    gr.pair_off = ud.pair_off;
+    gr.n_tok = ud.n_tok;
     const bool shared = gr.expert >= N;
-    const int kch = shared ? kchunks_s : 1;
-    const int blk = local / (parts * kch), kc = (local / parts) % kch, sub = local % parts;
-    gr.pair_off += sub * NMAX;
-    gr.n_tok = gr.n_tok - sub * NMAX < NMAX ? gr.n_tok - sub * NMAX : NMAX;
-    const int kdim = shared ? kdim_s : kdim_r;
-    const int kt_begin = kch > 1 ? kc * (I / kKTile) : 0;                                    // K tiles of this unit
-    const int kt_end = kch > 1 ? (kt_begin + I / kKTile < kdim / kKTile ? kt_begin + I / kKTile : kdim / kKTile) : kdim / kKTile;
+    const int blk = ud.blk, kt_begin = ud.kt_begin, kt_end = ud.kt_end;
     const int n_pad = (gr.n_tok + 15) & ~15;                                  // MMA N
     const int n_loads = (gr.n_tok + kXRowsPerLoad - 1) / kXRowsPerLoad;       // 32-row boxes of the B tile
 
@@ -259,7 +305,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       if (!shared) {
         slot = p.f.snap.expert_slot[gr.expert];
         if (slot < 0) ok = false;
-        if (ok && lane == 0) {
+        if (ok && lane == 0 && !((s_ready_mask >> gr.expert) & 1ull)) {
           const uint32_t need = p.f.snap.need_gen[gr.expert];
           const uint32_t* flag = p.f.slot_ready + slot;
           if ((int32_t)(ld_acquire_sys(flag) - need) < 0) {
@@ -317,6 +363,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         // two accumulator buffers of 256 TMEM columns: this unit's MMAs run while the epilogue warps
         // still read the previous unit's
         const uint32_t buf = unit_no & 1u;
+        TCTL(PHASE, unit_no * 16 + 15);
         if (unit_no >= 2) ok = mbar_wait(&tmem_empty[buf], ((unit_no >> 1) - 1) & 1, &s_abort, p.f.wait_limit_ns);
         tc_fence_after();
         TCTL(PHASE, unit_no * 16);
@@ -350,6 +397,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         TCTL(PHASE, unit_no * 16 + 11);
         if (ok) umma_commit(&tmem_full[buf]);
         else atomicExch(&s_abort, 1);
+        TCTL(PHASE, unit_no * 16 + 14);
       }
     } else {
       // ================= epilogue: warp w owns TMEM lanes 32*(w%4) .. +31
@@ -399,6 +447,8 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     }
     ++unit_no;
     if (*(volatile int*)&s_abort) break;
+  }
+    __syncthreads();  // every role is done with this chunk's descriptors (after an abort the later chunks fall through)
   }
   tc_fence_before();
   __syncthreads();

@@ -263,9 +263,12 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   // cold code cost each role more than a microsecond per unit.
   for (int chunk0 = blockIdx.x; chunk0 < n_units; chunk0 += (int)gridDim.x * kUnitChunk) {
     if (tid < kUnitChunk) {
-      const int uu = chunk0 + tid * (int)gridDim.x;
+      // units are taken from the end of the list: the shared expert's (the widest token tiles, the longest epilogues)
+      // come first, so that their epilogues overlap later units instead of forming the tail of the launch
+      const int uf = chunk0 + tid * (int)gridDim.x;
+      const int uu = n_units - 1 - uf;
       UnitDesc ud = {};
-      if (uu < n_units) {
+      if (uf < n_units) {
         int g = 0;
         while (uu >= s_ustart[g + 1]) ++g;
         Group gr = load_group(s_grp, g);

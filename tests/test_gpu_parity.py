@@ -325,6 +325,14 @@ def test_batched_router_group_shapes(d, N, k, C, B):
         assert stats["tokens"] == 2 * B and stats["routed"] == 2 * B * k
 
 
+def test_tensor_core_path_more_units_than_one_descriptor_chunk():
+    # gate/up GEMM: 64 experts x 112 row blocks = 7168 units, i.e. 49 per CTA on 148 SMs: the kernel describes its units 32
+    # at a time, so this runs two chunks (the second one partial)
+    cfg = synth.tiny_config(d=256, N=64, k=16, I=14336, C=64, T=1, sigma_p=1.0, cfg_id=377)
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=1, B=256, ffn_token_stride=64)
+    assert stats["tokens"] == 256 and rep.ffn_checked >= 4
+
+
 # ------------------------------------------------------------------ API behaviour
 def test_decode_token_matches_per_call_sequence_and_counts_launches():
     cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=6, L=2, T=4, cfg_id=218)

@@ -65,12 +65,23 @@ def rank_desc(z: np.ndarray) -> np.ndarray:
 
 def min_adjacent_gap(z: np.ndarray, upto: Optional[int] = None) -> float:
     """Smallest gap between neighbours of z sorted descending, among the first `upto`
-    neighbours (all if None).  Used only to flag near-ties."""
+    neighbour pairs (all if None): pair j is (position j, position j+1), so upto = m covers the
+    order inside the first m positions and the boundary below position m.  Used only to flag
+    near-ties."""
     s = np.sort(np.asarray(z, dtype=np.float64))[::-1]
     g = s[:-1] - s[1:]
     if upto is not None:
         g = g[:upto]
     return float(g.min()) if len(g) else float("inf")
+
+
+def boundary_gap(z: np.ndarray, m: int) -> float:
+    """Gap between the m-th and the (m+1)-th largest value of z: the one comparison that decides
+    which m elements form the top-m SET.  inf when there is no such boundary (m <= 0 or m >= len)."""
+    s = np.sort(np.asarray(z, dtype=np.float64))[::-1]
+    if m <= 0 or m >= len(s):
+        return float("inf")
+    return float(s[m - 1] - s[m])
 
 
 # --------------------------------------------------------------------------------------
@@ -116,7 +127,8 @@ def select_budget(q_p: np.ndarray, pi: np.ndarray, w: np.ndarray, theta: np.ndar
             if theta[delta] - s >= t_tau:
                 d_hat = delta
                 break
-        margin = float(np.min(np.abs(theta - s - t_tau)))
+        # only the comparisons that were taken decide delta_hat: delta = 0 .. delta_hat
+        margin = float(np.min(np.abs(theta[:d_hat + 1] - s - t_tau)))
     uncapped = d_hat
     d_hat = min(d_hat, C - k)
     return {"delta_hat": d_hat, "uncapped": uncapped, "capped": int(uncapped > d_hat),
@@ -159,19 +171,32 @@ def covered(K_r: Sequence[int], P: Sequence[int]) -> bool:
 # Stall-free execution set (Algorithm 1) and gates
 # --------------------------------------------------------------------------------------
 def stall_free_set(K_r: Sequence[int], alpha: np.ndarray, K_p: Sequence[int]) -> List[int]:
-    """Algorithm 1.  K_p is the set of experts that are available (the paper's prefetched set;
-    with a persistent cache, the resident set).  Garbled spots are read as C = K_p minus K~ and
-    S = Top_{|M|}(C; alpha); Top ranks by (alpha descending, index ascending).  If fewer than
-    |M| candidates exist the set stays short (cannot happen while |K_p| >= k)."""
-    K_p = set(int(e) for e in K_p)
+    """Execution set of the stall-free mode (Sec. IV-E (2), Alg. 1), stated as one ordering: the
+    available experts K_p (the paper's prefetched set; with a persistent cache, the resident set)
+    are ordered by (routed first, then router weight alpha descending, then index ascending) and
+    the first k = |K_r| of them are executed.  Every available routed expert is kept (there are at
+    most k of them) and the places of the missing ones go to the best remaining available experts:
+    Alg. 1's candidate pool is K_p minus the kept experts and its Top is by (alpha, then index).
+    If fewer than k experts are available the set stays short (cannot happen while |K_p| >= k).
+    Returned in ascending expert index.  tests/test_oracle_pins.py proves this equal to the
+    step-by-step algorithm by brute force over all subsets."""
     alpha = np.asarray(alpha, np.float64)
-    if set(K_r) <= K_p:
-        return sorted(int(e) for e in K_r)
-    keep = [e for e in K_r if e in K_p]
-    missing = [e for e in K_r if e not in K_p]
-    cand = sorted(K_p - set(keep), key=lambda e: (-alpha[e], e))
-    subs = cand[:len(missing)]
-    return sorted(keep + subs)
+    routed = set(int(e) for e in K_r)
+    order = sorted(set(int(e) for e in K_p), key=lambda e: (0 if e in routed else 1, -alpha[e], e))
+    return sorted(order[:len(routed)])
+
+
+def substitution_margin(z_r: np.ndarray, K_r: Sequence[int], K_p: Sequence[int]) -> float:
+    """Near-tie margin of Alg. 1's Top_{|M|}: the logit gap between the last substitute taken
+    and the best one left out (the order of alpha is the order of z_r).  inf when nothing is
+    substituted or every remaining available expert is taken."""
+    routed = set(int(e) for e in K_r)
+    avail = set(int(e) for e in K_p)
+    n_missing = len(routed - avail)
+    pool = sorted(avail - routed)
+    if n_missing == 0 or not pool:
+        return float("inf")
+    return boundary_gap(np.asarray(z_r, np.float64)[pool], n_missing)
 
 
 def gates(alpha: np.ndarray, K_exec: Sequence[int], norm_topk: bool = True) -> np.ndarray:
@@ -253,6 +278,12 @@ class SlotCache:
 
     def touch(self, e: int):
         self.slot_stamp[self.expert_slot[e]] = self.clock
+
+    def touch_all(self, experts: Sequence[int]):
+        """Recency update of a set of resident experts that were executed (stall-free mode: the
+        union of the execution sets; order is irrelevant, every stamp becomes the clock)."""
+        for e in sorted(set(int(x) for x in experts)):
+            self.touch(e)
 
     def _acquire(self, e: int, protect: set, deprioritise: set) -> Optional[Tuple[int, int]]:
         """Make e resident.  Returns (e, slot) if a copy is needed, None on a hit."""
@@ -337,8 +368,11 @@ def layer_step(cache: SlotCache, *, W_p, b_p, W_r, b_r, w, theta, tau: float, k:
     for b in range(B):
         z_p, q_p, pi = prefetch_scores(W_p, b_p, h[b])
         sel = select_budget(q_p, pi, w, theta, tau, k, cache.C)
+        # rank_margin decides the whole ranking pi; cand_margin only the ordered candidate list
+        # (order inside the first k + delta_hat positions and the boundary below them)
         tok = {"z_p": z_p, "q_p": q_p, "pi": pi, **sel,
-               "rank_margin": min_adjacent_gap(z_p)}
+               "rank_margin": min_adjacent_gap(z_p),
+               "cand_margin": min_adjacent_gap(z_p, upto=k + sel["delta_hat"])}
         out["tokens"].append(tok)
         P_sets.append(sel["P"])
     U, copies = cache.prefetch(P_sets)
@@ -375,17 +409,30 @@ def layer_step(cache: SlotCache, *, W_p, b_p, W_r, b_r, w, theta, tau: float, k:
         for tok in out["tokens"]:
             tok["K_exec"] = stall_free_set(tok["K_r"], tok["alpha"], R)
             tok["n_subst"] = len(set(tok["K_exec"]) - set(tok["K_r"]))
-            # near-tie accounting for the substitutes: gaps of z_r among available non-routed experts
-            cand = [e for e in R if e not in tok["K_r"]]
-            tok["subst_margin"] = min_adjacent_gap(tok["z_r"][cand]) if (tok["n_subst"] and len(cand) > 1) \
-                else float("inf")
+            tok["subst_margin"] = substitution_margin(tok["z_r"], tok["K_r"], R)
             used |= set(tok["K_exec"])
-        for e in sorted(used):
-            cache.touch(e)
+        cache.touch_all(used)
     else:
         raise ValueError(mode)
     for b, tok in enumerate(out["tokens"]):
         tok["gates"] = gates(tok["alpha"], tok["K_exec"], norm_topk)
         if compute_ffn and expert_weights is not None and (ffn_tokens is None or b in ffn_tokens):
             tok["y"] = moe_output(h_post[b], tok["K_exec"], tok["gates"], expert_weights, shared)
+    return out
+
+
+def near_tie_reasons(tok: Dict) -> List[str]:
+    """Which deciding comparisons of one token's step had a margin under the near-tie tolerance:
+    'cand' (order or boundary of the candidate list, z_p), 'threshold' (the test of Eq. (9)),
+    'route' (order or boundary of K_r, z_r), 'subst' (Alg. 1's Top boundary).  A GPU decision may
+    differ from the oracle's only where the matching reason is listed."""
+    out = []
+    if tok.get("cand_margin", float("inf")) < NEAR_TIE_LOGIT:
+        out.append("cand")
+    if tok.get("threshold_margin", float("inf")) < NEAR_TIE_THRESHOLD:
+        out.append("threshold")
+    if tok.get("route_margin", float("inf")) < NEAR_TIE_LOGIT:
+        out.append("route")
+    if tok.get("subst_margin", float("inf")) < NEAR_TIE_LOGIT:
+        out.append("subst")
     return out

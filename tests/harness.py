@@ -3,8 +3,12 @@
 Per layer-step the oracle is given the library's pre-step slot table, runs the step on the same
 inputs, and every decision is compared: ranking, budget, candidate set, slot plan, routed set,
 execution set, gates, demand plan, post-step table (bit-exact) and the FFN output (tolerance).
-A mismatch is excused only when the oracle flags the deciding comparison as a near-tie (logit gap
-below 1e-6, threshold margin below 1e-5); such steps are counted and reported."""
+A mismatch is excused only when the oracle flags THE comparison that decides it as a near-tie:
+a ranking position may hold another expert only if the two experts' logits differ by less than
+1e-6; the candidate list only by the z_p gaps up to its boundary k + delta_hat or the threshold
+margin (below 1e-5) of the comparisons Eq. (9) took; K_r only by the z_r gaps up to the boundary
+k; a substitute only by the boundary of Alg. 1's Top.  Such steps are counted, and the run fails
+when there are more of them than the caller allows (default: none)."""
 from __future__ import annotations
 
 import dataclasses
@@ -116,21 +120,26 @@ class Problem:
         return synth.split_store(w)
 
 
-def _excusable(tok, what: str) -> bool:
+def _excusable(tok, what: str, got=None) -> bool:
+    reasons = ao.near_tie_reasons(tok)
     if what == "rank":
-        return tok["rank_margin"] < ao.NEAR_TIE_LOGIT
+        # position by position: the expert the library ranked there and the oracle's must be tied
+        z = tok["z_p"]
+        return len(got) == len(tok["pi"]) and sorted(int(e) for e in got) == list(range(len(z))) and \
+            all(abs(float(z[int(a)]) - float(z[int(b)])) < ao.NEAR_TIE_LOGIT for a, b in zip(got, tok["pi"]))
     if what == "budget":
-        return tok["threshold_margin"] < ao.NEAR_TIE_THRESHOLD or tok["rank_margin"] < ao.NEAR_TIE_LOGIT
+        return "cand" in reasons or "threshold" in reasons
     if what == "route":
-        return tok["route_margin"] < ao.NEAR_TIE_LOGIT
+        return "route" in reasons
     if what == "exec":
-        return tok["subst_margin"] < ao.NEAR_TIE_LOGIT or tok["route_margin"] < ao.NEAR_TIE_LOGIT
+        return "subst" in reasons or "route" in reasons
     return False
 
 
 def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T: int, B: int = 1,
                  C: Optional[int] = None, norm_topk: bool = True, cache_reuse: bool = True,
-                 check_ffn_every: int = 1, use_prefetch: bool = True, t0: int = 0, ffn_token_stride: int = 1) -> Report:
+                 check_ffn_every: int = 1, use_prefetch: bool = True, t0: int = 0, ffn_token_stride: int = 1,
+                 max_near_ties: int = 0) -> Report:
     cfg = prob.cfg
     C = C or cfg.C
     N, k, d = cfg.N, cfg.k, cfg.d
@@ -184,7 +193,7 @@ def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T:
                     np.testing.assert_allclose(z_p[b], tok["z_p"], atol=2e-5, rtol=0)
                     np.testing.assert_allclose(q_p[b], tok["q_p"], atol=1e-6, rtol=1e-5)
                     if list(pi[b]) != list(tok["pi"]):
-                        assert _excusable(tok, "rank"), f"ranking differs t={t} l={l} b={b}"
+                        assert _excusable(tok, "rank", list(pi[b])), f"ranking differs t={t} l={l} b={b}"
                         excused = True
                     gP = [int(e) for e in g_cand[b][:g_ncand[b]]]
                     if gP != tok["P"] or g_ncand[b] != k + tok["delta_hat"]:
@@ -241,6 +250,8 @@ def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T:
                     rep.worst_max_abs = max(rep.worst_max_abs, mx)
                     rep.ffn_checked += 1
                     assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL, f"FFN output t={t} l={l} b={b}: rel-L2 {rel:.3e} max-abs {mx:.3e}"
+    print(f"lock-step: {rep.layer_steps} layer-steps, {rep.near_ties} excused as near-ties (allowed {max_near_ties})")
+    assert rep.near_ties <= max_near_ties, f"{rep.near_ties} near-tie steps, at most {max_near_ties} allowed: {rep}"
     return rep
 
 
@@ -255,7 +266,7 @@ def _oracle_step_without_prefetch(cache, W_r, b_r, k, h_post, mode, prob, layer,
     for b in range(B):
         z_r, K_r, alpha = ao.route_topk(W_r, b_r, h_post[b], k)
         out["tokens"].append({"z_r": z_r, "K_r": K_r, "alpha": alpha, "route_margin": ao.min_adjacent_gap(z_r, upto=k),
-                              "n_subst": 0, "subst_margin": float("inf")})
+                              "n_subst": 0, "subst_margin": float("inf"), "n_miss": sum(1 for e in K_r if e not in R)})
         Ks.append(K_r)
     if mode == "exact":
         missing, waves = cache.demand(Ks)
@@ -269,11 +280,9 @@ def _oracle_step_without_prefetch(cache, W_r, b_r, k, h_post, mode, prob, layer,
         for tok in out["tokens"]:
             tok["K_exec"] = ao.stall_free_set(tok["K_r"], tok["alpha"], R)
             tok["n_subst"] = len(set(tok["K_exec"]) - set(tok["K_r"]))
-            cand = [e for e in R if e not in tok["K_r"]]
-            tok["subst_margin"] = ao.min_adjacent_gap(tok["z_r"][cand]) if (tok["n_subst"] and len(cand) > 1) else float("inf")
+            tok["subst_margin"] = ao.substitution_margin(tok["z_r"], tok["K_r"], R)
             used |= set(tok["K_exec"])
-        for e in sorted(used):
-            cache.touch(e)
+        cache.touch_all(used)
     for b, tok in enumerate(out["tokens"]):
         tok["gates"] = ao.gates(tok["alpha"], tok["K_exec"], norm_topk)
         if do_ffn:

@@ -14,19 +14,21 @@ def _harness():
 
 
 def _run(cfg, *, mode, tau, T, B=1, layers=None, C=None, norm_topk=1, cache_reuse=1, check_ffn_every=1,
-         use_prefetch=True, prob=None, ffn_token_stride=1, flags=0):
+         use_prefetch=True, prob=None, ffn_token_stride=1, flags=0, max_near_ties=0):
     hz = _harness()
     prob = prob or hz.Problem(cfg, layers=layers)
     apex = prob.make_ctx(C=C, max_batch=B, norm_topk=norm_topk, cache_reuse=cache_reuse, flags=flags)
     try:
         rep = hz.run_lockstep(prob, apex, mode=mode, tau=tau, T=T, B=B, C=C, norm_topk=bool(norm_topk),
                               cache_reuse=bool(cache_reuse), check_ffn_every=check_ffn_every,
-                              use_prefetch=use_prefetch, ffn_token_stride=ffn_token_stride)
+                              use_prefetch=use_prefetch, ffn_token_stride=ffn_token_stride, max_near_ties=max_near_ties)
         stats = apex.get_stats()
     finally:
         apex.destroy()
+    assert rep.near_ties <= max_near_ties
     if use_prefetch and rep.near_ties == 0:
-        # S9: the device-side counters equal the oracle's metrics summed over the run
+        # S9: the device-side counters equal the oracle's metrics summed over the run (always, unless the caller
+        # allowed near-tie steps and some occurred: the library's counters then include steps the oracle's sums skip)
         for key in ("sum_delta_hat", "sum_delta_star", "sum_ncand", "hits_P", "hits_R", "covered", "capped"):
             assert stats[key] == getattr(rep, key), (key, stats[key], getattr(rep, key))
         assert stats["prefetch_copies"] == rep.n_prefetch_copies and stats["demand_copies"] == rep.n_demand_copies
@@ -41,7 +43,7 @@ def _run(cfg, *, mode, tau, T, B=1, layers=None, C=None, norm_topk=1, cache_reus
 def test_tiny_shapes_both_modes(d, N, k, I, C, mode):
     cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, T=12, sigma_p=1.0, cfg_id=200 + N)
     rep, stats = _run(cfg, mode=mode, tau=0.7, T=12)
-    assert rep.layer_steps == 12 and rep.ffn_checked + rep.near_ties >= 12
+    assert rep.layer_steps == 12 and rep.ffn_checked == 12 and rep.near_ties == 0
     assert stats["tokens"] == 12 and stats["routed"] == 12 * k
     if mode == "stall_free":
         assert rep.n_demand_copies == 0
@@ -106,7 +108,7 @@ def test_batched_tensor_core_path(B, mode):
     # shapes the tcgen05 grouped GEMM accepts (d, I, I_shared multiples of 128), B >= 16
     cfg = synth.tiny_config(d=256, N=12, k=3, I=128, C=8, T=3, I_shared=256, sigma_p=1.0, cfg_id=230)
     rep, stats = _run(cfg, mode=mode, tau=0.8, T=3, B=B)
-    assert stats["tokens"] == 3 * B and rep.ffn_checked + rep.near_ties >= 1
+    assert stats["tokens"] == 3 * B and rep.ffn_checked >= 1 and rep.near_ties == 0
     print("tc", B, mode, rep)
 
 
@@ -129,7 +131,7 @@ def _run_fp8(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1):
 def test_fp8_store_tiny_shapes(d, N, k, I, C, Ish, mode):
     cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, T=8, I_shared=Ish, sigma_p=1.0, cfg_id=260 + N)
     rep, stats = _run_fp8(cfg, mode=mode, tau=0.7, T=8)
-    assert rep.layer_steps == 8 and rep.ffn_checked + rep.near_ties >= 8
+    assert rep.layer_steps == 8 and rep.ffn_checked == 8 and rep.near_ties == 0
     assert stats["bytes_copied"] == (rep.n_prefetch_copies + rep.n_demand_copies) * I * (3 * d + 16)
     print("fp8", d, mode, rep)
 
@@ -162,7 +164,7 @@ def _run_fp4(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1):
 def test_fp4_store_tiny_shapes(d, N, k, I, C, Ish, mode):
     cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, T=8, I_shared=Ish, sigma_p=1.0, cfg_id=300 + N)
     rep, stats = _run_fp4(cfg, mode=mode, tau=0.7, T=8)
-    assert rep.layer_steps == 8 and rep.ffn_checked + rep.near_ties >= 8
+    assert rep.layer_steps == 8 and rep.ffn_checked == 8 and rep.near_ties == 0
     assert stats["bytes_copied"] == (rep.n_prefetch_copies + rep.n_demand_copies) * I * synth.fp4_row_bytes(d)
     print("fp4", d, mode, rep)
 
@@ -189,7 +191,7 @@ def test_speculative_fill_with_good_and_useless_predictor(sigma_p, mode):
     # gate's, so nearly every speculative copy is dropped and its stage refilled
     cfg = synth.tiny_config(d=1024, N=24, k=6, I=96, C=12, T=10, I_shared=32, sigma_p=sigma_p, cfg_id=280)
     rep, stats = _run(cfg, mode=mode, tau=0.6, T=10, flags=binding.FLAG_SPECULATE)
-    assert rep.layer_steps == 10 and rep.ffn_checked + rep.near_ties >= 10
+    assert rep.layer_steps == 10 and rep.ffn_checked == 10 and rep.near_ties == 0
     if sigma_p == 8.0:
         assert stats["hits_P"] < 0.8 * stats["routed"]
 
@@ -569,6 +571,7 @@ def test_config1_full_size_decode_token_sampled_layers(mode):
         hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
         y = torch.empty((cfg.L, 1, cfg.d), device="cuda")
         worst = 0.0
+        n_near = 0
         for t in range(T):
             pre = [apex.get_slot_table(l) for l in range(cfg.L)]
             apex.decode_token(h[t], hp[t], 1, 0.9, mode, y)
@@ -582,13 +585,13 @@ def test_config1_full_size_decode_token_sampled_layers(mode):
                 out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=0.9, k=cfg.k,
                                     h=hs[l][0][t], h_post=hs[l][1][t], mode=mode, expert_weights=prob.oracle_experts(l))
                 tok = out["tokens"][0]
-                near = (min(tok["rank_margin"], tok["route_margin"], tok["subst_margin"]) < ao.NEAR_TIE_LOGIT
-                        or tok["threshold_margin"] < ao.NEAR_TIE_THRESHOLD)
+                near = bool(ao.near_tie_reasons(tok))
                 post = apex.get_slot_table(l)
                 cp, dm = apex.get_last_copies(l)
                 same = (list(post[0]) == cache.expert_slot and list(post[1]) == cache.slot_stamp and post[2] == cache.clock
                         and cp == out["prefetch_copies"] and dm == out["demand_copies"])
                 assert same or near, f"slot decisions differ t={t} l={l}"
+                n_near += int(not same)
                 if same:
                     err = g_y[l, 0].astype(np.float64) - tok["y"]
                     rel = float(np.linalg.norm(err) / np.linalg.norm(tok["y"]))
@@ -596,7 +599,8 @@ def test_config1_full_size_decode_token_sampled_layers(mode):
                     assert rel <= hz.REL_L2_TOL and float(np.abs(err).max()) <= hz.MAX_ABS_TOL, (t, l, rel)
         st = apex.get_stats()
         assert st["tokens"] == T * cfg.L and st["timeouts"] == 0
-        print("config1 full", mode, "worst rel-L2", worst, st)
+        assert n_near == 0, f"{n_near} sampled layer-steps excused as near-ties"
+        print("config1 full", mode, "worst rel-L2", worst, "near-ties", n_near, st)
     finally:
         apex.destroy()
 
@@ -610,7 +614,7 @@ def test_config1_long_run_counts_near_ties():
     prob = hz.Problem(cfg, layers=1, cdf="fitted")
     apex = prob.make_ctx()
     try:
-        rep = hz.run_lockstep(prob, apex, mode="exact", tau=0.9, T=cfg.T, check_ffn_every=64)
+        rep = hz.run_lockstep(prob, apex, mode="exact", tau=0.9, T=cfg.T, check_ffn_every=64, max_near_ties=2)
     finally:
         apex.destroy()
     assert rep.layer_steps == 1024
@@ -626,15 +630,16 @@ def test_config1_long_run_stall_free_and_batched():
     prob = hz.Problem(cfg, layers=1, cdf="fitted")
     apex = prob.make_ctx()
     try:
-        rep = hz.run_lockstep(prob, apex, mode="stall_free", tau=0.9, T=cfg.T, check_ffn_every=64)
+        rep = hz.run_lockstep(prob, apex, mode="stall_free", tau=0.9, T=cfg.T, check_ffn_every=64, max_near_ties=2)
         st = apex.get_stats()
     finally:
         apex.destroy()
     assert rep.layer_steps == 1024 and rep.near_ties <= 2 and rep.n_demand_copies == 0
-    assert st["substitutions"] == rep.n_subst > 0
+    assert st["substitutions"] >= rep.n_subst > 0 and (rep.near_ties > 0 or st["substitutions"] == rep.n_subst)
     apex = prob.make_ctx(max_batch=8)
     try:
-        rep8 = hz.run_lockstep(prob, apex, mode="exact", tau=0.9, T=128, B=8, check_ffn_every=16, ffn_token_stride=3)
+        rep8 = hz.run_lockstep(prob, apex, mode="exact", tau=0.9, T=128, B=8, check_ffn_every=16, ffn_token_stride=3,
+                               max_near_ties=2)
     finally:
         apex.destroy()
     assert rep8.layer_steps == 128 and rep8.near_ties <= 2

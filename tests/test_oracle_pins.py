@@ -226,6 +226,146 @@ def test_stall_free_tie_break_prefers_lower_index():
     assert ao.stall_free_set([0, 4], alpha, [0, 2, 3]) == [0, 2]
 
 
+def _algorithm1_stepwise(K_r, alpha, avail):
+    """Alg. 1 as a procedure over sets, written for this test only: all routed experts available -> K_r; otherwise the
+    available routed ones stay and each missing one is replaced by the best expert (alpha, then lower index) still in
+    the pool of available, not yet chosen experts -- one replacement at a time."""
+    avail = set(avail)
+    chosen = [e for e in K_r if e in avail]
+    n_missing = len(K_r) - len(chosen)
+    for _ in range(n_missing):
+        pool = [e for e in avail if e not in chosen]
+        if not pool:
+            break
+        best = pool[0]
+        for e in pool[1:]:
+            if alpha[e] > alpha[best] or (alpha[e] == alpha[best] and e < best):
+                best = e
+        chosen.append(best)
+    return sorted(chosen)
+
+
+def test_stall_free_set_equals_algorithm1_taken_step_by_step():
+    rng = np.random.default_rng(81)
+    for trial in range(500):
+        N = int(rng.integers(2, 10)); k = int(rng.integers(1, N + 1))
+        # coarse values: many equal weights, so the index tie-break is exercised
+        alpha = rng.integers(1, 5, size=N).astype(np.float64); alpha /= alpha.sum()
+        K_r = [int(e) for e in ao.rank_desc(alpha)[:k]]
+        R = sorted(int(e) for e in rng.choice(N, size=int(rng.integers(1, N + 1)), replace=False))
+        assert ao.stall_free_set(K_r, alpha, R) == _algorithm1_stepwise(K_r, alpha, R)
+
+
+# ---------------------------------------------------------------- near-tie margins (they decide what the parity harness forgives)
+def test_min_adjacent_gap_is_the_closest_pair_and_respects_upto():
+    rng = np.random.default_rng(82)
+    for trial in range(300):
+        n = int(rng.integers(2, 10))
+        z = rng.standard_normal(n) if trial % 3 else rng.integers(-2, 3, size=n).astype(np.float64)
+        # all neighbours: the smallest distance between any two entries
+        brute = min(abs(z[i] - z[j]) for i in range(n) for j in range(i + 1, n))
+        assert ao.min_adjacent_gap(z) == pytest.approx(brute, abs=0)
+        # upto = m: pairs whose larger member is among the m largest entries (order inside the top m and its boundary)
+        order = [int(e) for e in ao.rank_desc(z)]
+        for m in range(0, n + 2):
+            top = order[:m]
+            pairs = [abs(z[a] - z[b]) for a in top for b in range(n) if b != a]
+            expect = min(pairs) if pairs else float("inf")
+            assert ao.min_adjacent_gap(z, upto=m) == pytest.approx(expect, abs=0)
+    assert ao.min_adjacent_gap(np.array([3.0, 1.0, 3.0])) == 0.0            # duplicated value
+    assert ao.min_adjacent_gap(np.array([3.0, 1.0, 3.0, 0.5]), upto=1) == 0.0
+    assert ao.min_adjacent_gap(np.array([5.0, 1.0, 1.0]), upto=1) == 4.0    # the tie lies below the first boundary
+    assert ao.min_adjacent_gap(np.array([2.0])) == float("inf")
+
+
+def test_boundary_gap_is_the_margin_of_the_top_m_set():
+    rng = np.random.default_rng(83)
+    for trial in range(300):
+        n = int(rng.integers(1, 9))
+        z = rng.standard_normal(n) if trial % 2 else rng.integers(-2, 3, size=n).astype(np.float64)
+        order = [int(e) for e in ao.rank_desc(z)]
+        for m in range(-1, n + 2):
+            inside, outside = order[:max(m, 0)], order[max(m, 0):]
+            expect = min((z[a] - z[b] for a in inside for b in outside), default=float("inf"))
+            assert ao.boundary_gap(z, m) == pytest.approx(expect, abs=0)
+            # moving every entry by less than half the gap cannot change the top-m set
+            if 0 < m < n and expect > 1e-9:
+                zz = z + rng.uniform(-0.49, 0.49, size=n) * expect
+                assert set(int(e) for e in ao.rank_desc(zz)[:m]) == set(inside)
+
+
+def test_threshold_margin_is_the_distance_to_a_different_budget():
+    rng = np.random.default_rng(84)
+    flipped = 0
+    for trial in range(400):
+        N = int(rng.integers(3, 12)); k = int(rng.integers(1, N)); C = N
+        q = ao.softmax(rng.standard_normal(N) * 2); pi = ao.rank_desc(q)
+        w = rng.standard_normal(N).astype(np.float32) * 3
+        theta = np.sort(rng.standard_normal(N - k + 1).astype(np.float32) * 2)
+        tau = float(rng.uniform(0.05, 0.99))
+        sel = ao.select_budget(q, pi, w, theta, tau, k, C)
+        # written out again with python floats: the comparisons Eq. (9) takes are delta = 0 .. delta_hat
+        s = sum(float(w[j]) * float(np.sort(q)[::-1][j]) for j in range(N))
+        t_tau = math.log(tau / (1.0 - tau))
+        brute = min(abs(float(theta[dl]) - s - t_tau) for dl in range(sel["uncapped"] + 1))
+        assert sel["threshold_margin"] == pytest.approx(brute, rel=1e-9, abs=1e-12)
+        m = sel["threshold_margin"]
+        if m < 1e-9:
+            continue
+        # a shift of the score by less than the margin leaves the budget alone ...
+        for sign in (-1.0, 1.0):
+            th2 = theta.astype(np.float64) + sign * 0.98 * m
+            assert ao.select_budget(q, pi, w, th2, tau, k, C)["delta_hat"] == sel["delta_hat"]
+        # ... and a shift just beyond it, in one of the two directions, changes it (unless the budget is the
+        # fall-back N - k that is taken when no comparison passes: failing one more comparison changes nothing)
+        d2 = {ao.select_budget(q, pi, w, theta.astype(np.float64) + sign * 1.02 * m, tau, k, C)["delta_hat"] for sign in (-1.0, 1.0)}
+        if sel["delta_hat"] < N - k:
+            assert d2 != {sel["delta_hat"]}
+            flipped += 1
+    assert flipped > 200
+    # comparisons beyond delta_hat are never taken and must not count: a threshold far above sits exactly on the test
+    q = ao.softmax(np.array([3.0, 1.0, 0.0, -1.0])); pi = ao.rank_desc(q)
+    t_tau = math.log(0.9 / 0.1)
+    sel = ao.select_budget(q, pi, np.zeros(4, np.float32), np.array([t_tau + 1.0, t_tau + 2.0, t_tau + 2.0 + 1e-9]), 0.9, 1, 4)
+    assert sel["delta_hat"] == 0 and sel["threshold_margin"] == pytest.approx(1.0)
+
+
+def test_substitution_margin_and_near_tie_reasons():
+    rng = np.random.default_rng(85)
+    for trial in range(300):
+        N = int(rng.integers(3, 9)); k = int(rng.integers(1, N))
+        z = rng.standard_normal(N) if trial % 2 else rng.integers(-2, 3, size=N).astype(np.float64)
+        alpha = ao.softmax(z)
+        K_r = [int(e) for e in ao.rank_desc(z)[:k]]
+        R = sorted(int(e) for e in rng.choice(N, size=int(rng.integers(k, N + 1)), replace=False))
+        K = ao.stall_free_set(K_r, alpha, R)
+        subs = [e for e in K if e not in K_r]
+        left = [e for e in R if e not in K_r and e not in K]
+        expect = min((z[a] - z[b] for a in subs for b in left), default=float("inf"))
+        assert ao.substitution_margin(z, K_r, R) == pytest.approx(expect, abs=0)
+    base = {"cand_margin": 1.0, "threshold_margin": 1.0, "route_margin": 1.0, "subst_margin": float("inf"), "rank_margin": 0.0}
+    assert ao.near_tie_reasons(base) == []                       # a tie elsewhere in the ranking excuses nothing
+    assert ao.near_tie_reasons({**base, "cand_margin": 9e-7}) == ["cand"]
+    assert ao.near_tie_reasons({**base, "threshold_margin": 9e-6}) == ["threshold"]
+    assert ao.near_tie_reasons({**base, "threshold_margin": 2e-5, "route_margin": 0.0, "subst_margin": 5e-7}) == ["route", "subst"]
+
+
+def test_layer_step_margins_follow_the_deciding_positions():
+    # a tie far down the prefetch ranking and one far down the router's ranking: neither decides anything
+    N, k, d = 8, 2, 8
+    W = np.zeros((N, d), np.float32)
+    for e, v in enumerate([5.0, 4.0, 3.0, 2.0, 1.0, 0.5, 0.0, 0.0]):       # experts 6 and 7 tie at the bottom
+        W[e, 0] = v
+    h = np.zeros((1, d), np.float32); h[0, 0] = 1.0
+    cache = ao.SlotCache(N, 4)
+    out = ao.layer_step(cache, W_p=W, b_p=None, W_r=W, b_r=None, w=np.zeros(N, np.float32),
+                        theta=np.linspace(-1, 5, N - k + 1).astype(np.float32), tau=0.6, k=k, h=h, h_post=h, mode="stall_free",
+                        compute_ffn=False)
+    tok = out["tokens"][0]
+    assert tok["rank_margin"] == 0.0 and tok["cand_margin"] == 1.0 and tok["route_margin"] == 1.0
+    assert ao.near_tie_reasons(tok) == []
+
+
 # ---------------------------------------------------------------- slot cache
 def test_slot_cache_hand_traced_example():
     # N=4, C=2.  Traced by hand from the replacement rule (smallest (stamp, slot) not protected).
@@ -245,6 +385,33 @@ def test_slot_cache_hand_traced_example():
     assert cp == [] and c.slot_stamp == [3, 2]
     miss, waves = c.demand([[0, 2]])            # both missing, C=2: one chunk; 0 -> slot1 (stamp 2 < 3), 2 -> slot0
     assert miss == [0, 2] and waves == [[(0, 1), (2, 0)]] and c.expert_slot == [1, -1, 0, -1]
+    # stall-free steps issue no demand copy; the executed experts are stamped instead.  Traced by hand:
+    c = ao.SlotCache(4, 3)
+    c.begin_step()                              # clock 1
+    c.prefetch([[0, 1, 2]])                     # slots 0, 1, 2 <- experts 0, 1, 2, all stamped 1
+    c.begin_step()                              # clock 2
+    U, cp = c.prefetch([[1]])                   # hit: slot1 stamp 2
+    c.touch_all([2, 1])                         # executed set {1, 2} (a substitute included): slots 1, 2 stamped 2
+    assert cp == [] and c.slot_stamp == [1, 2, 2]
+    c.begin_step()                              # clock 3
+    U, cp = c.prefetch([[3]])                   # the one slot not used last step (slot0, expert 0) is the victim
+    assert cp == [(3, 0)] and c.expert_slot == [-1, 1, 2, 0] and c.slot_stamp == [3, 2, 2]
+
+
+def test_stall_free_step_stamps_exactly_the_executed_experts():
+    cfg = synth.tiny_config(d=64, N=10, k=3, I=16, C=6, T=30, sigma_p=1.5)
+    W_r, b_r, W_p, b_p = synth.router_weights(cfg, 0)
+    w, theta = synth.handset_cdf_params(cfg)
+    h, hp = synth.hidden_states(cfg, 0, cfg.T, B=2)
+    cache = ao.SlotCache(cfg.N, cfg.C)
+    for t in range(cfg.T):
+        out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=0.5, k=cfg.k, h=h[t],
+                            h_post=hp[t], mode="stall_free", compute_ffn=False)
+        used = set(e for tok in out["tokens"] for e in tok["K_exec"])
+        planned = set(out["U"])
+        for e in cache.resident():
+            stamp = cache.slot_stamp[cache.expert_slot[e]]
+            assert (stamp == cache.clock) == (e in used or e in planned), (t, e)
 
 
 def test_slot_cache_invariants_random_walk():
@@ -298,14 +465,15 @@ def test_batched_prefetch_union_order_and_truncation():
 
 
 # ---------------------------------------------------------------- whole layer-step
-def _dense_topk_moe(W_r, b_r, hp, k, experts, shared):
+def _dense_topk_moe(W_r, b_r, hp, k, experts, shared, renormalise=True):
     """Written separately from the oracle, with torch fp64 ops: standard MoE layer that knows
-    nothing about prefetching or caches (softmax over all experts, top-k, renormalised gates)."""
+    nothing about prefetching or caches (softmax over all experts, top-k; gates renormalised over
+    the selected experts, or -- the other convention in use -- the plain softmax values)."""
     t = lambda a: torch.from_numpy(np.asarray(a, dtype=np.float64))
     logits = t(W_r) @ t(hp) + t(b_r)
     probs = torch.softmax(logits, 0)
     top = torch.topk(logits, k).indices
-    gate = probs[top] / probs[top].sum()
+    gate = probs[top] / probs[top].sum() if renormalise else probs[top]
     y = torch.zeros(len(hp), dtype=torch.float64)
     for g, e in zip(gate, top):
         Wg, Wu, Wd = (t(m) for m in experts(int(e)))
@@ -346,6 +514,21 @@ def test_exact_mode_equals_dense_topk_moe(tau, C, reuse):
         need = set(e for tok in out["tokens"] for e in tok["K_r"])
         if len(need) <= cfg.C:                  # otherwise the waves reuse slots within the step
             assert need <= set(cache.resident())
+
+
+def test_unnormalised_gates_equal_dense_moe_that_keeps_the_softmax_values():
+    cfg = synth.tiny_config(d=64, N=8, k=3, I=16, C=8, T=5, I_shared=8)
+    W_r, b_r, W_p, b_p, experts, shared, w, theta = _tiny_problem(cfg)
+    h, hp = synth.hidden_states(cfg, 0, cfg.T)
+    cache = ao.SlotCache(cfg.N, cfg.C)
+    for t in range(cfg.T):
+        out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=0.9, k=cfg.k, h=h[t],
+                            h_post=hp[t], mode="exact", expert_weights=experts, shared=shared, norm_topk=False)
+        tok = out["tokens"][0]
+        ref = _dense_topk_moe(W_r, b_r, hp[t, 0], cfg.k, experts, shared, renormalise=False)
+        np.testing.assert_allclose(tok["y"], ref, rtol=1e-10, atol=1e-13)
+        assert sum(tok["gates"]) < 1.0 - 1e-6                   # k < N: the weights do not sum to one
+        assert not np.allclose(tok["y"], _dense_topk_moe(W_r, b_r, hp[t, 0], cfg.k, experts, shared), rtol=1e-6, atol=1e-9)
 
 
 def test_stall_free_equals_exact_when_covered_and_differs_only_by_substitution():

@@ -70,6 +70,14 @@ extern "C" {
                                  directly, costs inside the decode loop, where the early copies delay the gate kernel; off by
                                  default */
 
+#define APEX_FLAG_HOST_WAVES 8 /* apex_config.flags: at B = 1 in exact mode a missing expert is NOT waited for inside the
+                                 running kernel; the first launch executes the resident routed experts and one further launch
+                                 per demand wave adds the rest (the scheme B > 1 always uses).  Needed wherever a kernel
+                                 launch does not return before the kernel has finished -- see apex_moe_ffn.  Set
+                                 automatically when the process runs with CUDA_LAUNCH_BLOCKING=1 or under a CUDA
+                                 injection tool (a profiler that serialises kernels), and after the first in-kernel wait
+                                 for a demand copy that ran out on this context */
+
 #define APEX_MAX_EXPERTS 64
 #define APEX_MAX_TOPK 16
 #define APEX_MAX_BATCH 256
@@ -125,6 +133,8 @@ typedef struct apex_step_stats {
  * Returns APEX_EINVAL for shapes outside the limits above, APEX_ENOMEM / APEX_ECUDA otherwise. */
 int apex_create(const apex_config* cfg, apex_ctx** out);
 int apex_destroy(apex_ctx* ctx);
+/* Text of the last error on this context.  With ctx == NULL: the reason the last apex_create on the calling
+ * thread failed (the context it was building no longer exists). */
 const char* apex_last_error(const apex_ctx* ctx);
 
 /* ---- parameters (host pointers, copied into library-owned device memory) ---------------- */
@@ -179,7 +189,12 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
  * missing expert and then executes it, at B > 1 further launches follow.  APEX_MODE_STALL_FREE executes
  * Algorithm 1 with K_p := the resident set.  exec_idx_dev [B][k] (ascending expert index) and
  * exec_gate_dev [B][k] may be NULL.  Device-side waits on slot-ready flags are bounded; when one
- * runs out the call (or the next call on this context) returns APEX_ETIMEOUT. */
+ * runs out the call (or the next call on this context) returns APEX_ETIMEOUT.
+ * Asynchronous launches are assumed at B = 1 in exact mode: the kernel waits for demand copies that this same
+ * call issues only after the launch has returned.  Where a launch blocks until the kernel is done
+ * (CUDA_LAUNCH_BLOCKING=1, a profiler or debugger that serialises kernels) that wait could only run out, so
+ * the context then uses APEX_FLAG_HOST_WAVES (detected at apex_create from the environment; it can also be
+ * set by hand): same results, one more launch per step that misses. */
 int apex_moe_ffn(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B, float* y_dev,
                  int32_t* exec_idx_dev, float* exec_gate_dev, void* stream);
 
@@ -237,6 +252,9 @@ int64_t apex_launch_count(const apex_ctx* ctx);
  * both escape the pool's accounting and stall the device.  No context is needed and nothing is
  * allocated or freed, here or in any library it calls.
  *   W_r_dev [N][d], b_r_dev [N] or NULL, hpost_dev [B][d]: device inputs, borrowed for the launch.
+ *   W_r_dev and b_r_dev must be complete in memory before the call is made, not merely ordered before it
+ *   on the stream: the kernel starts reading the weights while the kernel ahead of it on the stream may still
+ *   be finishing (hpost_dev, like every other input of this library, only needs stream order).
  *   idx_dev [B][k] (K_r in rank order) and alpha_dev [B][N] (softmax of the logits): device outputs.
  *   Limits: B <= APEX_STATIC_MAX_BATCH (64), N <= APEX_MAX_EXPERTS (64), k <= min(N, 16),
  *   d a multiple of 4 and d <= 4096.  Larger sizes are refused with APEX_EINVAL and a message.
@@ -245,7 +263,7 @@ int64_t apex_launch_count(const apex_ctx* ctx);
  * up the array's address on that device (make that first call outside any stream capture).  All
  * calls on a device share the array and it keeps the previous call's logits; the kernel overwrites
  * what it uses, so nothing has to be cleared, but two calls that overlap on the GPU (different
- * streams) race on it: serialise them.
+ * streams) race on it: serialise them.  First calls from several host threads are serialised inside.
  * err (optional, err_len bytes, caller-owned) receives a text on failure.  Returns APEX_OK,
  * APEX_EINVAL or APEX_ECUDA. */
 int apex_route_topk_static(const float* W_r_dev, const float* b_r_dev, const float* hpost_dev, int N, int d, int k,

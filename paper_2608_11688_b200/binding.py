@@ -21,6 +21,7 @@ MODES = {"exact": MODE_EXACT, "stall_free": MODE_STALL_FREE}
 FLAG_FP8_EXPERTS = 1
 FLAG_SPECULATE = 2
 FLAG_FP4_EXPERTS = 4
+FLAG_HOST_WAVES = 8
 ERR_NAMES = {0: "APEX_OK", -1: "APEX_EINVAL", -2: "APEX_ENOMEM", -3: "APEX_ECUDA", -4: "APEX_ETIMEOUT",
              -5: "APEX_ESTATE", -6: "APEX_ENOTIMPL"}
 
@@ -145,7 +146,7 @@ class Apex:
         h = C.c_void_p()
         rc = self.lib.apex_create(C.byref(self.cfg), C.byref(h))
         if rc != APEX_OK:
-            raise ApexError(rc, "apex_create failed")
+            raise ApexError(rc, self.lib.apex_last_error(None).decode() or "apex_create failed")
         self.h = h
         self._keep = []   # borrowed buffers that must outlive the context
 

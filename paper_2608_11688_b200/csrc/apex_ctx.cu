@@ -6,26 +6,56 @@ using namespace apex;
 
 extern "C" {
 
+namespace {
+// A kernel launch that does not return before the kernel has finished (CUDA_LAUNCH_BLOCKING, or a tool injected
+// into the CUDA runtime that serialises kernels) cannot be combined with a kernel that waits for the launching
+// thread's next action.
+bool launches_may_block() {
+  const char* b = getenv("CUDA_LAUNCH_BLOCKING");
+  if (b && *b && strcmp(b, "0") != 0) return true;
+  for (const char* name : {"CUDA_INJECTION64_PATH", "CUDA_INJECTION32_PATH", "NV_COMPUTE_PROFILER_PERFWORKS_DIR",
+                           "NV_NSIGHT_INJECTION_PORT_BASE", "NSIGHT_CUDA_DEBUGGER", "CUDA_DEBUGGER_SOFTWARE_PREEMPTION"}) {
+    const char* v = getenv(name);
+    if (v && *v) return true;
+  }
+  return false;
+}
+}  // namespace
+
 int apex_create(const apex_config* cfg, apex_ctx** out) {
-  if (!cfg || !out) return APEX_EINVAL;
+  create_error().clear();
+  if (!cfg || !out) {
+    create_error() = "apex_create: null argument";
+    return APEX_EINVAL;
+  }
   *out = nullptr;
   const apex_config& c = *cfg;
   if (c.N < 1 || c.N > APEX_MAX_EXPERTS || c.k < 1 || c.k > APEX_MAX_TOPK || c.k > c.N || c.C < c.k || c.C > c.N ||
       c.L < 1 || c.I < 1 || c.I_shared < 0 || c.max_batch < 1 || c.max_batch > APEX_MAX_BATCH || !ffn_shape_supported(c.d) ||
-      c.ctx_len < 0)
+      c.ctx_len < 0) {
+    create_error() = "apex_create: shape outside the limits of this build (see apex.h)";
     return APEX_EINVAL;
-  if (!(c.link_gbs >= 0.0)) return APEX_EINVAL;
+  }
+  if (!(c.link_gbs >= 0.0)) {
+    create_error() = "apex_create: link_gbs must be >= 0";
+    return APEX_EINVAL;
+  }
   // the kernels index (token, expert, intermediate index) rows with 31 bits
-  if ((long long)c.max_batch * (c.k + 1) * (long long)(c.I > c.I_shared ? c.I : c.I_shared) >= (1ll << 30)) return APEX_EINVAL;
+  if ((long long)c.max_batch * (c.k + 1) * (long long)(c.I > c.I_shared ? c.I : c.I_shared) >= (1ll << 30)) {
+    create_error() = "apex_create: max_batch * (k + 1) * I does not fit the kernels' row index";
+    return APEX_EINVAL;
+  }
   apex_ctx* ctx = new (std::nothrow) apex_ctx();
   if (!ctx) return APEX_ENOMEM;
   ctx->cfg = c;
+  ctx->host_waves = (c.flags & APEX_FLAG_HOST_WAVES) != 0 || launches_may_block();
   if (ctx->cfg.wait_limit_ns <= 0) ctx->cfg.wait_limit_ns = 2000000000ll;
   if (ctx->cfg.ctx_len == 0) ctx->cfg.ctx_len = 1024;
   const size_t L = c.L, N = c.N, C = c.C, d = c.d, MB = c.max_batch, k = c.k;
   const bool fp8 = (c.flags & APEX_FLAG_FP8_EXPERTS) != 0, fp4 = (c.flags & APEX_FLAG_FP4_EXPERTS) != 0;
   if ((fp8 && fp4) || ((fp8 || fp4) && !ffn_quantised_shape_supported(c.d))) {
     delete ctx;
+    create_error() = "apex_create: the quantised expert stores exclude each other and need d in {512, 1024, 1536, 2048, 4096}";
     return APEX_EINVAL;
   }
   ctx->fmt = fp4 ? 2 : (fp8 ? 1 : 0);
@@ -35,7 +65,7 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
 
   auto bail = [&](int code, const char* what, cudaError_t e) {
     fail(ctx, code, what, e);
-    fprintf(stderr, "apex_create: %s\n", ctx->err.c_str());
+    create_error() = ctx->err;
     apex_destroy(ctx);
     return code;
   };
@@ -195,7 +225,7 @@ int apex_destroy(apex_ctx* ctx) {
   return APEX_OK;
 }
 
-const char* apex_last_error(const apex_ctx* ctx) { return ctx ? ctx->err.c_str() : "null context"; }
+const char* apex_last_error(const apex_ctx* ctx) { return ctx ? ctx->err.c_str() : create_error().c_str(); }
 
 int apex_set_router(apex_ctx* ctx, int layer, const float* W, const float* b) {
   CHECK_CTX(ctx);

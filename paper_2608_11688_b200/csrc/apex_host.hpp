@@ -9,6 +9,8 @@
 #include <cstdlib>
 #include <cstring>
 #include <new>
+#include <string>
+#include <thread>
 #include <vector>
 
 #include "apex_internal.hpp"
@@ -70,21 +72,39 @@ inline int stream_write32(apex_ctx* ctx, cudaStream_t cs, uint32_t* dev, uint32_
   return APEX_OK;
 }
 
-// Bounded host wait for a mailbox sequence number.
+// Bounded host wait for a mailbox sequence number.  The records of the hit path arrive within microseconds, so the
+// first 50 us are a plain spin; after that the core is given up between polls (yield, then sleeps growing to 200 us),
+// so a wait behind a long copy or a stalled device does not burn a core until its limit.
 inline bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
   if ((int32_t)(*p - want) >= 0) return true;
   const auto t0 = std::chrono::steady_clock::now();
   const int64_t limit = ctx->cfg.wait_limit_ns * 2 + 1000000000ll;  // the device side gives up first
+  int64_t sleep_us = 0;
   for (uint32_t it = 0;; ++it) {
     if ((int32_t)(*p - want) >= 0) return true;
-    if ((it & 1023u) == 1023u) {
-      const int64_t ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
-      if (ns > limit) return false;
-    }
+    if (sleep_us == 0 && (it & 255u) != 255u) {
 #if defined(__x86_64__)
-    __builtin_ia32_pause();
+      __builtin_ia32_pause();
 #endif
+      continue;
+    }
+    const int64_t ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
+    if (ns > limit) return false;
+    if (ns < 50000) continue;
+    if (sleep_us == 0) {
+      sleep_us = 1;
+      std::this_thread::yield();
+    } else {
+      std::this_thread::sleep_for(std::chrono::microseconds(sleep_us));
+      sleep_us = sleep_us < 200 ? sleep_us * 2 : 200;
+    }
   }
+}
+
+// Why the last apex_create on this thread failed (the context it was building is gone by then).
+inline std::string& create_error() {
+  static thread_local std::string s;
+  return s;
 }
 
 // Copy machinery and device status (apex_step.cu)

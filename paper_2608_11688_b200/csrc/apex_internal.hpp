@@ -305,6 +305,7 @@ struct apex_ctx {
   int last_pred_layer = -1;             // layer whose prefetch stage (router, budget selection) was the last launch, else -1
   cudaEvent_t ev_wave = nullptr, ev_in = nullptr;
   int inject = 0;
+  bool host_waves = false;  // B = 1 exact mode: misses are corrected by further launches, not by a wait inside the kernel
   int64_t launches = 0;
   void* fn_write_value32 = nullptr;  // cuStreamWriteValue32 when the driver offers it
 };

@@ -114,7 +114,10 @@ int check_device_status(apex_ctx* ctx) {
   if (mhdr(ctx)->status != 0) {
     mhdr(ctx)->status = 0;
     release_withheld(ctx);
-    return fail(ctx, APEX_ETIMEOUT, "a device-side wait on a slot-ready flag ran out");
+    // If it was a wait for a demand copy inside the kernel, launches may not be asynchronous here (the copy is issued
+    // after the launch returns): from now on misses are corrected by further launches instead.
+    ctx->host_waves = true;
+    return fail(ctx, APEX_ETIMEOUT, "a device-side wait on a slot-ready flag or a demand copy ran out");
   }
   return APEX_OK;
 }
@@ -276,9 +279,19 @@ int apex_prefetch(apex_ctx* ctx, int layer, int B, void* copy_stream) {
     if (!ctx->tables[layer].plan_prefetch(cand, ncand, B, C, &copies)) return fail(ctx, APEX_ESTATE, "no evictable slot");
     ordered = copies;
   }
-  for (const auto& c : ordered) {
+  for (size_t i = 0; i < ordered.size(); ++i) {
+    const auto& c = ordered[i];
     int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->stream_of_slot(c.slot));
-    if (r != APEX_OK) return r;
+    if (r != APEX_OK) {
+      // The plan has already installed every candidate in the table.  What was not copied must not stay there as
+      // resident (the expert FFN would multiply by the previous occupant's bytes): those slots are left empty and
+      // the call can be repeated.
+      for (size_t j = i; j < ordered.size(); ++j) ctx->tables[layer].drop(ordered[j].expert);
+      ctx->host_stats[layer].prefetch_copies += (int64_t)i;
+      for (const auto& cc : copies)
+        if (ctx->tables[layer].expert_slot()[cc.expert] >= 0) ctx->last_copies[layer].push_back(cc);
+      return r;
+    }
   }
   ctx->host_stats[layer].prefetch_copies += (int64_t)copies.size();
   ctx->last_copies[layer].insert(ctx->last_copies[layer].end(), copies.begin(), copies.end());
@@ -458,7 +471,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.demand = ctx->d_demand + (size_t)layer * N;
   ctx->launch_tag = ctx->launch_tag % 0xfffffeu + 1u;
   p.demand_tag = ctx->launch_tag;
-  p.demand_in_kernel = (mode == APEX_MODE_EXACT && B == 1) ? 1 : 0;
+  p.demand_in_kernel = (mode == APEX_MODE_EXACT && B == 1 && !ctx->host_waves) ? 1 : 0;
   p.run_mask = p.demand_in_kernel ? ~0ull : p.snap.resident_mask;
   // Speculative first fill (opt-in): the kernel may start streaming the experts the prefetch router ranked
   // first before the gate's decision is visible.  Allowed when that ranking is certainly complete by
@@ -518,14 +531,21 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
     if (!tab.plan_demand(K_r, B, k, &copies, &need)) return fail(ctx, APEX_ESTATE, "no evictable slot");
     if (p.demand_in_kernel) {
       // the running kernel waits for these experts: copy, then publish (tag, slot)
-      for (const auto& c : copies) {
+      for (size_t i = 0; i < copies.size(); ++i) {
+        const auto& c = copies[i];
         const int prev = slot_expert_before[c.slot];
-        if (c.wave != 1 || (prev >= 0 && ((need >> prev) & 1))) return fail(ctx, APEX_ESTATE, "demand plan would evict an expert in use");
-        int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->stream_of_slot(c.slot));
-        if (r != APEX_OK) return r;
-        r = stream_write32(ctx, ctx->stream_of_slot(c.slot), ctx->d_demand + (size_t)layer * ctx->cfg.N + c.expert,
-                           (st.pend_tag << 8) | (uint32_t)c.slot);
-        if (r != APEX_OK) return r;
+        int r = APEX_OK;
+        if (c.wave != 1 || (prev >= 0 && ((need >> prev) & 1))) r = fail(ctx, APEX_ESTATE, "demand plan would evict an expert in use");
+        if (r == APEX_OK) r = issue_copy(ctx, layer, c.expert, c.slot, ctx->stream_of_slot(c.slot));
+        if (r == APEX_OK)
+          r = stream_write32(ctx, ctx->stream_of_slot(c.slot), ctx->d_demand + (size_t)layer * ctx->cfg.N + c.expert,
+                             (st.pend_tag << 8) | (uint32_t)c.slot);
+        if (r != APEX_OK) {
+          // experts whose copy was not issued (or not published) leave the table again; the running kernel's wait
+          // for them runs out and y stays incomplete: the caller sees the error and may repeat the expert FFN
+          for (size_t j = i; j < copies.size(); ++j) tab.drop(copies[j].expert);
+          return r;
+        }
       }
     } else {
       int n_waves = 0;
@@ -550,10 +570,16 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
             if (i == 0 || ctx->cur_copy_streams[i] != ctx->cur_copy_streams[0])
               CU_TRY(ctx, cudaStreamWaitEvent(ctx->cur_copy_streams[i], ctx->ev_wave, 0));
         }
-        for (const auto& c : copies)
+        for (size_t ci = 0; ci < copies.size(); ++ci) {
+          const auto& c = copies[ci];
           if (c.wave == w) {
             int r = issue_copy(ctx, layer, c.expert, c.slot, ctx->stream_of_slot(c.slot));
-            if (r != APEX_OK) return r;
+            if (r != APEX_OK) {
+              // (the plan lists the copies wave by wave) nothing from here on was copied: un-install it.  An expert of
+              // an earlier wave whose slot a later wave was going to reuse is no longer in the table either way.
+              for (size_t j = ci; j < copies.size(); ++j) tab.drop(copies[j].expert);
+              return r;
+            }
             const int prev = cur_slot_expert[c.slot];
             if (prev >= 0) {
               cur.expert_slot[prev] = -1;
@@ -564,6 +590,7 @@ int ffn_finalize(apex_ctx* ctx, int layer) {
             cur.need_gen[c.expert] = ctx->slot_gen[layer][c.slot];
             cur.resident_mask |= (1ull << c.expert);
           }
+        }
         FfnParams q = p;
         q.snap = cur;
         q.run_mask = chunk;

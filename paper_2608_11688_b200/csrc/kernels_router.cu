@@ -8,6 +8,8 @@
 // partial sums are combined by a 5-step xor-shuffle tree (offsets 16, 8, 4, 2, 1).
 #include <cooperative_groups.h>
 
+#include <mutex>
+
 #include "apex_internal.hpp"
 #include "ptx.cuh"
 
@@ -402,18 +404,24 @@ cudaError_t launch_router(const RouterParams& p, cudaStream_t s) {
     // rows in registers allow no more); further groups are walked by the same clusters
     static int n_sm_of[kMaxDevices];
     static bool configured[kMaxDevices];
+    static std::mutex setup_mutex;  // contexts of several host threads (and the context-free gate) share this set-up
     int dev = 0;
     cudaError_t e = cudaGetDevice(&dev);
     if (e != cudaSuccess) return e;
     if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
-    if (!configured[dev]) {
-      if ((e = cudaDeviceGetAttribute(&n_sm_of[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
-      if ((e = cudaFuncSetAttribute(router_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                    kRouterTok * kRouterMaxVec * 32 * (int)sizeof(float4))) != cudaSuccess)
-        return e;
-      configured[dev] = true;
+    int n_sm = 0;
+    {
+      std::lock_guard<std::mutex> lock(setup_mutex);
+      if (!configured[dev]) {
+        if ((e = cudaDeviceGetAttribute(&n_sm_of[dev], cudaDevAttrMultiProcessorCount, dev)) != cudaSuccess) return e;
+        if ((e = cudaFuncSetAttribute(router_batched_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                      kRouterTok * kRouterMaxVec * 32 * (int)sizeof(float4))) != cudaSuccess)
+          return e;
+        configured[dev] = true;
+      }
+      n_sm = n_sm_of[dev];
     }
-    int resident = n_sm_of[dev] / csize;
+    int resident = n_sm / csize;
     if (resident < 1) resident = 1;
     // small batches spread over the clusters (a token per cluster while they last); large ones fill the groups,
     // because a group costs a barrier and a round of shared-memory reads of all its tokens per warp

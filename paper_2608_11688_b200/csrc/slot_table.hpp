@@ -52,6 +52,16 @@ class SlotTable {
     if (e >= 0 && e < N_ && expert_slot_[e] >= 0) slot_stamp_[expert_slot_[e]] = clock_;
   }
 
+  // Takes e out of the table and leaves its slot empty (never used): for a planned install whose copy
+  // could not be issued.  The previous occupant was already taken out by the plan.
+  void drop(int e) {
+    if (e < 0 || e >= N_ || expert_slot_[e] < 0) return;
+    const int s = expert_slot_[e];
+    expert_slot_[e] = -1;
+    slot_expert_[s] = -1;
+    slot_stamp_[s] = -1;
+  }
+
   // Candidate lists of B tokens -> prefetch set U: experts ordered by (number of tokens that want
   // them descending, index ascending), truncated to C; planned in ascending index with U protected.
   // Returns false if no slot could be found (cannot happen while |U| <= C).

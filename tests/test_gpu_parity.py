@@ -75,6 +75,46 @@ def test_minimal_cache_C_equals_k():
     assert rep.n_subst > 0 and stats["substitutions"] == rep.n_subst
 
 
+@pytest.mark.parametrize("how", ["flag", "environment"])
+def test_exact_mode_with_host_side_miss_correction(how, monkeypatch):
+    # B = 1, exact mode, no wait for the host inside the kernel: resident routed experts first, one further launch per
+    # demand wave.  The setting for processes whose kernel launches block (it is chosen from the environment when the
+    # context is created).  Same decisions, same table, same output as the oracle.
+    cfg = synth.tiny_config(d=256, N=10, k=3, I=16, C=3, T=20, sigma_p=1.5, cfg_id=212)
+    if how == "environment":
+        monkeypatch.setenv("CUDA_LAUNCH_BLOCKING", "1")       # read by apex_create; the CUDA runtime of this process is already up
+    rep, stats = _run(cfg, mode="exact", tau=0.9, T=20, flags=binding.FLAG_HOST_WAVES if how == "flag" else 0)
+    assert rep.n_miss_steps > 0 and rep.ffn_checked == 20
+    assert stats["extra_waves"] == rep.n_miss_steps        # one more launch for every step that missed (C >= k: one wave)
+    assert stats["demand_copies"] == rep.n_demand_copies > 0 and stats["timeouts"] == 0
+    # through the pipelined whole-token call as well
+    hz = _harness()
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=4, L=3, T=5, sigma_p=1.5, cfg_id=231)
+    prob = hz.Problem(cfg)
+    hs = [synth.hidden_states(cfg, l, cfg.T, 1) for l in range(cfg.L)]
+    h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()
+    hp = torch.from_numpy(np.stack([x[1] for x in hs], 1)).cuda()
+    outs = []
+    for flags in (0, binding.FLAG_HOST_WAVES):
+        if how == "environment" and flags == 0:
+            monkeypatch.delenv("CUDA_LAUNCH_BLOCKING")
+        elif how == "environment":
+            monkeypatch.setenv("CUDA_LAUNCH_BLOCKING", "1")
+        apex = prob.make_ctx(flags=flags if how == "flag" else 0)
+        try:
+            y = torch.zeros((cfg.T, cfg.L, 1, cfg.d), dtype=torch.float32, device="cuda")
+            for t in range(cfg.T):
+                apex.decode_token(h[t], hp[t], 1, 0.8, "exact", y[t])
+            torch.cuda.synchronize()
+            st = apex.get_stats()
+            assert st["timeouts"] == 0 and (st["extra_waves"] > 0) == (flags != 0)
+            outs.append((y.cpu().numpy(), st["demand_copies"], [apex.get_slot_table(l)[0].tolist() for l in range(cfg.L)]))
+        finally:
+            apex.destroy()
+    assert outs[0][1] == outs[1][1] > 0 and outs[0][2] == outs[1][2]
+    np.testing.assert_allclose(outs[1][0], outs[0][0], rtol=0, atol=2e-6 * float(np.abs(outs[0][0]).max()))
+
+
 def test_load_use_evict_policy_and_unnormalised_gates():
     cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=7, T=12, sigma_p=1.0, cfg_id=213)
     rep, stats = _run(cfg, mode="stall_free", tau=0.8, T=12, cache_reuse=0)
@@ -495,6 +535,42 @@ def test_host_side_fault_hooks_copy_failure_and_withheld_flag():
         with pytest.raises(binding.ApexError) as ei:
             a.prefetch(0, 1)
         assert ei.value.code == binding.APEX_ECUDA
+        # the candidates whose copy was never issued must not count as resident: the same context goes on --
+        # prefetch again, gate, exact-mode FFN -- and the output is the dense top-k mixture of the oracle
+        from oracle import apex_oracle as ao
+        es, _, _ = a.get_slot_table(0)
+        cp, _ = a.get_last_copies(0)
+        assert sorted(e for e, s in enumerate(es) if s >= 0) == sorted(e for e, _ in cp)    # only what was really copied
+        a.prefetch(0, 1); a.attention_standin(0); a.route_topk(0, hpd[0], 1, idx, al)
+        a.moe_ffn(0, "exact", hpd[0], 1, y)
+        torch.cuda.synchronize()
+        W_r, b_r, _, _ = prob.routers[0]
+        _, K_r, alpha = ao.route_topk(W_r, b_r, hp[0, 0], cfg.k)
+        ref = ao.moe_output(hp[0, 0], K_r, ao.gates(alpha, K_r), prob.oracle_experts(0))
+        err = y[0].double().cpu().numpy() - ref
+        assert np.linalg.norm(err) / np.linalg.norm(ref) <= hz.REL_L2_TOL and np.abs(err).max() <= hz.MAX_ABS_TOL
+        assert sorted(idx[0].tolist()) == sorted(K_r)
+        # and a failure of a demand copy: the expert FFN reports it, the table does not keep the expert, a second
+        # attempt of the same layer-step's FFN completes
+        a.predict(0, hd[1], 1); a.select_candidates(0, 1, 0.0, cand, nc); a.prefetch(0, 1)
+        a.route_topk(0, hpd[1], 1, idx, al)
+        pre_es, _, _ = a.get_slot_table(0)
+        routed = idx[0].tolist()
+        if any(pre_es[e] < 0 for e in routed):                    # (seeded inputs: this step does miss)
+            a.test_inject(1)
+            with pytest.raises(binding.ApexError) as ei:
+                a.moe_ffn(0, "exact", hpd[1], 1, y)
+            assert ei.value.code in (binding.APEX_ECUDA, binding.APEX_ETIMEOUT)
+            torch.cuda.synchronize()
+            try:
+                a.moe_ffn(0, "exact", hpd[1], 1, y)
+            except binding.ApexError as e:     # the first attempt's wait that ran out, reported late; this attempt's work is queued in full
+                assert e.code == binding.APEX_ETIMEOUT
+            torch.cuda.synchronize()
+            _, K_r, alpha = ao.route_topk(W_r, b_r, hp[1, 0], cfg.k)
+            ref = ao.moe_output(hp[1, 0], K_r, ao.gates(alpha, K_r), prob.oracle_experts(0))
+            err = y[0].double().cpu().numpy() - ref
+            assert np.linalg.norm(err) / np.linalg.norm(ref) <= hz.REL_L2_TOL and np.abs(err).max() <= hz.MAX_ABS_TOL
         # 2: a slot-ready flag is withheld: the device-side wait runs out and the call reports it;
         # the context stays usable afterwards
         a2 = prob.make_ctx(wait_limit_ns=50_000_000)

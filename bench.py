@@ -31,9 +31,9 @@ NOMINAL_HBM_GBS = 8000.0
 FALLBACK_HBM_GBS = 6650.0
 TAU = 0.90
 
-# DRAM bytes per launch of the expert-FFN kernel (dram__bytes_read.sum + dram__bytes_write.sum) from
-# the ncu capture summarised in profiles/ (same kernel, same per-launch shape).  None = not captured.
-NCU_TRAFFIC_BYTES = {1: 37_854_500}   # profiles/moe_ffn_stream_kernel_config1.md: 37.809 MB read + ~0.045 MB written
+# DRAM bytes per launch (dram__bytes_read.sum + dram__bytes_write.sum) of the per-layer expert-FFN kernel from its ncu
+# capture on config 1 (37.809 MB read + 0.045 MB written).  None = not captured.
+NCU_TRAFFIC_BYTES = {1: 37_854_500}
 
 
 def measured_peak():
@@ -292,6 +292,33 @@ def time_ffn_kernel(apex, cfg, h, hp, B, tokens):
     return statistics.mean(per_launch) * 1e-3, statistics.median(per_launch) * 1e-3, len(per_launch) * cfg.L
 
 
+def time_token_kernel(cfg, prob, h, hp, y, tokens, standin):
+    """Average device time of one launch of the persistent token kernel (all L layer-steps of a token: prefetch
+    router, budget, gate, expert FFN, hand-over between layers), all experts resident, CUDA events on the launching
+    stream around `tokens` launches after a warm-up.  standin=False leaves the stand-in attention's bytes out, so the
+    launch moves the method's own bytes only."""
+    import torch
+    from paper_2608_11688_b200 import binding
+    a = make_ctx(cfg, prob, cfg.N, flags=0 if standin else binding.FLAG_SKIP_STANDIN)
+    try:
+        a.warm_all()
+        T = h.shape[0]
+        n0 = a.launch_count()
+        for t in range(4):
+            a.decode_token(h[t % T], hp[t % T], 1, TAU, "exact", y)
+        per_token = (a.launch_count() - n0) / 4
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(tokens):
+            a.decode_token(h[(4 + t) % T], hp[(4 + t) % T], 1, TAU, "exact", y)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) * 1e-3 / tokens, per_token
+    finally:
+        a.destroy()
+
+
 def oracle_tokens_per_s(cfg, prob, n_tokens):
     """The CPU oracle as it stands, timed on the host cores over n_tokens full decode tokens."""
     import torch
@@ -376,6 +403,10 @@ def main():
     ap.add_argument("--resident", action="store_true",
                     help="cache as large as the expert count, warmed up: no host-link copies (kernel launch lists)")
     ap.add_argument("--spec", action="store_true", help="A/B: expert FFN with the speculative first fill (FLAG_SPECULATE)")
+    ap.add_argument("--layer-launches", action="store_true",
+                    help="A/B: the per-layer kernel sequence instead of the persistent token kernel (FLAG_LAYER_LAUNCHES)")
+    ap.add_argument("--no-standin", action="store_true",
+                    help="leave the stand-in attention out of the decode step (FLAG_SKIP_STANDIN): the method's own bytes only")
     ap.add_argument("--fp8", action="store_true",
                     help="datatype study: e4m3 expert store with per-row scales (needs --ffn-only or --skip-extras)")
     ap.add_argument("--link-sweep", action="store_true",
@@ -428,6 +459,9 @@ def main():
         replicas.barrier()
         dist_sync = replicas.barrier
     B = args.batch
+    from paper_2608_11688_b200 import binding as _b
+    base_flags = (_b.FLAG_SPECULATE if args.spec else 0) | (_b.FLAG_LAYER_LAUNCHES if args.layer_launches else 0) | \
+                 (_b.FLAG_SKIP_STANDIN if args.no_standin else 0)
     prob = build_problem(cfg, dev, fp8=args.fp8, fp4=args.fp4)
     aux_info = None
     if args.train_aux:
@@ -443,7 +477,7 @@ def main():
     y_pin = torch.empty((cfg.L, B, cfg.d), dtype=torch.float32).pin_memory()
 
     if args.trace:
-        a = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B)
+        a = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B, flags=base_flags)
         if args.resident:
             a.warm_all()
         for t in range(args.warmup):
@@ -458,11 +492,16 @@ def main():
         per_layer = max(1, len(spans) // (n_tok * cfg.L))
         print(trace.format_spans(spans, limit=3 * per_layer + 2), file=sys.stderr)
         summary = trace.summarize(spans)
-        phases = trace.ffn_phase_medians(trace.read_ffn_cta_stamps(trace_lib, torch.cuda.get_device_properties(dev).multi_processor_count)) if B == 1 else {}
+        persistent = trace.KERNEL_NAMES[10] in summary
+        n_sm = torch.cuda.get_device_properties(dev).multi_processor_count
+        phases = trace.ffn_phase_medians(trace.read_ffn_cta_stamps(trace_lib, n_sm)) if (B == 1 and not persistent) else {}
+        dec = trace.decode_phase_medians(trace.read_decode_stamps(trace_lib, n_sm, cfg.L)) if persistent else {}
+        if persistent:
+            print(trace.format_decode_phases(dec), file=sys.stderr)
         print(json.dumps({"trace": summary, "tokens_traced": n_tok, "layers": cfg.L, "B": B,
                           "us_per_layer_step": summary["_all"]["wall_us"] / (n_tok * cfg.L),
-                          "ffn_cta_phase_median_cycles": phases, "config": f"config{cfg.cfg_id}",
-                          "resident": bool(args.resident)}), flush=True)
+                          "ffn_cta_phase_median_cycles": phases, "persistent_kernel_phase_median_us": dec,
+                          "config": f"config{cfg.cfg_id}", "resident": bool(args.resident)}), flush=True)
         a.destroy()
         return
 
@@ -501,7 +540,7 @@ def main():
         return
 
     # ---- headline: config cache size, exact (correctness-preserving) mode, inputs resident in HBM
-    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B, flags=2 if args.spec else 0)
+    apex = make_ctx(cfg, prob, cfg.N if args.resident else cfg.C, max_batch=B, flags=base_flags)
     if args.resident:
         apex.warm_all()
     sampler = ClockSampler(local_rank)
@@ -563,14 +602,34 @@ def main():
                                       "frac_of_8TBs": bytes_step * cfg.L * args.steps / sec_res / 1e9 / NOMINAL_HBM_GBS,
                                       "frac_of_peak": bytes_step * cfg.L * args.steps / sec_res / 1e9 / peak}
             extras["exact"]["exposed_stall_us_per_token"] = (sec / args.steps - sec_res / args.steps) * 1e6
-            # ---- the dominant kernel alone
+            # ---- the per-layer expert-FFN kernel alone (the kernel behind apex_moe_ffn)
             mean_s, med_s, n_l = time_ffn_kernel(a3, cfg, h_dev, hp_dev, B, tokens=max(2, min(8, args.steps)))
             achieved = bytes_ffn / mean_s / 1e9
-            roof = {"bound": "hbm", "kernel": "moe_ffn_stream_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
-                    "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / NOMINAL_HBM_GBS,
-                    "traffic": NCU_TRAFFIC_BYTES.get(cfg.cfg_id), "algorithmic_bytes_per_launch": bytes_ffn,
-                    "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6, "launches_timed": n_l}
+            ffn_alone = {"bound": "hbm", "kernel": "moe_ffn_stream_kernel", "achieved": achieved, "peak": peak, "unit": "GB/s",
+                         "frac": achieved / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": achieved / NOMINAL_HBM_GBS,
+                         "traffic": NCU_TRAFFIC_BYTES.get(cfg.cfg_id), "algorithmic_bytes_per_launch": bytes_ffn,
+                         "us_per_launch_mean": mean_s * 1e6, "us_per_launch_median": med_s * 1e6, "launches_timed": n_l}
             a3.destroy()
+            roof = ffn_alone
+            if B == 1 and not (args.layer_launches or args.fp8 or args.fp4):
+                # ---- the dominant kernel of the decode step: the persistent token kernel, one launch = all L layer-steps.
+                # Algorithmic bytes per launch: L x (routed expert weights + shared FFN + both routers + h, h', y).
+                n_tok = max(8, min(32, args.steps))
+                sec_tok, per_token = time_token_kernel(cfg, prob, h_dev, hp_dev, y_dev, n_tok, standin=False)
+                if per_token == 1.0:   # (a context that fell back to per-layer launches has no such kernel)
+                    bytes_tok = cfg.L * (bytes_step + cfg.d * 4)
+                    ach = bytes_tok / sec_tok / 1e9
+                    sec_att, _ = time_token_kernel(cfg, prob, h_dev, hp_dev, y_dev, n_tok, standin=True)
+                    attn_bytes = (4 * cfg.d * cfg.d + 2 * 1024 * cfg.d) * 2
+                    roof = {"bound": "hbm", "kernel": "decode_token_kernel", "achieved": ach, "peak": peak, "unit": "GB/s",
+                            "frac": ach / peak, "peak_kind": f"of {peak_kind}", "frac_of_8TBs": ach / NOMINAL_HBM_GBS,
+                            "traffic": None, "algorithmic_bytes_per_launch": bytes_tok, "us_per_launch_mean": sec_tok * 1e6,
+                            "us_per_layer_step": sec_tok * 1e6 / cfg.L, "launches_timed": n_tok,
+                            "launch": f"one token = {cfg.L} layer-steps, all experts resident, stand-in attention left out",
+                            "with_standin": {"us_per_launch_mean": sec_att * 1e6, "bytes_per_launch": bytes_tok + cfg.L * attn_bytes,
+                                             "achieved": (bytes_tok + cfg.L * attn_bytes) / sec_att / 1e9,
+                                             "frac": (bytes_tok + cfg.L * attn_bytes) / sec_att / 1e9 / peak},
+                            "per_layer_ffn_kernel_alone": ffn_alone}
             # ---- the oracle on the host cores (bounded sample)
             tps, cores, dt = oracle_tokens_per_s(cfg, prob, args.cpu_baseline_tokens)
             cpu = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",

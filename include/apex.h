@@ -76,7 +76,15 @@ extern "C" {
                                  launch does not return before the kernel has finished -- see apex_moe_ffn.  Set
                                  automatically when the process runs with CUDA_LAUNCH_BLOCKING=1 or under a CUDA
                                  injection tool (a profiler that serialises kernels), and after the first in-kernel wait
-                                 for a demand copy that ran out on this context */
+                                 for a demand copy that ran out on this context.  APEX_ASYNC_LAUNCHES=1 in the environment
+                                 switches the detection off (for profiling a run in which nothing can miss) */
+
+#define APEX_FLAG_LAYER_LAUNCHES 16 /* apex_config.flags: apex_decode_token always runs its per-layer kernel sequence.  Without it
+                                       a batch-1 token over bf16 stores runs as ONE persistent kernel over all layers (the
+                                       same steps, the same results; no launch and no host round trip between layers on the
+                                       hit path), unless launches may block (see APEX_FLAG_HOST_WAVES) */
+#define APEX_FLAG_SKIP_STANDIN 32   /* apex_config.flags: apex_decode_token leaves the stand-in attention out (the hiding
+                                       window of Eq. (12) is then empty: for measuring the method's own bytes) */
 
 #define APEX_MAX_EXPERTS 64
 #define APEX_MAX_TOPK 16
@@ -210,6 +218,10 @@ int apex_moe_ffn_begin(apex_ctx* ctx, int layer, int mode, const float* hpost_de
 int apex_moe_ffn_end(apex_ctx* ctx, int layer);
 
 /* All L layers of one decode step, in the order above.  h_dev, hpost_dev, y_dev are [L][B][d].
+ * At B = 1 with bf16 expert stores the whole token is one cooperative kernel launch that loops over the layers
+ * (prefetch router, stand-in attention, gate, expert FFN as roles inside it; layers handed over through bounded
+ * device-side counters); the host thread only plans and issues copies from the records the kernel posts and, on the
+ * hit path, is never waited for.  Otherwise, and with APEX_FLAG_LAYER_LAUNCHES, one kernel sequence per layer.
  * tau < 0 skips the prefetch stage altogether: the "No Prefetch" baseline of Sec. V-A, where every
  * non-resident routed expert is loaded on the critical path (static over-fetch baselines are a
  * confidence model with w = 0 and a step in theta). */

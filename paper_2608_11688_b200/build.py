@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libapex.so")
 TRACE_LIB = os.path.join(HERE, "libapex_trace.so")   # the same sources with the kernels' time stamps compiled in (trace.py)
-SOURCES = ["apex_ctx.cu", "apex_step.cu", "apex_observe.cu", "kernels_router.cu", "kernels_ffn.cu", "kernels_plan.cu", "kernels_ffn_tc.cu", "apex_noalloc.cu", "fit_cdf.cu", "distill.cu"]
+SOURCES = ["apex_ctx.cu", "apex_step.cu", "apex_observe.cu", "apex_decode.cu", "kernels_decode.cu", "kernels_router.cu", "kernels_ffn.cu", "kernels_plan.cu", "kernels_ffn_tc.cu", "apex_noalloc.cu", "fit_cdf.cu", "distill.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "--use_fast_math=false"]
 

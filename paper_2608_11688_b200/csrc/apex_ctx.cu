@@ -11,6 +11,8 @@ namespace {
 // into the CUDA runtime that serialises kernels) cannot be combined with a kernel that waits for the launching
 // thread's next action.
 bool launches_may_block() {
+  const char* a = getenv("APEX_ASYNC_LAUNCHES");  // the caller vouches for asynchronous launches (e.g. a profiler capture of
+  if (a && *a && strcmp(a, "0") != 0) return false;  // a run that cannot miss: every expert resident)
   const char* b = getenv("CUDA_LAUNCH_BLOCKING");
   if (b && *b && strcmp(b, "0") != 0) return true;
   for (const char* name : {"CUDA_INJECTION64_PATH", "CUDA_INJECTION32_PATH", "NV_COMPUTE_PROFILER_PERFWORKS_DIR",
@@ -198,6 +200,14 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   ctx->host_stats.assign(L, apex_step_stats{});
   ctx->step.assign(L, apex_ctx::StepState{});
   ctx->ffn_params.assign(L, FfnParams{});
+  {
+    const int r = decode_setup(ctx);
+    if (r != APEX_OK) {
+      create_error() = ctx->err;
+      apex_destroy(ctx);
+      return r;
+    }
+  }
   *out = ctx;
   return APEX_OK;
 }
@@ -213,6 +223,7 @@ int apex_destroy(apex_ctx* ctx) {
                  ctx->d_h_stage, ctx->d_hp_stage, ctx->d_y_stage};
   for (void* p : dev)
     if (p) cudaFree(p);
+  decode_teardown(ctx);
   if (ctx->mbox) cudaFreeHost(ctx->mbox);
   if (ctx->pad_src) cudaFreeHost(ctx->pad_src);
   if (ctx->pad_dst) cudaFree(ctx->pad_dst);
@@ -286,6 +297,8 @@ int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights) {
   if (ctx->cfg.I_shared <= 0) return fail(ctx, APEX_EINVAL, "the context was created with I_shared = 0");
   if (!dev_weights || ((uintptr_t)dev_weights & 15)) return fail(ctx, APEX_EINVAL, "shared expert: null or unaligned");
   ctx->shared_dev[layer] = static_cast<const uint8_t*>(dev_weights);
+  if (ctx->d_shared_ptrs)
+    CU_TRY(ctx, cudaMemcpy(ctx->d_shared_ptrs + layer, &dev_weights, sizeof(void*), cudaMemcpyHostToDevice));
   if (ctx->tc_ok) {
     TcMaps& m = ctx->tc_shared_maps[layer];
     if (!tc_make_weight_map(m.ws_gateup, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1, ctx->shared_bytes, 128) ||

@@ -73,7 +73,7 @@ inline int stream_write32(apex_ctx* ctx, cudaStream_t cs, uint32_t* dev, uint32_
 }
 
 // Bounded host wait for a mailbox sequence number.  The records of the hit path arrive within microseconds, so the
-// first 50 us are a plain spin; after that the core is given up between polls (yield, then sleeps growing to 200 us),
+// first 50 us are a plain spin; after that the core is given up between polls (yield, then sleeps growing to 32 us),
 // so a wait behind a long copy or a stalled device does not burn a core until its limit.
 inline bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
   if ((int32_t)(*p - want) >= 0) return true;
@@ -91,12 +91,13 @@ inline bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
     const int64_t ns = std::chrono::duration_cast<std::chrono::nanoseconds>(std::chrono::steady_clock::now() - t0).count();
     if (ns > limit) return false;
     if (ns < 50000) continue;
+    if (mhdr(ctx)->status != 0) return false;  // a kernel gave up: what it was going to post will not come
     if (sleep_us == 0) {
       sleep_us = 1;
       std::this_thread::yield();
     } else {
       std::this_thread::sleep_for(std::chrono::microseconds(sleep_us));
-      sleep_us = sleep_us < 200 ? sleep_us * 2 : 200;
+      sleep_us = sleep_us < 32 ? sleep_us * 2 : 32;
     }
   }
 }
@@ -112,6 +113,13 @@ int issue_copy(apex_ctx* ctx, int layer, int e, int slot, cudaStream_t cs);
 int release_withheld(apex_ctx* ctx);
 SlotSnapshot make_snapshot(apex_ctx* ctx, int layer);
 int check_device_status(apex_ctx* ctx);
+
+// Persistent decode path (apex_decode.cu)
+int decode_setup(apex_ctx* ctx);
+void decode_teardown(apex_ctx* ctx);
+bool decode_persistent_usable(const apex_ctx* ctx, int B);
+int decode_token_persistent(apex_ctx* ctx, const float* h_dev, const float* hpost_dev, float tau, int mode, float* y_dev,
+                            cudaStream_t cs);
 
 }  // namespace apex
 

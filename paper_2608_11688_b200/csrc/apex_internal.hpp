@@ -171,6 +171,63 @@ struct TcMaps {          // opaque 128-byte CUtensorMap objects
   alignas(64) unsigned char w_gateup[128], w_down[128], ws_gateup[128], ws_down[128], xg[128], act[128], act_lo[128];
 };
 
+// Persistent decode kernel (kernels_decode.cu): all layers of one token in one cooperative launch.
+constexpr int kDecWarps = 8;
+constexpr int kDecThreads = kDecWarps * 32;
+constexpr int kDecCluster = 8;  // CTAs per cluster: CTA r owns the router rows of experts 8r .. 8r+7, so N <= 64
+// A layer's new slot table, published by the host in mapped memory after it has issued the prefetch copies of the step.
+struct DecodeHostSnap {
+  SlotSnapshot tab;
+  uint32_t seq;  // sequence number of the token the snapshot belongs to; written last
+  uint32_t pad[3];
+};
+// Records of one layer-step for the host, in mapped memory; each record is one aligned 16-byte store that carries the
+// token's sequence number.
+struct DecodeMbox {
+  uint32_t sel_rec[4];   // candidate set: mask lo, mask hi, k + delta_hat, sequence number
+  uint32_t kr_rec[4];    // routed set: mask lo, mask hi, sequence number, 0
+  uint32_t exec_rec[4];  // execution set: the same
+  uint32_t pad[4];
+  int32_t cand[APEX_MAX_EXPERTS];  // candidates in rank order (advisory: the order in which the copies are issued)
+};
+struct DecodeParams {
+  const float* h;       // [L][d] pre-attention states
+  const float* hpost;   // [L][d] post-attention states
+  float* y;             // [L][d], zero at launch
+  const float *W_p, *b_p, *W_r, *b_r;  // [L][N][d], [L][N] (zeros where a layer has no bias)
+  const float *w, *theta;               // [L][N], [L][N-k+1]
+  const uint8_t* cache;                 // [L][C][slot_stride]
+  const uint8_t* const* shared_w;       // [L] pointers (device array), or null
+  const uint32_t* slot_ready;           // [L][C]
+  const uint32_t* demand;               // [L][N]
+  const SlotSnapshot* tab;              // [L] slot tables as they stand at launch (device memory)
+  const uint8_t* opt;                   // [L] 1: the host expects this layer's table to stay as it is in this step
+  const DecodeHostSnap* snap;           // [L] mapped host memory
+  DecodeHostSnap* snap_dev;             // [L] device memory: the same, passed on by the one warp that reads the host's
+  DecodeMbox* mbox;                     // [L] mapped host memory
+  volatile uint32_t* mbox_status;
+  DevStats* stats;                      // [L]
+  float *zp_out, *qp_out;               // [N] of the layer processed last
+  int32_t* pi_out;                      // [N]
+  float *zr_out, *alpha_out;            // [L] rows of zr_stride floats
+  int32_t* idx_out;                     // [L] rows of idx_stride ints
+  int32_t *ncand_keep, *cand_dev, *ncand_dev;  // context scratch of the selection
+  unsigned long long* cand_rec;         // [L][2] device: candidate mask of the layer-step, then the token's sequence number
+  unsigned long long* bar;              // [L][2] device counters: CTAs done with the expert FFN / with the stand-in
+  unsigned long long bar_target;        // value both counters reach when every CTA of this launch has counted itself in
+  unsigned int* abort_flag;             // device word: somebody gave up
+  const uint8_t* attn;
+  size_t attn_bytes;
+  int attn_layers, run_attn;
+  uint32_t seq;                         // this token's sequence number
+  uint32_t demand_tag;
+  float t_tau;
+  int force, prefetching;
+  size_t slot_stride, zr_stride, idx_stride;
+  long long wait_limit_ns;
+  int d, N, k, I, I_shared, C, L, mode, norm_topk, cache_reuse, n_sm;
+};
+
 struct AttnParams {
   const uint4* buf;
   size_t n_vec;  // 16-byte vectors
@@ -192,6 +249,8 @@ bool tc_shape_supported(int d, int I, int I_shared);
 bool ffn_shape_supported(int d);
 bool ffn_quantised_shape_supported(int d);   // widths the e4m3 / e2m1 kernels were built for
 size_t ffn_row_bytes(int fmt, int d);        // bytes of one intermediate index (three vectors and their scales)
+int decode_max_clusters(int d);              // clusters of kDecCluster CTAs the current device holds at once (0: not supported)
+cudaError_t launch_decode(const DecodeParams& p, int n_clusters, cudaStream_t s);
 
 }  // namespace apex
 
@@ -304,6 +363,26 @@ struct apex_ctx {
   uintptr_t last_ffn_y_lo = 0, last_ffn_y_hi = 0;  // output range of the last streaming-kernel launch
   int last_pred_layer = -1;             // layer whose prefetch stage (router, budget selection) was the last launch, else -1
   cudaEvent_t ev_wave = nullptr, ev_in = nullptr;
+  // persistent decode kernel (B = 1): device copies of the slot tables, mapped snapshots and records, counters
+  int dec_clusters = 0;                       // clusters per launch; 0: the persistent path is not available
+  apex::SlotSnapshot* d_dec_tab = nullptr;    // [L]
+  uint8_t* d_dec_opt = nullptr;               // [L]
+  uint8_t* dec_opt_stage = nullptr;           // pinned [2][L]
+  std::vector<uint8_t> dec_opt_host, dec_opt_last;  // expectation per layer: now / as uploaded
+  apex::SlotSnapshot* dec_tab_stage = nullptr;  // pinned [2][L]: staging of the table upload
+  std::vector<apex::SlotSnapshot> dec_tab_last;  // what the device holds
+  bool dec_tab_valid = false;
+  int dec_stage_sel = 0;
+  apex::DecodeHostSnap* dec_snap = nullptr;   // mapped [L]
+  apex::DecodeHostSnap* d_dec_snap = nullptr; // device [L]
+  apex::DecodeMbox* dec_mbox = nullptr;       // mapped [L]
+  unsigned long long* d_dec_bar = nullptr;    // [L][2]
+  unsigned long long* d_dec_cand = nullptr;   // [L][2]
+  unsigned int* d_dec_abort = nullptr;
+  const uint8_t** d_shared_ptrs = nullptr;    // [L]
+  unsigned long long dec_epoch = 0;           // persistent launches since the counters were last cleared
+  uint32_t dec_seq = 0;
+  bool dec_dirty = false;                     // a launch gave up: counters and abort flag must be cleared before the next
   int inject = 0;
   bool host_waves = false;  // B = 1 exact mode: misses are corrected by further launches, not by a wait inside the kernel
   int64_t launches = 0;

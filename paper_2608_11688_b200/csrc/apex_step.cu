@@ -117,6 +117,7 @@ int check_device_status(apex_ctx* ctx) {
     // If it was a wait for a demand copy inside the kernel, launches may not be asynchronous here (the copy is issued
     // after the launch returns): from now on misses are corrected by further launches instead.
     ctx->host_waves = true;
+    ctx->dec_dirty = true;  // a persistent decode launch that gave up leaves its counters short
     return fail(ctx, APEX_ETIMEOUT, "a device-side wait on a slot-ready flag or a demand copy ran out");
   }
   return APEX_OK;
@@ -652,8 +653,11 @@ int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev,
                       void* stream) {
   CHECK_CTX(ctx);
   if (!h_dev || !hpost_dev || !y_dev || B < 1 || B > ctx->cfg.max_batch) return fail(ctx, APEX_EINVAL, "apex_decode_token: bad argument");
+  if (decode_persistent_usable(ctx, B))  // one persistent kernel over all layers
+    return decode_token_persistent(ctx, h_dev, hpost_dev, tau, mode, y_dev, (cudaStream_t)stream);
   const size_t step = (size_t)B * ctx->cfg.d;
   const size_t MB = ctx->cfg.max_batch, k = ctx->cfg.k, N = ctx->cfg.N;
+  const bool standin = !(ctx->cfg.flags & APEX_FLAG_SKIP_STANDIN);
   int r;
   for (int l = 0; l < ctx->cfg.L; ++l) {
     int32_t* idx = ctx->d_idx + (size_t)l * MB * k;
@@ -662,7 +666,7 @@ int apex_decode_token(apex_ctx* ctx, const float* h_dev, const float* hpost_dev,
     if (prefetching &&
         (r = predict_select_fused(ctx, l, h_dev + l * step, B, tau, ctx->d_cand, ctx->d_cand_ncand, (cudaStream_t)stream)) != APEX_OK)
       return r;
-    if ((r = apex_attention_standin(ctx, l, stream)) != APEX_OK) return r;
+    if (standin && (r = apex_attention_standin(ctx, l, stream)) != APEX_OK) return r;
     if ((r = apex_route_topk(ctx, l, hpost_dev + l * step, B, idx, alpha, stream)) != APEX_OK) return r;
     if (l > 0 && (r = ffn_finalize(ctx, l - 1)) != APEX_OK) return r;
     if (prefetching && (r = apex_prefetch(ctx, l, B, nullptr)) != APEX_OK) return r;

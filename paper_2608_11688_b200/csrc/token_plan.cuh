@@ -53,21 +53,11 @@ __device__ __forceinline__ TokenLoads load_token(const int32_t* __restrict__ idx
   }
   return t;
 }
-__device__ __forceinline__ TokenPlan plan_token(const TokenLoads& t, int mode, int norm_topk, unsigned long long resident,
-                                                int lane) {
+// Execution set from the routed set (Alg. 1 in stall-free mode; K~ = K_r otherwise).  z0, z1: logits of experts lane,
+// lane + 32 (read in stall-free mode only).
+__device__ __forceinline__ unsigned long long exec_set(unsigned long long kr, int mode, unsigned long long resident, float z0,
+                                                       float z1, int lane) {
   const int e0 = lane, e1 = lane + 32;
-  const int my_idx = t.my_idx;
-  const float al0 = t.al0, al1 = t.al1, z0 = t.z0, z1 = t.z1;
-  unsigned lo = 0, hi = 0;
-  if (my_idx >= 0) {
-    if (my_idx < 32)
-      lo = 1u << my_idx;
-    else
-      hi = 1u << (my_idx - 32);
-  }
-  lo = __reduce_or_sync(0xffffffffu, lo);
-  hi = __reduce_or_sync(0xffffffffu, hi);
-  const unsigned long long kr = ((unsigned long long)hi << 32) | lo;
   unsigned long long exec = kr;
   if (mode == APEX_MODE_STALL_FREE && (kr & ~resident) != 0ull) {
     const unsigned long long keep = kr & resident;
@@ -87,15 +77,34 @@ __device__ __forceinline__ TokenPlan plan_token(const TokenLoads& t, int mode, i
     const unsigned b0 = __ballot_sync(0xffffffffu, s0), b1 = __ballot_sync(0xffffffffu, s1);
     exec = keep | (((unsigned long long)b1 << 32) | b0);
   }
-  const bool x0 = (exec >> e0) & 1, x1 = (exec >> e1) & 1;
+  return exec;
+}
+// Gates of the executed experts: alpha_e / sum over K~ (norm_topk) or alpha_e; 0 for the others.
+__device__ __forceinline__ void exec_gates(unsigned long long exec, float al0, float al1, int norm_topk, int lane, float* g0,
+                                           float* g1) {
+  const bool x0 = (exec >> lane) & 1, x1 = (exec >> (lane + 32)) & 1;
   const float a0 = x0 ? al0 : 0.f, a1 = x1 ? al1 : 0.f;
   float denom = 1.f;
   if (norm_topk) denom = warp_sum(a0 + a1);
+  *g0 = a0 / denom;
+  *g1 = a1 / denom;
+}
+__device__ __forceinline__ TokenPlan plan_token(const TokenLoads& t, int mode, int norm_topk, unsigned long long resident,
+                                                int lane) {
+  const int my_idx = t.my_idx;
+  unsigned lo = 0, hi = 0;
+  if (my_idx >= 0) {
+    if (my_idx < 32)
+      lo = 1u << my_idx;
+    else
+      hi = 1u << (my_idx - 32);
+  }
+  lo = __reduce_or_sync(0xffffffffu, lo);
+  hi = __reduce_or_sync(0xffffffffu, hi);
   TokenPlan tp;
-  tp.exec_mask = exec;
-  tp.kr_mask = kr;
-  tp.g0 = a0 / denom;
-  tp.g1 = a1 / denom;
+  tp.kr_mask = ((unsigned long long)hi << 32) | lo;
+  tp.exec_mask = exec_set(tp.kr_mask, mode, resident, t.z0, t.z1, lane);
+  exec_gates(tp.exec_mask, t.al0, t.al1, norm_topk, lane, &tp.g0, &tp.g1);
   return tp;
 }
 

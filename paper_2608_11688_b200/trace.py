@@ -29,12 +29,21 @@ KERNEL_NAMES = {
     7: "gather (B > 1)",
     8: "gate/up GEMM (B > 1)",
     9: "down GEMM (B > 1)",
+    10: "persistent token kernel (all layers, B = 1)",
 }
 LOG_RECORDS = 4096
 # stamps of one CTA of the streaming expert-FFN kernel (index -> meaning); 0, 11, 12 are %globaltimer (ns), the others clock64
 FFN_CTA_STAMPS = {0: "entry (ns)", 1: "entry", 4: "dependency wait over", 10: "gate outputs loaded", 2: "plan done",
                   3: "first row consumed", 7: "last row consumed", 8: "partials combined", 9: "exit",
                   11: "dependency wait over (ns)", 12: "exit (ns)"}
+
+# stamps of one (CTA, layer) of the persistent token kernel, %globaltimer (ns); per CTA the warp that writes last wins
+DECODE_STAMPS = {0: "layer start", 15: "previous layer's counter passed (W_p row owners)", 1: "prefetch logit sent",
+                 2: "candidate mask out (poster)", 10: "candidate record posted to the host (poster)", 3: "own share of the stand-in landed",
+                 14: "stand-in and previous layer's counters passed (W_r row owners)", 4: "gate logit sent", 5: "gate logits complete",
+                 6: "execution set and row space planned", 7: "first expert row landed", 8: "last expert row consumed",
+                 11: "warps' partial y in shared memory", 12: "cluster's partial y complete", 13: "y added", 9: "layer counted in"}
+DECODE_STAMP_ORDER = (15, 1, 2, 10, 3, 14, 4, 5, 6, 7, 8, 11, 12, 13, 9)
 
 Span = Tuple[int, int, int]   # (kernel id, start ns, end ns)
 
@@ -52,6 +61,8 @@ def use_trace_library() -> C.CDLL:
     lib.apex_debug_reset_spans.restype = C.c_int
     lib.apex_debug_read_timeline.argtypes = [C.c_void_p, C.c_int]
     lib.apex_debug_read_timeline.restype = C.c_int
+    lib.apex_debug_read_decode_timeline.argtypes = [C.c_void_p]
+    lib.apex_debug_read_decode_timeline.restype = C.c_int
     return lib
 
 
@@ -135,3 +146,39 @@ def ffn_phase_medians(stamps: np.ndarray) -> Dict[str, float]:
     if used.size == 0:
         return {}
     return {n: float(np.median(used[:, b] - used[:, a])) for n, a, b in zip(names, order[:-1], order[1:])}
+
+
+def read_decode_stamps(lib: C.CDLL, n_ctas: int, n_layers: int) -> np.ndarray:
+    """[n_ctas][n_layers][16] stamps of the last persistent-kernel launch (see DECODE_STAMPS); 0 = not written."""
+    buf = np.zeros((160, 64, 16), np.uint64)
+    rc = lib.apex_debug_read_decode_timeline(buf.ctypes.data)
+    if rc != 0:
+        raise RuntimeError(f"apex_debug_read_decode_timeline: CUDA error {rc}")
+    return buf[:min(n_ctas, 160), :min(n_layers, 64)].astype(np.int64)
+
+
+def decode_phase_medians(stamps: np.ndarray) -> Dict[str, float]:
+    """Per stamp: median over CTAs and layers (first and last layer left out) of the microseconds since the CTA's own
+    layer start; plus the median layer period."""
+    if stamps.shape[1] < 3:
+        return {}
+    out: Dict[str, float] = {}
+    inner = stamps[:, 1:-1]
+    for i in DECODE_STAMP_ORDER:
+        ok = (inner[:, :, i] > 0) & (inner[:, :, 0] > 0)
+        if ok.any():
+            out[DECODE_STAMPS[i]] = float(np.median((inner[:, :, i] - inner[:, :, 0])[ok])) / 1e3
+    start = stamps[:, :, 0]
+    ok = (start[:, 1:] > 0) & (start[:, :-1] > 0)
+    if ok.any():
+        out["layer period"] = float(np.median((start[:, 1:] - start[:, :-1])[ok])) / 1e3
+    return out
+
+
+def format_decode_phases(ph: Dict[str, float]) -> str:
+    if not ph:
+        return "(no persistent-kernel stamps recorded)"
+    lines = ["%-66s %9s" % ("persistent token kernel: event (median over CTAs and layers)", "us")]
+    for k, v in ph.items():
+        lines.append("%-66s %9.2f" % (k, v))
+    return "\n".join(lines)

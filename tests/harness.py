@@ -288,3 +288,86 @@ def _oracle_step_without_prefetch(cache, W_r, b_r, k, h_post, mode, prob, layer,
         if do_ffn:
             tok["y"] = ao.moe_output(h_post[b], tok["K_exec"], tok["gates"], prob.oracle_experts(layer), prob.oracle_shared(layer))
     return out
+
+
+def run_decode_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T: int, B: int = 1,
+                        C: Optional[int] = None, norm_topk: bool = True, cache_reuse: bool = True,
+                        layers_checked=None, ffn_token_stride: int = 1, max_near_ties: int = 0, host_buffers: bool = False) -> Report:
+    """The same lock-step comparison through apex_decode_token (all layers of a token in one call: the persistent
+    kernel at B = 1, the pipelined per-layer sequence otherwise).  Before every token the slot tables of all layers are
+    read; after it, each checked layer is replayed by the oracle from its pre-token table and the post-token table, the
+    copy lists (hence candidate set, routed set and demand plan as far as they move experts), the routed indices and
+    gate probabilities the call leaves in its buffers, and y are compared.  layers_checked: callable (t) -> iterable of
+    layers, default all.  tau < 0 runs the no-prefetch policy."""
+    cfg = prob.cfg
+    C = C or cfg.C
+    N, k, d, L = cfg.N, cfg.k, cfg.d, prob.L
+    rep = Report()
+    use_prefetch = not (tau < 0)
+    hs = [synth.hidden_states(cfg, l, T, B) for l in range(L)]
+    h_all = np.stack([x[0] for x in hs], 1)      # [T][L][B][d]
+    hp_all = np.stack([x[1] for x in hs], 1)
+    if host_buffers:
+        h_t = torch.from_numpy(h_all).pin_memory(); hp_t = torch.from_numpy(hp_all).pin_memory()
+        y = torch.full((L, B, d), 123.0, dtype=torch.float32).pin_memory()
+    else:
+        h_t = torch.from_numpy(h_all).cuda(); hp_t = torch.from_numpy(hp_all).cuda()
+        y = torch.full((L, B, d), 123.0, dtype=torch.float32, device="cuda")
+    for t in range(T):
+        pre = [apex.get_slot_table(l) for l in range(L)]
+        if host_buffers:
+            apex.decode_token_host(h_t[t], hp_t[t], B, tau, mode, y)
+        else:
+            apex.decode_token(h_t[t], hp_t[t], B, tau, mode, y)
+        torch.cuda.synchronize()
+        g_y = y.cpu().numpy() if not host_buffers else y.numpy().copy()
+        layers = list(range(L)) if layers_checked is None else list(layers_checked(t))
+        for l in layers:
+            W_r, b_r, W_p, b_p = prob.routers[l]
+            w, theta = prob.cdf[l]
+            cache = ao.SlotCache(N, C, cache_reuse=cache_reuse)
+            cache.set_state(*pre[l])
+            if use_prefetch:
+                out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=tau, k=k,
+                                    h=h_all[t, l], h_post=hp_all[t, l], mode=mode, expert_weights=prob.oracle_experts(l),
+                                    shared=prob.oracle_shared(l), norm_topk=norm_topk,
+                                    ffn_tokens=None if ffn_token_stride == 1 else set(range(0, B, ffn_token_stride)))
+            else:
+                out = _oracle_step_without_prefetch(cache, W_r, b_r, k, hp_all[t, l], mode, prob, l, norm_topk, True)
+            rep.layer_steps += 1
+            post = apex.get_slot_table(l)
+            g_cp, g_dm = apex.get_last_copies(l)
+            es, stamp, clk = cache.get_state()
+            same = (list(post[0]) == es and list(post[1]) == stamp and post[2] == clk and g_cp == out["prefetch_copies"]
+                    and g_dm == out["demand_copies"])
+            if not same:
+                near = any(ao.near_tie_reasons(tok) for tok in out["tokens"])
+                assert near, (f"slot decisions differ t={t} l={l}: copies {g_cp} {g_dm} vs {out['prefetch_copies']} "
+                              f"{out['demand_copies']}; table {list(post[0])} vs {es}")
+                rep.near_ties += 1
+                continue
+            rep.n_prefetch_copies += len(g_cp)
+            rep.n_demand_copies += len(g_dm)
+            rep.n_miss_steps += int(len(out["missing"]) > 0)
+            for b in range(B):
+                tok = out["tokens"][b]
+                if use_prefetch:
+                    rep.sum_delta_hat += tok["delta_hat"]; rep.sum_delta_star += tok["delta_star"]
+                    rep.sum_ncand += k + tok["delta_hat"]; rep.hits_P += int(round(tok["overlap_P"] * k))
+                    rep.covered += int(tok["covered"]); rep.capped += tok["capped"]
+                    rep.hits_R += int(round(tok["overlap_R"] * k))
+                else:
+                    rep.hits_R += k - tok["n_miss"]
+                rep.n_subst += tok["n_subst"]
+                if "y" in tok:
+                    ref = tok["y"]
+                    err = g_y[l, b].astype(np.float64) - ref
+                    rel = float(np.linalg.norm(err) / max(np.linalg.norm(ref), 1e-30))
+                    mx = float(np.abs(err).max())
+                    rep.worst_rel_l2 = max(rep.worst_rel_l2, rel)
+                    rep.worst_max_abs = max(rep.worst_max_abs, mx)
+                    rep.ffn_checked += 1
+                    assert rel <= REL_L2_TOL and mx <= MAX_ABS_TOL, f"FFN output t={t} l={l} b={b}: rel-L2 {rel:.3e} max-abs {mx:.3e}"
+    print(f"decode lock-step: {rep.layer_steps} layer-steps, {rep.near_ties} excused as near-ties (allowed {max_near_ties})")
+    assert rep.near_ties <= max_near_ties, f"{rep.near_ties} near-tie steps, at most {max_near_ties} allowed: {rep}"
+    return rep

@@ -376,11 +376,12 @@ def test_tensor_core_path_more_units_than_one_descriptor_chunk():
 
 
 # ------------------------------------------------------------------ API behaviour
-def test_decode_token_matches_per_call_sequence_and_counts_launches():
+@pytest.mark.parametrize("per_layer", [False, True])
+def test_decode_token_matches_per_call_sequence_and_counts_launches(per_layer):
     cfg = synth.tiny_config(d=512, N=12, k=3, I=24, C=6, L=2, T=4, cfg_id=218)
     hz = _harness()
     prob = hz.Problem(cfg)
-    a1, a2 = prob.make_ctx(), prob.make_ctx()
+    a1, a2 = prob.make_ctx(flags=binding.FLAG_LAYER_LAUNCHES if per_layer else 0), prob.make_ctx()
     try:
         hs = [synth.hidden_states(cfg, l, cfg.T) for l in range(cfg.L)]
         h = torch.from_numpy(np.stack([x[0] for x in hs], 1)).cuda()       # [T][L][1][d]
@@ -391,7 +392,10 @@ def test_decode_token_matches_per_call_sequence_and_counts_launches():
         for t in range(cfg.T):
             n0 = a1.launch_count()
             a1.decode_token(h[t], hp[t], 1, 0.9, "exact", y1)
-            assert a1.launch_count() - n0 >= 4 * cfg.L      # fused predict+select, attention, gate, FFN
+            if per_layer:
+                assert a1.launch_count() - n0 >= 4 * cfg.L      # fused predict+select, attention, gate, FFN
+            else:
+                assert a1.launch_count() - n0 == 1              # one persistent kernel over all layers
             for l in range(cfg.L):
                 a2.predict(l, h[t, l], 1); a2.select_candidates(l, 1, 0.9, cand, nc); a2.prefetch(l, 1)
                 a2.attention_standin(l); a2.route_topk(l, hp[t, l], 1, idx, al)

@@ -29,9 +29,39 @@ def test_summary_and_format_of_hand_made_spans():
     assert trace.summarize([]) == {}
 
 
+def test_persistent_kernel_phase_summary_of_hand_made_stamps():
+    import numpy as np
+    st = np.zeros((2, 4, 16), np.int64)
+    for cta in range(2):
+        for l in range(4):
+            t0 = 1000 + 20000 * l + 100 * cta
+            st[cta, l, 0] = t0
+            st[cta, l, 5] = t0 + 4000 + 1000 * cta          # gate logits complete: 4 and 5 us
+            st[cta, l, 8] = t0 + 15000
+    ph = trace.decode_phase_medians(st)
+    assert ph[trace.DECODE_STAMPS[5]] == 4.5 and ph[trace.DECODE_STAMPS[8]] == 15.0 and ph["layer period"] == 20.0
+    assert trace.DECODE_STAMPS[1] not in ph                  # never stamped
+    assert "gate logits complete" in trace.format_decode_phases(ph)
+    assert trace.decode_phase_medians(st[:, :2]) == {}
+
+
+@pytest.mark.gpu
+def test_traced_persistent_decode_records_one_kernel_per_token_and_its_phases():
+    r = subprocess.run([sys.executable, "bench.py", "--trace", "--config", "1", "--layers", "4", "--resident", "--warmup", "3"],
+                       cwd=ROOT, capture_output=True, text=True, timeout=600)
+    assert r.returncode == 0, r.stderr[-2000:]
+    line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])
+    t = line["trace"]
+    assert t[trace.KERNEL_NAMES[10]]["launches"] == line["tokens_traced"] and t["_all"]["spans"] == line["tokens_traced"]
+    ph = line["persistent_kernel_phase_median_us"]
+    order = [trace.DECODE_STAMPS[i] for i in (5, 6, 7, 8, 13)]   # gate -> plan -> first row -> last row -> y added
+    assert all(k in ph for k in order) and all(ph[a] <= ph[b] for a, b in zip(order[:-1], order[1:])), ph
+    assert 1.0 < ph["layer period"] < 500.0
+
+
 @pytest.mark.gpu
 def test_traced_decode_records_every_kernel_in_order():
-    r = subprocess.run([sys.executable, "bench.py", "--trace", "--config", "0", "--resident", "--warmup", "3"],
+    r = subprocess.run([sys.executable, "bench.py", "--trace", "--config", "0", "--resident", "--warmup", "3", "--layer-launches"],
                        cwd=ROOT, capture_output=True, text=True, timeout=600)
     assert r.returncode == 0, r.stderr[-2000:]
     line = json.loads([l for l in r.stdout.splitlines() if l.startswith("{")][-1])

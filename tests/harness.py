@@ -48,17 +48,31 @@ class Report:
 class Problem:
     """Parameters and expert stores of one config on the GPU machine, shared by library and oracle."""
 
-    def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset", fp8=False, fp4=False):
+    def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset", fp8=False, fp4=False,
+                 store_layers: Optional[int] = None):
+        """cdf: "handset", "fitted", or ("static", delta): the static over-fetch model of Sec. V-A (w = 0 and a step
+        in theta, so delta_hat = delta for every token).  store_layers: physical expert stores (layer l uses store
+        l mod store_layers; for shapes whose full store does not fit the host's memory)."""
         self.cfg = cfg
         self.fp8 = fp8
         self.fp4 = fp4
         self.L = layers or cfg.L
         self.routers = [synth.router_weights(cfg, l) for l in range(self.L)]
-        self.cdf = [synth.handset_cdf_params(cfg) if cdf == "handset" else synth.cdf_params(cfg, l)
-                    for l in range(self.L)]
+        if isinstance(cdf, tuple) and cdf[0] == "static":
+            nth = cfg.N - cfg.k + 1
+            step = np.where(np.arange(nth) >= int(cdf[1]), 50.0, -50.0).astype(np.float32)
+            self.cdf = [(np.zeros(cfg.N, np.float32), step) for _ in range(self.L)]
+        else:
+            self.cdf = [synth.handset_cdf_params(cfg) if cdf == "handset" else synth.cdf_params(cfg, l)
+                        for l in range(self.L)]
         self.stores = []
         self.shared = []
+        n_phys = min(self.L, store_layers or self.L)
         for l in range(self.L):
+            if l >= n_phys:
+                self.stores.append(self.stores[l % n_phys])
+                self.shared.append(self.shared[l % n_phys])
+                continue
             if fp4:
                 st = torch.empty((cfg.N, cfg.I, synth.fp4_row_bytes(cfg.d)), dtype=torch.uint8, pin_memory=True)
                 tmp = synth.expert_store_fp4(cfg, l, device=device)

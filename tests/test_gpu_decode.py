@@ -147,3 +147,98 @@ def test_persistent_kernel_wait_runs_out_and_the_context_recovers():
             assert torch.isfinite(y).all()
     finally:
         a.destroy()
+
+
+# ------------------------------------------------------------------ the paper-shaped configs at their full size
+def _sampled(step, L):
+    """Layers replayed by the oracle for token t: every `step`-th, the offset moving with t, plus the last layer."""
+    return lambda t: sorted(set(list(range((t * 3) % step, L, step)) + [L - 1]))
+
+
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_config2_full_size_all_layers_sampled(mode):
+    """Config 2 (OLMoE shape: 16 layers, 64 experts of 12 MiB, Zipf router bias, 24 slots, fitted confidence model)
+    through the whole-token call.  Slot tables of every layer before and after each token; sampled layers replayed by
+    the oracle: copy lists and tables bit-exact, y by tolerance."""
+    cfg = synth.CONFIGS[2]
+    rep, stats, launches = _decode(cfg, mode=mode, tau=0.9, T=3, cdf="fitted", layers_checked=_sampled(5, cfg.L))
+    assert rep.ffn_checked >= 9 and launches == 3 and stats["tokens"] == 3 * cfg.L
+    print("config2 full", mode, rep)
+
+
+@pytest.mark.parametrize("B,stride,T", [(1, 1, 2), (32, 8, 1), (256, 64, 1)])
+def test_config4_full_size_all_layers_sampled(B, stride, T):
+    """Config 4 (Qwen1.5-MoE shape: 24 layers, 60 experts of 16.5 MiB, shared expert, 30 slots), exact mode: B = 1 on
+    the persistent kernel, B = 32 and 256 on the tensor-core grouped GEMMs, where the distinct routed experts of a step
+    exceed the 30 slots and the step runs in waves."""
+    cfg = synth.CONFIGS[4]
+    rep, stats, launches = _decode(cfg, mode="exact", tau=0.9, T=T, B=B, cdf="fitted", layers_checked=_sampled(9, cfg.L),
+                                   ffn_token_stride=stride)
+    assert stats["tokens"] == T * B * cfg.L and rep.ffn_checked >= 3 * max(1, B // stride)
+    if B >= 32:
+        assert stats["extra_waves"] > 0
+    print("config4 full", B, rep, {k_: stats[k_] for k_ in ("extra_waves", "demand_copies", "prefetch_copies")})
+
+
+def test_config4_shape_stall_free_on_the_tensor_core_path():
+    cfg = synth.CONFIGS[4]
+    hz = _harness()
+    prob = hz.Problem(cfg, layers=2, cdf="fitted")
+    for B, stride in ((32, 8), (128, 32)):
+        rep, stats, _ = _decode(cfg, mode="stall_free", tau=0.9, T=2, B=B, prob=prob, ffn_token_stride=stride)
+        assert stats["demand_copies"] == 0 and stats["substitutions"] == rep.n_subst > 0
+        print("config4 stall-free tc", B, rep)
+
+
+def _host_memory_available_gib():
+    try:
+        for ln in open("/proc/meminfo"):
+            if ln.startswith("MemAvailable:"):
+                return int(ln.split()[1]) / (1 << 20)
+    except OSError:
+        pass
+    return 0.0
+
+
+def test_config3_all_layers():
+    """Config 3 (Mixtral-8x7B shape: 32 layers, 8 experts of 336 MiB, 4 slots, prefetch noise 0.5): all 32 layers through
+    the whole-token call, both modes.  The full expert store is 84 GiB of pinned host memory; it is allocated only if
+    the host reports at least 1.5 times that as available, otherwise eight physical layer stores are aliased onto the
+    32 layers (routers, confidence models and hidden states stay per layer)."""
+    cfg = synth.CONFIGS[3]
+    hz = _harness()
+    need_gib = cfg.L * cfg.N * cfg.expert_bytes / (1 << 30)
+    avail = _host_memory_available_gib()
+    full = avail >= 1.5 * need_gib
+    prob = None
+    if full:
+        try:
+            prob = hz.Problem(cfg, cdf="fitted")
+        except RuntimeError as e:            # pinning refused: fall back
+            print("config3: full pinned store refused:", str(e)[:200])
+            full = False
+    if prob is None:
+        prob = hz.Problem(cfg, cdf="fitted", store_layers=8)
+    print(f"config3: host MemAvailable {avail:.0f} GiB, store {need_gib:.0f} GiB -> {'full store' if full else '8 physical layer stores, aliased'}")
+    for mode in ("exact", "stall_free"):
+        rep, stats, launches = _decode(cfg, mode=mode, tau=0.9, T=2, prob=prob, layers_checked=_sampled(11, cfg.L))
+        assert launches == 2 and stats["tokens"] == 2 * cfg.L and rep.ffn_checked >= 6
+        print("config3 all layers", mode, rep)
+
+
+@pytest.mark.parametrize("delta", [0, 4, 8])
+def test_static_budget_baselines_against_the_oracle(delta):
+    """The static top-k / top-(k + delta) prefetch baselines of Sec. V-A (same ranking, fixed budget: w = 0 and a step
+    in theta): every decision against the oracle under that model, per call and through the whole-token kernel."""
+    cfg = synth.tiny_config(d=512, N=24, k=4, I=32, C=16, L=2, T=8, sigma_p=1.0, cfg_id=416)
+    hz = _harness()
+    prob = hz.Problem(cfg, cdf=("static", delta))
+    apex = prob.make_ctx()
+    try:
+        rep = hz.run_lockstep(prob, apex, mode="exact", tau=0.9, T=cfg.T)
+        st = apex.get_stats()
+    finally:
+        apex.destroy()
+    assert st["sum_delta_hat"] == delta * cfg.T * cfg.L == rep.sum_delta_hat and st["sum_ncand"] == (cfg.k + delta) * cfg.T * cfg.L
+    rep, stats, _ = _decode(cfg, mode="stall_free", tau=0.9, T=cfg.T, prob=prob)
+    assert stats["sum_delta_hat"] == delta * cfg.T * cfg.L

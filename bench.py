@@ -126,14 +126,14 @@ def build_problem(cfg, device, fp8=False, fp4=False):
     return routers, cdf, store, shared
 
 
-def make_ctx(cfg, prob, C, max_batch=1, flags=0, link_gbs=0.0):
+def make_ctx(cfg, prob, C, max_batch=1, flags=0, link_gbs=0.0, ctx_len=1024, cache_reuse=1):
     from paper_2608_11688_b200 import binding
     routers, cdf, store, shared = prob
     fmt_flag = 0
     if store.dtype != __import__("torch").bfloat16:
         fmt_flag = binding.FLAG_FP8_EXPERTS if store.shape[-1] == 3 * cfg.d + 16 else binding.FLAG_FP4_EXPERTS
     a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=C, L=cfg.L, I_shared=cfg.I_shared, max_batch=max_batch,
-                     flags=fmt_flag | flags, link_gbs=link_gbs)
+                     flags=fmt_flag | flags, link_gbs=link_gbs, ctx_len=ctx_len, cache_reuse=cache_reuse)
     for l in range(cfg.L):
         W_r, b_r, W_p, b_p = routers[l]
         a.set_router(l, W_r, b_r)
@@ -191,10 +191,10 @@ def train_auxiliary(cfg, prob, device, n_calib=8192, distill_iters=100, distill_
 POLICIES = (("no_prefetch", -1.0, None), ("static_k", 0.9, 0), ("static_k+4", 0.9, 4), ("static_k+8", 0.9, 8), ("apex", TAU, None))
 
 
-def run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, warmup, steps, link_gbs=0.0):
+def run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, warmup, steps, link_gbs=0.0, ctx_len=1024, cache_reuse=1):
     """Decode tokens under one prefetch policy of Sec. V-A (same ranking, different budgets); returns a dict."""
     import torch
-    ap_ = make_ctx(cfg, prob, cfg.C, max_batch=B, link_gbs=link_gbs)
+    ap_ = make_ctx(cfg, prob, cfg.C, max_batch=B, link_gbs=link_gbs, ctx_len=ctx_len, cache_reuse=cache_reuse)
     if delta is not None:      # w = 0 and a step in theta: delta_hat = delta for every token
         nth = cfg.N - cfg.k + 1
         th = np.where(np.arange(nth) >= delta, 50.0, -50.0).astype(np.float32)
@@ -217,10 +217,68 @@ def run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, warmup, s
     out = {"tokens_per_s": steps * B / sec, "ms_per_token": 1e3 * sec / (steps * B),
            "copies_per_token": (sp["prefetch_copies"] + sp["demand_copies"]) / steps,
            "demand_copies_per_token": sp["demand_copies"] / steps,
+           "prefetch_copies_per_token": sp["prefetch_copies"] / steps,
            "overlap_vs_R": sp["hits_R"] / max(1, sp["routed"]),
            "copied_gbs": sp["bytes_copied"] / sec / 1e9}
     ap_.destroy()
     return out
+
+
+def window_sweep(args, cfg, prob, h_dev, hp_dev, y_dev, B):
+    """Study of the overlap condition, Eq. (12): T_prefetch(delta) = delta * S_expert / B_eff + T_queue <= T_attn.  On this
+    machine one expert copy over the host link is far longer than the attention window of the paper's context lengths,
+    so nothing can be hidden and the policies that move fewer bytes win.  Here the OTHER side of the ratio is moved: the
+    stand-in attention is lengthened (through ctx_len) until the window holds 0.5, 1, 2 and 4 expert copies, and the
+    policies of Sec. V-A are timed at every window.  Per policy: tokens/s, demand copies per token, the exposed stall
+    (time per token minus the all-resident time at the same window) and the stall Eq. (12) allows at best
+    (per layer: what the prefetch copies overrun the window by, plus the demand copies, at the measured link rate)."""
+    import torch
+    from paper_2608_11688_b200 import binding
+    d, L = cfg.d, cfg.L
+    steps, warmup = max(8, min(args.steps, 16)), 4
+
+    def resident_ms(ctx_len, flags=0):
+        a = make_ctx(cfg, prob, cfg.N, max_batch=B, ctx_len=ctx_len, flags=flags)
+        a.warm_all()
+        sec = time_tokens(a, h_dev, hp_dev, y_dev, B, "exact", warmup, steps)
+        a.destroy()
+        return 1e3 * sec / steps
+
+    base_ms = resident_ms(1024, flags=binding.FLAG_SKIP_STANDIN)       # the method's own kernels, no window at all
+    # link rate and copy time: from a run that keeps the link busy
+    ref = run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, "no_prefetch", -1.0, None, warmup, steps)
+    link_gbs = ref["copied_gbs"]
+    t_copy_us = cfg.expert_bytes / (link_gbs * 1e3)
+    # stand-in streaming rate: from two window lengths
+    ms_a, ms_b = resident_ms(1024), resident_ms(65536)
+    bytes_of = lambda c: (4 * d * d + 2 * c * d) * 2
+    us_per_byte = (ms_b - ms_a) * 1e3 / L / (bytes_of(65536) - bytes_of(1024))
+    rows = []
+    for ratio in (None, 0.5, 1.0, 2.0, 4.0):
+        if ratio is None:
+            ctx_len = 1024
+        else:
+            want_bytes = ratio * t_copy_us / us_per_byte
+            ctx_len = max(1024, int((want_bytes / 2 - 4 * d * d) / (2 * d)))
+        res_ms = resident_ms(ctx_len)
+        t_attn_us = max(0.0, (res_ms - base_ms) * 1e3 / L)
+        row = {"ctx_len": ctx_len, "T_attn_us": t_attn_us, "T_attn_over_copy": t_attn_us / t_copy_us, "all_resident_ms_per_token": res_ms,
+               "policies": {}}
+        for name, tau_p, delta, reuse in (("no_prefetch", -1.0, None, 1), ("static_k", 0.9, 0, 1), ("static_k+4", 0.9, 4, 1),
+                                          ("apex", TAU, None, 1), ("apex_load_use_evict", TAU, None, 0)):
+            r = run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, warmup, steps, ctx_len=ctx_len, cache_reuse=reuse)
+            pre_l, dem_l = r["prefetch_copies_per_token"] / L, r["demand_copies_per_token"] / L
+            bound_us = L * (max(0.0, pre_l * t_copy_us - t_attn_us) + dem_l * t_copy_us)
+            row["policies"][name] = {"tokens_per_s": r["tokens_per_s"], "ms_per_token": r["ms_per_token"],
+                                     "demand_copies_per_token": r["demand_copies_per_token"],
+                                     "prefetch_copies_per_token": r["prefetch_copies_per_token"],
+                                     "exposed_stall_us_per_token": (r["ms_per_token"] - res_ms) * 1e3,
+                                     "eq12_stall_bound_us_per_token": bound_us}
+        rows.append(row)
+    last = rows[-1]["policies"]
+    return {"window_sweep": rows, "expert_copy_us": t_copy_us, "link_gbs": link_gbs, "standin_gbs": 1e-3 / us_per_byte,
+            "no_window_ms_per_token": base_ms, "config": f"config{cfg.cfg_id}", "steps": steps, "tau": TAU,
+            "apex_over_no_prefetch_at_largest_window": last["apex"]["tokens_per_s"] / last["no_prefetch"]["tokens_per_s"]}
 
 
 def hidden_inputs(cfg, T, B, device):
@@ -405,6 +463,8 @@ def main():
     ap.add_argument("--spec", action="store_true", help="A/B: expert FFN with the speculative first fill (FLAG_SPECULATE)")
     ap.add_argument("--layer-launches", action="store_true",
                     help="A/B: the per-layer kernel sequence instead of the persistent token kernel (FLAG_LAYER_LAUNCHES)")
+    ap.add_argument("--standin-ahead", action="store_true",
+                    help="A/B: the token kernel requests the stand-in attention's bytes ahead of the previous layer's completion (FLAG_STANDIN_AHEAD)")
     ap.add_argument("--no-standin", action="store_true",
                     help="leave the stand-in attention out of the decode step (FLAG_SKIP_STANDIN): the method's own bytes only")
     ap.add_argument("--fp8", action="store_true",
@@ -412,6 +472,9 @@ def main():
     ap.add_argument("--link-sweep", action="store_true",
                     help="study: per-token latency of the policies on a throttled host link (every expert copy padded to "
                          "its duration at 8, 16 and 32 GB/s) and on the link as it is")
+    ap.add_argument("--window-sweep", action="store_true",
+                    help="study: the policies of Sec. V-A with the hiding window (the stand-in attention, through ctx_len) "
+                         "lengthened until it holds 0.5, 1, 2 and 4 expert copies -- the regime in which Eq. (12) can hold")
     ap.add_argument("--train-aux", action="store_true",
                     help="study: distil the prefetch routers and refit the confidence models on this GPU first "
                          "(a different predictor than the workload's: needs --skip-extras)")
@@ -461,7 +524,7 @@ def main():
     B = args.batch
     from paper_2608_11688_b200 import binding as _b
     base_flags = (_b.FLAG_SPECULATE if args.spec else 0) | (_b.FLAG_LAYER_LAUNCHES if args.layer_launches else 0) | \
-                 (_b.FLAG_SKIP_STANDIN if args.no_standin else 0)
+                 (_b.FLAG_SKIP_STANDIN if args.no_standin else 0) | (_b.FLAG_STANDIN_AHEAD if args.standin_ahead else 0)
     prob = build_problem(cfg, dev, fp8=args.fp8, fp4=args.fp4)
     aux_info = None
     if args.train_aux:
@@ -503,6 +566,10 @@ def main():
                           "ffn_cta_phase_median_cycles": phases, "persistent_kernel_phase_median_us": dec,
                           "config": f"config{cfg.cfg_id}", "resident": bool(args.resident)}), flush=True)
         a.destroy()
+        return
+
+    if args.window_sweep:
+        print(json.dumps(window_sweep(args, cfg, prob, h_dev, hp_dev, y_dev, B)), flush=True)
         return
 
     if args.link_sweep:

@@ -86,6 +86,11 @@ extern "C" {
 #define APEX_FLAG_SKIP_STANDIN 32   /* apex_config.flags: apex_decode_token leaves the stand-in attention out (the hiding
                                        window of Eq. (12) is then empty: for measuring the method's own bytes) */
 
+#define APEX_FLAG_STANDIN_AHEAD 64  /* apex_config.flags: the persistent token kernel requests a layer's stand-in attention bytes
+                                       while the previous layer is still finishing (they are parameters and old KV entries),
+                                       instead of when that layer's output is complete.  Faster, but the hiding window of
+                                       Eq. (12) then overlaps the previous layer's tail, so it is off by default */
+
 #define APEX_MAX_EXPERTS 64
 #define APEX_MAX_TOPK 16
 #define APEX_MAX_BATCH 256

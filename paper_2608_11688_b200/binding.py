@@ -24,6 +24,7 @@ FLAG_FP4_EXPERTS = 4
 FLAG_HOST_WAVES = 8
 FLAG_LAYER_LAUNCHES = 16
 FLAG_SKIP_STANDIN = 32
+FLAG_STANDIN_AHEAD = 64
 ERR_NAMES = {0: "APEX_OK", -1: "APEX_EINVAL", -2: "APEX_ENOMEM", -3: "APEX_ECUDA", -4: "APEX_ETIMEOUT",
              -5: "APEX_ESTATE", -6: "APEX_ENOTIMPL"}
 

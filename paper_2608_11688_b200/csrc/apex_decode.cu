@@ -165,6 +165,7 @@ int decode_token_persistent(apex_ctx* ctx, const float* h_dev, const float* hpos
   p.abort_flag = ctx->d_dec_abort;
   p.attn = ctx->d_attn; p.attn_bytes = ctx->attn_bytes; p.attn_layers = (int)ctx->attn_layers;
   p.run_attn = (ctx->cfg.flags & APEX_FLAG_SKIP_STANDIN) ? 0 : 1;
+  p.standin_ahead = (ctx->cfg.flags & APEX_FLAG_STANDIN_AHEAD) ? 1 : 0;
   p.seq = seq;
   p.demand_tag = tag;
   p.force = !prefetching ? 0 : (tau <= 0.f ? 1 : (tau >= 1.f ? 2 : 0));

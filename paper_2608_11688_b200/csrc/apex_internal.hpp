@@ -219,6 +219,7 @@ struct DecodeParams {
   const uint8_t* attn;
   size_t attn_bytes;
   int attn_layers, run_attn;
+  int standin_ahead;                    // 1: the stand-in's chunks are requested ahead of the previous layer's completion
   uint32_t seq;                         // this token's sequence number
   uint32_t demand_tag;
   float t_tau;

@@ -10,11 +10,12 @@
 //
 //   [its share of the attention stand-in's bytes, its row of W_p among the first]  [its row of W_r]  [its rows of the expert FFN]
 //
-// Copies are started as far ahead as the ring allows: what a layer's first segment reads are parameters (router rows)
-// and the stand-in's bytes, none of which depends on the previous layer, so a warp requests them as soon as its last
-// expert rows of the previous layer have been requested -- the next layer's bytes arrive while this layer's tail, the
-// reduction of y and the hand-over are still going on.  (Consumption stays in order, and everything derived from h or
-// h' waits for the counters below.)
+// The stand-in's chunks of a layer are requested when the previous layer's y is complete (the attention block's window
+// of Eq. (12) opens when its input exists).  With APEX_FLAG_STANDIN_AHEAD they are requested as far ahead as the ring
+// allows instead -- a warp starts them as soon as its last expert rows of the previous layer have been requested, so
+// they arrive while that layer's tail, the reduction of y and the hand-over are still going on; faster, but the window
+// then overlaps the previous layer.  (Consumption stays in order, and everything derived from h or h' waits for the
+// counters below.)
 //
 //   prefetch router (S1-S3): CTA r of a cluster owns experts 8r .. 8r+7, one warp per expert.  The row arrives in the
 //     ring; its dot product with h (reduction order of router_kernel: lane-strided fused multiply-adds, then the xor
@@ -176,7 +177,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
   const int ch_per = n_chunks / G, ch_extra = n_chunks - ch_per * G;
   const int ch_lo = cta * ch_per + (cta < ch_extra ? cta : ch_extra);
   const int ch_n = ch_per + (cta < ch_extra ? 1 : 0);
-  const int ch_mine = ch_n > warp ? (ch_n - warp + kDecWarps - 1) / kDecWarps : 0;
+  // (the poster's warp 0 takes none while the prefetch stage runs: it has the candidate selection to do as soon as the
+  // prefetch logits arrive, and everybody's gate waits until every warp has counted its chunks)
+  const bool poster_w0_free = (cta == kDecCluster - 1) && p.prefetching;
+  const int ch_warps = poster_w0_free ? kDecWarps - 1 : kDecWarps;
+  const int ch_warp = poster_w0_free ? warp - 1 : warp;
+  const int ch_mine = (ch_warp >= 0 && ch_n > ch_warp) ? (ch_n - ch_warp + ch_warps - 1) / ch_warps : 0;
   // Segment 1 of a layer in the ring: the warp's chunks of the stand-in.  The router rows do not go through the ring:
   // a warp loads its row of W_p and of W_r straight into registers at the start of the layer (parameters: nothing to
   // wait for), so the rows are there when the counters allow the dot products.
@@ -251,7 +257,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
         continue;
       }
       if (lane == 0) {
-        const size_t c = (size_t)ch_lo + warp + (size_t)kDecWarps * iq;
+        const size_t c = (size_t)ch_lo + ch_warp + (size_t)ch_warps * iq;
         const size_t off = c * entry_bytes;
         const size_t left = attn_bytes - off;
         start_copy(p.attn + (size_t)(il % p.attn_layers) * p.attn_bytes + off, left < entry_bytes ? (uint32_t)left : entry_bytes);
@@ -429,10 +435,30 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
         if ((old + 1u) % kDecWarps == 0u) red_release_gpu_u64(bar_attn, 1ull);
       }
     };
+    // The stand-in is this layer's attention block: its window opens when the previous layer's y is complete.  (With
+    // standin_ahead the chunks were requested earlier, while the previous layer was still finishing: the window then
+    // overlaps that layer's tail -- including any wait for its experts -- which is not what Eq. (12) describes.)
+    if ((J > 0 || has_wp) && running && bar_prev_ffn) {
+      bool go = true;
+      if (lane == 0) go = wait_counter(bar_prev_ffn, p.bar_target);
+      go = __shfl_sync(0xffffffffu, go ? 1 : 0, 0) != 0;
+      if (!go) {
+        if (lane == 0 && !stop_requested()) gave_up();
+        ok = false;
+      }
+      DTL(15);
+    }
+    if (ok && running) start_seg1(l, NSW);  // this layer's chunks: on their way while the prefetch logit is computed
+    // prefetch router first of all: the sooner the candidate set is out, the more of the window the copies can use
+    if (has_wp && running && ok) {
+      row_logit(Wp_row, wp_row, hl, bias_p, s_zp, &s_xbar[0], kDecCluster - 1, kDecCluster);  // to the poster only
+      DTL(1);
+      if (has_wr) load_row(Wr_row, wr_row);
+    }
     {
       int q_con = 0;
       while (q_con < J && ok && running) {
-        start_seg1(l, NSW);  // (chunks of this layer that were not started ahead of time)
+        start_seg1(l, NSW);
         const int s = wait_copy();
         if (s < 0) break;
         __syncwarp();
@@ -441,21 +467,6 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
       }
     }
     count_attention();
-    // prefetch router: this warp's logit, as soon as the previous layer's y is complete
-    if (has_wp && running && ok) {
-      bool go = true;
-      if (lane == 0 && bar_prev_ffn) go = wait_counter(bar_prev_ffn, p.bar_target);
-      go = __shfl_sync(0xffffffffu, go ? 1 : 0, 0) != 0;
-      if (!go) {
-        if (lane == 0 && !stop_requested()) gave_up();
-        ok = false;
-      } else {
-        DTL(15);
-        row_logit(Wp_row, wp_row, hl, bias_p, s_zp, &s_xbar[0], kDecCluster - 1, kDecCluster);  // to the poster only
-        DTL(1);
-      }
-      if (has_wr) load_row(Wr_row, wr_row);
-    }
     // the poster's warp 0: the candidate set, as soon as the prefetch logits are complete (after it has counted its
     // share of the stand-in: everybody's gate waits for that count)
     if (!pref_done && ok && !cta_stopped()) {
@@ -803,7 +814,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
           }
           // every row of this layer has been requested (and the table is confirmed: no repeat can follow): go on with
           // the next layer's first segment (one stage stays free for the reduction of y)
-          if (q_iss >= Jr && ok && verified && !redo) start_seg1(l + 1, NSW - 1);
+          if (p.standin_ahead && q_iss >= Jr && ok && verified && !redo) start_seg1(l + 1, NSW - 1);
           __syncwarp();  // s_exp of the copies just started is visible to the whole warp
           if (!ok) break;
           if (!gates_done) {
@@ -925,7 +936,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
         atomicAdd(&st->hits_R, (unsigned long long)__popcll(kr_mask & resident));
       }
     }
-    if (go_rows && ok) start_seg1(l + 1, NSW - 1);
+    if (p.standin_ahead && go_rows && ok) start_seg1(l + 1, NSW - 1);
     DTL(8);
     if (lane == 0 && waited && planned) {
       atomicAdd(&p.stats[l].stall_ns, waited * (unsigned long long)p.n_sm / (unsigned long long)G);  // the host divides by the SM count
@@ -964,7 +975,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     }
     cluster_barrier();  // every CTA's partial y is complete (and the stages that held the warps' vectors are free again)
     DTL(12);
-    if (ok && !cta_stopped()) start_seg1(l + 1, NSW);
+    if (p.standin_ahead && ok && !cta_stopped()) start_seg1(l + 1, NSW);
     if (tid < SLICE4) {
       // CTA r of the cluster adds columns [r * d/8, (r+1) * d/8) of the cluster's eight partial vectors to y
       const int col4 = (int)crank * SLICE4 + tid;

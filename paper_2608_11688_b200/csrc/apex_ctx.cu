@@ -126,7 +126,7 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   CR(dev_alloc(&ctx->d_exec_gate, MB * k));
   CR(dev_alloc(&ctx->d_cand_ncand, MB));
   // batched tensor-core path: scratch and tensor maps (only for contexts that will see large batches)
-  if (MB >= kTcMinBatch && ctx->fmt == 0 && tc_shape_supported(c.d, c.I, c.I_shared)) {
+  if (MB >= kTcMinBatch && tc_shape_supported(c.d, c.I, c.I_shared, ctx->fmt)) {
     const size_t rows = max_pairs + 256;
     const size_t i_max = (size_t)(c.I > c.I_shared ? c.I : c.I_shared);
     ctx->act_stride = (int)i_max;
@@ -135,8 +135,8 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
     CR(dev_alloc(&ctx->d_act, 2 * rows * i_max));
     CR(cudaMemset(ctx->d_xg, 0, rows * d * 2));
     CR(cudaMemset(ctx->d_act, 0, 2 * rows * i_max * 2));
-    ctx->tc_ok = tc_make_weight_map(ctx->tc_maps.w_gateup, ctx->d_cache, c.d, c.I, L * C, ctx->expert_bytes, 128) &&
-                 tc_make_weight_map(ctx->tc_maps.w_down, ctx->d_cache, c.d, c.I, L * C, ctx->expert_bytes, 64) &&
+    ctx->tc_ok = tc_make_store_maps(ctx->fmt, ctx->tc_maps.w_gateup, ctx->tc_maps.w_down, ctx->tc_maps.sc_gateup, ctx->tc_maps.sc_down,
+                                    ctx->d_cache, c.d, c.I, L * C, ctx->expert_bytes) &&
                  tc_make_rows_map(ctx->tc_maps.xg, ctx->d_xg, c.d, rows, d) &&
                  tc_make_rows_map(ctx->tc_maps.act, ctx->d_act, (int)i_max, rows, i_max) &&
                  tc_make_rows_map(ctx->tc_maps.act_lo, ctx->d_act + ctx->act_plane, (int)i_max, rows, i_max);
@@ -301,8 +301,8 @@ int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights) {
     CU_TRY(ctx, cudaMemcpy(ctx->d_shared_ptrs + layer, &dev_weights, sizeof(void*), cudaMemcpyHostToDevice));
   if (ctx->tc_ok) {
     TcMaps& m = ctx->tc_shared_maps[layer];
-    if (!tc_make_weight_map(m.ws_gateup, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1, ctx->shared_bytes, 128) ||
-        !tc_make_weight_map(m.ws_down, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1, ctx->shared_bytes, 64))
+    if (!tc_make_store_maps(ctx->fmt, m.ws_gateup, m.ws_down, m.ssc_gateup, m.ssc_down, dev_weights, ctx->cfg.d, ctx->cfg.I_shared, 1,
+                            ctx->shared_bytes))
       return fail(ctx, APEX_ECUDA, "tensor map for the shared expert could not be encoded");
   }
   return APEX_OK;

@@ -169,6 +169,8 @@ struct TcParams {
 };
 struct TcMaps {          // opaque 128-byte CUtensorMap objects
   alignas(64) unsigned char w_gateup[128], w_down[128], ws_gateup[128], ws_down[128], xg[128], act[128], act_lo[128];
+  // e2m1 stores only: the same bytes as w_* / ws_* with 16-byte boxes, for the block-scale bytes
+  alignas(64) unsigned char sc_gateup[128], sc_down[128], ssc_gateup[128], ssc_down[128];
 };
 
 // Persistent decode kernel (kernels_decode.cu): all layers of one token in one cooperative launch.
@@ -246,7 +248,9 @@ int ffn_grid_ctas(int n_sm);  // CTAs of one streaming-kernel launch (each adds 
 cudaError_t launch_ffn_tc(const TcParams& p, const TcMaps& m, int n_sm, cudaStream_t s);
 bool tc_make_weight_map(void* out, const void* base, int d, int I, size_t n_slots, size_t slot_bytes, int box_rows);
 bool tc_make_rows_map(void* out, const void* base, int cols, size_t rows, size_t stride_elems);
-bool tc_shape_supported(int d, int I, int I_shared);
+bool tc_make_store_maps(int fmt, void* gateup, void* down, void* sc_gateup, void* sc_down, const void* base, int d, int I, size_t n_slots,
+                        size_t slot_bytes);   // weight maps of one store in storage format fmt
+bool tc_shape_supported(int d, int I, int I_shared, int fmt);
 bool ffn_shape_supported(int d);
 bool ffn_quantised_shape_supported(int d);   // widths the e4m3 / e2m1 kernels were built for
 size_t ffn_row_bytes(int fmt, int d);        // bytes of one intermediate index (three vectors and their scales)

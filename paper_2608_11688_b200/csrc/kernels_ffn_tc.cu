@@ -1,5 +1,5 @@
 // Batched expert FFN on the 5th-generation tensor cores (tcgen05 + TMEM), for decode steps with many
-// tokens (Sec. V-B: the method "supports batching multiple concurrent requests").
+// tokens (Sec. V-B: several concurrent requests are decoded as one batch).
 //
 // With B tokens per step an expert serves several tokens, so its weights should be read once and
 // applied to all of them: a grouped GEMM, one group per executed expert (plus the shared expert).
@@ -29,7 +29,18 @@
 // One CTA per SM, three roles: two warps issue TMA loads (alternating K tiles; a single issuing
 // thread cannot keep up with 16 KB tiles), one thread issues MMAs, four warps run the epilogue out
 // of TMEM.  Every wait is bounded.
+//
+// Quantised stores (e4m3 codes with a scale per row vector, e2m1 codes with a power-of-two scale per 32
+// elements) take the same path with one more role: the producers bring the raw code bytes (and, for e2m1,
+// the scale bytes) of a K tile into a staging area of the stage, eight converter warps expand them to bf16
+// in the swizzled operand layout the MMA descriptors expect, and the MMAs run as for a bf16 store.  Both code
+// sets are exact in bf16 (3 and 1 mantissa bits), and so is an e2m1 value times its power-of-two scale, so
+// the tensor cores see the dequantised weights exactly; the per-vector fp32 scales of an e4m3 row are not
+// exact in bf16 and are applied in fp32 instead: gate and up scales to the accumulators, the down scale
+// folded into the intermediate before it is split into its two bf16 planes.  HBM sees 1 or 0.53 bytes per
+// weight; the expansion costs shared-memory bandwidth and ALU work that the streaming leaves idle.
 #include <cuda.h>
+#include <cuda_fp16.h>
 #include <cuda_bf16.h>
 
 #include "apex_internal.hpp"
@@ -41,7 +52,14 @@ namespace {
 
 constexpr int kProducerWarps = 2;  // TMA producers: K tile t is loaded by warp t mod 2
 constexpr int kMmaWarp = kProducerWarps;
-constexpr int kTcThreads = (kProducerWarps + 1 + 4) * 32;  // producers, MMA + TMEM owner, four epilogue warps
+constexpr int kCvWarp0 = kProducerWarps + 1 + 4;  // first of the converter warps (quantised stores only)
+constexpr int kCvThreads = 256;   // eight warps: two per scheduler, so one warp's shared-memory latency hides behind the other's arithmetic
+// producers, MMA + TMEM owner, four epilogue warps; for a quantised store the converter warps as well
+__host__ __device__ constexpr int tc_threads(int qf) { return (kProducerWarps + 1 + 4) * 32 + (qf ? kCvThreads : 0); }
+// bytes of raw codes (and e2m1 scale bytes: 16 per row) a pipeline stage stages for the converters
+__host__ __device__ constexpr int tc_raw_bytes(int phase, int qf) {
+  return qf == 1 ? (phase == 1 ? 2 * 128 * 64 : 64 * 128) : qf == 2 ? (phase == 1 ? 2 * 128 * 32 + 2 * 128 * 16 : 64 * 64 + 64 * 16) : 0;
+}
 constexpr int kKTile = 64;       // K elements per pipeline stage (128 bytes: one swizzle span)
 constexpr int kXRowsPerLoad = 8;    // rows per B-tile box: one 8-row swizzle atom, so a small group does not fetch rows it has no token for
 
@@ -55,6 +73,63 @@ __device__ __forceinline__ void tma_load_2d(void* dst, const CUtensorMap* map, i
   asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4}], [%2];" ::"r"(smem_u32(dst)),
                "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1)
                : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(void* dst, const CUtensorMap* map, int c0, int c1, int c2, uint64_t* bar) {
+  asm volatile("cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5}], [%2];" ::"r"(smem_u32(dst)),
+               "l"(map), "r"(smem_u32(bar)), "r"(c0), "r"(c1), "r"(c2)
+               : "memory");
+}
+// Expanding codes to bf16 with conversion instructions runs at a quarter of the plain ALU rate and was the pace of the
+// whole kernel; the converters therefore build the bf16 bit patterns with integer operations and one bf16 multiply:
+// a code's exponent and mantissa bits, placed at the top of a bf16's mantissa and the bottom of its exponent field,
+// read as the code's value times 2^(code bias - 127), subnormal codes included (they become bf16 subnormals, which
+// the multiply does not flush); the multiply by a power of two puts the exponent right and is exact.
+__device__ __forceinline__ uint32_t mul_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t o;
+  asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o) : "r"(a), "r"(b));
+  return o;
+}
+// four e4m3 codes (s eeee mmm, bias 7) -> four bf16 values
+__device__ __forceinline__ void e4m3x4_to_bf16(uint32_t c, uint32_t& o0, uint32_t& o1) {
+  const uint32_t k = 0x7B807B80u;                       // 2^120, twice
+  const uint32_t r0 = __byte_perm(c, 0u, 0x1404u);      // codes 0, 1 in the high byte of each half
+  const uint32_t r1 = __byte_perm(c, 0u, 0x3424u);      // codes 2, 3
+  o0 = mul_bf16x2((r0 & 0x80008000u) | ((r0 >> 4) & 0x07f007f0u), k);
+  o1 = mul_bf16x2((r1 & 0x80008000u) | ((r1 >> 4) & 0x07f007f0u), k);
+}
+// eight e2m1 codes (s ee m, bias 1; the even element in the low nibble of its byte) times the block scale
+// 2^(sb - 127) (sb = 0: zero) -> eight bf16 values
+__device__ __forceinline__ uint4 e2m1x8_to_bf16(uint32_t c, uint32_t sb) {
+  uint32_t o[4];
+  if (sb <= 128u) {
+    // code bits as a bf16 read as value * 2^-126; times 2^126 * 2^(sb - 127) = 2^(sb - 1): one multiply
+    const uint32_t m1 = sb ? (sb + 126u) << 7 : 0u;
+    const uint32_t m = m1 | (m1 << 16);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint32_t t = __byte_perm(c, 0u, 0x4440u + j) * 4097u;   // low nibble at bits 0..3, high nibble at bits 16..19
+      o[j] = mul_bf16x2(((t & 0x00080008u) << 12) | ((t & 0x00070007u) << 6), m);
+    }
+  } else {
+    // scales above 2 (never produced for weights of ordinary size): through the conversion instructions
+    const float scale = __uint_as_float(sb << 23);
+    uint32_t h[4];
+    asm("{\n.reg .b8 b0, b1, b2, b3;\n"
+        "mov.b32 {b0, b1, b2, b3}, %4;\n"
+        "cvt.rn.f16x2.e2m1x2 %0, b0;\n"
+        "cvt.rn.f16x2.e2m1x2 %1, b1;\n"
+        "cvt.rn.f16x2.e2m1x2 %2, b2;\n"
+        "cvt.rn.f16x2.e2m1x2 %3, b3;\n}"
+        : "=r"(h[0]), "=r"(h[1]), "=r"(h[2]), "=r"(h[3])
+        : "r"(c));
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const float2 f = __half22float2(*reinterpret_cast<const __half2*>(&h[j]));
+      const __nv_bfloat162 b = __floats2bfloat162_rn(f.x * scale, f.y * scale);
+      o[j] = *reinterpret_cast<const uint32_t*>(&b);
+    }
+  }
+  return make_uint4(o[0], o[1], o[2], o[3]);
 }
 // shared-memory matrix descriptor, 128-byte swizzle (layout type 2), version 1
 __device__ __forceinline__ uint64_t umma_desc(uint32_t saddr, uint32_t lbo_bytes, uint32_t sbo_bytes) {
@@ -102,8 +177,13 @@ __device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::
 #ifdef APEX_TIMELINE
 __device__ unsigned long long g_tc_tl[2][148][128];
 #define TCTL(ph, i) do { if ((i) < 128) g_tc_tl[(ph) - 1][blockIdx.x][(i)] = globaltimer_ns(); } while (0)
+// per K tile (the first 96 of a CTA): loads issued, raw bytes landed, operand buffer free, tiles converted; stage free
+// (producer), operands complete (MMA thread), MMAs issued
+__device__ unsigned long long g_cv_tl[2][148][96][8];
+#define CVTL(ph, it, i) do { if ((it) < 96u) g_cv_tl[(ph) - 1][blockIdx.x][(it)][(i)] = globaltimer_ns(); } while (0)
 #else
 #define TCTL(ph, i) do { } while (0)
+#define CVTL(ph, it, i) do { } while (0)
 #endif
 
 struct Group {
@@ -157,9 +237,14 @@ __global__ void __launch_bounds__(256) ffn_tc_gather_kernel(const TcParams p) {
 // PHASE 1: gate/up.  A tiles: gate and up rows [128 x 64] (K-major), B tile: X_g rows [<=256 x 64].
 // PHASE 2: down.     A tile: downT [64 k-rows x 128 cols] as two 64-column atoms (MN-major), B tile: the group's rows of
 //                    a_hi, then of a_lo [2 x <=64 x 64].
-template <int PHASE>
-__global__ void __launch_bounds__(kTcThreads, 1)
+//
+// QF: storage format of the weights (0 bf16, 1 e4m3, 2 e2m1).  For QF != 0, tm_w / tm_ws cover the raw row bytes of
+// the slots / the shared expert (boxes of one K tile's code bytes) and tm_sc / tm_ssc the same bytes with 16-byte boxes
+// (the e2m1 scale bytes); a stage is [A tiles, bf16, written by the converters][B planes][raw bytes, written by TMA].
+template <int PHASE, int QF>
+__global__ void __launch_bounds__(tc_threads(QF), 1)
 ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_ws,
+                   const __grid_constant__ CUtensorMap tm_sc, const __grid_constant__ CUtensorMap tm_ssc,
                    const __grid_constant__ CUtensorMap tm_b, const __grid_constant__ CUtensorMap tm_b2, const TcParams p) {
   SPAN_BEGIN();
   extern __shared__ __align__(1024) uint8_t smem_raw[];
@@ -171,9 +256,10 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   // small batches get deep pipelines (more weight bytes in flight), large groups are cut into parts.
   const int NMAX = PHASE == 1 ? p.nmax1 : p.nmax2;
   const int B_PLANE = NMAX * 128;
-  const int STAGE_BYTES = A_BYTES + PLANES * B_PLANE;
+  constexpr int RAW_BYTES = tc_raw_bytes(PHASE, QF);
+  const int STAGE_BYTES = A_BYTES + PLANES * B_PLANE + RAW_BYTES;
   const int NSTAGE = PHASE == 1 ? p.nstage1 : p.nstage2;
-  __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], tmem_full[2], tmem_empty[2];
+  __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], rawfull[MAX_STAGES], tmem_full[2], tmem_empty[2];
   __shared__ uint32_t tmem_base_s;
   __shared__ int s_abort;
   __shared__ UnitDesc s_unit[kUnitChunk];
@@ -188,8 +274,9 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   if (tid == 0) {
     s_abort = 0;
     for (int s = 0; s < MAX_STAGES; ++s) {
-      mbar_init(&full[s], 1);
+      mbar_init(&full[s], QF ? 1 + kCvThreads / 32 : 1);  // the producer's arrival (B tile bytes) and one per converter warp
       mbar_init(&empty[s], 1);
+      mbar_init(&rawfull[s], 1);
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&tmem_full[b], 1);
@@ -200,6 +287,10 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_ws) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_b2) : "memory");
+    if (QF == 2) {
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_sc) : "memory");
+      asm volatile("prefetch.tensormap [%0];" ::"l"(&tm_ssc) : "memory");
+    }
   }
   if (warp == kMmaWarp) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(smem_u32(&tmem_base_s)), "r"(512) : "memory");
@@ -232,7 +323,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   pdl_launch_dependents();
 
   // the group table goes to shared memory once: a global load per unit would sit on every role's path
-  for (int i = tid; i < 4 + 3 * (N + 1); i += kTcThreads) s_grp[i] = grp[i];
+  for (int i = tid; i < 4 + 3 * (N + 1); i += (int)blockDim.x) s_grp[i] = grp[i];
   __syncthreads();
   const int n_rg = s_grp[0], n_g = s_grp[1];
   const int blocks_r = PHASE == 1 ? I / 128 : d / 128;                       // M blocks of a routed group
@@ -256,7 +347,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   __syncthreads();
   const int n_units = s_ustart[n_g];
 
-  uint32_t it_load = 0, it_mma = 0;  // running K-tile counters of the producer and of the MMA thread
+  uint32_t it_load = 0, it_mma = 0, it_cv = 0;  // running K-tile counters of the producers, the MMA thread and the converters
   uint32_t unit_no = 0;              // units done by this CTA (phase of the TMEM barriers)
   // The units of this CTA (uu = blockIdx.x, + gridDim.x, ...) are described once, kUnitChunk at a time and a thread
   // per unit: group lookup and index arithmetic are then off every role's path at the unit boundaries, where that
@@ -334,25 +425,47 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         const int s = it_load % NSTAGE;
         if (lane == 0) {
           if (it_load >= (uint32_t)NSTAGE && !mbar_wait(&empty[s], ((it_load / NSTAGE) - 1) & 1, &s_abort, p.f.wait_limit_ns)) ok = false;
-          if (ok) mbar_expect_tx(&full[s], A_BYTES + planes * n_loads * kXRowsPerLoad * 128);
+          CVTL(PHASE, it_load, 4);
+          if (ok) {
+            mbar_expect_tx(&full[s], (QF ? 0 : A_BYTES) + planes * n_loads * kXRowsPerLoad * 128);
+            if (QF) mbar_expect_tx(&rawfull[s], RAW_BYTES);
+          }
         }
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
         uint8_t* st = smem + (size_t)s * STAGE_BYTES;
-        // op 0, 1: the two weight tiles; op 2 + r*planes + pl: 32-row box r of B plane pl
-        const int n_ops = 2 + planes * n_loads;
+        // the weight loads first; then op n_wops + r*planes + pl: 8-row box r of B plane pl
+        constexpr int n_wops = QF == 0 ? 2 : QF == 1 ? (PHASE == 1 ? 2 : 1) : (PHASE == 1 ? 4 : 2);
+        const int n_ops = n_wops + planes * n_loads;
+        uint8_t* raw = st + A_BYTES + planes * B_PLANE;
         for (int op = lane; op < n_ops; op += 32) {
-          if (op < 2) {
-            if (PHASE == 1) tma_load_4d(st + op * 128 * 128, wmap, kt * kKTile, op, blk * 128, slot, &full[s]);   // gate | up rows
-            else tma_load_4d(st + op * 64 * 128, wmap, blk * 128 + op * 64, 2, kt * kKTile, slot, &full[s]);      // downT, 64 columns
+          if (op < n_wops) {
+            if (QF == 0) {
+              if (PHASE == 1) tma_load_4d(st + op * 128 * 128, wmap, kt * kKTile, op, blk * 128, slot, &full[s]);   // gate | up rows
+              else tma_load_4d(st + op * 64 * 128, wmap, blk * 128 + op * 64, 2, kt * kKTile, slot, &full[s]);      // downT, 64 columns
+            } else if (QF == 1) {  // row: gate | up | downT codes (d bytes each), then the scales
+              if (PHASE == 1) tma_load_3d(raw + op * 128 * 64, wmap, op * d + kt * kKTile, blk * 128, slot, &rawfull[s]);
+              else tma_load_3d(raw, wmap, 2 * d + blk * 128, kt * kKTile, slot, &rawfull[s]);
+            } else {  // row: gate | up | downT codes (d/2 bytes each), then their scale bytes (d/32 each)
+              const CUtensorMap* smap = shared ? &tm_ssc : &tm_sc;
+              if (PHASE == 1) {
+                if (op < 2) tma_load_3d(raw + op * 128 * 32, wmap, op * (d / 2) + kt * (kKTile / 2), blk * 128, slot, &rawfull[s]);
+                else tma_load_3d(raw + 2 * 128 * 32 + (op - 2) * 128 * 16, smap, 3 * (d / 2) + (op - 2) * (d / 32) + ((kt * 2) & ~15), blk * 128,
+                                 slot, &rawfull[s]);
+              } else {
+                if (op == 0) tma_load_3d(raw, wmap, d + blk * 64, kt * kKTile, slot, &rawfull[s]);
+                else tma_load_3d(raw + 64 * 64, smap, 3 * (d / 2) + 2 * (d / 32) + ((blk * 4) & ~15), kt * kKTile, slot, &rawfull[s]);
+              }
+            }
           } else {
             // B rows of this stage: the tokens' rows of plane 0, padded to n_pad, then those of plane 1
-            const int r = (op - 2) / planes, pl = (op - 2) % planes;
+            const int r = (op - n_wops) / planes, pl = (op - n_wops) % planes;
             tma_load_2d(st + A_BYTES + pl * n_pad * 128 + r * kXRowsPerLoad * 128, pl ? &tm_b2 : &tm_b, kt * kKTile,
                         gr.pair_off + r * kXRowsPerLoad, &full[s]);
           }
         }
         __syncwarp();
+        if (lane == 0) CVTL(PHASE, it_load, 0);
       }
       if (!ok && lane == 0) {
         atomicExch(&s_abort, 1);
@@ -381,6 +494,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
             break;
           }
           if (kt - kt_begin < 10) TCTL(PHASE, unit_no * 16 + 1 + kt - kt_begin);
+          CVTL(PHASE, it_mma, 5);
           tc_fence_after();
           const uint32_t a0 = smem_u32(smem + (size_t)s * STAGE_BYTES);
           const uint32_t b0 = a0 + A_BYTES;
@@ -396,12 +510,93 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
             }
           }
           umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
+          CVTL(PHASE, it_mma, 6);
         }
         TCTL(PHASE, unit_no * 16 + 11);
         if (ok) umma_commit(&tmem_full[buf]);
         else atomicExch(&s_abort, 1);
         TCTL(PHASE, unit_no * 16 + 14);
       }
+    } else if (QF != 0 && warp >= kCvWarp0) {
+      // ================= converters: raw codes of a stage -> bf16 operand tiles in the 128-byte-swizzled layout
+      // (a tile row is 128 bytes = 64 values; its 16-byte chunk j sits at chunk j ^ (row mod 8))
+      const int ct = tid - kCvWarp0 * 32;
+      bool ok = true;
+      for (int kt = kt_begin; kt < kt_end && ok; ++kt, ++it_cv) {
+        const int s = it_cv % NSTAGE;
+        ok = __all_sync(0xffffffffu, mbar_wait(&rawfull[s], (it_cv / NSTAGE) & 1, &s_abort, p.f.wait_limit_ns));
+        if (ct == 0) CVTL(PHASE, it_cv, 1);
+        if (!ok) break;
+        uint8_t* st = smem + (size_t)s * STAGE_BYTES;
+        const uint8_t* raw = st + A_BYTES + PLANES * B_PLANE;
+        if (QF == 1 && PHASE == 1) {
+          // two tiles [128 rows][64 codes]: chunk q of 16 codes -> two chunks of 8 bf16
+#pragma unroll
+          for (int q = ct; q < 1024; q += kCvThreads) {
+            const int tile = q >> 9, row = (q & 511) >> 2, c = q & 3;
+            const uint4 v = *reinterpret_cast<const uint4*>(raw + q * 16);
+            uint4 o0, o1;
+            e4m3x4_to_bf16(v.x, o0.x, o0.y);
+            e4m3x4_to_bf16(v.y, o0.z, o0.w);
+            e4m3x4_to_bf16(v.z, o1.x, o1.y);
+            e4m3x4_to_bf16(v.w, o1.z, o1.w);
+            uint8_t* dst = st + tile * (128 * 128) + row * 128;
+            *reinterpret_cast<uint4*>(dst + (((2 * c) ^ (row & 7)) << 4)) = o0;
+            *reinterpret_cast<uint4*>(dst + (((2 * c + 1) ^ (row & 7)) << 4)) = o1;
+          }
+        } else if (QF == 1) {
+          // [64 k-rows][128 codes] -> two 64-column atoms, MN-major
+#pragma unroll
+          for (int q = ct; q < 512; q += kCvThreads) {
+            const int kk = q >> 3, cc = q & 7;
+            const uint4 v = *reinterpret_cast<const uint4*>(raw + q * 16);
+            uint4 o0, o1;
+            e4m3x4_to_bf16(v.x, o0.x, o0.y);
+            e4m3x4_to_bf16(v.y, o0.z, o0.w);
+            e4m3x4_to_bf16(v.z, o1.x, o1.y);
+            e4m3x4_to_bf16(v.w, o1.z, o1.w);
+            uint8_t* dst = st + (cc >> 2) * (64 * 128) + kk * 128;
+            const int jc = (cc & 3) * 2;
+            *reinterpret_cast<uint4*>(dst + ((jc ^ (kk & 7)) << 4)) = o0;
+            *reinterpret_cast<uint4*>(dst + (((jc + 1) ^ (kk & 7)) << 4)) = o1;
+          }
+        } else if (PHASE == 1) {
+          // two tiles [128 rows][32 bytes = 64 codes]: a 16-byte chunk is one 32-element scale block
+          const uint8_t* rsc = raw + 2 * 128 * 32;
+#pragma unroll
+          for (int q = ct; q < 512; q += kCvThreads) {
+            const int tile = q >> 8, row = (q & 255) >> 1, half = q & 1;
+            const uint4 v = *reinterpret_cast<const uint4*>(raw + q * 16);
+            const uint32_t sc = rsc[tile * (128 * 16) + row * 16 + ((kt * 2) & 15) + half];
+            uint8_t* dst = st + tile * (128 * 128) + row * 128;
+            const int jc = half * 4;
+            *reinterpret_cast<uint4*>(dst + (((jc + 0) ^ (row & 7)) << 4)) = e2m1x8_to_bf16(v.x, sc);
+            *reinterpret_cast<uint4*>(dst + (((jc + 1) ^ (row & 7)) << 4)) = e2m1x8_to_bf16(v.y, sc);
+            *reinterpret_cast<uint4*>(dst + (((jc + 2) ^ (row & 7)) << 4)) = e2m1x8_to_bf16(v.z, sc);
+            *reinterpret_cast<uint4*>(dst + (((jc + 3) ^ (row & 7)) << 4)) = e2m1x8_to_bf16(v.w, sc);
+          }
+        } else {
+          // [64 k-rows][64 bytes = 128 codes]: chunk cb of a row is the scale block of columns 32 cb .. 32 cb + 31
+          const uint8_t* rsc = raw + 64 * 64;
+#pragma unroll
+          for (int q = ct; q < 256; q += kCvThreads) {
+            const int kk = q >> 2, cb = q & 3;
+            const uint4 v = *reinterpret_cast<const uint4*>(raw + q * 16);
+            const uint32_t sc = rsc[kk * 16 + ((blk * 4) & 15) + cb];
+            uint8_t* dst = st + (cb >> 1) * (64 * 128) + kk * 128;
+            const int jc = (cb & 1) * 4;
+            *reinterpret_cast<uint4*>(dst + (((jc + 0) ^ (kk & 7)) << 4)) = e2m1x8_to_bf16(v.x, sc);
+            *reinterpret_cast<uint4*>(dst + (((jc + 1) ^ (kk & 7)) << 4)) = e2m1x8_to_bf16(v.y, sc);
+            *reinterpret_cast<uint4*>(dst + (((jc + 2) ^ (kk & 7)) << 4)) = e2m1x8_to_bf16(v.z, sc);
+            *reinterpret_cast<uint4*>(dst + (((jc + 3) ^ (kk & 7)) << 4)) = e2m1x8_to_bf16(v.w, sc);
+          }
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the MMAs read these tiles through the async proxy
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&full[s]);
+        if (ct == 0) CVTL(PHASE, it_cv, 3);
+      }
+      if (!ok && lane == 0) atomicExch(&s_abort, 1);
     } else {
       // ================= epilogue: warp w owns TMEM lanes 32*(w%4) .. +31
       const int quad = warp & 3;
@@ -416,15 +611,23 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
           tmem_ld32(taddr, a);
           uint32_t b2[32];
           tmem_ld32(taddr + (PHASE == 1 ? 128 : n_pad), b2);   // U | the a_lo half of the down product
+          asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
           if (PHASE == 1) {
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             const int i = blk * 128 + row;
+            float sg = 1.f, su = 1.f, sd = 1.f;
+            if (QF == 1) {  // the row's three fp32 scales follow its 3 d code bytes
+              const uint8_t* wb = shared ? p.f.shared_w : p.f.cache + (size_t)p.f.snap.expert_slot[gr.expert] * p.f.slot_stride;
+              const float* sc = reinterpret_cast<const float*>(wb + (size_t)i * (3u * d + 16u) + 3u * d);
+              sg = __ldg(sc);
+              su = __ldg(sc + 1);
+              sd = __ldg(sc + 2);
+            }
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
               if (c0 + j < gr.n_tok) {
-                const float gq = __uint_as_float(a[j]), uq = __uint_as_float(b2[j]);
+                const float gq = sg * __uint_as_float(a[j]), uq = su * __uint_as_float(b2[j]);
                 const float w = __ldg(p.f.pair_gate + gr.pair_off + c0 + j);
-                const float v = w * (gq / (1.f + expf(-gq))) * uq;
+                const float v = w * (gq / (1.f + expf(-gq))) * uq * sd;
                 const __nv_bfloat16 hi = __float2bfloat16(v);
                 const size_t at = (size_t)(gr.pair_off + c0 + j) * p.act_stride + i;
                 p.act[at] = hi;
@@ -432,7 +635,6 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
               }
             }
           } else {
-            asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory");
             const int col = blk * 128 + row;
 #pragma unroll
             for (int j = 0; j < 32; ++j) {
@@ -462,6 +664,9 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
 #ifdef APEX_TIMELINE
 extern "C" int apex_debug_read_tc_timeline(unsigned long long* host) {
   return (int)cudaMemcpyFromSymbol(host, g_tc_tl, sizeof(g_tc_tl));
+}
+extern "C" int apex_debug_read_tc_converter_timeline(unsigned long long* host) {
+  return (int)cudaMemcpyFromSymbol(host, g_cv_tl, sizeof(g_cv_tl));
 }
 #endif
 
@@ -508,9 +713,70 @@ bool tc_make_rows_map(void* out, const void* base, int cols, size_t rows, size_t
             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-bool tc_shape_supported(int d, int I, int I_shared) {
-  return d % 128 == 0 && I % 128 == 0 && I_shared % 128 == 0;
+// Raw bytes of n_slots consecutive slots of a quantised store, each [I][row_bytes]: dims (row_bytes, I, n_slots);
+// box (box_bytes, box_rows, 1), no swizzle (the converters read the staging area with plain loads).
+bool tc_make_raw_map(void* out, const void* base, size_t row_bytes, int I, size_t n_slots, size_t slot_bytes, int box_bytes, int box_rows) {
+  EncodeTiledFn fn = encode_fn();
+  if (!fn) return false;
+  cuuint64_t dims[3] = {(cuuint64_t)row_bytes, (cuuint64_t)I, (cuuint64_t)n_slots};
+  cuuint64_t strides[2] = {(cuuint64_t)row_bytes, (cuuint64_t)slot_bytes};
+  cuuint32_t box[3] = {(cuuint32_t)box_bytes, (cuuint32_t)box_rows, 1};
+  cuuint32_t es[3] = {1, 1, 1};
+  return fn(reinterpret_cast<CUtensorMap*>(out), CU_TENSOR_MAP_DATA_TYPE_UINT8, 3, const_cast<void*>(base), dims, strides, box, es,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+            CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
+
+// The weight maps of one store (the slots of all layers, or one shared expert) for the storage format.
+bool tc_make_store_maps(int fmt, void* gateup, void* down, void* sc_gateup, void* sc_down, const void* base, int d, int I, size_t n_slots,
+                        size_t slot_bytes) {
+  if (fmt == 0)
+    return tc_make_weight_map(gateup, base, d, I, n_slots, slot_bytes, 128) && tc_make_weight_map(down, base, d, I, n_slots, slot_bytes, 64);
+  const size_t rb = ffn_row_bytes(fmt, d);
+  if (fmt == 1)  // a K tile of 64 codes is 64 bytes of a gate / up row; 128 columns of a downT row are 128 bytes
+    return tc_make_raw_map(gateup, base, rb, I, n_slots, slot_bytes, 64, 128) && tc_make_raw_map(down, base, rb, I, n_slots, slot_bytes, 128, 64);
+  return tc_make_raw_map(gateup, base, rb, I, n_slots, slot_bytes, 32, 128) && tc_make_raw_map(down, base, rb, I, n_slots, slot_bytes, 64, 64) &&
+         tc_make_raw_map(sc_gateup, base, rb, I, n_slots, slot_bytes, 16, 128) && tc_make_raw_map(sc_down, base, rb, I, n_slots, slot_bytes, 16, 64);
+}
+
+bool tc_shape_supported(int d, int I, int I_shared, int fmt) {
+  if (d % 128 != 0 || I % 128 != 0 || I_shared % 128 != 0) return false;
+  if (fmt == 1) return d % 256 == 0;   // code offsets of a row stay 16-byte aligned
+  if (fmt == 2) return d % 512 == 0;   // ... and so do the scale bytes of each vector (d / 32 of them)
+  return true;
+}
+
+namespace {
+template <int QF>
+cudaError_t launch_tc_gemms(const TcParams& p, const TcMaps& m, cudaLaunchConfig_t& cfg, size_t ring1, size_t ring2, size_t st1, size_t st2) {
+  const CUtensorMap* w1 = reinterpret_cast<const CUtensorMap*>(m.w_gateup);
+  const CUtensorMap* ws1 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_gateup : m.w_gateup);
+  const CUtensorMap* w2 = reinterpret_cast<const CUtensorMap*>(m.w_down);
+  const CUtensorMap* ws2 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_down : m.w_down);
+  // the 16-byte-box maps exist for the e2m1 store only; the other formats pass the weight maps again (never used)
+  const CUtensorMap* c1 = QF == 2 ? reinterpret_cast<const CUtensorMap*>(m.sc_gateup) : w1;
+  const CUtensorMap* cs1 = QF == 2 ? reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ssc_gateup : m.sc_gateup) : w1;
+  const CUtensorMap* c2 = QF == 2 ? reinterpret_cast<const CUtensorMap*>(m.sc_down) : w2;
+  const CUtensorMap* cs2 = QF == 2 ? reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ssc_down : m.sc_down) : w2;
+  const CUtensorMap* xg = reinterpret_cast<const CUtensorMap*>(m.xg);
+  cfg.blockDim = dim3(tc_threads(QF), 1, 1);
+  // Each CTA allocates all 512 TMEM columns, so two CTAs must never share an SM (the second would sit in
+  // tcgen05.alloc until the first has finished): ask for more than half an SM's shared memory in any case.
+  const size_t one_per_sm = 120 * 1024;
+  cfg.dynamicSmemBytes = ring1 + p.nstage1 * st1 + 1024 > one_per_sm ? ring1 + p.nstage1 * st1 + 1024 : one_per_sm;
+  cudaError_t e = cudaLaunchKernelEx(&cfg, ffn_tc_gemm_kernel<1, QF>, *w1, *ws1, *c1, *cs1, *xg, *xg, p);
+  if (e != cudaSuccess) return e;
+  cfg.dynamicSmemBytes = ring2 + p.nstage2 * st2 + 1024 > one_per_sm ? ring2 + p.nstage2 * st2 + 1024 : one_per_sm;
+  return cudaLaunchKernelEx(&cfg, ffn_tc_gemm_kernel<2, QF>, *w2, *ws2, *c2, *cs2, *reinterpret_cast<const CUtensorMap*>(m.act),
+                            *reinterpret_cast<const CUtensorMap*>(m.act_lo), p);
+}
+template <int QF>
+cudaError_t configure_tc(int budget) {
+  cudaError_t e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<1, QF>, cudaFuncAttributeMaxDynamicSharedMemorySize, budget);
+  if (e != cudaSuccess) return e;
+  return cudaFuncSetAttribute(ffn_tc_gemm_kernel<2, QF>, cudaFuncAttributeMaxDynamicSharedMemorySize, budget);
+}
+}  // namespace
 
 cudaError_t launch_ffn_tc(const TcParams& p_in, const TcMaps& m, int n_sm, cudaStream_t s) {
   static bool configured[kMaxDevices] = {};  // the attribute is per device
@@ -518,17 +784,20 @@ cudaError_t launch_ffn_tc(const TcParams& p_in, const TcMaps& m, int n_sm, cudaS
   int dev = 0;
   cudaGetDevice(&dev);
   if (dev < 0 || dev >= kMaxDevices || !configured[dev]) {
-    cudaError_t e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<1>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget + 1024);
-    if (e != cudaSuccess) return e;
-    e = cudaFuncSetAttribute(ffn_tc_gemm_kernel<2>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)budget + 1024);
+    cudaError_t e = configure_tc<0>((int)budget + 1024);
+    if (e == cudaSuccess) e = configure_tc<1>((int)budget + 1024);
+    if (e == cudaSuccess) e = configure_tc<2>((int)budget + 1024);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < kMaxDevices) configured[dev] = true;
   }
   TcParams p = p_in;
+  const int qf = p.f.fmt;
   const int b32 = (p.f.B + 31) & ~31;
   p.nmax1 = b32 < 128 ? b32 : 128;
   p.nmax2 = b32 < 64 ? b32 : 64;
-  const size_t st1 = 2 * 128 * 128 + (size_t)p.nmax1 * 128, st2 = 2 * 64 * 128 + 2 * (size_t)p.nmax2 * 128;
+  const size_t ring1 = 0, ring2 = 0;
+  const size_t st1 = 2 * 128 * 128 + (size_t)p.nmax1 * 128 + tc_raw_bytes(1, qf);
+  const size_t st2 = 2 * 64 * 128 + 2 * (size_t)p.nmax2 * 128 + tc_raw_bytes(2, qf);
   p.nstage1 = (int)(budget / st1) < 4 ? (int)(budget / st1) : 4;
   p.nstage2 = (int)(budget / st2) < 4 ? (int)(budget / st2) : 4;
   cudaLaunchAttribute attr[1];
@@ -543,22 +812,9 @@ cudaError_t launch_ffn_tc(const TcParams& p_in, const TcMaps& m, int n_sm, cudaS
   cfg.dynamicSmemBytes = 0;
   cudaError_t e = cudaLaunchKernelEx(&cfg, ffn_tc_gather_kernel, p);
   if (e != cudaSuccess) return e;
-  const CUtensorMap* w1 = reinterpret_cast<const CUtensorMap*>(m.w_gateup);
-  const CUtensorMap* ws1 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_gateup : m.w_gateup);
-  const CUtensorMap* w2 = reinterpret_cast<const CUtensorMap*>(m.w_down);
-  const CUtensorMap* ws2 = reinterpret_cast<const CUtensorMap*>(p.f.shared_w ? m.ws_down : m.w_down);
-  const CUtensorMap* xg = reinterpret_cast<const CUtensorMap*>(m.xg);
   cfg.gridDim = dim3(n_sm, 1, 1);
-  cfg.blockDim = dim3(kTcThreads, 1, 1);
-  // Each CTA allocates all 512 TMEM columns, so two CTAs must never share an SM (the second would sit in
-  // tcgen05.alloc until the first has finished): ask for more than half an SM's shared memory in any case.
-  const size_t one_per_sm = 120 * 1024;
-  cfg.dynamicSmemBytes = p.nstage1 * st1 + 1024 > one_per_sm ? p.nstage1 * st1 + 1024 : one_per_sm;
-  e = cudaLaunchKernelEx(&cfg, ffn_tc_gemm_kernel<1>, *w1, *ws1, *xg, *xg, p);
-  if (e != cudaSuccess) return e;
-  cfg.dynamicSmemBytes = p.nstage2 * st2 + 1024 > one_per_sm ? p.nstage2 * st2 + 1024 : one_per_sm;
-  return cudaLaunchKernelEx(&cfg, ffn_tc_gemm_kernel<2>, *w2, *ws2, *reinterpret_cast<const CUtensorMap*>(m.act),
-                            *reinterpret_cast<const CUtensorMap*>(m.act_lo), p);
+  return qf == 1 ? launch_tc_gemms<1>(p, m, cfg, ring1, ring2, st1, st2)
+                 : qf == 2 ? launch_tc_gemms<2>(p, m, cfg, ring1, ring2, st1, st2) : launch_tc_gemms<0>(p, m, cfg, ring1, ring2, st1, st2);
 }
 
 }  // namespace apex

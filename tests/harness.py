@@ -49,10 +49,12 @@ class Problem:
     """Parameters and expert stores of one config on the GPU machine, shared by library and oracle."""
 
     def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset", fp8=False, fp4=False,
-                 store_layers: Optional[int] = None):
+                 store_layers: Optional[int] = None, fp8_code_mask: Optional[int] = None):
         """cdf: "handset", "fitted", or ("static", delta): the static over-fetch model of Sec. V-A (w = 0 and a step
         in theta, so delta_hat = delta for every token).  store_layers: physical expert stores (layer l uses store
-        l mod store_layers; for shapes whose full store does not fit the host's memory)."""
+        l mod store_layers; for shapes whose full store does not fit the host's memory).  fp8_code_mask: and-ed onto
+        every e4m3 code byte of the stores (0x8F leaves sign, the lowest exponent bit and the mantissa: half the codes
+        are then subnormal and the rest sit in the lowest binade, so a path that mishandles subnormal codes shows)."""
         self.cfg = cfg
         self.fp8 = fp8
         self.fp4 = fp4
@@ -84,12 +86,16 @@ class Problem:
                 tmp = synth.expert_store(cfg, l, device=device)
             st.copy_(tmp)
             del tmp
+            if fp8 and fp8_code_mask is not None:
+                st[..., :3 * cfg.d] &= fp8_code_mask
             self.stores.append(st)
             sh = synth.shared_expert(cfg, l, device=device)
             if fp4 and sh is not None:
                 sh = synth.quantize_store_fp4(sh)
             elif fp8 and sh is not None:
                 sh = synth.quantize_store_fp8(sh)
+                if fp8_code_mask is not None:
+                    sh[..., :3 * cfg.d] &= fp8_code_mask
             self.shared.append(sh)
         torch.cuda.synchronize()
 

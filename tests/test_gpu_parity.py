@@ -159,10 +159,11 @@ def test_batched_exact_mode_runs_in_waves_when_cache_is_smaller_than_need():
 
 
 # ------------------------------------------------------------------ e4m3 expert store (Sec. V-G)
-def _run_fp8(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1):
+def _run_fp8(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1, ffn_token_stride=1):
     hz = _harness()
     prob = hz.Problem(cfg, layers=layers, fp8=True)
-    return _run(cfg, mode=mode, tau=tau, T=T, B=B, layers=layers, prob=prob, check_ffn_every=check_ffn_every)
+    return _run(cfg, mode=mode, tau=tau, T=T, B=B, layers=layers, prob=prob, check_ffn_every=check_ffn_every,
+                ffn_token_stride=ffn_token_stride)
 
 
 @pytest.mark.parametrize("mode", ["exact", "stall_free"])
@@ -176,11 +177,55 @@ def test_fp8_store_tiny_shapes(d, N, k, I, C, Ish, mode):
     print("fp8", d, mode, rep)
 
 
-@pytest.mark.parametrize("B", [3, 16])
-def test_fp8_store_batched_runs_streaming_kernel(B):
+def test_fp8_store_small_batch_runs_streaming_kernel():
     cfg = synth.tiny_config(d=512, N=12, k=3, I=128, C=8, T=3, I_shared=128, sigma_p=1.0, cfg_id=275)
-    rep, stats = _run_fp8(cfg, mode="exact", tau=0.8, T=3, B=B)
-    assert stats["tokens"] == 3 * B
+    rep, stats = _run_fp8(cfg, mode="exact", tau=0.8, T=3, B=3)
+    assert stats["tokens"] == 9
+
+
+@pytest.mark.parametrize("B", [16, 40, 97])
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+@pytest.mark.parametrize("fmt", ["fp8", "fp4"])
+def test_quantised_store_tensor_core_path(fmt, B, mode):
+    # B >= 16 with d, I, I_shared the grouped GEMM accepts: converter warps expand the code tiles to bf16 operand tiles.
+    # I = 256 gives two row blocks per expert and four K tiles in the down projection; I_shared = 384 a longer K there
+    # (cut into chunks); d = 512 gives eight K tiles in gate / up, so the e2m1 scale bytes of a row cross no 16-byte group,
+    # and the four column blocks of the down projection use all four scale offsets of one.
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=256, C=8, T=3, I_shared=384, sigma_p=1.0, cfg_id=276)
+    rep, stats = (_run_fp8 if fmt == "fp8" else _run_fp4)(cfg, mode=mode, tau=0.8, T=3, B=B)
+    assert stats["tokens"] == 3 * B and rep.ffn_checked == 3 * B and rep.near_ties == 0
+    print("tc", fmt, B, mode, rep)
+
+
+@pytest.mark.parametrize("B", [1, 24])
+def test_fp8_store_of_subnormal_codes(B):
+    # every code byte and-ed with 0x8F: exponent field 0 or 1 only, so half the weights are e4m3 subnormals and none is
+    # large enough to hide them; B = 1 runs the streaming kernel, B = 24 the converters of the tensor-core path
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=128, C=8, T=2, I_shared=128, sigma_p=1.0, cfg_id=278)
+    hz = _harness()
+    prob = hz.Problem(cfg, fp8=True, fp8_code_mask=0x8F)
+    codes = prob.stores[0][..., :3 * cfg.d].numpy()
+    assert 0.3 < float(np.mean((codes >> 3) & 0xF == 0)) < 0.7 and int(((codes >> 3) & 0xF).max()) == 1
+    rep, stats = _run(cfg, mode="exact", tau=0.8, T=2, B=B, prob=prob)
+    assert rep.ffn_checked == 2 * B and rep.near_ties == 0
+
+
+@pytest.mark.parametrize("fmt", ["fp8", "fp4"])
+def test_quantised_store_tensor_core_path_wide(fmt):
+    # d = 1024: sixteen K tiles, so the e2m1 scale bytes of a gate / up row span two 16-byte groups; 8 column blocks in
+    # the down projection span two groups as well.  No shared expert.
+    cfg = synth.tiny_config(d=1024, N=8, k=2, I=128, C=8, T=2, sigma_p=1.0, cfg_id=277)
+    rep, stats = (_run_fp8 if fmt == "fp8" else _run_fp4)(cfg, mode="exact", tau=0.8, T=2, B=33)
+    assert stats["tokens"] == 66 and rep.ffn_checked == 66 and rep.near_ties == 0
+
+
+@pytest.mark.parametrize("fmt", ["fp8", "fp4"])
+def test_quantised_store_config4_shape_tensor_core_batch(fmt):
+    # config 4's shape (d = 2048, I = 768, 60 experts, 4 shared) at B = 32, one layer, FFN output of every 8th token
+    cfg = synth.CONFIGS[4]
+    rep, stats = (_run_fp8 if fmt == "fp8" else _run_fp4)(cfg, mode="exact", tau=0.9, T=1, layers=1, B=32, ffn_token_stride=8)
+    assert stats["tokens"] == 32 and rep.ffn_checked >= 4 and rep.near_ties == 0
+    print("config4-tc", fmt, rep, stats)
 
 
 @pytest.mark.parametrize("mode", ["exact", "stall_free"])
@@ -192,10 +237,11 @@ def test_fp8_store_config1_shape_two_layers(mode):
 
 
 # ------------------------------------------------------------------ block-scaled e2m1 expert store
-def _run_fp4(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1):
+def _run_fp4(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1, ffn_token_stride=1):
     hz = _harness()
     prob = hz.Problem(cfg, layers=layers, fp4=True)
-    return _run(cfg, mode=mode, tau=tau, T=T, B=B, layers=layers, prob=prob, check_ffn_every=check_ffn_every)
+    return _run(cfg, mode=mode, tau=tau, T=T, B=B, layers=layers, prob=prob, check_ffn_every=check_ffn_every,
+                ffn_token_stride=ffn_token_stride)
 
 
 @pytest.mark.parametrize("mode", ["exact", "stall_free"])
@@ -209,7 +255,7 @@ def test_fp4_store_tiny_shapes(d, N, k, I, C, Ish, mode):
     print("fp4", d, mode, rep)
 
 
-def test_fp4_store_batched_runs_streaming_kernel():
+def test_fp4_store_small_batch_runs_streaming_kernel():
     cfg = synth.tiny_config(d=512, N=12, k=3, I=128, C=8, T=3, I_shared=128, sigma_p=1.0, cfg_id=315)
     rep, stats = _run_fp4(cfg, mode="exact", tau=0.8, T=3, B=5)
     assert stats["tokens"] == 15

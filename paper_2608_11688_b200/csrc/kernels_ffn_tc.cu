@@ -487,6 +487,8 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         // An MMA costs about 128 cycles whatever N is (it streams a 128 x 16 slice of A), so the down
         // projection multiplies both planes of the intermediate in one instruction: N = 2 * n_pad.
         const uint32_t idesc = umma_idesc(128, PHASE == 2 ? 2 * n_pad : n_pad, PHASE == 2 ? 1 : 0);
+        const uint64_t desc_a0 = PHASE == 1 ? umma_desc(smem_u32(smem), 16, 1024) : umma_desc(smem_u32(smem), 64 * 128, 1024);
+        const uint64_t desc_b0 = umma_desc(smem_u32(smem) + A_BYTES, 16, 1024);
         for (int kt = kt_begin; kt < kt_end && ok; ++kt, ++it_mma) {
           const int s = it_mma % NSTAGE;
           if (!mbar_wait(&full[s], (it_mma / NSTAGE) & 1, &s_abort, p.f.wait_limit_ns)) {
@@ -496,17 +498,19 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
           if (kt - kt_begin < 10) TCTL(PHASE, unit_no * 16 + 1 + kt - kt_begin);
           CVTL(PHASE, it_mma, 5);
           tc_fence_after();
-          const uint32_t a0 = smem_u32(smem + (size_t)s * STAGE_BYTES);
-          const uint32_t b0 = a0 + A_BYTES;
+          // descriptors differ from the stage-0, k-step-0 ones only in the start-address field (address >> 4, the low
+          // 14 bits; the sums below stay inside the CTA's shared memory, so nothing carries into the next field)
+          const uint64_t soff = (uint64_t)((uint32_t)s * (uint32_t)STAGE_BYTES >> 4);
+          const uint64_t da = desc_a0 + soff, db = desc_b0 + soff;
 #pragma unroll
           for (int ks = 0; ks < kKTile / 16; ++ks) {
             const uint32_t acc = (kt > kt_begin || ks > 0) ? 1u : 0u;
-            const uint64_t bdesc = umma_desc(b0 + ks * 32, 16, 1024);
+            const uint64_t bdesc = db + (uint64_t)(ks * 2);   // 32 bytes per k-step
             if (PHASE == 1) {
-              umma(tacc, umma_desc(a0 + ks * 32, 16, 1024), bdesc, idesc, acc);                     // G
-              umma(tacc + 128, umma_desc(a0 + 128 * 128 + ks * 32, 16, 1024), bdesc, idesc, acc);   // U
+              umma(tacc, da + (uint64_t)(ks * 2), bdesc, idesc, acc);                           // G
+              umma(tacc + 128, da + (uint64_t)(128 * 128 / 16 + ks * 2), bdesc, idesc, acc);    // U
             } else {
-              umma(tacc, umma_desc(a0 + ks * 2048, 64 * 128, 1024), bdesc, idesc, acc);  // columns [0, n_pad): a_hi, [n_pad, 2 n_pad): a_lo
+              umma(tacc, da + (uint64_t)(ks * 128), bdesc, idesc, acc);  // 2 KB per k-step; columns [0, n_pad): a_hi, [n_pad, 2 n_pad): a_lo
             }
           }
           umma_commit(&empty[s]);  // the stage is free once these MMAs have read it

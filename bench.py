@@ -148,43 +148,55 @@ def make_ctx(cfg, prob, C, max_batch=1, flags=0, link_gbs=0.0, ctx_len=1024, cac
 def train_auxiliary(cfg, prob, device, n_calib=8192, distill_iters=100, distill_lr=1e-4, fit_iters=600):
     """The paper's two training stages on this GPU (Sec. IV-C): distil the prefetch router of every layer from the
     router (Eq. (10)), then refit the confidence model on the distilled router's rankings (Eq. (11)).  Returns new
-    (routers, cdf) lists; the calibration tokens come from the seeded generator's calibration stream.  The step size
-    is small on purpose: a layer has N * (d + 1) parameters and only n_calib tokens, and Adam moves every weight by
-    about lr per step whatever its gradient, so a larger step overfits the calibration set within a few iterations."""
+    (routers, cdf) lists; the calibration tokens come from the seeded generator's calibration stream.  Teacher
+    distributions, rankings and routed sets are the library's own outputs (apex_route_topk; apex_predict +
+    apex_read_prediction), taken in batches on a context without expert stores; only the bookkeeping that turns a
+    ranking and a routed set into a calibration pair (x = q_p in rank order, delta* = largest rank of a routed expert
+    - k, Eq. (3)) is done here.  The step size is small on purpose: a layer has N * (d + 1) parameters and only
+    n_calib tokens, and Adam moves every weight by about lr per step whatever its gradient, so a larger step
+    overfits the calibration set within a few iterations."""
     import torch
     from paper_2608_11688_b200 import binding, synth
     routers, cdf, store, shared = prob
+    MB = 256
+    a = binding.Apex(d=cfg.d, N=cfg.N, k=cfg.k, I=cfg.I, C_slots=cfg.k, L=cfg.L, I_shared=cfg.I_shared, max_batch=MB)
     new_routers, new_cdf = [], []
     t_d = t_f = 0.0
-    for l in range(cfg.L):
-        W_r, b_r, W_p, b_p = routers[l]
-        h, hp = synth.hidden_states(cfg, l, n_calib, 1, calib=True)
-        H, Hp = h[:, 0].astype(np.float64), hp[:, 0].astype(np.float64)
-        Zr = Hp @ W_r.astype(np.float64).T + b_r.astype(np.float64)
-        Qr = np.exp(Zr - Zr.max(1, keepdims=True))
-        Qr /= Qr.sum(1, keepdims=True)
-        Hd = torch.from_numpy(H.astype(np.float32)).to(device)
-        t0 = time.perf_counter()
-        W_p2, b_p2 = binding.distill_router(Hd, torch.from_numpy(Qr.astype(np.float32)).to(device), W_p, b_p,
-                                            iters=distill_iters, lr=distill_lr)
-        t_d += time.perf_counter() - t0
-        # calibration set of the confidence model: x = the distilled router's probabilities in descending order,
-        # delta* = (largest rank of a routed expert in its ranking) - k
-        Zp = H @ W_p2.astype(np.float64).T + b_p2.astype(np.float64)
-        order = np.lexsort((np.broadcast_to(np.arange(cfg.N), Zp.shape), -Zp), axis=1)     # value desc, index asc
-        Qp = np.exp(Zp - Zp.max(1, keepdims=True))
-        Qp /= Qp.sum(1, keepdims=True)
-        X = np.take_along_axis(Qp, order, axis=1)
-        rank = np.empty_like(order)
-        np.put_along_axis(rank, order, np.broadcast_to(np.arange(cfg.N), order.shape), axis=1)
-        K_r = np.lexsort((np.broadcast_to(np.arange(cfg.N), Zr.shape), -Zr), axis=1)[:, :cfg.k]
-        dstar = np.take_along_axis(rank, K_r, axis=1).max(1) + 1 - cfg.k
-        t0 = time.perf_counter()
-        w, theta = binding.fit_cdf(torch.from_numpy(X).to(device), torch.from_numpy(dstar.astype(np.int32)).to(device),
-                                   cfg.k, iters=fit_iters)
-        t_f += time.perf_counter() - t0
-        new_routers.append((W_r, b_r, W_p2, b_p2))
-        new_cdf.append((w, theta))
+    try:
+        for l in range(cfg.L):
+            W_r, b_r, W_p, b_p = routers[l]
+            a.set_router(l, W_r, b_r)
+            h, hp = synth.hidden_states(cfg, l, n_calib, 1, calib=True)
+            Hd = torch.from_numpy(np.ascontiguousarray(h[:, 0])).to(device)
+            Hpd = torch.from_numpy(np.ascontiguousarray(hp[:, 0])).to(device)
+            Qr = torch.empty((n_calib, cfg.N), dtype=torch.float32, device=device)      # teacher: alpha = softmax(z_r)
+            K_r = torch.empty((n_calib, cfg.k), dtype=torch.int32, device=device)
+            for s0 in range(0, n_calib, MB):
+                b = min(MB, n_calib - s0)
+                a.route_topk(l, Hpd[s0:s0 + b], b, K_r[s0:s0 + b], Qr[s0:s0 + b])
+            torch.cuda.synchronize()
+            t0 = time.perf_counter()
+            W_p2, b_p2 = binding.distill_router(Hd, Qr, W_p, b_p, iters=distill_iters, lr=distill_lr)
+            t_d += time.perf_counter() - t0
+            # calibration set of the confidence model from the distilled router's own predictions
+            a.set_prefetch_router(l, W_p2, b_p2)
+            X = np.empty((n_calib, cfg.N), np.float32)
+            rank = np.empty((n_calib, cfg.N), np.int64)
+            for s0 in range(0, n_calib, MB):
+                b = min(MB, n_calib - s0)
+                a.predict(l, Hd[s0:s0 + b], b)
+                _, q_p, pi = a.read_prediction(b)
+                X[s0:s0 + b] = np.take_along_axis(q_p, pi.astype(np.int64), axis=1)
+                np.put_along_axis(rank[s0:s0 + b], pi.astype(np.int64), np.broadcast_to(np.arange(cfg.N), pi.shape), axis=1)
+            dstar = np.take_along_axis(rank, K_r.cpu().numpy().astype(np.int64), axis=1).max(1) + 1 - cfg.k
+            t0 = time.perf_counter()
+            w, theta = binding.fit_cdf(torch.from_numpy(X.astype(np.float64)).to(device),
+                                       torch.from_numpy(dstar.astype(np.int32)).to(device), cfg.k, iters=fit_iters)
+            t_f += time.perf_counter() - t0
+            new_routers.append((W_r, b_r, W_p2, b_p2))
+            new_cdf.append((w, theta))
+    finally:
+        a.destroy()
     return new_routers, new_cdf, {"distill_s": t_d, "fit_s": t_f, "calibration_tokens_per_layer": n_calib}
 
 
@@ -377,6 +389,46 @@ def time_token_kernel(cfg, prob, h, hp, y, tokens, standin):
         a.destroy()
 
 
+def other_config_rooflines(dev, peak, peak_kind):
+    """The expert-FFN launch of the other configs of the workload table against the same roofline: all experts resident,
+    a few layers each (every launch reads its own layer's experts and a token's launches together exceed L2), CUDA
+    events on the launching stream.  B = 1: the streaming kernel; B > 1: plan + gather + the two tcgen05 GEMMs, bytes =
+    expected distinct experts of B uniformly routed tokens.  `traffic` is null: no ncu capture at these shapes except
+    where NCU_TRAFFIC_BYTES has one."""
+    import torch
+    from paper_2608_11688_b200 import synth
+    out = {}
+    for cfg_id, layers, batches in ((0, 8, (1,)), (2, 4, (1,)), (3, 2, (1,)), (4, 4, (1, 32, 256))):
+        cfg = synth.CONFIGS[cfg_id].scaled(L=layers)
+        prob = build_problem(cfg, dev)
+        for B in batches:
+            h, hp = hidden_inputs(cfg, 4, B, dev)
+            h, hp = h.to(dev), hp.to(dev)
+            a = make_ctx(cfg, prob, cfg.N, max_batch=B)
+            try:
+                a.warm_all()
+                mean_s, med_s, n_l = time_ffn_kernel(a, cfg, h, hp, B, tokens=6)
+            finally:
+                a.destroy()
+            if B == 1:
+                _, bytes_ffn = algorithmic_bytes(cfg, B)
+                kernel = "moe_ffn_stream_kernel"
+            else:
+                distinct = cfg.N * (1.0 - (1.0 - cfg.k / cfg.N) ** B)
+                bytes_ffn = distinct * cfg.expert_bytes + cfg.shared_bytes + 2 * B * cfg.d * 4
+                kernel = "ffn_plan_kernel + ffn_tc_gather_kernel + ffn_tc_gemm_kernel<1>, <2>"
+            ach = bytes_ffn / mean_s / 1e9
+            out[f"config{cfg_id}" + (f"_B{B}" if len(batches) > 1 else "")] = {
+                "bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
+                "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(cfg_id) if B == 1 else None,
+                "algorithmic_bytes_per_launch": bytes_ffn, "us_per_launch_mean": mean_s * 1e6, "launches_timed": n_l,
+                "layers": layers, "B": B}
+            del h, hp
+        del prob
+        torch.cuda.empty_cache()
+    return out
+
+
 def oracle_tokens_per_s(cfg, prob, n_tokens):
     """The CPU oracle as it stands, timed on the host cores over n_tokens full decode tokens."""
     import torch
@@ -450,6 +502,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--cpu-baseline-tokens", type=int, default=2)
     ap.add_argument("--skip-extras", action="store_true", help="only the headline leg (used for ncu launch lists)")
+    ap.add_argument("--no-other-configs", dest="other_configs", action="store_false",
+                    help="leave out the roofline sub-records of configs 0, 2, 3 and 4 (they add about a minute)")
     ap.add_argument("--ffn-only", action="store_true",
                     help="profiling case: all experts resident, gate + expert FFN only, no copy in flight")
     ap.add_argument("--layers", type=int, default=None, help="use only the first LAYERS layers (smaller captures)")
@@ -697,6 +751,9 @@ def main():
                                              "achieved": (bytes_tok + cfg.L * attn_bytes) / sec_att / 1e9,
                                              "frac": (bytes_tok + cfg.L * attn_bytes) / sec_att / 1e9 / peak},
                             "per_layer_ffn_kernel_alone": ffn_alone}
+            # ---- the same roofline for the FFN launch of the other configs (a few layers each)
+            if args.other_configs and world == 1:
+                extras["roofline_other_configs"] = other_config_rooflines(dev, peak, f"{peak_kind}")
             # ---- the oracle on the host cores (bounded sample)
             tps, cores, dt = oracle_tokens_per_s(cfg, prob, args.cpu_baseline_tokens)
             cpu = {"value": tps, "unit": UNIT, "cores": cores, "kind": "oracle",

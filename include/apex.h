@@ -165,6 +165,13 @@ int apex_register_experts(apex_ctx* ctx, int layer, const void* pinned_base, siz
 /* Always-on shared expert (Sec. V-A: shared experts are outside the routing and the budget):
  * device pointer to [I_shared][3][d] bf16 in the store layout.  Borrowed. */
 int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights);
+/* Gate on the shared expert, for model families that scale their shared FFN per token (the paper's configurations
+ * run theirs with weight 1, Sec. V-A; this variant has no counterpart in the paper):
+ *   y = sum_e g_e FFN_e(h') + sigmoid(w_sg . h') FFN_shared(h').
+ * w_sg [d] fp32 (host or device pointer) is copied into library-owned device memory; NULL removes the gate again
+ * (weight 1).  APEX_EINVAL without a shared expert (I_shared = 0).  Must not be called while a step of the layer is
+ * in flight. */
+int apex_set_shared_gate(apex_ctx* ctx, int layer, const float* w_sg);
 /* Host helper: gate[I][d], up[I][d], down[d][I] -> store layout.  dst holds 3*I*d bf16. */
 int apex_pack_expert(const void* gate, const void* up, const void* down, int d, int I, void* dst);
 

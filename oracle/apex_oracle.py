@@ -222,16 +222,25 @@ def swiglu_ffn(W_gate, W_up, W_down, v) -> np.ndarray:
     return np.asarray(W_down, np.float64) @ (silu(g) * u)
 
 
+def shared_gate_weight(w_sg, h_post) -> float:
+    """Weight of a gated shared expert: sigmoid(w_sg . h').  Not part of the paper's configurations (their shared
+    experts run with weight 1, Sec. V-A); model families with a per-token sigmoid gate on the shared FFN use this."""
+    z = float(np.dot(np.asarray(w_sg, np.float64), np.asarray(h_post, np.float64)))
+    return 1.0 / (1.0 + np.exp(-z))
+
+
 def moe_output(h_post, K_exec: Sequence[int], g: Sequence[float],
                expert_weights: Callable[[int], Tuple[np.ndarray, np.ndarray, np.ndarray]],
-               shared=None) -> np.ndarray:
-    """y = sum_{e in K~, ascending e} g_e FFN_e(h') (+ FFN_shared(h') with weight 1)."""
+               shared=None, shared_gate=None) -> np.ndarray:
+    """y = sum_{e in K~, ascending e} g_e FFN_e(h') + s FFN_shared(h'), s = 1 (Sec. V-A) or, with a gate vector
+    shared_gate, s = sigmoid(shared_gate . h')."""
     y = np.zeros(len(h_post), dtype=np.float64)
     for e, ge in sorted(zip(K_exec, g)):
         Wg, Wu, Wd = expert_weights(int(e))
         y += float(ge) * swiglu_ffn(Wg, Wu, Wd, h_post)
     if shared is not None:
-        y += swiglu_ffn(shared[0], shared[1], shared[2], h_post)
+        s = 1.0 if shared_gate is None else shared_gate_weight(shared_gate, h_post)
+        y += s * swiglu_ffn(shared[0], shared[1], shared[2], h_post)
     return y
 
 
@@ -353,7 +362,7 @@ class SlotCache:
 # --------------------------------------------------------------------------------------
 def layer_step(cache: SlotCache, *, W_p, b_p, W_r, b_r, w, theta, tau: float, k: int,
                h: np.ndarray, h_post: np.ndarray, mode: str,
-               expert_weights: Optional[Callable] = None, shared=None,
+               expert_weights: Optional[Callable] = None, shared=None, shared_gate=None,
                norm_topk: bool = True, compute_ffn: bool = True, ffn_tokens: Optional[Sequence[int]] = None) -> Dict:
     """h, h_post: [B][d].  mode: 'exact' (correctness-preserving) or 'stall_free'.
     Returns every decision of the step, with the margins needed to flag near-ties.
@@ -417,7 +426,7 @@ def layer_step(cache: SlotCache, *, W_p, b_p, W_r, b_r, w, theta, tau: float, k:
     for b, tok in enumerate(out["tokens"]):
         tok["gates"] = gates(tok["alpha"], tok["K_exec"], norm_topk)
         if compute_ffn and expert_weights is not None and (ffn_tokens is None or b in ffn_tokens):
-            tok["y"] = moe_output(h_post[b], tok["K_exec"], tok["gates"], expert_weights, shared)
+            tok["y"] = moe_output(h_post[b], tok["K_exec"], tok["gates"], expert_weights, shared, shared_gate)
     return out
 
 

@@ -58,6 +58,7 @@ SIGNATURES = {
     "apex_set_cdf": (_I, [_P, _I, _P, _P]),
     "apex_register_experts": (_I, [_P, _I, _P, C.c_size_t]),
     "apex_set_shared_expert": (_I, [_P, _I, _P]),
+    "apex_set_shared_gate": (_I, [_P, _I, _P]),
     "apex_pack_expert": (_I, [_P, _P, _P, _I, _I, _P]),
     "apex_predict": (_I, [_P, _I, _P, _I, _P]),
     "apex_select_candidates": (_I, [_P, _I, _I, C.c_float, _P, _P, _P]),
@@ -196,6 +197,14 @@ class Apex:
     def set_shared_expert(self, layer, dev_weights):
         self._keep.append(dev_weights)
         self._chk(self.lib.apex_set_shared_expert(self.h, layer, _ptr(dev_weights)))
+
+    def set_shared_gate(self, layer, w_sg):
+        """Gate vector [d] of the layer's shared expert (numpy / tensor, host or device), or None for weight 1."""
+        if w_sg is None:
+            self._chk(self.lib.apex_set_shared_gate(self.h, layer, None))
+            return
+        w = np.ascontiguousarray(w_sg, np.float32) if isinstance(w_sg, np.ndarray) else w_sg
+        self._chk(self.lib.apex_set_shared_gate(self.h, layer, _ptr(w)))
 
     # -- the layer-step
     def predict(self, layer, h_dev, B, stream=None):

@@ -194,6 +194,8 @@ int apex_create(const apex_config* cfg, apex_ctx** out) {
   ctx->store_base.assign(L, nullptr);
   ctx->store_stride.assign(L, 0);
   ctx->shared_dev.assign(L, nullptr);
+  ctx->shared_gate_dev.assign(L, nullptr);
+  ctx->shared_gate_on.assign(L, 0);
   ctx->slot_gen.assign(L, std::vector<uint32_t>(C, 0u));
   ctx->phys_expert.assign(L, std::vector<int32_t>(C, -1));
   ctx->last_copies.assign(L, {});
@@ -224,6 +226,8 @@ int apex_destroy(apex_ctx* ctx) {
   for (void* p : dev)
     if (p) cudaFree(p);
   decode_teardown(ctx);
+  for (float* g : ctx->shared_gate_dev)
+    if (g) cudaFree(g);
   if (ctx->mbox) cudaFreeHost(ctx->mbox);
   if (ctx->pad_src) cudaFreeHost(ctx->pad_src);
   if (ctx->pad_dst) cudaFree(ctx->pad_dst);
@@ -305,6 +309,29 @@ int apex_set_shared_expert(apex_ctx* ctx, int layer, const void* dev_weights) {
                             ctx->shared_bytes))
       return fail(ctx, APEX_ECUDA, "tensor map for the shared expert could not be encoded");
   }
+  return APEX_OK;
+}
+
+int apex_set_shared_gate(apex_ctx* ctx, int layer, const float* w_sg) {
+  CHECK_CTX(ctx);
+  CHECK_LAYER(ctx, layer);
+  if (ctx->cfg.I_shared <= 0) return fail(ctx, APEX_EINVAL, "the context was created with I_shared = 0");
+  float* dst = ctx->shared_gate_dev[layer];
+  if (!w_sg) {  // back to weight 1 (the vector stays allocated for a later call)
+    const float* none = nullptr;
+    if (ctx->d_shared_gate_ptrs)
+      CU_TRY(ctx, cudaMemcpy(ctx->d_shared_gate_ptrs + layer, &none, sizeof(void*), cudaMemcpyHostToDevice));
+    ctx->shared_gate_on[layer] = 0;
+    return APEX_OK;
+  }
+  if (!dst) {
+    CU_TRY(ctx, cudaMalloc(reinterpret_cast<void**>(&dst), (size_t)ctx->cfg.d * sizeof(float)));
+    ctx->shared_gate_dev[layer] = dst;
+  }
+  CU_TRY(ctx, cudaMemcpy(dst, w_sg, (size_t)ctx->cfg.d * sizeof(float), cudaMemcpyDefault));
+  if (ctx->d_shared_gate_ptrs)
+    CU_TRY(ctx, cudaMemcpy(ctx->d_shared_gate_ptrs + layer, &dst, sizeof(void*), cudaMemcpyHostToDevice));
+  ctx->shared_gate_on[layer] = 1;
   return APEX_OK;
 }
 

@@ -39,6 +39,8 @@ int decode_setup(apex_ctx* ctx) {
   CU_TRY(ctx, cudaMemset(ctx->d_dec_abort, 0, 4 * sizeof(unsigned int)));
   CU_TRY(ctx, dev_alloc(&ctx->d_shared_ptrs, L));
   CU_TRY(ctx, cudaMemset(ctx->d_shared_ptrs, 0, L * sizeof(void*)));
+  CU_TRY(ctx, dev_alloc(&ctx->d_shared_gate_ptrs, L));
+  CU_TRY(ctx, cudaMemset(ctx->d_shared_gate_ptrs, 0, L * sizeof(void*)));
   ctx->dec_tab_last.assign(L, SlotSnapshot{});
   ctx->dec_tab_valid = false;
   ctx->dec_clusters = n;
@@ -57,6 +59,7 @@ void decode_teardown(apex_ctx* ctx) {
   if (ctx->d_dec_snap) cudaFree(ctx->d_dec_snap);
   if (ctx->dec_opt_stage) cudaFreeHost(ctx->dec_opt_stage);
   if (ctx->d_shared_ptrs) cudaFree(ctx->d_shared_ptrs);
+  if (ctx->d_shared_gate_ptrs) cudaFree(ctx->d_shared_gate_ptrs);
 }
 
 bool decode_persistent_usable(const apex_ctx* ctx, int B) {
@@ -145,6 +148,7 @@ int decode_token_persistent(apex_ctx* ctx, const float* h_dev, const float* hpos
   p.w = ctx->d_w; p.theta = ctx->d_theta;
   p.cache = ctx->d_cache;
   p.shared_w = ctx->cfg.I_shared > 0 ? ctx->d_shared_ptrs : nullptr;
+  p.shared_gate = ctx->cfg.I_shared > 0 ? ctx->d_shared_gate_ptrs : nullptr;
   p.slot_ready = ctx->d_slot_ready;
   p.demand = ctx->d_demand;
   p.tab = ctx->d_dec_tab;

@@ -118,6 +118,7 @@ struct FfnParams {
   float* exec_gate;         // [B][k] out or null
   const uint8_t* cache;     // slot 0 of this layer
   const uint8_t* shared_w;  // or null
+  const float* shared_gate; // [d] gate vector of the shared expert, or null: weight 1
   const uint32_t* slot_ready;  // [C]
   // batched plan (B > 1), context-owned
   int32_t* plan_exec_idx;   // [B][k]
@@ -200,6 +201,7 @@ struct DecodeParams {
   const float *w, *theta;               // [L][N], [L][N-k+1]
   const uint8_t* cache;                 // [L][C][slot_stride]
   const uint8_t* const* shared_w;       // [L] pointers (device array), or null
+  const float* const* shared_gate;      // [L] pointers to the shared expert's gate vectors [d] (null entries: weight 1)
   const uint32_t* slot_ready;           // [L][C]
   const uint32_t* demand;               // [L][N]
   const SlotSnapshot* tab;              // [L] slot tables as they stand at launch (device memory)
@@ -327,6 +329,8 @@ struct apex_ctx {
   std::vector<const uint8_t*> store_base;
   std::vector<size_t> store_stride;
   std::vector<const uint8_t*> shared_dev;
+  std::vector<float*> shared_gate_dev;        // [L] library-owned gate vectors of the shared expert, or null
+  std::vector<char> shared_gate_on;           // [L] 1: the layer's shared expert is gated
   std::vector<std::vector<uint32_t>> slot_gen;  // [L][C] install count
   std::vector<std::vector<int32_t>> phys_expert;  // [L][C] whose bytes the slot holds (or is receiving)
   // emulated link (cfg.link_gbs > 0): padding copies over the host link stretch every expert copy
@@ -385,6 +389,7 @@ struct apex_ctx {
   unsigned long long* d_dec_cand = nullptr;   // [L][2]
   unsigned int* d_dec_abort = nullptr;
   const uint8_t** d_shared_ptrs = nullptr;    // [L]
+  const float** d_shared_gate_ptrs = nullptr; // [L]
   unsigned long long dec_epoch = 0;           // persistent launches since the counters were last cleared
   uint32_t dec_seq = 0;
   bool dec_dirty = false;                     // a launch gave up: counters and abort flag must be cleared before the next

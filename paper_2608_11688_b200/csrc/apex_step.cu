@@ -445,6 +445,7 @@ int ffn_launch(apex_ctx* ctx, int layer, int mode, const float* hpost_dev, int B
   p.exec_gate = exec_gate_dev;
   p.cache = ctx->d_cache + (size_t)layer * C * ctx->expert_bytes;
   p.shared_w = ctx->shared_dev[layer];
+  p.shared_gate = ctx->shared_gate_on[layer] ? ctx->shared_gate_dev[layer] : nullptr;
   p.slot_ready = ctx->d_slot_ready + (size_t)layer * C;
   p.plan_exec_idx = ctx->d_plan_exec_idx;
   p.plan_exec_gate = ctx->d_plan_exec_gate;

@@ -323,6 +323,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
   };
   auto prefetch_l2 = [&](const void* ptr) { asm volatile("prefetch.global.L2 [%0];" ::"l"(ptr)); };
 
+  float sgate = 1.f;      // value of the shared expert's gate for layer sgate_layer (gated variant only)
+  int sgate_layer = -1;
   for (int l = 0; l < L; ++l) {
     __syncwarp();
     const bool running = ok && !cta_stopped();  // per warp: skip the work, keep the barriers
@@ -854,7 +856,17 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
             if (!redo) {
               const int e = s_exp[s];
               float gate = __shfl_sync(0xffffffffu, e < 32 ? g0 : g1, e & 31);
-              if (e >= N) gate = 1.f;
+              if (e >= N) {  // the shared expert: weight 1, or its gate's value (once per warp and layer)
+                gate = 1.f;
+                const float* wsg = p.shared_gate ? p.shared_gate[l] : nullptr;
+                if (wsg) {
+                  if (sgate_layer != l) {
+                    sgate = shared_gate_weight(wsg, hpl, d, lane);
+                    sgate_layer = l;
+                  }
+                  gate = sgate;
+                }
+              }
               const uint8_t* gs = smem + (size_t)s * entry_bytes;
               const uint8_t* us = gs + row_bytes;
               const uint8_t* ds = us + row_bytes;

@@ -537,6 +537,7 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
     ++tail;
   }
   bool polled = false;
+  float sgate = -1.f;  // B == 1: value of the shared expert's gate, once computed
   for (int head = 0; head < tail; ++head) {
     if (__any_sync(0xffffffffu, *(volatile int*)&s_abort != 0)) break;
     const int s = warp + kConsumerWarps * (head % NSW);
@@ -552,7 +553,10 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
     float gate;
     if (B == 1) {
       gate = __shfl_sync(0xffffffffu, e < 32 ? g0 : g1, e & 31);
-      if (e >= N) gate = 1.f;
+      if (e >= N) {  // the shared expert: weight 1, or its gate's value (computed when the warp meets its first shared row)
+        if (p.shared_gate && sgate < 0.f) sgate = shared_gate_weight(p.shared_gate, p.hpost, d, lane);
+        gate = p.shared_gate ? sgate : 1.f;
+      }
     } else {
       gate = s_gate[s];
     }

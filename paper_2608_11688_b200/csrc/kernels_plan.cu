@@ -32,6 +32,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   const unsigned crank = cluster.block_rank();
   __shared__ unsigned long long s_exec[APEX_MAX_BATCH];
   __shared__ float s_pgate[APEX_MAX_BATCH][APEX_MAX_TOPK];  // gate of the j-th executed expert of each token
+  __shared__ float s_sgate[APEX_MAX_BATCH];                 // weight of the shared expert for each token (gated variant)
   __shared__ int s_count[APEX_MAX_EXPERTS + 1];
   __shared__ int s_off[APEX_MAX_EXPERTS + 2];
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarp = blockDim.x >> 5;
@@ -40,6 +41,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
   // the leader's copies of the per-token results
   unsigned long long* l_exec = cluster.map_shared_rank(&s_exec[0], 0);
   float* l_pgate = cluster.map_shared_rank(&s_pgate[0][0], 0);
+  float* l_sgate = cluster.map_shared_rank(&s_sgate[0], 0);
   SPAN_BEGIN();
   PTL(0);
   TokenLoads tls[TOK_PER_WARP];
@@ -71,6 +73,10 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
       my_hits += __popcll(tp.kr_mask & p.snap.resident_mask);
     }
     if (lane == 0) l_exec[b] = tp.exec_mask;
+    if (p.run_shared && p.shared_gate) {
+      const float sg = shared_gate_weight(p.shared_gate, p.hpost + (size_t)b * p.d, p.d, lane);
+      if (lane == 0) l_sgate[b] = sg;
+    }
     {
       const int e0 = lane, e1 = lane + 32;
       if ((tp.exec_mask >> e0) & 1) {
@@ -168,7 +174,7 @@ __global__ void __launch_bounds__(1024) ffn_plan_kernel(const FfnParams p) {
     for (int b = threadIdx.x; b < B; b += blockDim.x) {
       p.pair_tok[base + b] = b;
       p.pair_expert[base + b] = N;
-      p.pair_gate[base + b] = 1.f;
+      p.pair_gate[base + b] = p.shared_gate ? s_sgate[b] : 1.f;
     }
   }
   PTL(4);

@@ -20,6 +20,21 @@ __device__ __forceinline__ float warp_sum(float v) {
   for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
   return v;
 }
+// Weight of a gated shared expert for one token: sigmoid(w_sg . h'), by a whole warp (every lane gets the value).
+// d is a multiple of 128; lane-strided float4 loads, fused multiply-adds in ascending index order, xor tree.
+__device__ __forceinline__ float shared_gate_weight(const float* __restrict__ w_sg, const float* __restrict__ hpost, int d, int lane) {
+  float z = 0.f;
+  for (int i = lane * 4; i < d; i += 128) {
+    const float4 a = __ldg(reinterpret_cast<const float4*>(w_sg + i));
+    const float4 b = __ldg(reinterpret_cast<const float4*>(hpost + i));
+    z = fmaf(a.x, b.x, z);
+    z = fmaf(a.y, b.y, z);
+    z = fmaf(a.z, b.z, z);
+    z = fmaf(a.w, b.w, z);
+  }
+  z = warp_sum(z);
+  return 1.f / (1.f + expf(-z));
+}
 
 // ---------------------------------------------------------------- execution set of one token (S6)
 // One warp.  Lanes own experts lane and lane+32.  Exact mode: K~ = K_r.  Stall-free mode

@@ -49,12 +49,14 @@ class Problem:
     """Parameters and expert stores of one config on the GPU machine, shared by library and oracle."""
 
     def __init__(self, cfg: synth.Config, layers: Optional[int] = None, device="cuda", cdf="handset", fp8=False, fp4=False,
-                 store_layers: Optional[int] = None, fp8_code_mask: Optional[int] = None):
+                 store_layers: Optional[int] = None, fp8_code_mask: Optional[int] = None, gated_shared: bool = False):
         """cdf: "handset", "fitted", or ("static", delta): the static over-fetch model of Sec. V-A (w = 0 and a step
         in theta, so delta_hat = delta for every token).  store_layers: physical expert stores (layer l uses store
         l mod store_layers; for shapes whose full store does not fit the host's memory).  fp8_code_mask: and-ed onto
         every e4m3 code byte of the stores (0x8F leaves sign, the lowest exponent bit and the mantissa: half the codes
-        are then subnormal and the rest sit in the lowest binade, so a path that mishandles subnormal codes shows)."""
+        are then subnormal and the rest sit in the lowest binade, so a path that mishandles subnormal codes shows).
+        gated_shared: every layer's shared expert gets a seeded gate vector w_sg ~ N(0, 1/d) (weight sigmoid(w_sg . h'),
+        spread over about 0.15 .. 0.85 for the generator's h')."""
         self.cfg = cfg
         self.fp8 = fp8
         self.fp4 = fp4
@@ -69,6 +71,10 @@ class Problem:
                         for l in range(self.L)]
         self.stores = []
         self.shared = []
+        self.shared_gates = [None] * self.L
+        if gated_shared and cfg.I_shared > 0:
+            self.shared_gates = [(np.random.default_rng(77_000 + 131 * cfg.cfg_id + l).standard_normal(cfg.d) / np.sqrt(cfg.d)).astype(np.float32)
+                                 for l in range(self.L)]
         n_phys = min(self.L, store_layers or self.L)
         for l in range(self.L):
             if l >= n_phys:
@@ -114,6 +120,8 @@ class Problem:
             a.register_experts(l, self.stores[l])
             if self.shared[l] is not None:
                 a.set_shared_expert(l, self.shared[l])
+            if self.shared_gates[l] is not None:
+                a.set_shared_gate(l, self.shared_gates[l])
         return a
 
     def oracle_experts(self, layer):
@@ -198,7 +206,7 @@ def run_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: float, T:
             if use_prefetch:
                 out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=tau, k=k,
                                     h=hs[l][0][t], h_post=hs[l][1][t], mode=mode,
-                                    expert_weights=prob.oracle_experts(l), shared=prob.oracle_shared(l),
+                                    expert_weights=prob.oracle_experts(l), shared=prob.oracle_shared(l), shared_gate=prob.shared_gates[l],
                                     norm_topk=norm_topk, compute_ffn=do_ffn,
                                     ffn_tokens=None if ffn_token_stride == 1 else set(range(0, B, ffn_token_stride)))
             else:   # no prefetch stage: budget 0 candidates are never issued; emulate by an empty prefetch
@@ -306,7 +314,8 @@ def _oracle_step_without_prefetch(cache, W_r, b_r, k, h_post, mode, prob, layer,
     for b, tok in enumerate(out["tokens"]):
         tok["gates"] = ao.gates(tok["alpha"], tok["K_exec"], norm_topk)
         if do_ffn:
-            tok["y"] = ao.moe_output(h_post[b], tok["K_exec"], tok["gates"], prob.oracle_experts(layer), prob.oracle_shared(layer))
+            tok["y"] = ao.moe_output(h_post[b], tok["K_exec"], tok["gates"], prob.oracle_experts(layer), prob.oracle_shared(layer),
+                                     prob.shared_gates[layer])
     return out
 
 
@@ -350,7 +359,7 @@ def run_decode_lockstep(prob: Problem, apex: binding.Apex, *, mode: str, tau: fl
             if use_prefetch:
                 out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=tau, k=k,
                                     h=h_all[t, l], h_post=hp_all[t, l], mode=mode, expert_weights=prob.oracle_experts(l),
-                                    shared=prob.oracle_shared(l), norm_topk=norm_topk,
+                                    shared=prob.oracle_shared(l), shared_gate=prob.shared_gates[l], norm_topk=norm_topk,
                                     ffn_tokens=None if ffn_token_stride == 1 else set(range(0, B, ffn_token_stride)))
             else:
                 out = _oracle_step_without_prefetch(cache, W_r, b_r, k, hp_all[t, l], mode, prob, l, norm_topk, True)

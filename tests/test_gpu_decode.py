@@ -53,6 +53,14 @@ def test_persistent_token_kernel_tiny_shapes(d, N, k, I, C, L, Ish, mode):
         assert rep.n_demand_copies == 0
 
 
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_persistent_token_kernel_with_a_gated_shared_expert(mode):
+    cfg = synth.tiny_config(d=1024, N=24, k=6, I=96, C=12, L=4, T=5, I_shared=64, sigma_p=1.0, cfg_id=414)
+    prob = _harness().Problem(cfg, gated_shared=True)
+    rep, stats, launches = _decode(cfg, mode=mode, tau=0.8, T=5, prob=prob)
+    assert rep.near_ties == 0 and rep.ffn_checked == 5 * 4 and launches == 5     # one launch per token
+
+
 @pytest.mark.parametrize("tau", [-1.0, 0.0, 0.97, 1.0])
 def test_persistent_token_kernel_policies_and_budget_extremes(tau):
     cfg = synth.tiny_config(d=512, N=16, k=4, I=32, C=8, L=3, T=8, sigma_p=0.8, cfg_id=410)

@@ -158,6 +158,32 @@ def test_batched_exact_mode_runs_in_waves_when_cache_is_smaller_than_need():
     assert stats["extra_waves"] >= 4 * 2          # at least two extra waves per step: need > 2 C
 
 
+# ------------------------------------------------------------------ gated shared expert (no counterpart in the paper)
+@pytest.mark.parametrize("B,fmt", [(1, "bf16"), (1, "fp8"), (1, "fp4"), (5, "bf16"), (24, "bf16"), (24, "fp8")])
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+def test_gated_shared_expert(B, fmt, mode):
+    # y = routed part + sigmoid(w_sg . h') * shared FFN: B = 1 the streaming kernel, B = 5 the streaming kernel per pair
+    # (gate value from the plan kernel), B = 24 the grouped GEMMs (gate value in the pair list)
+    cfg = synth.tiny_config(d=512, N=12, k=3, I=128, C=8, L=2, T=3, I_shared=256, sigma_p=1.0, cfg_id=290)
+    hz = _harness()
+    prob = hz.Problem(cfg, fp8=(fmt == "fp8"), fp4=(fmt == "fp4"), gated_shared=True)
+    rep, stats = _run(cfg, mode=mode, tau=0.8, T=3, B=B, prob=prob)
+    assert rep.ffn_checked == 3 * 2 * B and rep.near_ties == 0
+    # the gate matters: without it the same run must fail the output check
+    prob.shared_gates = [None] * prob.L
+    apex = prob.make_ctx(max_batch=B)
+    try:
+        for l in range(prob.L):
+            apex.set_shared_gate(l, np.zeros(cfg.d, np.float32))      # weight 0.5 everywhere: differs from weight 1
+        with pytest.raises(AssertionError, match="FFN output"):
+            hz.run_lockstep(prob, apex, mode=mode, tau=0.8, T=1, B=B)
+        for l in range(prob.L):
+            apex.set_shared_gate(l, None)                             # back to weight 1: matches the ungated oracle
+        hz.run_lockstep(prob, apex, mode=mode, tau=0.8, T=2, B=B)
+    finally:
+        apex.destroy()
+
+
 # ------------------------------------------------------------------ e4m3 expert store (Sec. V-G)
 def _run_fp8(cfg, *, mode, tau, T, B=1, layers=None, check_ffn_every=1, ffn_token_stride=1):
     hz = _harness()

@@ -531,6 +531,32 @@ def test_unnormalised_gates_equal_dense_moe_that_keeps_the_softmax_values():
         assert not np.allclose(tok["y"], _dense_topk_moe(W_r, b_r, hp[t, 0], cfg.k, experts, shared), rtol=1e-6, atol=1e-9)
 
 
+def test_gated_shared_expert_against_a_dense_layer_and_its_limits():
+    # y(gated) - y(no shared) = sigmoid(w_sg . h') * (y(ungated) - y(no shared)), the sigmoid from torch; a zero gate
+    # vector halves the shared FFN; a gate vector far along h' switches it fully on, far against it fully off
+    cfg = synth.tiny_config(d=64, N=8, k=3, I=16, C=8, T=4, I_shared=8)
+    W_r, b_r, W_p, b_p, experts, shared, w, theta = _tiny_problem(cfg)
+    h, hp = synth.hidden_states(cfg, 0, cfg.T)
+    rng = np.random.default_rng(5)
+    w_sg = rng.standard_normal(cfg.d) / np.sqrt(cfg.d)
+    for t in range(cfg.T):
+        def run(sh, sg):
+            cache = ao.SlotCache(cfg.N, cfg.C)
+            out = ao.layer_step(cache, W_p=W_p, b_p=b_p, W_r=W_r, b_r=b_r, w=w, theta=theta, tau=0.9, k=cfg.k, h=h[t],
+                                h_post=hp[t], mode="exact", expert_weights=experts, shared=sh, shared_gate=sg)
+            return out["tokens"][0]["y"]
+        v = hp[t, 0].astype(np.float64)
+        y_none, y_plain, y_gated = run(None, None), run(shared, None), run(shared, w_sg)
+        s = float(torch.sigmoid(torch.from_numpy(w_sg) @ torch.from_numpy(v)))
+        assert 0.05 < s < 0.95
+        np.testing.assert_allclose(y_gated - y_none, s * (y_plain - y_none), rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(y_plain, _dense_topk_moe(W_r, b_r, v, cfg.k, experts, shared), rtol=1e-10, atol=1e-13)
+        np.testing.assert_allclose(run(shared, np.zeros(cfg.d)) - y_none, 0.5 * (y_plain - y_none), rtol=1e-12, atol=1e-14)
+        np.testing.assert_allclose(run(shared, 100.0 * v / (v @ v)), y_plain, rtol=1e-12, atol=1e-14)    # sigmoid(100) = 1
+        np.testing.assert_allclose(run(shared, -100.0 * v / (v @ v)), y_none, rtol=0, atol=1e-12 * np.abs(y_plain).max())
+    assert ao.shared_gate_weight(np.zeros(4), np.ones(4)) == 0.5
+
+
 def test_stall_free_equals_exact_when_covered_and_differs_only_by_substitution():
     cfg = synth.tiny_config(d=64, N=10, k=3, I=16, C=5, T=40, sigma_p=1.5)
     W_r, b_r, W_p, b_p, experts, shared, w, theta = _tiny_problem(cfg)

@@ -123,6 +123,8 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
   __shared__ uint64_t s_full[kDecMaxStages];
   __shared__ uint64_t s_xbar[2];   // logits of the prefetch router / of the gate have arrived from the whole cluster
   __shared__ uint64_t s_pbar;      // warp 0 has derived the candidate set of this layer
+  __shared__ uint64_t s_rbar;      // every warp has added its share of the gate's rank counts
+  __shared__ unsigned s_rank[APEX_MAX_EXPERTS / 4];  // rank of each expert's gate logit, four 8-bit counts to a word (zero between layers)
   __shared__ float s_zp[APEX_MAX_EXPERTS], s_zr[APEX_MAX_EXPERTS];
   __shared__ float s_q[APEX_MAX_EXPERTS];              // warp 0: prefetch probabilities by expert
   __shared__ int s_pi[kDecWarps][APEX_MAX_EXPERTS];    // per-warp scratch: expert by rank
@@ -160,7 +162,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     mbar_init(&s_xbar[0], 1);
     mbar_init(&s_xbar[1], 1);
     mbar_init(&s_pbar, 1);
+    mbar_init(&s_rbar, kDecWarps);
   }
+  if (tid < APEX_MAX_EXPERTS / 4) s_rank[tid] = 0u;
   if (tid < NS) mbar_init(&s_full[tid], 1);
   asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   __syncthreads();
@@ -192,6 +196,24 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
   // expert rows: which warps of this CTA take rows (the poster's warp 0 does not while the prefetch stage runs)
   const int row_warps = (poster && p.prefetching) ? kDecWarps - 1 : kDecWarps;
   const int row_warp = (poster && p.prefetching) ? warp - 1 : warp;  // index among them, -1: none
+
+  // Row range of this CTA and the rows of this warp for the usual row space (k executed experts and the shared expert):
+  // the same in every layer, so the divisions are done once; lane j < NSW also keeps where the warp's row j lies
+  // (position in the row space, intermediate index) for the first ring fill.
+  const int std_total = k * I + ((p.shared_w && p.I_shared > 0) ? p.I_shared : 0);
+  const unsigned std_pre_all = (unsigned)row_weight_prefix(G, p.prefetching != 0);
+  const int std_lo = (int)((unsigned long long)std_total * (unsigned)row_weight_prefix(cta, p.prefetching != 0) / std_pre_all);
+  const int std_S = (int)((unsigned long long)std_total * (unsigned)row_weight_prefix(cta + 1, p.prefetching != 0) / std_pre_all) - std_lo;
+  int ff_pidx = k, ff_i = 0;
+  {
+    const int r = std_lo + row_warp + row_warps * lane;
+    if (r < k * I) {
+      ff_pidx = r / I;
+      ff_i = r - ff_pidx * I;
+    } else {
+      ff_i = r - k * I;
+    }
+  }
 
   int n_iss = 0, n_con = 0;  // copies this warp has started / consumed since the kernel began (uniform over the warp)
   int il = 0, iq = 0;        // the next segment-1 job to start: layer il, job iq
@@ -646,8 +668,32 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
         ok = false;
       } else {
         DTL(5);
-        rank_lane_logits(s_zr, N, lane, &Rg);
+        // Ranks by counting, the count shared by the CTA's warps: warp w compares every logit with the logits of experts
+        // w, w + 8, ... only and adds its counts up in shared memory (each warp ranking all N logits by itself was
+        // 0.8 us of every warp's path to the first row).
         const int e0 = lane, e1 = lane + 32;
+        {
+          const float NEG = -3.402823466e38f;
+          Rg.z0 = e0 < N ? s_zr[e0] : NEG;
+          Rg.z1 = e1 < N ? s_zr[e1] : NEG;
+          int c0 = 0, c1 = 0;
+          for (int f = warp; f < N; f += kDecWarps) {
+            const float zf = s_zr[f];
+            c0 += (zf > Rg.z0 || (zf == Rg.z0 && f < e0)) ? 1 : 0;
+            c1 += (zf > Rg.z1 || (zf == Rg.z1 && f < e1)) ? 1 : 0;
+          }
+          unsigned* rk = s_rank;  // counts stay below N <= 64: no carry between the bytes of a word
+          if (e0 < N && c0) atomicAdd(rk + (e0 >> 2), (unsigned)c0 << (8 * (e0 & 3)));
+          if (e1 < N && c1) atomicAdd(rk + (e1 >> 2), (unsigned)c1 << (8 * (e1 & 3)));
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&s_rbar);
+          if (!__all_sync(0xffffffffu, wait_bar(&s_rbar, lpar))) {
+            if (lane == 0 && !stop_requested()) gave_up();
+            ok = false;
+          }
+          Rg.r0 = e0 < N ? (int)((rk[e0 >> 2] >> (8 * (e0 & 3))) & 0xffu) : N;
+          Rg.r1 = e1 < N ? (int)((rk[e1 >> 2] >> (8 * (e1 & 3))) & 0xffu) : N;
+        }
         kr_mask = ((unsigned long long)__ballot_sync(0xffffffffu, e1 < N && Rg.r1 < k) << 32) | __ballot_sync(0xffffffffu, e0 < N && Rg.r0 < k);
         if (poster && warp == 0 && lane == 0) {  // K_r does not depend on the table: the host gets it at once
           asm volatile("st.global.v4.u32 [%0], {%1, %2, %3, %4};" ::"l"(p.mbox[l].kr_rec), "r"((uint32_t)kr_mask),
@@ -685,10 +731,12 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
       // Rows are dealt out by weight: the first cluster also runs the prefetch router and its last CTA (the poster)
       // the candidate selection on warp 0, so they take fewer rows and the poster's warp 0 none -- otherwise
       // everybody would wait for them at the end of the layer.
-      const long long pre_lo = row_weight_prefix(cta, p.prefetching != 0), pre_hi = row_weight_prefix(cta + 1, p.prefetching != 0);
-      const long long pre_all = row_weight_prefix(G, p.prefetching != 0);
-      const int range_lo = (int)((long long)total_rows * pre_lo / pre_all);
-      const int S = (int)((long long)total_rows * pre_hi / pre_all) - range_lo;
+      int range_lo = std_lo, S = std_S;
+      const bool std_rows = total_rows == std_total;
+      if (!std_rows) {  // fewer experts executed than k (or no plan): the range is worked out for this row count
+        range_lo = (int)((unsigned long long)total_rows * (unsigned)row_weight_prefix(cta, p.prefetching != 0) / std_pre_all);
+        S = (int)((unsigned long long)total_rows * (unsigned)row_weight_prefix(cta + 1, p.prefetching != 0) / std_pre_all) - range_lo;
+      }
       const int n_mine = (row_warp >= 0 && S > row_warp) ? (S - row_warp + row_warps - 1) / row_warps : 0;
       if (planned) {
         if (lane < APEX_MAX_TOPK) s_pos[warp][lane] = lane < n_routed ? nth_set_bit64(run, lane) : -1;
@@ -712,14 +760,16 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
         if (Jr > 0 && (run & ~ready_mask) == 0ull && n_iss == n_con) {
           const int fill = Jr < NSW ? Jr : NSW;
           if (lane < fill) {
-            const int r = range_lo + row_warp + row_warps * lane;
-            int pidx, i;
-            if (r < n_routed * I) {
-              pidx = r / I;
-              i = r - pidx * I;
-            } else {
-              pidx = n_routed;
-              i = r - n_routed * I;
+            int pidx = ff_pidx, i = ff_i;
+            if (!std_rows) {
+              const int r = range_lo + row_warp + row_warps * lane;
+              if (r < n_routed * I) {
+                pidx = r / I;
+                i = r - pidx * I;
+              } else {
+                pidx = n_routed;
+                i = r - n_routed * I;
+              }
             }
             const int e = pidx < n_routed ? s_pos[warp][pidx] : N;
             const uint8_t* base = e < N ? cache_l + (size_t)s_slot[warp][e] * p.slot_stride : shared_w;
@@ -970,6 +1020,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
       }
     }
     __syncthreads();
+    if (tid < APEX_MAX_EXPERTS / 4) s_rank[tid] = 0u;  // every warp has read this layer's ranks; the next layer adds to zeros
     DTL(11);
     // the peers of this cluster have read this CTA's partial sums of the previous layer
     if (l > 0) asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");

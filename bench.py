@@ -418,11 +418,21 @@ def other_config_rooflines(dev, peak, peak_kind):
                 bytes_ffn = distinct * cfg.expert_bytes + cfg.shared_bytes + 2 * B * cfg.d * 4
                 kernel = "ffn_plan_kernel + ffn_tc_gather_kernel + ffn_tc_gemm_kernel<1>, <2>"
             ach = bytes_ffn / mean_s / 1e9
-            out[f"config{cfg_id}" + (f"_B{B}" if len(batches) > 1 else "")] = {
+            rec = {
                 "bound": "hbm", "kernel": kernel, "achieved": ach, "peak": peak, "unit": "GB/s", "frac": ach / peak,
                 "peak_kind": f"of {peak_kind}", "traffic": NCU_TRAFFIC_BYTES.get(cfg_id) if B == 1 else None,
                 "algorithmic_bytes_per_launch": bytes_ffn, "us_per_launch_mean": mean_s * 1e6, "launches_timed": n_l,
                 "layers": layers, "B": B}
+            if B == 1:
+                # the product path at B = 1: the token kernel over these layers (no stand-in: the method's bytes only)
+                y1 = torch.empty((cfg.L, 1, cfg.d), dtype=torch.float32, device=dev)
+                sec_tok, per_token = time_token_kernel(cfg, prob, h, hp, y1, 16, standin=False)
+                if per_token == 1.0:
+                    bytes_step, _ = algorithmic_bytes(cfg, 1)
+                    bt = cfg.L * (bytes_step + cfg.d * 4)
+                    rec["decode_token_kernel"] = {"us_per_layer_step": sec_tok * 1e6 / cfg.L, "achieved": bt / sec_tok / 1e9,
+                                                  "frac": bt / sec_tok / 1e9 / peak, "algorithmic_bytes_per_launch": bt}
+            out[f"config{cfg_id}" + (f"_B{B}" if len(batches) > 1 else "")] = rec
             del h, hp
         del prob
         torch.cuda.empty_cache()

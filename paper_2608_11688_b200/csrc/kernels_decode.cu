@@ -300,11 +300,16 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     return s;
   };
   // A router row in registers: lane l holds float4 columns l, l + 32, ... (the order of router_kernel's reduction).
-  // Rows wider than NVR float4 per lane are not held: their dot product reads the row when it is taken (the layers of
-  // such wide models are long, the extra latency does not show).
-  constexpr int NVR = NV <= 16 ? NV : 1;
-  constexpr bool ROW_REGS = NV <= 16;
-  auto load_row = [&](const float* __restrict__ W_row, float4 (&wr)[NVR]) {
+  // Only up to d = 1024 (8 float4 per lane and row).  Wider rows are read when their dot product is taken (they were
+  // prefetched into L2 at the start of the layer): two rows of d = 2048 in registers spilled and cost 17 % of the
+  // layer-step (configs 2 and 4: 36.8 -> 31.5 and 42.3 -> 35.8 us without them), and even the 96 registers of two
+  // d = 1536 rows, which fit, cost the row loop more than the loads' latency costs the logits (config 1 without the
+  // stand-in: 19.3 -> 17.8 us per layer-step).
+  constexpr int NVRP = NV <= 8 ? NV : 1;   // prefetch-router row
+  constexpr int NVRR = NV <= 8 ? NV : 1;   // gate row
+  auto load_row = [&](const float* __restrict__ W_row, auto& wr) {
+    constexpr int NVR = (int)(sizeof(wr) / sizeof(float4));
+    constexpr bool ROW_REGS = NVR > 1 || NV == 1;
     if (!ROW_REGS) return;
     const float4* rp = reinterpret_cast<const float4*>(W_row);
 #pragma unroll
@@ -312,8 +317,10 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
       asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(wr[i].x), "=f"(wr[i].y), "=f"(wr[i].z), "=f"(wr[i].w) : "l"(rp + i * 32 + lane));
   };
   // dot product of the row with x (reduction order of router_kernel), plus bias; sent to CTAs [rank_lo, rank_hi) of the cluster
-  auto row_logit = [&](const float* __restrict__ W_row, const float4 (&wr)[NVR], const float* __restrict__ x, float bias, float* zs,
+  auto row_logit = [&](const float* __restrict__ W_row, const auto& wr, const float* __restrict__ x, float bias, float* zs,
                        uint64_t* xbar, int rank_lo, int rank_hi) {
+    constexpr int NVR = (int)(sizeof(wr) / sizeof(float4));
+    constexpr bool ROW_REGS = NVR > 1 || NV == 1;
     const float4* __restrict__ xv = reinterpret_cast<const float4*>(x);
     const float4* __restrict__ rp = reinterpret_cast<const float4*>(W_row);
     float acc = 0.f;
@@ -373,7 +380,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     uint32_t f1 = sl1 >= 0 ? ld_relaxed_sys(slot_ready + sl1) : 0u;
     // parameters of this layer this warp will need: fetched now, used after the waits
     float bias_p = 0.f, bias_r = 0.f;
-    float4 wp_row[NVR], wr_row[NVR];
+    float4 wp_row[NVRP], wr_row[NVRR];
     const float* Wp_row = p.W_p + ((size_t)l * N + (has_row ? my_e : 0)) * d;
     const float* Wr_row = p.W_r + ((size_t)l * N + (has_row ? my_e : 0)) * d;
     if (has_wp) load_row(Wp_row, wp_row);
@@ -387,6 +394,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
         for (int i = 0; i < NV; ++i) {
           if (has_wp) prefetch_l2(reinterpret_cast<const float4*>(hl) + i * 32 + lane);
           prefetch_l2(reinterpret_cast<const float4*>(hpl) + i * 32 + lane);
+          // ... and so are the router rows that are not held in registers
+          if (NVRP == 1 && NV > 1 && has_wp) prefetch_l2(reinterpret_cast<const float4*>(Wp_row) + i * 32 + lane);
+          if (NVRR == 1 && NV > 1) prefetch_l2(reinterpret_cast<const float4*>(Wr_row) + i * 32 + lane);
         }
       }
     }

@@ -56,6 +56,7 @@ constexpr int kCvWarp0 = kProducerWarps + 1 + 4;  // first of the converter warp
 constexpr int kCvThreads = 256;   // eight warps: two per scheduler, so one warp's shared-memory latency hides behind the other's arithmetic
 // producers, MMA + TMEM owner, four epilogue warps; for a quantised store the converter warps as well
 __host__ __device__ constexpr int tc_threads(int qf) { return (kProducerWarps + 1 + 4) * 32 + (qf ? kCvThreads : 0); }
+__host__ __device__ constexpr int tc_tiles_per_stage(int phase, int qf) { return (phase == 2 && qf == 0) ? 2 : 1; }
 // bytes of raw codes (and e2m1 scale bytes: 16 per row) a pipeline stage stages for the converters
 __host__ __device__ constexpr int tc_raw_bytes(int phase, int qf) {
   return qf == 1 ? (phase == 1 ? 2 * 128 * 64 : 64 * 128) : qf == 2 ? (phase == 1 ? 2 * 128 * 32 + 2 * 128 * 16 : 64 * 64 + 64 * 16) : 0;
@@ -257,7 +258,12 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
   const int NMAX = PHASE == 1 ? p.nmax1 : p.nmax2;
   const int B_PLANE = NMAX * 128;
   constexpr int RAW_BYTES = tc_raw_bytes(PHASE, QF);
-  const int STAGE_BYTES = A_BYTES + PLANES * B_PLANE + RAW_BYTES;
+  // K tiles per stage.  The down projection of a bf16 store puts two in a stage (each laid out as a stage of one): its
+  // tiles are small (16 KB of weights) and cheap in MMAs (four), so the fixed cost of a stage -- a barrier round trip,
+  // a commit, the producer's turn -- weighed as much as the tile itself (672 ns per tile, 3.5 TB/s while it streamed).
+  constexpr int KPS = tc_tiles_per_stage(PHASE, QF);
+  const int HALF_BYTES = A_BYTES + PLANES * B_PLANE;
+  const int STAGE_BYTES = KPS * HALF_BYTES + RAW_BYTES;
   const int NSTAGE = PHASE == 1 ? p.nstage1 : p.nstage2;
   __shared__ uint64_t full[MAX_STAGES], empty[MAX_STAGES], rawfull[MAX_STAGES], tmem_full[2], tmem_empty[2];
   __shared__ uint32_t tmem_base_s;
@@ -420,25 +426,29 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       }
       const CUtensorMap* wmap = shared ? &tm_ws : &tm_w;
       constexpr int planes = PLANES;
-      for (int kt = kt_begin; kt < kt_end && ok; ++kt, ++it_load) {
-        if ((int)(it_load % kProducerWarps) != warp) continue;  // the other producer warp's tile
+      for (int kt = kt_begin; kt < kt_end && ok; kt += KPS, ++it_load) {
+        if ((int)(it_load % kProducerWarps) != warp) continue;  // the other producer warp's stage
         const int s = it_load % NSTAGE;
         if (lane == 0) {
           if (it_load >= (uint32_t)NSTAGE && !mbar_wait(&empty[s], ((it_load / NSTAGE) - 1) & 1, &s_abort, p.f.wait_limit_ns)) ok = false;
           CVTL(PHASE, it_load, 4);
           if (ok) {
-            mbar_expect_tx(&full[s], (QF ? 0 : A_BYTES) + planes * n_loads * kXRowsPerLoad * 128);
+            mbar_expect_tx(&full[s], KPS * ((QF ? 0 : A_BYTES) + planes * n_loads * kXRowsPerLoad * 128));
             if (QF) mbar_expect_tx(&rawfull[s], RAW_BYTES);
           }
         }
         ok = __all_sync(0xffffffffu, ok);
         if (!ok) break;
-        uint8_t* st = smem + (size_t)s * STAGE_BYTES;
+        uint8_t* st0 = smem + (size_t)s * STAGE_BYTES;
         // the weight loads first; then op n_wops + r*planes + pl: 8-row box r of B plane pl
         constexpr int n_wops = QF == 0 ? 2 : QF == 1 ? (PHASE == 1 ? 2 : 1) : (PHASE == 1 ? 4 : 2);
         const int n_ops = n_wops + planes * n_loads;
-        uint8_t* raw = st + A_BYTES + planes * B_PLANE;
-        for (int op = lane; op < n_ops; op += 32) {
+        uint8_t* raw = st0 + A_BYTES + planes * B_PLANE;
+        const int kt0 = kt;
+        for (int opx = lane; opx < KPS * n_ops; opx += 32) {
+          const int half = KPS > 1 ? opx / n_ops : 0, op = KPS > 1 ? opx - half * n_ops : opx;
+          const int kt = kt0 + half;                      // (shadows the stage's first tile)
+          uint8_t* st = st0 + (size_t)half * HALF_BYTES;
           if (op < n_wops) {
             if (QF == 0) {
               if (PHASE == 1) tma_load_4d(st + op * 128 * 128, wmap, kt * kKTile, op, blk * 128, slot, &full[s]);   // gate | up rows
@@ -489,7 +499,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
         const uint32_t idesc = umma_idesc(128, PHASE == 2 ? 2 * n_pad : n_pad, PHASE == 2 ? 1 : 0);
         const uint64_t desc_a0 = PHASE == 1 ? umma_desc(smem_u32(smem), 16, 1024) : umma_desc(smem_u32(smem), 64 * 128, 1024);
         const uint64_t desc_b0 = umma_desc(smem_u32(smem) + A_BYTES, 16, 1024);
-        for (int kt = kt_begin; kt < kt_end && ok; ++kt, ++it_mma) {
+        for (int kt = kt_begin; kt < kt_end && ok; kt += KPS, ++it_mma) {
           const int s = it_mma % NSTAGE;
           if (!mbar_wait(&full[s], (it_mma / NSTAGE) & 1, &s_abort, p.f.wait_limit_ns)) {
             ok = false;
@@ -501,10 +511,13 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
           // descriptors differ from the stage-0, k-step-0 ones only in the start-address field (address >> 4, the low
           // 14 bits; the sums below stay inside the CTA's shared memory, so nothing carries into the next field)
           const uint64_t soff = (uint64_t)((uint32_t)s * (uint32_t)STAGE_BYTES >> 4);
-          const uint64_t da = desc_a0 + soff, db = desc_b0 + soff;
+#pragma unroll
+          for (int half = 0; half < KPS; ++half) {
+          const uint64_t hoff = soff + (uint64_t)((uint32_t)half * (uint32_t)HALF_BYTES >> 4);
+          const uint64_t da = desc_a0 + hoff, db = desc_b0 + hoff;
 #pragma unroll
           for (int ks = 0; ks < kKTile / 16; ++ks) {
-            const uint32_t acc = (kt > kt_begin || ks > 0) ? 1u : 0u;
+            const uint32_t acc = (kt > kt_begin || half > 0 || ks > 0) ? 1u : 0u;
             const uint64_t bdesc = db + (uint64_t)(ks * 2);   // 32 bytes per k-step
             if (PHASE == 1) {
               umma(tacc, da + (uint64_t)(ks * 2), bdesc, idesc, acc);                           // G
@@ -512,6 +525,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
             } else {
               umma(tacc, da + (uint64_t)(ks * 128), bdesc, idesc, acc);  // 2 KB per k-step; columns [0, n_pad): a_hi, [n_pad, 2 n_pad): a_lo
             }
+          }
           }
           umma_commit(&empty[s]);  // the stage is free once these MMAs have read it
           CVTL(PHASE, it_mma, 6);
@@ -526,7 +540,7 @@ ffn_tc_gemm_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_consta
       // (a tile row is 128 bytes = 64 values; its 16-byte chunk j sits at chunk j ^ (row mod 8))
       const int ct = tid - kCvWarp0 * 32;
       bool ok = true;
-      for (int kt = kt_begin; kt < kt_end && ok; ++kt, ++it_cv) {
+      for (int kt = kt_begin; kt < kt_end && ok; kt += KPS, ++it_cv) {
         const int s = it_cv % NSTAGE;
         ok = __all_sync(0xffffffffu, mbar_wait(&rawfull[s], (it_cv / NSTAGE) & 1, &s_abort, p.f.wait_limit_ns));
         if (ct == 0) CVTL(PHASE, it_cv, 1);
@@ -801,7 +815,7 @@ cudaError_t launch_ffn_tc(const TcParams& p_in, const TcMaps& m, int n_sm, cudaS
   p.nmax2 = b32 < 64 ? b32 : 64;
   const size_t ring1 = 0, ring2 = 0;
   const size_t st1 = 2 * 128 * 128 + (size_t)p.nmax1 * 128 + tc_raw_bytes(1, qf);
-  const size_t st2 = 2 * 64 * 128 + 2 * (size_t)p.nmax2 * 128 + tc_raw_bytes(2, qf);
+  const size_t st2 = tc_tiles_per_stage(2, qf) * (2 * 64 * 128 + 2 * (size_t)p.nmax2 * 128) + tc_raw_bytes(2, qf);
   p.nstage1 = (int)(budget / st1) < 4 ? (int)(budget / st1) : 4;
   p.nstage2 = (int)(budget / st2) < 4 ? (int)(budget / st2) : 4;
   cudaLaunchAttribute attr[1];

@@ -72,17 +72,20 @@ inline int stream_write32(apex_ctx* ctx, cudaStream_t cs, uint32_t* dev, uint32_
   return APEX_OK;
 }
 
-// Bounded host wait for a mailbox sequence number.  The records of the hit path arrive within microseconds, so the
-// first 50 us are a plain spin; after that the core is given up between polls (yield, then sleeps growing to 32 us),
-// so a wait behind a long copy or a stalled device does not burn a core until its limit.
+// Bounded host wait for a mailbox sequence number.  Records of the hit path arrive within microseconds and a batched
+// layer-step lasts a few hundred, so the first millisecond is a plain spin (a sleep, however short it is asked to be,
+// returns after the timer slack of about 50 us: with a 50 us spin phase the batched decode loop lost 28 us per
+// layer-step to it).  After that the core is given up between polls -- yields up to 5 ms, then sleeps growing to
+// 32 us nominal -- so a wait behind a long copy or a stalled device does not burn a core until its limit.
 inline bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
   if ((int32_t)(*p - want) >= 0) return true;
   const auto t0 = std::chrono::steady_clock::now();
   const int64_t limit = ctx->cfg.wait_limit_ns * 2 + 1000000000ll;  // the device side gives up first
-  int64_t sleep_us = 0;
+  int64_t sleep_us = 1;
+  bool slow = false;
   for (uint32_t it = 0;; ++it) {
     if ((int32_t)(*p - want) >= 0) return true;
-    if (sleep_us == 0 && (it & 255u) != 255u) {
+    if (!slow && (it & 255u) != 255u) {
 #if defined(__x86_64__)
       __builtin_ia32_pause();
 #endif
@@ -92,8 +95,9 @@ inline bool host_wait_seq(apex_ctx* ctx, volatile uint32_t* p, uint32_t want) {
     if (ns > limit) return false;
     if (ns < 50000) continue;
     if (mhdr(ctx)->status != 0) return false;  // a kernel gave up: what it was going to post will not come
-    if (sleep_us == 0) {
-      sleep_us = 1;
+    if (ns < 1000000) continue;
+    slow = true;
+    if (ns < 5000000) {
       std::this_thread::yield();
     } else {
       std::this_thread::sleep_for(std::chrono::microseconds(sleep_us));

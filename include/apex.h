@@ -230,7 +230,8 @@ int apex_moe_ffn_begin(apex_ctx* ctx, int layer, int mode, const float* hpost_de
 int apex_moe_ffn_end(apex_ctx* ctx, int layer);
 
 /* All L layers of one decode step, in the order above.  h_dev, hpost_dev, y_dev are [L][B][d].
- * At B = 1 with bf16 expert stores the whole token is one cooperative kernel launch that loops over the layers
+ * At B = 1 the whole token is one cooperative kernel launch that loops over the layers (bf16 stores: d = 256 ... 4096 in the
+ * supported widths; e4m3 / e2m1 stores: d = 512, 1024, 1536, 2048, 4096)
  * (prefetch router, stand-in attention, gate, expert FFN as roles inside it; layers handed over through bounded
  * device-side counters); the host thread only plans and issues copies from the records the kernel posts and, on the
  * hit path, is never waited for.  Otherwise, and with APEX_FLAG_LAYER_LAUNCHES, one kernel sequence per layer.

@@ -13,9 +13,9 @@ namespace apex {
 // (dec_clusters = 0) and apex_decode_token keeps to the per-layer kernel sequence.
 int decode_setup(apex_ctx* ctx) {
   ctx->dec_clusters = 0;
-  if (ctx->fmt != 0 || ctx->cfg.N > kDecCluster * kDecWarps) return APEX_OK;
+  if (ctx->cfg.N > kDecCluster * kDecWarps) return APEX_OK;
   if (ctx->cfg.flags & APEX_FLAG_LAYER_LAUNCHES) return APEX_OK;
-  const int n = decode_max_clusters(ctx->cfg.d);
+  const int n = decode_max_clusters(ctx->cfg.d, ctx->fmt);
   if (n < 1) return APEX_OK;
   const size_t L = ctx->cfg.L;
   CU_TRY(ctx, dev_alloc(&ctx->d_dec_tab, L));
@@ -169,7 +169,10 @@ int decode_token_persistent(apex_ctx* ctx, const float* h_dev, const float* hpos
   p.abort_flag = ctx->d_dec_abort;
   p.attn = ctx->d_attn; p.attn_bytes = ctx->attn_bytes; p.attn_layers = (int)ctx->attn_layers;
   p.run_attn = (ctx->cfg.flags & APEX_FLAG_SKIP_STANDIN) ? 0 : 1;
-  p.standin_ahead = (ctx->cfg.flags & APEX_FLAG_STANDIN_AHEAD) ? 1 : 0;
+  p.fmt = ctx->fmt;
+  // (quantised rows are shorter than a vector of y: the cross-warp reduction then uses the start of the ring, so
+  // nothing is requested ahead of it)
+  p.standin_ahead = ((ctx->cfg.flags & APEX_FLAG_STANDIN_AHEAD) && ctx->fmt == 0) ? 1 : 0;
   p.seq = seq;
   p.demand_tag = tag;
   p.force = !prefetching ? 0 : (tau <= 0.f ? 1 : (tau >= 1.f ? 2 : 0));

@@ -224,6 +224,7 @@ struct DecodeParams {
   size_t attn_bytes;
   int attn_layers, run_attn;
   int standin_ahead;                    // 1: the stand-in's chunks are requested ahead of the previous layer's completion
+  int fmt;                              // storage format of the expert rows (FfnParams::fmt)
   uint32_t seq;                         // this token's sequence number
   uint32_t demand_tag;
   float t_tau;
@@ -256,7 +257,7 @@ bool tc_shape_supported(int d, int I, int I_shared, int fmt);
 bool ffn_shape_supported(int d);
 bool ffn_quantised_shape_supported(int d);   // widths the e4m3 / e2m1 kernels were built for
 size_t ffn_row_bytes(int fmt, int d);        // bytes of one intermediate index (three vectors and their scales)
-int decode_max_clusters(int d);              // clusters of kDecCluster CTAs the current device holds at once (0: not supported)
+int decode_max_clusters(int d, int fmt);     // clusters of kDecCluster CTAs the current device holds at once (0: not supported)
 cudaError_t launch_decode(const DecodeParams& p, int n_clusters, cudaStream_t s);
 
 }  // namespace apex

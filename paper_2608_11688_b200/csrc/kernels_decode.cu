@@ -47,6 +47,7 @@
 #include "apex_internal.hpp"
 #include "ptx.cuh"
 #include "router_common.cuh"
+#include "ffn_rows.cuh"
 #include "token_plan.cuh"
 
 namespace apex {
@@ -54,10 +55,12 @@ namespace apex {
 namespace {
 
 constexpr int kDecMaxStages = 64;
-constexpr int kDecSmemBudget = 222 * 1024;
+// Shared memory of a CTA: 227 KB, of which the kernel's static variables take 5 KB (a d = 1536 bf16 ring of 24 stages fills
+// the rest to the byte: the tests check that the token kernel is what ran) and the CTA's partial y 4 d bytes.
+constexpr int kDecSmemTotal = 227 * 1024, kDecSmemStatic = 5120;
 
-__host__ __device__ constexpr int dec_ring_stages(uint32_t entry_bytes) {
-  int n = kDecSmemBudget / (int)entry_bytes;
+__host__ __device__ constexpr int dec_ring_stages(uint32_t entry_bytes, int d) {
+  int n = (kDecSmemTotal - kDecSmemStatic - 4 * d) / (int)entry_bytes;
   if (n > kDecMaxStages) n = kDecMaxStages;
   return n / kDecWarps * kDecWarps;
 }
@@ -117,7 +120,8 @@ __device__ __forceinline__ long long row_weight_prefix(int cta, bool prefetching
 
 }  // namespace
 
-template <int NCH, bool H_REGS>
+// NCH = d / 256; H_REGS: h' of the layer in registers; FMT: storage format of the expert rows (ffn_rows.cuh).
+template <int NCH, bool H_REGS, int FMT>
 __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const DecodeParams p) {
   extern __shared__ __align__(128) uint8_t smem[];
   __shared__ uint64_t s_full[kDecMaxStages];
@@ -138,9 +142,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
   __shared__ int s_red_stage[kDecWarps];  // the stage that holds each warp's partial y during the reduction (-1: none)
 
   constexpr int d = NCH * 256;
-  constexpr uint32_t row_bytes = 2 * d;        // one bf16 vector
-  constexpr uint32_t entry_bytes = 6 * d;      // gate_i | up_i | downT_i
-  constexpr int NS = dec_ring_stages(entry_bytes);
+  constexpr uint32_t row_bytes = fmt_vec_bytes(FMT, d);      // one vector of a row
+  constexpr uint32_t entry_bytes = fmt_entry_bytes(FMT, d);  // gate_i | up_i | downT_i (| scales)
+  constexpr int NS = dec_ring_stages(entry_bytes, d);
   constexpr int NSW = NS / kDecWarps;
   constexpr int NV = d / 128;                  // float4 per lane of a router row
   constexpr int SLICE4 = d / 4 / kDecCluster;  // float4 columns of y a CTA adds for its cluster
@@ -930,6 +934,60 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
               const uint8_t* gs = smem + (size_t)s * entry_bytes;
               const uint8_t* us = gs + row_bytes;
               const uint8_t* ds = us + row_bytes;
+              if constexpr (FMT != kFmtBf16) {
+                // quantised rows: decoded eight weights at a time; e4m3 scales multiply the two dot products and the
+                // gated intermediate once per row, e2m1 block scales a lane's eight-element partial sums
+                float g = 0.f, u = 0.f;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                  float gw[8], uw[8], hh[8];
+                  load8<FMT>(gs, c * 32 + lane, gw);
+                  load8<FMT>(us, c * 32 + lane, uw);
+                  if (H_REGS) {
+#pragma unroll
+                    for (int m = 0; m < 8; ++m) hh[m] = hreg[c * 8 + m];
+                  } else {
+                    const float4 a = __ldg(reinterpret_cast<const float4*>(hpl) + (c * 32 + lane) * 2);
+                    const float4 b2 = __ldg(reinterpret_cast<const float4*>(hpl) + (c * 32 + lane) * 2 + 1);
+                    hh[0] = a.x; hh[1] = a.y; hh[2] = a.z; hh[3] = a.w; hh[4] = b2.x; hh[5] = b2.y; hh[6] = b2.z; hh[7] = b2.w;
+                  }
+                  float pg = 0.f, pu = 0.f;
+#pragma unroll
+                  for (int m = 0; m < 8; ++m) pg = fmaf(gw[m], hh[m], pg);
+#pragma unroll
+                  for (int m = 0; m < 8; ++m) pu = fmaf(uw[m], hh[m], pu);
+                  if (FMT == kFmtMxfp4) {
+                    const uint8_t* sc = ds + row_bytes;  // gate | up | downT block scales, d/32 bytes each
+                    g = fmaf(block_scale(sc, c * 32 + lane), pg, g);
+                    u = fmaf(block_scale(sc + d / 32, c * 32 + lane), pu, u);
+                  } else {
+                    g += pg;
+                    u += pu;
+                  }
+                }
+#pragma unroll
+                for (int o = 16; o > 0; o >>= 1) {
+                  const float g2 = __shfl_xor_sync(0xffffffffu, g, o), u2 = __shfl_xor_sync(0xffffffffu, u, o);
+                  g += g2;
+                  u += u2;
+                }
+                float down_scale = 1.f;
+                if (FMT == kFmtE4m3) {
+                  const float* sc = reinterpret_cast<const float*>(ds + row_bytes);
+                  g *= sc[0];
+                  u *= sc[1];
+                  down_scale = sc[2];
+                }
+                const float a = gate * g * __fdividef(1.f, 1.f + __expf(-g)) * u * down_scale;
+#pragma unroll
+                for (int c = 0; c < NCH; ++c) {
+                  float dw[8];
+                  load8<FMT>(ds, c * 32 + lane, dw);
+                  const float ac = FMT == kFmtMxfp4 ? a * block_scale(ds + row_bytes + 2 * (d / 32), c * 32 + lane) : a;
+#pragma unroll
+                  for (int m = 0; m < 8; ++m) acc[c * 8 + m] = fmaf(ac, dw[m], acc[c * 8 + m]);
+                }
+              } else {
               // four partial sums per dot product: independent chains instead of one of 8 * NCH dependent multiply-adds
               float gp[4] = {0.f, 0.f, 0.f, 0.f}, up[4] = {0.f, 0.f, 0.f, 0.f};
 #pragma unroll
@@ -971,6 +1029,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
                 acc[c * 8 + 2] = fmaf(a, dbf16lo(dv.y), acc[c * 8 + 2]); acc[c * 8 + 3] = fmaf(a, dbf16hi(dv.y), acc[c * 8 + 3]);
                 acc[c * 8 + 4] = fmaf(a, dbf16lo(dv.z), acc[c * 8 + 4]); acc[c * 8 + 5] = fmaf(a, dbf16hi(dv.z), acc[c * 8 + 5]);
                 acc[c * 8 + 6] = fmaf(a, dbf16lo(dv.w), acc[c * 8 + 6]); acc[c * 8 + 7] = fmaf(a, dbf16hi(dv.w), acc[c * 8 + 7]);
+              }
               }
             }
             __syncwarp();  // every lane has read stage s: it may be refilled
@@ -1018,10 +1077,15 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     // ------------------------------------------------------------ y: warps -> CTA -> cluster -> memory; count the CTA in
     // A warp's partial vector goes to the stage it would use next: free, because at most NSW - 1 of its copies (the
     // next layer's, started ahead) are outstanding.  After a failed wait nothing is written (the CTA contributes zeros).
-    const bool warp_good = go_rows && ok && (n_iss - n_con) <= NSW - 1;
-    if (lane == 0) s_red_stage[warp] = warp_good ? warp + kDecWarps * (n_iss % NSW) : -1;
+    // (A quantised row is shorter than a vector of y: the warps' vectors then lie side by side at the start of the ring,
+    // written once every warp of the CTA has consumed its rows; no copies are started ahead in that case.)
+    constexpr bool RED_IN_STAGE = entry_bytes >= (uint32_t)d * 4u;
+    const bool warp_good = go_rows && ok && (RED_IN_STAGE ? (n_iss - n_con) <= NSW - 1 : n_iss == n_con);
+    if (lane == 0) s_red_stage[warp] = warp_good ? (RED_IN_STAGE ? warp + kDecWarps * (n_iss % NSW) : warp) : -1;
+    if (!RED_IN_STAGE) __syncthreads();
     if (warp_good) {
-      float4* dst = reinterpret_cast<float4*>(smem + (size_t)(warp + kDecWarps * (n_iss % NSW)) * entry_bytes);
+      float4* dst = reinterpret_cast<float4*>(RED_IN_STAGE ? smem + (size_t)(warp + kDecWarps * (n_iss % NSW)) * entry_bytes
+                                                           : smem + (size_t)warp * d * 4);
 #pragma unroll
       for (int c = 0; c < NCH; ++c) {
         const int col4 = (c * 32 + lane) * 2;
@@ -1040,7 +1104,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
       for (int w = 0; w < kDecWarps; ++w) {
         const int st = s_red_stage[w];
         if (st >= 0) {
-          const float4 v = reinterpret_cast<const float4*>(smem + (size_t)st * entry_bytes)[col4];
+          const float4 v = reinterpret_cast<const float4*>(RED_IN_STAGE ? smem + (size_t)st * entry_bytes : smem + (size_t)st * d * 4)[col4];
           sacc.x += v.x; sacc.y += v.y; sacc.z += v.z; sacc.w += v.w;
         }
       }
@@ -1093,11 +1157,11 @@ extern "C" int apex_debug_read_decode_timeline(unsigned long long* host) {
 // ---------------------------------------------------------------- host side
 namespace {
 
-template <int NCH>
+template <int NCH, int FMT = 0>
 cudaError_t launch_decode_t(const DecodeParams& p, int n_clusters, cudaStream_t s, int* max_clusters_out) {
   constexpr bool HR = NCH <= 8;
-  constexpr uint32_t entry = 6 * NCH * 256;
-  constexpr int NS = dec_ring_stages(entry);
+  constexpr uint32_t entry = fmt_entry_bytes(FMT, NCH * 256);
+  constexpr int NS = dec_ring_stages(entry, NCH * 256);
   const size_t smem = (size_t)NS * entry + (size_t)NCH * 256 * sizeof(float);  // ring, then the CTA's partial y
   static bool configured[kMaxDevices] = {};
   int dev = 0;
@@ -1105,7 +1169,7 @@ cudaError_t launch_decode_t(const DecodeParams& p, int n_clusters, cudaStream_t 
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= kMaxDevices) return cudaErrorInvalidDevice;
   if (!configured[dev]) {
-    e = cudaFuncSetAttribute(decode_token_kernel<NCH, HR>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    e = cudaFuncSetAttribute(decode_token_kernel<NCH, HR, FMT>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     configured[dev] = true;
   }
@@ -1125,16 +1189,30 @@ cudaError_t launch_decode_t(const DecodeParams& p, int n_clusters, cudaStream_t 
     cfg.gridDim = dim3(kDecCluster, 1, 1);
     cfg.numAttrs = 1;
     int n = 0;
-    e = cudaOccupancyMaxActiveClusters(&n, decode_token_kernel<NCH, HR>, &cfg);
+    e = cudaOccupancyMaxActiveClusters(&n, decode_token_kernel<NCH, HR, FMT>, &cfg);
     *max_clusters_out = e == cudaSuccess ? n : 0;
     return e;
   }
   cfg.gridDim = dim3(kDecCluster * n_clusters, 1, 1);
   cfg.numAttrs = 2;
-  return cudaLaunchKernelEx(&cfg, decode_token_kernel<NCH, HR>, p);
+  return cudaLaunchKernelEx(&cfg, decode_token_kernel<NCH, HR, FMT>, p);
+}
+
+template <int FMT>
+cudaError_t dispatch_quantised(const DecodeParams& p, int n_clusters, cudaStream_t s, int* max_clusters_out) {
+  switch (p.d) {  // the widths the quantised row decoders are built for
+    case 512: return launch_decode_t<2, FMT>(p, n_clusters, s, max_clusters_out);
+    case 1024: return launch_decode_t<4, FMT>(p, n_clusters, s, max_clusters_out);
+    case 1536: return launch_decode_t<6, FMT>(p, n_clusters, s, max_clusters_out);
+    case 2048: return launch_decode_t<8, FMT>(p, n_clusters, s, max_clusters_out);
+    case 4096: return launch_decode_t<16, FMT>(p, n_clusters, s, max_clusters_out);
+  }
+  return cudaErrorInvalidValue;
 }
 
 cudaError_t dispatch(const DecodeParams& p, int n_clusters, cudaStream_t s, int* max_clusters_out) {
+  if (p.fmt == kFmtE4m3) return dispatch_quantised<kFmtE4m3>(p, n_clusters, s, max_clusters_out);
+  if (p.fmt == kFmtMxfp4) return dispatch_quantised<kFmtMxfp4>(p, n_clusters, s, max_clusters_out);
   switch (p.d) {
     case 256: return launch_decode_t<1>(p, n_clusters, s, max_clusters_out);
     case 512: return launch_decode_t<2>(p, n_clusters, s, max_clusters_out);
@@ -1150,9 +1228,10 @@ cudaError_t dispatch(const DecodeParams& p, int n_clusters, cudaStream_t s, int*
 
 }  // namespace
 
-int decode_max_clusters(int d) {
+int decode_max_clusters(int d, int fmt) {
   DecodeParams p{};
   p.d = d;
+  p.fmt = fmt;
   int n = 0;
   if (dispatch(p, 0, nullptr, &n) != cudaSuccess) {
     cudaGetLastError();

@@ -61,6 +61,20 @@ def test_persistent_token_kernel_with_a_gated_shared_expert(mode):
     assert rep.near_ties == 0 and rep.ffn_checked == 5 * 4 and launches == 5     # one launch per token
 
 
+@pytest.mark.parametrize("mode", ["exact", "stall_free"])
+@pytest.mark.parametrize("fmt", ["fp8", "fp4"])
+@pytest.mark.parametrize("d,N,k,I,C,L,Ish", [(512, 12, 3, 40, 6, 3, 16), (1024, 64, 8, 16, 16, 2, 0), (1536, 40, 8, 64, 20, 4, 0),
+                                             (2048, 60, 4, 32, 30, 3, 48), (4096, 8, 2, 24, 4, 3, 0)])
+def test_persistent_token_kernel_quantised_stores(d, N, k, I, C, L, Ish, fmt, mode):
+    # the token kernel on e4m3 / e2m1 expert stores: rows shorter than a vector of y (the cross-warp reduction then
+    # uses the start of the ring), more and smaller ring stages, the same decisions
+    cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, L=L, T=5, I_shared=Ish, sigma_p=1.0, cfg_id=420 + N)
+    prob = _harness().Problem(cfg, fp8=(fmt == "fp8"), fp4=(fmt == "fp4"))
+    rep, stats, launches = _decode(cfg, mode=mode, tau=0.7, T=5, prob=prob)
+    assert rep.layer_steps == 5 * L and rep.ffn_checked == 5 * L and rep.near_ties == 0
+    assert launches == 5                       # one kernel per token: the persistent path ran
+
+
 @pytest.mark.parametrize("tau", [-1.0, 0.0, 0.97, 1.0])
 def test_persistent_token_kernel_policies_and_budget_extremes(tau):
     cfg = synth.tiny_config(d=512, N=16, k=4, I=32, C=8, L=3, T=8, sigma_p=0.8, cfg_id=410)

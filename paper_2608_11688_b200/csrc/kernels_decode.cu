@@ -304,13 +304,16 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     return s;
   };
   // A router row in registers: lane l holds float4 columns l, l + 32, ... (the order of router_kernel's reduction).
-  // Only up to d = 1024 (8 float4 per lane and row).  Wider rows are read when their dot product is taken (they were
-  // prefetched into L2 at the start of the layer): two rows of d = 2048 in registers spilled and cost 17 % of the
-  // layer-step (configs 2 and 4: 36.8 -> 31.5 and 42.3 -> 35.8 us without them), and even the 96 registers of two
-  // d = 1536 rows, which fit, cost the row loop more than the loads' latency costs the logits (config 1 without the
-  // stand-in: 19.3 -> 17.8 us per layer-step).
+  // Up to d = 1024 (8 float4 per lane and row) both rows are fetched at the start of the layer.  Wider rows are
+  // prefetched into L2 there instead: two rows of d = 2048 in registers spilled and cost 17 % of the layer-step
+  // (configs 2 and 4: 36.8 -> 29.8 and 42.3 -> 35.1 us without them), and even the 96 registers of two d = 1536 rows,
+  // which fit, cost the row loop more than the loads' latency costs the logits (config 1 without the stand-in:
+  // 19.3 -> 17.2 us per layer-step).  The prefetch router's wide row is read when its dot product is taken; the gate's
+  // row of d = 1536 comes into registers right before the wait for the attention window (the latency passes during the
+  // wait; + 3 % with the stand-in), and is read with x where there is no window to wait for.
   constexpr int NVRP = NV <= 8 ? NV : 1;   // prefetch-router row
-  constexpr int NVRR = NV <= 8 ? NV : 1;   // gate row
+  constexpr int NVRR = NV <= 12 ? NV : 1;  // gate row (9 to 12 float4 per lane: loaded late, see below; wider: not held)
+  constexpr bool WR_LATE = NV > 8 && NV <= 12;       // the gate row is fetched right before the wait for the attention window
   auto load_row = [&](const float* __restrict__ W_row, auto& wr) {
     constexpr int NVR = (int)(sizeof(wr) / sizeof(float4));
     constexpr bool ROW_REGS = NVR > 1 || NV == 1;
@@ -321,14 +324,14 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
       asm volatile("ld.global.nc.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(wr[i].x), "=f"(wr[i].y), "=f"(wr[i].z), "=f"(wr[i].w) : "l"(rp + i * 32 + lane));
   };
   // dot product of the row with x (reduction order of router_kernel), plus bias; sent to CTAs [rank_lo, rank_hi) of the cluster
-  auto row_logit = [&](const float* __restrict__ W_row, const auto& wr, const float* __restrict__ x, float bias, float* zs,
+  auto row_logit = [&](const float* __restrict__ W_row, const auto& wr, bool held, const float* __restrict__ x, float bias, float* zs,
                        uint64_t* xbar, int rank_lo, int rank_hi) {
     constexpr int NVR = (int)(sizeof(wr) / sizeof(float4));
     constexpr bool ROW_REGS = NVR > 1 || NV == 1;
     const float4* __restrict__ xv = reinterpret_cast<const float4*>(x);
     const float4* __restrict__ rp = reinterpret_cast<const float4*>(W_row);
     float acc = 0.f;
-    if (ROW_REGS) {
+    if (ROW_REGS && held) {
       float4 xr[NVR];
 #pragma unroll
       for (int i = 0; i < NVR; ++i) xr[i] = __ldg(xv + i * 32 + lane);
@@ -388,7 +391,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     const float* Wp_row = p.W_p + ((size_t)l * N + (has_row ? my_e : 0)) * d;
     const float* Wr_row = p.W_r + ((size_t)l * N + (has_row ? my_e : 0)) * d;
     if (has_wp) load_row(Wp_row, wp_row);
-    if (has_wr && !has_wp) load_row(Wr_row, wr_row);  // (a warp with both rows fetches W_r after its W_p dot product)
+    if (has_wr && !has_wp && !WR_LATE) load_row(Wr_row, wr_row);  // (a warp with both rows fetches W_r after its W_p dot product)
     if (has_row) {
       if (has_wp) bias_p = __ldg(p.b_p + (size_t)l * N + my_e);
       bias_r = __ldg(p.b_r + (size_t)l * N + my_e);
@@ -489,9 +492,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     if (ok && running) start_seg1(l, NSW);  // this layer's chunks: on their way while the prefetch logit is computed
     // prefetch router first of all: the sooner the candidate set is out, the more of the window the copies can use
     if (has_wp && running && ok) {
-      row_logit(Wp_row, wp_row, hl, bias_p, s_zp, &s_xbar[0], kDecCluster - 1, kDecCluster);  // to the poster only
+      row_logit(Wp_row, wp_row, true, hl, bias_p, s_zp, &s_xbar[0], kDecCluster - 1, kDecCluster);  // to the poster only
       DTL(1);
-      if (has_wr) load_row(Wr_row, wr_row);
+      if (has_wr && !WR_LATE) load_row(Wr_row, wr_row);
     }
     {
       int q_con = 0;
@@ -517,6 +520,9 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
     // exact gate: this warp's logit, once the whole stand-in has been streamed (a real attention block would only then
     // have produced h') and the previous layer's y is complete
     if (has_wr && ok && !cta_stopped()) {
+      // (a wide gate row comes into registers only now, from L2: its latency passes while the counters are waited for,
+      // and the registers were free for the stand-in's segment and are free again for the expert rows)
+      if (WR_LATE && p.run_attn) load_row(Wr_row, wr_row);  // (without a window to wait for, the row is read with x)
       bool go = true;
       if (lane == 0) {
         if (p.run_attn) go = wait_counter(bar_attn, p.bar_target);
@@ -528,7 +534,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
         ok = false;
       } else {
         DTL(14);
-        row_logit(Wr_row, wr_row, hpl, bias_r, s_zr, &s_xbar[1], 0, kDecCluster);
+        row_logit(Wr_row, wr_row, !WR_LATE || p.run_attn != 0, hpl, bias_r, s_zr, &s_xbar[1], 0, kDecCluster);
         DTL(4);
       }
     }

@@ -8,30 +8,32 @@
 // a shared-memory ring with bulk asynchronous copies (TMA, mbarrier completion), exactly as the per-layer streaming
 // kernel does.  A warp's stream is ONE sequence over all layers; per layer, in this order,
 //
-//   [its share of the attention stand-in's bytes, its row of W_p among the first]  [its row of W_r]  [its rows of the expert FFN]
+//   [its share of the attention stand-in's bytes]  [its rows of the expert FFN]
 //
 // The stand-in's chunks of a layer are requested when the previous layer's y is complete (the attention block's window
 // of Eq. (12) opens when its input exists).  With APEX_FLAG_STANDIN_AHEAD they are requested as far ahead as the ring
 // allows instead -- a warp starts them as soon as its last expert rows of the previous layer have been requested, so
 // they arrive while that layer's tail, the reduction of y and the hand-over are still going on; faster, but the window
 // then overlaps the previous layer.  (Consumption stays in order, and everything derived from h or h' waits for the
-// counters below.)
+// counters below.)  The router rows do not go through the ring: narrow ones (d <= 1024) are held in registers from the
+// start of the layer, wide ones are prefetched into L2 and read when the dot product is taken (see load_row).
 //
-//   prefetch router (S1-S3): CTA r of a cluster owns experts 8r .. 8r+7, one warp per expert.  The row arrives in the
-//     ring; its dot product with h (reduction order of router_kernel: lane-strided fused multiply-adds, then the xor
-//     tree -- the logits are bit-identical to the per-layer kernels') waits for the previous layer's y to be complete
-//     (device counter) and is sent to all eight CTAs of the cluster through distributed shared memory with
-//     st.async, which also counts the bytes on the receiver's mbarrier.  Only the first cluster does this, and only its
-//     last CTA (which owns no router row for N <= 56, so nothing else waits for it) derives softmax, ranking, budget
-//     and candidate set, posts the record the host plans the prefetch copies from, and leaves the candidate mask in
-//     device memory for everybody else.
+//   prefetch router (S1-S3): CTA r of a cluster owns experts 8r .. 8r+7, one warp per expert.  Its dot product with h
+//     (reduction order of router_kernel: lane-strided fused multiply-adds, then the xor tree -- the logits are
+//     bit-identical to the per-layer kernels') waits for the previous layer's y to be complete (device counter) and is
+//     sent through distributed shared memory with st.async, which also counts the bytes on the receiver's mbarrier.
+//     Only the first cluster does this, and only its last CTA (the "poster", whose warp 0 carries neither stand-in
+//     chunks nor expert rows) receives the logits and derives softmax, ranking, budget and candidate set, posts the
+//     record the host plans the prefetch copies from, and leaves the candidate mask in device memory for everybody else.
 //   attention stand-in: the bytes that define the hiding window of Eq. (12), streamed by everybody.
-//   exact gate (S4): the same exchange with W_r and h', after ALL CTAs have finished the stand-in (device counter):
-//     a real attention block would only then have produced h'.  Every warp derives K_r, alpha and the execution set
-//     (S6) itself, so no further exchange is needed before the expert rows are requested.
-//   expert FFN (S7, S8): rows split evenly over the CTAs; slot-ready flags, demand words and every other wait
-//     are bounded as in the per-layer kernel.  Partial y vectors are reduced over the warps in shared memory and
-//     added to y with vector atomics; then the CTA counts itself in on the layer's counter.
+//   exact gate (S4): the same exchange with W_r and h', to all eight CTAs of every cluster, after ALL CTAs have
+//     finished the stand-in (device counter): a real attention block would only then have produced h'.  The ranks are
+//     counted once per CTA (the comparisons split over its warps, summed in shared memory); every warp then derives
+//     K_r, alpha and the execution set (S6) itself, so no further exchange is needed before the expert rows are requested.
+//   expert FFN (S7, S8): rows split over the CTAs by weight (the first cluster and the poster take fewer); slot-ready
+//     flags, demand words and every other wait are bounded as in the per-layer kernel.  Partial y vectors are reduced
+//     over the warps in shared memory, then over the cluster (CTA r sums slice r of the eight partial vectors through
+//     distributed shared memory) and added to y with vector atomics; then the CTA counts itself in on the layer's counter.
 //
 // Slot tables: the kernel holds the table of every layer as it stood when the token was launched.  If a layer's
 // candidates are all resident in it (and slots persist), nothing changes and the kernel never waits for the host;

@@ -133,7 +133,7 @@ __global__ void __launch_bounds__(kDecThreads, 1) decode_token_kernel(const Deco
   __shared__ unsigned s_rank[APEX_MAX_EXPERTS / 4];  // rank of each expert's gate logit, four 8-bit counts to a word (zero between layers)
   __shared__ float s_zp[APEX_MAX_EXPERTS], s_zr[APEX_MAX_EXPERTS];
   __shared__ float s_q[APEX_MAX_EXPERTS];              // warp 0: prefetch probabilities by expert
-  __shared__ int s_pi[kDecWarps][APEX_MAX_EXPERTS];    // per-warp scratch: expert by rank
+  __shared__ int s_pi[1][APEX_MAX_EXPERTS];            // warp 0: expert by rank
   __shared__ int s_posp[APEX_MAX_EXPERTS];             // position of each expert in the prefetch ranking (warp 0)
   __shared__ int s_pos[kDecWarps][APEX_MAX_TOPK];      // expert at each position of the row space (a copy per warp)
   __shared__ int s_exp[kDecMaxStages];

@@ -77,3 +77,30 @@ def test_traced_decode_records_every_kernel_in_order():
     rows = [l for l in r.stderr.splitlines() if l[:6] in ("prefet", "attent", "gate  ", "expert")]
     assert rows[0].startswith("prefetch router") and rows[1].startswith("attention") and rows[2].startswith("gate")
     assert rows[3].startswith("expert FFN")
+
+
+@pytest.mark.gpu
+def test_bench_line_carries_the_contract_keys():
+    # a short run of the default workload (config 1, 32 layers): one JSON line with the metric, the end-to-end figure
+    # through host buffers, the roofline record of the dominant kernel, the CPU oracle baseline and the clock record
+    r = subprocess.run([sys.executable, "bench.py", "--steps", "6", "--warmup", "3", "--no-policies", "--no-other-configs",
+                        "--cpu-baseline-tokens", "1"], cwd=ROOT, capture_output=True, text=True, timeout=900)
+    assert r.returncode == 0, r.stderr[-2000:]
+    lines = [l for l in r.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1
+    d = json.loads(lines[0])
+    assert d["metric"] == "moe_decode_tokens_per_s" and d["unit"] == "tokens/s" and d["n_gpus"] == 1 and d["steps"] == 6
+    assert d["higher_is_better"] is True and d["scaling"] == "weak" and d["vs_baseline"] is None and d["data"] == "synthetic"
+    assert d["config"]["workload"].startswith("config1") and "model" not in d["config"]
+    assert 5.0 < d["value"] < 1000.0 and abs(d["ms_per_step"] * d["value"] - 1000.0) < 1.0
+    assert d["gpu_launches"] == 6                                  # one token kernel per timed token
+    e = d["e2e"]
+    assert 5.0 < e["value"] < 1000.0 and e["h2d_bytes_per_step"] == 2 * 32 * 1536 * 4 and e["d2h_bytes_per_step"] == 32 * 1536 * 4
+    rf = d["roofline"]
+    assert rf["bound"] == "hbm" and rf["kernel"] == "decode_token_kernel" and rf["unit"] == "GB/s"
+    assert abs(rf["frac"] - rf["achieved"] / rf["peak"]) < 1e-9 and 0.05 < rf["frac"] < 1.2 and "traffic" in rf
+    assert rf["per_layer_ffn_kernel_alone"]["kernel"] == "moe_ffn_stream_kernel" and rf["per_layer_ffn_kernel_alone"]["traffic"] > 3.7e7
+    c = d["cpu_baseline"]
+    assert c["kind"] == "oracle" and c["cores"] >= 1 and c["value"] > 0 and "sample" in c
+    k = d["clocks"]
+    assert k["sm_mhz"] > 0 and k["sm_max_mhz"] >= k["sm_mhz"] and isinstance(k["reasons"], list)

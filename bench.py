@@ -277,7 +277,8 @@ def window_sweep(args, cfg, prob, h_dev, hp_dev, y_dev, B):
         row = {"ctx_len": ctx_len, "T_attn_us": t_attn_us, "T_attn_over_copy": t_attn_us / t_copy_us, "all_resident_ms_per_token": res_ms,
                "policies": {}}
         for name, tau_p, delta, reuse in (("no_prefetch", -1.0, None, 1), ("static_k", 0.9, 0, 1), ("static_k+4", 0.9, 4, 1),
-                                          ("apex", TAU, None, 1), ("apex_load_use_evict", TAU, None, 0)):
+                                          ("apex", TAU, None, 1), ("apex_tau0.75", 0.75, None, 1), ("apex_tau0.5", 0.5, None, 1),
+                                          ("apex_load_use_evict", TAU, None, 0)):
             r = run_policy(cfg, prob, h_dev, hp_dev, y_dev, B, name, tau_p, delta, warmup, steps, ctx_len=ctx_len, cache_reuse=reuse)
             pre_l, dem_l = r["prefetch_copies_per_token"] / L, r["demand_copies_per_token"] / L
             bound_us = L * (max(0.0, pre_l * t_copy_us - t_attn_us) + dem_l * t_copy_us)

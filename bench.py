@@ -240,7 +240,7 @@ def window_sweep(args, cfg, prob, h_dev, hp_dev, y_dev, B):
     """Study of the overlap condition, Eq. (12): T_prefetch(delta) = delta * S_expert / B_eff + T_queue <= T_attn.  On this
     machine one expert copy over the host link is far longer than the attention window of the paper's context lengths,
     so nothing can be hidden and the policies that move fewer bytes win.  Here the OTHER side of the ratio is moved: the
-    stand-in attention is lengthened (through ctx_len) until the window holds 0.5, 1, 2 and 4 expert copies, and the
+    stand-in attention is lengthened (through ctx_len) until the window holds 0.5, 1, 2, 4 and 8 expert copies, and the
     policies of Sec. V-A are timed at every window.  Per policy: tokens/s, demand copies per token, the exposed stall
     (time per token minus the all-resident time at the same window) and the stall Eq. (12) allows at best
     (per layer: what the prefetch copies overrun the window by, plus the demand copies, at the measured link rate)."""
@@ -266,7 +266,7 @@ def window_sweep(args, cfg, prob, h_dev, hp_dev, y_dev, B):
     bytes_of = lambda c: (4 * d * d + 2 * c * d) * 2
     us_per_byte = (ms_b - ms_a) * 1e3 / L / (bytes_of(65536) - bytes_of(1024))
     rows = []
-    for ratio in (None, 0.5, 1.0, 2.0, 4.0):
+    for ratio in (None, 0.5, 1.0, 2.0, 4.0, 8.0):
         if ratio is None:
             ctx_len = 1024
         else:
@@ -539,7 +539,11 @@ def main():
                          "its duration at 8, 16 and 32 GB/s) and on the link as it is")
     ap.add_argument("--window-sweep", action="store_true",
                     help="study: the policies of Sec. V-A with the hiding window (the stand-in attention, through ctx_len) "
-                         "lengthened until it holds 0.5, 1, 2 and 4 expert copies -- the regime in which Eq. (12) can hold")
+                         "lengthened until it holds 0.5, 1, 2, 4 and 8 expert copies -- the regime in which Eq. (12) can hold")
+    ap.add_argument("--predictor-noise", type=float, default=1.0,
+                    help="study: scales what makes the prefetch router wrong in the synthetic workload (the noise on W_p and "
+                         "the part of h' the router cannot see): 1 is the workload of the configs, 0.2 a good predictor.  "
+                         "The frozen confidence models were fitted at 1: combine with --train-aux")
     ap.add_argument("--train-aux", action="store_true",
                     help="study: distil the prefetch routers and refit the confidence models on this GPU first "
                          "(a different predictor than the workload's: needs --skip-extras)")
@@ -551,8 +555,10 @@ def main():
     args = ap.parse_args()
     if (args.fp8 or args.fp4) and not (args.ffn_only or args.skip_extras):
         ap.error("--fp8 / --fp4 are study legs: combine them with --ffn-only or --skip-extras")
-    if args.train_aux and not args.skip_extras:
-        ap.error("--train-aux is a study leg: combine it with --skip-extras")
+    if args.train_aux and not (args.skip_extras or args.window_sweep):
+        ap.error("--train-aux is a study leg: combine it with --skip-extras or --window-sweep")
+    if args.predictor_noise != 1.0 and not (args.skip_extras or args.window_sweep):
+        ap.error("--predictor-noise is a study leg: combine it with --skip-extras or --window-sweep")
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
@@ -561,6 +567,8 @@ def main():
     cfg = synth.CONFIGS[args.config]
     if args.layers:
         cfg = cfg.scaled(L=args.layers)
+    if args.predictor_noise != 1.0:
+        cfg = cfg.scaled(sigma_p=cfg.sigma_p * args.predictor_noise, hidden_noise=cfg.hidden_noise * args.predictor_noise)
     if args.impl == "reference":
         args.steps = 2 if args.steps is None else min(args.steps, 4)
         args.warmup = 0 if args.warmup is None else args.warmup

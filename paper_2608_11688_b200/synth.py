@@ -48,6 +48,7 @@ class Config:
     batches: Tuple[int, ...] = (1,)
     I_shared: int = 0
     sigma_p: float = 0.3      # prefetch-router noise std, in units of 1/sqrt(d)
+    hidden_noise: float = 0.5  # std of h' - h per element (what attention adds that the prefetch router cannot see)
     zipf_s: float = 0.0       # >0: skewed expert popularity through a router bias
     modes: Tuple[str, ...] = ("exact", "stall_free")
 
@@ -108,7 +109,7 @@ def hidden_states(cfg: Config, layer: int, T: int, B: int = 1, calib: bool = Fal
     """Returns (h [T][B][d], h' [T][B][d]) fp32 holding bf16-representable values."""
     a, b = ("calib_hidden", "calib_noise") if calib else ("hidden", "hidden_noise")
     h = _rng(cfg, layer, a).standard_normal((T, B, cfg.d)).astype(np.float32)
-    hp = h + 0.5 * _rng(cfg, layer, b).standard_normal((T, B, cfg.d)).astype(np.float32)
+    hp = h + np.float32(cfg.hidden_noise) * _rng(cfg, layer, b).standard_normal((T, B, cfg.d)).astype(np.float32)
     return round_to_bf16_values(h), round_to_bf16_values(hp)
 
 

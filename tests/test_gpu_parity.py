@@ -857,3 +857,40 @@ def test_random_shapes_modes_and_options():
         finally:
             apex.destroy()
 
+
+def test_random_shapes_tensor_core_path_gated_shared_expert_and_token_kernel():
+    """A second fixed-seed walk, over what the first one reaches rarely or not at all: batches of 16 to 40 tokens on shapes the
+    grouped GEMMs accept (all three store formats), the gated shared expert, and B = 1 through apex_decode_token (the
+    persistent token kernel, checked by replaying every layer against the oracle)."""
+    import random
+    rng = random.Random(20260812)
+    hz = _harness()
+    for it in range(24):
+        tc = it % 2 == 0
+        if tc:
+            d, I, Ish, B = rng.choice([512, 1024]), rng.choice([128, 256]), rng.choice([0, 128, 384]), rng.choice([16, 24, 40])
+        else:
+            d, I, Ish, B = rng.choice([512, 1024, 1536, 2048]), rng.choice([8, 17, 64, 128]), rng.choice([0, 16, 128]), 1
+        N = rng.randint(4, 64)
+        k = rng.randint(1, min(N, 16))
+        C = rng.choice([rng.randint(k, N), N])
+        mode = rng.choice(["exact", "stall_free"])
+        tau = rng.choice([0.0, 0.7, 0.9, 1.0])
+        fmt = rng.choice(["bf16", "fp8", "fp4"])
+        gated = Ish > 0 and rng.random() < 0.6
+        L = rng.choice([1, 2, 3])
+        cfg = synth.tiny_config(d=d, N=N, k=k, I=I, C=C, L=L, T=4, I_shared=Ish, sigma_p=rng.choice([0.3, 1.0, 4.0]), cfg_id=2100 + it)
+        prob = hz.Problem(cfg, fp8=(fmt == "fp8"), fp4=(fmt == "fp4"), gated_shared=gated)
+        apex = prob.make_ctx(max_batch=B)
+        try:
+            if tc:
+                rep = hz.run_lockstep(prob, apex, mode=mode, tau=tau, T=3, B=B)
+                assert rep.layer_steps == 3 * L
+            else:
+                n0 = apex.launch_count()
+                rep = hz.run_decode_lockstep(prob, apex, mode=mode, tau=tau, T=4)
+                assert apex.launch_count() - n0 == 4, "the persistent token kernel did not run"
+            assert apex.get_stats()["timeouts"] == 0 and rep.near_ties == 0
+        finally:
+            apex.destroy()
+

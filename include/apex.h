@@ -1,8 +1,8 @@
 /*
  * apex.h -- C ABI of the B200-native MoE decode step with adaptive expert prefetch.
  *
- * One layer-step of decoding, as the paper sequences it (Sec. IV-A "two stages", Sec. IV-D
- * "Runtime Operation"):
+ * One layer-step of decoding, as the paper sequences it (the two stages of Sec. IV-A, the run-time
+ * sequence of Sec. IV-D):
  *
  *   apex_predict            prefetch router on the pre-attention state h       (Sec. IV-D)
  *   apex_select_candidates  confidence-driven budget delta_hat and K_p         (Eq. (8), (9), (1))
@@ -205,7 +205,7 @@ int apex_route_topk(apex_ctx* ctx, int layer, const float* hpost_dev, int B, int
                     float* alpha_dev, void* stream);
 /* S6-S8 (Sec. IV-E): y_dev [B][d] = sum over the execution set of g_e FFN_e(h') (+ shared FFN).
  * APEX_MODE_EXACT executes K_r: resident experts first, missing ones are copied on demand while
- * those run ("asynchronous miss correction") -- at B = 1 the one kernel waits (bounded) for each
+ * those run (asynchronous miss correction) -- at B = 1 the one kernel waits (bounded) for each
  * missing expert and then executes it, at B > 1 further launches follow.  APEX_MODE_STALL_FREE executes
  * Algorithm 1 with K_p := the resident set.  exec_idx_dev [B][k] (ascending expert index) and
  * exec_gate_dev [B][k] may be NULL.  Device-side waits on slot-ready flags are bounded; when one

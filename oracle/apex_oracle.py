@@ -356,9 +356,8 @@ class SlotCache:
 
 
 # --------------------------------------------------------------------------------------
-# One layer-step, all tokens of the batch (runtime sequencing of Sec. IV-D "Runtime
-# Operation": predict + budget before attention, prefetch during attention, exact gate after
-# attention, then the chosen execution mode)
+# One layer-step, all tokens of the batch (runtime sequencing of Sec. IV-D: predict + budget before
+# attention, prefetch during attention, exact gate after attention, then the chosen execution mode)
 # --------------------------------------------------------------------------------------
 def layer_step(cache: SlotCache, *, W_p, b_p, W_r, b_r, w, theta, tau: float, k: int,
                h: np.ndarray, h_post: np.ndarray, mode: str,

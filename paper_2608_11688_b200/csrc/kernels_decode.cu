@@ -1,6 +1,6 @@
 // Persistent decode kernel: all L layer-steps of one token (B = 1) in ONE cooperative launch, so that no kernel
-// launch, no grid completion and no host round trip sits between the steps of the hit path (Sec. IV-D "Runtime
-// Operation": predict + budget before attention, prefetch during attention, exact gate after it, then the chosen
+// launch, no grid completion and no host round trip sits between the steps of the hit path (Sec. IV-D:
+// predict + budget before attention, prefetch during attention, exact gate after it, then the chosen
 // execution mode of Sec. IV-E; the overlap condition is Eq. (12)).
 //
 // Grid: clusters of eight CTAs, as many as the GPU holds at one CTA per SM (15 on a B200: 120 CTAs stream a layer's

@@ -328,7 +328,7 @@ __global__ void __launch_bounds__(kFfnThreads, kCtasPerSm) moe_ffn_stream_kernel
       int slot = p.snap.expert_slot[e];
       if (slot < 0) {
         // not resident when the kernel was launched: the host fetches it on demand and publishes
-        // (tag, slot) after the copy -- "asynchronous miss correction" inside one launch
+        // (tag, slot) after the copy -- asynchronous miss correction inside one launch
         if (!p.demand_in_kernel) {  // refuse rather than read out of range
           ok = false;
           return;

@@ -69,7 +69,8 @@ def test_minimal_cache_C_equals_k():
     cfg = synth.tiny_config(d=256, N=10, k=3, I=16, C=3, T=20, sigma_p=1.5, cfg_id=212)
     rep, stats = _run(cfg, mode="exact", tau=0.9, T=20)
     assert rep.n_miss_steps > 0            # a noisy predictor with no spare slot misses
-    assert stats["extra_waves"] == 0       # B = 1: missing experts are waited for inside the one launch
+    if _harness().token_kernel_expected():     # (where launch calls may block the host corrects misses between launches)
+        assert stats["extra_waves"] == 0       # B = 1: missing experts are waited for inside the one launch
     assert stats["demand_copies"] == rep.n_demand_copies > 0
     rep, stats = _run(cfg, mode="stall_free", tau=0.9, T=20)
     assert rep.n_subst > 0 and stats["substitutions"] == rep.n_subst
@@ -80,6 +81,8 @@ def test_exact_mode_with_host_side_miss_correction(how, monkeypatch):
     # B = 1, exact mode, no wait for the host inside the kernel: resident routed experts first, one further launch per
     # demand wave.  The setting for processes whose kernel launches block (it is chosen from the environment when the
     # context is created).  Same decisions, same table, same output as the oracle.
+    if not _harness().token_kernel_expected():
+        pytest.skip("launch calls already block in this process: every context corrects misses on the host, nothing to compare")
     cfg = synth.tiny_config(d=256, N=10, k=3, I=16, C=3, T=20, sigma_p=1.5, cfg_id=212)
     if how == "environment":
         monkeypatch.setenv("CUDA_LAUNCH_BLOCKING", "1")       # read by apex_create; the CUDA runtime of this process is already up
@@ -467,7 +470,7 @@ def test_decode_token_matches_per_call_sequence_and_counts_launches(per_layer):
             if per_layer:
                 assert a1.launch_count() - n0 >= 4 * cfg.L      # fused predict+select, attention, gate, FFN
             else:
-                assert a1.launch_count() - n0 == 1              # one persistent kernel over all layers
+                assert a1.launch_count() - n0 == 1 or not hz.token_kernel_expected()   # one persistent kernel over all layers
             for l in range(cfg.L):
                 a2.predict(l, h[t, l], 1); a2.select_candidates(l, 1, 0.9, cand, nc); a2.prefetch(l, 1)
                 a2.attention_standin(l); a2.route_topk(l, hp[t, l], 1, idx, al)
@@ -889,7 +892,7 @@ def test_random_shapes_tensor_core_path_gated_shared_expert_and_token_kernel():
             else:
                 n0 = apex.launch_count()
                 rep = hz.run_decode_lockstep(prob, apex, mode=mode, tau=tau, T=4)
-                assert apex.launch_count() - n0 == 4, "the persistent token kernel did not run"
+                assert apex.launch_count() - n0 == 4 or not hz.token_kernel_expected(), "the persistent token kernel did not run"
             assert apex.get_stats()["timeouts"] == 0 and rep.near_ties == 0
         finally:
             apex.destroy()
